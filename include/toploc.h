@@ -1,0 +1,211 @@
+/*
+ * toploc.h -- C ABI of the TopLoc proof hot path for NVIDIA B200 (sm_100a).
+ *
+ * TopLoc ("A Locality Sensitive Hashing Scheme for Trustless Verifiable
+ * Inference") commits, once per chunk of L tokens, to the k largest-magnitude
+ * entries of the last-layer hidden states by interpolating a polynomial
+ * congruence through (index mod m, value bits) and storing m plus the k
+ * coefficients (Algorithm 1; 258 bytes at k = 128, Section 5.7).  A validator
+ * recomputes the activations, repeats the top-k, evaluates the committed
+ * polynomial at the recomputed indices and thresholds the exponent / mantissa
+ * differences (Algorithm 2, thresholds in Section 5.2).
+ *
+ * Everything here is plain C: fixed-layout structs, raw pointers and sizes.
+ * Each pointer argument says whether it is HOST or DEVICE memory.  The caller
+ * owns every buffer; unless an entry point says otherwise the library
+ * allocates no device memory, frees nothing of the caller's and only enqueues
+ * work on the given CUDA stream.  No C++ exception crosses this boundary and
+ * no kernel traps: host-detected problems come back as a negative return code,
+ * per-chunk conditions as a status byte.
+ */
+#ifndef TOPLOC_H_
+#define TOPLOC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- constants -------------------------------------------------------- */
+
+/* Activation element types.  fp32 chunks are ranked on the full 31-bit
+ * magnitude but commit only the upper 16 bits of each selected pattern (the
+ * "fp32 mantissa scaled to match bf16" of Section 5.6), so proofs keep the
+ * 2 + 2k byte size. */
+#define TOPLOC_DTYPE_BF16 0
+#define TOPLOC_DTYPE_FP32 1
+
+/* Largest k the kernels are built for and largest chunk (elements). */
+#define TOPLOC_MAX_K 256
+#define TOPLOC_MAX_CHUNK_ELEMS (1 << 24)
+
+/* Host-side return codes (0 = success, negative = nothing was enqueued). */
+#define TOPLOC_OK 0
+#define TOPLOC_ERR_INVALID_ARGUMENT (-1)  /* NULL pointer, non-positive size, k out of range, ... */
+#define TOPLOC_ERR_UNSUPPORTED (-2)       /* dtype / k / chunk size outside what the kernels handle */
+#define TOPLOC_ERR_WORKSPACE (-3)         /* workspace or staging buffer smaller than required */
+#define TOPLOC_ERR_CUDA (-4)              /* a CUDA runtime call or a launch failed */
+#define TOPLOC_ERR_ARCH (-5)              /* current device is not compute capability 10.x */
+
+/* Per-chunk status codes (d_status of build, .status of a verify result). */
+#define TOPLOC_CHUNK_OK 0
+#define TOPLOC_CHUNK_NO_INJECTIVE_MODULUS 1 /* Algorithm 6 ran out of candidates (its "raise") */
+#define TOPLOC_CHUNK_K_EXCEEDS_CHUNK 2      /* the chunk holds fewer than k elements */
+#define TOPLOC_CHUNK_BAD_PROOF 3            /* decoded modulus outside [2^15+1, 2^16] or a coefficient >= p */
+#define TOPLOC_CHUNK_NONFINITE_COMMITTED 4  /* a selected 16-bit pattern is >= p (a negative NaN); the
+                                               proof is still produced but cannot reproduce that value */
+
+/* ---- structs ---------------------------------------------------------- */
+
+/* Batch layout.  Activations are a row-major matrix [total_tokens, hidden]
+ * with row_stride elements between consecutive token rows.  Sequences occupy
+ * consecutive row ranges; every sequence is cut into chunks of chunk_len rows
+ * (the last chunk of a sequence may be shorter), and a chunk is flattened
+ * row-major: flat index = token_in_chunk * hidden + channel (Section 4: an
+ * index needs 4 bytes because 32 x 4096 > 2^16). */
+typedef struct {
+  int32_t dtype;              /* TOPLOC_DTYPE_* */
+  int32_t hidden;             /* H > 0 */
+  int32_t chunk_len;          /* L > 0 tokens per chunk (32 in Section 5.5) */
+  int32_t k;                  /* 1..TOPLOC_MAX_K (128 in the paper) */
+  int32_t num_seqs;           /* > 0 */
+  int32_t reserved;           /* must be 0 */
+  int64_t tokens_per_seq;     /* uniform sequence length; used when seq_offsets == NULL */
+  const int64_t* seq_offsets; /* HOST, optional: num_seqs + 1 ascending row offsets (ragged batch);
+                                 read before the call returns */
+  int64_t row_stride;         /* elements between token rows, >= hidden */
+} toploc_layout;
+
+/* Acceptance thresholds of Algorithm 2 (Section 5.2: 38 / 10 / 8 for bf16).
+ * A chunk is rejected iff exp_mismatch > t_exp or mean > t_mean or
+ * median > t_median, or nothing matched, or its status is not OK.
+ * sign_in_exponent != 0 compares the sign bit together with the 8 exponent
+ * bits (bits 15..7), so a sign flip counts as an exponent mismatch;
+ * 0 compares bits 14..7 only. */
+typedef struct {
+  int32_t t_exp;
+  int32_t sign_in_exponent;
+  double t_mean;
+  double t_median;
+} toploc_thresholds;
+
+/* One per chunk, 40 bytes. */
+typedef struct {
+  uint32_t exp_mismatch;  /* err_e of Algorithm 2 */
+  uint32_t n_match;       /* |err_m|: points whose exponent fields agree */
+  uint32_t mant_diff_sum; /* exact sum of the |mantissa differences| in err_m */
+  int32_t topk_mismatch;  /* k - |generator indices ∩ validator indices| (Section 5.4),
+                             -1 when generator indices were not supplied */
+  double mant_mean;       /* mant_diff_sum / n_match in fp64, 0 when n_match == 0 */
+  double mant_median;     /* median of err_m (mean of the two middle values for an even
+                             count), 0 when n_match == 0 */
+  uint32_t modulus;       /* decoded m */
+  uint8_t accept;         /* 1 = valid, 0 = rejected */
+  uint8_t status;         /* TOPLOC_CHUNK_* */
+  uint8_t pad[2];
+} toploc_chunk_result;
+
+/* ---- queries (host only, no CUDA calls) ------------------------------- */
+
+/* Number of chunks the layout describes (sum over sequences of
+ * ceil(len / chunk_len)); negative error code for an invalid layout. */
+int64_t toploc_num_chunks(const toploc_layout* lay);
+
+/* 2 + 2k: a 2-byte modulus and k 2-byte coefficients (Section 4, Section 5.7). */
+size_t toploc_proof_bytes(int32_t k);
+
+/* Bytes of device scratch build/verify need for this layout: 0 for uniform
+ * batches, a per-chunk row table for ragged ones (seq_offsets != NULL). */
+size_t toploc_workspace_bytes(const toploc_layout* lay);
+
+/* Smallest device staging buffer the *_host entry points accept for this
+ * layout: room for the longest sequence's activations plus its outputs. */
+size_t toploc_staging_bytes(const toploc_layout* lay);
+
+/* Field prime p (largest prime below 2^16; Algorithm 3's modulus M must be a
+ * prime that fits the 2-byte coefficients) and the inclusive modulus search
+ * range of Algorithm 6. */
+void toploc_get_constants(uint32_t* p, uint32_t* m_lo, uint32_t* m_hi);
+
+const char* toploc_status_string(int chunk_status);
+const char* toploc_error_string(int return_code);
+
+/* ---- hot path --------------------------------------------------------- */
+
+/*
+ * Proof generation, Algorithm 1, for every chunk of the batch:
+ *   top-k by magnitude (key = bit pattern without the sign bit, ties to the
+ *   lower flat index)  ->  largest m in [2^15+1, 2^16] for which
+ *   (index mod m) mod p is injective (Algorithm 6)  ->  x = (index mod m) mod p,
+ *   y = selected 16-bit pattern mod p  ->  coefficients of the unique
+ *   polynomial of degree < k through the points over Z_p (Algorithm 3)  ->
+ *   proof bytes: m & 0xFFFF little-endian (0 stands for 65536), then the k
+ *   coefficients in ascending degree, 2 bytes little-endian each.
+ *
+ * d_act         DEVICE  activations, layout as described by *lay
+ * lay           HOST    read before return
+ * d_proofs      DEVICE  out, [num_chunks, 2 + 2k] bytes, chunks in batch order
+ *                       (sequence-major); zero-filled for a chunk whose status
+ *                       is NO_INJECTIVE_MODULUS or K_EXCEEDS_CHUNK
+ * d_status      DEVICE  out, [num_chunks] TOPLOC_CHUNK_* bytes
+ * d_indices_opt DEVICE  out, optional (NULL to skip): [num_chunks, k] selected
+ *                       flat indices ordered by (magnitude desc, index asc)
+ * d_workspace   DEVICE  scratch of at least toploc_workspace_bytes(lay) bytes,
+ *                       8-byte aligned; may be NULL when that is 0
+ * cuda_stream   a cudaStream_t (NULL = default stream)
+ *
+ * Asynchronous: returns after enqueueing; results are valid once the stream
+ * has been synchronised.  Returns TOPLOC_OK or a negative TOPLOC_ERR_*.
+ */
+int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_proofs,
+                        uint8_t* d_status, int32_t* d_indices_opt, void* d_workspace,
+                        size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Proof validation, Algorithm 2, for every chunk: decode (k from the layout
+ * must equal (proof length - 2) / 2), top-k on the recomputed activations,
+ * x' = (index mod m) mod p, Horner evaluation of the committed polynomial at
+ * every x' (Algorithm 5), split both 16-bit patterns into exponent field and
+ * 7-bit mantissa, count exponent mismatches and collect |mantissa difference|
+ * where the exponents agree, then threshold (strict >) as described at
+ * toploc_thresholds.
+ *
+ * d_act             DEVICE  recomputed activations (same layout as at build)
+ * d_proofs          DEVICE  [num_chunks, 2 + 2k] proofs
+ * thr               HOST    thresholds, read before return
+ * d_results         DEVICE  out, [num_chunks] toploc_chunk_result
+ * d_gen_indices_opt DEVICE  optional: the generator's [num_chunks, k] indices
+ *                           (d_indices_opt of build) for topk_mismatch
+ * other arguments as for toploc_build_proofs.
+ */
+int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint8_t* d_proofs,
+                         const toploc_thresholds* thr, toploc_chunk_result* d_results,
+                         const int32_t* d_gen_indices_opt, void* d_workspace,
+                         size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same two operations for callers whose data lives in HOST memory
+ * (pinned memory gives asynchronous copies; pageable memory works).  The
+ * batch is cut into groups of whole sequences that fit the staging buffer;
+ * each group is copied host->device, processed, and its proofs / results are
+ * copied device->host, all on cuda_stream.  The stream is synchronised before
+ * returning, so the host outputs are complete on return.
+ *
+ * h_act / h_proofs / h_status / h_results  HOST buffers, shapes as above
+ * d_staging  DEVICE scratch of staging_bytes >= toploc_staging_bytes(lay),
+ *            256-byte aligned; a larger buffer means fewer, larger groups
+ */
+int toploc_build_proofs_host(const void* h_act, const toploc_layout* lay, uint8_t* h_proofs,
+                             uint8_t* h_status, void* d_staging, size_t staging_bytes,
+                             void* cuda_stream);
+
+int toploc_verify_proofs_host(const void* h_act, const toploc_layout* lay, const uint8_t* h_proofs,
+                              const toploc_thresholds* thr, toploc_chunk_result* h_results,
+                              void* d_staging, size_t staging_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOPLOC_H_ */

@@ -1,0 +1,171 @@
+"""CPU oracle of the TopLoc proof path (ctypes view of oracle/toploc_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's CPU-baseline leg.  The product package never imports this module
+and this module never imports the product package.
+
+All functions take and return numpy arrays on the host.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+P_FIELD = 65521          # largest prime below 2^16 (Algorithm 3 needs a prime that fits 2 bytes)
+M_HIGH = 65536           # Algorithm 6 search range, inclusive
+M_LOW = 2 ** 15 + 1
+
+ST_OK, ST_NO_MODULUS, ST_K_EXCEEDS, ST_BAD_PROOF, ST_NONFINITE = range(5)
+
+RESULT_DTYPE = np.dtype([
+    ("exp_mismatch", "<u4"), ("n_match", "<u4"), ("mant_diff_sum", "<u4"), ("topk_mismatch", "<i4"),
+    ("mant_mean", "<f8"), ("mant_median", "<f8"), ("modulus", "<u4"),
+    ("accept", "u1"), ("status", "u1"), ("pad", "u1", (2,)),
+])
+assert RESULT_DTYPE.itemsize == 40
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(_build.build())
+        _lib.oracle_find_injective_modulus.restype = ctypes.c_uint32
+        _lib.oracle_mod_inverse.restype = ctypes.c_uint32
+        _lib.oracle_mod_inverse_euclid.restype = ctypes.c_int64
+        _lib.oracle_horner.restype = ctypes.c_uint32
+        _lib.oracle_num_chunks.restype = ctypes.c_int64
+    return _lib
+
+
+def _ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _dtype_code(act):
+    """bf16 chunks travel as uint16 bit patterns, fp32 chunks as float32 or uint32."""
+    if act.dtype == np.uint16:
+        return 0
+    if act.dtype in (np.float32, np.uint32):
+        return 1
+    raise TypeError("activations must be uint16 (bf16 patterns), float32 or uint32")
+
+
+def default_threads():
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def topk(chunk, k):
+    """chunk: 2-D [rows, hidden] array -> (indices uint32[k], bits uint16[k]) in rank order,
+    or None when k exceeds the chunk."""
+    chunk = np.ascontiguousarray(chunk)
+    rows, hidden = chunk.shape
+    idx = np.zeros(k, np.uint32)
+    bits = np.zeros(k, np.uint16)
+    st = lib().oracle_topk(_ptr(chunk), _dtype_code(chunk), rows, hidden, ctypes.c_int64(hidden), k,
+                           _ptr(idx), _ptr(bits))
+    return None if st != ST_OK else (idx, bits)
+
+
+def find_injective_modulus(indices, field_distinct=True):
+    """Algorithm 6; returns 0 when there is none."""
+    idx = np.ascontiguousarray(indices, np.uint32)
+    return int(lib().oracle_find_injective_modulus(_ptr(idx), len(idx), int(bool(field_distinct))))
+
+
+def mod_inverse(a):
+    return int(lib().oracle_mod_inverse(ctypes.c_uint32(a)))
+
+
+def mod_inverse_euclid(a, m):
+    return int(lib().oracle_mod_inverse_euclid(ctypes.c_int64(a), ctypes.c_int64(m)))
+
+
+def interpolate(x, y, newton=False):
+    """Coefficients (ascending degree, uint16) of the polynomial through (x_j, y_j) over Z_p."""
+    x = np.ascontiguousarray(x, np.uint32)
+    y = np.ascontiguousarray(y, np.uint32)
+    c = np.zeros(len(x), np.uint16)
+    fn = lib().oracle_interpolate_newton if newton else lib().oracle_interpolate
+    if fn(_ptr(x), _ptr(y), len(x), _ptr(c)) != 0:
+        raise ValueError("x values are not distinct mod p")
+    return c
+
+
+def horner(coeffs, x):
+    c = np.ascontiguousarray(coeffs, np.uint16)
+    return int(lib().oracle_horner(_ptr(c), len(c), ctypes.c_uint32(x)))
+
+
+def encode(m, coeffs):
+    c = np.ascontiguousarray(coeffs, np.uint16)
+    proof = np.zeros(2 + 2 * len(c), np.uint8)
+    lib().oracle_encode(ctypes.c_uint32(m), _ptr(c), len(c), _ptr(proof))
+    return proof
+
+
+def decode(proof):
+    """-> (status, k, m, coeffs)."""
+    proof = np.ascontiguousarray(proof, np.uint8)
+    k = ctypes.c_int(0)
+    m = ctypes.c_uint32(0)
+    c = np.zeros(max(1, len(proof) // 2), np.uint16)
+    st = lib().oracle_decode(_ptr(proof), ctypes.c_int64(len(proof)), ctypes.byref(k), ctypes.byref(m),
+                             _ptr(c))
+    return st, k.value, m.value, c[:k.value]
+
+
+def num_chunks(num_seqs, tokens_per_seq, chunk_len, seq_offsets=None):
+    so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
+    return int(lib().oracle_num_chunks(num_seqs, ctypes.c_int64(tokens_per_seq),
+                                       None if so is None else _ptr(so), chunk_len))
+
+
+def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None, first_chunk=0,
+                 last_chunk=-1, want_indices=True, threads=None):
+    """act: 2-D [total_tokens, hidden] host array (uint16 bf16 patterns or float32).
+
+    Returns (proofs uint8[n, 2+2k], status uint8[n], indices int32[n, k] or None), all indexed by
+    absolute chunk number; only rows first_chunk..last_chunk-1 are filled."""
+    assert act.ndim == 2 and act.strides[1] == act.itemsize
+    hidden = act.shape[1]
+    row_stride = act.strides[0] // act.itemsize
+    so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
+    n = num_chunks(num_seqs, tokens_per_seq, chunk_len, so)
+    proofs = np.zeros((n, 2 + 2 * k), np.uint8)
+    status = np.zeros(n, np.uint8)
+    indices = np.zeros((n, k), np.int32) if want_indices else None
+    lib().oracle_build_proofs(
+        _ptr(act), _dtype_code(act), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
+        None if so is None else _ptr(so), ctypes.c_int64(row_stride), ctypes.c_int64(first_chunk),
+        ctypes.c_int64(last_chunk), _ptr(proofs), _ptr(status),
+        None if indices is None else _ptr(indices), threads or default_threads())
+    return proofs, status, indices
+
+
+def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None,
+                  t_exp=38, t_mean=10.0, t_median=8.0, sign_in_exponent=True, gen_indices=None,
+                  first_chunk=0, last_chunk=-1, threads=None):
+    """Returns a structured array (RESULT_DTYPE) with one entry per chunk."""
+    assert act.ndim == 2 and act.strides[1] == act.itemsize
+    hidden = act.shape[1]
+    row_stride = act.strides[0] // act.itemsize
+    so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
+    n = num_chunks(num_seqs, tokens_per_seq, chunk_len, so)
+    proofs = np.ascontiguousarray(proofs, np.uint8)
+    assert proofs.shape == (n, 2 + 2 * k)
+    gi = None if gen_indices is None else np.ascontiguousarray(gen_indices, np.int32)
+    results = np.zeros(n, RESULT_DTYPE)
+    lib().oracle_verify_proofs(
+        _ptr(act), _dtype_code(act), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
+        None if so is None else _ptr(so), ctypes.c_int64(row_stride), ctypes.c_int64(first_chunk),
+        ctypes.c_int64(last_chunk), _ptr(proofs), int(t_exp), ctypes.c_double(t_mean),
+        ctypes.c_double(t_median), int(bool(sign_in_exponent)), None if gi is None else _ptr(gi),
+        _ptr(results), threads or default_threads())
+    return results

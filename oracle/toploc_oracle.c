@@ -1,0 +1,569 @@
+/*
+ * toploc_oracle.c -- slow, plain CPU statement of the TopLoc proof path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the parity reference for the CUDA
+ * library and the timed CPU baseline of the benchmark; nothing on the product
+ * path may call it, and it shares no code, header, table or constant with the
+ * CUDA side.  Every routine is written for being checked by eye against the
+ * paper, not for speed: a full sort for top-k, a brute-force modulus search,
+ * Gaussian elimination on the Vandermonde system for the interpolant.
+ *
+ * Readings of points the paper leaves open (each is repeated where it is used):
+ *   - ranking key: the bit pattern with the sign bit cleared, compared as an
+ *     unsigned integer; ties go to the lower flat index;
+ *   - field prime p = 65521, the largest prime below 2^16 (Algorithm 3 needs a
+ *     prime modulus, Section 4 fixes 2-byte coefficients);
+ *   - a candidate modulus m is accepted only if (index mod m) mod p is
+ *     injective, because m may exceed p;
+ *   - proof layout: m & 0xFFFF little-endian (0 means 65536), then the k
+ *     coefficients in ascending degree, 2 bytes little-endian each;
+ *   - fp32 activations rank on the 31-bit magnitude and commit the upper 16
+ *     bits of the pattern (Section 5.6, mantissa scaled to bf16).
+ *
+ * Pins (tests/test_oracle_*.py): worked examples and the paper's printed
+ * values under tests/golden/, brute force on tiny inputs, P(x_j) = y_j with
+ * Python integers, exhaustive a * inverse(a) = 1, Newton (Algorithm 3) against
+ * elimination, the modulus distribution of Table 11.  Unpinned: byte
+ * compatibility with the upstream project's proofs (its code is not
+ * available here) -- "parity unpinned" for that claim only.
+ */
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define P_FIELD 65521u /* largest prime below 2^16 */
+#define M_HIGH 65536u  /* Algorithm 6: "for i = 65536 downto 2^15 + 1" */
+#define M_LOW 32769u
+
+enum { ST_OK = 0, ST_NO_MODULUS = 1, ST_K_EXCEEDS = 2, ST_BAD_PROOF = 3, ST_NONFINITE = 4 };
+
+typedef struct {
+  uint32_t exp_mismatch;
+  uint32_t n_match;
+  uint32_t mant_diff_sum;
+  int32_t topk_mismatch;
+  double mant_mean;
+  double mant_median;
+  uint32_t modulus;
+  uint8_t accept;
+  uint8_t status;
+  uint8_t pad[2];
+} oracle_result;
+
+/* ------------------------------------------------------------------ */
+/* Section 5.3 "top-k magnitude elements"; Algorithm 1 step topk(h,k). */
+/* ------------------------------------------------------------------ */
+
+typedef struct {
+  uint32_t key;  /* magnitude: pattern without its sign bit */
+  uint32_t flat; /* token_in_chunk * hidden + channel */
+  uint16_t bits; /* the 16-bit pattern that gets committed */
+} ranked;
+
+static int by_magnitude_then_index(const void* a, const void* b) {
+  const ranked* p = (const ranked*)a;
+  const ranked* q = (const ranked*)b;
+  if (p->key != q->key) return p->key > q->key ? -1 : 1; /* larger magnitude first */
+  if (p->flat != q->flat) return p->flat < q->flat ? -1 : 1; /* then lower index */
+  return 0;
+}
+
+/* chunk: first element of the chunk's first row; rows x hidden elements,
+ * row_stride elements between rows.  dtype 0 = bf16 (uint16 patterns),
+ * 1 = fp32 (uint32 patterns).  Writes k indices and 16-bit patterns in rank
+ * order.  Returns ST_OK or ST_K_EXCEEDS. */
+int oracle_topk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
+                uint32_t* idx_out, uint16_t* bits_out) {
+  int64_t n = (int64_t)rows * hidden;
+  if (k > n) return ST_K_EXCEEDS;
+  ranked* all = (ranked*)malloc((size_t)n * sizeof(ranked));
+  for (int t = 0; t < rows; ++t) {
+    for (int c = 0; c < hidden; ++c) {
+      ranked* r = &all[(int64_t)t * hidden + c];
+      r->flat = (uint32_t)((int64_t)t * hidden + c);
+      if (dtype == 0) {
+        uint16_t v = ((const uint16_t*)chunk)[(int64_t)t * row_stride + c];
+        r->key = v & 0x7FFFu;
+        r->bits = v;
+      } else {
+        uint32_t v = ((const uint32_t*)chunk)[(int64_t)t * row_stride + c];
+        r->key = v & 0x7FFFFFFFu;
+        r->bits = (uint16_t)(v >> 16);
+      }
+    }
+  }
+  qsort(all, (size_t)n, sizeof(ranked), by_magnitude_then_index);
+  for (int j = 0; j < k; ++j) {
+    idx_out[j] = all[j].flat;
+    bits_out[j] = all[j].bits;
+  }
+  free(all);
+  return ST_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 6, Find Injective Modulus.                                */
+/* ------------------------------------------------------------------ */
+
+/* Largest m in [2^15+1, 2^16] such that the residues are pairwise distinct.
+ * field_distinct != 0: the residues compared are (idx mod m) mod p (the
+ * reading used by the proof path, since two residues below m can differ by
+ * exactly p); 0: idx mod m, Algorithm 6 as printed.  Returns 0 when no
+ * candidate works (the algorithm's "raise"). */
+uint32_t oracle_find_injective_modulus(const uint32_t* idx, int k, int field_distinct) {
+  uint32_t* r = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t found = 0;
+  for (uint32_t m = M_HIGH; m >= M_LOW && !found; --m) {
+    for (int j = 0; j < k; ++j) {
+      r[j] = idx[j] % m;
+      if (field_distinct) r[j] %= P_FIELD;
+    }
+    int injective = 1;
+    for (int a = 0; a < k && injective; ++a)
+      for (int b = a + 1; b < k; ++b)
+        if (r[a] == r[b]) {
+          injective = 0;
+          break;
+        }
+    if (injective) found = m;
+  }
+  free(r);
+  return found;
+}
+
+/* ------------------------------------------------------------------ */
+/* Arithmetic in Z_p.                                                  */
+/* ------------------------------------------------------------------ */
+
+static uint32_t mulp(uint32_t a, uint32_t b) { return (uint32_t)(((uint64_t)a * b) % P_FIELD); }
+static uint32_t addp(uint32_t a, uint32_t b) { return (a + b) % P_FIELD; }
+static uint32_t subp(uint32_t a, uint32_t b) { return (a + P_FIELD - b) % P_FIELD; }
+
+/* Inverse in Z_p by Fermat's little theorem, a^(p-2).  (Algorithm 4 uses the
+ * extended Euclidean algorithm; the inverse is unique, so the method is
+ * free.)  a must be in [1, p). */
+uint32_t oracle_mod_inverse(uint32_t a) {
+  uint32_t result = 1, base = a % P_FIELD;
+  uint32_t e = P_FIELD - 2;
+  while (e) {
+    if (e & 1u) result = mulp(result, base);
+    base = mulp(base, base);
+    e >>= 1;
+  }
+  return result;
+}
+
+/* Algorithm 4 as an algorithm: extended Euclid on (a, m), Bezout coefficient
+ * of a brought into [0, m).  Returns 0 when m <= 1; returns m (an impossible
+ * inverse) when gcd(a, m) != 1, standing for the algorithm's "throw". */
+int64_t oracle_mod_inverse_euclid(int64_t a, int64_t m) {
+  if (m <= 1) return 0;
+  int64_t r0 = a, r1 = m, s0 = 1, s1 = 0;
+  while (r1 != 0) {
+    int64_t q = r0 / r1;
+    int64_t r2 = r0 - q * r1;
+    r0 = r1;
+    r1 = r2;
+    int64_t s2 = s0 - q * s1;
+    s0 = s1;
+    s1 = s2;
+  }
+  if (r0 != 1) return m;
+  int64_t s = s0 % m;
+  if (s < 0) s += m;
+  return s;
+}
+
+/* Algorithm 5, Horner: c[0..k-1] ascending degree, result in [0, p). */
+uint32_t oracle_horner(const uint16_t* c, int k, uint32_t x) {
+  uint32_t acc = c[k - 1] % P_FIELD;
+  x %= P_FIELD;
+  for (int d = k - 2; d >= 0; --d) acc = addp(mulp(acc, x), c[d] % P_FIELD);
+  return acc;
+}
+
+/* ------------------------------------------------------------------ */
+/* Section 4: "there always exists a unique k-1-degree polynomial that  */
+/* goes through the points".  The interpolant is the solution of the   */
+/* Vandermonde system  sum_d c_d x_j^d = y_j  over Z_p; solved here by  */
+/* Gaussian elimination.  x must be pairwise distinct mod p.           */
+/* Returns 0 on success, 1 if the system is singular.                  */
+/* ------------------------------------------------------------------ */
+int oracle_interpolate(const uint32_t* x, const uint32_t* y, int k, uint16_t* c) {
+  int w = k + 1;
+  uint32_t* a = (uint32_t*)malloc((size_t)k * w * sizeof(uint32_t));
+  for (int j = 0; j < k; ++j) {
+    uint32_t pw = 1, xj = x[j] % P_FIELD;
+    for (int d = 0; d < k; ++d) {
+      a[j * w + d] = pw;
+      pw = mulp(pw, xj);
+    }
+    a[j * w + k] = y[j] % P_FIELD;
+  }
+  /* forward elimination to upper-triangular with unit diagonal */
+  for (int col = 0; col < k; ++col) {
+    int piv = -1;
+    for (int r = col; r < k; ++r)
+      if (a[r * w + col] != 0) {
+        piv = r;
+        break;
+      }
+    if (piv < 0) {
+      free(a);
+      return 1;
+    }
+    if (piv != col)
+      for (int d = 0; d < w; ++d) {
+        uint32_t t = a[col * w + d];
+        a[col * w + d] = a[piv * w + d];
+        a[piv * w + d] = t;
+      }
+    uint32_t inv = oracle_mod_inverse(a[col * w + col]);
+    for (int d = col; d < w; ++d) a[col * w + d] = mulp(a[col * w + d], inv);
+    for (int r = col + 1; r < k; ++r) {
+      uint32_t f = a[r * w + col];
+      if (f == 0) continue;
+      for (int d = col; d < w; ++d) a[r * w + d] = subp(a[r * w + d], mulp(f, a[col * w + d]));
+    }
+  }
+  /* back substitution */
+  uint32_t* sol = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  for (int row = k - 1; row >= 0; --row) {
+    uint32_t s = a[row * w + k];
+    for (int d = row + 1; d < k; ++d) s = subp(s, mulp(a[row * w + d], sol[d]));
+    sol[row] = s;
+  }
+  for (int d = 0; d < k; ++d) c[d] = (uint16_t)sol[d];
+  free(sol);
+  free(a);
+  return 0;
+}
+
+/* Algorithm 3, Newton interpolation, kept beside the elimination above as a
+ * second statement of the same polynomial (the two must agree because the
+ * interpolant is unique).  Divided differences first, then the Newton form
+ * a_0 + (x - x_0)(a_1 + (x - x_1)(...)) is multiplied out from the inside.
+ * Inverses by the extended Euclidean routine (Algorithm 4). */
+int oracle_interpolate_newton(const uint32_t* x, const uint32_t* y, int k, uint16_t* c) {
+  uint32_t* dd = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* poly = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+  for (int j = 0; j < k; ++j) dd[j] = y[j] % P_FIELD;
+  for (int level = 1; level < k; ++level)
+    for (int i = k - 1; i >= level; --i) {
+      uint32_t num = subp(dd[i], dd[i - 1]);
+      uint32_t den = subp(x[i] % P_FIELD, x[i - level] % P_FIELD);
+      int64_t inv = oracle_mod_inverse_euclid((int64_t)den, (int64_t)P_FIELD);
+      if (den == 0 || inv == (int64_t)P_FIELD) {
+        free(dd);
+        free(poly);
+        return 1;
+      }
+      dd[i] = mulp(num, (uint32_t)inv);
+    }
+  /* poly <- dd[k-1]; then for i = k-2..0: poly <- poly * (x - x_i) + dd[i] */
+  poly[0] = dd[k - 1];
+  int deg = 0;
+  for (int i = k - 2; i >= 0; --i) {
+    uint32_t neg_xi = subp(0, x[i] % P_FIELD);
+    for (int d = deg + 1; d >= 1; --d) poly[d] = addp(poly[d - 1], mulp(poly[d], neg_xi));
+    poly[0] = addp(mulp(poly[0], neg_xi), dd[i]);
+    ++deg;
+  }
+  for (int d = 0; d < k; ++d) c[d] = (uint16_t)poly[d];
+  free(dd);
+  free(poly);
+  return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* encode / decode (Algorithm 1 last step, Algorithm 2 first step).    */
+/* 2 + 2k bytes: Section 4 (2-byte coefficients), Section 5.7 (256 B of */
+/* coefficients per interval), abstract (258 B).                       */
+/* ------------------------------------------------------------------ */
+void oracle_encode(uint32_t m, const uint16_t* c, int k, uint8_t* proof) {
+  uint32_t m16 = m & 0xFFFFu; /* 65536 -> 0 */
+  proof[0] = (uint8_t)(m16 & 0xFF);
+  proof[1] = (uint8_t)(m16 >> 8);
+  for (int d = 0; d < k; ++d) {
+    proof[2 + 2 * d] = (uint8_t)(c[d] & 0xFF);
+    proof[3 + 2 * d] = (uint8_t)(c[d] >> 8);
+  }
+}
+
+/* Returns ST_OK or ST_BAD_PROOF (odd or too short length, modulus outside
+ * the search range, a coefficient >= p).  *k_out = (len - 2) / 2. */
+int oracle_decode(const uint8_t* proof, int64_t len, int* k_out, uint32_t* m_out, uint16_t* c) {
+  if (len < 4 || (len & 1)) return ST_BAD_PROOF;
+  int k = (int)((len - 2) / 2);
+  uint32_t m = (uint32_t)proof[0] | ((uint32_t)proof[1] << 8);
+  if (m == 0) m = 65536u;
+  *k_out = k;
+  *m_out = m;
+  int bad = (m < M_LOW || m > M_HIGH);
+  for (int d = 0; d < k; ++d) {
+    c[d] = (uint16_t)(proof[2 + 2 * d] | (proof[3 + 2 * d] << 8));
+    if (c[d] >= P_FIELD) bad = 1;
+  }
+  return bad ? ST_BAD_PROOF : ST_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 1 for one chunk.                                          */
+/* ------------------------------------------------------------------ */
+int oracle_build_chunk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
+                       uint8_t* proof, int32_t* indices_opt) {
+  size_t nbytes = 2 + 2 * (size_t)k;
+  memset(proof, 0, nbytes);
+  if (indices_opt) memset(indices_opt, 0, (size_t)k * sizeof(int32_t));
+  uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* bits = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  uint32_t* xs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* ys = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* coef = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  int status = oracle_topk(chunk, dtype, rows, hidden, row_stride, k, idx, bits);
+  if (status == ST_OK) {
+    if (indices_opt)
+      for (int j = 0; j < k; ++j) indices_opt[j] = (int32_t)idx[j];
+    uint32_t m = oracle_find_injective_modulus(idx, k, 1);
+    if (m == 0) {
+      status = ST_NO_MODULUS;
+    } else {
+      for (int j = 0; j < k; ++j) {
+        xs[j] = (idx[j] % m) % P_FIELD;
+        ys[j] = (uint32_t)bits[j] % P_FIELD; /* "dd <- y mod M" */
+        if (bits[j] >= P_FIELD) status = ST_NONFINITE;
+      }
+      oracle_interpolate(xs, ys, k, coef);
+      oracle_encode(m, coef, k, proof);
+    }
+  }
+  free(idx);
+  free(bits);
+  free(xs);
+  free(ys);
+  free(coef);
+  return status;
+}
+
+static int ascending_u32(const void* a, const void* b) {
+  uint32_t p = *(const uint32_t*)a, q = *(const uint32_t*)b;
+  return p < q ? -1 : (p > q ? 1 : 0);
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 2 for one chunk.  Thresholds: Section 5.2.                */
+/* 16-bit pattern: bit 15 sign, bits 14..7 exponent, bits 6..0         */
+/* mantissa (bf16 has 7 mantissa bits, Section 5.2).                   */
+/* ------------------------------------------------------------------ */
+void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
+                         const uint8_t* proof, int t_exp, double t_mean, double t_median,
+                         int sign_in_exponent, const int32_t* gen_indices_opt, oracle_result* out) {
+  memset(out, 0, sizeof(*out));
+  out->topk_mismatch = -1;
+  uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* bits = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  uint16_t* coef = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  uint32_t* diffs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  int kk = 0;
+  uint32_t m = 0;
+  int status = oracle_decode(proof, 2 + 2 * (int64_t)k, &kk, &m, coef);
+  out->modulus = m;
+  if (status == ST_OK) status = oracle_topk(chunk, dtype, rows, hidden, row_stride, k, idx, bits);
+  if (status == ST_OK) {
+    uint32_t err_e = 0, n = 0, sum = 0;
+    for (int j = 0; j < k; ++j) {
+      uint32_t xj = (idx[j] % m) % P_FIELD;
+      uint32_t committed = oracle_horner(coef, k, xj); /* P[i_m[j]] */
+      uint32_t seen = bits[j];
+      uint32_t e_p, e_v;
+      if (sign_in_exponent) {
+        e_p = committed >> 7; /* sign + exponent, 9 bits */
+        e_v = seen >> 7;
+      } else {
+        e_p = (committed >> 7) & 0xFFu;
+        e_v = (seen >> 7) & 0xFFu;
+      }
+      uint32_t m_p = committed & 0x7Fu, m_v = seen & 0x7Fu;
+      if (e_p == e_v) {
+        uint32_t d = m_p > m_v ? m_p - m_v : m_v - m_p;
+        diffs[n++] = d;
+        sum += d;
+      } else {
+        ++err_e;
+      }
+    }
+    out->exp_mismatch = err_e;
+    out->n_match = n;
+    out->mant_diff_sum = sum;
+    if (n > 0) {
+      out->mant_mean = (double)sum / (double)n;
+      qsort(diffs, n, sizeof(uint32_t), ascending_u32);
+      out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
+    }
+    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    if (n == 0) reject = 1; /* nothing matched: no statistic to accept on */
+    out->accept = reject ? 0 : 1;
+    if (gen_indices_opt) {
+      int common = 0;
+      for (int a = 0; a < k; ++a)
+        for (int b = 0; b < k; ++b)
+          if ((uint32_t)gen_indices_opt[a] == idx[b]) {
+            ++common;
+            break;
+          }
+      out->topk_mismatch = k - common;
+    }
+  }
+  out->status = (uint8_t)status;
+  if (status != ST_OK) out->accept = 0;
+  free(idx);
+  free(bits);
+  free(coef);
+  free(diffs);
+}
+
+/* ------------------------------------------------------------------ */
+/* Batch drivers: chunks of chunk_len rows per sequence (Section 5.5:   */
+/* one proof per 32 new tokens), the last chunk of a sequence may be    */
+/* shorter.  seq_offsets: num_seqs + 1 row offsets, or NULL for        */
+/* uniform sequences of tokens_per_seq rows.  Threads split chunks.    */
+/* ------------------------------------------------------------------ */
+
+typedef struct {
+  int64_t row0;
+  int32_t rows;
+} chunk_span;
+
+static int64_t enumerate_chunks(int num_seqs, int64_t tokens_per_seq, const int64_t* seq_offsets,
+                                int chunk_len, chunk_span* out) {
+  int64_t n = 0;
+  for (int s = 0; s < num_seqs; ++s) {
+    int64_t begin = seq_offsets ? seq_offsets[s] : (int64_t)s * tokens_per_seq;
+    int64_t end = seq_offsets ? seq_offsets[s + 1] : begin + tokens_per_seq;
+    for (int64_t r = begin; r < end; r += chunk_len) {
+      if (out) {
+        out[n].row0 = r;
+        out[n].rows = (int32_t)((end - r) < chunk_len ? (end - r) : chunk_len);
+      }
+      ++n;
+    }
+  }
+  return n;
+}
+
+int64_t oracle_num_chunks(int num_seqs, int64_t tokens_per_seq, const int64_t* seq_offsets, int chunk_len) {
+  return enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, NULL);
+}
+
+typedef struct {
+  int tid, nthreads, verify;
+  const uint8_t* act;
+  int dtype, hidden, k;
+  int64_t row_stride;
+  const chunk_span* spans;
+  int64_t first, last; /* chunk range [first, last) */
+  uint8_t* proofs;
+  uint8_t* status;
+  int32_t* indices;
+  const uint8_t* proofs_in;
+  const int32_t* gen_indices;
+  oracle_result* results;
+  int t_exp, sign_in_exponent;
+  double t_mean, t_median;
+} job;
+
+static void* worker(void* arg) {
+  job* jb = (job*)arg;
+  size_t esz = jb->dtype == 0 ? 2 : 4;
+  size_t pbytes = 2 + 2 * (size_t)jb->k;
+  for (int64_t c = jb->first + jb->tid; c < jb->last; c += jb->nthreads) {
+    const void* chunk = jb->act + (size_t)jb->spans[c].row0 * (size_t)jb->row_stride * esz;
+    if (!jb->verify) {
+      int st = oracle_build_chunk(chunk, jb->dtype, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
+                                  jb->proofs + (size_t)c * pbytes,
+                                  jb->indices ? jb->indices + (size_t)c * jb->k : NULL);
+      jb->status[c] = (uint8_t)st;
+    } else {
+      oracle_verify_chunk(chunk, jb->dtype, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
+                          jb->proofs_in + (size_t)c * pbytes, jb->t_exp, jb->t_mean, jb->t_median,
+                          jb->sign_in_exponent,
+                          jb->gen_indices ? jb->gen_indices + (size_t)c * jb->k : NULL, &jb->results[c]);
+    }
+  }
+  return NULL;
+}
+
+static int run_jobs(job* proto, int nthreads) {
+  if (nthreads < 1) nthreads = 1;
+  pthread_t* th = (pthread_t*)malloc((size_t)nthreads * sizeof(pthread_t));
+  job* jobs = (job*)malloc((size_t)nthreads * sizeof(job));
+  for (int t = 0; t < nthreads; ++t) {
+    jobs[t] = *proto;
+    jobs[t].tid = t;
+    jobs[t].nthreads = nthreads;
+    pthread_create(&th[t], NULL, worker, &jobs[t]);
+  }
+  for (int t = 0; t < nthreads; ++t) pthread_join(th[t], NULL);
+  free(jobs);
+  free(th);
+  return 0;
+}
+
+/* Proofs for chunks [first_chunk, last_chunk) of the batch (last_chunk < 0:
+ * all).  Outputs are indexed by absolute chunk number. */
+int oracle_build_proofs(const void* act, int dtype, int hidden, int chunk_len, int k, int num_seqs,
+                        int64_t tokens_per_seq, const int64_t* seq_offsets, int64_t row_stride,
+                        int64_t first_chunk, int64_t last_chunk, uint8_t* proofs, uint8_t* status,
+                        int32_t* indices_opt, int nthreads) {
+  int64_t n = enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, NULL);
+  chunk_span* spans = (chunk_span*)malloc((size_t)(n > 0 ? n : 1) * sizeof(chunk_span));
+  enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, spans);
+  job jb;
+  memset(&jb, 0, sizeof(jb));
+  jb.act = (const uint8_t*)act;
+  jb.dtype = dtype;
+  jb.hidden = hidden;
+  jb.k = k;
+  jb.row_stride = row_stride;
+  jb.spans = spans;
+  jb.first = first_chunk;
+  jb.last = last_chunk < 0 ? n : last_chunk;
+  jb.proofs = proofs;
+  jb.status = status;
+  jb.indices = indices_opt;
+  run_jobs(&jb, nthreads);
+  free(spans);
+  return 0;
+}
+
+int oracle_verify_proofs(const void* act, int dtype, int hidden, int chunk_len, int k, int num_seqs,
+                         int64_t tokens_per_seq, const int64_t* seq_offsets, int64_t row_stride,
+                         int64_t first_chunk, int64_t last_chunk, const uint8_t* proofs, int t_exp,
+                         double t_mean, double t_median, int sign_in_exponent,
+                         const int32_t* gen_indices_opt, oracle_result* results, int nthreads) {
+  int64_t n = enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, NULL);
+  chunk_span* spans = (chunk_span*)malloc((size_t)(n > 0 ? n : 1) * sizeof(chunk_span));
+  enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, spans);
+  job jb;
+  memset(&jb, 0, sizeof(jb));
+  jb.verify = 1;
+  jb.act = (const uint8_t*)act;
+  jb.dtype = dtype;
+  jb.hidden = hidden;
+  jb.k = k;
+  jb.row_stride = row_stride;
+  jb.spans = spans;
+  jb.first = first_chunk;
+  jb.last = last_chunk < 0 ? n : last_chunk;
+  jb.proofs_in = proofs;
+  jb.gen_indices = gen_indices_opt;
+  jb.results = results;
+  jb.t_exp = t_exp;
+  jb.t_mean = t_mean;
+  jb.t_median = t_median;
+  jb.sign_in_exponent = sign_in_exponent;
+  run_jobs(&jb, nthreads);
+  free(spans);
+  return 0;
+}

@@ -1,0 +1,274 @@
+"""Python view of include/toploc.h: same names, argument marshalling only.
+
+Every step of the proof path runs in the CUDA library (csrc/libtoploc.so).  torch is
+used for device memory and streams, nothing else.  There is no fallback: if the library
+is missing or the arguments are wrong, the call raises.
+"""
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+__all__ = [
+    "TOPLOC_DTYPE_BF16", "TOPLOC_DTYPE_FP32", "TOPLOC_MAX_K", "RESULT_DTYPE", "ToplocError",
+    "ToplocLayout", "ToplocThresholds", "make_layout", "library_path", "load_library",
+    "toploc_num_chunks", "toploc_proof_bytes", "toploc_workspace_bytes", "toploc_staging_bytes",
+    "toploc_get_constants", "toploc_status_string", "toploc_error_string",
+    "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
+    "toploc_verify_proofs_host",
+]
+
+TOPLOC_DTYPE_BF16 = 0
+TOPLOC_DTYPE_FP32 = 1
+TOPLOC_MAX_K = 256
+
+RESULT_DTYPE = np.dtype([
+    ("exp_mismatch", "<u4"), ("n_match", "<u4"), ("mant_diff_sum", "<u4"), ("topk_mismatch", "<i4"),
+    ("mant_mean", "<f8"), ("mant_median", "<f8"), ("modulus", "<u4"),
+    ("accept", "u1"), ("status", "u1"), ("pad", "u1", (2,)),
+])
+
+
+class ToplocError(RuntimeError):
+    pass
+
+
+class ToplocLayout(ctypes.Structure):
+    _fields_ = [
+        ("dtype", ctypes.c_int32), ("hidden", ctypes.c_int32), ("chunk_len", ctypes.c_int32),
+        ("k", ctypes.c_int32), ("num_seqs", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("tokens_per_seq", ctypes.c_int64), ("seq_offsets", ctypes.POINTER(ctypes.c_int64)),
+        ("row_stride", ctypes.c_int64),
+    ]
+
+
+class ToplocThresholds(ctypes.Structure):
+    _fields_ = [
+        ("t_exp", ctypes.c_int32), ("sign_in_exponent", ctypes.c_int32),
+        ("t_mean", ctypes.c_double), ("t_median", ctypes.c_double),
+    ]
+
+
+_LIB = None
+
+
+def library_path():
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libtoploc.so")
+
+
+def load_library():
+    """Loads csrc/libtoploc.so (built by csrc/build.py); raises if it is not there."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise ToplocError(
+            "%s is missing: build it with `python -m paper_2501_16007_b200.csrc.build` "
+            "(there is no CPU fallback)" % path)
+    lib = ctypes.CDLL(path)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    lay_p, thr_p = ctypes.POINTER(ToplocLayout), ctypes.POINTER(ToplocThresholds)
+    lib.toploc_num_chunks.restype, lib.toploc_num_chunks.argtypes = i64, [lay_p]
+    lib.toploc_proof_bytes.restype, lib.toploc_proof_bytes.argtypes = sz, [i32]
+    lib.toploc_workspace_bytes.restype, lib.toploc_workspace_bytes.argtypes = sz, [lay_p]
+    lib.toploc_staging_bytes.restype, lib.toploc_staging_bytes.argtypes = sz, [lay_p]
+    lib.toploc_get_constants.restype = None
+    lib.toploc_get_constants.argtypes = [ctypes.POINTER(ctypes.c_uint32)] * 3
+    lib.toploc_status_string.restype, lib.toploc_status_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
+    lib.toploc_error_string.restype, lib.toploc_error_string.argtypes = ctypes.c_char_p, [ctypes.c_int]
+    lib.toploc_build_proofs.restype = ctypes.c_int
+    lib.toploc_build_proofs.argtypes = [vp, lay_p, vp, vp, vp, vp, sz, vp]
+    lib.toploc_verify_proofs.restype = ctypes.c_int
+    lib.toploc_verify_proofs.argtypes = [vp, lay_p, vp, thr_p, vp, vp, vp, sz, vp]
+    lib.toploc_build_proofs_host.restype = ctypes.c_int
+    lib.toploc_build_proofs_host.argtypes = [vp, lay_p, vp, vp, vp, sz, vp]
+    lib.toploc_verify_proofs_host.restype = ctypes.c_int
+    lib.toploc_verify_proofs_host.argtypes = [vp, lay_p, vp, thr_p, vp, vp, sz, vp]
+    _LIB = lib
+    return lib
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise ToplocError("%s failed: %s (%d)" % (what, toploc_error_string(rc), rc))
+
+
+def _dtype_code(t):
+    if t.dtype == torch.bfloat16:
+        return TOPLOC_DTYPE_BF16
+    if t.dtype == torch.float32:
+        return TOPLOC_DTYPE_FP32
+    raise ToplocError("activations must be bfloat16 or float32, got %s" % t.dtype)
+
+
+def make_layout(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None):
+    """Layout of a 2-D activation tensor [total_tokens, hidden] (last dimension contiguous).
+
+    Returns (layout, keepalive): keepalive holds the host seq_offsets array the struct points to."""
+    if act.dim() != 2 or act.stride(1) != 1:
+        raise ToplocError("activations must be 2-D with a contiguous last dimension")
+    lay = ToplocLayout()
+    lay.dtype = _dtype_code(act)
+    lay.hidden = act.shape[1]
+    lay.chunk_len = chunk_len
+    lay.k = k
+    lay.num_seqs = num_seqs
+    lay.reserved = 0
+    lay.tokens_per_seq = tokens_per_seq
+    lay.row_stride = act.stride(0) if act.shape[0] > 1 else act.shape[1]
+    keep = None
+    if seq_offsets is not None:
+        keep = np.ascontiguousarray(seq_offsets, np.int64)
+        if keep.shape != (num_seqs + 1,):
+            raise ToplocError("seq_offsets must have num_seqs + 1 entries")
+        lay.seq_offsets = keep.ctypes.data_as(ctypes.POINTER(ctypes.c_int64))
+        total = int(keep[-1])
+    else:
+        total = num_seqs * tokens_per_seq
+    if total > act.shape[0]:
+        raise ToplocError("layout describes %d rows, tensor has %d" % (total, act.shape[0]))
+    return lay, keep
+
+
+def toploc_num_chunks(lay):
+    n = load_library().toploc_num_chunks(ctypes.byref(lay))
+    if n < 0:
+        raise ToplocError("invalid layout: %s" % toploc_error_string(int(n)))
+    return int(n)
+
+
+def toploc_proof_bytes(k):
+    return int(load_library().toploc_proof_bytes(k))
+
+
+def toploc_workspace_bytes(lay):
+    return int(load_library().toploc_workspace_bytes(ctypes.byref(lay)))
+
+
+def toploc_staging_bytes(lay):
+    return int(load_library().toploc_staging_bytes(ctypes.byref(lay)))
+
+
+def toploc_get_constants():
+    p, lo, hi = ctypes.c_uint32(), ctypes.c_uint32(), ctypes.c_uint32()
+    load_library().toploc_get_constants(ctypes.byref(p), ctypes.byref(lo), ctypes.byref(hi))
+    return p.value, lo.value, hi.value
+
+
+def toploc_status_string(code):
+    return load_library().toploc_status_string(int(code)).decode()
+
+
+def toploc_error_string(code):
+    return load_library().toploc_error_string(int(code)).decode()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dev_ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _workspace(lay, workspace, device):
+    need = toploc_workspace_bytes(lay)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace, (0 if workspace is None else workspace.numel() * workspace.element_size())
+
+
+def toploc_build_proofs(act, lay, proofs=None, status=None, indices=None, workspace=None, stream=None,
+                        want_indices=False):
+    """Enqueues proof generation for the batch `lay` describes on `stream` (default: torch's
+    current stream).  act: CUDA tensor.  Output tensors are allocated when not given.
+    Returns (proofs uint8[n, 2+2k], status uint8[n], indices int32[n, k] or None)."""
+    if not act.is_cuda:
+        raise ToplocError("toploc_build_proofs needs a CUDA tensor (use toploc_build_proofs_host)")
+    n = toploc_num_chunks(lay)
+    pb = toploc_proof_bytes(lay.k)
+    dev = act.device
+    if proofs is None:
+        proofs = torch.empty((n, pb), dtype=torch.uint8, device=dev)
+    if status is None:
+        status = torch.empty((n,), dtype=torch.uint8, device=dev)
+    if indices is None and want_indices:
+        indices = torch.empty((n, lay.k), dtype=torch.int32, device=dev)
+    assert proofs.is_contiguous() and proofs.numel() == n * pb and status.numel() == n
+    assert indices is None or (indices.is_contiguous() and indices.numel() == n * lay.k
+                               and indices.dtype == torch.int32)
+    workspace, wbytes = _workspace(lay, workspace, dev)
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_build_proofs(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(proofs), _dev_ptr(status), _dev_ptr(indices),
+            _dev_ptr(workspace), wbytes, _stream_ptr(stream))
+    _check(rc, "toploc_build_proofs")
+    return proofs, status, indices
+
+
+def toploc_verify_proofs(act, lay, proofs, thresholds=None, results=None, gen_indices=None,
+                         workspace=None, stream=None):
+    """Enqueues validation.  Returns a uint8 CUDA tensor [n, 40]; view it on the host with
+    results.cpu().numpy().view(RESULT_DTYPE).reshape(-1)."""
+    if not act.is_cuda:
+        raise ToplocError("toploc_verify_proofs needs a CUDA tensor (use toploc_verify_proofs_host)")
+    n = toploc_num_chunks(lay)
+    dev = act.device
+    thr = thresholds if thresholds is not None else default_thresholds()
+    if results is None:
+        results = torch.empty((n, RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    assert proofs.is_contiguous() and proofs.numel() == n * toploc_proof_bytes(lay.k)
+    assert results.is_contiguous() and results.numel() == n * RESULT_DTYPE.itemsize
+    assert gen_indices is None or (gen_indices.is_contiguous() and gen_indices.dtype == torch.int32
+                                   and gen_indices.numel() == n * lay.k)
+    workspace, wbytes = _workspace(lay, workspace, dev)
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_verify_proofs(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(proofs), ctypes.byref(thr), _dev_ptr(results),
+            _dev_ptr(gen_indices), _dev_ptr(workspace), wbytes, _stream_ptr(stream))
+    _check(rc, "toploc_verify_proofs")
+    return results
+
+
+def default_thresholds(k=128, sign_in_exponent=True):
+    """Section 5.2 thresholds for bf16 (38 / 10 / 8 at k = 128); the exponent threshold
+    scales with k for other proof sizes."""
+    thr = ToplocThresholds()
+    thr.t_exp = (38 * k) // 128
+    thr.sign_in_exponent = 1 if sign_in_exponent else 0
+    thr.t_mean = 10.0
+    thr.t_median = 8.0
+    return thr
+
+
+__all__.append("default_thresholds")
+
+
+def toploc_build_proofs_host(act, lay, proofs, status, staging, stream=None):
+    """Host-memory variant: act / proofs / status are CPU tensors (pinned for asynchronous
+    copies), staging is a CUDA uint8 tensor of at least toploc_staging_bytes(lay) bytes.
+    Blocks until the host outputs are complete."""
+    if act.is_cuda or proofs.is_cuda or status.is_cuda or not staging.is_cuda:
+        raise ToplocError("host variant: act/proofs/status on the CPU, staging on the GPU")
+    with torch.cuda.device(staging.device):
+        rc = load_library().toploc_build_proofs_host(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(proofs), _dev_ptr(status), _dev_ptr(staging),
+            staging.numel() * staging.element_size(), _stream_ptr(stream))
+    _check(rc, "toploc_build_proofs_host")
+    return proofs, status
+
+
+def toploc_verify_proofs_host(act, lay, proofs, thresholds, results, staging, stream=None):
+    if act.is_cuda or proofs.is_cuda or results.is_cuda or not staging.is_cuda:
+        raise ToplocError("host variant: act/proofs/results on the CPU, staging on the GPU")
+    thr = thresholds if thresholds is not None else default_thresholds(lay.k)
+    with torch.cuda.device(staging.device):
+        rc = load_library().toploc_verify_proofs_host(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(proofs), ctypes.byref(thr), _dev_ptr(results),
+            _dev_ptr(staging), staging.numel() * staging.element_size(), _stream_ptr(stream))
+    _check(rc, "toploc_verify_proofs_host")
+    return results
