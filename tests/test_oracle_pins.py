@@ -151,7 +151,10 @@ def test_modulus_worked_outlier_sets():
         m = oracle.find_injective_modulus(idx)
         check_modulus_by_definition(idx, m)
     assert oracle.find_injective_modulus(a) == 65532
-    assert oracle.find_injective_modulus(b) == 65528
+    assert oracle.find_injective_modulus(b) == 65532
+    c8 = [t * 8192 + c for t in range(16) for c in range(8)]   # 8 adjacent channels instead
+    check_modulus_by_definition(c8, oracle.find_injective_modulus(c8))
+    assert oracle.find_injective_modulus(c8) == 65528
     assert oracle.find_injective_modulus(small) == 65536  # all indices below 2^15 + 1
 
 
