@@ -1,0 +1,330 @@
+"""Benchmark of the TopLoc proof hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 70b|8b] [--impl ours|reference]
+
+One step = proof generation for every chunk of the batch followed by validation of every
+proof against recomputed activations (honest-noise copy), i.e. one pass of the whole path.
+The default workload is the Llama-3.1-70B-shaped batch: 256 sequences x 4096 tokens,
+H = 8192, bf16 (17.18 GB), 32-token chunks, k = 128 -> 32768 proofs of 258 bytes.
+
+Rank 0 prints one JSON line.  `value` counts chunks generated-and-validated per second with
+the activations resident in HBM; `e2e` is the same through the host-buffer entry points
+(pinned host memory, copies inside the timed region).  With N > 1 (torchrun) every rank
+processes its own full batch: weak scaling, no collective on the data path.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # name: (sequences, tokens per sequence, hidden, chunk_len, k, seed)
+    "70b": (256, 4096, 8192, 32, 128, 4),
+    "8b": (64, 2048, 4096, 32, 128, 2),
+}
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=5)
+        sm, smax, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for row in self.rows:
+            if len(row) != 6:
+                continue
+            try:
+                sm.append(float(row[0]))
+                smax = float(row[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, row[2:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def reference_arm(args, rank):
+    """The CPU oracle, as it stands, on the host cores: each step builds and validates the proofs
+    of a bounded sample (the first sequence) of the workload."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2501_16007_b200 import synth
+    S, T, H, L, k, seed = WORKLOADS[args.workload]
+    act = synth.make_activations(1, T, H, torch.bfloat16, seed=seed, device="cpu")
+    noisy = synth.honest_noise(act, seed=seed + 1)
+    host, host_noisy = synth.host_patterns(act), synth.host_patterns(noisy)
+    chunks = T // L
+    cores = oracle.default_threads()
+
+    def step():
+        proofs, status, idx = oracle.build_proofs(host, L, k, 1, T, threads=cores)
+        oracle.verify_proofs(host_noisy, proofs, L, k, 1, T, gen_indices=idx, threads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = chunks / dt
+    line = {
+        "impl": "reference", "metric": "proof_chunks_per_s_generate_plus_verify", "value": value,
+        "unit": "chunks/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u16/u32 integer (bf16 bit patterns)", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload), "sample": "first sequence (%d chunks) per step" % chunks},
+        "cpu_baseline": {"value": value, "unit": "chunks/s", "cores": cores, "kind": "oracle",
+                         "sample": "first sequence: %d chunks of %d x %d bf16, build + verify" % (chunks, L, H)},
+        "e2e": {"value": value, "unit": "chunks/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(key):
+    S, T, H, L, k, seed = WORKLOADS[key]
+    return "%s-shaped: %d seq x %d tok, H=%d bf16, L=%d, k=%d" % (
+        {"70b": "Llama-3.1-70B", "8b": "Llama-3.1-8B"}[key], S, T, H, L, k)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="70b")
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        reference_arm(args, rank)
+        return
+
+    import paper_2501_16007_b200 as tl
+    from paper_2501_16007_b200 import synth
+    import torch.distributed as dist
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    S, T, H, L, k, seed = WORKLOADS[args.workload]
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=seed + 10007 * rank, device=dev)
+    recomputed = synth.honest_noise(act, seed=seed + 1)
+    lay, _ = tl.make_layout(act, L, k, S, T)
+    n = tl.toploc_num_chunks(lay)
+    act_bytes = act.numel() * act.element_size()
+    proofs = torch.empty((n, tl.toploc_proof_bytes(k)), dtype=torch.uint8, device=dev)
+    status = torch.empty((n,), dtype=torch.uint8, device=dev)
+    results = torch.empty((n, 40), dtype=torch.uint8, device=dev)
+    thr = tl.default_thresholds(k)
+
+    def step(ev=None):
+        if ev:
+            ev[0].record()
+        tl.toploc_build_proofs(act, lay, proofs, status)
+        if ev:
+            ev[1].record()
+        tl.toploc_verify_proofs(recomputed, lay, proofs, thr, results)
+        if ev:
+            ev[2].record()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(args.steps):
+        step(events[i])
+    stop.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    total_ms = start.elapsed_time(stop)
+    build_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
+    verify_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
+    if world > 1:
+        t = torch.tensor([total_ms, build_ms, verify_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, build_ms, verify_ms = t.tolist()
+    ms_per_step = total_ms / args.steps
+
+    accepted = int(results.cpu().numpy().view(tl.RESULT_DTYPE)["accept"].sum())
+    bad_status = int(status.count_nonzero().item())
+
+    # end to end through the host-buffer entry points (pinned memory, copies timed)
+    e2e = None
+    if not args.no_e2e:
+        e2e = measure_e2e(tl, act, lay, n, k, thr, dev, args.e2e_steps, world)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_hbm_peak()
+    build_gbs = act_bytes / (build_ms * 1e-3) / 1e9
+    verify_gbs = act_bytes / (verify_ms * 1e-3) / 1e9
+    line = {
+        "metric": "proof_chunks_per_s_generate_plus_verify",
+        "value": n * world / (ms_per_step * 1e-3), "unit": "chunks/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u16/u32 integer (bf16 bit patterns)", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload), "chunks": n, "proof_bytes": 2 + 2 * k,
+                   "activation_bytes": act_bytes, "l2": "inputs larger than L2 (no flush needed)",
+                   "recomputed": "honest reorder noise, relative 2^-8", "parallelism": "chunks sharded, no collective"},
+        "generate": {"ms": build_ms, "chunks_per_s": n / (build_ms * 1e-3), "GB_per_s": build_gbs,
+                     "frac_of_measured_copy_peak": build_gbs / peak, "frac_of_8TBs_nominal": build_gbs / 8000.0},
+        "verify": {"ms": verify_ms, "chunks_per_s": n / (verify_ms * 1e-3), "GB_per_s": verify_gbs,
+                   "frac_of_measured_copy_peak": verify_gbs / peak, "frac_of_8TBs_nominal": verify_gbs / 8000.0},
+        "activation_GB_per_s": 2 * act_bytes / (ms_per_step * 1e-3) / 1e9,
+        "roofline": {"bound": "hbm", "kernel": "toploc_build_kernel<bf16, flat>",
+                     "achieved": build_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": build_gbs / peak, "traffic": None},
+        "roofline_verify": {"bound": "hbm", "kernel": "toploc_verify_kernel<bf16, flat>",
+                            "achieved": verify_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                            "frac": verify_gbs / peak, "traffic": None},
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+        "checks": {"accepted_chunks": accepted, "chunks_with_status": bad_status},
+        "e2e": e2e,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(act, recomputed, S, T, H, L, k)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure_e2e(tl, act, lay, n, k, thr, dev, steps, world):
+    """Host-buffer path: activations in pinned host memory, proofs and results returned to the host."""
+    import torch.distributed as dist
+    act_bytes = act.numel() * act.element_size()
+    try:
+        h_act = torch.empty(act.shape, dtype=act.dtype, pin_memory=True)
+    except RuntimeError as e:
+        return {"value": None, "unit": "chunks/s", "error": "pinned allocation failed: %s" % e}
+    h_act.copy_(act)
+    h_proofs = torch.empty((n, 2 + 2 * k), dtype=torch.uint8, pin_memory=True)
+    h_status = torch.empty((n,), dtype=torch.uint8, pin_memory=True)
+    h_results = torch.empty((n, 40), dtype=torch.uint8, pin_memory=True)
+    staging = torch.empty(max(tl.toploc_staging_bytes(lay) * 8, 1 << 20), dtype=torch.uint8, device=dev)
+
+    def step():
+        tl.toploc_build_proofs_host(h_act, lay, h_proofs, h_status, staging)
+        tl.toploc_verify_proofs_host(h_act, lay, h_proofs, thr, h_results, staging)
+
+    step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / steps
+    if world > 1:
+        t = torch.tensor([dt], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = t.item()
+    proofs_b = n * (2 + 2 * k)
+    return {"value": n * world / dt, "unit": "chunks/s", "ms_per_step": dt * 1e3, "steps": steps,
+            "h2d_bytes_per_step": 2 * act_bytes + proofs_b, "d2h_bytes_per_step": proofs_b + n + n * 40,
+            "note": "build then verify (identical copy) from pinned host memory; PCIe-bound"}
+
+
+def cpu_baseline(act, recomputed, S, T, H, L, k):
+    import oracle
+    from paper_2501_16007_b200 import synth
+    host = synth.host_patterns(act[:T])
+    host_rec = synth.host_patterns(recomputed[:T])
+    cores = oracle.default_threads()
+    chunks = T // L
+    t0 = time.perf_counter()
+    proofs, status, idx = oracle.build_proofs(host, L, k, 1, T, threads=cores)
+    t1 = time.perf_counter()
+    oracle.verify_proofs(host_rec, proofs, L, k, 1, T, gen_indices=idx, threads=cores)
+    t2 = time.perf_counter()
+    return {"value": chunks / (t2 - t0), "unit": "chunks/s", "cores": cores, "kind": "oracle",
+            "sample": "first sequence: %d chunks of %d x %d bf16, build + verify" % (chunks, L, H),
+            "generate_chunks_per_s": chunks / (t1 - t0), "verify_chunks_per_s": chunks / (t2 - t1)}
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,251 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded bytes.  Proof bytes, selected indices, statuses and every integer statistic must be
+identical; fp64 mean / median within 1e-9 (helpers.MEAN_TOL)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2501_16007_b200 as tl
+from paper_2501_16007_b200 import synth
+
+from helpers import (assert_build_equal, assert_results_equal, gpu_build, gpu_verify, oracle_thresholds,
+                     parity_case)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def from_patterns(pat):
+    """uint16 numpy patterns -> bf16 CUDA tensor with those exact bits."""
+    return torch.from_numpy(pat.view(np.int16).copy()).view(torch.bfloat16).to(DEV)
+
+
+# ------------------------------------------------------------------ small shapes, every code path
+
+@pytest.mark.parametrize("hidden,rows,chunk_len,k", [
+    (4096, 96, 32, 128),     # three chunks of the paper's shape
+    (2048, 50, 16, 32),      # ragged last chunk (50 = 3 * 16 + 2)
+    (8192, 64, 64, 256),     # 2 MiB-class chunk in fp32 terms, largest k
+    (1000, 40, 8, 64),       # hidden not a multiple of 8: element-wise loads
+    (64, 7, 7, 5),           # smaller than one tile
+    (520, 33, 32, 128),      # 16-byte aligned rows, odd tile remainder
+])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_small_shapes(hidden, rows, chunk_len, k, dtype):
+    act = synth.make_activations(2, rows, hidden, dtype, seed=hidden + rows, device=DEV,
+                                 outliers="jitter")
+    noisy = synth.honest_noise(act, seed=5)
+    other = synth.make_activations(2, rows, hidden, dtype, seed=999, device=DEV, outliers="jitter")
+    parity_case(act, chunk_len, k, 2, rows, recomputed={"honest": noisy, "other": other},
+                where="H%d L%d k%d %s" % (hidden, chunk_len, k, dtype))
+
+
+@pytest.mark.parametrize("outliers", ["fixed", "none"])
+def test_outlier_recipes(outliers):
+    act = synth.make_activations(3, 64, 4096, torch.bfloat16, seed=3, device=DEV, outliers=outliers)
+    fp8 = synth.fp8_roundtrip(act)
+    parity_case(act, 32, 128, 3, 64, recomputed={"fp8": fp8}, where=outliers)
+
+
+def test_padded_rows_take_the_strided_path():
+    wide = synth.make_activations(1, 70, 1024 + 64, torch.bfloat16, seed=8, device=DEV, outliers="none")
+    act = wide[:, :1024]                       # row stride 1088, hidden 1024: aligned rows with padding
+    assert not act.is_contiguous()
+    parity_case(act, 32, 64, 1, 70, where="strided")
+    odd = wide[:, 1:1001]                      # misaligned start: element-wise path
+    host = synth.host_patterns(wide)[:, 1:1001]
+    g = gpu_build(odd, 32, 64, 1, 70)
+    r = oracle.build_proofs(host, 32, 64, 1, 70)
+    assert_build_equal(g, r, "misaligned")
+
+
+def test_ragged_batch_with_empty_sequence():
+    act = synth.make_activations(1, 23 + 40, 512, torch.bfloat16, seed=12, device=DEV, outliers="jitter")
+    offsets = [0, 9, 9, 23, 63]
+    parity_case(act, 4, 16, 4, seq_offsets=offsets, where="ragged")
+
+
+# ------------------------------------------------------------------ degenerate inputs
+
+def test_all_equal_and_all_zero_chunks():
+    for pattern in (0x0000, 0x42A0, 0x8000):
+        pat = np.full((64, 2048), pattern, np.uint16)
+        act = from_patterns(pat)
+        g = gpu_build(act, 32, 128, 1, 64)
+        r = oracle.build_proofs(pat, 32, 128, 1, 64)
+        assert_build_equal(g, r, "constant %04x" % pattern)
+        assert g[2].cpu().numpy()[0].tolist() == list(range(128))
+
+
+def test_growing_magnitudes_overflow_the_candidate_buffer():
+    # every element beats all earlier ones: the filter never rejects anything
+    n = 32 * 1024
+    pat = (np.arange(n, dtype=np.uint32) // 2 + 0x0100).astype(np.uint16).reshape(32, 1024)
+    act = from_patterns(pat)
+    g = gpu_build(act, 32, 128, 1, 32)
+    r = oracle.build_proofs(pat, 32, 128, 1, 32)
+    assert_build_equal(g, r, "ascending")
+    # and the mirror image: the first tile already holds the answer
+    pat2 = pat.reshape(-1)[::-1].copy().reshape(32, 1024)
+    g = gpu_build(from_patterns(pat2), 32, 128, 1, 32)
+    r = oracle.build_proofs(pat2, 32, 128, 1, 32)
+    assert_build_equal(g, r, "descending")
+
+
+def test_heavy_ties_at_the_cut():
+    rng = np.random.default_rng(4)
+    vals = rng.integers(0, 5, size=(32, 4096)).astype(np.uint16) * 0x0080 + 0x3F80  # 5 magnitudes
+    vals ^= (rng.integers(0, 2, size=vals.shape).astype(np.uint16) << 15)
+    act = from_patterns(vals)
+    for k in (1, 7, 128, 256):
+        g = gpu_build(act, 32, k, 1, 32)
+        r = oracle.build_proofs(vals, 32, k, 1, 32)
+        assert_build_equal(g, r, "ties k=%d" % k)
+
+
+def test_chunk_smaller_than_k_and_nan_patterns():
+    pat = np.zeros((3, 40), np.uint16)
+    pat[0, 3] = 0xFFF5          # negative NaN pattern >= p
+    pat[1, 7] = 0x7FC0          # positive NaN: ranks above everything finite
+    pat[2, 1] = 0x7F80          # +Inf
+    act = from_patterns(pat)
+    # chunk_len 2 -> chunks of 80 and 40 elements; k = 64 exceeds the second
+    g = gpu_build(act, 2, 64, 1, 3)
+    r = oracle.build_proofs(pat, 2, 64, 1, 3)
+    assert_build_equal(g, r, "nan")
+    assert r[1].tolist() == [oracle.ST_NONFINITE, oracle.ST_K_EXCEEDS]
+    gv = gpu_verify(act, g[0], 2, 64, 1, 3, gen_indices=g[2])
+    rv = oracle.verify_proofs(pat, r[0], 2, 64, 1, 3, gen_indices=r[2], **oracle_thresholds(64))
+    assert_results_equal(gv, rv, "nan verify")
+
+
+def test_malformed_proofs_are_reported_not_trusted():
+    act = synth.make_activations(1, 64, 1024, torch.bfloat16, seed=2, device=DEV)
+    g = gpu_build(act, 32, 32, 1, 64)
+    proofs = g[0].clone()
+    proofs[0, 0], proofs[0, 1] = 0x00, 0x80      # m = 32768
+    proofs[1, 4], proofs[1, 5] = 0xF1, 0xFF      # coefficient = p
+    gv = gpu_verify(act, proofs, 32, 32, 1, 64)
+    rv = oracle.verify_proofs(synth.host_patterns(act), proofs.cpu().numpy(), 32, 32, 1, 64,
+                              **oracle_thresholds(32))
+    assert_results_equal(gv, rv, "bad proof")
+    assert gv["status"].tolist() == [3, 3]
+
+
+def test_sign_bit_reading_switch():
+    act = synth.make_activations(1, 64, 4096, torch.bfloat16, seed=6, device=DEV)
+    other = synth.make_activations(1, 64, 4096, torch.bfloat16, seed=1006, device=DEV)
+    g = gpu_build(act, 32, 128, 1, 64)
+    for sign in (True, False):
+        thr = tl.default_thresholds(128, sign_in_exponent=sign)
+        gv = gpu_verify(other, g[0], 32, 128, 1, 64, thresholds=thr)
+        rv = oracle.verify_proofs(synth.host_patterns(other), g[0].cpu().numpy(), 32, 128, 1, 64,
+                                  **oracle_thresholds(128, sign))
+        assert_results_equal(gv, rv, "sign=%s" % sign)
+
+
+def test_host_buffer_entry_points_match_device_ones():
+    act = synth.make_activations(5, 96, 2048, torch.bfloat16, seed=21, device=DEV, outliers="jitter")
+    lay, _ = tl.make_layout(act, 32, 128, 5, 96)
+    n = tl.toploc_num_chunks(lay)
+    g = gpu_build(act, 32, 128, 5, 96)
+    h_act = act.cpu().pin_memory()
+    h_proofs = torch.empty((n, 258), dtype=torch.uint8).pin_memory()
+    h_status = torch.empty((n,), dtype=torch.uint8).pin_memory()
+    # staging for two sequences at a time: the batch goes through in three groups
+    staging = torch.empty(2 * tl.toploc_staging_bytes(lay) + 4096, dtype=torch.uint8, device=DEV)
+    tl.toploc_build_proofs_host(h_act, lay, h_proofs, h_status, staging)
+    assert torch.equal(h_proofs, g[0].cpu()) and torch.equal(h_status, g[1].cpu())
+    h_res = torch.empty((n, 40), dtype=torch.uint8).pin_memory()
+    tl.toploc_verify_proofs_host(h_act, lay, h_proofs, tl.default_thresholds(), h_res, staging)
+    gv = gpu_verify(act, g[0], 32, 128, 5, 96)
+    hv = h_res.numpy().view(tl.RESULT_DTYPE).reshape(-1)
+    assert_results_equal(hv, gv, "host variant")
+    small = torch.empty(1024, dtype=torch.uint8, device=DEV)
+    with pytest.raises(tl.ToplocError):
+        tl.toploc_build_proofs_host(h_act, lay, h_proofs, h_status, small)
+
+
+# ------------------------------------------------------------------ the named configurations
+
+def test_config_tiny():
+    """1 sequence, 4 chunks of 32 x 4096 bf16, seed 0, k = 128: generate, validate an identical
+    copy and a +1-ulp copy."""
+    act = synth.make_activations(1, 128, 4096, torch.bfloat16, seed=0, device=DEV)
+    ulp = synth.plus_one_ulp(act, seed=0)
+    r, v = parity_case(act, 32, 128, 1, 128, recomputed={"ulp": ulp}, where="tiny")
+    assert r[0].shape == (4, 258)
+    assert v["same"]["accept"].tolist() == [1] * 4 and not v["same"]["mant_diff_sum"].any()
+    assert v["ulp"]["accept"].tolist() == [1] * 4
+
+
+def test_config_8b_decode_and_validation_sweep():
+    """64 sequences x 2048 tokens, H = 4096 (4096 proofs), then the validation sweep: honest
+    reorder noise, other seed, fp8 round trip, 16-token prefix shift -- every chunk compared."""
+    S, T, H = 64, 2048, 4096
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=2, device=DEV)
+    other = synth.make_activations(S, T, H, torch.bfloat16, seed=1002, device=DEV)
+    rec = {
+        "honest": synth.honest_noise(act, seed=3),
+        "other_seed": other,
+        "fp8": synth.fp8_roundtrip(act),
+        "prefix_shift": synth.prefix_shift(act, other, S, T, 16),
+    }
+    r, v = parity_case(act, 32, 128, S, T, recomputed=rec, where="8B")
+    assert r[0].shape == (4096, 258) and not r[1].any()
+    assert v["same"]["accept"].all() and v["honest"]["accept"].all()
+    assert not v["other_seed"]["accept"].any() and not v["prefix_shift"]["accept"].any()
+
+
+def test_config_70b_full_size_sampled():
+    """256 sequences x 4096 tokens, H = 8192 (~17 GB): generate and validate at full size in the
+    launch configuration the benchmark times; the oracle checks whole sampled sequences, and
+    properties that hold for every chunk are checked on all 32768."""
+    S, T, H = 256, 4096, 8192
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2 ** 30:
+        pytest.skip("needs 40 GB of free device memory")
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=4, device=DEV)
+    g = gpu_build(act, 32, 128, S, T)
+    assert not g[1].any().item()
+    same = gpu_verify(act, g[0], 32, 128, S, T, gen_indices=g[2])
+    assert same["accept"].all() and not same["exp_mismatch"].any() and not same["mant_diff_sum"].any()
+    assert (same["n_match"] == 128).all() and not same["topk_mismatch"].any()
+    assert ((same["modulus"] >= 32769) & (same["modulus"] <= 65536)).all()
+    noisy = synth.honest_noise(act, seed=5)
+    honest = gpu_verify(noisy, g[0], 32, 128, S, T, gen_indices=g[2])
+    cps = T // 32
+    for s in (0, 77, 255):
+        rows = slice(s * T, (s + 1) * T)
+        host = synth.host_patterns(act[rows])
+        r = oracle.build_proofs(host, 32, 128, 1, T)
+        sub = (g[0][s * cps:(s + 1) * cps], g[1][s * cps:(s + 1) * cps], g[2][s * cps:(s + 1) * cps])
+        assert_build_equal(sub, r, "70B seq %d" % s)
+        rv = oracle.verify_proofs(synth.host_patterns(noisy[rows]), r[0], 32, 128, 1, T, gen_indices=r[2],
+                                  **oracle_thresholds(128))
+        assert_results_equal(honest[s * cps:(s + 1) * cps], rv, "70B honest seq %d" % s)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("hidden", [2048, 4096, 8192])
+def test_config_sweep(hidden, dtype):
+    """k in {32, 64, 128, 256} x chunk length in {16, 32, 64} at 128 sequences x 1024 tokens;
+    the GPU runs the full point, the oracle checks two whole sequences of it."""
+    S, T = 128, 1024
+    act = synth.make_activations(S, T, hidden, dtype, seed=50 + hidden // 1024, device=DEV)
+    noisy = synth.honest_noise(act, seed=9)
+    for chunk_len in (16, 32, 64):
+        cps = T // chunk_len
+        for k in (32, 64, 128, 256):
+            g = gpu_build(act, chunk_len, k, S, T)
+            gv = gpu_verify(noisy, g[0], chunk_len, k, S, T, gen_indices=g[2])
+            for s in (1, 126):
+                rows = slice(s * T, (s + 1) * T)
+                r = oracle.build_proofs(synth.host_patterns(act[rows]), chunk_len, k, 1, T)
+                sub = tuple(t[s * cps:(s + 1) * cps] for t in g)
+                where = "sweep H%d L%d k%d %s seq %d" % (hidden, chunk_len, k, dtype, s)
+                assert_build_equal(sub, r, where)
+                rv = oracle.verify_proofs(synth.host_patterns(noisy[rows]), r[0], chunk_len, k, 1, T,
+                                          gen_indices=r[2], **oracle_thresholds(k))
+                assert_results_equal(gv[s * cps:(s + 1) * cps], rv, where)

@@ -1,0 +1,95 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header declares, and its
+host-only queries behave.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2501_16007_b200 as tl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built_library():
+    from paper_2501_16007_b200.csrc import build
+    build.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "toploc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(toploc_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    lib = tl.load_library()
+    names = declared_functions()
+    assert "toploc_build_proofs" in names and "toploc_verify_proofs" in names and len(names) >= 11
+    for name in names:
+        assert hasattr(lib, name), name
+        assert hasattr(tl, name), "binding lacks %s" % name
+
+
+def test_struct_sizes_match_the_header():
+    assert ctypes.sizeof(tl.ToplocLayout) == 48
+    assert ctypes.sizeof(tl.ToplocThresholds) == 24
+    assert tl.RESULT_DTYPE.itemsize == 40
+
+
+def layout(**kw):
+    lay = tl.ToplocLayout()
+    base = dict(dtype=0, hidden=4096, chunk_len=32, k=128, num_seqs=2, reserved=0, tokens_per_seq=100,
+                row_stride=4096)
+    base.update(kw)
+    for key, val in base.items():
+        setattr(lay, key, val)
+    return lay
+
+
+def test_constants_and_sizes():
+    assert tl.toploc_get_constants() == (65521, 32769, 65536)
+    assert tl.toploc_proof_bytes(128) == 258
+    assert [tl.toploc_proof_bytes(k) for k in (32, 64, 256)] == [66, 130, 514]
+    assert tl.toploc_status_string(0) == "ok" and "modulus" in tl.toploc_status_string(1)
+    assert tl.toploc_error_string(-3).startswith("workspace")
+
+
+def test_chunk_counting():
+    assert tl.toploc_num_chunks(layout()) == 2 * 4          # ceil(100 / 32) per sequence
+    assert tl.toploc_num_chunks(layout(tokens_per_seq=4096, num_seqs=256)) == 32768
+    assert tl.toploc_workspace_bytes(layout()) == 0
+    offs = np.array([0, 9, 9, 23], np.int64)
+    lay = layout(num_seqs=3, chunk_len=4)
+    lay.seq_offsets = offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64))
+    assert tl.toploc_num_chunks(lay) == 7
+    assert tl.toploc_workspace_bytes(lay) == 7 * 16
+    assert tl.toploc_staging_bytes(layout()) >= 100 * 4096 * 2 + 4 * 258
+
+
+@pytest.mark.parametrize("bad", [dict(k=0), dict(k=257), dict(hidden=0), dict(chunk_len=0), dict(num_seqs=0),
+                                 dict(dtype=7), dict(row_stride=100), dict(tokens_per_seq=0),
+                                 dict(reserved=1), dict(hidden=1 << 20, chunk_len=64, row_stride=1 << 20)])
+def test_invalid_layouts_are_refused(bad):
+    with pytest.raises(tl.ToplocError):
+        tl.toploc_num_chunks(layout(**bad))
+
+
+def test_device_entry_points_refuse_host_tensors():
+    act = torch.zeros((64, 64), dtype=torch.bfloat16)
+    lay, _ = tl.make_layout(act, 32, 8, 1, 64)
+    with pytest.raises(tl.ToplocError):
+        tl.toploc_build_proofs(act, lay)
+
+
+def test_null_pointers_are_refused_before_any_cuda_call():
+    lib = tl.load_library()
+    lay = layout()
+    assert lib.toploc_build_proofs(None, ctypes.byref(lay), None, None, None, None, 0, None) == -1
+    thr = tl.default_thresholds()
+    assert lib.toploc_verify_proofs(None, ctypes.byref(lay), None, ctypes.byref(thr), None, None, None, 0,
+                                    None) == -1
+    assert lib.toploc_build_proofs_host(None, ctypes.byref(lay), None, None, None, 0, None) == -1
