@@ -116,8 +116,10 @@ int64_t toploc_num_chunks(const toploc_layout* lay);
 /* 2 + 2k: a 2-byte modulus and k 2-byte coefficients (Section 4, Section 5.7). */
 size_t toploc_proof_bytes(int32_t k);
 
-/* Bytes of device scratch build/verify need for this layout: 0 for uniform
- * batches, a per-chunk row table for ragged ones (seq_offsets != NULL). */
+/* Bytes of device scratch build/verify need for this layout: the selected
+ * (index, pattern) pairs of every chunk (6k + 1 bytes per chunk) that the
+ * select kernel hands to the arithmetic kernel, plus a per-chunk row table for
+ * ragged batches (seq_offsets != NULL). */
 size_t toploc_workspace_bytes(const toploc_layout* lay);
 
 /* Smallest device staging buffer the *_host entry points accept for this
@@ -153,7 +155,7 @@ const char* toploc_error_string(int return_code);
  * d_indices_opt DEVICE  out, optional (NULL to skip): [num_chunks, k] selected
  *                       flat indices ordered by (magnitude desc, index asc)
  * d_workspace   DEVICE  scratch of at least toploc_workspace_bytes(lay) bytes,
- *                       8-byte aligned; may be NULL when that is 0
+ *                       16-byte aligned; contents are undefined afterwards
  * cuda_stream   a cudaStream_t (NULL = default stream)
  *
  * Asynchronous: returns after enqueueing; results are valid once the stream

@@ -1,12 +1,20 @@
-// TopLoc proof hot path for sm_100a: one thread block per chunk streams the
-// chunk from HBM once, keeps the exact top-k on chip, and finishes the chunk in
-// the same kernel (build: injective modulus, interpolation over Z_p, packing;
-// verify: Horner evaluation, bit-field comparison, statistics, verdict).
+// TopLoc proof hot path for sm_100a.
+//
+// Two kernels per call:
+//   select   one 128-thread block per chunk streams the chunk from HBM exactly
+//            once and keeps the exact top-k on chip (Algorithm 1 / 2, topk());
+//            for proof generation it also runs the injective-modulus search
+//            (Algorithm 6).  The k (index, pattern) pairs go to scratch memory.
+//   tail     one warp per chunk does the arithmetic over Z_p: Newton
+//            interpolation and packing (Algorithm 3, proof generation) or
+//            Horner evaluation, bit-field comparison, statistics and verdict
+//            (Algorithms 5 and 2, validation).
 //
 // The path is a selection over data read once plus integer modular arithmetic:
 // HBM bandwidth is the roofline, there is no dense contraction and therefore no
-// tensor-core work.  Blocks of 128 threads, many per SM, so that blocks that
-// are in their arithmetic tail overlap with blocks that are streaming.
+// tensor-core work.  The select kernel is built to keep many 16-byte loads in
+// flight per SM (small blocks, many per SM, software-pipelined tiles) and to
+// spend about one instruction per element on the elements that lose.
 #include "toploc.h"
 
 #include <cuda_runtime.h>
@@ -26,17 +34,26 @@ constexpr uint32_t kModLow = 32769u;
 // ---------------------------------------------------------------------------
 // launch shape
 // ---------------------------------------------------------------------------
-constexpr int kThreads = 128;            // threads per block
-constexpr int kUnroll = 4;               // 16-byte loads in flight per thread and tile
-constexpr int kCandCap = 1536;           // candidate buffer entries (8 bytes each)
+#ifndef TOPLOC_SELECT_MIN_BLOCKS
+#define TOPLOC_SELECT_MIN_BLOCKS 13      // select: one-warp blocks per SM (shared memory allows 13)
+#endif
+#ifndef TOPLOC_SELECT_STAGES
+#define TOPLOC_SELECT_STAGES 3           // select: tiles in flight per warp
+#endif
+constexpr int kThreads = 32;             // select: one warp per chunk
+constexpr int kUnroll = 4;               // select: 16-byte loads per lane and tile
+constexpr int kStages = TOPLOC_SELECT_STAGES;
+constexpr int kCandCap = 640;            // select: candidate buffer entries (8 bytes each)
+constexpr int kHitCap = 96;              // select: vectors that can be parked between drains
+constexpr int kHitTrigger = 32;          // select: drain once this many are parked
 constexpr int kMaxK = TOPLOC_MAX_K;
-constexpr int kEntriesPerThread = kMaxK / kThreads;  // tail arrays: entries owned per thread
+constexpr int kMaxSlots = kMaxK / 32;    // tail: entries a lane owns at most
 constexpr int kIdxBits = 24;             // flat index field of a candidate
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
+constexpr int kInterpWarps = 32;         // interpolation kernel: warps (= chunks in flight) per block
+constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
-static_assert(kMaxK % kThreads == 0, "tail loops assume whole entries per thread");
-static_assert(kCandCap >= kMaxK + kThreads * 8, "a safe sub-tile must fit after a compaction");
-static_assert(kCandCap * 8 >= 8192 && kCandCap * 8 >= 6 * kMaxK * 4, "buffer is reused by the tail");
+static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
 
 struct ChunkSpan {   // one per chunk of a ragged batch, built on the host
   long long row0;
@@ -55,10 +72,13 @@ struct BatchParams {
   int chunks_per_seq;
 };
 
-struct BuildOut {
-  uint8_t* proofs;
-  uint8_t* status;
-  int32_t* indices;            // optional
+// What the select kernel leaves behind for the tail kernel.
+struct Selection {
+  uint32_t* idx;       // [num_chunks, k] selected flat indices
+  uint16_t* bits;      // [num_chunks, k] their 16-bit patterns
+  uint8_t* status;     // [num_chunks] TOPLOC_CHUNK_*; the caller's d_status during proof generation
+  uint8_t* proofs;     // proof generation only: receives the modulus (or zeros)
+  int32_t* indices;    // optional: indices in rank order
 };
 
 struct VerifyIo {
@@ -78,18 +98,46 @@ __device__ __forceinline__ unsigned long long make_candidate(uint32_t key, uint3
   return ((unsigned long long)key << (kIdxBits + 1)) | ((unsigned long long)(kIdxMask - flat) << 1) | sign;
 }
 
-struct __align__(16) BlockShared {
-  unsigned long long cand[kCandCap];  // candidates; later the modulus bitmap, then the tail arrays
-  uint32_t hist[256];
-  uint32_t idx[kMaxK];                // selected flat indices in rank order
-  uint16_t bits[kMaxK];               // selected 16-bit patterns in rank order
-  int count;
+struct __align__(16) SelectShared {
+  uint4 ring[kStages * kUnroll * kThreads];  // tiles on their way from HBM (asynchronous copies)
+  unsigned long long cand[kCandCap];  // candidates held; ring + cand later serve as the residue set
+  uint4 hit_vec[kHitCap];             // vectors that passed the streaming filter, not yet unpacked
+  uint32_t hit_idx[kHitCap];          // their vector index within the chunk
+  uint32_t hist[256];                 // digit histogram of a compaction pass
+  uint32_t top_hist[256];             // held candidates by the upper 8 bits of their 15-bit key
+  uint32_t low_hist[128];             // those whose upper bits equal top_bin, by the lower 7 bits
+  int count;                          // candidates held
+  int nhits;                          // hit vectors held
+  uint32_t top_bin;                   // which upper-bits value low_hist describes (kNoBin: none)
   uint32_t digit;
+  uint32_t bin;
   int want;
-  uint32_t err_e;
-  uint32_t diff_sum;
-  uint32_t common;
 };
+constexpr uint32_t kNoBin = 0xFFFFFFFFu;
+static_assert(sizeof(uint4) * kStages * kUnroll * kThreads + 8 * kCandCap >= 8192,
+              "ring + candidates double as the 65536-bit residue set");
+
+// The block is one warp, so a block barrier is a warp barrier that also orders
+// shared memory.
+__device__ __forceinline__ void warp_barrier() { __syncwarp(); }
+
+// A shared-memory word as the whole warp agrees on it: lane 0 reads, everyone
+// receives.  Used for every value that steers a branch, so that a lane running
+// ahead (and already appending again) cannot make the others see another value.
+template <typename T>
+__device__ __forceinline__ T uniform_load(const T* p) {
+  T v = T();
+  if (threadIdx.x == 0) v = *p;
+  return __shfl_sync(0xFFFFFFFFu, v, 0);
+}
+
+// The 15-bit key the running threshold is kept in: a bf16 key as it is, the
+// upper half of an fp32 key.
+template <int DT>
+__device__ __forceinline__ uint32_t coarse_key(unsigned long long cand) {
+  const uint32_t key = (uint32_t)(cand >> (kIdxBits + 1));
+  return DT == 0 ? key : (key >> 16);
+}
 
 __device__ __forceinline__ uint4 load_streaming(const uint4* p) {
   uint4 v;
@@ -99,9 +147,32 @@ __device__ __forceinline__ uint4 load_streaming(const uint4* p) {
   return v;
 }
 
-__device__ __forceinline__ void push_candidate(BlockShared& sh, unsigned long long c, int& max_pos) {
+// 16 bytes global -> shared without passing through registers; completion is
+// tracked per thread in commit groups (a thread only ever reads what it copied).
+__device__ __forceinline__ void copy_async_16(void* smem_dst, const void* gmem_src) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void copy_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <int DT>
+__device__ __forceinline__ void count_candidate(SelectShared& sh, unsigned long long c) {
+  const uint32_t key = coarse_key<DT>(c);
+  atomicAdd(&sh.top_hist[key >> 7], 1u);
+  if ((key >> 7) == sh.top_bin) atomicAdd(&sh.low_hist[key & 127u], 1u);
+}
+
+template <int DT>
+__device__ __forceinline__ void push_candidate(SelectShared& sh, unsigned long long c, int& max_pos) {
   int pos = atomicAdd(&sh.count, 1);
-  if (pos < kCandCap) sh.cand[pos] = c;
+  if (pos < kCandCap) {
+    sh.cand[pos] = c;
+    count_candidate<DT>(sh, c);
+  }
   max_pos = max(max_pos, pos);
 }
 
@@ -120,14 +191,17 @@ struct ChunkSource {
   int hidden;
   int vecs_per_row;
 
+  // address of vector v (MODE 0 and 1 only)
+  __device__ __forceinline__ const void* address(int v) const {
+    if (MODE == 0) return reinterpret_cast<const uint4*>(base) + v;
+    int t = v / vecs_per_row;
+    int c = v - t * vecs_per_row;
+    return base + ((long long)t * row_stride + (long long)c * kVec) * kElemBytes;
+  }
+
   __device__ __forceinline__ uint4 load(int v) const {
-    if (MODE == 0) {
-      return load_streaming(reinterpret_cast<const uint4*>(base) + v);
-    } else if (MODE == 1) {
-      int t = v / vecs_per_row;
-      int c = v - t * vecs_per_row;
-      const char* p = base + ((long long)t * row_stride + (long long)c * kVec) * kElemBytes;
-      return load_streaming(reinterpret_cast<const uint4*>(p));
+    if (MODE != 2) {
+      return load_streaming(reinterpret_cast<const uint4*>(address(v)));
     } else {
       int t = v / hidden;
       int c = v - t * hidden;
@@ -140,243 +214,388 @@ struct ChunkSource {
   }
 };
 
-// Appends every element of one vector whose key is >= thr.  flat0 = flat index
-// of the vector's first element.  bf16 fast test: with both 15-bit keys of a
-// word in separate 16-bit lanes, adding (0x8000 - thr) to each lane sets the
-// lane's top bit exactly when key >= thr (no carry leaves a lane).
+// Does any element of the vector have key >= thr?  bf16: both 15-bit keys of a
+// word sit in separate 16-bit lanes, and adding (0x8000 - thr) to a lane sets
+// its top bit exactly when key >= thr (no carry leaves a lane).  The OR of the
+// four words is tested first: a bitwise OR is never below any of its operands,
+// so a vector whose OR fails the test holds no candidate.
 template <int DT, int VEC>
-__device__ __forceinline__ void filter_vector(BlockShared& sh, const uint4& w, uint32_t thr, uint32_t flat0,
-                                              int& max_pos) {
+__device__ __forceinline__ bool vector_has_candidate(const uint4& w, uint32_t thr, uint32_t add) {
+  if (VEC == 1) {
+    return (DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu)) >= thr;
+  } else if (DT == 0) {
+    const uint32_t any = (w.x | w.y | w.z | w.w) & 0x7FFF7FFFu;
+    if (((any + add) & 0x80008000u) == 0) return false;
+    const uint32_t t0 = (w.x & 0x7FFF7FFFu) + add, t1 = (w.y & 0x7FFF7FFFu) + add;
+    const uint32_t t2 = (w.z & 0x7FFF7FFFu) + add, t3 = (w.w & 0x7FFF7FFFu) + add;
+    return ((t0 | t1 | t2 | t3) & 0x80008000u) != 0;
+  } else {
+    const uint32_t any = (w.x | w.y | w.z | w.w) & 0x7FFFFFFFu;
+    if (any < thr) return false;
+    return (w.x & 0x7FFFFFFFu) >= thr || (w.y & 0x7FFFFFFFu) >= thr || (w.z & 0x7FFFFFFFu) >= thr ||
+           (w.w & 0x7FFFFFFFu) >= thr;
+  }
+}
+
+__device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
+
+// Appends every element of one vector whose key is >= thr to the candidate
+// buffer.  flat0 = flat index of the vector's first element.
+template <int DT, int VEC>
+__device__ __forceinline__ void push_vector(SelectShared& sh, const uint4& w, uint32_t thr, uint32_t flat0,
+                                            int& max_pos) {
   if (VEC == 1) {
     uint32_t key = DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu);
     uint32_t sign = DT == 0 ? (w.x >> 15) & 1u : (w.x >> 31);
-    if (key >= thr) push_candidate(sh, make_candidate(key, flat0, sign), max_pos);
+    if (key >= thr) push_candidate<DT>(sh, make_candidate(key, flat0, sign), max_pos);
   } else if (DT == 0) {
-    const uint32_t add = (0x8000u - thr) * 0x00010001u;
-    uint32_t t0 = (w.x & 0x7FFF7FFFu) + add;
-    uint32_t t1 = (w.y & 0x7FFF7FFFu) + add;
-    uint32_t t2 = (w.z & 0x7FFF7FFFu) + add;
-    uint32_t t3 = (w.w & 0x7FFF7FFFu) + add;
-    if ((t0 | t1 | t2 | t3) & 0x80008000u) {
-      const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-      const uint32_t tests[4] = {t0, t1, t2, t3};
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        if (tests[i] & 0x00008000u)
-          push_candidate(sh, make_candidate(words[i] & 0x7FFFu, flat0 + 2 * i, (words[i] >> 15) & 1u), max_pos);
-        if (tests[i] & 0x80000000u)
-          push_candidate(sh, make_candidate((words[i] >> 16) & 0x7FFFu, flat0 + 2 * i + 1, words[i] >> 31),
-                         max_pos);
-      }
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t lo = words[i] & 0x7FFFu, hi = (words[i] >> 16) & 0x7FFFu;
+      if (lo >= thr) push_candidate<DT>(sh, make_candidate(lo, flat0 + 2 * i, (words[i] >> 15) & 1u), max_pos);
+      if (hi >= thr) push_candidate<DT>(sh, make_candidate(hi, flat0 + 2 * i + 1, words[i] >> 31), max_pos);
     }
   } else {
     const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-    bool any = false;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) any |= (words[i] & 0x7FFFFFFFu) >= thr;
-    if (any) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        uint32_t key = words[i] & 0x7FFFFFFFu;
-        if (key >= thr) push_candidate(sh, make_candidate(key, flat0 + i, words[i] >> 31), max_pos);
-      }
+    for (int i = 0; i < 4; ++i) {
+      uint32_t key = words[i] & 0x7FFFFFFFu;
+      if (key >= thr) push_candidate<DT>(sh, make_candidate(key, flat0 + i, words[i] >> 31), max_pos);
     }
   }
 }
 
-// Keeps the k best candidates (radix select on the 56 meaningful bits, most
-// significant digit first) and raises the threshold to "strictly better than
-// the k-th": every later element of the chunk has a higher flat index, so one
-// that only ties the k-th key can no longer be selected.  All threads call it.
-template <int DT>
-__device__ void compact_candidates(BlockShared& sh, int k, uint32_t& thr) {
-  const int tid = threadIdx.x;
-  __syncthreads();
-  const int n = min(sh.count, kCandCap);
-  __syncthreads();
-  if (n <= k) return;
-  constexpr int kPer = kCandCap / kThreads;
-  unsigned long long mine[kPer];
+// The warp walks a histogram from its highest bin down and finds the bin in
+// which the want-th entry (counted from the top) falls; lane l owns bins
+// PER_LANE * l .. PER_LANE * l + PER_LANE - 1.  Writes sh.digit (the bin, or
+// kNoBin when the histogram holds fewer than want entries), sh.bin (its
+// population) and sh.want (the rank wanted inside it).
+template <int PER_LANE>
+__device__ __forceinline__ void find_from_top(SelectShared& sh, const uint32_t* hist, int want) {
+  const int lane = threadIdx.x;
+  warp_barrier();  // results of an earlier call have been read by every lane
+  uint32_t local[PER_LANE];
+  uint32_t sum = 0;
 #pragma unroll
-  for (int i = 0; i < kPer; ++i) {
-    int e = tid + i * kThreads;
-    mine[i] = e < n ? sh.cand[e] : 0ull;
+  for (int b = 0; b < PER_LANE; ++b) {
+    local[b] = hist[lane * PER_LANE + b];
+    sum += local[b];
   }
+  uint32_t incl = sum;  // becomes the sum over lanes >= this one
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    uint32_t other = __shfl_down_sync(0xFFFFFFFFu, incl, off);
+    if (lane + off < 32) incl += other;
+  }
+  const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 0);
+  if (lane == 0 && total < (uint32_t)want) sh.digit = kNoBin;
+  const uint32_t above = incl - sum;  // entries in higher lanes
+  if (above < (uint32_t)want && incl >= (uint32_t)want) {
+    uint32_t acc = above;
+#pragma unroll
+    for (int b = PER_LANE - 1; b >= 0; --b) {
+      if (acc < (uint32_t)want && acc + local[b] >= (uint32_t)want) {
+        sh.digit = (uint32_t)(lane * PER_LANE + b);
+        sh.bin = local[b];
+        sh.want = want - (int)acc;
+      }
+      acc += local[b];
+    }
+  }
+  warp_barrier();
+}
+
+// Raises the threshold from the two key histograms, without touching the
+// candidates: the k-th largest 15-bit key among the held candidates is found
+// by walking top_hist, then low_hist, from the top.  For bf16 that key is
+// exact, and since at least k held candidates reach it and every later element
+// has a higher flat index, later elements must beat it strictly.  For fp32 the
+// 15 bits are only the upper half of the key, so later elements need only
+// reach it.
+template <int DT>
+__device__ __noinline__ uint32_t raise_threshold(SelectShared& sh, int k, uint32_t thr) {
+  const int lane = threadIdx.x;
+  warp_barrier();  // every append and its histogram updates are in
+  find_from_top<8>(sh, sh.top_hist, k);
+  const uint32_t top = sh.digit;
+  const int want = sh.want;
+  if (top == kNoBin) return thr;  // fewer than k candidates so far
+  if (top != sh.top_bin) {
+    // the boundary moved into another upper-bits bin: describe that one
+    warp_barrier();
+    for (int b = lane; b < 128; b += kThreads) sh.low_hist[b] = 0;
+    if (lane == 0) sh.top_bin = top;
+    warp_barrier();
+    const int n = min(uniform_load(&sh.count), kCandCap);
+    for (int e = lane; e < n; e += kThreads) {
+      const uint32_t key = coarse_key<DT>(sh.cand[e]);
+      if ((key >> 7) == top) atomicAdd(&sh.low_hist[key & 127u], 1u);
+    }
+    warp_barrier();
+  }
+  find_from_top<4>(sh, sh.low_hist, want);
+  const uint32_t key = (top << 7) | sh.digit;
+  const uint32_t raised = DT == 0 ? key + 1u : key << 16;
+  warp_barrier();
+  return max(thr, raised);
+}
+
+// Keeps the best candidates (radix select on the 56 meaningful bits, most
+// significant digit first) and returns the raised threshold "strictly better
+// than the k-th".  Ties on the key are only broken by index when it matters:
+// once the key digits are settled the scan stops if the boundary bin can be
+// kept whole -- because exactly k candidates remain, or, for a compaction in
+// mid-stream (exact == false), because at most kMaxK remain; only the last
+// compaction of a chunk must leave exactly k.
+template <int DT>
+__device__ __noinline__ uint32_t compact_candidates(SelectShared& sh, int k, uint32_t thr, bool exact) {
+  const int lane = threadIdx.x;
+  warp_barrier();
+  const int n = min(uniform_load(&sh.count), kCandCap);
+  if (n <= k) return thr;
   unsigned long long prefix = 0ull, mask = 0ull;
   int want = k;
   // bf16 keys have 15 bits: candidate bits 40..55 are zero, two digit passes fewer
+#pragma unroll 1
   for (int shift = (DT == 0 ? 32 : 48); shift >= 0; shift -= 8) {
-    sh.hist[tid] = 0;
-    sh.hist[tid + kThreads] = 0;
-    __syncthreads();
-#pragma unroll
-    for (int i = 0; i < kPer; ++i) {
-      int e = tid + i * kThreads;
-      if (e < n && (mine[i] & mask) == prefix) atomicAdd(&sh.hist[(uint32_t)(mine[i] >> shift) & 255u], 1u);
+    for (int b = lane; b < 256; b += kThreads) sh.hist[b] = 0;
+    warp_barrier();
+    for (int e = lane; e < n; e += kThreads) {
+      const unsigned long long c = sh.cand[e];
+      if ((c & mask) == prefix) atomicAdd(&sh.hist[(uint32_t)(c >> shift) & 255u], 1u);
     }
-    __syncthreads();
-    if (tid < 32) {
-      // lane l owns digits 8l..8l+7; find the largest digit d with
-      // (#candidates with digit >= d) >= want
-      uint32_t local[8];
-      uint32_t sum = 0;
-#pragma unroll
-      for (int b = 0; b < 8; ++b) {
-        local[b] = sh.hist[tid * 8 + b];
-        sum += local[b];
-      }
-      uint32_t incl = sum;  // becomes the sum over lanes >= this one
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        uint32_t other = __shfl_down_sync(0xFFFFFFFFu, incl, off);
-        if (tid + off < 32) incl += other;
-      }
-      uint32_t above = incl - sum;  // candidates in higher lanes
-      if (above < (uint32_t)want && incl >= (uint32_t)want) {
-        uint32_t acc = above;
-#pragma unroll
-        for (int b = 7; b >= 0; --b) {
-          if (acc < (uint32_t)want && acc + local[b] >= (uint32_t)want) {
-            sh.digit = (uint32_t)(tid * 8 + b);
-            sh.want = want - (int)acc;
-          }
-          acc += local[b];
-        }
-      }
-    }
-    __syncthreads();
+    warp_barrier();
+    find_from_top<8>(sh, sh.hist, want);  // largest digit with enough candidates at or above it
     prefix |= (unsigned long long)sh.digit << shift;
     mask |= 255ull << shift;
     want = sh.want;
+    const int kept = k - want + (int)sh.bin;
+    warp_barrier();
+    // lower bits of the pivot stay 0: the boundary bin is kept whole
+    if (shift <= 24 && (kept == k || (!exact && kept <= kMaxK))) break;
   }
-  const unsigned long long pivot = prefix;  // the k-th best candidate itself
-  if (tid == 0) sh.count = 0;
-  __syncthreads();
-#pragma unroll
-  for (int i = 0; i < kPer; ++i) {
-    int e = tid + i * kThreads;
-    if (e < n && mine[i] >= pivot) sh.cand[atomicAdd(&sh.count, 1)] = mine[i];
+  const unsigned long long pivot = prefix;  // everything >= pivot is kept
+  // in-place, in order: a slot is overwritten only after it has been read
+  int out = 0;
+  for (int base = 0; base < n; base += kThreads) {
+    const int e = base + lane;
+    const unsigned long long c = e < n ? sh.cand[e] : 0ull;
+    const bool keep = e < n && c >= pivot;
+    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, keep);
+    const int pos = out + __popc(votes & ((1u << lane) - 1u));
+    warp_barrier();
+    if (keep) sh.cand[pos] = c;
+    out += __popc(votes);
   }
-  __syncthreads();
-  thr = (uint32_t)(pivot >> (kIdxBits + 1)) + 1u;
+  // the key histograms describe the survivors only
+  for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
+  if (lane == 0) {
+    sh.count = out;
+    sh.top_bin = kNoBin;
+  }
+  warp_barrier();
+  for (int e = lane; e < out; e += kThreads) atomicAdd(&sh.top_hist[coarse_key<DT>(sh.cand[e]) >> 7], 1u);
+  warp_barrier();
+  return max(thr, (uint32_t)(pivot >> (kIdxBits + 1)) + 1u);
 }
 
-// Processes vectors [vb, ve) one vector per thread at a time, compacting
-// whenever another round might not fit.  Precondition: count <= k.
+// Processes vectors [vb, ve) one vector per lane at a time, raising the
+// threshold after every round and compacting whenever another round might not
+// fit.
 template <int DT, int MODE>
-__device__ void select_carefully(BlockShared& sh, const ChunkSource<DT, MODE>& src, int vb, int ve, int k,
-                                 uint32_t& thr) {
+__device__ __noinline__ uint32_t select_carefully(SelectShared& sh, const ChunkSource<DT, MODE> src, int vb,
+                                                  int ve, int k, uint32_t thr) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
-  const int tid = threadIdx.x;
-  int max_pos = -1;
+  const int lane = threadIdx.x;
   for (int s = vb; s < ve; s += kThreads) {
-    int v = s + tid;
-    if (v < ve) filter_vector<DT, VEC>(sh, src.load(v), thr, (uint32_t)v * VEC, max_pos);
-    if (__syncthreads_or(max_pos + 1 + kThreads * VEC > kCandCap)) {
-      compact_candidates<DT>(sh, k, thr);
-      max_pos = -1;
-    }
+    warp_barrier();
+    if (uniform_load(&sh.count) + kThreads * VEC > kCandCap) thr = compact_candidates<DT>(sh, k, thr, false);
+    const int v = s + lane;
+    int max_pos = -1;
+    if (v < ve) push_vector<DT, VEC>(sh, src.load(v), thr, (uint32_t)v * VEC, max_pos);
+    thr = raise_threshold<DT>(sh, k, thr);
   }
+  return thr;
 }
 
-// Exact top-k of one chunk.  On return sh.idx / sh.bits hold the k selected
-// flat indices and 16-bit patterns in rank order (magnitude descending, index
-// ascending).  n_elems >= k is the caller's business.
+// Unpacks the held hit vectors into candidates (against the current, possibly
+// higher, threshold), one vector per lane and round, then raises the threshold.
+template <int DT, int VEC>
+__device__ __noinline__ uint32_t drain_hits(SelectShared& sh, int k, uint32_t thr) {
+  const int lane = threadIdx.x;
+  warp_barrier();
+  const int nh = min(uniform_load(&sh.nhits), kHitCap);
+  for (int base = 0; base < nh; base += kThreads) {
+    warp_barrier();
+    if (uniform_load(&sh.count) + kThreads * VEC > kCandCap) thr = compact_candidates<DT>(sh, k, thr, false);
+    const int h = base + lane;
+    int max_pos = -1;
+    if (h < nh) push_vector<DT, VEC>(sh, sh.hit_vec[h], thr, sh.hit_idx[h] * VEC, max_pos);
+    thr = raise_threshold<DT>(sh, k, thr);
+  }
+  warp_barrier();
+  if (lane == 0) sh.nhits = 0;
+  warp_barrier();
+  return thr;
+}
+
+// Forgets everything held.
+__device__ void reset_selection(SelectShared& sh) {
+  const int lane = threadIdx.x;
+  warp_barrier();
+  for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
+  if (lane == 0) {
+    sh.count = 0;
+    sh.nhits = 0;
+    sh.top_bin = kNoBin;
+  }
+  warp_barrier();
+}
+
+// Exact top-k of one chunk by one warp: on return sh.cand[0..k) holds the k
+// selected candidates (in no particular order).  n_elems >= k is the caller's
+// business.
+//
+// The chunk is streamed in index order.  A warm-up over the first vectors
+// establishes a threshold; after that a lane only tests whether a 16-byte
+// vector holds anything at or above the threshold and, if so, parks the whole
+// vector in shared memory.  Parked vectors are unpacked by the whole warp at
+// once, so the rare slow work is done with every lane busy.  Nothing here
+// waits on another warp: a chunk's serial steps only delay that chunk, while
+// the other warps of the SM keep their own loads in flight.
 template <int DT, int MODE>
-__device__ void select_topk(BlockShared& sh, const ChunkSource<DT, MODE>& src, int n_elems, int k) {
+__device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, int n_elems, int k) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   constexpr int kTileVecs = kThreads * kUnroll;
-  const int tid = threadIdx.x;
+  const int lane = threadIdx.x;
   const int n_vecs = n_elems / VEC;
-  const int trigger = max(4 * k, 256);  // compact once this many candidates are held
 
-  if (tid == 0) sh.count = 0;
-  __syncthreads();
+  reset_selection(sh);
   uint32_t thr = 0;  // accept everything until k candidates exist
 
-  // Warm-up on the first tile, then raise the threshold as far as it goes.
-  const int first = min(n_vecs, kTileVecs);
-  select_carefully<DT, MODE>(sh, src, 0, first, k, thr);
-  compact_candidates<DT>(sh, k, thr);
+  // Warm-up: enough elements that afterwards only a minority of vectors hit.
+  const int warm = min(n_vecs, (32 / VEC) * max(k, 128));
+  const int n_tiles = (n_vecs - warm) / kTileVecs;
+  const int full_end = warm + n_tiles * kTileVecs;
 
-  // Streaming tiles: kUnroll independent 16-byte loads per thread, then the
-  // filter.  The block only synchronises to agree on whether to compact.
-  int v0 = first;
-  int max_pos = -1;
+  // Streaming tiles travel through a ring of kStages tiles in shared memory,
+  // filled by asynchronous 16-byte copies: the loads of the next tiles are in
+  // flight, at no cost in registers, while this tile is filtered and while the
+  // warp drains or compacts.  Slot (stage, u, lane) is private to its lane.
+  // The first tiles are requested before the warm-up starts.
+  constexpr bool kRing = (MODE != 2);
+  auto request_tile = [&](int tile) {
+    if (kRing && tile < n_tiles) {
+      const int stage = tile % kStages;
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u)
+        copy_async_16(&sh.ring[(stage * kUnroll + u) * kThreads + lane],
+                      src.address(warm + tile * kTileVecs + u * kThreads + lane));
+    }
+    if (kRing) copy_async_commit();
+  };
+  for (int t = 0; t < kStages; ++t) request_tile(t);
+
+  thr = select_carefully<DT, MODE>(sh, src, 0, warm, k, thr);
+
+  int max_hit = -1;
   bool overflow = false;
-  for (; v0 + kTileVecs <= n_vecs; v0 += kTileVecs) {
+  for (int tile = 0; tile < n_tiles; ++tile) {
+    const int v0 = warm + tile * kTileVecs;
     uint4 w[kUnroll];
+    if (kRing) {
+      copy_async_wait<kStages - 1>();  // this lane's copies of `tile` have landed
+      const int stage = tile % kStages;
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) w[u] = src.load(v0 + u * kThreads + tid);
+      for (int u = 0; u < kUnroll; ++u) w[u] = sh.ring[(stage * kUnroll + u) * kThreads + lane];
+    } else {
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u)
-      filter_vector<DT, VEC>(sh, w[u], thr, (uint32_t)(v0 + u * kThreads + tid) * VEC, max_pos);
-    if (__syncthreads_or(max_pos + 1 >= trigger)) {
-      if (sh.count > kCandCap) {  // uniform: nobody appends until the next tile
+      for (int u = 0; u < kUnroll; ++u) w[u] = src.load(v0 + u * kThreads + lane);
+    }
+    const uint32_t add = bf16_lane_add(thr);
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (vector_has_candidate<DT, VEC>(w[u], thr, add)) {
+        const int pos = atomicAdd(&sh.nhits, 1);
+        if (pos < kHitCap) {
+          sh.hit_vec[pos] = w[u];
+          sh.hit_idx[pos] = (uint32_t)(v0 + u * kThreads + lane);
+        }
+        max_hit = max(max_hit, pos);
+      }
+    }
+    request_tile(tile + kStages);  // refill the stage just consumed
+    if (__any_sync(0xFFFFFFFFu, max_hit + 1 >= kHitTrigger)) {
+      warp_barrier();
+      if (uniform_load(&sh.nhits) > kHitCap) {
         overflow = true;
         break;
       }
-      compact_candidates<DT>(sh, k, thr);
-      max_pos = -1;
+      thr = drain_hits<DT, VEC>(sh, k, thr);
+      max_hit = -1;
     }
   }
+  if (kRing) copy_async_wait<0>();
   if (overflow) {
-    // More candidates than the buffer holds arrived within one tile (e.g.
-    // magnitudes that keep growing).  Start over, carefully.
-    __syncthreads();
-    if (tid == 0) sh.count = 0;
-    __syncthreads();
-    thr = 0;
-    select_carefully<DT, MODE>(sh, src, 0, n_vecs, k, thr);
+    // More vectors hit within one tile than can be parked (e.g. magnitudes
+    // that keep growing).  Start over, carefully.
+    reset_selection(sh);
+    thr = select_carefully<DT, MODE>(sh, src, 0, n_vecs, k, 0u);
   } else {
-    compact_candidates<DT>(sh, k, thr);
-    select_carefully<DT, MODE>(sh, src, v0, n_vecs, k, thr);
+    thr = drain_hits<DT, VEC>(sh, k, thr);
+    thr = select_carefully<DT, MODE>(sh, src, full_end, n_vecs, k, thr);
   }
-  compact_candidates<DT>(sh, k, thr);  // exactly k remain
-
-  // Rank by counting: position = number of better candidates.
-  __syncthreads();
-  for (int j = tid; j < k; j += kThreads) {
-    const unsigned long long cj = sh.cand[j];
-    int rank = 0;
-    for (int i = 0; i < k; ++i) rank += sh.cand[i] > cj;
-    const uint32_t key = (uint32_t)(cj >> (kIdxBits + 1));
-    const uint32_t sign = (uint32_t)cj & 1u;
-    sh.idx[rank] = kIdxMask - ((uint32_t)(cj >> 1) & kIdxMask);
-    sh.bits[rank] = (uint16_t)((sign << 15) | (DT == 0 ? key : (key >> 16)));
-  }
-  __syncthreads();
+  compact_candidates<DT>(sh, k, thr, true);  // exactly k remain
 }
 
 // ---------------------------------------------------------------------------
 // arithmetic in Z_p (all operands < p < 2^16, so a * b + c fits 32 bits)
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t mul_mod(uint32_t a, uint32_t b) { return (a * b) % kPrime; }
+__host__ __device__ constexpr uint32_t mul_mod(uint32_t a, uint32_t b) { return (a * b) % kPrime; }
 __device__ __forceinline__ uint32_t mad_mod(uint32_t a, uint32_t b, uint32_t c) { return (a * b + c) % kPrime; }
 __device__ __forceinline__ uint32_t sub_mod(uint32_t a, uint32_t b) { return a >= b ? a - b : a + kPrime - b; }
 
-// a^(p-2): the inverse of a != 0 (the inverse is unique, Algorithm 4 computes
-// the same value by the extended Euclidean algorithm).
-__device__ uint32_t inverse_mod(uint32_t a) {
-  uint32_t result = 1, base = a;
-  uint32_t e = kPrime - 2u;
-#pragma unroll 1
+__host__ __device__ constexpr uint32_t pow_mod(uint32_t a, uint32_t e) {
+  uint32_t r = 1;
   while (e) {
-    if (e & 1u) result = mul_mod(result, base);
-    base = mul_mod(base, base);
+    if (e & 1u) r = mul_mod(r, a);
+    a = mul_mod(a, a);
     e >>= 1;
   }
-  return result;
+  return r;
 }
+
+// Smallest generator of the multiplicative group of Z_p (p - 1 = 2^4 3^2 5 7 13).
+constexpr uint32_t find_generator() {
+  for (uint32_t g = 2; g < kPrime; ++g) {
+    bool ok = true;
+    for (uint32_t q : {2u, 3u, 5u, 7u, 13u})
+      if (pow_mod(g, (kPrime - 1) / q) == 1u) ok = false;
+    if (ok) return g;
+  }
+  return 0;
+}
+constexpr uint32_t kGenerator = find_generator();
+constexpr uint32_t kGeneratorInv = pow_mod(kGenerator, kPrime - 2);
+static_assert(kGenerator != 0 && mul_mod(kGenerator, kGeneratorInv) == 1u, "generator of Z_p^*");
 
 // Algorithm 6: largest m in [2^15 + 1, 2^16] for which the selected indices
 // stay distinct as (index mod m) mod p -- the second reduction because the
 // x-coordinates live in Z_p and m may exceed p.  Returns 0 if there is none.
-// x_out[e] receives the residue of entry tid + e * kThreads.  Uses the
-// candidate buffer as a 65536-bit set.
-__device__ uint32_t find_injective_modulus(BlockShared& sh, int k, uint32_t (&x_out)[kEntriesPerThread]) {
+// The selected candidates sit in sh.cand[0..k) on entry and are consumed: the
+// tile ring and the candidate buffer become the 65536-bit set of residues seen.
+__device__ uint32_t find_injective_modulus(SelectShared& sh, int k) {
   const int tid = threadIdx.x;
-  uint32_t* seen = reinterpret_cast<uint32_t*>(sh.cand);
+  uint32_t idx[kMaxK / kThreads], res[kMaxK / kThreads];
+#pragma unroll
+  for (int e = 0; e < kMaxK / kThreads; ++e) {
+    int j = tid + e * kThreads;
+    idx[e] = j < k ? kIdxMask - ((uint32_t)(sh.cand[j] >> 1) & kIdxMask) : 0u;
+    res[e] = 0;
+  }
+  __syncthreads();
+  uint32_t* seen = reinterpret_cast<uint32_t*>(sh.ring);  // ring and cand are adjacent: 11 KB
   for (int i = tid; i < 2048; i += kThreads) seen[i] = 0;
   __syncthreads();
   uint32_t found = 0;
@@ -384,21 +603,21 @@ __device__ uint32_t find_injective_modulus(BlockShared& sh, int k, uint32_t (&x_
   for (uint32_t m = kModHigh; m >= kModLow; --m) {
     uint32_t dup = 0;
 #pragma unroll
-    for (int e = 0; e < kEntriesPerThread; ++e) {
+    for (int e = 0; e < kMaxK / kThreads; ++e) {
       int j = tid + e * kThreads;
       if (j < k) {
-        uint32_t r = sh.idx[j] % m;
+        uint32_t r = idx[e] % m;
         if (r >= kPrime) r -= kPrime;
-        x_out[e] = r;
+        res[e] = r;
         uint32_t bit = 1u << (r & 31u);
         dup |= atomicOr(&seen[r >> 5], bit) & bit;
       }
     }
     const int clash = __syncthreads_or(dup != 0);
 #pragma unroll
-    for (int e = 0; e < kEntriesPerThread; ++e) {
+    for (int e = 0; e < kMaxK / kThreads; ++e) {
       int j = tid + e * kThreads;
-      if (j < k) seen[x_out[e] >> 5] = 0;
+      if (j < k) seen[res[e] >> 5] = 0;
     }
     __syncthreads();
     if (!clash) {
@@ -407,94 +626,6 @@ __device__ uint32_t find_injective_modulus(BlockShared& sh, int k, uint32_t (&x_
     }
   }
   return found;
-}
-
-// Algorithm 3 (Newton interpolation over Z_p) with the divisions postponed:
-// every divided difference is carried as a fraction num / den, one level per
-// block-wide step, and each Newton coefficient takes a single inverse at the
-// end.  The Newton form is then multiplied out from the innermost bracket:
-//   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0.
-// Entry j of every array belongs to thread j % kThreads.  On return coef[]
-// (shared, k entries, ascending degree) holds the polynomial.
-__device__ uint32_t* interpolate(BlockShared& sh, int k, const uint32_t (&x_in)[kEntriesPerThread]) {
-  const int tid = threadIdx.x;
-  uint32_t* X = reinterpret_cast<uint32_t*>(sh.cand);
-  uint32_t* A = X + kMaxK;
-  uint32_t* num[2] = {A + kMaxK, A + 2 * kMaxK};
-  uint32_t* den[2] = {A + 3 * kMaxK, A + 4 * kMaxK};
-  uint32_t fin_num[kEntriesPerThread], fin_den[kEntriesPerThread];
-#pragma unroll
-  for (int e = 0; e < kEntriesPerThread; ++e) {
-    int j = tid + e * kThreads;
-    fin_num[e] = 0;
-    fin_den[e] = 1;
-    if (j < k) {
-      uint32_t y = sh.bits[j];
-      if (y >= kPrime) y -= kPrime;  // "dd <- y mod M"
-      X[j] = x_in[e];
-      num[0][j] = y;
-      den[0][j] = 1;
-      fin_num[e] = y;  // entry 0 is already final; the others are overwritten at level j
-    }
-  }
-  __syncthreads();
-  int cur = 0;
-#pragma unroll 1
-  for (int level = 1; level < k; ++level) {
-    const uint32_t* nc = num[cur];
-    const uint32_t* dc = den[cur];
-    uint32_t* nn = num[cur ^ 1];
-    uint32_t* dn = den[cur ^ 1];
-#pragma unroll
-    for (int e = 0; e < kEntriesPerThread; ++e) {
-      int j = tid + e * kThreads;
-      if (j < k && j >= level) {
-        // (n_j/d_j - n_{j-1}/d_{j-1}) / (x_j - x_{j-level})
-        uint32_t nj = nc[j], np = nc[j - 1], dj = dc[j], dp = dc[j - 1];
-        uint32_t span = sub_mod(X[j], X[j - level]);
-        uint32_t n_new = mad_mod(kPrime - np, dj, mul_mod(nj, dp));
-        uint32_t d_new = mul_mod(mul_mod(dj, dp), span);
-        nn[j] = n_new;
-        dn[j] = d_new;
-        if (j == level) {
-          fin_num[e] = n_new;
-          fin_den[e] = d_new;
-        }
-      }
-    }
-    __syncthreads();
-    cur ^= 1;
-  }
-#pragma unroll
-  for (int e = 0; e < kEntriesPerThread; ++e) {
-    int j = tid + e * kThreads;
-    if (j < k) A[j] = mul_mod(fin_num[e], inverse_mod(fin_den[e]));
-  }
-  uint32_t* poly[2] = {num[0], num[1]};
-  __syncthreads();  // A complete; num[] free for reuse (every level's reads are done)
-  for (int d = tid; d < k; d += kThreads) poly[0][d] = (d == 0) ? A[k - 1] : 0u;
-  __syncthreads();
-  cur = 0;
-#pragma unroll 1
-  for (int i = k - 2; i >= 0; --i) {
-    const uint32_t neg_x = (kPrime - X[i]) % kPrime;
-    const uint32_t a_i = A[i];
-    const int top = k - 1 - i;  // degree after this step
-    const uint32_t* pc = poly[cur];
-    uint32_t* pn = poly[cur ^ 1];
-#pragma unroll
-    for (int e = 0; e < kEntriesPerThread; ++e) {
-      int d = tid + e * kThreads;
-      if (d <= top) {
-        const uint32_t carry = d > 0 ? pc[d - 1] : a_i;
-        const uint32_t here = d < top ? pc[d] : 0u;  // the old polynomial has degree top - 1
-        pn[d] = mad_mod(here, neg_x, carry);
-      }
-    }
-    __syncthreads();
-    cur ^= 1;
-  }
-  return poly[cur];
 }
 
 struct ChunkPlace {
@@ -523,25 +654,26 @@ __device__ __forceinline__ ChunkPlace locate_chunk(const BatchParams& bp, long l
 }
 
 // ---------------------------------------------------------------------------
-// Algorithm 1 for one chunk per block.
+// select kernel: topk() of Algorithms 1 and 2, one chunk per block; for proof
+// generation (sel.proofs != nullptr) also findInjectiveModulus() of Algorithm 1.
 // ---------------------------------------------------------------------------
 template <int DT, int MODE>
-__global__ void __launch_bounds__(kThreads) toploc_build_kernel(BatchParams bp, BuildOut out) {
-  __shared__ BlockShared sh;
+__global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_select_kernel(BatchParams bp, Selection sel) {
+  __shared__ SelectShared sh;
   const int tid = threadIdx.x;
   const long long chunk = blockIdx.x;
   const int k = bp.k;
-  const size_t proof_bytes = 2 + 2 * (size_t)k;
-  uint16_t* proof = reinterpret_cast<uint16_t*>(out.proofs + chunk * proof_bytes);
-  int32_t* indices = out.indices ? out.indices + chunk * k : nullptr;
+  uint16_t* proof = sel.proofs ? reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 2 * (size_t)k)) : nullptr;
+  int32_t* indices = sel.indices ? sel.indices + chunk * k : nullptr;
 
   const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
   const long long n_elems = (long long)pl.rows * bp.hidden;
   if (n_elems < k) {
-    for (int i = tid; i < k + 1; i += kThreads) proof[i] = 0;
+    if (proof)
+      for (int i = tid; i < k + 1; i += kThreads) proof[i] = 0;
     if (indices)
       for (int i = tid; i < k; i += kThreads) indices[i] = 0;
-    if (tid == 0) out.status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+    if (tid == 0) sel.status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
     return;
   }
   ChunkSource<DT, MODE> src;
@@ -551,39 +683,197 @@ __global__ void __launch_bounds__(kThreads) toploc_build_kernel(BatchParams bp, 
   src.vecs_per_row = bp.hidden / ChunkSource<DT, MODE>::kVec;
   select_topk<DT, MODE>(sh, src, (int)n_elems, k);
 
-  if (indices)
-    for (int j = tid; j < k; j += kThreads) indices[j] = (int32_t)sh.idx[j];
+  // hand the selection to the tail kernel; rank order only where the caller asked for indices
   uint32_t unrepresentable = 0;
-  for (int j = tid; j < k; j += kThreads) unrepresentable |= sh.bits[j] >= kPrime;
-  const int nonfinite = __syncthreads_or(unrepresentable != 0);
-
-  uint32_t x[kEntriesPerThread];
-  const uint32_t m = find_injective_modulus(sh, k, x);
-  if (m == 0) {
-    for (int i = tid; i < k + 1; i += kThreads) proof[i] = 0;
-    if (tid == 0) out.status[chunk] = TOPLOC_CHUNK_NO_INJECTIVE_MODULUS;
+  for (int j = tid; j < k; j += kThreads) {
+    const unsigned long long cj = sh.cand[j];
+    const uint32_t key = (uint32_t)(cj >> (kIdxBits + 1));
+    const uint32_t sign = (uint32_t)cj & 1u;
+    const uint32_t flat = kIdxMask - ((uint32_t)(cj >> 1) & kIdxMask);
+    const uint32_t bits = (sign << 15) | (DT == 0 ? key : (key >> 16));
+    unrepresentable |= bits >= kPrime;
+    sel.idx[chunk * k + j] = flat;
+    sel.bits[chunk * k + j] = (uint16_t)bits;
+    if (indices) {
+      int rank = 0;  // position = number of better candidates
+      for (int i = 0; i < k; ++i) rank += sh.cand[i] > cj;
+      indices[rank] = (int32_t)flat;
+    }
+  }
+  if (proof == nullptr) {
+    if (tid == 0) sel.status[chunk] = TOPLOC_CHUNK_OK;
     return;
   }
-  const uint32_t* coef = interpolate(sh, k, x);
-  // proof: m & 0xFFFF (65536 -> 0), then k coefficients, little-endian 16-bit words
-  if (tid == 0) {
-    proof[0] = (uint16_t)(m & 0xFFFFu);
-    out.status[chunk] = nonfinite ? TOPLOC_CHUNK_NONFINITE_COMMITTED : TOPLOC_CHUNK_OK;
+  const int nonfinite = __syncthreads_or(unrepresentable != 0);
+  const uint32_t m = find_injective_modulus(sh, k);
+  if (m == 0) {
+    for (int i = tid; i < k + 1; i += kThreads) proof[i] = 0;
+    if (tid == 0) sel.status[chunk] = TOPLOC_CHUNK_NO_INJECTIVE_MODULUS;
+    return;
   }
-  for (int d = tid; d < k; d += kThreads) proof[1 + d] = (uint16_t)coef[d];
+  if (tid == 0) {
+    proof[0] = (uint16_t)(m & 0xFFFFu);  // 65536 is stored as 0
+    sel.status[chunk] = nonfinite ? TOPLOC_CHUNK_NONFINITE_COMMITTED : TOPLOC_CHUNK_OK;
+  }
 }
 
 // ---------------------------------------------------------------------------
-// Algorithm 2 for one chunk per block.
+// tail kernels: one warp per chunk.  Entry j of a chunk's k points belongs to
+// lane j % 32, slot j / 32 of that lane.
 // ---------------------------------------------------------------------------
-template <int DT, int MODE>
-__global__ void __launch_bounds__(kThreads) toploc_verify_kernel(BatchParams bp, VerifyIo io) {
-  __shared__ BlockShared sh;
+
+// value of entry j - 1 as seen from entry j (lane 0 takes lane 31 of the slot below)
+template <int S>
+__device__ __forceinline__ uint32_t left_neighbour(const uint32_t (&v)[S], int s, int lane, uint32_t first) {
+  uint32_t prev = __shfl_up_sync(0xFFFFFFFFu, v[s], 1);
+  if (s > 0) {
+    const uint32_t carry = __shfl_sync(0xFFFFFFFFu, v[s > 0 ? s - 1 : 0], 31);
+    if (lane == 0) prev = carry;
+  } else if (lane == 0) {
+    prev = first;
+  }
+  return prev;
+}
+
+// Algorithm 3 for the chunks of one warp.  inv[] is the table of inverses in
+// Z_p; xw / aw are this warp's scratch rows (k entries each).
+template <int SLOTS>
+__device__ __forceinline__ void interpolate_chunk(const uint16_t* inv, uint16_t* xw, uint16_t* aw, int k,
+                                                  const uint32_t* idx, const uint16_t* bits, uint32_t m,
+                                                  uint16_t* proof) {
+  const int lane = threadIdx.x & 31;
+  uint32_t x[SLOTS], dd[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int j = s * 32 + lane;
+    x[s] = 0;
+    dd[s] = 0;
+    if (j < k) {
+      uint32_t r = idx[j] % m;       // i_m = i mod m, then into Z_p
+      if (r >= kPrime) r -= kPrime;
+      uint32_t y = bits[j];          // "dd <- y mod M"
+      if (y >= kPrime) y -= kPrime;
+      x[s] = r;
+      dd[s] = y;
+      xw[j] = (uint16_t)r;
+    }
+  }
+  __syncwarp();
+  // divided differences: after level l entry j >= l holds f[x_{j-l}, ..., x_j]
+#pragma unroll 1
+  for (int level = 1; level < k; ++level) {
+    const int s_lo = level >> 5;
+#pragma unroll
+    for (int s = SLOTS - 1; s >= 0; --s) {
+      if (s >= s_lo) {
+        const int j = s * 32 + lane;
+        const uint32_t prev = left_neighbour<SLOTS>(dd, s, lane, 0u);
+        const bool active = j >= level && j < k;
+        const uint32_t span = active ? sub_mod(x[s], xw[j - level]) : 0u;
+        const uint32_t next = mul_mod(sub_mod(dd[s], prev), inv[span]);
+        dd[s] = active ? next : dd[s];
+      }
+    }
+  }
+  // dd[j] is the Newton coefficient a_j; multiply the Newton form out from the inside:
+  //   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int j = s * 32 + lane;
+    if (j < k) aw[j] = (uint16_t)dd[s];
+  }
+  __syncwarp();
+  uint32_t c[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) c[s] = 0;
+  if (lane == 0) c[0] = aw[k - 1];
+#pragma unroll 1
+  for (int i = k - 2; i >= 0; --i) {
+    const uint32_t xi = xw[i];
+    const uint32_t neg_x = xi ? kPrime - xi : 0u;
+    const uint32_t a_i = aw[i];
+    const int top = k - 1 - i;  // degree after this step
+    const int s_hi = top >> 5;
+#pragma unroll
+    for (int s = SLOTS - 1; s >= 0; --s) {
+      if (s <= s_hi) {
+        const int d = s * 32 + lane;
+        const uint32_t prev = left_neighbour<SLOTS>(c, s, lane, a_i);
+        const uint32_t next = mad_mod(c[s], neg_x, prev);
+        c[s] = d <= top ? next : 0u;
+      }
+    }
+  }
+  // proof bytes 2 + 2d, 3 + 2d: coefficient of degree d, little-endian
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int d = s * 32 + lane;
+    if (d < k) proof[1 + d] = (uint16_t)c[s];
+  }
+  __syncwarp();
+}
+
+// InterpolateModPolynomial() and encode() of Algorithm 1 for every chunk the
+// select kernel finished.  Each block first fills a table of all inverses in
+// Z_p (walking the powers of a generator forwards and backwards), then every
+// warp takes chunks in turn.
+__global__ void __launch_bounds__(kInterpWarps * 32, 1)
+toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
+  extern __shared__ __align__(16) uint16_t dyn_smem[];
+  uint16_t* inv = dyn_smem;                               // 65536 entries
+  uint16_t* scratch = dyn_smem + 65536;                   // 2 rows of kMaxK per warp
   const int tid = threadIdx.x;
-  const long long chunk = blockIdx.x;
-  const int k = bp.k;
+  const int warp = tid >> 5;
+  {
+    // thread t owns exponents 64t .. 64t + 63 of the generator
+    const uint32_t e0 = (uint32_t)tid * 64u;
+    uint32_t a = pow_mod(kGenerator, e0);
+    uint32_t b = pow_mod(kGeneratorInv, e0);
+    if (tid == 0) inv[0] = 0;
+#pragma unroll 4
+    for (int i = 0; i < 64; ++i) {
+      if (e0 + i < kPrime - 1) inv[a] = (uint16_t)b;
+      a = mul_mod(a, kGenerator);
+      b = mul_mod(b, kGeneratorInv);
+    }
+  }
+  __syncthreads();
+  uint16_t* xw = scratch + warp * 2 * kMaxK;
+  uint16_t* aw = xw + kMaxK;
   const size_t proof_bytes = 2 + 2 * (size_t)k;
-  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * proof_bytes);
+  for (long long chunk = (long long)blockIdx.x * kInterpWarps + warp; chunk < num_chunks;
+       chunk += (long long)gridDim.x * kInterpWarps) {
+    const uint8_t st = sel.status[chunk];
+    if (st == TOPLOC_CHUNK_NO_INJECTIVE_MODULUS || st == TOPLOC_CHUNK_K_EXCEEDS_CHUNK) continue;
+    uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_bytes);
+    uint32_t m = proof[0];
+    if (m == 0) m = 65536u;
+    const uint32_t* idx = sel.idx + chunk * k;
+    const uint16_t* bits = sel.bits + chunk * k;
+    if (k <= 32) interpolate_chunk<1>(inv, xw, aw, k, idx, bits, m, proof);
+    else if (k <= 64) interpolate_chunk<2>(inv, xw, aw, k, idx, bits, m, proof);
+    else if (k <= 128) interpolate_chunk<4>(inv, xw, aw, k, idx, bits, m, proof);
+    else interpolate_chunk<kMaxSlots>(inv, xw, aw, k, idx, bits, m, proof);
+  }
+}
+
+struct VerifyWarpShared {
+  uint16_t coef[kMaxK];
+  uint32_t gen[kMaxK];
+  uint32_t hist[128];  // a 7-bit mantissa difference is at most 127
+};
+
+// decode(), Horner evaluation (Algorithm 5), extractBits(), the error
+// accumulation and the verdict of Algorithm 2, one warp per chunk.
+__global__ void __launch_bounds__(kVerifyWarps * 32)
+toploc_evaluate_kernel(Selection sel, VerifyIo io, int k, long long num_chunks) {
+  __shared__ VerifyWarpShared wsh[kVerifyWarps];
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const long long chunk = (long long)blockIdx.x * kVerifyWarps + warp;
+  if (chunk >= num_chunks) return;
+  VerifyWarpShared& ws = wsh[warp];
+  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 2 * (size_t)k));
 
   toploc_chunk_result res;
   res.exp_mismatch = 0;
@@ -596,52 +886,39 @@ __global__ void __launch_bounds__(kThreads) toploc_verify_kernel(BatchParams bp,
   res.status = TOPLOC_CHUNK_OK;
   res.pad[0] = res.pad[1] = 0;
 
-  // decode
   uint32_t m = proof[0];
   if (m == 0) m = 65536u;
   res.modulus = m;
   uint32_t bad = (m < kModLow || m > kModHigh);
-  for (int d = tid; d < k; d += kThreads) bad |= proof[1 + d] >= kPrime;
-  if (__syncthreads_or(bad != 0)) {
+  for (int d = lane; d < k; d += 32) {
+    const uint16_t cd = proof[1 + d];
+    ws.coef[d] = cd;
+    bad |= cd >= kPrime;
+  }
+  if (__any_sync(0xFFFFFFFFu, bad != 0)) {
     res.status = TOPLOC_CHUNK_BAD_PROOF;
-    if (tid == 0) io.results[chunk] = res;
+    if (lane == 0) io.results[chunk] = res;
     return;
   }
-  const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
-  const long long n_elems = (long long)pl.rows * bp.hidden;
-  if (n_elems < k) {
-    res.status = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
-    if (tid == 0) io.results[chunk] = res;
+  if (sel.status[chunk] != TOPLOC_CHUNK_OK) {
+    res.status = sel.status[chunk];
+    if (lane == 0) io.results[chunk] = res;
     return;
   }
-  ChunkSource<DT, MODE> src;
-  src.base = pl.base;
-  src.row_stride = bp.row_stride;
-  src.hidden = bp.hidden;
-  src.vecs_per_row = bp.hidden / ChunkSource<DT, MODE>::kVec;
-  select_topk<DT, MODE>(sh, src, (int)n_elems, k);
-
-  // the candidate buffer is free now: coefficients, then the generator's indices
-  uint32_t* coef = reinterpret_cast<uint32_t*>(sh.cand);
-  uint32_t* gen = coef + kMaxK;
-  for (int d = tid; d < k; d += kThreads) coef[d] = proof[1 + d];
   if (io.gen_indices)
-    for (int j = tid; j < k; j += kThreads) gen[j] = (uint32_t)io.gen_indices[chunk * k + j];
-  sh.hist[tid] = 0;  // 128 bins: a 7-bit mantissa difference is at most 127
-  if (tid == 0) {
-    sh.err_e = 0;
-    sh.diff_sum = 0;
-    sh.common = 0;
-  }
-  __syncthreads();
-  for (int j = tid; j < k; j += kThreads) {
-    uint32_t x = sh.idx[j] % m;
+    for (int j = lane; j < k; j += 32) ws.gen[j] = (uint32_t)io.gen_indices[chunk * k + j];
+  for (int b = lane; b < 128; b += 32) ws.hist[b] = 0;
+  __syncwarp();
+
+  uint32_t err_e = 0, diff_sum = 0, common = 0;
+  for (int j = lane; j < k; j += 32) {
+    const uint32_t flat = sel.idx[chunk * k + j];
+    const uint32_t seen = sel.bits[chunk * k + j];
+    uint32_t x = flat % m;
     if (x >= kPrime) x -= kPrime;
-    // Algorithm 5 (Horner), highest degree first
-    uint32_t acc = coef[k - 1];
+    uint32_t acc = ws.coef[k - 1];  // Horner, highest degree first
 #pragma unroll 4
-    for (int d = k - 2; d >= 0; --d) acc = mad_mod(acc, x, coef[d]);
-    const uint32_t seen = sh.bits[j];
+    for (int d = k - 2; d >= 0; --d) acc = mad_mod(acc, x, ws.coef[d]);
     uint32_t e_p = acc >> 7, e_v = seen >> 7;  // sign + 8 exponent bits
     if (!io.sign_in_exponent) {
       e_p &= 0xFFu;
@@ -650,37 +927,63 @@ __global__ void __launch_bounds__(kThreads) toploc_verify_kernel(BatchParams bp,
     if (e_p == e_v) {
       int diff = (int)(acc & 0x7Fu) - (int)(seen & 0x7Fu);
       diff = diff < 0 ? -diff : diff;
-      atomicAdd(&sh.hist[diff], 1u);
-      atomicAdd(&sh.diff_sum, (uint32_t)diff);
+      atomicAdd(&ws.hist[diff], 1u);
+      diff_sum += (uint32_t)diff;
     } else {
-      atomicAdd(&sh.err_e, 1u);
+      ++err_e;
     }
     if (io.gen_indices) {
-      const uint32_t mine = sh.idx[j];
       uint32_t hit = 0;
-      for (int i = 0; i < k; ++i) hit |= gen[i] == mine;
-      if (hit) atomicAdd(&sh.common, 1u);
+      for (int i = 0; i < k; ++i) hit |= ws.gen[i] == flat;
+      common += hit;
     }
   }
-  __syncthreads();
-  if (tid == 0) {
-    const uint32_t n = (uint32_t)k - sh.err_e;
-    res.exp_mismatch = sh.err_e;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    err_e += __shfl_xor_sync(0xFFFFFFFFu, err_e, off);
+    diff_sum += __shfl_xor_sync(0xFFFFFFFFu, diff_sum, off);
+    common += __shfl_xor_sync(0xFFFFFFFFu, common, off);
+  }
+  __syncwarp();
+  // median from the histogram: sorted positions (n - 1) / 2 and n / 2; lane l owns bins 4l .. 4l + 3
+  const uint32_t n = (uint32_t)k - err_e;
+  uint32_t local[4], sum = 0;
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    local[b] = ws.hist[lane * 4 + b];
+    sum += local[b];
+  }
+  uint32_t incl = sum;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t other = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    if (lane >= off) incl += other;
+  }
+  int lo_val = -1, hi_val = -1;
+  if (n > 0) {
+    const uint32_t lo_pos = (n - 1) / 2, hi_pos = n / 2;
+    uint32_t below = incl - sum;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const uint32_t upto = below + local[b];
+      if (below <= lo_pos && lo_pos < upto) lo_val = lane * 4 + b;
+      if (below <= hi_pos && hi_pos < upto) hi_val = lane * 4 + b;
+      below = upto;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    lo_val = max(lo_val, __shfl_xor_sync(0xFFFFFFFFu, lo_val, off));
+    hi_val = max(hi_val, __shfl_xor_sync(0xFFFFFFFFu, hi_val, off));
+  }
+  if (lane == 0) {
+    res.exp_mismatch = err_e;
     res.n_match = n;
-    res.mant_diff_sum = sh.diff_sum;
-    if (io.gen_indices) res.topk_mismatch = k - (int)sh.common;
+    res.mant_diff_sum = diff_sum;
+    if (io.gen_indices) res.topk_mismatch = k - (int)common;
     bool reject = true;  // nothing matched: nothing to accept on
     if (n > 0) {
-      res.mant_mean = (double)sh.diff_sum / (double)n;
-      // median from the histogram: sorted positions (n-1)/2 and n/2
-      const uint32_t lo_pos = (n - 1) / 2, hi_pos = n / 2;
-      uint32_t seen_cnt = 0;
-      int lo_val = -1, hi_val = -1;
-      for (int v = 0; v < 128 && hi_val < 0; ++v) {
-        seen_cnt += sh.hist[v];
-        if (lo_val < 0 && seen_cnt > lo_pos) lo_val = v;
-        if (seen_cnt > hi_pos) hi_val = v;
-      }
+      res.mant_mean = (double)diff_sum / (double)n;
       res.mant_median = ((double)lo_val + (double)hi_val) * 0.5;
       reject = (res.exp_mismatch > (uint32_t)io.t_exp) || (res.mant_mean > io.t_mean) ||
                (res.mant_median > io.t_median);
@@ -734,20 +1037,36 @@ int plan_layout(const toploc_layout* lay, HostPlan* plan) {
   return TOPLOC_OK;
 }
 
-int check_device() {
+struct DeviceInfo {
+  bool known;
+  int major;
+  int sms;
+  bool interp_smem_set;
+};
+
+size_t interp_smem_bytes() { return (65536 + (size_t)kInterpWarps * 2 * kMaxK) * sizeof(uint16_t); }
+
+int device_info(DeviceInfo** out) {
+  static DeviceInfo table[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return TOPLOC_ERR_CUDA;
-  static int major_of[64];
-  static bool known[64];
   if (dev < 0 || dev >= 64) return TOPLOC_ERR_UNSUPPORTED;
-  if (!known[dev]) {
-    int major = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+  DeviceInfo& d = table[dev];
+  if (!d.known) {
+    if (cudaDeviceGetAttribute(&d.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return TOPLOC_ERR_CUDA;
-    major_of[dev] = major;
-    known[dev] = true;
+    d.known = true;
   }
-  return major_of[dev] == 10 ? TOPLOC_OK : TOPLOC_ERR_ARCH;
+  if (d.major != 10) return TOPLOC_ERR_ARCH;
+  if (!d.interp_smem_set) {
+    if (cudaFuncSetAttribute(toploc_interpolate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)interp_smem_bytes()) != cudaSuccess)
+      return TOPLOC_ERR_CUDA;
+    d.interp_smem_set = true;
+  }
+  *out = &d;
+  return TOPLOC_OK;
 }
 
 // 0: flat vectors, 1: aligned rows with padding, 2: element-wise
@@ -760,14 +1079,31 @@ int pick_mode(const void* act, const toploc_layout* lay) {
   return lay->row_stride == lay->hidden ? 0 : 1;
 }
 
-// Fills the device row table of a ragged batch (in the caller's workspace).
-int upload_spans(const toploc_layout* lay, const HostPlan& plan, void* d_workspace, size_t workspace_bytes,
-                 cudaStream_t stream, const ChunkSpan** d_spans) {
-  *d_spans = nullptr;
-  if (!plan.ragged || plan.num_chunks == 0) return TOPLOC_OK;
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Scratch of one call: ragged row table, then the selection.
+struct WorkspacePlan {
+  size_t spans_off, idx_off, bits_off, status_off, total;
+};
+
+WorkspacePlan plan_workspace(bool ragged, long long chunks, int k) {
+  WorkspacePlan w;
+  size_t off = 0;
+  w.spans_off = off;
+  off += ragged ? round_up((size_t)chunks * sizeof(ChunkSpan), 256) : 0;
+  w.idx_off = off;
+  off += round_up((size_t)chunks * k * sizeof(uint32_t), 256);
+  w.bits_off = off;
+  off += round_up((size_t)chunks * k * sizeof(uint16_t), 256);
+  w.status_off = off;
+  off += round_up((size_t)chunks, 256);
+  w.total = off;
+  return w;
+}
+
+// Fills the device row table of a ragged batch.
+int upload_spans(const toploc_layout* lay, const HostPlan& plan, void* d_spans, cudaStream_t stream) {
   const size_t need = (size_t)plan.num_chunks * sizeof(ChunkSpan);
-  if (d_workspace == nullptr || workspace_bytes < need) return TOPLOC_ERR_WORKSPACE;
-  if (reinterpret_cast<uintptr_t>(d_workspace) % 8 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
   ChunkSpan* spans = static_cast<ChunkSpan*>(malloc(need));
   if (spans == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
   long long c = 0;
@@ -781,60 +1117,70 @@ int upload_spans(const toploc_layout* lay, const HostPlan& plan, void* d_workspa
     }
   }
   // pageable source: the runtime has staged the bytes by the time this returns
-  cudaError_t err = cudaMemcpyAsync(d_workspace, spans, need, cudaMemcpyHostToDevice, stream);
+  cudaError_t err = cudaMemcpyAsync(d_spans, spans, need, cudaMemcpyHostToDevice, stream);
   free(spans);
-  if (err != cudaSuccess) return TOPLOC_ERR_CUDA;
-  *d_spans = static_cast<const ChunkSpan*>(d_workspace);
-  return TOPLOC_OK;
+  return err == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
-BatchParams make_params(const void* d_act, const toploc_layout* lay, const HostPlan& plan,
-                        const ChunkSpan* d_spans) {
+template <int DT>
+void launch_select(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const Selection& sel) {
+  if (mode == 0) toploc_select_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, sel);
+  else if (mode == 1) toploc_select_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, sel);
+  else toploc_select_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, sel);
+}
+
+// Common front half of both entry points: checks, scratch carving, row table, select kernel.
+int run_select(const void* d_act, const toploc_layout* lay, void* d_workspace, size_t workspace_bytes,
+               cudaStream_t stream, uint8_t* d_status_or_null, uint8_t* d_proofs_or_null,
+               int32_t* d_indices_opt, HostPlan* plan, Selection* sel, DeviceInfo** dev) {
+  int rc = device_info(dev);
+  if (rc != TOPLOC_OK) return rc;
+  const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k);
+  if (d_workspace == nullptr || workspace_bytes < wp.total) return TOPLOC_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(d_workspace) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  char* ws = static_cast<char*>(d_workspace);
   BatchParams bp;
   bp.act = d_act;
   bp.row_stride = lay->row_stride;
   bp.tokens_per_seq = lay->tokens_per_seq;
-  bp.spans = d_spans;
+  bp.spans = nullptr;
   bp.hidden = lay->hidden;
   bp.chunk_len = lay->chunk_len;
   bp.k = lay->k;
-  bp.chunks_per_seq = plan.chunks_per_seq;
-  return bp;
+  bp.chunks_per_seq = plan->chunks_per_seq;
+  if (plan->ragged) {
+    if ((rc = upload_spans(lay, *plan, ws + wp.spans_off, stream)) != TOPLOC_OK) return rc;
+    bp.spans = reinterpret_cast<const ChunkSpan*>(ws + wp.spans_off);
+  }
+  sel->idx = reinterpret_cast<uint32_t*>(ws + wp.idx_off);
+  sel->bits = reinterpret_cast<uint16_t*>(ws + wp.bits_off);
+  sel->status = d_status_or_null ? d_status_or_null : reinterpret_cast<uint8_t*>(ws + wp.status_off);
+  sel->proofs = d_proofs_or_null;
+  sel->indices = d_indices_opt;
+  const int mode = pick_mode(d_act, lay);
+  if (lay->dtype == TOPLOC_DTYPE_BF16) launch_select<0>(mode, (unsigned)plan->num_chunks, stream, bp, *sel);
+  else launch_select<1>(mode, (unsigned)plan->num_chunks, stream, bp, *sel);
+  return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
-
-template <int DT>
-void launch_build(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const BuildOut& out) {
-  if (mode == 0) toploc_build_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, out);
-  else if (mode == 1) toploc_build_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, out);
-  else toploc_build_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, out);
-}
-
-template <int DT>
-void launch_verify(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const VerifyIo& io) {
-  if (mode == 0) toploc_verify_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, io);
-  else if (mode == 1) toploc_verify_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, io);
-  else toploc_verify_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, io);
-}
-
-size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Carves the staging buffer of the *_host entry points for a group of
-// sequences: activations, per-chunk outputs, proofs, ragged row table.
+// sequences: activations, per-chunk outputs, proofs, scratch.
 struct StagingPlan {
-  size_t act_off, small_off, proofs_off, spans_off, total;
+  size_t act_off, small_off, proofs_off, work_off, work_bytes, total;
 };
 
-StagingPlan carve_staging(const toploc_layout* lay, long long rows, long long chunks, size_t small_elem) {
+StagingPlan carve_staging(const toploc_layout* lay, long long rows, long long chunks) {
   const size_t esz = lay->dtype == TOPLOC_DTYPE_BF16 ? 2 : 4;
   StagingPlan sp;
   sp.act_off = 0;
   size_t off = round_up((size_t)rows * (size_t)lay->row_stride * esz, 256);
   sp.small_off = off;
-  off += round_up((size_t)chunks * small_elem, 256);
+  off += round_up((size_t)chunks * sizeof(toploc_chunk_result), 256);
   sp.proofs_off = off;
   off += round_up((size_t)chunks * (2 + 2 * (size_t)lay->k), 256);
-  sp.spans_off = off;
-  off += round_up((size_t)chunks * sizeof(ChunkSpan), 256);
+  sp.work_off = off;
+  sp.work_bytes = plan_workspace(true, chunks, lay->k).total;
+  off += sp.work_bytes;
   sp.total = off;
   return sp;
 }
@@ -869,15 +1215,15 @@ size_t toploc_proof_bytes(int32_t k) { return k > 0 ? 2 + 2 * (size_t)k : 0; }
 
 size_t toploc_workspace_bytes(const toploc_layout* lay) {
   HostPlan plan;
-  if (plan_layout(lay, &plan) != TOPLOC_OK || !plan.ragged) return 0;
-  return (size_t)plan.num_chunks * sizeof(ChunkSpan);
+  if (plan_layout(lay, &plan) != TOPLOC_OK) return 0;
+  return plan_workspace(plan.ragged, plan.num_chunks, lay->k).total;
 }
 
 size_t toploc_staging_bytes(const toploc_layout* lay) {
   HostPlan plan;
   if (plan_layout(lay, &plan) != TOPLOC_OK) return 0;
   long long chunks = (plan.max_seq_rows + lay->chunk_len - 1) / lay->chunk_len;
-  return carve_staging(lay, plan.max_seq_rows, chunks, sizeof(toploc_chunk_result)).total;
+  return carve_staging(lay, plan.max_seq_rows, chunks).total;
 }
 
 void toploc_get_constants(uint32_t* p, uint32_t* m_lo, uint32_t* m_hi) {
@@ -917,19 +1263,18 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
   if (rc != TOPLOC_OK) return rc;
   if (d_act == nullptr || d_proofs == nullptr || d_status == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(d_proofs) % 2 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if ((rc = check_device()) != TOPLOC_OK) return rc;
   if (plan.num_chunks == 0) return TOPLOC_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const ChunkSpan* d_spans = nullptr;
-  if ((rc = upload_spans(lay, plan, d_workspace, workspace_bytes, stream, &d_spans)) != TOPLOC_OK) return rc;
-  const BatchParams bp = make_params(d_act, lay, plan, d_spans);
-  BuildOut out;
-  out.proofs = d_proofs;
-  out.status = d_status;
-  out.indices = d_indices_opt;
-  const int mode = pick_mode(d_act, lay);
-  if (lay->dtype == TOPLOC_DTYPE_BF16) launch_build<0>(mode, (unsigned)plan.num_chunks, stream, bp, out);
-  else launch_build<1>(mode, (unsigned)plan.num_chunks, stream, bp, out);
+  Selection sel;
+  DeviceInfo* dev = nullptr;
+  rc = run_select(d_act, lay, d_workspace, workspace_bytes, stream, d_status, d_proofs, d_indices_opt, &plan,
+                  &sel, &dev);
+  if (rc != TOPLOC_OK) return rc;
+  const long long per_wave = kInterpWarps;
+  long long blocks = (plan.num_chunks + per_wave - 1) / per_wave;
+  if (blocks > dev->sms) blocks = dev->sms;
+  toploc_interpolate_kernel<<<(unsigned)blocks, kInterpWarps * 32, interp_smem_bytes(), stream>>>(
+      sel, lay->k, plan.num_chunks);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
@@ -945,12 +1290,13 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   if (reinterpret_cast<uintptr_t>(d_proofs) % 2 != 0 || reinterpret_cast<uintptr_t>(d_results) % 8 != 0)
     return TOPLOC_ERR_INVALID_ARGUMENT;
   if (thr->t_exp < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if ((rc = check_device()) != TOPLOC_OK) return rc;
   if (plan.num_chunks == 0) return TOPLOC_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const ChunkSpan* d_spans = nullptr;
-  if ((rc = upload_spans(lay, plan, d_workspace, workspace_bytes, stream, &d_spans)) != TOPLOC_OK) return rc;
-  const BatchParams bp = make_params(d_act, lay, plan, d_spans);
+  Selection sel;
+  DeviceInfo* dev = nullptr;
+  rc = run_select(d_act, lay, d_workspace, workspace_bytes, stream, nullptr, nullptr, nullptr, &plan, &sel,
+                  &dev);
+  if (rc != TOPLOC_OK) return rc;
   VerifyIo io;
   io.proofs = d_proofs;
   io.results = d_results;
@@ -959,14 +1305,13 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   io.sign_in_exponent = thr->sign_in_exponent;
   io.t_mean = thr->t_mean;
   io.t_median = thr->t_median;
-  const int mode = pick_mode(d_act, lay);
-  if (lay->dtype == TOPLOC_DTYPE_BF16) launch_verify<0>(mode, (unsigned)plan.num_chunks, stream, bp, io);
-  else launch_verify<1>(mode, (unsigned)plan.num_chunks, stream, bp, io);
+  const long long blocks = (plan.num_chunks + kVerifyWarps - 1) / kVerifyWarps;
+  toploc_evaluate_kernel<<<(unsigned)blocks, kVerifyWarps * 32, 0, stream>>>(sel, io, lay->k, plan.num_chunks);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
 // Shared driver of the two host-memory entry points: groups of whole sequences
-// go host -> staging -> kernel -> host, in stream order.
+// go host -> staging -> kernels -> host, in stream order.
 static int run_from_host(bool verify, const void* h_act, const toploc_layout* lay, uint8_t* h_proofs_out,
                          const uint8_t* h_proofs_in, uint8_t* h_status, const toploc_thresholds* thr,
                          toploc_chunk_result* h_results, void* d_staging, size_t staging_bytes,
@@ -980,7 +1325,6 @@ static int run_from_host(bool verify, const void* h_act, const toploc_layout* la
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t esz = lay->dtype == TOPLOC_DTYPE_BF16 ? 2 : 4;
   const size_t pb = 2 + 2 * (size_t)lay->k;
-  const size_t small_elem = verify ? sizeof(toploc_chunk_result) : 1;
   char* stage = static_cast<char*>(d_staging);
   int64_t* rebased = static_cast<int64_t*>(malloc(((size_t)lay->num_seqs + 1) * sizeof(int64_t)));
   if (rebased == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
@@ -989,11 +1333,10 @@ static int run_from_host(bool verify, const void* h_act, const toploc_layout* la
   while (s0 < lay->num_seqs && rc == TOPLOC_OK) {
     // largest group of sequences starting at s0 that fits
     int s1 = s0 + 1;
-    StagingPlan sp = carve_staging(lay, seq_begin(lay, s1) - seq_begin(lay, s0), chunks_between(lay, s0, s1),
-                                   sizeof(toploc_chunk_result));
+    StagingPlan sp = carve_staging(lay, seq_begin(lay, s1) - seq_begin(lay, s0), chunks_between(lay, s0, s1));
     while (s1 < lay->num_seqs) {
-      StagingPlan bigger = carve_staging(lay, seq_begin(lay, s1 + 1) - seq_begin(lay, s0),
-                                         chunks_between(lay, s0, s1 + 1), sizeof(toploc_chunk_result));
+      StagingPlan bigger =
+          carve_staging(lay, seq_begin(lay, s1 + 1) - seq_begin(lay, s0), chunks_between(lay, s0, s1 + 1));
       if (bigger.total > staging_bytes) break;
       sp = bigger;
       ++s1;
@@ -1014,7 +1357,7 @@ static int run_from_host(bool verify, const void* h_act, const toploc_layout* la
       if (rc == TOPLOC_OK && !verify) {
         rc = toploc_build_proofs(stage + sp.act_off, &sub, reinterpret_cast<uint8_t*>(stage + sp.proofs_off),
                                  reinterpret_cast<uint8_t*>(stage + sp.small_off), nullptr,
-                                 stage + sp.spans_off, sp.total - sp.spans_off, stream);
+                                 stage + sp.work_off, sp.work_bytes, stream);
         if (rc == TOPLOC_OK &&
             (cudaMemcpyAsync(h_proofs_out + (size_t)chunk0 * pb, stage + sp.proofs_off, (size_t)chunks * pb,
                              cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
@@ -1028,14 +1371,13 @@ static int run_from_host(bool verify, const void* h_act, const toploc_layout* la
         if (rc == TOPLOC_OK)
           rc = toploc_verify_proofs(stage + sp.act_off, &sub, reinterpret_cast<uint8_t*>(stage + sp.proofs_off),
                                     thr, reinterpret_cast<toploc_chunk_result*>(stage + sp.small_off), nullptr,
-                                    stage + sp.spans_off, sp.total - sp.spans_off, stream);
+                                    stage + sp.work_off, sp.work_bytes, stream);
         if (rc == TOPLOC_OK &&
-            cudaMemcpyAsync(h_results + chunk0, stage + sp.small_off, (size_t)chunks * small_elem,
-                            cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+            cudaMemcpyAsync(h_results + chunk0, stage + sp.small_off,
+                            (size_t)chunks * sizeof(toploc_chunk_result), cudaMemcpyDeviceToHost,
+                            stream) != cudaSuccess)
           rc = TOPLOC_ERR_CUDA;
       }
-      // the ragged row table of this group is read from `rebased` before the call returns,
-      // and staged copies of pageable memory are complete on return: safe to reuse both
     }
     chunk0 += chunks;
     s0 = s1;

@@ -61,12 +61,13 @@ def test_constants_and_sizes():
 def test_chunk_counting():
     assert tl.toploc_num_chunks(layout()) == 2 * 4          # ceil(100 / 32) per sequence
     assert tl.toploc_num_chunks(layout(tokens_per_seq=4096, num_seqs=256)) == 32768
-    assert tl.toploc_workspace_bytes(layout()) == 0
+    per_chunk = 128 * 4 + 128 * 2 + 1
+    assert 8 * per_chunk <= tl.toploc_workspace_bytes(layout()) <= 8 * per_chunk + 3 * 256
     offs = np.array([0, 9, 9, 23], np.int64)
     lay = layout(num_seqs=3, chunk_len=4)
     lay.seq_offsets = offs.ctypes.data_as(ctypes.POINTER(ctypes.c_int64))
     assert tl.toploc_num_chunks(lay) == 7
-    assert tl.toploc_workspace_bytes(lay) == 7 * 16
+    assert tl.toploc_workspace_bytes(lay) >= 7 * 16 + 7 * per_chunk
     assert tl.toploc_staging_bytes(layout()) >= 100 * 4096 * 2 + 4 * 258
 
 
