@@ -38,13 +38,13 @@ constexpr uint32_t kModLow = 32769u;
 #define TOPLOC_SELECT_MIN_BLOCKS 13      // select: one-warp blocks per SM (shared memory allows 13)
 #endif
 #ifndef TOPLOC_SELECT_STAGES
-#define TOPLOC_SELECT_STAGES 3           // select: tiles in flight per warp
+#define TOPLOC_SELECT_STAGES 2           // select: tiles in flight per warp
 #endif
 constexpr int kThreads = 32;             // select: one warp per chunk
 constexpr int kUnroll = 4;               // select: 16-byte loads per lane and tile
 constexpr int kStages = TOPLOC_SELECT_STAGES;
-constexpr int kCandCap = 640;            // select: candidate buffer entries (8 bytes each)
-constexpr int kHitCap = 96;              // select: vectors that can be parked between drains
+constexpr int kCandCap = 768;            // select: candidate buffer entries (8 bytes each)
+constexpr int kHitCap = 160;             // select: vectors that can be parked between drains
 constexpr int kHitTrigger = 32;          // select: drain once this many are parked
 constexpr int kMaxK = TOPLOC_MAX_K;
 constexpr int kMaxSlots = kMaxK / 32;    // tail: entries a lane owns at most
@@ -54,6 +54,7 @@ constexpr int kInterpWarps = 32;         // interpolation kernel: warps (= chunk
 constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
 static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
+static_assert(kHitCap >= kHitTrigger - 1 + kThreads * kUnroll, "a tile's hits must fit below the drain trigger");
 
 struct ChunkSpan {   // one per chunk of a ragged batch, built on the host
   long long row0;
@@ -106,8 +107,6 @@ struct __align__(16) SelectShared {
   uint32_t hist[256];                 // digit histogram of a compaction pass
   uint32_t top_hist[256];             // held candidates by the upper 8 bits of their 15-bit key
   uint32_t low_hist[128];             // those whose upper bits equal top_bin, by the lower 7 bits
-  int count;                          // candidates held
-  int nhits;                          // hit vectors held
   uint32_t top_bin;                   // which upper-bits value low_hist describes (kNoBin: none)
   uint32_t digit;
   uint32_t bin;
@@ -117,19 +116,16 @@ constexpr uint32_t kNoBin = 0xFFFFFFFFu;
 static_assert(sizeof(uint4) * kStages * kUnroll * kThreads + 8 * kCandCap >= 8192,
               "ring + candidates double as the 65536-bit residue set");
 
-// The block is one warp, so a block barrier is a warp barrier that also orders
-// shared memory.
-__device__ __forceinline__ void warp_barrier() { __syncwarp(); }
+// What the warp knows about its chunk so far.  Every lane holds the same
+// values: appends are agreed on by ballot, so the counters need no atomics.
+struct WarpState {
+  uint32_t thr;  // an element is a candidate iff its key is >= thr
+  int count;     // candidates held in sh.cand
+  int nhits;     // vectors parked in sh.hit_vec
+};
 
-// A shared-memory word as the whole warp agrees on it: lane 0 reads, everyone
-// receives.  Used for every value that steers a branch, so that a lane running
-// ahead (and already appending again) cannot make the others see another value.
-template <typename T>
-__device__ __forceinline__ T uniform_load(const T* p) {
-  T v = T();
-  if (threadIdx.x == 0) v = *p;
-  return __shfl_sync(0xFFFFFFFFu, v, 0);
-}
+// The block is one warp, so a warp barrier orders its shared memory.
+__device__ __forceinline__ void warp_barrier() { __syncwarp(); }
 
 // The 15-bit key the running threshold is kept in: a bf16 key as it is, the
 // upper half of an fp32 key.
@@ -149,31 +145,13 @@ __device__ __forceinline__ uint4 load_streaming(const uint4* p) {
 
 // 16 bytes global -> shared without passing through registers; completion is
 // tracked per thread in commit groups (a thread only ever reads what it copied).
-__device__ __forceinline__ void copy_async_16(void* smem_dst, const void* gmem_src) {
-  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+__device__ __forceinline__ void copy_async_16(uint32_t smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void copy_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-template <int DT>
-__device__ __forceinline__ void count_candidate(SelectShared& sh, unsigned long long c) {
-  const uint32_t key = coarse_key<DT>(c);
-  atomicAdd(&sh.top_hist[key >> 7], 1u);
-  if ((key >> 7) == sh.top_bin) atomicAdd(&sh.low_hist[key & 127u], 1u);
-}
-
-template <int DT>
-__device__ __forceinline__ void push_candidate(SelectShared& sh, unsigned long long c, int& max_pos) {
-  int pos = atomicAdd(&sh.count, 1);
-  if (pos < kCandCap) {
-    sh.cand[pos] = c;
-    count_candidate<DT>(sh, c);
-  }
-  max_pos = max(max_pos, pos);
 }
 
 // ---------------------------------------------------------------------------
@@ -239,30 +217,20 @@ __device__ __forceinline__ bool vector_has_candidate(const uint4& w, uint32_t th
 
 __device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
 
-// Appends every element of one vector whose key is >= thr to the candidate
-// buffer.  flat0 = flat index of the vector's first element.
+// Element e of a vector as (key, sign).
 template <int DT, int VEC>
-__device__ __forceinline__ void push_vector(SelectShared& sh, const uint4& w, uint32_t thr, uint32_t flat0,
-                                            int& max_pos) {
+__device__ __forceinline__ void vector_element(const uint4& w, int e, uint32_t* key, uint32_t* sign) {
+  const uint32_t words[4] = {w.x, w.y, w.z, w.w};
   if (VEC == 1) {
-    uint32_t key = DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu);
-    uint32_t sign = DT == 0 ? (w.x >> 15) & 1u : (w.x >> 31);
-    if (key >= thr) push_candidate<DT>(sh, make_candidate(key, flat0, sign), max_pos);
+    *key = DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu);
+    *sign = DT == 0 ? (w.x >> 15) & 1u : (w.x >> 31);
   } else if (DT == 0) {
-    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t lo = words[i] & 0x7FFFu, hi = (words[i] >> 16) & 0x7FFFu;
-      if (lo >= thr) push_candidate<DT>(sh, make_candidate(lo, flat0 + 2 * i, (words[i] >> 15) & 1u), max_pos);
-      if (hi >= thr) push_candidate<DT>(sh, make_candidate(hi, flat0 + 2 * i + 1, words[i] >> 31), max_pos);
-    }
+    const uint32_t half = (words[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu;
+    *key = half & 0x7FFFu;
+    *sign = half >> 15;
   } else {
-    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint32_t key = words[i] & 0x7FFFFFFFu;
-      if (key >= thr) push_candidate<DT>(sh, make_candidate(key, flat0 + i, words[i] >> 31), max_pos);
-    }
+    *key = words[e & 3] & 0x7FFFFFFFu;
+    *sign = words[e & 3] >> 31;
   }
 }
 
@@ -274,7 +242,7 @@ __device__ __forceinline__ void push_vector(SelectShared& sh, const uint4& w, ui
 template <int PER_LANE>
 __device__ __forceinline__ void find_from_top(SelectShared& sh, const uint32_t* hist, int want) {
   const int lane = threadIdx.x;
-  warp_barrier();  // results of an earlier call have been read by every lane
+  warp_barrier();  // histogram updates are in; results of an earlier call have been read
   uint32_t local[PER_LANE];
   uint32_t sum = 0;
 #pragma unroll
@@ -314,70 +282,65 @@ __device__ __forceinline__ void find_from_top(SelectShared& sh, const uint32_t* 
 // 15 bits are only the upper half of the key, so later elements need only
 // reach it.
 template <int DT>
-__device__ __noinline__ uint32_t raise_threshold(SelectShared& sh, int k, uint32_t thr) {
+__device__ __noinline__ uint32_t raise_threshold(SelectShared& sh, int k, uint32_t thr, int count) {
   const int lane = threadIdx.x;
-  warp_barrier();  // every append and its histogram updates are in
+  if (count < k) return thr;
   find_from_top<8>(sh, sh.top_hist, k);
   const uint32_t top = sh.digit;
   const int want = sh.want;
-  if (top == kNoBin) return thr;  // fewer than k candidates so far
   if (top != sh.top_bin) {
     // the boundary moved into another upper-bits bin: describe that one
     warp_barrier();
     for (int b = lane; b < 128; b += kThreads) sh.low_hist[b] = 0;
     if (lane == 0) sh.top_bin = top;
     warp_barrier();
-    const int n = min(uniform_load(&sh.count), kCandCap);
-    for (int e = lane; e < n; e += kThreads) {
+    for (int e = lane; e < count; e += kThreads) {
       const uint32_t key = coarse_key<DT>(sh.cand[e]);
       if ((key >> 7) == top) atomicAdd(&sh.low_hist[key & 127u], 1u);
     }
-    warp_barrier();
   }
   find_from_top<4>(sh, sh.low_hist, want);
   const uint32_t key = (top << 7) | sh.digit;
   const uint32_t raised = DT == 0 ? key + 1u : key << 16;
-  warp_barrier();
   return max(thr, raised);
 }
 
 // Keeps the best candidates (radix select on the 56 meaningful bits, most
-// significant digit first) and returns the raised threshold "strictly better
-// than the k-th".  Ties on the key are only broken by index when it matters:
-// once the key digits are settled the scan stops if the boundary bin can be
-// kept whole -- because exactly k candidates remain, or, for a compaction in
+// significant digit first) and sets the threshold to "strictly better than
+// the k-th".  Ties on the key are only broken by index when it matters: once
+// the key digits are settled the scan stops if the boundary bin can be kept
+// whole -- because exactly k candidates remain, or, for a compaction in
 // mid-stream (exact == false), because at most kMaxK remain; only the last
-// compaction of a chunk must leave exactly k.
+// compaction of a chunk must leave exactly k.  Returns the new state.
 template <int DT>
-__device__ __noinline__ uint32_t compact_candidates(SelectShared& sh, int k, uint32_t thr, bool exact) {
+__device__ __noinline__ WarpState compact_candidates(SelectShared& sh, int k, WarpState st, bool exact) {
   const int lane = threadIdx.x;
-  warp_barrier();
-  const int n = min(uniform_load(&sh.count), kCandCap);
-  if (n <= k) return thr;
+  const int n = st.count;
+  if (n <= k) return st;
   unsigned long long prefix = 0ull, mask = 0ull;
   int want = k;
   // bf16 keys have 15 bits: candidate bits 40..55 are zero, two digit passes fewer
 #pragma unroll 1
   for (int shift = (DT == 0 ? 32 : 48); shift >= 0; shift -= 8) {
+    warp_barrier();
     for (int b = lane; b < 256; b += kThreads) sh.hist[b] = 0;
     warp_barrier();
     for (int e = lane; e < n; e += kThreads) {
       const unsigned long long c = sh.cand[e];
       if ((c & mask) == prefix) atomicAdd(&sh.hist[(uint32_t)(c >> shift) & 255u], 1u);
     }
-    warp_barrier();
     find_from_top<8>(sh, sh.hist, want);  // largest digit with enough candidates at or above it
     prefix |= (unsigned long long)sh.digit << shift;
     mask |= 255ull << shift;
     want = sh.want;
     const int kept = k - want + (int)sh.bin;
-    warp_barrier();
     // lower bits of the pivot stay 0: the boundary bin is kept whole
     if (shift <= 24 && (kept == k || (!exact && kept <= kMaxK))) break;
   }
   const unsigned long long pivot = prefix;  // everything >= pivot is kept
-  // in-place, in order: a slot is overwritten only after it has been read
+  // in place, in order: a slot is overwritten only after it has been read
   int out = 0;
+  warp_barrier();
   for (int base = 0; base < n; base += kThreads) {
     const int e = base + lane;
     const unsigned long long c = e < n ? sh.cand[e] : 0ull;
@@ -390,67 +353,98 @@ __device__ __noinline__ uint32_t compact_candidates(SelectShared& sh, int k, uin
   }
   // the key histograms describe the survivors only
   for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
-  if (lane == 0) {
-    sh.count = out;
-    sh.top_bin = kNoBin;
-  }
+  if (lane == 0) sh.top_bin = kNoBin;
   warp_barrier();
   for (int e = lane; e < out; e += kThreads) atomicAdd(&sh.top_hist[coarse_key<DT>(sh.cand[e]) >> 7], 1u);
   warp_barrier();
-  return max(thr, (uint32_t)(pivot >> (kIdxBits + 1)) + 1u);
+  st.count = out;
+  st.thr = max(st.thr, (uint32_t)(pivot >> (kIdxBits + 1)) + 1u);
+  return st;
+}
+
+// Appends the elements of one vector per lane that reach the threshold.  The
+// lanes agree on the slots by ballot, element position by element position, so
+// the whole warp stays in step and the counter needs no atomic.  Makes room
+// first (a mid-stream compaction) if the round would not fit.
+template <int DT, int VEC>
+__device__ __forceinline__ void append_round(SelectShared& sh, int k, WarpState& st, const uint4& w, bool valid,
+                                             uint32_t flat0) {
+  const int lane = threadIdx.x;
+  const uint32_t below = (1u << lane) - 1u;
+  uint32_t votes[VEC];
+  int total = 0;
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    uint32_t key, sign;
+    vector_element<DT, VEC>(w, e, &key, &sign);
+    votes[e] = __ballot_sync(0xFFFFFFFFu, valid && key >= st.thr);
+    total += __popc(votes[e]);
+  }
+  if (st.count + total > kCandCap) {
+    st = compact_candidates<DT>(sh, k, st, false);  // leaves at most kMaxK; a round adds at most 32 * VEC
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+      uint32_t key, sign;
+      vector_element<DT, VEC>(w, e, &key, &sign);
+      votes[e] = __ballot_sync(0xFFFFFFFFu, valid && key >= st.thr);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    if (votes[e]) {  // the same for every lane
+      if ((votes[e] >> lane) & 1u) {
+        uint32_t key, sign;
+        vector_element<DT, VEC>(w, e, &key, &sign);
+        const unsigned long long c = make_candidate(key, flat0 + e, sign);
+        sh.cand[st.count + __popc(votes[e] & below)] = c;
+        const uint32_t ck = coarse_key<DT>(c);
+        atomicAdd(&sh.top_hist[ck >> 7], 1u);
+        if ((ck >> 7) == sh.top_bin) atomicAdd(&sh.low_hist[ck & 127u], 1u);
+      }
+      st.count += __popc(votes[e]);
+    }
+  }
 }
 
 // Processes vectors [vb, ve) one vector per lane at a time, raising the
-// threshold after every round and compacting whenever another round might not
-// fit.
+// threshold after every round.
 template <int DT, int MODE>
-__device__ __noinline__ uint32_t select_carefully(SelectShared& sh, const ChunkSource<DT, MODE> src, int vb,
-                                                  int ve, int k, uint32_t thr) {
+__device__ __noinline__ WarpState select_carefully(SelectShared& sh, const ChunkSource<DT, MODE> src, int vb,
+                                                   int ve, int k, WarpState st) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x;
   for (int s = vb; s < ve; s += kThreads) {
-    warp_barrier();
-    if (uniform_load(&sh.count) + kThreads * VEC > kCandCap) thr = compact_candidates<DT>(sh, k, thr, false);
     const int v = s + lane;
-    int max_pos = -1;
-    if (v < ve) push_vector<DT, VEC>(sh, src.load(v), thr, (uint32_t)v * VEC, max_pos);
-    thr = raise_threshold<DT>(sh, k, thr);
+    const bool valid = v < ve;
+    uint4 w = make_uint4(0, 0, 0, 0);
+    if (valid) w = src.load(v);
+    append_round<DT, VEC>(sh, k, st, w, valid, (uint32_t)v * VEC);
+    st.thr = raise_threshold<DT>(sh, k, st.thr, st.count);
   }
-  return thr;
+  return st;
 }
 
-// Unpacks the held hit vectors into candidates (against the current, possibly
-// higher, threshold), one vector per lane and round, then raises the threshold.
+// Unpacks the parked hit vectors into candidates (against the current,
+// possibly higher, threshold), one vector per lane and round, then raises the
+// threshold.
 template <int DT, int VEC>
-__device__ __noinline__ uint32_t drain_hits(SelectShared& sh, int k, uint32_t thr) {
+__device__ __noinline__ WarpState drain_hits(SelectShared& sh, int k, WarpState st) {
   const int lane = threadIdx.x;
-  warp_barrier();
-  const int nh = min(uniform_load(&sh.nhits), kHitCap);
-  for (int base = 0; base < nh; base += kThreads) {
-    warp_barrier();
-    if (uniform_load(&sh.count) + kThreads * VEC > kCandCap) thr = compact_candidates<DT>(sh, k, thr, false);
+  warp_barrier();  // the parked vectors are visible
+  for (int base = 0; base < st.nhits; base += kThreads) {
     const int h = base + lane;
-    int max_pos = -1;
-    if (h < nh) push_vector<DT, VEC>(sh, sh.hit_vec[h], thr, sh.hit_idx[h] * VEC, max_pos);
-    thr = raise_threshold<DT>(sh, k, thr);
+    const bool valid = h < st.nhits;
+    uint4 w = make_uint4(0, 0, 0, 0);
+    uint32_t v = 0;
+    if (valid) {
+      w = sh.hit_vec[h];
+      v = sh.hit_idx[h];
+    }
+    append_round<DT, VEC>(sh, k, st, w, valid, v * VEC);
   }
-  warp_barrier();
-  if (lane == 0) sh.nhits = 0;
-  warp_barrier();
-  return thr;
-}
-
-// Forgets everything held.
-__device__ void reset_selection(SelectShared& sh) {
-  const int lane = threadIdx.x;
-  warp_barrier();
-  for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
-  if (lane == 0) {
-    sh.count = 0;
-    sh.nhits = 0;
-    sh.top_bin = kNoBin;
-  }
-  warp_barrier();
+  st.nhits = 0;
+  st.thr = raise_threshold<DT>(sh, k, st.thr, st.count);
+  return st;
 }
 
 // Exact top-k of one chunk by one warp: on return sh.cand[0..k) holds the k
@@ -459,8 +453,8 @@ __device__ void reset_selection(SelectShared& sh) {
 //
 // The chunk is streamed in index order.  A warm-up over the first vectors
 // establishes a threshold; after that a lane only tests whether a 16-byte
-// vector holds anything at or above the threshold and, if so, parks the whole
-// vector in shared memory.  Parked vectors are unpacked by the whole warp at
+// vector holds anything at or above the threshold and, if so, the vector is
+// parked in shared memory.  Parked vectors are unpacked by the whole warp at
 // once, so the rare slow work is done with every lane busy.  Nothing here
 // waits on another warp: a chunk's serial steps only delay that chunk, while
 // the other warps of the SM keep their own loads in flight.
@@ -469,10 +463,15 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   constexpr int kTileVecs = kThreads * kUnroll;
   const int lane = threadIdx.x;
+  const uint32_t below = (1u << lane) - 1u;
   const int n_vecs = n_elems / VEC;
 
-  reset_selection(sh);
-  uint32_t thr = 0;  // accept everything until k candidates exist
+  for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
+  if (lane == 0) sh.top_bin = kNoBin;
+  WarpState st;
+  st.thr = 0;  // accept everything until k candidates exist
+  st.count = 0;
+  st.nhits = 0;
 
   // Warm-up: enough elements that afterwards only a minority of vectors hit.
   const int warm = min(n_vecs, (32 / VEC) * max(k, 128));
@@ -485,22 +484,22 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
   // warp drains or compacts.  Slot (stage, u, lane) is private to its lane.
   // The first tiles are requested before the warm-up starts.
   constexpr bool kRing = (MODE != 2);
+  const uint32_t ring_lane = (uint32_t)__cvta_generic_to_shared(&sh.ring[lane]);
   auto request_tile = [&](int tile) {
     if (kRing && tile < n_tiles) {
-      const int stage = tile % kStages;
+      const uint32_t dst = ring_lane + (uint32_t)((tile % kStages) * kUnroll * kThreads * sizeof(uint4));
+      const int v = warm + tile * kTileVecs + lane;
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u)
-        copy_async_16(&sh.ring[(stage * kUnroll + u) * kThreads + lane],
-                      src.address(warm + tile * kTileVecs + u * kThreads + lane));
+        copy_async_16(dst + (uint32_t)(u * kThreads * sizeof(uint4)), src.address(v + u * kThreads));
     }
     if (kRing) copy_async_commit();
   };
   for (int t = 0; t < kStages; ++t) request_tile(t);
+  warp_barrier();
 
-  thr = select_carefully<DT, MODE>(sh, src, 0, warm, k, thr);
+  st = select_carefully<DT, MODE>(sh, src, 0, warm, k, st);
 
-  int max_hit = -1;
-  bool overflow = false;
   for (int tile = 0; tile < n_tiles; ++tile) {
     const int v0 = warm + tile * kTileVecs;
     uint4 w[kUnroll];
@@ -513,40 +512,29 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) w[u] = src.load(v0 + u * kThreads + lane);
     }
-    const uint32_t add = bf16_lane_add(thr);
+    const uint32_t add = bf16_lane_add(st.thr);
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      if (vector_has_candidate<DT, VEC>(w[u], thr, add)) {
-        const int pos = atomicAdd(&sh.nhits, 1);
-        if (pos < kHitCap) {
+      const bool hit = vector_has_candidate<DT, VEC>(w[u], st.thr, add);
+      const uint32_t votes = __ballot_sync(0xFFFFFFFFu, hit);
+      if (votes) {  // the same for every lane
+        if (hit) {
+          const int pos = st.nhits + __popc(votes & below);
           sh.hit_vec[pos] = w[u];
           sh.hit_idx[pos] = (uint32_t)(v0 + u * kThreads + lane);
         }
-        max_hit = max(max_hit, pos);
+        st.nhits += __popc(votes);
       }
     }
     request_tile(tile + kStages);  // refill the stage just consumed
-    if (__any_sync(0xFFFFFFFFu, max_hit + 1 >= kHitTrigger)) {
-      warp_barrier();
-      if (uniform_load(&sh.nhits) > kHitCap) {
-        overflow = true;
-        break;
-      }
-      thr = drain_hits<DT, VEC>(sh, k, thr);
-      max_hit = -1;
-    }
+    // a tile parks at most kTileVecs vectors, so the buffer cannot overflow
+    if (st.nhits >= kHitTrigger) st = drain_hits<DT, VEC>(sh, k, st);
   }
   if (kRing) copy_async_wait<0>();
-  if (overflow) {
-    // More vectors hit within one tile than can be parked (e.g. magnitudes
-    // that keep growing).  Start over, carefully.
-    reset_selection(sh);
-    thr = select_carefully<DT, MODE>(sh, src, 0, n_vecs, k, 0u);
-  } else {
-    thr = drain_hits<DT, VEC>(sh, k, thr);
-    thr = select_carefully<DT, MODE>(sh, src, full_end, n_vecs, k, thr);
-  }
-  compact_candidates<DT>(sh, k, thr, true);  // exactly k remain
+  st = drain_hits<DT, VEC>(sh, k, st);
+  st = select_carefully<DT, MODE>(sh, src, full_end, n_vecs, k, st);
+  compact_candidates<DT>(sh, k, st, true);  // exactly k remain
+  warp_barrier();
 }
 
 // ---------------------------------------------------------------------------
