@@ -53,6 +53,7 @@ constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
 constexpr int kInterpWarps = 32;         // interpolation kernel: warps (= chunks in flight) per block
 constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
+static_assert(kUnroll % 2 == 0, "vectors are tested in pairs");
 static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
 static_assert(kHitCap >= kHitTrigger - 1 + kThreads * kUnroll, "a tile's hits must fit below the drain trigger");
 
@@ -217,20 +218,20 @@ __device__ __forceinline__ bool vector_has_candidate(const uint4& w, uint32_t th
 
 __device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
 
-// Element e of a vector as (key, sign).
+// Cheap necessary condition for "one of these two vectors holds a candidate":
+// the OR of all their keys reaches the threshold (an OR is never below any of
+// its operands).  One test per 32 bytes on the elements that lose.
 template <int DT, int VEC>
-__device__ __forceinline__ void vector_element(const uint4& w, int e, uint32_t* key, uint32_t* sign) {
-  const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+__device__ __forceinline__ bool pair_may_hold_candidate(const uint4& a, const uint4& b, uint32_t thr, uint32_t add) {
   if (VEC == 1) {
-    *key = DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu);
-    *sign = DT == 0 ? (w.x >> 15) & 1u : (w.x >> 31);
+    const uint32_t m = DT == 0 ? 0x7FFFu : 0x7FFFFFFFu;
+    return ((a.x | b.x) & m) >= thr;
   } else if (DT == 0) {
-    const uint32_t half = (words[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu;
-    *key = half & 0x7FFFu;
-    *sign = half >> 15;
+    const uint32_t any = ((a.x | a.y | a.z) | (a.w | b.x | b.y) | (b.z | b.w)) & 0x7FFF7FFFu;
+    return ((any + add) & 0x80008000u) != 0;
   } else {
-    *key = words[e & 3] & 0x7FFFFFFFu;
-    *sign = words[e & 3] >> 31;
+    const uint32_t any = ((a.x | a.y | a.z) | (a.w | b.x | b.y) | (b.z | b.w)) & 0x7FFFFFFFu;
+    return any >= thr;
   }
 }
 
@@ -362,48 +363,87 @@ __device__ __noinline__ WarpState compact_candidates(SelectShared& sh, int k, Wa
   return st;
 }
 
-// Appends the elements of one vector per lane that reach the threshold.  The
-// lanes agree on the slots by ballot, element position by element position, so
-// the whole warp stays in step and the counter needs no atomic.  Makes room
-// first (a mid-stream compaction) if the round would not fit.
+// Bit e of the result is set iff element e of the vector has key >= thr.
+template <int DT, int VEC>
+__device__ __forceinline__ uint32_t passing_mask(const uint4& w, uint32_t thr) {
+  if (VEC == 1) {
+    return ((DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu)) >= thr) ? 1u : 0u;
+  } else if (DT == 0) {
+    const uint32_t add = bf16_lane_add(thr);
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t t = (words[i] & 0x7FFF7FFFu) + add;  // top bit of each half: key >= thr
+      m |= ((t >> 15) & 1u) << (2 * i);
+      m |= (t >> 31) << (2 * i + 1);
+    }
+    return m;
+  } else {
+    return ((w.x & 0x7FFFFFFFu) >= thr ? 1u : 0u) | ((w.y & 0x7FFFFFFFu) >= thr ? 2u : 0u) |
+           ((w.z & 0x7FFFFFFFu) >= thr ? 4u : 0u) | ((w.w & 0x7FFFFFFFu) >= thr ? 8u : 0u);
+  }
+}
+
+// Element e (a run-time position) of a vector as (key, sign), by selects.
+template <int DT, int VEC>
+__device__ __forceinline__ void pick_element(const uint4& w, uint32_t e, uint32_t* key, uint32_t* sign) {
+  if (VEC == 1) {
+    *key = DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu);
+    *sign = DT == 0 ? (w.x >> 15) & 1u : (w.x >> 31);
+  } else {
+    const uint32_t wi = DT == 0 ? (e >> 1) : e;
+    const uint32_t word = (wi & 2u) ? ((wi & 1u) ? w.w : w.z) : ((wi & 1u) ? w.y : w.x);
+    if (DT == 0) {
+      const uint32_t half = (word >> ((e & 1u) * 16u)) & 0xFFFFu;
+      *key = half & 0x7FFFu;
+      *sign = half >> 15;
+    } else {
+      *key = word & 0x7FFFFFFFu;
+      *sign = word >> 31;
+    }
+  }
+}
+
+// Appends the elements of one vector per lane that reach the threshold.  Each
+// lane counts its passing elements, a warp prefix sum hands out the slots (the
+// counter is warp-uniform, no atomic), then every lane stores its own few.
+// Makes room first (a mid-stream compaction) if the round would not fit.
 template <int DT, int VEC>
 __device__ __forceinline__ void append_round(SelectShared& sh, int k, WarpState& st, const uint4& w, bool valid,
                                              uint32_t flat0) {
   const int lane = threadIdx.x;
-  const uint32_t below = (1u << lane) - 1u;
-  uint32_t votes[VEC];
-  int total = 0;
+  uint32_t mask = 0;
+  int incl = 0, total = 0;
+#pragma unroll 1
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    mask = valid ? passing_mask<DT, VEC>(w, st.thr) : 0u;
+    incl = __popc(mask);
 #pragma unroll
-  for (int e = 0; e < VEC; ++e) {
+    for (int off = 1; off < 32; off <<= 1) {
+      const int other = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+      if (lane >= off) incl += other;
+    }
+    total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    if (st.count + total <= kCandCap) break;
+    // leaves at most kMaxK and may raise the threshold; a round adds at most 32 * VEC
+    st = compact_candidates<DT>(sh, k, st, false);
+  }
+  int pos = st.count + incl - __popc(mask);
+  const uint32_t top_bin = sh.top_bin;
+  while (mask) {
+    const uint32_t e = (uint32_t)__ffs((int)mask) - 1u;
+    mask &= mask - 1u;
     uint32_t key, sign;
-    vector_element<DT, VEC>(w, e, &key, &sign);
-    votes[e] = __ballot_sync(0xFFFFFFFFu, valid && key >= st.thr);
-    total += __popc(votes[e]);
+    pick_element<DT, VEC>(w, e, &key, &sign);
+    const unsigned long long c = make_candidate(key, flat0 + e, sign);
+    sh.cand[pos++] = c;
+    const uint32_t ck = coarse_key<DT>(c);
+    atomicAdd(&sh.top_hist[ck >> 7], 1u);
+    if ((ck >> 7) == top_bin) atomicAdd(&sh.low_hist[ck & 127u], 1u);
   }
-  if (st.count + total > kCandCap) {
-    st = compact_candidates<DT>(sh, k, st, false);  // leaves at most kMaxK; a round adds at most 32 * VEC
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) {
-      uint32_t key, sign;
-      vector_element<DT, VEC>(w, e, &key, &sign);
-      votes[e] = __ballot_sync(0xFFFFFFFFu, valid && key >= st.thr);
-    }
-  }
-#pragma unroll
-  for (int e = 0; e < VEC; ++e) {
-    if (votes[e]) {  // the same for every lane
-      if ((votes[e] >> lane) & 1u) {
-        uint32_t key, sign;
-        vector_element<DT, VEC>(w, e, &key, &sign);
-        const unsigned long long c = make_candidate(key, flat0 + e, sign);
-        sh.cand[st.count + __popc(votes[e] & below)] = c;
-        const uint32_t ck = coarse_key<DT>(c);
-        atomicAdd(&sh.top_hist[ck >> 7], 1u);
-        if ((ck >> 7) == sh.top_bin) atomicAdd(&sh.low_hist[ck & 127u], 1u);
-      }
-      st.count += __popc(votes[e]);
-    }
-  }
+  __syncwarp();
+  st.count += total;
 }
 
 // Processes vectors [vb, ve) one vector per lane at a time, raising the
@@ -514,16 +554,20 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
     }
     const uint32_t add = bf16_lane_add(st.thr);
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const bool hit = vector_has_candidate<DT, VEC>(w[u], st.thr, add);
-      const uint32_t votes = __ballot_sync(0xFFFFFFFFu, hit);
-      if (votes) {  // the same for every lane
-        if (hit) {
-          const int pos = st.nhits + __popc(votes & below);
-          sh.hit_vec[pos] = w[u];
-          sh.hit_idx[pos] = (uint32_t)(v0 + u * kThreads + lane);
+    for (int u = 0; u < kUnroll; u += 2) {
+      // most pairs of vectors are dismissed by one test; `if (any)` is warp-uniform
+      if (__any_sync(0xFFFFFFFFu, pair_may_hold_candidate<DT, VEC>(w[u], w[u + 1], st.thr, add))) {
+#pragma unroll
+        for (int h = u; h < u + 2; ++h) {
+          const bool hit = vector_has_candidate<DT, VEC>(w[h], st.thr, add);
+          const uint32_t votes = __ballot_sync(0xFFFFFFFFu, hit);
+          if (hit) {
+            const int pos = st.nhits + __popc(votes & below);
+            sh.hit_vec[pos] = w[h];
+            sh.hit_idx[pos] = (uint32_t)(v0 + h * kThreads + lane);
+          }
+          st.nhits += __popc(votes);
         }
-        st.nhits += __popc(votes);
       }
     }
     request_tile(tile + kStages);  // refill the stage just consumed
