@@ -53,7 +53,6 @@ constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
 constexpr int kInterpWarps = 32;         // interpolation kernel: warps (= chunks in flight) per block
 constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
-static_assert(kUnroll % 2 == 0, "vectors are tested in pairs");
 static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
 static_assert(kHitCap >= kHitTrigger - 1 + kThreads * kUnroll, "a tile's hits must fit below the drain trigger");
 
@@ -195,43 +194,19 @@ struct ChunkSource {
 
 // Does any element of the vector have key >= thr?  bf16: both 15-bit keys of a
 // word sit in separate 16-bit lanes, and adding (0x8000 - thr) to a lane sets
-// its top bit exactly when key >= thr (no carry leaves a lane).  The OR of the
-// four words is tested first: a bitwise OR is never below any of its operands,
-// so a vector whose OR fails the test holds no candidate.
+// its top bit exactly when key >= thr (no carry leaves a lane).
+__device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
+
 template <int DT, int VEC>
-__device__ __forceinline__ bool vector_has_candidate(const uint4& w, uint32_t thr, uint32_t add) {
+__device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uint32_t add) {
   if (VEC == 1) {
     return (DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu)) >= thr;
   } else if (DT == 0) {
-    const uint32_t any = (w.x | w.y | w.z | w.w) & 0x7FFF7FFFu;
-    if (((any + add) & 0x80008000u) == 0) return false;
     const uint32_t t0 = (w.x & 0x7FFF7FFFu) + add, t1 = (w.y & 0x7FFF7FFFu) + add;
     const uint32_t t2 = (w.z & 0x7FFF7FFFu) + add, t3 = (w.w & 0x7FFF7FFFu) + add;
-    return ((t0 | t1 | t2 | t3) & 0x80008000u) != 0;
+    return (((t0 | t1 | t2) | t3) & 0x80008000u) != 0;
   } else {
-    const uint32_t any = (w.x | w.y | w.z | w.w) & 0x7FFFFFFFu;
-    if (any < thr) return false;
-    return (w.x & 0x7FFFFFFFu) >= thr || (w.y & 0x7FFFFFFFu) >= thr || (w.z & 0x7FFFFFFFu) >= thr ||
-           (w.w & 0x7FFFFFFFu) >= thr;
-  }
-}
-
-__device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
-
-// Cheap necessary condition for "one of these two vectors holds a candidate":
-// the OR of all their keys reaches the threshold (an OR is never below any of
-// its operands).  One test per 32 bytes on the elements that lose.
-template <int DT, int VEC>
-__device__ __forceinline__ bool pair_may_hold_candidate(const uint4& a, const uint4& b, uint32_t thr, uint32_t add) {
-  if (VEC == 1) {
-    const uint32_t m = DT == 0 ? 0x7FFFu : 0x7FFFFFFFu;
-    return ((a.x | b.x) & m) >= thr;
-  } else if (DT == 0) {
-    const uint32_t any = ((a.x | a.y | a.z) | (a.w | b.x | b.y) | (b.z | b.w)) & 0x7FFF7FFFu;
-    return ((any + add) & 0x80008000u) != 0;
-  } else {
-    const uint32_t any = ((a.x | a.y | a.z) | (a.w | b.x | b.y) | (b.z | b.w)) & 0x7FFFFFFFu;
-    return any >= thr;
+    return max(max(w.x & 0x7FFFFFFFu, w.y & 0x7FFFFFFFu), max(w.z & 0x7FFFFFFFu, w.w & 0x7FFFFFFFu)) >= thr;
   }
 }
 
@@ -459,7 +434,10 @@ __device__ __noinline__ WarpState select_carefully(SelectShared& sh, const Chunk
     uint4 w = make_uint4(0, 0, 0, 0);
     if (valid) w = src.load(v);
     append_round<DT, VEC>(sh, k, st, w, valid, (uint32_t)v * VEC);
-    st.thr = raise_threshold<DT>(sh, k, st.thr, st.count);
+    // early rounds move the threshold a lot, later ones little: raise after every round at
+    // first, then after every other one (and after the last)
+    const int round = (s - vb) / kThreads;
+    if (round < 6 || (round & 1) || s + kThreads >= ve) st.thr = raise_threshold<DT>(sh, k, st.thr, st.count);
   }
   return st;
 }
@@ -553,21 +531,27 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
       for (int u = 0; u < kUnroll; ++u) w[u] = src.load(v0 + u * kThreads + lane);
     }
     const uint32_t add = bf16_lane_add(st.thr);
+    // the tests of a tile's vectors are independent of each other: all of them first,
+    // then the votes, then one warp-uniform branch for the (less common) tile with a hit
+    bool hit[kUnroll];
+    uint32_t votes[kUnroll];
+    uint32_t any_votes = 0;
 #pragma unroll
-    for (int u = 0; u < kUnroll; u += 2) {
-      // most pairs of vectors are dismissed by one test; `if (any)` is warp-uniform
-      if (__any_sync(0xFFFFFFFFu, pair_may_hold_candidate<DT, VEC>(w[u], w[u + 1], st.thr, add))) {
+    for (int u = 0; u < kUnroll; ++u) hit[u] = vector_reaches<DT, VEC>(w[u], st.thr, add);
 #pragma unroll
-        for (int h = u; h < u + 2; ++h) {
-          const bool hit = vector_has_candidate<DT, VEC>(w[h], st.thr, add);
-          const uint32_t votes = __ballot_sync(0xFFFFFFFFu, hit);
-          if (hit) {
-            const int pos = st.nhits + __popc(votes & below);
-            sh.hit_vec[pos] = w[h];
-            sh.hit_idx[pos] = (uint32_t)(v0 + h * kThreads + lane);
-          }
-          st.nhits += __popc(votes);
+    for (int u = 0; u < kUnroll; ++u) {
+      votes[u] = __ballot_sync(0xFFFFFFFFu, hit[u]);
+      any_votes |= votes[u];
+    }
+    if (any_votes) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (hit[u]) {
+          const int pos = st.nhits + __popc(votes[u] & below);
+          sh.hit_vec[pos] = w[u];
+          sh.hit_idx[pos] = (uint32_t)(v0 + u * kThreads + lane);
         }
+        st.nhits += __popc(votes[u]);
       }
     }
     request_tile(tile + kStages);  // refill the stage just consumed
