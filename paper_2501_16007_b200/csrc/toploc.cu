@@ -17,6 +17,7 @@
 // spend about one instruction per element on the elements that lose.
 #include "toploc.h"
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -35,7 +36,7 @@ constexpr uint32_t kModLow = 32769u;
 // launch shape
 // ---------------------------------------------------------------------------
 #ifndef TOPLOC_SELECT_MIN_BLOCKS
-#define TOPLOC_SELECT_MIN_BLOCKS 13      // select: one-warp blocks per SM (shared memory allows 13)
+#define TOPLOC_SELECT_MIN_BLOCKS 15      // select: one-warp blocks per SM (shared memory allows 15)
 #endif
 #ifndef TOPLOC_SELECT_STAGES
 #define TOPLOC_SELECT_STAGES 2           // select: tiles in flight per warp
@@ -43,7 +44,7 @@ constexpr uint32_t kModLow = 32769u;
 constexpr int kThreads = 32;             // select: one warp per chunk
 constexpr int kUnroll = 4;               // select: 16-byte loads per lane and tile
 constexpr int kStages = TOPLOC_SELECT_STAGES;
-constexpr int kCandCap = 768;            // select: candidate buffer entries (8 bytes each)
+constexpr int kCandCap = 640;            // select: candidate buffer entries (8 bytes each)
 constexpr int kHitCap = 160;             // select: vectors that can be parked between drains
 constexpr int kHitTrigger = 32;          // select: drain once this many are parked
 constexpr int kMaxK = TOPLOC_MAX_K;
@@ -104,8 +105,8 @@ struct __align__(16) SelectShared {
   unsigned long long cand[kCandCap];  // candidates held; ring + cand later serve as the residue set
   uint4 hit_vec[kHitCap];             // vectors that passed the streaming filter, not yet unpacked
   uint32_t hit_idx[kHitCap];          // their vector index within the chunk
-  uint32_t hist[256];                 // digit histogram of a compaction pass
-  uint32_t top_hist[256];             // held candidates by the upper 8 bits of their 15-bit key
+  uint32_t top_hist[256];             // held candidates by the upper 8 bits of their 15-bit key; a
+                                      // compaction borrows it for its digit histograms
   uint32_t low_hist[128];             // those whose upper bits equal top_bin, by the lower 7 bits
   uint32_t top_bin;                   // which upper-bits value low_hist describes (kNoBin: none)
   uint32_t digit;
@@ -196,6 +197,22 @@ struct ChunkSource {
 // word sit in separate 16-bit lanes, and adding (0x8000 - thr) to a lane sets
 // its top bit exactly when key >= thr (no carry leaves a lane).
 __device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
+
+// The same test for bf16 through the half-precision compare unit: |x| >= t as
+// floating-point numbers orders finite magnitudes exactly like their bit
+// patterns, and the unordered form lets NaN patterns through (a superset is
+// fine here, the unpacking step repeats the test on integers).  Only valid
+// for thresholds that are normal numbers or infinity.
+__device__ __forceinline__ bool bf16_vector_reaches(const uint4& w, uint32_t thr2) {
+  const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(&thr2);
+  const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+  uint32_t any = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    any |= __hgeu2_mask(__habs2(*reinterpret_cast<const __nv_bfloat162*>(&words[i])), t);
+  return any != 0;
+}
+__device__ __forceinline__ bool bf16_threshold_is_ordinary(uint32_t thr) { return thr >= 0x0080u && thr <= 0x7F80u; }
 
 template <int DT, int VEC>
 __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uint32_t add) {
@@ -299,13 +316,13 @@ __device__ __noinline__ WarpState compact_candidates(SelectShared& sh, int k, Wa
 #pragma unroll 1
   for (int shift = (DT == 0 ? 32 : 48); shift >= 0; shift -= 8) {
     warp_barrier();
-    for (int b = lane; b < 256; b += kThreads) sh.hist[b] = 0;
+    for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
     warp_barrier();
     for (int e = lane; e < n; e += kThreads) {
       const unsigned long long c = sh.cand[e];
-      if ((c & mask) == prefix) atomicAdd(&sh.hist[(uint32_t)(c >> shift) & 255u], 1u);
+      if ((c & mask) == prefix) atomicAdd(&sh.top_hist[(uint32_t)(c >> shift) & 255u], 1u);
     }
-    find_from_top<8>(sh, sh.hist, want);  // largest digit with enough candidates at or above it
+    find_from_top<8>(sh, sh.top_hist, want);  // largest digit with enough candidates at or above it
     prefix |= (unsigned long long)sh.digit << shift;
     mask |= 255ull << shift;
     want = sh.want;
@@ -536,8 +553,14 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
     bool hit[kUnroll];
     uint32_t votes[kUnroll];
     uint32_t any_votes = 0;
+    if (DT == 0 && VEC == 8 && bf16_threshold_is_ordinary(st.thr)) {
+      const uint32_t thr2 = st.thr * 0x00010001u;
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) hit[u] = vector_reaches<DT, VEC>(w[u], st.thr, add);
+      for (int u = 0; u < kUnroll; ++u) hit[u] = bf16_vector_reaches(w[u], thr2);
+    } else {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) hit[u] = vector_reaches<DT, VEC>(w[u], st.thr, add);
+    }
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       votes[u] = __ballot_sync(0xFFFFFFFFu, hit[u]);

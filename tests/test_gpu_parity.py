@@ -104,6 +104,26 @@ def test_heavy_ties_at_the_cut():
         assert_build_equal(g, r, "ties k=%d" % k)
 
 
+def test_subnormal_and_nonfinite_thresholds():
+    """The streaming filter switches between a floating-point and an integer compare depending
+    on the threshold: exercise thresholds in the subnormal range and above infinity."""
+    rng = np.random.default_rng(17)
+    tiny = rng.integers(0, 0x0080, size=(64, 4096)).astype(np.uint16)          # zeros and subnormals only
+    tiny ^= (rng.integers(0, 2, size=tiny.shape).astype(np.uint16) << 15)
+    mixed = tiny.copy()
+    mixed[:, ::7] = rng.integers(0x0080, 0x0200, size=mixed[:, ::7].shape).astype(np.uint16)  # small normals
+    wild = rng.integers(0x3000, 0x4400, size=(64, 4096)).astype(np.uint16)
+    spots = rng.random(wild.shape) < 0.002                                      # ~500 NaN/Inf per chunk
+    wild[spots] = rng.integers(0x7F80, 0x8000, size=int(spots.sum())).astype(np.uint16)
+    wild ^= (rng.integers(0, 2, size=wild.shape).astype(np.uint16) << 15)
+    for name, pat in (("subnormal", tiny), ("mixed", mixed), ("nonfinite", wild)):
+        act = from_patterns(pat)
+        for k in (128, 256):
+            g = gpu_build(act, 32, k, 1, 64)
+            r = oracle.build_proofs(pat, 32, k, 1, 64)
+            assert_build_equal(g, r, "%s k=%d" % (name, k))
+
+
 def test_chunk_smaller_than_k_and_nan_patterns():
     pat = np.zeros((3, 40), np.uint16)
     pat[0, 3] = 0xFFF5          # negative NaN pattern >= p
