@@ -36,7 +36,7 @@ constexpr uint32_t kModLow = 32769u;
 // launch shape
 // ---------------------------------------------------------------------------
 #ifndef TOPLOC_SELECT_MIN_BLOCKS
-#define TOPLOC_SELECT_MIN_BLOCKS 15      // select: one-warp blocks per SM (shared memory allows 15)
+#define TOPLOC_SELECT_MIN_BLOCKS 18      // select: one-warp blocks per SM (shared memory allows 18)
 #endif
 #ifndef TOPLOC_SELECT_STAGES
 #define TOPLOC_SELECT_STAGES 2           // select: tiles in flight per warp
@@ -45,8 +45,11 @@ constexpr int kThreads = 32;             // select: one warp per chunk
 constexpr int kUnroll = 4;               // select: 16-byte loads per lane and tile
 constexpr int kStages = TOPLOC_SELECT_STAGES;
 constexpr int kCandCap = 640;            // select: candidate buffer entries (8 bytes each)
-constexpr int kHitCap = 160;             // select: vectors that can be parked between drains
-constexpr int kHitTrigger = 32;          // select: drain once this many are parked
+#ifndef TOPLOC_HIT_TRIGGER
+#define TOPLOC_HIT_TRIGGER 32
+#endif
+constexpr int kHitCap = TOPLOC_HIT_TRIGGER + 128;             // select: vectors that can be parked between drains
+constexpr int kHitTrigger = TOPLOC_HIT_TRIGGER;          // select: drain once this many are parked
 constexpr int kMaxK = TOPLOC_MAX_K;
 constexpr int kMaxSlots = kMaxK / 32;    // tail: entries a lane owns at most
 constexpr int kIdxBits = 24;             // flat index field of a candidate
@@ -103,8 +106,8 @@ __device__ __forceinline__ unsigned long long make_candidate(uint32_t key, uint3
 struct __align__(16) SelectShared {
   uint4 ring[kStages * kUnroll * kThreads];  // tiles on their way from HBM (asynchronous copies)
   unsigned long long cand[kCandCap];  // candidates held; ring + cand later serve as the residue set
-  uint4 hit_vec[kHitCap];             // vectors that passed the streaming filter, not yet unpacked
-  uint32_t hit_idx[kHitCap];          // their vector index within the chunk
+  uint32_t hit_idx[kHitCap];          // vectors that passed the streaming filter, not yet unpacked
+                                      // (index within the chunk; they are fetched again when unpacked)
   uint32_t top_hist[256];             // held candidates by the upper 8 bits of their 15-bit key; a
                                       // compaction borrows it for its digit histograms
   uint32_t low_hist[128];             // those whose upper bits equal top_bin, by the lower 7 bits
@@ -122,7 +125,7 @@ static_assert(sizeof(uint4) * kStages * kUnroll * kThreads + 8 * kCandCap >= 819
 struct WarpState {
   uint32_t thr;  // an element is a candidate iff its key is >= thr
   int count;     // candidates held in sh.cand
-  int nhits;     // vectors parked in sh.hit_vec
+  int nhits;     // vectors parked in sh.hit_idx
 };
 
 // The block is one warp, so a warp barrier orders its shared memory.
@@ -461,19 +464,22 @@ __device__ __noinline__ WarpState select_carefully(SelectShared& sh, const Chunk
 
 // Unpacks the parked hit vectors into candidates (against the current,
 // possibly higher, threshold), one vector per lane and round, then raises the
-// threshold.
-template <int DT, int VEC>
-__device__ __noinline__ WarpState drain_hits(SelectShared& sh, int k, WarpState st) {
+// threshold.  Only the vector's index was parked: the 16 bytes are fetched
+// again (they were read moments ago, so this rarely reaches DRAM).
+template <int DT, int MODE>
+__device__ __noinline__ WarpState drain_hits(SelectShared& sh, const ChunkSource<DT, MODE> src, int k,
+                                             WarpState st) {
+  constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x;
-  warp_barrier();  // the parked vectors are visible
+  warp_barrier();  // the parked indices are visible
   for (int base = 0; base < st.nhits; base += kThreads) {
     const int h = base + lane;
     const bool valid = h < st.nhits;
     uint4 w = make_uint4(0, 0, 0, 0);
     uint32_t v = 0;
     if (valid) {
-      w = sh.hit_vec[h];
       v = sh.hit_idx[h];
+      w = src.load((int)v);
     }
     append_round<DT, VEC>(sh, k, st, w, valid, v * VEC);
   }
@@ -571,7 +577,6 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
       for (int u = 0; u < kUnroll; ++u) {
         if (hit[u]) {
           const int pos = st.nhits + __popc(votes[u] & below);
-          sh.hit_vec[pos] = w[u];
           sh.hit_idx[pos] = (uint32_t)(v0 + u * kThreads + lane);
         }
         st.nhits += __popc(votes[u]);
@@ -579,10 +584,10 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
     }
     request_tile(tile + kStages);  // refill the stage just consumed
     // a tile parks at most kTileVecs vectors, so the buffer cannot overflow
-    if (st.nhits >= kHitTrigger) st = drain_hits<DT, VEC>(sh, k, st);
+    if (st.nhits >= kHitTrigger) st = drain_hits<DT, MODE>(sh, src, k, st);
   }
   if (kRing) copy_async_wait<0>();
-  st = drain_hits<DT, VEC>(sh, k, st);
+  st = drain_hits<DT, MODE>(sh, src, k, st);
   st = select_carefully<DT, MODE>(sh, src, full_end, n_vecs, k, st);
   compact_candidates<DT>(sh, k, st, true);  // exactly k remain
   warp_barrier();
