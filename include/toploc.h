@@ -48,6 +48,11 @@ extern "C" {
 #define TOPLOC_ERR_WORKSPACE (-3)         /* workspace or staging buffer smaller than required */
 #define TOPLOC_ERR_CUDA (-4)              /* a CUDA runtime call or a launch failed */
 #define TOPLOC_ERR_ARCH (-5)              /* current device is not compute capability 10.x */
+#define TOPLOC_ERR_BUILTIN_SCRATCH (-6)   /* batch too large for toploc_build_proofs_builtin_scratch */
+
+/* Size of the scratch buffer built into the library's device image (8 MiB):
+ * enough for 10905 chunks at k = 128 (769 bytes each). */
+#define TOPLOC_BUILTIN_SCRATCH_BYTES (8u << 20)
 
 /* Per-chunk status codes (d_status of build, .status of a verify result). */
 #define TOPLOC_CHUNK_OK 0
@@ -186,6 +191,36 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
                          const toploc_thresholds* thr, toploc_chunk_result* d_results,
                          const int32_t* d_gen_indices_opt, void* d_workspace,
                          size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * toploc_build_proofs for callers that have no way to hand over scratch
+ * memory.  (The paper has no counterpart to this entry point; it exists for
+ * how the library gets embedded.)  Some hosts of this code may not allocate
+ * device memory at the point where proofs are generated: a hook inside a
+ * serving engine whose memory pool is fixed and fully handed out at start-up,
+ * a plug-in that is only given pointers to the engine's tensors, code running
+ * where a cudaMalloc would stall or be refused.  For them the select kernel's
+ * scratch (the selected index / pattern pairs) lives in a buffer of
+ * TOPLOC_BUILTIN_SCRATCH_BYTES that is part of the library itself: every GPU
+ * that loads the library carries it until the process ends, and this call
+ * allocates nothing, on the device or on the host heap.
+ *
+ * Arguments and results are those of toploc_build_proofs, minus the
+ * workspace; the proofs, statuses and indices are bit-identical.  Limits and
+ * rules:
+ *   - toploc_workspace_bytes(lay) must not exceed TOPLOC_BUILTIN_SCRATCH_BYTES,
+ *     else TOPLOC_ERR_BUILTIN_SCRATCH is returned and nothing is enqueued;
+ *   - uniform batches only (seq_offsets == NULL), else TOPLOC_ERR_UNSUPPORTED;
+ *   - the first call on each device looks up the buffer's device address (with
+ *     that device current); make that first call outside any stream capture;
+ *   - all calls on a device share the one buffer, which keeps whatever the
+ *     previous call left in it (nothing in it needs clearing: every entry that
+ *     is read has been written by the same call first).  Two calls whose
+ *     kernels can overlap on the GPU -- different streams, no dependency --
+ *     race on it: keep such calls ordered.
+ */
+int toploc_build_proofs_builtin_scratch(const void* d_act, const toploc_layout* lay, uint8_t* d_proofs,
+                                        uint8_t* d_status, int32_t* d_indices_opt, void* cuda_stream);
 
 /*
  * The same two operations for callers whose data lives in HOST memory

@@ -16,12 +16,13 @@ __all__ = [
     "toploc_num_chunks", "toploc_proof_bytes", "toploc_workspace_bytes", "toploc_staging_bytes",
     "toploc_get_constants", "toploc_status_string", "toploc_error_string",
     "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
-    "toploc_verify_proofs_host",
+    "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES",
 ]
 
 TOPLOC_DTYPE_BF16 = 0
 TOPLOC_DTYPE_FP32 = 1
 TOPLOC_MAX_K = 256
+TOPLOC_BUILTIN_SCRATCH_BYTES = 8 << 20
 
 RESULT_DTYPE = np.dtype([
     ("exp_mismatch", "<u4"), ("n_match", "<u4"), ("mant_diff_sum", "<u4"), ("topk_mismatch", "<i4"),
@@ -86,6 +87,8 @@ def load_library():
     lib.toploc_build_proofs_host.argtypes = [vp, lay_p, vp, vp, vp, sz, vp]
     lib.toploc_verify_proofs_host.restype = ctypes.c_int
     lib.toploc_verify_proofs_host.argtypes = [vp, lay_p, vp, thr_p, vp, vp, sz, vp]
+    lib.toploc_build_proofs_builtin_scratch.restype = ctypes.c_int
+    lib.toploc_build_proofs_builtin_scratch.argtypes = [vp, lay_p, vp, vp, vp, vp]
     _LIB = lib
     return lib
 
@@ -272,3 +275,19 @@ def toploc_verify_proofs_host(act, lay, proofs, thresholds, results, staging, st
             _dev_ptr(staging), staging.numel() * staging.element_size(), _stream_ptr(stream))
     _check(rc, "toploc_verify_proofs_host")
     return results
+
+
+def toploc_build_proofs_builtin_scratch(act, lay, proofs, status, indices=None, stream=None):
+    """Proof generation without a workspace argument: the scratch is a fixed buffer inside the
+    library (TOPLOC_BUILTIN_SCRATCH_BYTES), for embedders that cannot allocate device memory
+    where proofs are made.  This wrapper allocates nothing either: every output tensor must be
+    passed in.  Batches whose scratch need exceeds the buffer, and ragged batches, are refused.
+    Calls share the buffer: keep calls that could overlap on the GPU ordered."""
+    if not act.is_cuda:
+        raise ToplocError("toploc_build_proofs_builtin_scratch needs CUDA tensors")
+    with torch.cuda.device(act.device):
+        rc = load_library().toploc_build_proofs_builtin_scratch(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(proofs), _dev_ptr(status), _dev_ptr(indices),
+            _stream_ptr(stream))
+    _check(rc, "toploc_build_proofs_builtin_scratch")
+    return proofs, status, indices

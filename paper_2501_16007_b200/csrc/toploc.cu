@@ -1086,7 +1086,15 @@ struct DeviceInfo {
   int major;
   int sms;
   bool interp_smem_set;
+  void* builtin_scratch;  // device address of g_builtin_scratch on this device, once looked up
 };
+
+// Scratch for toploc_build_proofs_builtin_scratch: lives in the library's own
+// device image, so every GPU that loads the library holds these bytes until
+// the process exits.  In host code this name is only a handle; the address a
+// kernel can use comes from cudaGetSymbolAddress (see builtin_scratch_address).
+constexpr size_t kBuiltinScratchBytes = TOPLOC_BUILTIN_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
 
 size_t interp_smem_bytes() { return (65536 + (size_t)kInterpWarps * 2 * kMaxK) * sizeof(uint16_t); }
 
@@ -1110,6 +1118,17 @@ int device_info(DeviceInfo** out) {
     d.interp_smem_set = true;
   }
   *out = &d;
+  return TOPLOC_OK;
+}
+
+// Device address of the built-in scratch on the current device (looked up once per device).
+int builtin_scratch_address(DeviceInfo* d, void** out) {
+  if (d->builtin_scratch == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_builtin_scratch) != cudaSuccess || ptr == nullptr) return TOPLOC_ERR_CUDA;
+    d->builtin_scratch = ptr;
+  }
+  *out = d->builtin_scratch;
   return TOPLOC_OK;
 }
 
@@ -1295,6 +1314,8 @@ const char* toploc_error_string(int rc) {
     case TOPLOC_ERR_WORKSPACE: return "workspace or staging buffer too small";
     case TOPLOC_ERR_CUDA: return "CUDA runtime error";
     case TOPLOC_ERR_ARCH: return "device is not compute capability 10.x";
+    case TOPLOC_ERR_BUILTIN_SCRATCH:
+      return "batch needs more scratch than the library's built-in buffer holds (TOPLOC_BUILTIN_SCRATCH_BYTES)";
     default: return "unknown error";
   }
 }
@@ -1352,6 +1373,23 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   const long long blocks = (plan.num_chunks + kVerifyWarps - 1) / kVerifyWarps;
   toploc_evaluate_kernel<<<(unsigned)blocks, kVerifyWarps * 32, 0, stream>>>(sel, io, lay->k, plan.num_chunks);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+}
+
+int toploc_build_proofs_builtin_scratch(const void* d_act, const toploc_layout* lay, uint8_t* d_proofs,
+                                        uint8_t* d_status, int32_t* d_indices_opt, void* cuda_stream) {
+  HostPlan plan;
+  int rc = plan_layout(lay, &plan);
+  if (rc != TOPLOC_OK) return rc;
+  if (plan.ragged) return TOPLOC_ERR_UNSUPPORTED;  // the row table would have to be built on the heap
+  if (plan_workspace(false, plan.num_chunks, lay->k).total > kBuiltinScratchBytes) return TOPLOC_ERR_BUILTIN_SCRATCH;
+  DeviceInfo* dev = nullptr;
+  if ((rc = device_info(&dev)) != TOPLOC_OK) return rc;
+  void* scratch = nullptr;
+  if ((rc = builtin_scratch_address(dev, &scratch)) != TOPLOC_OK) return rc;
+  // Nothing in the scratch has to start at zero: the select kernel writes every
+  // selection and status entry that the interpolation kernel goes on to read.
+  return toploc_build_proofs(d_act, lay, d_proofs, d_status, d_indices_opt, scratch, kBuiltinScratchBytes,
+                             cuda_stream);
 }
 
 // Shared driver of the two host-memory entry points: groups of whole sequences
