@@ -54,7 +54,11 @@ constexpr int kMaxK = TOPLOC_MAX_K;
 constexpr int kMaxSlots = kMaxK / 32;    // tail: entries a lane owns at most
 constexpr int kIdxBits = 24;             // flat index field of a candidate
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
-constexpr int kInterpWarps = 32;         // interpolation kernel: warps (= chunks in flight) per block
+constexpr int kInterpWarps = 32;         // interpolation kernel: warps per block
+#ifndef TOPLOC_INTERP_CHUNKS
+#define TOPLOC_INTERP_CHUNKS 2
+#endif
+constexpr int kInterpChunks = TOPLOC_INTERP_CHUNKS;  // interpolation kernel: chunks a warp works on at once
 constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
 static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
@@ -779,27 +783,42 @@ __device__ __forceinline__ uint32_t left_neighbour(const uint32_t (&v)[S], int s
   return prev;
 }
 
-// Algorithm 3 for the chunks of one warp.  inv[] is the table of inverses in
-// Z_p; xw / aw are this warp's scratch rows (k entries each).
-template <int SLOTS>
-__device__ __forceinline__ void interpolate_chunk(const uint16_t* inv, uint16_t* xw, uint16_t* aw, int k,
-                                                  const uint32_t* idx, const uint16_t* bits, uint32_t m,
-                                                  uint16_t* proof) {
+// Algorithm 3 for NCH chunks of one warp at a time (their dependency chains are
+// independent, which keeps the issue slots of a latency-bound loop filled).
+// inv[] is the table of inverses in Z_p; xw / aw are this warp's scratch rows
+// (NCH x kMaxK entries each).  A chunk that is not live is carried along with
+// zeros and not written.
+template <int SLOTS, int NCH>
+__device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t* xw, uint16_t* aw, int k,
+                                                   const Selection& sel, const long long (&chunk)[NCH],
+                                                   const bool (&live)[NCH]) {
   const int lane = threadIdx.x & 31;
-  uint32_t x[SLOTS], dd[SLOTS];
+  const size_t proof_bytes = 2 + 2 * (size_t)k;
+  uint32_t x[NCH][SLOTS], dd[NCH][SLOTS];
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) {
-    const int j = s * 32 + lane;
-    x[s] = 0;
-    dd[s] = 0;
-    if (j < k) {
-      uint32_t r = idx[j] % m;       // i_m = i mod m, then into Z_p
-      if (r >= kPrime) r -= kPrime;
-      uint32_t y = bits[j];          // "dd <- y mod M"
-      if (y >= kPrime) y -= kPrime;
-      x[s] = r;
-      dd[s] = y;
-      xw[j] = (uint16_t)r;
+  for (int c = 0; c < NCH; ++c) {
+    uint32_t m = 65536u;
+    if (live[c]) {
+      m = reinterpret_cast<const uint16_t*>(sel.proofs + chunk[c] * proof_bytes)[0];
+      if (m == 0) m = 65536u;
+    }
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const int j = s * 32 + lane;
+      x[c][s] = 0;
+      dd[c][s] = 0;
+      if (j < k) {
+        uint32_t r = 0, y = 0;
+        if (live[c]) {
+          r = sel.idx[chunk[c] * k + j] % m;  // i_m = i mod m, then into Z_p
+          if (r >= kPrime) r -= kPrime;
+          y = sel.bits[chunk[c] * k + j];     // "dd <- y mod M"
+          if (y >= kPrime) y -= kPrime;
+        }
+        x[c][s] = r;
+        dd[c][s] = y;
+        xw[c * kMaxK + j] = (uint16_t)r;
+      }
     }
   }
   __syncwarp();
@@ -811,48 +830,68 @@ __device__ __forceinline__ void interpolate_chunk(const uint16_t* inv, uint16_t*
     for (int s = SLOTS - 1; s >= 0; --s) {
       if (s >= s_lo) {
         const int j = s * 32 + lane;
-        const uint32_t prev = left_neighbour<SLOTS>(dd, s, lane, 0u);
         const bool active = j >= level && j < k;
-        const uint32_t span = active ? sub_mod(x[s], xw[j - level]) : 0u;
-        const uint32_t next = mul_mod(sub_mod(dd[s], prev), inv[span]);
-        dd[s] = active ? next : dd[s];
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const uint32_t prev = left_neighbour<SLOTS>(dd[c], s, lane, 0u);
+          const uint32_t span = active ? sub_mod(x[c][s], xw[c * kMaxK + j - level]) : 0u;
+          const uint32_t next = mul_mod(sub_mod(dd[c][s], prev), inv[span]);
+          dd[c][s] = active ? next : dd[c][s];
+        }
       }
     }
   }
   // dd[j] is the Newton coefficient a_j; multiply the Newton form out from the inside:
   //   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) {
-    const int j = s * 32 + lane;
-    if (j < k) aw[j] = (uint16_t)dd[s];
-  }
-  __syncwarp();
-  uint32_t c[SLOTS];
+  for (int c = 0; c < NCH; ++c)
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) c[s] = 0;
-  if (lane == 0) c[0] = aw[k - 1];
+    for (int s = 0; s < SLOTS; ++s) {
+      const int j = s * 32 + lane;
+      if (j < k) aw[c * kMaxK + j] = (uint16_t)dd[c][s];
+    }
+  __syncwarp();
+  uint32_t co[NCH][SLOTS];
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) co[c][s] = 0;
+    if (lane == 0) co[c][0] = aw[c * kMaxK + k - 1];
+  }
 #pragma unroll 1
   for (int i = k - 2; i >= 0; --i) {
-    const uint32_t xi = xw[i];
-    const uint32_t neg_x = xi ? kPrime - xi : 0u;
-    const uint32_t a_i = aw[i];
     const int top = k - 1 - i;  // degree after this step
     const int s_hi = top >> 5;
+    uint32_t neg_x[NCH], a_i[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const uint32_t xi = xw[c * kMaxK + i];
+      neg_x[c] = xi ? kPrime - xi : 0u;
+      a_i[c] = aw[c * kMaxK + i];
+    }
 #pragma unroll
     for (int s = SLOTS - 1; s >= 0; --s) {
       if (s <= s_hi) {
         const int d = s * 32 + lane;
-        const uint32_t prev = left_neighbour<SLOTS>(c, s, lane, a_i);
-        const uint32_t next = mad_mod(c[s], neg_x, prev);
-        c[s] = d <= top ? next : 0u;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const uint32_t prev = left_neighbour<SLOTS>(co[c], s, lane, a_i[c]);
+          const uint32_t next = mad_mod(co[c][s], neg_x[c], prev);
+          co[c][s] = d <= top ? next : 0u;
+        }
       }
     }
   }
   // proof bytes 2 + 2d, 3 + 2d: coefficient of degree d, little-endian
 #pragma unroll
-  for (int s = 0; s < SLOTS; ++s) {
-    const int d = s * 32 + lane;
-    if (d < k) proof[1 + d] = (uint16_t)c[s];
+  for (int c = 0; c < NCH; ++c) {
+    if (!live[c]) continue;
+    uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk[c] * proof_bytes);
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const int d = s * 32 + lane;
+      if (d < k) proof[1 + d] = (uint16_t)co[c][s];
+    }
   }
   __syncwarp();
 }
@@ -860,12 +899,12 @@ __device__ __forceinline__ void interpolate_chunk(const uint16_t* inv, uint16_t*
 // InterpolateModPolynomial() and encode() of Algorithm 1 for every chunk the
 // select kernel finished.  Each block first fills a table of all inverses in
 // Z_p (walking the powers of a generator forwards and backwards), then every
-// warp takes chunks in turn.
+// warp takes chunks in turn, kInterpChunks at a time.
 __global__ void __launch_bounds__(kInterpWarps * 32, 1)
 toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
   extern __shared__ __align__(16) uint16_t dyn_smem[];
   uint16_t* inv = dyn_smem;                               // 65536 entries
-  uint16_t* scratch = dyn_smem + 65536;                   // 2 rows of kMaxK per warp
+  uint16_t* scratch = dyn_smem + 65536;                   // 2 * kInterpChunks rows of kMaxK per warp
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   {
@@ -882,22 +921,29 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
     }
   }
   __syncthreads();
-  uint16_t* xw = scratch + warp * 2 * kMaxK;
-  uint16_t* aw = xw + kMaxK;
-  const size_t proof_bytes = 2 + 2 * (size_t)k;
-  for (long long chunk = (long long)blockIdx.x * kInterpWarps + warp; chunk < num_chunks;
-       chunk += (long long)gridDim.x * kInterpWarps) {
-    const uint8_t st = sel.status[chunk];
-    if (st == TOPLOC_CHUNK_NO_INJECTIVE_MODULUS || st == TOPLOC_CHUNK_K_EXCEEDS_CHUNK) continue;
-    uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_bytes);
-    uint32_t m = proof[0];
-    if (m == 0) m = 65536u;
-    const uint32_t* idx = sel.idx + chunk * k;
-    const uint16_t* bits = sel.bits + chunk * k;
-    if (k <= 32) interpolate_chunk<1>(inv, xw, aw, k, idx, bits, m, proof);
-    else if (k <= 64) interpolate_chunk<2>(inv, xw, aw, k, idx, bits, m, proof);
-    else if (k <= 128) interpolate_chunk<4>(inv, xw, aw, k, idx, bits, m, proof);
-    else interpolate_chunk<kMaxSlots>(inv, xw, aw, k, idx, bits, m, proof);
+  uint16_t* xw = scratch + warp * 2 * kInterpChunks * kMaxK;
+  uint16_t* aw = xw + kInterpChunks * kMaxK;
+  const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
+  for (long long g = (long long)blockIdx.x * kInterpWarps + warp; g < groups;
+       g += (long long)gridDim.x * kInterpWarps) {
+    long long chunk[kInterpChunks];
+    bool live[kInterpChunks];
+    bool any = false;
+#pragma unroll
+    for (int c = 0; c < kInterpChunks; ++c) {
+      chunk[c] = g * kInterpChunks + c;
+      live[c] = false;
+      if (chunk[c] < num_chunks) {
+        const uint8_t st = sel.status[chunk[c]];
+        live[c] = st != TOPLOC_CHUNK_NO_INJECTIVE_MODULUS && st != TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+      }
+      any |= live[c];
+    }
+    if (!any) continue;
+    if (k <= 32) interpolate_chunks<1, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
+    else if (k <= 64) interpolate_chunks<2, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
+    else if (k <= 128) interpolate_chunks<4, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
+    else interpolate_chunks<kMaxSlots, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
   }
 }
 
@@ -1096,7 +1142,7 @@ struct DeviceInfo {
 constexpr size_t kBuiltinScratchBytes = TOPLOC_BUILTIN_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
 
-size_t interp_smem_bytes() { return (65536 + (size_t)kInterpWarps * 2 * kMaxK) * sizeof(uint16_t); }
+size_t interp_smem_bytes() { return (65536 + (size_t)kInterpWarps * 2 * kInterpChunks * kMaxK) * sizeof(uint16_t); }
 
 int device_info(DeviceInfo** out) {
   static DeviceInfo table[64];
@@ -1335,7 +1381,7 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
   rc = run_select(d_act, lay, d_workspace, workspace_bytes, stream, d_status, d_proofs, d_indices_opt, &plan,
                   &sel, &dev);
   if (rc != TOPLOC_OK) return rc;
-  const long long per_wave = kInterpWarps;
+  const long long per_wave = (long long)kInterpWarps * kInterpChunks;
   long long blocks = (plan.num_chunks + per_wave - 1) / per_wave;
   if (blocks > dev->sms) blocks = dev->sms;
   toploc_interpolate_kernel<<<(unsigned)blocks, kInterpWarps * 32, interp_smem_bytes(), stream>>>(
