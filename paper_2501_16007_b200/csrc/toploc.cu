@@ -61,6 +61,7 @@ constexpr int kInterpWarps = 32;         // interpolation kernel: warps per bloc
 constexpr int kInterpChunks = TOPLOC_INTERP_CHUNKS;  // interpolation kernel: chunks a warp works on at once
 constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
+static_assert(kCandCap * 8 >= 8 * kMaxK * 2, "the candidate buffer holds the maxima of the first vectors");
 static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
 static_assert(kHitCap >= kHitTrigger - 1 + kThreads * kUnroll, "a tile's hits must fit below the drain trigger");
 
@@ -492,6 +493,55 @@ __device__ __noinline__ WarpState drain_hits(SelectShared& sh, const ChunkSource
   return st;
 }
 
+// Largest key in one vector, as the 15-bit key the threshold is kept in.
+template <int DT, int VEC>
+__device__ __forceinline__ uint32_t vector_max_coarse_key(const uint4& w) {
+  if (VEC == 1) {
+    return DT == 0 ? (w.x & 0x7FFFu) : ((w.x & 0x7FFFFFFFu) >> 16);
+  } else if (DT == 0) {
+    const uint32_t m = __vmaxu2(__vmaxu2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu),
+                                __vmaxu2(w.z & 0x7FFF7FFFu, w.w & 0x7FFF7FFFu));
+    return max(m & 0xFFFFu, m >> 16);
+  } else {
+    return max(max(w.x & 0x7FFFFFFFu, w.y & 0x7FFFFFFFu), max(w.z & 0x7FFFFFFFu, w.w & 0x7FFFFFFFu)) >> 16;
+  }
+}
+
+// A sound first threshold from the chunk's first n_first vectors (n_first >= k):
+// the k-th largest of their per-vector maxima.  Each maximum is a different
+// element, so at least k elements of the chunk reach it and the k-th largest
+// element cannot lie below it.  Uses the candidate buffer to hold the maxima
+// and leaves the histograms empty again.
+template <int DT, int MODE>
+__device__ __noinline__ uint32_t sound_first_threshold(SelectShared& sh, const ChunkSource<DT, MODE> src,
+                                                       int n_first, int k) {
+  constexpr int VEC = ChunkSource<DT, MODE>::kVec;
+  const int lane = threadIdx.x;
+  uint16_t* maxima = reinterpret_cast<uint16_t*>(sh.cand);
+  warp_barrier();
+#pragma unroll 4
+  for (int v = lane; v < n_first; v += kThreads) {
+    const uint32_t key = vector_max_coarse_key<DT, VEC>(src.load(v));
+    maxima[v] = (uint16_t)key;
+    atomicAdd(&sh.top_hist[key >> 7], 1u);
+  }
+  find_from_top<8>(sh, sh.top_hist, k);
+  const uint32_t top = sh.digit;
+  const int want = sh.want;
+  for (int b = lane; b < 128; b += kThreads) sh.low_hist[b] = 0;
+  warp_barrier();
+  for (int v = lane; v < n_first; v += kThreads) {
+    const uint32_t key = maxima[v];
+    if ((key >> 7) == top) atomicAdd(&sh.low_hist[key & 127u], 1u);
+  }
+  find_from_top<4>(sh, sh.low_hist, want);
+  const uint32_t key = (top << 7) | sh.digit;
+  warp_barrier();
+  for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
+  warp_barrier();
+  return DT == 0 ? key : key << 16;
+}
+
 // Exact top-k of one chunk by one warp: on return sh.cand[0..k) holds the k
 // selected candidates (in no particular order).  n_elems >= k is the caller's
 // business.
@@ -518,8 +568,13 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
   st.count = 0;
   st.nhits = 0;
 
-  // Warm-up: enough elements that afterwards only a minority of vectors hit.
-  const int warm = min(n_vecs, (32 / VEC) * max(k, 128));
+  // Before streaming, a threshold that only a minority of vectors reach.  Large
+  // aligned chunks get it from a look at the maxima of their first vectors
+  // (which are then streamed like everything else); otherwise the first vectors
+  // are selected from directly.
+  const int first = (32 / VEC) * max(k, 128);
+  const bool look_ahead = (MODE != 2) && n_vecs >= first;
+  const int warm = look_ahead ? 0 : min(n_vecs, first);
   const int n_tiles = (n_vecs - warm) / kTileVecs;
   const int full_end = warm + n_tiles * kTileVecs;
 
@@ -543,7 +598,8 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
   for (int t = 0; t < kStages; ++t) request_tile(t);
   warp_barrier();
 
-  st = select_carefully<DT, MODE>(sh, src, 0, warm, k, st);
+  if (look_ahead) st.thr = sound_first_threshold<DT, MODE>(sh, src, first, k);
+  else st = select_carefully<DT, MODE>(sh, src, 0, warm, k, st);
 
   for (int tile = 0; tile < n_tiles; ++tile) {
     const int v0 = warm + tile * kTileVecs;
