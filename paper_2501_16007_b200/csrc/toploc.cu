@@ -17,7 +17,6 @@
 // spend about one instruction per element on the elements that lose.
 #include "toploc.h"
 
-#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -205,22 +204,6 @@ struct ChunkSource {
 // word sit in separate 16-bit lanes, and adding (0x8000 - thr) to a lane sets
 // its top bit exactly when key >= thr (no carry leaves a lane).
 __device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
-
-// The same test for bf16 through the half-precision compare unit: |x| >= t as
-// floating-point numbers orders finite magnitudes exactly like their bit
-// patterns, and the unordered form lets NaN patterns through (a superset is
-// fine here, the unpacking step repeats the test on integers).  Only valid
-// for thresholds that are normal numbers or infinity.
-__device__ __forceinline__ bool bf16_vector_reaches(const uint4& w, uint32_t thr2) {
-  const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(&thr2);
-  const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-  uint32_t any = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-    any |= __hgeu2_mask(__habs2(*reinterpret_cast<const __nv_bfloat162*>(&words[i])), t);
-  return any != 0;
-}
-__device__ __forceinline__ bool bf16_threshold_is_ordinary(uint32_t thr) { return thr >= 0x0080u && thr <= 0x7F80u; }
 
 template <int DT, int VEC>
 __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uint32_t add) {
@@ -585,66 +568,74 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
   // The first tiles are requested before the warm-up starts.
   constexpr bool kRing = (MODE != 2);
   const uint32_t ring_lane = (uint32_t)__cvta_generic_to_shared(&sh.ring[lane]);
-  auto request_tile = [&](int tile) {
+  constexpr uint32_t kStageBytes = kUnroll * kThreads * sizeof(uint4);
+  // stage is a compile-time constant at every call site (the tile loop is unrolled by kStages)
+  auto request_tile = [&](int tile, int stage) {
     if (kRing && tile < n_tiles) {
-      const uint32_t dst = ring_lane + (uint32_t)((tile % kStages) * kUnroll * kThreads * sizeof(uint4));
-      const int v = warm + tile * kTileVecs + lane;
+      const uint32_t dst = ring_lane + (uint32_t)stage * kStageBytes;
+      if (MODE == 0) {
+        const char* g = src.base + ((size_t)(warm + tile * kTileVecs + lane)) * sizeof(uint4);
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u)
-        copy_async_16(dst + (uint32_t)(u * kThreads * sizeof(uint4)), src.address(v + u * kThreads));
+        for (int u = 0; u < kUnroll; ++u)
+          copy_async_16(dst + (uint32_t)(u * kThreads * sizeof(uint4)), g + u * kThreads * sizeof(uint4));
+      } else {
+        const int v = warm + tile * kTileVecs + lane;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          copy_async_16(dst + (uint32_t)(u * kThreads * sizeof(uint4)), src.address(v + u * kThreads));
+      }
     }
     if (kRing) copy_async_commit();
   };
-  for (int t = 0; t < kStages; ++t) request_tile(t);
+#pragma unroll
+  for (int t = 0; t < kStages; ++t) request_tile(t, t);
   warp_barrier();
 
   if (look_ahead) st.thr = sound_first_threshold<DT, MODE>(sh, src, first, k);
   else st = select_carefully<DT, MODE>(sh, src, 0, warm, k, st);
 
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    const int v0 = warm + tile * kTileVecs;
-    uint4 w[kUnroll];
-    if (kRing) {
-      copy_async_wait<kStages - 1>();  // this lane's copies of `tile` have landed
-      const int stage = tile % kStages;
+  for (int tile0 = 0; tile0 < n_tiles; tile0 += kStages) {
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) w[u] = sh.ring[(stage * kUnroll + u) * kThreads + lane];
-    } else {
+    for (int stage = 0; stage < kStages; ++stage) {
+      const int tile = tile0 + stage;
+      if (tile >= n_tiles) break;
+      const int v0 = warm + tile * kTileVecs;
+      uint4 w[kUnroll];
+      if (kRing) {
+        copy_async_wait<kStages - 1>();  // this lane's copies of `tile` have landed
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) w[u] = src.load(v0 + u * kThreads + lane);
-    }
-    const uint32_t add = bf16_lane_add(st.thr);
-    // the tests of a tile's vectors are independent of each other: all of them first,
-    // then the votes, then one warp-uniform branch for the (less common) tile with a hit
-    bool hit[kUnroll];
-    uint32_t votes[kUnroll];
-    uint32_t any_votes = 0;
-    if (DT == 0 && VEC == 8 && bf16_threshold_is_ordinary(st.thr)) {
-      const uint32_t thr2 = st.thr * 0x00010001u;
+        for (int u = 0; u < kUnroll; ++u) w[u] = sh.ring[(stage * kUnroll + u) * kThreads + lane];
+      } else {
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) hit[u] = bf16_vector_reaches(w[u], thr2);
-    } else {
+        for (int u = 0; u < kUnroll; ++u) w[u] = src.load(v0 + u * kThreads + lane);
+      }
+      const uint32_t add = bf16_lane_add(st.thr);
+      // the tests of a tile's vectors are independent of each other: all of them first,
+      // then the votes, then one warp-uniform branch for the (less common) tile with a hit
+      bool hit[kUnroll];
+      uint32_t votes[kUnroll];
+      uint32_t any_votes = 0;
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) hit[u] = vector_reaches<DT, VEC>(w[u], st.thr, add);
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      votes[u] = __ballot_sync(0xFFFFFFFFu, hit[u]);
-      any_votes |= votes[u];
-    }
-    if (any_votes) {
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        if (hit[u]) {
-          const int pos = st.nhits + __popc(votes[u] & below);
-          sh.hit_idx[pos] = (uint32_t)(v0 + u * kThreads + lane);
-        }
-        st.nhits += __popc(votes[u]);
+        votes[u] = __ballot_sync(0xFFFFFFFFu, hit[u]);
+        any_votes |= votes[u];
       }
+      if (any_votes) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+          if (hit[u]) {
+            const int pos = st.nhits + __popc(votes[u] & below);
+            sh.hit_idx[pos] = (uint32_t)(v0 + u * kThreads + lane);
+          }
+          st.nhits += __popc(votes[u]);
+        }
+      }
+      request_tile(tile + kStages, stage);  // refill the stage just consumed
+      // a tile parks at most kTileVecs vectors, so the buffer cannot overflow
+      if (st.nhits >= kHitTrigger) st = drain_hits<DT, MODE>(sh, src, k, st);
     }
-    request_tile(tile + kStages);  // refill the stage just consumed
-    // a tile parks at most kTileVecs vectors, so the buffer cannot overflow
-    if (st.nhits >= kHitTrigger) st = drain_hits<DT, MODE>(sh, src, k, st);
   }
   if (kRing) copy_async_wait<0>();
   st = drain_hits<DT, MODE>(sh, src, k, st);
