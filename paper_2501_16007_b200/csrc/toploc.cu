@@ -210,9 +210,11 @@ __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uin
   if (VEC == 1) {
     return (DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu)) >= thr;
   } else if (DT == 0) {
-    const uint32_t t0 = (w.x & 0x7FFF7FFFu) + add, t1 = (w.y & 0x7FFF7FFFu) + add;
-    const uint32_t t2 = (w.z & 0x7FFF7FFFu) + add, t3 = (w.w & 0x7FFF7FFFu) + add;
-    return (((t0 | t1 | t2) | t3) & 0x80008000u) != 0;
+    // largest key of each 16-bit lane over the four words (three-input packed maximum), then
+    // the add-and-test-top-bit comparison once
+    const uint32_t m = __vimax3_u16x2(__vimax3_u16x2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu, w.z & 0x7FFF7FFFu),
+                                      w.w & 0x7FFF7FFFu, 0u);
+    return ((m + add) & 0x80008000u) != 0;
   } else {
     return max(max(w.x & 0x7FFFFFFFu, w.y & 0x7FFFFFFFu), max(w.z & 0x7FFFFFFFu, w.w & 0x7FFFFFFFu)) >= thr;
   }
