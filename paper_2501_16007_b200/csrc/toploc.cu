@@ -35,15 +35,18 @@ constexpr uint32_t kModLow = 32769u;
 // launch shape
 // ---------------------------------------------------------------------------
 #ifndef TOPLOC_SELECT_MIN_BLOCKS
-#define TOPLOC_SELECT_MIN_BLOCKS 18      // select: one-warp blocks per SM (shared memory allows 18)
+#define TOPLOC_SELECT_MIN_BLOCKS 15      // select: one-warp blocks per SM (shared memory allows 15)
 #endif
 #ifndef TOPLOC_SELECT_STAGES
-#define TOPLOC_SELECT_STAGES 2           // select: tiles in flight per warp
+#define TOPLOC_SELECT_STAGES 3           // select: tiles in flight per warp
 #endif
 constexpr int kThreads = 32;             // select: one warp per chunk
 constexpr int kUnroll = 4;               // select: 16-byte loads per lane and tile
 constexpr int kStages = TOPLOC_SELECT_STAGES;
-constexpr int kCandCap = 640;            // select: candidate buffer entries (8 bytes each)
+#ifndef TOPLOC_CAND_CAP
+#define TOPLOC_CAND_CAP 640
+#endif
+constexpr int kCandCap = TOPLOC_CAND_CAP;            // select: candidate buffer entries (8 bytes each)
 #ifndef TOPLOC_HIT_TRIGGER
 #define TOPLOC_HIT_TRIGGER 32
 #endif
@@ -819,31 +822,28 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
 // lane j % 32, slot j / 32 of that lane.
 // ---------------------------------------------------------------------------
 
-// value of entry j - 1 as seen from entry j (lane 0 takes lane 31 of the slot below)
-template <int S>
-__device__ __forceinline__ uint32_t left_neighbour(const uint32_t (&v)[S], int s, int lane, uint32_t first) {
-  uint32_t prev = __shfl_up_sync(0xFFFFFFFFu, v[s], 1);
-  if (s > 0) {
-    const uint32_t carry = __shfl_sync(0xFFFFFFFFu, v[s > 0 ? s - 1 : 0], 31);
-    if (lane == 0) prev = carry;
-  } else if (lane == 0) {
-    prev = first;
-  }
-  return prev;
-}
-
 // Algorithm 3 for NCH chunks of one warp at a time (their dependency chains are
-// independent, which keeps the issue slots of a latency-bound loop filled).
-// inv[] is the table of inverses in Z_p; xw / aw are this warp's scratch rows
-// (NCH x kMaxK entries each).  A chunk that is not live is carried along with
-// zeros and not written.
+// independent, which keeps the issue slots filled).  inv[] is the table of
+// inverses in Z_p; xw / aw are this warp's scratch rows (NCH x kMaxK entries
+// each).  A chunk that is not live is carried along with zeros and not written.
+//
+// Divided differences are taken point by point instead of level by level (the
+// same table, visited row-wise): with a_0 = y_0, step i lets every later point j
+// do  t_j <- (t_j - a_i) / (x_j - x_i), after which t_{i+1} is the Newton
+// coefficient a_{i+1}.  All points advance together and only a_i and x_i are
+// broadcast, so no value has to travel between neighbouring entries.  Point j
+// lives in lane j % 32, slot j / 32.
+// The Newton form is then multiplied out from the inside,
+//   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0,
+// with coefficient d in lane d / SLOTS, slot d % SLOTS, so that the shift by one
+// degree stays inside a lane except for one value per lane and step.
 template <int SLOTS, int NCH>
 __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t* xw, uint16_t* aw, int k,
                                                    const Selection& sel, const long long (&chunk)[NCH],
                                                    const bool (&live)[NCH]) {
   const int lane = threadIdx.x & 31;
   const size_t proof_bytes = 2 + 2 * (size_t)k;
-  uint32_t x[NCH][SLOTS], dd[NCH][SLOTS];
+  uint32_t x[NCH][SLOTS], t[NCH][SLOTS];
 #pragma unroll
   for (int c = 0; c < NCH; ++c) {
     uint32_t m = 65536u;
@@ -855,7 +855,7 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t
     for (int s = 0; s < SLOTS; ++s) {
       const int j = s * 32 + lane;
       x[c][s] = 0;
-      dd[c][s] = 0;
+      t[c][s] = 0;
       if (j < k) {
         uint32_t r = 0, y = 0;
         if (live[c]) {
@@ -865,70 +865,58 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t
           if (y >= kPrime) y -= kPrime;
         }
         x[c][s] = r;
-        dd[c][s] = y;
+        t[c][s] = y;
         xw[c * kMaxK + j] = (uint16_t)r;
+        if (j == 0) aw[c * kMaxK] = (uint16_t)y;
       }
     }
   }
-  __syncwarp();
-  // divided differences: after level l entry j >= l holds f[x_{j-l}, ..., x_j]
 #pragma unroll 1
-  for (int level = 1; level < k; ++level) {
-    const int s_lo = level >> 5;
+  for (int i = 0; i + 1 < k; ++i) {
+    __syncwarp();  // a_i has been stored
+    uint32_t a_i[NCH], x_i[NCH];
 #pragma unroll
-    for (int s = SLOTS - 1; s >= 0; --s) {
+    for (int c = 0; c < NCH; ++c) {
+      a_i[c] = aw[c * kMaxK + i];
+      x_i[c] = xw[c * kMaxK + i];
+    }
+    const int s_lo = (i + 1) >> 5;
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
       if (s >= s_lo) {
         const int j = s * 32 + lane;
-        const bool active = j >= level && j < k;
+        const bool active = j > i && j < k;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
-          const uint32_t prev = left_neighbour<SLOTS>(dd[c], s, lane, 0u);
-          const uint32_t span = active ? sub_mod(x[c][s], xw[c * kMaxK + j - level]) : 0u;
-          const uint32_t next = mul_mod(sub_mod(dd[c][s], prev), inv[span]);
-          dd[c][s] = active ? next : dd[c][s];
+          const uint32_t span = active ? sub_mod(x[c][s], x_i[c]) : 0u;
+          const uint32_t next = mul_mod(sub_mod(t[c][s], a_i[c]), inv[span]);
+          t[c][s] = active ? next : t[c][s];
+          if (s == s_lo && j == i + 1) aw[c * kMaxK + j] = (uint16_t)next;
         }
       }
     }
   }
-  // dd[j] is the Newton coefficient a_j; multiply the Newton form out from the inside:
-  //   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0
-#pragma unroll
-  for (int c = 0; c < NCH; ++c)
-#pragma unroll
-    for (int s = 0; s < SLOTS; ++s) {
-      const int j = s * 32 + lane;
-      if (j < k) aw[c * kMaxK + j] = (uint16_t)dd[c][s];
-    }
   __syncwarp();
   uint32_t co[NCH][SLOTS];
 #pragma unroll
   for (int c = 0; c < NCH; ++c) {
 #pragma unroll
-    for (int s = 0; s < SLOTS; ++s) co[c][s] = 0;
+    for (int b = 0; b < SLOTS; ++b) co[c][b] = 0;
     if (lane == 0) co[c][0] = aw[c * kMaxK + k - 1];
   }
 #pragma unroll 1
   for (int i = k - 2; i >= 0; --i) {
-    const int top = k - 1 - i;  // degree after this step
-    const int s_hi = top >> 5;
-    uint32_t neg_x[NCH], a_i[NCH];
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
       const uint32_t xi = xw[c * kMaxK + i];
-      neg_x[c] = xi ? kPrime - xi : 0u;
-      a_i[c] = aw[c * kMaxK + i];
-    }
+      const uint32_t neg_x = xi ? kPrime - xi : 0u;
+      const uint32_t a_i = aw[c * kMaxK + i];
+      // coefficient d takes  c[d-1] + (-x_i) c[d];  entries above the current degree are 0 and stay 0
+      uint32_t carry = __shfl_up_sync(0xFFFFFFFFu, co[c][SLOTS - 1], 1);
+      if (lane == 0) carry = a_i;
 #pragma unroll
-    for (int s = SLOTS - 1; s >= 0; --s) {
-      if (s <= s_hi) {
-        const int d = s * 32 + lane;
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-          const uint32_t prev = left_neighbour<SLOTS>(co[c], s, lane, a_i[c]);
-          const uint32_t next = mad_mod(co[c][s], neg_x[c], prev);
-          co[c][s] = d <= top ? next : 0u;
-        }
-      }
+      for (int b = SLOTS - 1; b >= 1; --b) co[c][b] = mad_mod(co[c][b], neg_x, co[c][b - 1]);
+      co[c][0] = mad_mod(co[c][0], neg_x, carry);
     }
   }
   // proof bytes 2 + 2d, 3 + 2d: coefficient of degree d, little-endian
@@ -937,9 +925,9 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t
     if (!live[c]) continue;
     uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk[c] * proof_bytes);
 #pragma unroll
-    for (int s = 0; s < SLOTS; ++s) {
-      const int d = s * 32 + lane;
-      if (d < k) proof[1 + d] = (uint16_t)co[c][s];
+    for (int b = 0; b < SLOTS; ++b) {
+      const int d = lane * SLOTS + b;
+      if (d < k) proof[1 + d] = (uint16_t)co[c][b];
     }
   }
   __syncwarp();
