@@ -136,6 +136,22 @@ def reference_arm(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of a list of per-rank numbers over all ranks (identity for one rank)."""
+    if world <= 1:
+        return list(values)
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_rate(units_per_rank, world, seconds):
+    """Whole-job throughput: every rank processed units_per_rank units, the job took `seconds`
+    (the slowest rank's time)."""
+    return units_per_rank * world / seconds
+
+
 def workload_name(key):
     S, T, H, L, k, seed = WORKLOADS[key]
     return "%s-shaped: %d seq x %d tok, H=%d bf16, L=%d, k=%d" % (
@@ -219,10 +235,7 @@ def main():
     total_ms = start.elapsed_time(stop)
     build_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
     verify_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
-    if world > 1:
-        t = torch.tensor([total_ms, build_ms, verify_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, build_ms, verify_ms = t.tolist()
+    total_ms, build_ms, verify_ms = max_over_ranks([total_ms, build_ms, verify_ms], dev, world)
     ms_per_step = total_ms / args.steps
 
     accepted = int(results.cpu().numpy().view(tl.RESULT_DTYPE)["accept"].sum())
@@ -243,7 +256,7 @@ def main():
     verify_gbs = act_bytes / (verify_ms * 1e-3) / 1e9
     line = {
         "metric": "proof_chunks_per_s_generate_plus_verify",
-        "value": n * world / (ms_per_step * 1e-3), "unit": "chunks/s",
+        "value": aggregate_rate(n, world, ms_per_step * 1e-3), "unit": "chunks/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u16/u32 integer (bf16 bit patterns)", "data": "synthetic",
@@ -300,12 +313,9 @@ def measure_e2e(tl, act, lay, n, k, thr, dev, steps, world):
         step()
     torch.cuda.synchronize()
     dt = (time.perf_counter() - t0) / steps
-    if world > 1:
-        t = torch.tensor([dt], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = t.item()
+    dt = max_over_ranks([dt], dev, world)[0]
     proofs_b = n * (2 + 2 * k)
-    return {"value": n * world / dt, "unit": "chunks/s", "ms_per_step": dt * 1e3, "steps": steps,
+    return {"value": aggregate_rate(n, world, dt), "unit": "chunks/s", "ms_per_step": dt * 1e3, "steps": steps,
             "h2d_bytes_per_step": 2 * act_bytes + proofs_b, "d2h_bytes_per_step": proofs_b + n + n * 40,
             "note": "build then verify (identical copy) from pinned host memory; PCIe-bound"}
 
