@@ -193,6 +193,24 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
                          size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The selection step on its own: topk(h, k) of Algorithms 1 and 2 for every
+ * chunk (Section 5.5 describes the engine-side hook as obtaining exactly
+ * this: the top-k values of the last hidden layer).  Same ranking as above:
+ * magnitude key, ties to the lower flat index.
+ *
+ * d_sel_indices         DEVICE out, [num_chunks, k] u32: the selected flat indices of each
+ *                       chunk, as a set (order within a chunk is unspecified)
+ * d_sel_patterns        DEVICE out, [num_chunks, k] u16: their 16-bit patterns, same order
+ * d_status              DEVICE out, [num_chunks]: TOPLOC_CHUNK_OK or K_EXCEEDS_CHUNK (whose rows
+ *                       of the two arrays above are left untouched)
+ * d_ranked_indices_opt  DEVICE out, optional: [num_chunks, k] i32 indices in rank order
+ * other arguments as for toploc_build_proofs.  Asynchronous.
+ */
+int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_sel_indices,
+                       uint16_t* d_sel_patterns, uint8_t* d_status, int32_t* d_ranked_indices_opt,
+                       void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * toploc_build_proofs for callers that have no way to hand over scratch
  * memory.  (The paper has no counterpart to this entry point; it exists for
  * how the library gets embedded.)  Some hosts of this code may not allocate

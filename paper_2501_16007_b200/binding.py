@@ -16,7 +16,7 @@ __all__ = [
     "toploc_num_chunks", "toploc_proof_bytes", "toploc_workspace_bytes", "toploc_staging_bytes",
     "toploc_get_constants", "toploc_status_string", "toploc_error_string",
     "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
-    "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES",
+    "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES", "toploc_select_topk",
 ]
 
 TOPLOC_DTYPE_BF16 = 0
@@ -87,6 +87,8 @@ def load_library():
     lib.toploc_build_proofs_host.argtypes = [vp, lay_p, vp, vp, vp, sz, vp]
     lib.toploc_verify_proofs_host.restype = ctypes.c_int
     lib.toploc_verify_proofs_host.argtypes = [vp, lay_p, vp, thr_p, vp, vp, sz, vp]
+    lib.toploc_select_topk.restype = ctypes.c_int
+    lib.toploc_select_topk.argtypes = [vp, lay_p, vp, vp, vp, vp, vp, sz, vp]
     lib.toploc_build_proofs_builtin_scratch.restype = ctypes.c_int
     lib.toploc_build_proofs_builtin_scratch.argtypes = [vp, lay_p, vp, vp, vp, vp]
     _LIB = lib
@@ -291,3 +293,29 @@ def toploc_build_proofs_builtin_scratch(act, lay, proofs, status, indices=None, 
             _stream_ptr(stream))
     _check(rc, "toploc_build_proofs_builtin_scratch")
     return proofs, status, indices
+
+
+def toploc_select_topk(act, lay, sel_indices=None, sel_patterns=None, status=None, ranked_indices=None,
+                       workspace=None, stream=None, want_ranked=False):
+    """The selection step alone.  Returns (sel_indices int32-viewable uint32 [n, k] as an int32
+    tensor, sel_patterns int16 tensor holding the 16-bit patterns [n, k], status uint8 [n],
+    ranked_indices int32 [n, k] or None)."""
+    if not act.is_cuda:
+        raise ToplocError("toploc_select_topk needs a CUDA tensor")
+    n = toploc_num_chunks(lay)
+    dev = act.device
+    if sel_indices is None:
+        sel_indices = torch.empty((n, lay.k), dtype=torch.int32, device=dev)
+    if sel_patterns is None:
+        sel_patterns = torch.empty((n, lay.k), dtype=torch.int16, device=dev)
+    if status is None:
+        status = torch.empty((n,), dtype=torch.uint8, device=dev)
+    if ranked_indices is None and want_ranked:
+        ranked_indices = torch.empty((n, lay.k), dtype=torch.int32, device=dev)
+    workspace, wbytes = _workspace(lay, workspace, dev)
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_select_topk(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(sel_indices), _dev_ptr(sel_patterns), _dev_ptr(status),
+            _dev_ptr(ranked_indices), _dev_ptr(workspace), wbytes, _stream_ptr(stream))
+    _check(rc, "toploc_select_topk")
+    return sel_indices, sel_patterns, status, ranked_indices

@@ -1278,7 +1278,8 @@ void launch_select(int mode, unsigned grid, cudaStream_t stream, const BatchPara
 // Common front half of both entry points: checks, scratch carving, row table, select kernel.
 int run_select(const void* d_act, const toploc_layout* lay, void* d_workspace, size_t workspace_bytes,
                cudaStream_t stream, uint8_t* d_status_or_null, uint8_t* d_proofs_or_null,
-               int32_t* d_indices_opt, HostPlan* plan, Selection* sel, DeviceInfo** dev) {
+               int32_t* d_indices_opt, HostPlan* plan, Selection* sel, DeviceInfo** dev,
+               uint32_t* d_sel_idx_or_null = nullptr, uint16_t* d_sel_bits_or_null = nullptr) {
   int rc = device_info(dev);
   if (rc != TOPLOC_OK) return rc;
   const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k);
@@ -1298,8 +1299,8 @@ int run_select(const void* d_act, const toploc_layout* lay, void* d_workspace, s
     if ((rc = upload_spans(lay, *plan, ws + wp.spans_off, stream)) != TOPLOC_OK) return rc;
     bp.spans = reinterpret_cast<const ChunkSpan*>(ws + wp.spans_off);
   }
-  sel->idx = reinterpret_cast<uint32_t*>(ws + wp.idx_off);
-  sel->bits = reinterpret_cast<uint16_t*>(ws + wp.bits_off);
+  sel->idx = d_sel_idx_or_null ? d_sel_idx_or_null : reinterpret_cast<uint32_t*>(ws + wp.idx_off);
+  sel->bits = d_sel_bits_or_null ? d_sel_bits_or_null : reinterpret_cast<uint16_t*>(ws + wp.bits_off);
   sel->status = d_status_or_null ? d_status_or_null : reinterpret_cast<uint8_t*>(ws + wp.status_off);
   sel->proofs = d_proofs_or_null;
   sel->indices = d_indices_opt;
@@ -1456,6 +1457,23 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   const long long blocks = (plan.num_chunks + kVerifyWarps - 1) / kVerifyWarps;
   toploc_evaluate_kernel<<<(unsigned)blocks, kVerifyWarps * 32, 0, stream>>>(sel, io, lay->k, plan.num_chunks);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+}
+
+int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_sel_indices,
+                       uint16_t* d_sel_patterns, uint8_t* d_status, int32_t* d_ranked_indices_opt,
+                       void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+  HostPlan plan;
+  int rc = plan_layout(lay, &plan);
+  if (rc != TOPLOC_OK) return rc;
+  if (d_act == nullptr || d_sel_indices == nullptr || d_sel_patterns == nullptr || d_status == nullptr)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(d_sel_indices) % 4 != 0 || reinterpret_cast<uintptr_t>(d_sel_patterns) % 2 != 0)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (plan.num_chunks == 0) return TOPLOC_OK;
+  Selection sel;
+  DeviceInfo* dev = nullptr;
+  return run_select(d_act, lay, d_workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream), d_status,
+                    nullptr, d_ranked_indices_opt, &plan, &sel, &dev, d_sel_indices, d_sel_patterns);
 }
 
 int toploc_build_proofs_builtin_scratch(const void* d_act, const toploc_layout* lay, uint8_t* d_proofs,

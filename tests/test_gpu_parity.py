@@ -153,6 +153,23 @@ def test_malformed_proofs_are_reported_not_trusted():
     assert gv["status"].tolist() == [3, 3]
 
 
+def test_selection_entry_point_matches_the_oracle_topk():
+    act = synth.make_activations(2, 96, 4096, torch.bfloat16, seed=41, device=DEV, outliers="jitter")
+    lay, _ = tl.make_layout(act, 32, 128, 2, 96)
+    idx, pat, status, ranked = tl.toploc_select_topk(act, lay, want_ranked=True)
+    torch.cuda.synchronize()
+    host = synth.host_patterns(act)
+    idx, pat, ranked = idx.cpu().numpy(), pat.cpu().numpy().view(np.uint16), ranked.cpu().numpy()
+    assert not status.any().item()
+    for c in range(6):
+        want_idx, want_bits = oracle.topk(host[c * 32:(c + 1) * 32], 128)
+        assert ranked[c].tolist() == want_idx.tolist()
+        order = np.argsort(idx[c])
+        ref = np.argsort(want_idx)
+        assert idx[c][order].tolist() == want_idx[ref].tolist()           # same set ...
+        assert pat[c][order].tolist() == want_bits[ref].tolist()          # ... with the same values
+
+
 def test_sign_bit_reading_switch():
     act = synth.make_activations(1, 64, 4096, torch.bfloat16, seed=6, device=DEV)
     other = synth.make_activations(1, 64, 4096, torch.bfloat16, seed=1006, device=DEV)
