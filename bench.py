@@ -171,6 +171,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time the parameter sweep (k x chunk length x H x dtype) instead of the main workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -190,6 +192,11 @@ def main():
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
+
+    if args.sweep:
+        if rank == 0:
+            print(json.dumps(sweep(tl, synth, dev)), flush=True)
+        return
 
     S, T, H, L, k, seed = WORKLOADS[args.workload]
     act = synth.make_activations(S, T, H, torch.bfloat16, seed=seed + 10007 * rank, device=dev)
@@ -306,6 +313,51 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def sweep(tl, synth, dev, reps=5):
+    """k in {32, 64, 128, 256} x chunk length in {16, 32, 64} x H in {2048, 4096, 8192} x {bf16, fp32},
+    128 sequences x 1024 tokens each: generate and verify times per point (CUDA events, mean of reps)."""
+    peak, peak_kind = measured_hbm_peak()
+    S, T = 128, 1024
+    points = []
+    for dtype, name in ((torch.bfloat16, "bf16"), (torch.float32, "fp32")):
+        for H in (2048, 4096, 8192):
+            act = synth.make_activations(S, T, H, dtype, seed=50 + H // 1024, device=dev)
+            rec = synth.honest_noise(act, seed=9)
+            nbytes = act.numel() * act.element_size()
+            for L in (16, 32, 64):
+                for k in (32, 64, 128, 256):
+                    lay, _ = tl.make_layout(act, L, k, S, T)
+                    n = tl.toploc_num_chunks(lay)
+                    proofs = torch.empty((n, 2 + 2 * k), dtype=torch.uint8, device=dev)
+                    status = torch.empty((n,), dtype=torch.uint8, device=dev)
+                    results = torch.empty((n, 40), dtype=torch.uint8, device=dev)
+                    ws = torch.empty(tl.toploc_workspace_bytes(lay), dtype=torch.uint8, device=dev)
+                    thr = tl.default_thresholds(k)
+
+                    def timed(fn):
+                        for _ in range(2):
+                            fn()
+                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a.record()
+                        for _ in range(reps):
+                            fn()
+                        b.record()
+                        torch.cuda.synchronize()
+                        return a.elapsed_time(b) / reps
+
+                    g = timed(lambda: tl.toploc_build_proofs(act, lay, proofs, status, workspace=ws))
+                    v = timed(lambda: tl.toploc_verify_proofs(rec, lay, proofs, thr, results, workspace=ws))
+                    acc = int(results.cpu().numpy().view(tl.RESULT_DTYPE)["accept"].sum())
+                    points.append({"dtype": name, "H": H, "L": L, "k": k, "chunks": n,
+                                   "generate_ms": round(g, 4), "verify_ms": round(v, 4),
+                                   "generate_chunks_per_s": round(n / g * 1e3), "verify_chunks_per_s": round(n / v * 1e3),
+                                   "generate_frac_of_peak": round(nbytes / g / 1e6 / peak, 3),
+                                   "verify_frac_of_peak": round(nbytes / v / 1e6 / peak, 3), "accepted": acc})
+            del act, rec
+    return {"metric": "sweep", "peak_GB_per_s": peak, "peak_kind": peak_kind, "unit": "fraction of HBM peak",
+            "batch": "%d sequences x %d tokens" % (S, T), "points": points}
 
 
 def measure_e2e(tl, act, lay, n, k, thr, dev, steps, world):
