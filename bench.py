@@ -130,7 +130,7 @@ def reference_arm(args, rank):
         "impl": "reference", "metric": "proof_chunks_per_s_generate_plus_verify", "value": value,
         "unit": "chunks/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u16/u32 integer (bf16 bit patterns)", "data": "synthetic",
+        "dtype": "u32", "data": "synthetic",
         "config": {"workload": workload_name(args.workload), "sample": "first sequence (%d chunks) per step" % chunks},
         "cpu_baseline": {"value": value, "unit": "chunks/s", "cores": cores, "kind": "oracle",
                          "sample": "first sequence: %d chunks of %d x %d bf16, build + verify" % (chunks, L, H)},
@@ -285,7 +285,7 @@ def main():
         "value": aggregate_rate(n, world, ms_per_step * 1e-3), "unit": "chunks/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u16/u32 integer (bf16 bit patterns)", "data": "synthetic",
+        "dtype": "u32", "data": "synthetic",
         "config": {"workload": workload_name(args.workload), "chunks": n, "proof_bytes": 2 + 2 * k,
                    "activation_bytes": act_bytes, "l2": "inputs larger than L2 (no flush needed)",
                    "recomputed": "honest reorder noise, relative 2^-8", "parallelism": "chunks sharded, no collective"},
