@@ -1,10 +1,11 @@
 // TopLoc proof hot path for sm_100a.
 //
 // Two kernels per call:
-//   select   one 128-thread block per chunk streams the chunk from HBM exactly
-//            once and keeps the exact top-k on chip (Algorithm 1 / 2, topk());
-//            for proof generation it also runs the injective-modulus search
-//            (Algorithm 6).  The k (index, pattern) pairs go to scratch memory.
+//   select   one warp (a 32-thread block) per chunk streams the chunk from HBM
+//            exactly once and keeps the exact top-k on chip (Algorithm 1 / 2,
+//            topk()); for proof generation it also runs the injective-modulus
+//            search (Algorithm 6).  The k (index, pattern) pairs go to scratch
+//            memory.
 //   tail     one warp per chunk does the arithmetic over Z_p: Newton
 //            interpolation and packing (Algorithm 3, proof generation) or
 //            Horner evaluation, bit-field comparison, statistics and verdict
@@ -12,9 +13,10 @@
 //
 // The path is a selection over data read once plus integer modular arithmetic:
 // HBM bandwidth is the roofline, there is no dense contraction and therefore no
-// tensor-core work.  The select kernel is built to keep many 16-byte loads in
-// flight per SM (small blocks, many per SM, software-pipelined tiles) and to
-// spend about one instruction per element on the elements that lose.
+// tensor-core work.  The select kernel keeps its loads in flight as
+// asynchronous copies into a small shared-memory ring per warp (many
+// independent warps per SM, none waits on another) and spends about one
+// instruction per five elements on the elements that lose.
 #include "toploc.h"
 
 #include <cuda_runtime.h>
@@ -46,12 +48,12 @@ constexpr int kStages = TOPLOC_SELECT_STAGES;
 #ifndef TOPLOC_CAND_CAP
 #define TOPLOC_CAND_CAP 640
 #endif
-constexpr int kCandCap = TOPLOC_CAND_CAP;            // select: candidate buffer entries (8 bytes each)
+constexpr int kCandCap = TOPLOC_CAND_CAP;  // select: candidate buffer entries (8 bytes each)
 #ifndef TOPLOC_HIT_TRIGGER
 #define TOPLOC_HIT_TRIGGER 32
 #endif
-constexpr int kHitCap = TOPLOC_HIT_TRIGGER + 128;             // select: vectors that can be parked between drains
-constexpr int kHitTrigger = TOPLOC_HIT_TRIGGER;          // select: drain once this many are parked
+constexpr int kHitCap = TOPLOC_HIT_TRIGGER + 128;  // select: vectors that can be parked between drains
+constexpr int kHitTrigger = TOPLOC_HIT_TRIGGER;    // select: drain once this many are parked
 constexpr int kMaxK = TOPLOC_MAX_K;
 constexpr int kMaxSlots = kMaxK / 32;    // tail: entries a lane owns at most
 constexpr int kIdxBits = 24;             // flat index field of a candidate
