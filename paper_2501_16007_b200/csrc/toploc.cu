@@ -63,6 +63,8 @@ constexpr int kInterpWarps = 32;         // interpolation kernel: warps per bloc
 #define TOPLOC_INTERP_CHUNKS 2
 #endif
 constexpr int kInterpChunks = TOPLOC_INTERP_CHUNKS;  // interpolation kernel: chunks a warp works on at once
+static_assert((65536 + kInterpWarps * 2 * kInterpChunks * TOPLOC_MAX_K) * 2 <= 227 * 1024,
+              "table of inverses + per-warp rows must fit the shared memory of one block");
 constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
 static_assert(kCandCap * 8 >= 8 * kMaxK * 2, "the candidate buffer holds the maxima of the first vectors");
