@@ -204,6 +204,36 @@ def test_host_buffer_entry_points_match_device_ones():
         tl.toploc_build_proofs_host(h_act, lay, h_proofs, h_status, small)
 
 
+def test_host_detected_errors_leave_nothing_enqueued():
+    """Bad arguments come back as error codes before any launch: a workspace that is too small or
+    misaligned, an odd proof pointer, a negative threshold."""
+    import ctypes
+    act = synth.make_activations(1, 64, 1024, torch.bfloat16, seed=2, device=DEV)
+    lay, _ = tl.make_layout(act, 32, 32, 1, 64)
+    n = tl.toploc_num_chunks(lay)
+    need = tl.toploc_workspace_bytes(lay)
+    proofs = torch.zeros((n, 66), dtype=torch.uint8, device=DEV)
+    status = torch.full((n,), 77, dtype=torch.uint8, device=DEV)
+    small = torch.empty(need - 1, dtype=torch.uint8, device=DEV)
+    with pytest.raises(tl.ToplocError, match="workspace"):
+        tl.toploc_build_proofs(act, lay, proofs, status, workspace=small)
+    big = torch.empty(need + 64, dtype=torch.uint8, device=DEV)
+    with pytest.raises(tl.ToplocError, match="invalid argument"):
+        tl.toploc_build_proofs(act, lay, proofs, status, workspace=big[8:])          # not 16-byte aligned
+    lib = tl.load_library()
+    odd = ctypes.c_void_p(proofs.data_ptr() + 1)
+    rc = lib.toploc_build_proofs(ctypes.c_void_p(act.data_ptr()), ctypes.byref(lay), odd,
+                                 ctypes.c_void_p(status.data_ptr()), None, ctypes.c_void_p(big.data_ptr()),
+                                 need, None)
+    assert rc == -1
+    thr = tl.default_thresholds(32)
+    thr.t_exp = -1
+    with pytest.raises(tl.ToplocError, match="invalid argument"):
+        tl.toploc_verify_proofs(act, lay, proofs, thr)
+    torch.cuda.synchronize()
+    assert (status == 77).all().item() and not proofs.any().item()                   # nothing ran
+
+
 # ------------------------------------------------------------------ the named configurations
 
 def test_config_tiny():
