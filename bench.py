@@ -35,7 +35,7 @@ WORKLOADS = {
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one toploc_select_kernel launch on the full
 # batch (ncu, profiles/launch_list_70b_shape.md); None where no capture of the current kernel exists
-SELECT_DRAM_BYTES_PER_LAUNCH = {"70b": 17483756288 + 25687501}
+SELECT_DRAM_BYTES_PER_LAUNCH = {"70b": 17475660032 + 25806822}
 
 
 def measured_hbm_peak():
@@ -302,8 +302,8 @@ def main():
                      "traffic": SELECT_DRAM_BYTES_PER_LAUNCH.get(args.workload),
                      "frac_of_8TBs_nominal": select_gbs / 8000.0},
         "roofline_calls": {"generate_frac_of_peak": build_gbs / peak, "verify_frac_of_peak": verify_gbs / peak,
-                           "note": "whole calls: select + arithmetic kernels"},
-        "gpu_launches": 4 * args.steps + sel_steps,
+                           "note": "whole calls: generate = select + interpolate kernels, verify = one kernel"},
+        "gpu_launches": 3 * args.steps + sel_steps,  # build: select + interpolate; verify: one kernel
         "clocks": clocks,
         "checks": {"accepted_chunks": accepted, "chunks_with_status": bad_status},
         "e2e": e2e,

@@ -1,22 +1,24 @@
 // TopLoc proof hot path for sm_100a.
 //
-// Two kernels per call:
-//   select   one warp (a 32-thread block) per chunk streams the chunk from HBM
-//            exactly once and keeps the exact top-k on chip (Algorithm 1 / 2,
-//            topk()); for proof generation it also runs the injective-modulus
-//            search (Algorithm 6).  The k (index, pattern) pairs go to scratch
-//            memory.
-//   tail     one warp per chunk does the arithmetic over Z_p: Newton
-//            interpolation and packing (Algorithm 3, proof generation) or
-//            Horner evaluation, bit-field comparison, statistics and verdict
-//            (Algorithms 5 and 2, validation).
+// Proof generation, two kernels per call:
+//   select        one warp (a 32-thread block) per chunk streams the chunk from
+//                 HBM exactly once and keeps the exact top-k on chip (Algorithm 1,
+//                 topk()), then runs the injective-modulus search (Algorithm 6).
+//                 The k (index, pattern) pairs go to scratch memory.
+//   interpolate   one warp per chunk does the arithmetic over Z_p: Newton
+//                 interpolation and packing (Algorithm 3).
+// Validation, one kernel per call:
+//   verify        the same selection (Algorithm 2, topk()), after which the same
+//                 warp evaluates the committed polynomial at its k points
+//                 (Algorithm 5), compares bit fields, and writes statistics and
+//                 verdict.  Nothing goes through scratch memory.
 //
 // The path is a selection over data read once plus integer modular arithmetic:
 // HBM bandwidth is the roofline, there is no dense contraction and therefore no
-// tensor-core work.  The select kernel keeps its loads in flight as
-// asynchronous copies into a small shared-memory ring per warp (many
-// independent warps per SM, none waits on another) and spends about one
-// instruction per five elements on the elements that lose.
+// tensor-core work.  The selection keeps its loads in flight as asynchronous
+// copies into a small shared-memory ring per warp (many independent warps per
+// SM, none waits on another) and spends about one instruction per five
+// elements on the elements that lose.
 #include "toploc.h"
 
 #include <cuda_runtime.h>
@@ -65,7 +67,6 @@ constexpr int kInterpWarps = 32;         // interpolation kernel: warps per bloc
 constexpr int kInterpChunks = TOPLOC_INTERP_CHUNKS;  // interpolation kernel: chunks a warp works on at once
 static_assert((65536 + kInterpWarps * 2 * kInterpChunks * TOPLOC_MAX_K) * 2 <= 227 * 1024,
               "table of inverses + per-warp rows must fit the shared memory of one block");
-constexpr int kVerifyWarps = 8;          // evaluation kernel: warps per block
 
 static_assert(kCandCap * 8 >= 8 * kMaxK * 2, "the candidate buffer holds the maxima of the first vectors");
 static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
@@ -88,7 +89,7 @@ struct BatchParams {
   int chunks_per_seq;
 };
 
-// What the select kernel leaves behind for the tail kernel.
+// What the select kernel leaves behind for the interpolation kernel (or hands to the caller).
 struct Selection {
   uint32_t* idx;       // [num_chunks, k] selected flat indices
   uint16_t* bits;      // [num_chunks, k] their 16-bit patterns
@@ -787,7 +788,7 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
   src.vecs_per_row = bp.hidden / ChunkSource<DT, MODE>::kVec;
   select_topk<DT, MODE>(sh, src, (int)n_elems, k);
 
-  // hand the selection to the tail kernel; rank order only where the caller asked for indices
+  // hand the selection to the interpolation kernel; rank order only where the caller asked for indices
   uint32_t unrepresentable = 0;
   for (int j = tid; j < k; j += kThreads) {
     const unsigned long long cj = sh.cand[j];
@@ -822,8 +823,8 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
 }
 
 // ---------------------------------------------------------------------------
-// tail kernels: one warp per chunk.  Entry j of a chunk's k points belongs to
-// lane j % 32, slot j / 32 of that lane.
+// arithmetic over Z_p, one warp per chunk.  Entry j of a chunk's k points
+// belongs to lane j % 32, slot j / 32 of that lane.
 // ---------------------------------------------------------------------------
 
 // Algorithm 3 for NCH chunks of one warp at a time (their dependency chains are
@@ -988,84 +989,62 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
   }
 }
 
-struct VerifyWarpShared {
-  uint16_t coef[kMaxK];
-  uint32_t gen[kMaxK];
-  uint32_t hist[128];  // a 7-bit mantissa difference is at most 127
-};
-
 // decode(), Horner evaluation (Algorithm 5), extractBits(), the error
-// accumulation and the verdict of Algorithm 2, one warp per chunk.
-__global__ void __launch_bounds__(kVerifyWarps * 32)
-toploc_evaluate_kernel(Selection sel, VerifyIo io, int k, long long num_chunks) {
-  __shared__ VerifyWarpShared wsh[kVerifyWarps];
-  const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
-  const long long chunk = (long long)blockIdx.x * kVerifyWarps + warp;
-  if (chunk >= num_chunks) return;
-  VerifyWarpShared& ws = wsh[warp];
+// accumulation and the verdict of Algorithm 2 for one chunk, by the warp that
+// selected it.  res arrives initialised and with the decoded modulus.
+template <int SLOTS>
+__device__ __forceinline__ void evaluate_warp(SelectShared& sh, int k, long long chunk, const uint32_t (&idx)[SLOTS],
+                                              const uint32_t (&bits)[SLOTS], const VerifyIo& io,
+                                              toploc_chunk_result res) {
+  const int lane = threadIdx.x;
   const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 2 * (size_t)k));
-
-  toploc_chunk_result res;
-  res.exp_mismatch = 0;
-  res.n_match = 0;
-  res.mant_diff_sum = 0;
-  res.topk_mismatch = -1;
-  res.mant_mean = 0.0;
-  res.mant_median = 0.0;
-  res.accept = 0;
-  res.status = TOPLOC_CHUNK_OK;
-  res.pad[0] = res.pad[1] = 0;
-
-  uint32_t m = proof[0];
-  if (m == 0) m = 65536u;
-  res.modulus = m;
-  uint32_t bad = (m < kModLow || m > kModHigh);
-  for (int d = lane; d < k; d += 32) {
-    const uint16_t cd = proof[1 + d];
-    ws.coef[d] = cd;
-    bad |= cd >= kPrime;
-  }
-  if (__any_sync(0xFFFFFFFFu, bad != 0)) {
-    res.status = TOPLOC_CHUNK_BAD_PROOF;
-    if (lane == 0) io.results[chunk] = res;
-    return;
-  }
-  if (sel.status[chunk] != TOPLOC_CHUNK_OK) {
-    res.status = sel.status[chunk];
-    if (lane == 0) io.results[chunk] = res;
-    return;
-  }
+  // the selection has left shared memory (it is in idx / bits), so the ring is free
+  uint32_t* coef = reinterpret_cast<uint32_t*>(sh.ring);  // kMaxK words
+  uint32_t* gen = coef + kMaxK;                           // kMaxK words
+  uint32_t* hist = sh.top_hist;                           // a 7-bit mantissa difference is at most 127
+  warp_barrier();
+  for (int d = lane; d < k; d += 32) coef[d] = proof[1 + d];
   if (io.gen_indices)
-    for (int j = lane; j < k; j += 32) ws.gen[j] = (uint32_t)io.gen_indices[chunk * k + j];
-  for (int b = lane; b < 128; b += 32) ws.hist[b] = 0;
-  __syncwarp();
+    for (int j = lane; j < k; j += 32) gen[j] = (uint32_t)io.gen_indices[chunk * k + j];
+  for (int b = lane; b < 128; b += 32) hist[b] = 0;
+  warp_barrier();
 
-  uint32_t err_e = 0, diff_sum = 0, common = 0;
-  for (int j = lane; j < k; j += 32) {
-    const uint32_t flat = sel.idx[chunk * k + j];
-    const uint32_t seen = sel.bits[chunk * k + j];
-    uint32_t x = flat % m;
-    if (x >= kPrime) x -= kPrime;
-    uint32_t acc = ws.coef[k - 1];  // Horner, highest degree first
+  const uint32_t m = res.modulus;
+  uint32_t x[SLOTS], acc[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    uint32_t r = idx[s] % m;
+    if (r >= kPrime) r -= kPrime;
+    x[s] = r;
+    acc[s] = coef[k - 1];  // Horner, highest degree first
+  }
 #pragma unroll 4
-    for (int d = k - 2; d >= 0; --d) acc = mad_mod(acc, x, ws.coef[d]);
-    uint32_t e_p = acc >> 7, e_v = seen >> 7;  // sign + 8 exponent bits
+  for (int d = k - 2; d >= 0; --d) {
+    const uint32_t cd = coef[d];
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) acc[s] = mad_mod(acc[s], x[s], cd);
+  }
+  uint32_t err_e = 0, diff_sum = 0, common = 0;
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    if (s * 32 + lane >= k) continue;
+    const uint32_t seen = bits[s];
+    uint32_t e_p = acc[s] >> 7, e_v = seen >> 7;  // sign + 8 exponent bits
     if (!io.sign_in_exponent) {
       e_p &= 0xFFu;
       e_v &= 0xFFu;
     }
     if (e_p == e_v) {
-      int diff = (int)(acc & 0x7Fu) - (int)(seen & 0x7Fu);
+      int diff = (int)(acc[s] & 0x7Fu) - (int)(seen & 0x7Fu);
       diff = diff < 0 ? -diff : diff;
-      atomicAdd(&ws.hist[diff], 1u);
+      atomicAdd(&hist[diff], 1u);
       diff_sum += (uint32_t)diff;
     } else {
       ++err_e;
     }
     if (io.gen_indices) {
       uint32_t hit = 0;
-      for (int i = 0; i < k; ++i) hit |= ws.gen[i] == flat;
+      for (int i = 0; i < k; ++i) hit |= gen[i] == idx[s];
       common += hit;
     }
   }
@@ -1075,13 +1054,13 @@ toploc_evaluate_kernel(Selection sel, VerifyIo io, int k, long long num_chunks) 
     diff_sum += __shfl_xor_sync(0xFFFFFFFFu, diff_sum, off);
     common += __shfl_xor_sync(0xFFFFFFFFu, common, off);
   }
-  __syncwarp();
+  warp_barrier();
   // median from the histogram: sorted positions (n - 1) / 2 and n / 2; lane l owns bins 4l .. 4l + 3
   const uint32_t n = (uint32_t)k - err_e;
   uint32_t local[4], sum = 0;
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
-    local[b] = ws.hist[lane * 4 + b];
+    local[b] = hist[lane * 4 + b];
     sum += local[b];
   }
   uint32_t incl = sum;
@@ -1122,6 +1101,82 @@ toploc_evaluate_kernel(Selection sel, VerifyIo io, int k, long long num_chunks) 
     res.accept = reject ? 0 : 1;
     io.results[chunk] = res;
   }
+}
+
+template <int DT, int SLOTS>
+__device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, long long chunk, const VerifyIo& io,
+                                             const toploc_chunk_result& res) {
+  const int lane = threadIdx.x;
+  uint32_t idx[SLOTS], bits[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int j = s * 32 + lane;
+    idx[s] = 0;
+    bits[s] = 0;
+    if (j < k) {
+      const unsigned long long cj = sh.cand[j];
+      const uint32_t key = (uint32_t)(cj >> (kIdxBits + 1));
+      const uint32_t sign = (uint32_t)cj & 1u;
+      idx[s] = kIdxMask - ((uint32_t)(cj >> 1) & kIdxMask);
+      bits[s] = (sign << 15) | (DT == 0 ? key : (key >> 16));
+    }
+  }
+  evaluate_warp<SLOTS>(sh, k, chunk, idx, bits, io, res);
+}
+
+// ---------------------------------------------------------------------------
+// verify kernel: Algorithm 2 for one chunk per block (one warp): decode(),
+// topk() while the chunk streams in, then Horner evaluation, comparison and
+// verdict by the same warp.  Validation needs no scratch memory beyond the row
+// table of a ragged batch.
+// ---------------------------------------------------------------------------
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_verify_kernel(BatchParams bp, VerifyIo io) {
+  __shared__ SelectShared sh;
+  const int tid = threadIdx.x;
+  const long long chunk = blockIdx.x;
+  const int k = bp.k;
+
+  toploc_chunk_result res;
+  res.exp_mismatch = 0;
+  res.n_match = 0;
+  res.mant_diff_sum = 0;
+  res.topk_mismatch = -1;
+  res.mant_mean = 0.0;
+  res.mant_median = 0.0;
+  res.accept = 0;
+  res.status = TOPLOC_CHUNK_OK;
+  res.pad[0] = res.pad[1] = 0;
+  // decode(): a malformed proof is reported without looking at the activations
+  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 2 * (size_t)k));
+  uint32_t m = proof[0];
+  if (m == 0) m = 65536u;
+  res.modulus = m;
+  uint32_t bad = (m < kModLow || m > kModHigh);
+  for (int d = tid; d < k; d += kThreads) bad |= proof[1 + d] >= kPrime;
+  if (__any_sync(0xFFFFFFFFu, bad != 0)) {
+    res.status = TOPLOC_CHUNK_BAD_PROOF;
+    if (tid == 0) io.results[chunk] = res;
+    return;
+  }
+  const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
+  const long long n_elems = (long long)pl.rows * bp.hidden;
+  if (n_elems < k) {
+    res.status = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+    if (tid == 0) io.results[chunk] = res;
+    return;
+  }
+  ChunkSource<DT, MODE> src;
+  src.base = pl.base;
+  src.row_stride = bp.row_stride;
+  src.hidden = bp.hidden;
+  src.vecs_per_row = bp.hidden / ChunkSource<DT, MODE>::kVec;
+  select_topk<DT, MODE>(sh, src, (int)n_elems, k);
+
+  if (k <= 32) verify_chunk<DT, 1>(sh, k, chunk, io, res);
+  else if (k <= 64) verify_chunk<DT, 2>(sh, k, chunk, io, res);
+  else if (k <= 128) verify_chunk<DT, 4>(sh, k, chunk, io, res);
+  else verify_chunk<DT, kMaxSlots>(sh, k, chunk, io, res);
 }
 
 // ---------------------------------------------------------------------------
@@ -1279,30 +1334,47 @@ void launch_select(int mode, unsigned grid, cudaStream_t stream, const BatchPara
   else toploc_select_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, sel);
 }
 
-// Common front half of both entry points: checks, scratch carving, row table, select kernel.
-int run_select(const void* d_act, const toploc_layout* lay, void* d_workspace, size_t workspace_bytes,
-               cudaStream_t stream, uint8_t* d_status_or_null, uint8_t* d_proofs_or_null,
-               int32_t* d_indices_opt, HostPlan* plan, Selection* sel, DeviceInfo** dev,
-               uint32_t* d_sel_idx_or_null = nullptr, uint16_t* d_sel_bits_or_null = nullptr) {
+template <int DT>
+void launch_verify(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const VerifyIo& io) {
+  if (mode == 0) toploc_verify_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, io);
+  else if (mode == 1) toploc_verify_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, io);
+  else toploc_verify_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, io);
+}
+
+// Checks the scratch and describes the batch to the kernels; a ragged batch's row table is uploaded.
+int prepare_batch(const void* d_act, const toploc_layout* lay, void* d_workspace, size_t workspace_bytes,
+                  cudaStream_t stream, const HostPlan* plan, DeviceInfo** dev, BatchParams* bp) {
   int rc = device_info(dev);
   if (rc != TOPLOC_OK) return rc;
   const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k);
   if (d_workspace == nullptr || workspace_bytes < wp.total) return TOPLOC_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(d_workspace) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
   char* ws = static_cast<char*>(d_workspace);
-  BatchParams bp;
-  bp.act = d_act;
-  bp.row_stride = lay->row_stride;
-  bp.tokens_per_seq = lay->tokens_per_seq;
-  bp.spans = nullptr;
-  bp.hidden = lay->hidden;
-  bp.chunk_len = lay->chunk_len;
-  bp.k = lay->k;
-  bp.chunks_per_seq = plan->chunks_per_seq;
+  bp->act = d_act;
+  bp->row_stride = lay->row_stride;
+  bp->tokens_per_seq = lay->tokens_per_seq;
+  bp->spans = nullptr;
+  bp->hidden = lay->hidden;
+  bp->chunk_len = lay->chunk_len;
+  bp->k = lay->k;
+  bp->chunks_per_seq = plan->chunks_per_seq;
   if (plan->ragged) {
     if ((rc = upload_spans(lay, *plan, ws + wp.spans_off, stream)) != TOPLOC_OK) return rc;
-    bp.spans = reinterpret_cast<const ChunkSpan*>(ws + wp.spans_off);
+    bp->spans = reinterpret_cast<const ChunkSpan*>(ws + wp.spans_off);
   }
+  return TOPLOC_OK;
+}
+
+// Front half of proof generation and of toploc_select_topk: scratch carving and the select kernel.
+int run_select(const void* d_act, const toploc_layout* lay, void* d_workspace, size_t workspace_bytes,
+               cudaStream_t stream, uint8_t* d_status_or_null, uint8_t* d_proofs_or_null,
+               int32_t* d_indices_opt, HostPlan* plan, Selection* sel, DeviceInfo** dev,
+               uint32_t* d_sel_idx_or_null = nullptr, uint16_t* d_sel_bits_or_null = nullptr) {
+  BatchParams bp;
+  int rc = prepare_batch(d_act, lay, d_workspace, workspace_bytes, stream, plan, dev, &bp);
+  if (rc != TOPLOC_OK) return rc;
+  const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k);
+  char* ws = static_cast<char*>(d_workspace);
   sel->idx = d_sel_idx_or_null ? d_sel_idx_or_null : reinterpret_cast<uint32_t*>(ws + wp.idx_off);
   sel->bits = d_sel_bits_or_null ? d_sel_bits_or_null : reinterpret_cast<uint16_t*>(ws + wp.bits_off);
   sel->status = d_status_or_null ? d_status_or_null : reinterpret_cast<uint8_t*>(ws + wp.status_off);
@@ -1445,10 +1517,9 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   if (thr->t_exp < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (plan.num_chunks == 0) return TOPLOC_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  Selection sel;
   DeviceInfo* dev = nullptr;
-  rc = run_select(d_act, lay, d_workspace, workspace_bytes, stream, nullptr, nullptr, nullptr, &plan, &sel,
-                  &dev);
+  BatchParams bp;
+  rc = prepare_batch(d_act, lay, d_workspace, workspace_bytes, stream, &plan, &dev, &bp);
   if (rc != TOPLOC_OK) return rc;
   VerifyIo io;
   io.proofs = d_proofs;
@@ -1458,8 +1529,9 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   io.sign_in_exponent = thr->sign_in_exponent;
   io.t_mean = thr->t_mean;
   io.t_median = thr->t_median;
-  const long long blocks = (plan.num_chunks + kVerifyWarps - 1) / kVerifyWarps;
-  toploc_evaluate_kernel<<<(unsigned)blocks, kVerifyWarps * 32, 0, stream>>>(sel, io, lay->k, plan.num_chunks);
+  const int mode = pick_mode(d_act, lay);
+  if (lay->dtype == TOPLOC_DTYPE_BF16) launch_verify<0>(mode, (unsigned)plan.num_chunks, stream, bp, io);
+  else launch_verify<1>(mode, (unsigned)plan.num_chunks, stream, bp, io);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
