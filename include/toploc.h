@@ -37,9 +37,14 @@ extern "C" {
 #define TOPLOC_DTYPE_BF16 0
 #define TOPLOC_DTYPE_FP32 1
 
-/* Largest k the kernels are built for and largest chunk (elements). */
+/* Largest k the kernels are built for and largest chunk (elements; only chunks
+ * the layout really contains count, so chunk_len may exceed every sequence).
+ * A chunk of more than 2^19 elements -- a prompt committed as one chunk,
+ * Section 5.5 -- is selected in segments of whole rows, one warp each, whose
+ * winners are merged; the result is the same top-k.  hidden itself may not
+ * exceed 2^24. */
 #define TOPLOC_MAX_K 256
-#define TOPLOC_MAX_CHUNK_ELEMS (1 << 24)
+#define TOPLOC_MAX_CHUNK_ELEMS 0x7FFFFFFF
 
 /* Host-side return codes (0 = success, negative = nothing was enqueued). */
 #define TOPLOC_OK 0
@@ -124,7 +129,9 @@ size_t toploc_proof_bytes(int32_t k);
 /* Bytes of device scratch build/verify need for this layout: the selected
  * (index, pattern) pairs of every chunk (6k + 1 bytes per chunk) that the
  * select kernel hands to the arithmetic kernel, plus a per-chunk row table for
- * ragged batches (seq_offsets != NULL). */
+ * ragged batches (seq_offsets != NULL).  A layout with a long chunk (see
+ * TOPLOC_MAX_CHUNK_ELEMS) also needs 14k + 17 bytes per segment and 16 bytes
+ * per chunk.  One size serves every entry point. */
 size_t toploc_workspace_bytes(const toploc_layout* lay);
 
 /* Smallest device staging buffer the *_host entry points accept for this
@@ -228,7 +235,9 @@ int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_
  * rules:
  *   - toploc_workspace_bytes(lay) must not exceed TOPLOC_BUILTIN_SCRATCH_BYTES,
  *     else TOPLOC_ERR_BUILTIN_SCRATCH is returned and nothing is enqueued;
- *   - uniform batches only (seq_offsets == NULL), else TOPLOC_ERR_UNSUPPORTED;
+ *   - uniform batches only (seq_offsets == NULL) and no long chunks (more
+ *     than 2^19 elements), else TOPLOC_ERR_UNSUPPORTED: their row tables would
+ *     have to be built on the host heap;
  *   - the first call on each device looks up the buffer's device address (with
  *     that device current); make that first call outside any stream capture;
  *   - all calls on a device share the one buffer, which keeps whatever the

@@ -78,6 +78,14 @@ struct ChunkSpan {   // one per chunk of a ragged batch, built on the host
   int pad;
 };
 
+// Long chunks (a prompt processed as one chunk) are selected in segments of
+// whole rows, one warp per segment, and the segments' winners are merged.
+struct ChunkSegments {  // one per chunk of a batch that holds a long chunk, built on the host
+  long long row0;       // first row of the chunk
+  int first_seg;        // its segments are first_seg .. first_seg + n_segs - 1
+  int n_segs;
+};
+
 struct BatchParams {
   const void* act;
   long long row_stride;        // elements
@@ -96,6 +104,16 @@ struct Selection {
   uint8_t* status;     // [num_chunks] TOPLOC_CHUNK_*; the caller's d_status during proof generation
   uint8_t* proofs;     // proof generation only: receives the modulus (or zeros)
   int32_t* indices;    // optional: indices in rank order
+};
+
+// Inputs of the merge kernel: the per-segment selections (indices local to the segment).
+struct MergeParams {
+  const ChunkSegments* chunks;
+  const ChunkSpan* segs;
+  const uint32_t* seg_idx;      // [num_segs, k]
+  const uint16_t* seg_bits;     // [num_segs, k]
+  const uint8_t* seg_status;    // [num_segs]
+  unsigned long long* words;    // [num_segs, k] scratch: the candidates of a chunk as ranking words
 };
 
 struct VerifyIo {
@@ -688,18 +706,15 @@ static_assert(kGenerator != 0 && mul_mod(kGenerator, kGeneratorInv) == 1u, "gene
 // Algorithm 6: largest m in [2^15 + 1, 2^16] for which the selected indices
 // stay distinct as (index mod m) mod p -- the second reduction because the
 // x-coordinates live in Z_p and m may exceed p.  Returns 0 if there is none.
-// The selected candidates sit in sh.cand[0..k) on entry and are consumed: the
-// tile ring and the candidate buffer become the 65536-bit set of residues seen.
-__device__ uint32_t find_injective_modulus(SelectShared& sh, int k) {
+// idx[e] is the flat index of point 32 e + lane.  The selection in shared
+// memory is consumed: the tile ring and the candidate buffer become the
+// 65536-bit set of residues seen.
+__device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32_t (&idx)[kMaxK / kThreads]) {
   const int tid = threadIdx.x;
-  uint32_t idx[kMaxK / kThreads], res[kMaxK / kThreads];
+  uint32_t res[kMaxK / kThreads];
 #pragma unroll
-  for (int e = 0; e < kMaxK / kThreads; ++e) {
-    int j = tid + e * kThreads;
-    idx[e] = j < k ? kIdxMask - ((uint32_t)(sh.cand[j] >> 1) & kIdxMask) : 0u;
-    res[e] = 0;
-  }
-  __syncthreads();
+  for (int e = 0; e < kMaxK / kThreads; ++e) res[e] = 0;
+  __syncthreads();  // every lane has taken its candidates out of sh.cand
   uint32_t* seen = reinterpret_cast<uint32_t*>(sh.ring);  // ring and cand are adjacent: 11 KB
   for (int i = tid; i < 2048; i += kThreads) seen[i] = 0;
   __syncthreads();
@@ -810,7 +825,13 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
     return;
   }
   const int nonfinite = __syncthreads_or(unrepresentable != 0);
-  const uint32_t m = find_injective_modulus(sh, k);
+  uint32_t picked[kMaxK / kThreads];
+#pragma unroll
+  for (int e = 0; e < kMaxK / kThreads; ++e) {
+    const int j = tid + e * kThreads;
+    picked[e] = j < k ? kIdxMask - ((uint32_t)(sh.cand[j] >> 1) & kIdxMask) : 0u;
+  }
+  const uint32_t m = find_injective_modulus(sh, k, picked);
   if (m == 0) {
     for (int i = tid; i < k + 1; i += kThreads) proof[i] = 0;
     if (tid == 0) sel.status[chunk] = TOPLOC_CHUNK_NO_INJECTIVE_MODULUS;
@@ -1124,6 +1145,35 @@ __device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, long long 
   evaluate_warp<SLOTS>(sh, k, chunk, idx, bits, io, res);
 }
 
+// decode() of Algorithm 2 for one chunk, by one warp: fills res with zeros and
+// the decoded modulus.  A malformed proof (modulus outside [2^15 + 1, 2^16] or a
+// coefficient >= p) is reported without looking at the activations: its result
+// is written and false returned.
+__device__ __forceinline__ bool decode_proof(const VerifyIo& io, long long chunk, int k, toploc_chunk_result* res) {
+  const int lane = threadIdx.x;
+  res->exp_mismatch = 0;
+  res->n_match = 0;
+  res->mant_diff_sum = 0;
+  res->topk_mismatch = -1;
+  res->mant_mean = 0.0;
+  res->mant_median = 0.0;
+  res->accept = 0;
+  res->status = TOPLOC_CHUNK_OK;
+  res->pad[0] = res->pad[1] = 0;
+  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 2 * (size_t)k));
+  uint32_t m = proof[0];
+  if (m == 0) m = 65536u;
+  res->modulus = m;
+  uint32_t bad = (m < kModLow || m > kModHigh);
+  for (int d = lane; d < k; d += kThreads) bad |= proof[1 + d] >= kPrime;
+  if (__any_sync(0xFFFFFFFFu, bad != 0)) {
+    res->status = TOPLOC_CHUNK_BAD_PROOF;
+    if (lane == 0) io.results[chunk] = *res;
+    return false;
+  }
+  return true;
+}
+
 // ---------------------------------------------------------------------------
 // verify kernel: Algorithm 2 for one chunk per block (one warp): decode(),
 // topk() while the chunk streams in, then Horner evaluation, comparison and
@@ -1138,27 +1188,7 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
   const int k = bp.k;
 
   toploc_chunk_result res;
-  res.exp_mismatch = 0;
-  res.n_match = 0;
-  res.mant_diff_sum = 0;
-  res.topk_mismatch = -1;
-  res.mant_mean = 0.0;
-  res.mant_median = 0.0;
-  res.accept = 0;
-  res.status = TOPLOC_CHUNK_OK;
-  res.pad[0] = res.pad[1] = 0;
-  // decode(): a malformed proof is reported without looking at the activations
-  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 2 * (size_t)k));
-  uint32_t m = proof[0];
-  if (m == 0) m = 65536u;
-  res.modulus = m;
-  uint32_t bad = (m < kModLow || m > kModHigh);
-  for (int d = tid; d < k; d += kThreads) bad |= proof[1 + d] >= kPrime;
-  if (__any_sync(0xFFFFFFFFu, bad != 0)) {
-    res.status = TOPLOC_CHUNK_BAD_PROOF;
-    if (tid == 0) io.results[chunk] = res;
-    return;
-  }
+  if (!decode_proof(io, chunk, k, &res)) return;
   const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
   const long long n_elems = (long long)pl.rows * bp.hidden;
   if (n_elems < k) {
@@ -1180,14 +1210,201 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
 }
 
 // ---------------------------------------------------------------------------
+// merge kernel: the top-k of a chunk from the top-k of its segments, one warp
+// per chunk, then the same tails as the select and verify kernels.  Every
+// candidate becomes one 64-bit word whose unsigned order is the ranking order
+// over the whole chunk: key << 33 | (2^32 - 1 - flat index) << 1 | sign.  The
+// k-th largest word is found digit by digit (MSB-first radix select, eight
+// 8-bit passes over the chunk's words in scratch memory); the words that reach
+// it are the chunk's selection.  A chunk of one segment passes through.
+// TAIL: 0 hand the selection out, 1 proof generation (also the modulus),
+// 2 validation.
+// ---------------------------------------------------------------------------
+template <int DT, int TAIL, int SLOTS>
+__device__ __forceinline__ void finish_merged(SelectShared& sh, int k, long long chunk, const Selection& sel,
+                                              const VerifyIo& io, const toploc_chunk_result& res) {
+  const int lane = threadIdx.x;
+  uint32_t idx[kMaxK / kThreads], bits[SLOTS];
+  uint32_t unrepresentable = 0;
+#pragma unroll
+  for (int e = 0; e < kMaxK / kThreads; ++e) idx[e] = 0;
+#pragma unroll
+  for (int e = 0; e < SLOTS; ++e) {
+    const int j = e * 32 + lane;
+    bits[e] = 0;
+    if (j < k) {
+      const unsigned long long w = sh.cand[j];
+      const uint32_t key = (uint32_t)(w >> 33);
+      const uint32_t sign = (uint32_t)w & 1u;
+      idx[e] = 0xFFFFFFFFu - (uint32_t)(w >> 1);
+      bits[e] = (sign << 15) | (DT == 0 ? key : (key >> 16));
+      unrepresentable |= bits[e] >= kPrime;
+      if (TAIL != 2) {
+        sel.idx[chunk * k + j] = idx[e];
+        sel.bits[chunk * k + j] = (uint16_t)bits[e];
+        if (sel.indices) {
+          int rank = 0;  // position = number of better candidates
+          for (int i = 0; i < k; ++i) rank += sh.cand[i] > w;
+          sel.indices[chunk * k + rank] = (int32_t)idx[e];
+        }
+      }
+    }
+  }
+  if (TAIL == 0) {
+    if (lane == 0) sel.status[chunk] = TOPLOC_CHUNK_OK;
+  } else if (TAIL == 1) {
+    uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 2 * (size_t)k));
+    const int nonfinite = __syncthreads_or(unrepresentable != 0);
+    const uint32_t m = find_injective_modulus(sh, k, idx);
+    if (m == 0) {
+      for (int i = lane; i < k + 1; i += kThreads) proof[i] = 0;
+      if (lane == 0) sel.status[chunk] = TOPLOC_CHUNK_NO_INJECTIVE_MODULUS;
+      return;
+    }
+    if (lane == 0) {
+      proof[0] = (uint16_t)(m & 0xFFFFu);  // 65536 is stored as 0
+      sel.status[chunk] = nonfinite ? TOPLOC_CHUNK_NONFINITE_COMMITTED : TOPLOC_CHUNK_OK;
+    }
+  } else {
+    uint32_t own[SLOTS];
+#pragma unroll
+    for (int e = 0; e < SLOTS; ++e) own[e] = idx[e];
+    evaluate_warp<SLOTS>(sh, k, chunk, own, bits, io, res);
+  }
+}
+
+template <int DT, int TAIL>
+__global__ void __launch_bounds__(kThreads)
+toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) {
+  __shared__ SelectShared sh;
+  const int lane = threadIdx.x;
+  const uint32_t below = (1u << lane) - 1u;
+  const long long chunk = blockIdx.x;
+  const int k = bp.k;
+  toploc_chunk_result res;
+  if (TAIL == 2 && !decode_proof(io, chunk, k, &res)) return;
+
+  const ChunkSegments cs = mp.chunks[chunk];
+  if (mp.seg_status[cs.first_seg] != TOPLOC_CHUNK_OK) {
+    // fewer than k elements: such a chunk is one segment, which said so
+    if (TAIL == 2) {
+      res.status = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+      if (lane == 0) io.results[chunk] = res;
+      return;
+    }
+    if (TAIL == 1) {
+      uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 2 * (size_t)k));
+      for (int i = lane; i < k + 1; i += kThreads) proof[i] = 0;
+    }
+    if (sel.indices)
+      for (int i = lane; i < k; i += kThreads) sel.indices[chunk * k + i] = 0;
+    if (lane == 0) sel.status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+    return;
+  }
+
+  const int n = cs.n_segs * k;
+  unsigned long long* words = mp.words + (size_t)cs.first_seg * k;
+  for (int c = lane; c < n; c += kThreads) {
+    const int seg = c / k;
+    const size_t at = (size_t)(cs.first_seg + seg) * k + (size_t)(c - seg * k);
+    const long long seg_row0 = mp.segs[cs.first_seg + seg].row0;
+    const uint32_t local = mp.seg_idx[at];
+    const uint32_t flat = (uint32_t)((seg_row0 - cs.row0) * bp.hidden) + local;
+    uint32_t key, sign;
+    if (DT == 0) {
+      const uint32_t pattern = mp.seg_bits[at];
+      key = pattern & 0x7FFFu;
+      sign = pattern >> 15;
+    } else {
+      // the segment kept only the upper half of the pattern: read the element again
+      const long long row = seg_row0 + local / (uint32_t)bp.hidden;
+      const uint32_t col = local % (uint32_t)bp.hidden;
+      const uint32_t pattern = static_cast<const uint32_t*>(bp.act)[row * bp.row_stride + col];
+      key = pattern & 0x7FFFFFFFu;
+      sign = pattern >> 31;
+    }
+    words[c] = ((unsigned long long)key << 33) | ((unsigned long long)(0xFFFFFFFFu - flat) << 1) | sign;
+  }
+  __syncwarp();
+
+  unsigned long long kth = 0;  // the k-th largest word; all of them if the chunk is one segment
+  if (n > k) {
+    unsigned long long prefix = 0;
+    int want = k;
+#pragma unroll 1
+    for (int pass = 0; pass < 8; ++pass) {
+      const int shift = 56 - 8 * pass;
+      warp_barrier();
+      for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
+      warp_barrier();
+      for (int c = lane; c < n; c += kThreads) {
+        const unsigned long long w = words[c];
+        if (pass == 0 || (w >> (shift + 8)) == prefix) atomicAdd(&sh.top_hist[(uint32_t)(w >> shift) & 255u], 1u);
+      }
+      find_from_top<8>(sh, sh.top_hist, want);
+      prefix = (prefix << 8) | sh.digit;
+      want = sh.want;
+    }
+    kth = prefix;
+  }
+  int count = 0;
+  for (int c0 = 0; c0 < n; c0 += kThreads) {
+    const int c = c0 + lane;
+    const unsigned long long w = c < n ? words[c] : 0ull;
+    const bool keep = c < n && w >= kth;
+    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, keep);
+    if (keep) sh.cand[count + __popc(votes & below)] = w;  // words are distinct: exactly k are kept
+    count += __popc(votes);
+  }
+  warp_barrier();
+
+  if (k <= 32) finish_merged<DT, TAIL, 1>(sh, k, chunk, sel, io, res);
+  else if (k <= 64) finish_merged<DT, TAIL, 2>(sh, k, chunk, sel, io, res);
+  else if (k <= 128) finish_merged<DT, TAIL, 4>(sh, k, chunk, sel, io, res);
+  else finish_merged<DT, TAIL, kMaxSlots>(sh, k, chunk, sel, io, res);
+}
+
+// ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
 struct HostPlan {
   long long num_chunks;
   long long max_seq_rows;
+  long long num_segs;  // segments over all chunks; equals num_chunks unless some chunk is long
   int chunks_per_seq;  // uniform only
   bool ragged;
+  bool split;          // some chunk is selected in more than one segment
 };
+
+// A chunk of more than kLongChunkElems elements is selected in segments of whole
+// rows (about kSegmentElems elements each, at most kMaxSegmentsPerChunk unless
+// the 24-bit index field of a candidate forces more) whose winners are merged.
+constexpr long long kLongChunkElems = 1ll << 19;
+constexpr long long kSegmentElems = 1ll << 18;
+constexpr long long kMaxSegmentsPerChunk = 64;
+constexpr long long kMaxSegmentElems = 1ll << kIdxBits;
+
+// Segments of a chunk of `rows` rows (1: the chunk is selected directly).
+// Segment g covers rows [rows * g / n, rows * (g + 1) / n).
+long long segments_of(long long rows, long long hidden) {
+  const long long n = rows * hidden;
+  if (n <= kLongChunkElems) return 1;
+  long long segs = (n + kSegmentElems - 1) / kSegmentElems;
+  if (segs > kMaxSegmentsPerChunk) segs = kMaxSegmentsPerChunk;
+  const long long rows_fit = kMaxSegmentElems / hidden;  // rows whose indices fit the candidate's field
+  const long long forced = (rows + rows_fit - 1) / rows_fit;
+  if (segs < forced) segs = forced;
+  if (segs > rows) segs = rows;
+  return segs;
+}
+
+// Chunks and segments of a sequence of len rows: len / L full chunks and perhaps a shorter last one.
+void count_sequence(const toploc_layout* lay, long long len, long long* chunks, long long* segs) {
+  const long long full = len / lay->chunk_len, rest = len % lay->chunk_len;
+  *chunks += full + (rest ? 1 : 0);
+  if (full) *segs += full * segments_of(lay->chunk_len, lay->hidden);
+  if (rest) *segs += segments_of(rest, lay->hidden);
+}
 
 int plan_layout(const toploc_layout* lay, HostPlan* plan) {
   if (lay == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
@@ -1197,16 +1414,22 @@ int plan_layout(const toploc_layout* lay, HostPlan* plan) {
   if (lay->k < 1) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (lay->k > TOPLOC_MAX_K) return TOPLOC_ERR_UNSUPPORTED;
   if (lay->row_stride < lay->hidden) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if ((long long)lay->hidden * lay->chunk_len > TOPLOC_MAX_CHUNK_ELEMS) return TOPLOC_ERR_UNSUPPORTED;
+  if (lay->hidden > kMaxSegmentElems) return TOPLOC_ERR_UNSUPPORTED;  // a row must fit one segment
   plan->ragged = lay->seq_offsets != nullptr;
   plan->chunks_per_seq = 0;
-  long long n = 0, longest = 0;
+  long long n = 0, longest = 0, segs = 0;
+  // only chunks that exist count against the size limit
+  auto largest_chunk_fits = [&](long long len) {
+    const long long rows = len < lay->chunk_len ? len : lay->chunk_len;
+    return rows * lay->hidden <= (long long)TOPLOC_MAX_CHUNK_ELEMS;
+  };
   if (plan->ragged) {
     if (lay->seq_offsets[0] < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
     for (int s = 0; s < lay->num_seqs; ++s) {
       long long len = lay->seq_offsets[s + 1] - lay->seq_offsets[s];
       if (len < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
-      n += (len + lay->chunk_len - 1) / lay->chunk_len;
+      if (!largest_chunk_fits(len)) return TOPLOC_ERR_UNSUPPORTED;
+      count_sequence(lay, len, &n, &segs);
       if (len > longest) longest = len;
     }
   } else {
@@ -1214,11 +1437,16 @@ int plan_layout(const toploc_layout* lay, HostPlan* plan) {
     long long cps = (lay->tokens_per_seq + lay->chunk_len - 1) / lay->chunk_len;
     if (cps > 0x7FFFFFFFll) return TOPLOC_ERR_UNSUPPORTED;
     plan->chunks_per_seq = (int)cps;
-    n = cps * lay->num_seqs;
+    if (!largest_chunk_fits(lay->tokens_per_seq)) return TOPLOC_ERR_UNSUPPORTED;
+    count_sequence(lay, lay->tokens_per_seq, &n, &segs);
+    n *= lay->num_seqs;
+    segs *= lay->num_seqs;
     longest = lay->tokens_per_seq;
   }
-  if (n > 0x7FFFFFFFll) return TOPLOC_ERR_UNSUPPORTED;
+  if (n > 0x7FFFFFFFll || segs > 0x7FFFFFFFll) return TOPLOC_ERR_UNSUPPORTED;
   plan->num_chunks = n;
+  plan->num_segs = segs;
+  plan->split = segs != n;
   plan->max_seq_rows = longest;
   return TOPLOC_OK;
 }
@@ -1286,16 +1514,30 @@ int pick_mode(const void* act, const toploc_layout* lay) {
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Scratch of one call: ragged row table, then the selection.
+// Scratch of one call: ragged row table, then the selection; with long chunks
+// (segs != chunks) the row table describes segments and is followed by the
+// chunk table, the segments' selections and the merge's words.
 struct WorkspacePlan {
-  size_t spans_off, idx_off, bits_off, status_off, total;
+  size_t spans_off, chunk_table_off, seg_idx_off, seg_bits_off, seg_status_off, words_off;
+  size_t idx_off, bits_off, status_off, total;
 };
 
-WorkspacePlan plan_workspace(bool ragged, long long chunks, int k) {
+WorkspacePlan plan_workspace(bool ragged, long long chunks, int k, long long segs) {
   WorkspacePlan w;
+  const bool split = segs != chunks;
   size_t off = 0;
   w.spans_off = off;
-  off += ragged ? round_up((size_t)chunks * sizeof(ChunkSpan), 256) : 0;
+  off += (ragged || split) ? round_up((size_t)segs * sizeof(ChunkSpan), 256) : 0;
+  w.chunk_table_off = off;
+  off += split ? round_up((size_t)chunks * sizeof(ChunkSegments), 256) : 0;
+  w.seg_idx_off = off;
+  off += split ? round_up((size_t)segs * k * sizeof(uint32_t), 256) : 0;
+  w.seg_bits_off = off;
+  off += split ? round_up((size_t)segs * k * sizeof(uint16_t), 256) : 0;
+  w.seg_status_off = off;
+  off += split ? round_up((size_t)segs, 256) : 0;
+  w.words_off = off;
+  off += split ? round_up((size_t)segs * k * sizeof(unsigned long long), 256) : 0;
   w.idx_off = off;
   off += round_up((size_t)chunks * k * sizeof(uint32_t), 256);
   w.bits_off = off;
@@ -1306,24 +1548,51 @@ WorkspacePlan plan_workspace(bool ragged, long long chunks, int k) {
   return w;
 }
 
-// Fills the device row table of a ragged batch.
-int upload_spans(const toploc_layout* lay, const HostPlan& plan, void* d_spans, cudaStream_t stream) {
-  const size_t need = (size_t)plan.num_chunks * sizeof(ChunkSpan);
-  ChunkSpan* spans = static_cast<ChunkSpan*>(malloc(need));
-  if (spans == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
-  long long c = 0;
+long long seq_begin(const toploc_layout* lay, int s) {
+  return lay->seq_offsets ? lay->seq_offsets[s] : (long long)s * lay->tokens_per_seq;
+}
+
+// Fills the device row table (one span per segment; a chunk that is not long
+// is its own segment) and, for a batch with long chunks, the chunk table.
+int upload_spans(const toploc_layout* lay, const HostPlan& plan, void* d_spans, void* d_chunk_table,
+                 cudaStream_t stream) {
+  const size_t span_bytes = (size_t)plan.num_segs * sizeof(ChunkSpan);
+  const size_t table_bytes = plan.split ? (size_t)plan.num_chunks * sizeof(ChunkSegments) : 0;
+  ChunkSpan* spans = static_cast<ChunkSpan*>(malloc(span_bytes));
+  ChunkSegments* table = plan.split ? static_cast<ChunkSegments*>(malloc(table_bytes)) : nullptr;
+  if (spans == nullptr || (plan.split && table == nullptr)) {
+    free(spans);
+    free(table);
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  }
+  long long c = 0, g = 0;
   for (int s = 0; s < lay->num_seqs; ++s) {
-    for (long long r = lay->seq_offsets[s]; r < lay->seq_offsets[s + 1]; r += lay->chunk_len) {
-      long long left = lay->seq_offsets[s + 1] - r;
-      spans[c].row0 = r;
-      spans[c].rows = (int)(left < lay->chunk_len ? left : lay->chunk_len);
-      spans[c].pad = 0;
+    const long long end = seq_begin(lay, s + 1);
+    for (long long r = seq_begin(lay, s); r < end; r += lay->chunk_len) {
+      const long long left = end - r;
+      const long long rows = left < lay->chunk_len ? left : lay->chunk_len;
+      const long long n_segs = segments_of(rows, lay->hidden);
+      if (table) {
+        table[c].row0 = r;
+        table[c].first_seg = (int)g;
+        table[c].n_segs = (int)n_segs;
+      }
+      for (long long i = 0; i < n_segs; ++i) {
+        const long long a = rows * i / n_segs, b = rows * (i + 1) / n_segs;
+        spans[g].row0 = r + a;
+        spans[g].rows = (int)(b - a);
+        spans[g].pad = 0;
+        ++g;
+      }
       ++c;
     }
   }
-  // pageable source: the runtime has staged the bytes by the time this returns
-  cudaError_t err = cudaMemcpyAsync(d_spans, spans, need, cudaMemcpyHostToDevice, stream);
+  // pageable sources: the runtime has staged the bytes by the time these return
+  cudaError_t err = cudaMemcpyAsync(d_spans, spans, span_bytes, cudaMemcpyHostToDevice, stream);
+  if (err == cudaSuccess && table)
+    err = cudaMemcpyAsync(d_chunk_table, table, table_bytes, cudaMemcpyHostToDevice, stream);
   free(spans);
+  free(table);
   return err == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
@@ -1341,15 +1610,38 @@ void launch_verify(int mode, unsigned grid, cudaStream_t stream, const BatchPara
   else toploc_verify_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, io);
 }
 
-// Checks the scratch and describes the batch to the kernels; a ragged batch's row table is uploaded.
+template <int DT>
+void launch_merge(int tail, unsigned grid, cudaStream_t stream, const BatchParams& bp, const MergeParams& mp,
+                  const Selection& sel, const VerifyIo& io) {
+  if (tail == 0) toploc_merge_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, mp, sel, io);
+  else if (tail == 1) toploc_merge_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, mp, sel, io);
+  else toploc_merge_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, mp, sel, io);
+}
+
+// A batch as the kernels see it.
+struct PreparedBatch {
+  BatchParams bp;       // chunks; in a batch with long chunks: segments (one warp each)
+  MergeParams mp;       // batches with long chunks only
+  Selection segs;       // where the segment selections go (batches with long chunks only)
+  WorkspacePlan wp;
+  char* ws;
+  unsigned grid;        // blocks of the select / verify kernel
+};
+
+// Checks the scratch and describes the batch to the kernels; the row table of a
+// ragged batch or of one with long chunks is uploaded.
 int prepare_batch(const void* d_act, const toploc_layout* lay, void* d_workspace, size_t workspace_bytes,
-                  cudaStream_t stream, const HostPlan* plan, DeviceInfo** dev, BatchParams* bp) {
+                  cudaStream_t stream, const HostPlan* plan, DeviceInfo** dev, PreparedBatch* pb) {
   int rc = device_info(dev);
   if (rc != TOPLOC_OK) return rc;
-  const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k);
+  const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k, plan->num_segs);
   if (d_workspace == nullptr || workspace_bytes < wp.total) return TOPLOC_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(d_workspace) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
   char* ws = static_cast<char*>(d_workspace);
+  pb->wp = wp;
+  pb->ws = ws;
+  pb->grid = (unsigned)plan->num_segs;
+  BatchParams* bp = &pb->bp;
   bp->act = d_act;
   bp->row_stride = lay->row_stride;
   bp->tokens_per_seq = lay->tokens_per_seq;
@@ -1358,31 +1650,53 @@ int prepare_batch(const void* d_act, const toploc_layout* lay, void* d_workspace
   bp->chunk_len = lay->chunk_len;
   bp->k = lay->k;
   bp->chunks_per_seq = plan->chunks_per_seq;
-  if (plan->ragged) {
-    if ((rc = upload_spans(lay, *plan, ws + wp.spans_off, stream)) != TOPLOC_OK) return rc;
+  if (plan->ragged || plan->split) {
+    if ((rc = upload_spans(lay, *plan, ws + wp.spans_off, ws + wp.chunk_table_off, stream)) != TOPLOC_OK) return rc;
     bp->spans = reinterpret_cast<const ChunkSpan*>(ws + wp.spans_off);
+  }
+  if (plan->split) {
+    pb->segs.idx = reinterpret_cast<uint32_t*>(ws + wp.seg_idx_off);
+    pb->segs.bits = reinterpret_cast<uint16_t*>(ws + wp.seg_bits_off);
+    pb->segs.status = reinterpret_cast<uint8_t*>(ws + wp.seg_status_off);
+    pb->segs.proofs = nullptr;
+    pb->segs.indices = nullptr;
+    pb->mp.chunks = reinterpret_cast<const ChunkSegments*>(ws + wp.chunk_table_off);
+    pb->mp.segs = bp->spans;
+    pb->mp.seg_idx = pb->segs.idx;
+    pb->mp.seg_bits = pb->segs.bits;
+    pb->mp.seg_status = pb->segs.status;
+    pb->mp.words = reinterpret_cast<unsigned long long*>(ws + wp.words_off);
   }
   return TOPLOC_OK;
 }
 
-// Front half of proof generation and of toploc_select_topk: scratch carving and the select kernel.
+// Front half of proof generation and of toploc_select_topk: scratch carving and
+// the select kernel (for a batch with long chunks: per segment, then the merge).
 int run_select(const void* d_act, const toploc_layout* lay, void* d_workspace, size_t workspace_bytes,
                cudaStream_t stream, uint8_t* d_status_or_null, uint8_t* d_proofs_or_null,
                int32_t* d_indices_opt, HostPlan* plan, Selection* sel, DeviceInfo** dev,
                uint32_t* d_sel_idx_or_null = nullptr, uint16_t* d_sel_bits_or_null = nullptr) {
-  BatchParams bp;
-  int rc = prepare_batch(d_act, lay, d_workspace, workspace_bytes, stream, plan, dev, &bp);
+  PreparedBatch pb;
+  int rc = prepare_batch(d_act, lay, d_workspace, workspace_bytes, stream, plan, dev, &pb);
   if (rc != TOPLOC_OK) return rc;
-  const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k);
-  char* ws = static_cast<char*>(d_workspace);
-  sel->idx = d_sel_idx_or_null ? d_sel_idx_or_null : reinterpret_cast<uint32_t*>(ws + wp.idx_off);
-  sel->bits = d_sel_bits_or_null ? d_sel_bits_or_null : reinterpret_cast<uint16_t*>(ws + wp.bits_off);
-  sel->status = d_status_or_null ? d_status_or_null : reinterpret_cast<uint8_t*>(ws + wp.status_off);
+  sel->idx = d_sel_idx_or_null ? d_sel_idx_or_null : reinterpret_cast<uint32_t*>(pb.ws + pb.wp.idx_off);
+  sel->bits = d_sel_bits_or_null ? d_sel_bits_or_null : reinterpret_cast<uint16_t*>(pb.ws + pb.wp.bits_off);
+  sel->status = d_status_or_null ? d_status_or_null : reinterpret_cast<uint8_t*>(pb.ws + pb.wp.status_off);
   sel->proofs = d_proofs_or_null;
   sel->indices = d_indices_opt;
   const int mode = pick_mode(d_act, lay);
-  if (lay->dtype == TOPLOC_DTYPE_BF16) launch_select<0>(mode, (unsigned)plan->num_chunks, stream, bp, *sel);
-  else launch_select<1>(mode, (unsigned)plan->num_chunks, stream, bp, *sel);
+  const bool bf16 = lay->dtype == TOPLOC_DTYPE_BF16;
+  if (!plan->split) {
+    if (bf16) launch_select<0>(mode, pb.grid, stream, pb.bp, *sel);
+    else launch_select<1>(mode, pb.grid, stream, pb.bp, *sel);
+  } else {
+    if (bf16) launch_select<0>(mode, pb.grid, stream, pb.bp, pb.segs);
+    else launch_select<1>(mode, pb.grid, stream, pb.bp, pb.segs);
+    const VerifyIo none = {};
+    const int tail = d_proofs_or_null ? 1 : 0;
+    if (bf16) launch_merge<0>(tail, (unsigned)plan->num_chunks, stream, pb.bp, pb.mp, *sel, none);
+    else launch_merge<1>(tail, (unsigned)plan->num_chunks, stream, pb.bp, pb.mp, *sel, none);
+  }
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
@@ -1392,7 +1706,7 @@ struct StagingPlan {
   size_t act_off, small_off, proofs_off, work_off, work_bytes, total;
 };
 
-StagingPlan carve_staging(const toploc_layout* lay, long long rows, long long chunks) {
+StagingPlan carve_staging(const toploc_layout* lay, long long rows, long long chunks, long long segs) {
   const size_t esz = lay->dtype == TOPLOC_DTYPE_BF16 ? 2 : 4;
   StagingPlan sp;
   sp.act_off = 0;
@@ -1402,23 +1716,23 @@ StagingPlan carve_staging(const toploc_layout* lay, long long rows, long long ch
   sp.proofs_off = off;
   off += round_up((size_t)chunks * (2 + 2 * (size_t)lay->k), 256);
   sp.work_off = off;
-  sp.work_bytes = plan_workspace(true, chunks, lay->k).total;
+  sp.work_bytes = plan_workspace(true, chunks, lay->k, segs).total;
   off += sp.work_bytes;
   sp.total = off;
   return sp;
 }
 
-long long seq_begin(const toploc_layout* lay, int s) {
-  return lay->seq_offsets ? lay->seq_offsets[s] : (long long)s * lay->tokens_per_seq;
+// Chunks and segments of sequences s0 .. s1 - 1.
+void count_between(const toploc_layout* lay, int s0, int s1, long long* chunks, long long* segs) {
+  *chunks = 0;
+  *segs = 0;
+  for (int s = s0; s < s1; ++s) count_sequence(lay, seq_begin(lay, s + 1) - seq_begin(lay, s), chunks, segs);
 }
 
-long long chunks_between(const toploc_layout* lay, int s0, int s1) {
-  long long n = 0;
-  for (int s = s0; s < s1; ++s) {
-    long long len = seq_begin(lay, s + 1) - seq_begin(lay, s);
-    n += (len + lay->chunk_len - 1) / lay->chunk_len;
-  }
-  return n;
+StagingPlan carve_staging_for(const toploc_layout* lay, int s0, int s1) {
+  long long chunks, segs;
+  count_between(lay, s0, s1, &chunks, &segs);
+  return carve_staging(lay, seq_begin(lay, s1) - seq_begin(lay, s0), chunks, segs);
 }
 
 }  // namespace
@@ -1439,14 +1753,15 @@ size_t toploc_proof_bytes(int32_t k) { return k > 0 ? 2 + 2 * (size_t)k : 0; }
 size_t toploc_workspace_bytes(const toploc_layout* lay) {
   HostPlan plan;
   if (plan_layout(lay, &plan) != TOPLOC_OK) return 0;
-  return plan_workspace(plan.ragged, plan.num_chunks, lay->k).total;
+  return plan_workspace(plan.ragged, plan.num_chunks, lay->k, plan.num_segs).total;
 }
 
 size_t toploc_staging_bytes(const toploc_layout* lay) {
   HostPlan plan;
   if (plan_layout(lay, &plan) != TOPLOC_OK) return 0;
-  long long chunks = (plan.max_seq_rows + lay->chunk_len - 1) / lay->chunk_len;
-  return carve_staging(lay, plan.max_seq_rows, chunks).total;
+  long long chunks = 0, segs = 0;
+  count_sequence(lay, plan.max_seq_rows, &chunks, &segs);
+  return carve_staging(lay, plan.max_seq_rows, chunks, segs).total;
 }
 
 void toploc_get_constants(uint32_t* p, uint32_t* m_lo, uint32_t* m_hi) {
@@ -1518,8 +1833,8 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   if (plan.num_chunks == 0) return TOPLOC_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   DeviceInfo* dev = nullptr;
-  BatchParams bp;
-  rc = prepare_batch(d_act, lay, d_workspace, workspace_bytes, stream, &plan, &dev, &bp);
+  PreparedBatch pb;
+  rc = prepare_batch(d_act, lay, d_workspace, workspace_bytes, stream, &plan, &dev, &pb);
   if (rc != TOPLOC_OK) return rc;
   VerifyIo io;
   io.proofs = d_proofs;
@@ -1530,8 +1845,18 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   io.t_mean = thr->t_mean;
   io.t_median = thr->t_median;
   const int mode = pick_mode(d_act, lay);
-  if (lay->dtype == TOPLOC_DTYPE_BF16) launch_verify<0>(mode, (unsigned)plan.num_chunks, stream, bp, io);
-  else launch_verify<1>(mode, (unsigned)plan.num_chunks, stream, bp, io);
+  const bool bf16 = lay->dtype == TOPLOC_DTYPE_BF16;
+  if (!plan.split) {
+    if (bf16) launch_verify<0>(mode, pb.grid, stream, pb.bp, io);
+    else launch_verify<1>(mode, pb.grid, stream, pb.bp, io);
+  } else {
+    // long chunks: select per segment, then merge and validate per chunk
+    if (bf16) launch_select<0>(mode, pb.grid, stream, pb.bp, pb.segs);
+    else launch_select<1>(mode, pb.grid, stream, pb.bp, pb.segs);
+    const Selection none = {};
+    if (bf16) launch_merge<0>(2, (unsigned)plan.num_chunks, stream, pb.bp, pb.mp, none, io);
+    else launch_merge<1>(2, (unsigned)plan.num_chunks, stream, pb.bp, pb.mp, none, io);
+  }
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
@@ -1557,8 +1882,9 @@ int toploc_build_proofs_builtin_scratch(const void* d_act, const toploc_layout* 
   HostPlan plan;
   int rc = plan_layout(lay, &plan);
   if (rc != TOPLOC_OK) return rc;
-  if (plan.ragged) return TOPLOC_ERR_UNSUPPORTED;  // the row table would have to be built on the heap
-  if (plan_workspace(false, plan.num_chunks, lay->k).total > kBuiltinScratchBytes) return TOPLOC_ERR_BUILTIN_SCRATCH;
+  if (plan.ragged || plan.split) return TOPLOC_ERR_UNSUPPORTED;  // the row table would have to be built on the heap
+  if (plan_workspace(false, plan.num_chunks, lay->k, plan.num_segs).total > kBuiltinScratchBytes)
+    return TOPLOC_ERR_BUILTIN_SCRATCH;
   DeviceInfo* dev = nullptr;
   if ((rc = device_info(&dev)) != TOPLOC_OK) return rc;
   void* scratch = nullptr;
@@ -1592,16 +1918,16 @@ static int run_from_host(bool verify, const void* h_act, const toploc_layout* la
   while (s0 < lay->num_seqs && rc == TOPLOC_OK) {
     // largest group of sequences starting at s0 that fits
     int s1 = s0 + 1;
-    StagingPlan sp = carve_staging(lay, seq_begin(lay, s1) - seq_begin(lay, s0), chunks_between(lay, s0, s1));
+    StagingPlan sp = carve_staging_for(lay, s0, s1);
     while (s1 < lay->num_seqs) {
-      StagingPlan bigger =
-          carve_staging(lay, seq_begin(lay, s1 + 1) - seq_begin(lay, s0), chunks_between(lay, s0, s1 + 1));
+      StagingPlan bigger = carve_staging_for(lay, s0, s1 + 1);
       if (bigger.total > staging_bytes) break;
       sp = bigger;
       ++s1;
     }
     const long long row_a = seq_begin(lay, s0), row_b = seq_begin(lay, s1);
-    const long long chunks = chunks_between(lay, s0, s1);
+    long long chunks, group_segs;
+    count_between(lay, s0, s1, &chunks, &group_segs);
     if (row_b > row_a && chunks > 0) {
       toploc_layout sub = *lay;
       sub.num_seqs = s1 - s0;

@@ -71,9 +71,29 @@ def test_chunk_counting():
     assert tl.toploc_staging_bytes(layout()) >= 100 * 4096 * 2 + 4 * 258
 
 
+def test_long_chunks_are_planned_in_segments():
+    """A chunk above 2^19 elements is selected in segments of about 2^18 elements (whole rows) and
+    merged: the scratch grows by the segments' selections and the merge's words; the chunk count
+    does not change.  Only chunks that exist count against the size limit."""
+    long_one = layout(hidden=4096, row_stride=4096, chunk_len=700, tokens_per_seq=700, num_seqs=1, k=128)
+    assert tl.toploc_num_chunks(long_one) == 1
+    segs = 11                                                     # ceil(700 * 4096 / 2^18)
+    per_seg = 128 * (4 + 2 + 8) + 1 + 16
+    assert tl.toploc_workspace_bytes(long_one) >= segs * per_seg + 128 * 6
+    direct = layout(hidden=4096, row_stride=4096, chunk_len=128, tokens_per_seq=128, num_seqs=1, k=128)
+    assert tl.toploc_workspace_bytes(direct) < 2 * 1024           # 2^19 elements: selected directly
+    huge_len = layout(hidden=8192, row_stride=8192, chunk_len=1 << 30, tokens_per_seq=5000, num_seqs=2, k=128)
+    assert tl.toploc_num_chunks(huge_len) == 2                    # 5000 x 8192 = 41 M elements each
+    lib = tl.load_library()
+    assert lib.toploc_build_proofs_builtin_scratch(ctypes.c_void_p(16), ctypes.byref(long_one), ctypes.c_void_p(16),
+                                                   ctypes.c_void_p(16), None, None) == -2
+
+
 @pytest.mark.parametrize("bad", [dict(k=0), dict(k=257), dict(hidden=0), dict(chunk_len=0), dict(num_seqs=0),
                                  dict(dtype=7), dict(row_stride=100), dict(tokens_per_seq=0),
-                                 dict(reserved=1), dict(hidden=1 << 20, chunk_len=64, row_stride=1 << 20)])
+                                 dict(reserved=1),
+                                 dict(hidden=1 << 20, chunk_len=2048, tokens_per_seq=4096, row_stride=1 << 20),
+                                 dict(hidden=(1 << 24) + 8, row_stride=(1 << 24) + 8)])
 def test_invalid_layouts_are_refused(bad):
     with pytest.raises(tl.ToplocError):
         tl.toploc_num_chunks(layout(**bad))
