@@ -16,6 +16,7 @@ from . import build as _build
 P_FIELD = 65521          # largest prime below 2^16 (Algorithm 3 needs a prime that fits 2 bytes)
 M_HIGH = 65536           # Algorithm 6 search range, inclusive
 M_LOW = 2 ** 15 + 1
+Q_FIELD = 2 ** 32 - 5    # 32-bit field variant: largest prime below 2^32 (fits 4-byte coefficients)
 
 ST_OK, ST_NO_MODULUS, ST_K_EXCEEDS, ST_BAD_PROOF, ST_NONFINITE = range(5)
 
@@ -38,6 +39,8 @@ def lib():
         _lib.oracle_mod_inverse_euclid.restype = ctypes.c_int64
         _lib.oracle_horner.restype = ctypes.c_uint32
         _lib.oracle_num_chunks.restype = ctypes.c_int64
+        _lib.oracle_mod_inverse32.restype = ctypes.c_uint32
+        _lib.oracle_horner32.restype = ctypes.c_uint32
     return _lib
 
 
@@ -121,6 +124,53 @@ def decode(proof):
     return st, k.value, m.value, c[:k.value]
 
 
+def mod_inverse32(a):
+    return int(lib().oracle_mod_inverse32(ctypes.c_uint32(a)))
+
+
+def interpolate32(x, y, newton=False):
+    """Coefficients (ascending degree, uint32) of the polynomial through (x_j, y_j) over Z_q."""
+    x = np.ascontiguousarray(x, np.uint32)
+    y = np.ascontiguousarray(y, np.uint32)
+    c = np.zeros(len(x), np.uint32)
+    fn = lib().oracle_interpolate32_newton if newton else lib().oracle_interpolate32
+    if fn(_ptr(x), _ptr(y), len(x), _ptr(c)) != 0:
+        raise ValueError("x values are not distinct mod q")
+    return c
+
+
+def horner32(coeffs, x):
+    c = np.ascontiguousarray(coeffs, np.uint32)
+    return int(lib().oracle_horner32(_ptr(c), len(c), ctypes.c_uint32(x)))
+
+
+def encode32(m, coeffs):
+    c = np.ascontiguousarray(coeffs, np.uint32)
+    proof = np.zeros(2 + 4 * len(c), np.uint8)
+    lib().oracle_encode32(ctypes.c_uint32(m), _ptr(c), len(c), _ptr(proof))
+    return proof
+
+
+def decode32(proof):
+    """-> (status, k, m, coeffs)."""
+    proof = np.ascontiguousarray(proof, np.uint8)
+    k = ctypes.c_int(0)
+    m = ctypes.c_uint32(0)
+    c = np.zeros(max(1, len(proof) // 4), np.uint32)
+    st = lib().oracle_decode32(_ptr(proof), ctypes.c_int64(len(proof)), ctypes.byref(k), ctypes.byref(m),
+                               _ptr(c))
+    return st, k.value, m.value, c[:k.value]
+
+
+def _batch_dtype_code(act, wide):
+    code = _dtype_code(act)
+    if wide:
+        if code != 1:
+            raise TypeError("the 32-bit field variant commits fp32 activations")
+        return 2
+    return code
+
+
 def num_chunks(num_seqs, tokens_per_seq, chunk_len, seq_offsets=None):
     so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
     return int(lib().oracle_num_chunks(num_seqs, ctypes.c_int64(tokens_per_seq),
@@ -128,8 +178,9 @@ def num_chunks(num_seqs, tokens_per_seq, chunk_len, seq_offsets=None):
 
 
 def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None, first_chunk=0,
-                 last_chunk=-1, want_indices=True, threads=None):
+                 last_chunk=-1, want_indices=True, threads=None, wide=False):
     """act: 2-D [total_tokens, hidden] host array (uint16 bf16 patterns or float32).
+    wide: the 32-bit field variant (fp32 only; proofs of 2 + 4k bytes).
 
     Returns (proofs uint8[n, 2+2k], status uint8[n], indices int32[n, k] or None), all indexed by
     absolute chunk number; only rows first_chunk..last_chunk-1 are filled."""
@@ -138,11 +189,11 @@ def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None
     row_stride = act.strides[0] // act.itemsize
     so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
     n = num_chunks(num_seqs, tokens_per_seq, chunk_len, so)
-    proofs = np.zeros((n, 2 + 2 * k), np.uint8)
+    proofs = np.zeros((n, 2 + (4 if wide else 2) * k), np.uint8)
     status = np.zeros(n, np.uint8)
     indices = np.zeros((n, k), np.int32) if want_indices else None
     lib().oracle_build_proofs(
-        _ptr(act), _dtype_code(act), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
+        _ptr(act), _batch_dtype_code(act, wide), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
         None if so is None else _ptr(so), ctypes.c_int64(row_stride), ctypes.c_int64(first_chunk),
         ctypes.c_int64(last_chunk), _ptr(proofs), _ptr(status),
         None if indices is None else _ptr(indices), threads or default_threads())
@@ -151,7 +202,7 @@ def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None
 
 def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None,
                   t_exp=38, t_mean=10.0, t_median=8.0, sign_in_exponent=True, gen_indices=None,
-                  first_chunk=0, last_chunk=-1, threads=None):
+                  first_chunk=0, last_chunk=-1, threads=None, wide=False):
     """Returns a structured array (RESULT_DTYPE) with one entry per chunk."""
     assert act.ndim == 2 and act.strides[1] == act.itemsize
     hidden = act.shape[1]
@@ -159,11 +210,11 @@ def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_off
     so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
     n = num_chunks(num_seqs, tokens_per_seq, chunk_len, so)
     proofs = np.ascontiguousarray(proofs, np.uint8)
-    assert proofs.shape == (n, 2 + 2 * k)
+    assert proofs.shape == (n, 2 + (4 if wide else 2) * k)
     gi = None if gen_indices is None else np.ascontiguousarray(gen_indices, np.int32)
     results = np.zeros(n, RESULT_DTYPE)
     lib().oracle_verify_proofs(
-        _ptr(act), _dtype_code(act), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
+        _ptr(act), _batch_dtype_code(act, wide), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
         None if so is None else _ptr(so), ctypes.c_int64(row_stride), ctypes.c_int64(first_chunk),
         ctypes.c_int64(last_chunk), _ptr(proofs), int(t_exp), ctypes.c_double(t_mean),
         ctypes.c_double(t_median), int(bool(sign_in_exponent)), None if gi is None else _ptr(gi),

@@ -18,7 +18,9 @@
  *   - proof layout: m & 0xFFFF little-endian (0 means 65536), then the k
  *     coefficients in ascending degree, 2 bytes little-endian each;
  *   - fp32 activations rank on the 31-bit magnitude and commit the upper 16
- *     bits of the pattern (Section 5.6, mantissa scaled to bf16).
+ *     bits of the pattern (Section 5.6, mantissa scaled to bf16), or, in the
+ *     32-bit field variant further down (dtype code 2 of the batch drivers),
+ *     the whole pattern over Z_q, q = 2^32 - 5.
  *
  * Pins (tests/test_oracle_*.py): worked examples and the paper's printed
  * values under tests/golden/, brute force on tiny inputs, P(x_j) = y_j with
@@ -423,6 +425,271 @@ void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int
   free(diffs);
 }
 
+/* ================================================================== */
+/* 32-bit field variant: an fp32 chunk commits the full 32-bit pattern */
+/* of each selected value.  The paper uses it without printing its     */
+/* layout: Section 5.2 gives thresholds "for fp32 inference" (8 / 256 / */
+/* 128, on 23-bit mantissas, cf. the fp32 rows of the precision table   */
+/* in Section 5.6), and the subroutines appendix names "2^32 for        */
+/* 32-bit types" as the size of the modulus.  Readings used here:      */
+/*   - field prime q = 4294967291 = 2^32 - 5, the largest prime below  */
+/*     2^32 (a prime that fits 4-byte coefficients, as p fits 2 bytes); */
+/*   - proof: the same 2 modulus bytes, then k coefficients of 4 bytes  */
+/*     little-endian, ascending degree: 2 + 4k bytes;                  */
+/*   - x = index mod m needs no second reduction (m <= 2^16 < q), so    */
+/*     Algorithm 6 applies as printed;                                 */
+/*   - y = the 32-bit pattern mod q; the five patterns >= q (negative   */
+/*     NaNs) are flagged like their 16-bit counterparts;               */
+/*   - extractBits: bit 31 sign, bits 30..23 exponent, bits 22..0       */
+/*     mantissa (fp32 has 23 mantissa bits, Section 5.2).              */
+/* Everything else (ranking, ties, statistics, verdict) is as above.   */
+/* ================================================================== */
+#define Q_FIELD 4294967291u
+
+static uint32_t mulq(uint32_t a, uint32_t b) { return (uint32_t)(((uint64_t)a * b) % Q_FIELD); }
+static uint32_t addq(uint32_t a, uint32_t b) { return (uint32_t)(((uint64_t)a + b) % Q_FIELD); }
+static uint32_t subq(uint32_t a, uint32_t b) { return (uint32_t)(((uint64_t)a + Q_FIELD - b) % Q_FIELD); }
+
+/* a^(q-2) in Z_q; a in [1, q). */
+uint32_t oracle_mod_inverse32(uint32_t a) {
+  uint32_t result = 1, base = a % Q_FIELD;
+  uint32_t e = Q_FIELD - 2;
+  while (e) {
+    if (e & 1u) result = mulq(result, base);
+    base = mulq(base, base);
+    e >>= 1;
+  }
+  return result;
+}
+
+/* Algorithm 5 over Z_q. */
+uint32_t oracle_horner32(const uint32_t* c, int k, uint32_t x) {
+  uint32_t acc = c[k - 1] % Q_FIELD;
+  x %= Q_FIELD;
+  for (int d = k - 2; d >= 0; --d) acc = addq(mulq(acc, x), c[d] % Q_FIELD);
+  return acc;
+}
+
+/* The unique interpolant over Z_q: Gaussian elimination on the Vandermonde
+ * system, as oracle_interpolate.  Returns 1 if the system is singular. */
+int oracle_interpolate32(const uint32_t* x, const uint32_t* y, int k, uint32_t* c) {
+  int w = k + 1;
+  uint32_t* a = (uint32_t*)malloc((size_t)k * w * sizeof(uint32_t));
+  for (int j = 0; j < k; ++j) {
+    uint32_t pw = 1, xj = x[j] % Q_FIELD;
+    for (int d = 0; d < k; ++d) {
+      a[j * w + d] = pw;
+      pw = mulq(pw, xj);
+    }
+    a[j * w + k] = y[j] % Q_FIELD;
+  }
+  for (int col = 0; col < k; ++col) {
+    int piv = -1;
+    for (int r = col; r < k; ++r)
+      if (a[r * w + col] != 0) {
+        piv = r;
+        break;
+      }
+    if (piv < 0) {
+      free(a);
+      return 1;
+    }
+    if (piv != col)
+      for (int d = 0; d < w; ++d) {
+        uint32_t t = a[col * w + d];
+        a[col * w + d] = a[piv * w + d];
+        a[piv * w + d] = t;
+      }
+    uint32_t inv = oracle_mod_inverse32(a[col * w + col]);
+    for (int d = col; d < w; ++d) a[col * w + d] = mulq(a[col * w + d], inv);
+    for (int r = col + 1; r < k; ++r) {
+      uint32_t f = a[r * w + col];
+      if (f == 0) continue;
+      for (int d = col; d < w; ++d) a[r * w + d] = subq(a[r * w + d], mulq(f, a[col * w + d]));
+    }
+  }
+  for (int row = k - 1; row >= 0; --row) {
+    uint32_t s = a[row * w + k];
+    for (int d = row + 1; d < k; ++d) s = subq(s, mulq(a[row * w + d], c[d]));
+    c[row] = s;
+  }
+  free(a);
+  return 0;
+}
+
+/* Algorithm 3 over Z_q with the inverses of Algorithm 4: the second statement
+ * of the same polynomial. */
+int oracle_interpolate32_newton(const uint32_t* x, const uint32_t* y, int k, uint32_t* c) {
+  uint32_t* dd = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+  for (int j = 0; j < k; ++j) {
+    dd[j] = y[j] % Q_FIELD;
+    c[j] = 0;
+  }
+  for (int level = 1; level < k; ++level)
+    for (int i = k - 1; i >= level; --i) {
+      uint32_t num = subq(dd[i], dd[i - 1]);
+      uint32_t den = subq(x[i] % Q_FIELD, x[i - level] % Q_FIELD);
+      int64_t inv = oracle_mod_inverse_euclid((int64_t)den, (int64_t)Q_FIELD);
+      if (den == 0 || inv == (int64_t)Q_FIELD) {
+        free(dd);
+        return 1;
+      }
+      dd[i] = mulq(num, (uint32_t)inv);
+    }
+  c[0] = dd[k - 1];
+  int deg = 0;
+  for (int i = k - 2; i >= 0; --i) {
+    uint32_t neg_xi = subq(0, x[i] % Q_FIELD);
+    for (int d = deg + 1; d >= 1; --d) c[d] = addq(c[d - 1], mulq(c[d], neg_xi));
+    c[0] = addq(mulq(c[0], neg_xi), dd[i]);
+    ++deg;
+  }
+  free(dd);
+  return 0;
+}
+
+/* 2 + 4k bytes. */
+void oracle_encode32(uint32_t m, const uint32_t* c, int k, uint8_t* proof) {
+  uint32_t m16 = m & 0xFFFFu; /* 65536 -> 0 */
+  proof[0] = (uint8_t)(m16 & 0xFF);
+  proof[1] = (uint8_t)(m16 >> 8);
+  for (int d = 0; d < k; ++d)
+    for (int b = 0; b < 4; ++b) proof[2 + 4 * d + b] = (uint8_t)(c[d] >> (8 * b));
+}
+
+/* ST_OK or ST_BAD_PROOF (length not 2 + 4k, modulus outside the search
+ * range, a coefficient >= q).  *k_out = (len - 2) / 4. */
+int oracle_decode32(const uint8_t* proof, int64_t len, int* k_out, uint32_t* m_out, uint32_t* c) {
+  if (len < 6 || ((len - 2) & 3)) return ST_BAD_PROOF;
+  int k = (int)((len - 2) / 4);
+  uint32_t m = (uint32_t)proof[0] | ((uint32_t)proof[1] << 8);
+  if (m == 0) m = 65536u;
+  *k_out = k;
+  *m_out = m;
+  int bad = (m < M_LOW || m > M_HIGH);
+  for (int d = 0; d < k; ++d) {
+    c[d] = 0;
+    for (int b = 0; b < 4; ++b) c[d] |= (uint32_t)proof[2 + 4 * d + b] << (8 * b);
+    if (c[d] >= Q_FIELD) bad = 1;
+  }
+  return bad ? ST_BAD_PROOF : ST_OK;
+}
+
+/* top-k of an fp32 chunk with the full patterns of the selected elements. */
+static int topk_patterns32(const void* chunk, int rows, int hidden, int64_t row_stride, int k, uint32_t* idx,
+                           uint32_t* pattern) {
+  uint16_t* upper = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  int status = oracle_topk(chunk, 1, rows, hidden, row_stride, k, idx, upper);
+  free(upper);
+  if (status != ST_OK) return status;
+  for (int j = 0; j < k; ++j) {
+    int64_t t = idx[j] / (uint32_t)hidden, col = idx[j] % (uint32_t)hidden;
+    pattern[j] = ((const uint32_t*)chunk)[t * row_stride + col];
+  }
+  return ST_OK;
+}
+
+/* Algorithm 1 for one fp32 chunk over Z_q. */
+int oracle_build_chunk32(const void* chunk, int rows, int hidden, int64_t row_stride, int k, uint8_t* proof,
+                         int32_t* indices_opt) {
+  memset(proof, 0, 2 + 4 * (size_t)k);
+  if (indices_opt) memset(indices_opt, 0, (size_t)k * sizeof(int32_t));
+  uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* pattern = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* xs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* ys = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* coef = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  int status = topk_patterns32(chunk, rows, hidden, row_stride, k, idx, pattern);
+  if (status == ST_OK) {
+    if (indices_opt)
+      for (int j = 0; j < k; ++j) indices_opt[j] = (int32_t)idx[j];
+    uint32_t m = oracle_find_injective_modulus(idx, k, 0); /* residues below 2^16 are distinct in Z_q */
+    if (m == 0) {
+      status = ST_NO_MODULUS;
+    } else {
+      for (int j = 0; j < k; ++j) {
+        xs[j] = idx[j] % m;
+        ys[j] = pattern[j] % Q_FIELD;
+        if (pattern[j] >= Q_FIELD) status = ST_NONFINITE;
+      }
+      oracle_interpolate32(xs, ys, k, coef);
+      oracle_encode32(m, coef, k, proof);
+    }
+  }
+  free(idx);
+  free(pattern);
+  free(xs);
+  free(ys);
+  free(coef);
+  return status;
+}
+
+/* Algorithm 2 for one fp32 chunk over Z_q (thresholds of Section 5.2 for
+ * fp32 inference: 8 / 256 / 128 at k = 128). */
+void oracle_verify_chunk32(const void* chunk, int rows, int hidden, int64_t row_stride, int k,
+                           const uint8_t* proof, int t_exp, double t_mean, double t_median,
+                           int sign_in_exponent, const int32_t* gen_indices_opt, oracle_result* out) {
+  memset(out, 0, sizeof(*out));
+  out->topk_mismatch = -1;
+  uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* pattern = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* coef = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* diffs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  int kk = 0;
+  uint32_t m = 0;
+  int status = oracle_decode32(proof, 2 + 4 * (int64_t)k, &kk, &m, coef);
+  out->modulus = m;
+  if (status == ST_OK) status = topk_patterns32(chunk, rows, hidden, row_stride, k, idx, pattern);
+  if (status == ST_OK) {
+    uint32_t err_e = 0, n = 0;
+    uint64_t sum = 0;
+    for (int j = 0; j < k; ++j) {
+      uint32_t committed = oracle_horner32(coef, k, idx[j] % m);
+      uint32_t seen = pattern[j];
+      uint32_t e_p = committed >> 23, e_v = seen >> 23; /* sign + exponent, 9 bits */
+      if (!sign_in_exponent) {
+        e_p &= 0xFFu;
+        e_v &= 0xFFu;
+      }
+      uint32_t m_p = committed & 0x7FFFFFu, m_v = seen & 0x7FFFFFu;
+      if (e_p == e_v) {
+        uint32_t d = m_p > m_v ? m_p - m_v : m_v - m_p;
+        diffs[n++] = d;
+        sum += d;
+      } else {
+        ++err_e;
+      }
+    }
+    out->exp_mismatch = err_e;
+    out->n_match = n;
+    out->mant_diff_sum = (uint32_t)sum; /* k <= 256 differences below 2^23 */
+    if (n > 0) {
+      out->mant_mean = (double)sum / (double)n;
+      qsort(diffs, n, sizeof(uint32_t), ascending_u32);
+      out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
+    }
+    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    if (n == 0) reject = 1;
+    out->accept = reject ? 0 : 1;
+    if (gen_indices_opt) {
+      int common = 0;
+      for (int a = 0; a < k; ++a)
+        for (int b = 0; b < k; ++b)
+          if ((uint32_t)gen_indices_opt[a] == idx[b]) {
+            ++common;
+            break;
+          }
+      out->topk_mismatch = k - common;
+    }
+  }
+  out->status = (uint8_t)status;
+  if (status != ST_OK) out->accept = 0;
+  free(idx);
+  free(pattern);
+  free(coef);
+  free(diffs);
+}
+
 /* ------------------------------------------------------------------ */
 /* Batch drivers: chunks of chunk_len rows per sequence (Section 5.5:   */
 /* one proof per 32 new tokens), the last chunk of a sequence may be    */
@@ -476,10 +743,20 @@ typedef struct {
 static void* worker(void* arg) {
   job* jb = (job*)arg;
   size_t esz = jb->dtype == 0 ? 2 : 4;
-  size_t pbytes = 2 + 2 * (size_t)jb->k;
+  int wide = jb->dtype == 2; /* fp32 chunks committed over Z_q */
+  size_t pbytes = 2 + (wide ? 4 : 2) * (size_t)jb->k;
   for (int64_t c = jb->first + jb->tid; c < jb->last; c += jb->nthreads) {
     const void* chunk = jb->act + (size_t)jb->spans[c].row0 * (size_t)jb->row_stride * esz;
-    if (!jb->verify) {
+    if (!jb->verify && wide) {
+      jb->status[c] = (uint8_t)oracle_build_chunk32(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
+                                                    jb->proofs + (size_t)c * pbytes,
+                                                    jb->indices ? jb->indices + (size_t)c * jb->k : NULL);
+    } else if (wide) {
+      oracle_verify_chunk32(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
+                            jb->proofs_in + (size_t)c * pbytes, jb->t_exp, jb->t_mean, jb->t_median,
+                            jb->sign_in_exponent,
+                            jb->gen_indices ? jb->gen_indices + (size_t)c * jb->k : NULL, &jb->results[c]);
+    } else if (!jb->verify) {
       int st = oracle_build_chunk(chunk, jb->dtype, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
                                   jb->proofs + (size_t)c * pbytes,
                                   jb->indices ? jb->indices + (size_t)c * jb->k : NULL);
