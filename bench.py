@@ -33,7 +33,10 @@ WORKLOADS = {
     "8b": (64, 2048, 4096, 32, 128, 2),
     # every 4096-token prompt as ONE chunk of 33.5 M elements (selected in 64 segments and merged)
     "prompt70b": (64, 4096, 8192, 4096, 128, 6),
+    # fp32 activations committed whole over the 32-bit field (2 + 4k byte proofs, fp32 thresholds)
+    "70b-fp32-wide": (128, 4096, 8192, 32, 128, 7),
 }
+WIDE_WORKLOADS = ("70b-fp32-wide",)
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one toploc_select_kernel launch on the full
 # batch (ncu, profiles/launch_list_70b_shape.md); None where no capture of the current kernel exists
@@ -159,8 +162,10 @@ def aggregate_rate(units_per_rank, world, seconds):
 
 def workload_name(key):
     S, T, H, L, k, seed = WORKLOADS[key]
-    return "%s-shaped: %d seq x %d tok, H=%d bf16, L=%d, k=%d" % (
-        {"70b": "Llama-3.1-70B", "8b": "Llama-3.1-8B", "prompt70b": "Llama-3.1-70B prompt chunks"}[key], S, T, H, L, k)
+    return "%s-shaped: %d seq x %d tok, H=%d %s, L=%d, k=%d" % (
+        {"70b": "Llama-3.1-70B", "8b": "Llama-3.1-8B", "prompt70b": "Llama-3.1-70B prompt chunks",
+         "70b-fp32-wide": "Llama-3.1-70B"}[key], S, T, H,
+        "fp32 over the 32-bit field" if key in WIDE_WORKLOADS else "bf16", L, k)
 
 
 def main():
@@ -201,18 +206,25 @@ def main():
         return
 
     S, T, H, L, k, seed = WORKLOADS[args.workload]
-    act = synth.make_activations(S, T, H, torch.bfloat16, seed=seed + 10007 * rank, device=dev)
+    wide = args.workload in WIDE_WORKLOADS
+    field = tl.TOPLOC_FIELD_32 if wide else tl.TOPLOC_FIELD_16
+    # fp32: outlier magnitudes jittered -- exact ties at +-80 would be broken at random by any fp32 noise
+    act = synth.make_activations(S, T, H, torch.float32 if wide else torch.bfloat16, seed=seed + 10007 * rank,
+                                 device=dev, outliers="jitter" if wide else "fixed")
     # A prompt-sized bf16 chunk has thousands of elements tied at its largest magnitude, so the cut
     # is decided by index and any noise changes the selected set: that workload validates an exact copy.
     long_chunks = L * H > (1 << 19)
-    recomputed = act.clone() if long_chunks else synth.honest_noise(act, seed=seed + 1)
-    lay, _ = tl.make_layout(act, L, k, S, T)
+    # fp32 recomputation differs in the last mantissa bits only: relative 2^-22
+    noise_rel = 2.0 ** -22 if wide else 2.0 ** -8
+    recomputed = act.clone() if long_chunks else synth.honest_noise(act, seed=seed + 1, rel=noise_rel)
+    lay, _ = tl.make_layout(act, L, k, S, T, field=field)
+    lay_select, _ = tl.make_layout(act, L, k, S, T)   # toploc_select_topk hands out 16-bit patterns
     n = tl.toploc_num_chunks(lay)
     act_bytes = act.numel() * act.element_size()
-    proofs = torch.empty((n, tl.toploc_proof_bytes(k)), dtype=torch.uint8, device=dev)
+    proofs = torch.empty((n, tl.toploc_layout_proof_bytes(lay)), dtype=torch.uint8, device=dev)
     status = torch.empty((n,), dtype=torch.uint8, device=dev)
     results = torch.empty((n, 40), dtype=torch.uint8, device=dev)
-    thr = tl.default_thresholds(k)
+    thr = tl.default_thresholds(k, field=field)
     workspace = torch.empty(tl.toploc_workspace_bytes(lay), dtype=torch.uint8, device=dev)
 
     def step(ev=None):
@@ -258,12 +270,12 @@ def main():
     sel_pat = torch.empty((n, k), dtype=torch.int16, device=dev)
     sel_steps = min(args.steps, 20)
     for _ in range(3):
-        tl.toploc_select_topk(recomputed, lay, sel_idx, sel_pat, status, workspace=workspace)
+        tl.toploc_select_topk(recomputed, lay_select, sel_idx, sel_pat, status, workspace=workspace)
     torch.cuda.synchronize()
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s0.record()
     for _ in range(sel_steps):
-        tl.toploc_select_topk(recomputed, lay, sel_idx, sel_pat, status, workspace=workspace)
+        tl.toploc_select_topk(recomputed, lay_select, sel_idx, sel_pat, status, workspace=workspace)
     s1.record()
     torch.cuda.synchronize()
     select_ms = max_over_ranks([s0.elapsed_time(s1) / sel_steps], dev, world)[0]
@@ -291,9 +303,10 @@ def main():
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u32", "data": "synthetic",
-        "config": {"workload": workload_name(args.workload), "chunks": n, "proof_bytes": 2 + 2 * k,
+        "config": {"workload": workload_name(args.workload), "chunks": n, "proof_bytes": proofs.shape[1],
                    "activation_bytes": act_bytes, "l2": "inputs larger than L2 (no flush needed)",
-                   "recomputed": "exact copy" if long_chunks else "honest reorder noise, relative 2^-8",
+                   "recomputed": "exact copy" if long_chunks else "honest reorder noise, relative 2^%d" % (-22 if wide else -8),
+                   "outliers": "jittered magnitudes" if wide else "+-80 on fixed channels",
                    "parallelism": "chunks sharded, no collective"},
         "generate": {"ms": build_ms, "chunks_per_s": n / (build_ms * 1e-3), "GB_per_s": build_gbs,
                      "frac_of_measured_copy_peak": build_gbs / peak, "frac_of_8TBs_nominal": build_gbs / 8000.0},
@@ -301,7 +314,7 @@ def main():
                    "frac_of_measured_copy_peak": verify_gbs / peak, "frac_of_8TBs_nominal": verify_gbs / 8000.0},
         "activation_GB_per_s": 2 * act_bytes / (ms_per_step * 1e-3) / 1e9,
         # dominant kernel (87 % of the library's GPU time): algorithmic bytes = the activations, once
-        "roofline": {"bound": "hbm", "kernel": "toploc_select_kernel<bf16, flat>",
+        "roofline": {"bound": "hbm", "kernel": "toploc_select_kernel<%s, flat>" % ("fp32" if wide else "bf16"),
                      "achieved": select_gbs, "peak": peak, "peak_kind": peak_kind + " (torch copy, burst)",
                      "unit": "GB/s", "frac": select_gbs / peak, "ms_per_launch": select_ms,
                      "algorithmic_bytes_per_launch": act_bytes,
@@ -316,7 +329,7 @@ def main():
         "e2e": e2e,
     }
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = cpu_baseline(act, recomputed, S, T, H, L, k)
+        line["cpu_baseline"] = cpu_baseline(act, recomputed, S, T, H, L, k, wide)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -376,7 +389,7 @@ def measure_e2e(tl, act, lay, n, k, thr, dev, steps, world):
     except RuntimeError as e:
         return {"value": None, "unit": "chunks/s", "error": "pinned allocation failed: %s" % e}
     h_act.copy_(act)
-    h_proofs = torch.empty((n, 2 + 2 * k), dtype=torch.uint8, pin_memory=True)
+    h_proofs = torch.empty((n, tl.toploc_layout_proof_bytes(lay)), dtype=torch.uint8, pin_memory=True)
     h_status = torch.empty((n,), dtype=torch.uint8, pin_memory=True)
     h_results = torch.empty((n, 40), dtype=torch.uint8, pin_memory=True)
     staging = torch.empty(max(tl.toploc_staging_bytes(lay) * 8, 1 << 20), dtype=torch.uint8, device=dev)
@@ -395,13 +408,13 @@ def measure_e2e(tl, act, lay, n, k, thr, dev, steps, world):
     torch.cuda.synchronize()
     dt = (time.perf_counter() - t0) / steps
     dt = max_over_ranks([dt], dev, world)[0]
-    proofs_b = n * (2 + 2 * k)
+    proofs_b = n * tl.toploc_layout_proof_bytes(lay)
     return {"value": aggregate_rate(n, world, dt), "unit": "chunks/s", "ms_per_step": dt * 1e3, "steps": steps,
             "h2d_bytes_per_step": 2 * act_bytes + proofs_b, "d2h_bytes_per_step": proofs_b + n + n * 40,
             "note": "build then verify (identical copy) from pinned host memory; PCIe-bound"}
 
 
-def cpu_baseline(act, recomputed, S, T, H, L, k):
+def cpu_baseline(act, recomputed, S, T, H, L, k, wide=False):
     import oracle
     from paper_2501_16007_b200 import synth
     host = synth.host_patterns(act[:T])
@@ -409,12 +422,14 @@ def cpu_baseline(act, recomputed, S, T, H, L, k):
     cores = oracle.default_threads()
     chunks = T // L
     t0 = time.perf_counter()
-    proofs, status, idx = oracle.build_proofs(host, L, k, 1, T, threads=cores)
+    proofs, status, idx = oracle.build_proofs(host, L, k, 1, T, threads=cores, wide=wide)
     t1 = time.perf_counter()
-    oracle.verify_proofs(host_rec, proofs, L, k, 1, T, gen_indices=idx, threads=cores)
+    oracle.verify_proofs(host_rec, proofs, L, k, 1, T, gen_indices=idx, threads=cores, wide=wide,
+                         **({"t_exp": 8 * k // 128, "t_mean": 256.0, "t_median": 128.0} if wide else {}))
     t2 = time.perf_counter()
     return {"value": chunks / (t2 - t0), "unit": "chunks/s", "cores": cores, "kind": "oracle",
-            "sample": "first sequence: %d chunks of %d x %d bf16, build + verify" % (chunks, L, H),
+            "sample": "first sequence: %d chunks of %d x %d %s, build + verify" % (
+            chunks, L, H, "fp32 (32-bit field)" if wide else "bf16"),
             "generate_chunks_per_s": chunks / (t1 - t0), "verify_chunks_per_s": chunks / (t2 - t1)}
 
 

@@ -37,6 +37,21 @@ extern "C" {
 #define TOPLOC_DTYPE_BF16 0
 #define TOPLOC_DTYPE_FP32 1
 
+/* Field of the committed polynomial.  TOPLOC_FIELD_16: Z_p with p = 65521,
+ * 2-byte coefficients, proofs of 2 + 2k bytes (bf16 chunks; fp32 chunks scaled
+ * to 16 bits as above).  TOPLOC_FIELD_32, fp32 chunks only: every selected
+ * value commits its whole 32-bit pattern, the arithmetic runs in Z_q with
+ * q = 4294967291 = 2^32 - 5 (the largest prime below 2^32; the subroutines
+ * appendix names 2^32 as the modulus size for 32-bit types), coefficients take
+ * 4 bytes little-endian and a proof 2 + 4k bytes.  Validation then compares
+ * fp32 bit fields (sign, 8 exponent bits, 23 mantissa bits), which is what the
+ * thresholds "for fp32 inference" of Section 5.2 (8 / 256 / 128) are stated
+ * on.  The paper prints neither q nor this layout; they are this library's
+ * reading. */
+#define TOPLOC_FIELD_16 0
+#define TOPLOC_FIELD_32 1
+#define TOPLOC_FIELD_32_PRIME 4294967291u
+
 /* Largest k the kernels are built for and largest chunk (elements; only chunks
  * the layout really contains count, so chunk_len may exceed every sequence).
  * A chunk of more than 2^19 elements -- a prompt committed as one chunk,
@@ -81,7 +96,7 @@ typedef struct {
   int32_t chunk_len;          /* L > 0 tokens per chunk (32 in Section 5.5) */
   int32_t k;                  /* 1..TOPLOC_MAX_K (128 in the paper) */
   int32_t num_seqs;           /* > 0 */
-  int32_t reserved;           /* must be 0 */
+  int32_t field;              /* TOPLOC_FIELD_* (0 = 16-bit field, the default) */
   int64_t tokens_per_seq;     /* uniform sequence length; used when seq_offsets == NULL */
   const int64_t* seq_offsets; /* HOST, optional: num_seqs + 1 ascending row offsets (ragged batch);
                                  read before the call returns */
@@ -126,6 +141,10 @@ int64_t toploc_num_chunks(const toploc_layout* lay);
 /* 2 + 2k: a 2-byte modulus and k 2-byte coefficients (Section 4, Section 5.7). */
 size_t toploc_proof_bytes(int32_t k);
 
+/* Proof bytes per chunk of this layout: 2 + 2k, or 2 + 4k with TOPLOC_FIELD_32;
+ * 0 for an invalid layout.  Every proof buffer is [num_chunks, this many]. */
+size_t toploc_layout_proof_bytes(const toploc_layout* lay);
+
 /* Bytes of device scratch build/verify need for this layout: the selected
  * (index, pattern) pairs of every chunk (6k + 1 bytes per chunk) that the
  * select kernel hands to the arithmetic kernel, plus a per-chunk row table for
@@ -160,7 +179,8 @@ const char* toploc_error_string(int return_code);
  *
  * d_act         DEVICE  activations, layout as described by *lay
  * lay           HOST    read before return
- * d_proofs      DEVICE  out, [num_chunks, 2 + 2k] bytes, chunks in batch order
+ * d_proofs      DEVICE  out, [num_chunks, toploc_layout_proof_bytes(lay)] bytes (2 + 2k; 2 + 4k with
+ *                        TOPLOC_FIELD_32), chunks in batch order
  *                       (sequence-major); zero-filled for a chunk whose status
  *                       is NO_INJECTIVE_MODULUS or K_EXCEEDS_CHUNK
  * d_status      DEVICE  out, [num_chunks] TOPLOC_CHUNK_* bytes
@@ -187,7 +207,7 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
  * toploc_thresholds.
  *
  * d_act             DEVICE  recomputed activations (same layout as at build)
- * d_proofs          DEVICE  [num_chunks, 2 + 2k] proofs
+ * d_proofs          DEVICE  [num_chunks, toploc_layout_proof_bytes(lay)] proofs
  * thr               HOST    thresholds, read before return
  * d_results         DEVICE  out, [num_chunks] toploc_chunk_result
  * d_gen_indices_opt DEVICE  optional: the generator's [num_chunks, k] indices
@@ -208,6 +228,7 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
  * d_sel_indices         DEVICE out, [num_chunks, k] u32: the selected flat indices of each
  *                       chunk, as a set (order within a chunk is unspecified)
  * d_sel_patterns        DEVICE out, [num_chunks, k] u16: their 16-bit patterns, same order
+ *                        (TOPLOC_FIELD_16 layouts only, else TOPLOC_ERR_UNSUPPORTED)
  * d_status              DEVICE out, [num_chunks]: TOPLOC_CHUNK_OK or K_EXCEEDS_CHUNK (whose rows
  *                       of the two arrays above are left untouched)
  * d_ranked_indices_opt  DEVICE out, optional: [num_chunks, k] i32 indices in rank order

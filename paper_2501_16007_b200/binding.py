@@ -13,13 +13,17 @@ import torch
 __all__ = [
     "TOPLOC_DTYPE_BF16", "TOPLOC_DTYPE_FP32", "TOPLOC_MAX_K", "RESULT_DTYPE", "ToplocError",
     "ToplocLayout", "ToplocThresholds", "make_layout", "library_path", "load_library",
-    "toploc_num_chunks", "toploc_proof_bytes", "toploc_workspace_bytes", "toploc_staging_bytes",
+    "toploc_num_chunks", "toploc_proof_bytes", "toploc_layout_proof_bytes", "toploc_workspace_bytes",
+    "toploc_staging_bytes", "TOPLOC_FIELD_16", "TOPLOC_FIELD_32", "TOPLOC_FIELD_32_PRIME",
     "toploc_get_constants", "toploc_status_string", "toploc_error_string",
     "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
     "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES", "toploc_select_topk",
 ]
 
 TOPLOC_DTYPE_BF16 = 0
+TOPLOC_FIELD_16 = 0
+TOPLOC_FIELD_32 = 1
+TOPLOC_FIELD_32_PRIME = 4294967291
 TOPLOC_DTYPE_FP32 = 1
 TOPLOC_MAX_K = 256
 TOPLOC_BUILTIN_SCRATCH_BYTES = 8 << 20
@@ -38,7 +42,7 @@ class ToplocError(RuntimeError):
 class ToplocLayout(ctypes.Structure):
     _fields_ = [
         ("dtype", ctypes.c_int32), ("hidden", ctypes.c_int32), ("chunk_len", ctypes.c_int32),
-        ("k", ctypes.c_int32), ("num_seqs", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("k", ctypes.c_int32), ("num_seqs", ctypes.c_int32), ("field", ctypes.c_int32),
         ("tokens_per_seq", ctypes.c_int64), ("seq_offsets", ctypes.POINTER(ctypes.c_int64)),
         ("row_stride", ctypes.c_int64),
     ]
@@ -73,6 +77,7 @@ def load_library():
     lay_p, thr_p = ctypes.POINTER(ToplocLayout), ctypes.POINTER(ToplocThresholds)
     lib.toploc_num_chunks.restype, lib.toploc_num_chunks.argtypes = i64, [lay_p]
     lib.toploc_proof_bytes.restype, lib.toploc_proof_bytes.argtypes = sz, [i32]
+    lib.toploc_layout_proof_bytes.restype = sz
     lib.toploc_workspace_bytes.restype, lib.toploc_workspace_bytes.argtypes = sz, [lay_p]
     lib.toploc_staging_bytes.restype, lib.toploc_staging_bytes.argtypes = sz, [lay_p]
     lib.toploc_get_constants.restype = None
@@ -108,8 +113,9 @@ def _dtype_code(t):
     raise ToplocError("activations must be bfloat16 or float32, got %s" % t.dtype)
 
 
-def make_layout(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None):
+def make_layout(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None, field=TOPLOC_FIELD_16):
     """Layout of a 2-D activation tensor [total_tokens, hidden] (last dimension contiguous).
+    field=TOPLOC_FIELD_32 (float32 activations only): whole patterns over Z_q, proofs of 2 + 4k bytes.
 
     Returns (layout, keepalive): keepalive holds the host seq_offsets array the struct points to."""
     if act.dim() != 2 or act.stride(1) != 1:
@@ -120,7 +126,7 @@ def make_layout(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None)
     lay.chunk_len = chunk_len
     lay.k = k
     lay.num_seqs = num_seqs
-    lay.reserved = 0
+    lay.field = field
     lay.tokens_per_seq = tokens_per_seq
     lay.row_stride = act.stride(0) if act.shape[0] > 1 else act.shape[1]
     keep = None
@@ -146,6 +152,10 @@ def toploc_num_chunks(lay):
 
 def toploc_proof_bytes(k):
     return int(load_library().toploc_proof_bytes(k))
+
+
+def toploc_layout_proof_bytes(lay):
+    return int(load_library().toploc_layout_proof_bytes(ctypes.byref(lay)))
 
 
 def toploc_workspace_bytes(lay):
@@ -195,7 +205,7 @@ def toploc_build_proofs(act, lay, proofs=None, status=None, indices=None, worksp
     if not act.is_cuda:
         raise ToplocError("toploc_build_proofs needs a CUDA tensor (use toploc_build_proofs_host)")
     n = toploc_num_chunks(lay)
-    pb = toploc_proof_bytes(lay.k)
+    pb = toploc_layout_proof_bytes(lay)
     dev = act.device
     if proofs is None:
         proofs = torch.empty((n, pb), dtype=torch.uint8, device=dev)
@@ -226,7 +236,7 @@ def toploc_verify_proofs(act, lay, proofs, thresholds=None, results=None, gen_in
     thr = thresholds if thresholds is not None else default_thresholds()
     if results is None:
         results = torch.empty((n, RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
-    assert proofs.is_contiguous() and proofs.numel() == n * toploc_proof_bytes(lay.k)
+    assert proofs.is_contiguous() and proofs.numel() == n * toploc_layout_proof_bytes(lay)
     assert results.is_contiguous() and results.numel() == n * RESULT_DTYPE.itemsize
     assert gen_indices is None or (gen_indices.is_contiguous() and gen_indices.dtype == torch.int32
                                    and gen_indices.numel() == n * lay.k)
@@ -239,14 +249,16 @@ def toploc_verify_proofs(act, lay, proofs, thresholds=None, results=None, gen_in
     return results
 
 
-def default_thresholds(k=128, sign_in_exponent=True):
-    """Section 5.2 thresholds for bf16 (38 / 10 / 8 at k = 128); the exponent threshold
-    scales with k for other proof sizes."""
+def default_thresholds(k=128, sign_in_exponent=True, field=TOPLOC_FIELD_16):
+    """Section 5.2 thresholds: 38 / 10 / 8 at k = 128 for bf16 (and fp32 scaled to 16 bits), 8 / 256 / 128
+    for fp32 inference (TOPLOC_FIELD_32, 23-bit mantissas); the exponent threshold scales with k for
+    other proof sizes."""
     thr = ToplocThresholds()
-    thr.t_exp = (38 * k) // 128
+    wide = field == TOPLOC_FIELD_32
+    thr.t_exp = ((8 if wide else 38) * k) // 128
     thr.sign_in_exponent = 1 if sign_in_exponent else 0
-    thr.t_mean = 10.0
-    thr.t_median = 8.0
+    thr.t_mean = 256.0 if wide else 10.0
+    thr.t_median = 128.0 if wide else 8.0
     return thr
 
 

@@ -32,6 +32,7 @@ namespace {
 // constants of the method
 // ---------------------------------------------------------------------------
 constexpr uint32_t kPrime = 65521u;      // field modulus: largest prime below 2^16
+constexpr uint32_t kPrime32 = 4294967291u;  // 32-bit field (fp32 chunks committing whole patterns): 2^32 - 5
 constexpr uint32_t kModHigh = 65536u;    // Algorithm 6 scans 65536 down to 2^15 + 1
 constexpr uint32_t kModLow = 32769u;
 
@@ -95,12 +96,17 @@ struct BatchParams {
   int chunk_len;
   int k;
   int chunks_per_seq;
+  int coef_bytes;              // 2: coefficients in Z_p; 4: fp32 chunks over Z_q, q = 2^32 - 5
 };
+
+__device__ __forceinline__ size_t proof_stride(const BatchParams& bp) { return 2 + (size_t)bp.coef_bytes * bp.k; }
+__device__ __forceinline__ int proof_words(const BatchParams& bp) { return 1 + (bp.coef_bytes / 2) * bp.k; }
 
 // What the select kernel leaves behind for the interpolation kernel (or hands to the caller).
 struct Selection {
   uint32_t* idx;       // [num_chunks, k] selected flat indices
   uint16_t* bits;      // [num_chunks, k] their 16-bit patterns
+  uint32_t* bits32;    // 32-bit field: [num_chunks, k] their whole patterns instead
   uint8_t* status;     // [num_chunks] TOPLOC_CHUNK_*; the caller's d_status during proof generation
   uint8_t* proofs;     // proof generation only: receives the modulus (or zeros)
   int32_t* indices;    // optional: indices in rank order
@@ -111,7 +117,7 @@ struct MergeParams {
   const ChunkSegments* chunks;
   const ChunkSpan* segs;
   const uint32_t* seg_idx;      // [num_segs, k]
-  const uint16_t* seg_bits;     // [num_segs, k]
+  const uint16_t* seg_bits;     // [num_segs, k] (unused by fp32 chunks, whose patterns are read again)
   const uint8_t* seg_status;    // [num_segs]
   unsigned long long* words;    // [num_segs, k] scratch: the candidates of a chunk as ranking words
 };
@@ -705,11 +711,13 @@ static_assert(kGenerator != 0 && mul_mod(kGenerator, kGeneratorInv) == 1u, "gene
 
 // Algorithm 6: largest m in [2^15 + 1, 2^16] for which the selected indices
 // stay distinct as (index mod m) mod p -- the second reduction because the
-// x-coordinates live in Z_p and m may exceed p.  Returns 0 if there is none.
+// x-coordinates live in Z_p and m may exceed p (in the 32-bit field m < q and
+// Algorithm 6 applies as printed).  Returns 0 if there is none.
 // idx[e] is the flat index of point 32 e + lane.  The selection in shared
 // memory is consumed: the tile ring and the candidate buffer become the
 // 65536-bit set of residues seen.
-__device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32_t (&idx)[kMaxK / kThreads]) {
+__device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32_t (&idx)[kMaxK / kThreads],
+                                           bool wide_field) {
   const int tid = threadIdx.x;
   uint32_t res[kMaxK / kThreads];
 #pragma unroll
@@ -727,7 +735,7 @@ __device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32
       int j = tid + e * kThreads;
       if (j < k) {
         uint32_t r = idx[e] % m;
-        if (r >= kPrime) r -= kPrime;
+        if (!wide_field && r >= kPrime) r -= kPrime;  // every residue is below q = 2^32 - 5 as it is
         res[e] = r;
         uint32_t bit = 1u << (r & 31u);
         dup |= atomicOr(&seen[r >> 5], bit) & bit;
@@ -783,14 +791,15 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
   const int tid = threadIdx.x;
   const long long chunk = blockIdx.x;
   const int k = bp.k;
-  uint16_t* proof = sel.proofs ? reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 2 * (size_t)k)) : nullptr;
+  uint16_t* proof = sel.proofs ? reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_stride(bp)) : nullptr;
+  const bool wide = DT == 1 && bp.coef_bytes == 4;
   int32_t* indices = sel.indices ? sel.indices + chunk * k : nullptr;
 
   const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
   const long long n_elems = (long long)pl.rows * bp.hidden;
   if (n_elems < k) {
     if (proof)
-      for (int i = tid; i < k + 1; i += kThreads) proof[i] = 0;
+      for (int i = tid; i < proof_words(bp); i += kThreads) proof[i] = 0;
     if (indices)
       for (int i = tid; i < k; i += kThreads) indices[i] = 0;
     if (tid == 0) sel.status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
@@ -810,10 +819,16 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
     const uint32_t key = (uint32_t)(cj >> (kIdxBits + 1));
     const uint32_t sign = (uint32_t)cj & 1u;
     const uint32_t flat = kIdxMask - ((uint32_t)(cj >> 1) & kIdxMask);
-    const uint32_t bits = (sign << 15) | (DT == 0 ? key : (key >> 16));
-    unrepresentable |= bits >= kPrime;
     sel.idx[chunk * k + j] = flat;
-    sel.bits[chunk * k + j] = (uint16_t)bits;
+    if (wide) {
+      const uint32_t pattern = (sign << 31) | key;
+      unrepresentable |= pattern >= kPrime32;
+      sel.bits32[chunk * k + j] = pattern;
+    } else {
+      const uint32_t bits = (sign << 15) | (DT == 0 ? key : (key >> 16));
+      unrepresentable |= bits >= kPrime;
+      sel.bits[chunk * k + j] = (uint16_t)bits;
+    }
     if (indices) {
       int rank = 0;  // position = number of better candidates
       for (int i = 0; i < k; ++i) rank += sh.cand[i] > cj;
@@ -831,9 +846,9 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
     const int j = tid + e * kThreads;
     picked[e] = j < k ? kIdxMask - ((uint32_t)(sh.cand[j] >> 1) & kIdxMask) : 0u;
   }
-  const uint32_t m = find_injective_modulus(sh, k, picked);
+  const uint32_t m = find_injective_modulus(sh, k, picked, wide);
   if (m == 0) {
-    for (int i = tid; i < k + 1; i += kThreads) proof[i] = 0;
+    for (int i = tid; i < proof_words(bp); i += kThreads) proof[i] = 0;
     if (tid == 0) sel.status[chunk] = TOPLOC_CHUNK_NO_INJECTIVE_MODULUS;
     return;
   }
@@ -1124,8 +1139,278 @@ __device__ __forceinline__ void evaluate_warp(SelectShared& sh, int k, long long
   }
 }
 
+// ---------------------------------------------------------------------------
+// The 32-bit field: fp32 chunks that commit whole patterns work in Z_q,
+// q = 2^32 - 5 (products are 64 bits wide and 2^32 = 5 folds them back).  A
+// table of inverses is out of reach, so Algorithm 3 is arranged around k
+// inversions per chunk instead of k^2 / 2.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t reduce_q(unsigned long long t) {
+  unsigned long long s = (t & 0xFFFFFFFFull) + 5ull * (t >> 32);  // < 6 * 2^32
+  s = (s & 0xFFFFFFFFull) + 5ull * (s >> 32);                     // < 2^32 + 25 < 2q
+  return (uint32_t)(s >= kPrime32 ? s - kPrime32 : s);
+}
+__device__ __forceinline__ uint32_t mul_q(uint32_t a, uint32_t b) { return reduce_q((unsigned long long)a * b); }
+__device__ __forceinline__ uint32_t mad_q(uint32_t a, uint32_t b, uint32_t c) {
+  return reduce_q((unsigned long long)a * b + c);
+}
+__device__ __forceinline__ uint32_t sub_q(uint32_t a, uint32_t b) { return a >= b ? a - b : a + (kPrime32 - b); }
+
+// a^(q - 2): the inverse of a != 0 in Z_q (0 for a = 0).  The inverse is unique,
+// so this agrees with the extended Euclid of Algorithm 4.
+__device__ __forceinline__ uint32_t inv_q(uint32_t a) {
+  uint32_t r = a;
+#pragma unroll 1
+  for (int bit = 30; bit >= 0; --bit) {
+    r = mul_q(r, r);
+    if (((kPrime32 - 2u) >> bit) & 1u) r = mul_q(r, a);
+  }
+  return r;
+}
+
+// Algorithm 3 (InterpolateModPolynomial) over Z_q for one chunk, by one warp.
+// Point j lives in lane j % 32, slot j / 32.  The Newton coefficient of point i is
+//   a_i = (y_i - P_{i-1}(x_i)) / N_i(x_i),   N_i(x) = prod_{l < i} (x - x_l),
+// where P_{i-1} interpolates the first i points.  A first sweep forms every
+// denominator N_j(x_j) (they do not depend on y) and inverts the k of them; a
+// second sweep carries, for every later point j, the partial sum
+// S_j = P_{i-1}(x_j) and the partial product N_i(x_j); only a_i and x_i are
+// broadcast per step.  The Newton form is then multiplied out from the inside,
+//   P <- P * (x - x_i) + a_i  for i = k-2 .. 0,
+// with coefficient d in lane d / SLOTS, slot d % SLOTS, so the shift by one
+// degree stays inside a lane except for one value per lane and step.
+// row_x / row_a: this warp's scratch rows of kMaxK words in shared memory.
+template <int SLOTS>
+__device__ __forceinline__ void interpolate_warp_q(int k, const uint32_t (&x)[SLOTS], const uint32_t (&y)[SLOTS],
+                                                   uint32_t* row_x, uint32_t* row_a, uint16_t* proof) {
+  const int lane = threadIdx.x & 31;
+  constexpr uint32_t kFull = 0xFFFFFFFFu;
+  uint32_t den[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) den[s] = 1u;
+#pragma unroll
+  for (int b = 0; b < SLOTS; ++b) {
+    const int steps = min(32, k - 1 - 32 * b);  // points i = 32b + ii with i + 1 < k
+#pragma unroll 1
+    for (int ii = 0; ii < steps; ++ii) {
+      const uint32_t xi = __shfl_sync(kFull, x[b], ii);
+      den[b] = mul_q(den[b], lane > ii ? sub_q(x[b], xi) : 1u);
+#pragma unroll
+      for (int s = b + 1; s < SLOTS; ++s) den[s] = mul_q(den[s], sub_q(x[s], xi));
+    }
+  }
+  uint32_t inv_den[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) inv_den[s] = inv_q(den[s]);
+
+  uint32_t part[SLOTS], prod[SLOTS];  // S_j and N_i(x_j)
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    part[s] = 0u;
+    prod[s] = 1u;
+    if (s * 32 + lane < k) row_x[s * 32 + lane] = x[s];
+  }
+#pragma unroll
+  for (int b = 0; b < SLOTS; ++b) {
+    const int steps = min(32, k - 32 * b);  // includes the last point, which only yields its a
+#pragma unroll 1
+    for (int ii = 0; ii < steps; ++ii) {
+      // every lane forms the quotient of its own slot-b point; lane ii's is a_i
+      const uint32_t quot = mul_q(sub_q(y[b], part[b]), inv_den[b]);
+      const uint32_t a_i = __shfl_sync(kFull, quot, ii);
+      const uint32_t xi = __shfl_sync(kFull, x[b], ii);
+      if (lane == ii) row_a[32 * b + ii] = a_i;
+      const bool later = lane > ii;
+      const uint32_t part_b = mad_q(a_i, prod[b], part[b]);
+      const uint32_t prod_b = mul_q(prod[b], sub_q(x[b], xi));
+      part[b] = later ? part_b : part[b];
+      prod[b] = later ? prod_b : prod[b];
+#pragma unroll
+      for (int s = b + 1; s < SLOTS; ++s) {
+        part[s] = mad_q(a_i, prod[s], part[s]);
+        prod[s] = mul_q(prod[s], sub_q(x[s], xi));
+      }
+    }
+  }
+  __syncwarp();
+  uint32_t co[SLOTS];
+#pragma unroll
+  for (int b = 0; b < SLOTS; ++b) co[b] = 0u;
+  if (lane == 0) co[0] = row_a[k - 1];
+#pragma unroll 1
+  for (int i = k - 2; i >= 0; --i) {
+    const uint32_t neg_x = sub_q(0u, row_x[i]);
+    const uint32_t a_i = row_a[i];
+    // coefficient d takes  c[d-1] + (-x_i) c[d];  entries above the current degree are 0 and stay 0
+    uint32_t carry = __shfl_up_sync(kFull, co[SLOTS - 1], 1);
+    if (lane == 0) carry = a_i;
+#pragma unroll
+    for (int b = SLOTS - 1; b >= 1; --b) co[b] = mad_q(co[b], neg_x, co[b - 1]);
+    co[0] = mad_q(co[0], neg_x, carry);
+  }
+  // proof bytes 2 + 4d .. 5 + 4d: coefficient of degree d, little-endian (the proof is 2-byte aligned)
+#pragma unroll
+  for (int b = 0; b < SLOTS; ++b) {
+    const int d = lane * SLOTS + b;
+    if (d < k) {
+      proof[1 + 2 * d] = (uint16_t)(co[b] & 0xFFFFu);
+      proof[2 + 2 * d] = (uint16_t)(co[b] >> 16);
+    }
+  }
+}
+
+constexpr int kInterpQWarps = 8;  // 32-bit field interpolation: warps (chunks) per block
+
+// InterpolateModPolynomial() and encode() of Algorithm 1 over Z_q for every
+// chunk the select (or merge) kernel finished, one warp per chunk.
+template <int SLOTS>
+__device__ __forceinline__ void interpolate_chunk_q(const Selection& sel, int k, long long chunk, uint32_t* rows) {
+  const int lane = threadIdx.x & 31;
+  uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 4 * (size_t)k));
+  uint32_t m = proof[0];
+  if (m == 0) m = 65536u;
+  uint32_t x[SLOTS], y[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int j = s * 32 + lane;
+    x[s] = 0;
+    y[s] = 0;
+    if (j < k) {
+      x[s] = sel.idx[chunk * k + j] % m;  // i_m = i mod m (below 2^16 < q)
+      const uint32_t pattern = sel.bits32[chunk * k + j];
+      y[s] = pattern >= kPrime32 ? pattern - kPrime32 : pattern;  // "dd <- y mod M"
+    }
+  }
+  interpolate_warp_q<SLOTS>(k, x, y, rows, rows + kMaxK, proof);
+}
+
+__global__ void __launch_bounds__(kInterpQWarps * 32)
+toploc_interpolate_q_kernel(Selection sel, int k, long long num_chunks) {
+  __shared__ uint32_t rows[kInterpQWarps][2 * kMaxK];
+  const int warp = threadIdx.x >> 5;
+  const long long chunk = (long long)blockIdx.x * kInterpQWarps + warp;
+  if (chunk >= num_chunks) return;
+  const uint8_t st = sel.status[chunk];
+  if (st == TOPLOC_CHUNK_NO_INJECTIVE_MODULUS || st == TOPLOC_CHUNK_K_EXCEEDS_CHUNK) return;
+  if (k <= 32) interpolate_chunk_q<1>(sel, k, chunk, rows[warp]);
+  else if (k <= 64) interpolate_chunk_q<2>(sel, k, chunk, rows[warp]);
+  else if (k <= 128) interpolate_chunk_q<4>(sel, k, chunk, rows[warp]);
+  else interpolate_chunk_q<kMaxSlots>(sel, k, chunk, rows[warp]);
+}
+
+// Algorithm 2 after the selection, over Z_q, for one chunk whose selected
+// indices and whole fp32 patterns are in registers: Horner evaluation
+// (Algorithm 5), extractBits() (bit 31 sign, bits 30..23 exponent, bits 22..0
+// mantissa), error accumulation, verdict.  The median of up to k 23-bit
+// differences is found by rank counting (no histogram fits).
+template <int SLOTS>
+__device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long long chunk, const uint32_t (&idx)[SLOTS],
+                                                const uint32_t (&pattern)[SLOTS], const VerifyIo& io,
+                                                toploc_chunk_result res) {
+  const int lane = threadIdx.x;
+  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 4 * (size_t)k));
+  // the selection has left shared memory, so the ring is free: three rows of kMaxK words
+  uint32_t* coef = reinterpret_cast<uint32_t*>(sh.ring);
+  uint32_t* gen = coef + kMaxK;
+  uint32_t* diffs = gen + kMaxK;
+  constexpr uint32_t kNoMatch = 0xFFFFFFFFu;  // larger than any 23-bit difference
+  warp_barrier();
+  for (int d = lane; d < k; d += 32) coef[d] = (uint32_t)proof[1 + 2 * d] | ((uint32_t)proof[2 + 2 * d] << 16);
+  if (io.gen_indices)
+    for (int j = lane; j < k; j += 32) gen[j] = (uint32_t)io.gen_indices[chunk * k + j];
+  warp_barrier();
+
+  const uint32_t m = res.modulus;
+  uint32_t x[SLOTS], acc[SLOTS];
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    x[s] = idx[s] % m;
+    acc[s] = coef[k - 1];  // Horner, highest degree first
+  }
+#pragma unroll 2
+  for (int d = k - 2; d >= 0; --d) {
+    const uint32_t cd = coef[d];
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) acc[s] = mad_q(acc[s], x[s], cd);
+  }
+  uint32_t err_e = 0, diff_sum = 0, common = 0;
+#pragma unroll
+  for (int s = 0; s < SLOTS; ++s) {
+    const int j = s * 32 + lane;
+    if (j >= k) continue;
+    const uint32_t seen = pattern[s];
+    uint32_t e_p = acc[s] >> 23, e_v = seen >> 23;  // sign + 8 exponent bits
+    if (!io.sign_in_exponent) {
+      e_p &= 0xFFu;
+      e_v &= 0xFFu;
+    }
+    uint32_t diff = kNoMatch;
+    if (e_p == e_v) {
+      const uint32_t m_p = acc[s] & 0x7FFFFFu, m_v = seen & 0x7FFFFFu;
+      diff = m_p > m_v ? m_p - m_v : m_v - m_p;
+      diff_sum += diff;  // at most 256 differences below 2^23
+    } else {
+      ++err_e;
+    }
+    diffs[j] = diff;
+    if (io.gen_indices) {
+      uint32_t hit = 0;
+      for (int i = 0; i < k; ++i) hit |= gen[i] == idx[s];
+      common += hit;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    err_e += __shfl_xor_sync(0xFFFFFFFFu, err_e, off);
+    diff_sum += __shfl_xor_sync(0xFFFFFFFFu, diff_sum, off);
+    common += __shfl_xor_sync(0xFFFFFFFFu, common, off);
+  }
+  warp_barrier();
+  // median: the differences at sorted positions (n - 1) / 2 and n / 2, a difference's position being
+  // the number of differences that precede it (smaller, or equal and earlier)
+  const uint32_t n = (uint32_t)k - err_e;
+  int lo_val = -1, hi_val = -1;
+  if (n > 0) {
+    const uint32_t lo_pos = (n - 1) / 2, hi_pos = n / 2;
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) {
+      const int j = s * 32 + lane;
+      if (j >= k) continue;
+      const uint32_t mine = diffs[j];
+      if (mine == kNoMatch) continue;
+      uint32_t before = 0;
+      for (int i = 0; i < k; ++i) {
+        const uint32_t other = diffs[i];
+        before += (other < mine) || (other == mine && i < j);
+      }
+      if (before == lo_pos) lo_val = (int)mine;
+      if (before == hi_pos) hi_val = (int)mine;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    lo_val = max(lo_val, __shfl_xor_sync(0xFFFFFFFFu, lo_val, off));
+    hi_val = max(hi_val, __shfl_xor_sync(0xFFFFFFFFu, hi_val, off));
+  }
+  if (lane == 0) {
+    res.exp_mismatch = err_e;
+    res.n_match = n;
+    res.mant_diff_sum = diff_sum;
+    if (io.gen_indices) res.topk_mismatch = k - (int)common;
+    bool reject = true;  // nothing matched: nothing to accept on
+    if (n > 0) {
+      res.mant_mean = (double)diff_sum / (double)n;
+      res.mant_median = ((double)lo_val + (double)hi_val) * 0.5;
+      reject = (res.exp_mismatch > (uint32_t)io.t_exp) || (res.mant_mean > io.t_mean) ||
+               (res.mant_median > io.t_median);
+    }
+    res.accept = reject ? 0 : 1;
+    io.results[chunk] = res;
+  }
+}
+
 template <int DT, int SLOTS>
-__device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, long long chunk, const VerifyIo& io,
+__device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, bool wide, long long chunk, const VerifyIo& io,
                                              const toploc_chunk_result& res) {
   const int lane = threadIdx.x;
   uint32_t idx[SLOTS], bits[SLOTS];
@@ -1139,17 +1424,19 @@ __device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, long long 
       const uint32_t key = (uint32_t)(cj >> (kIdxBits + 1));
       const uint32_t sign = (uint32_t)cj & 1u;
       idx[s] = kIdxMask - ((uint32_t)(cj >> 1) & kIdxMask);
-      bits[s] = (sign << 15) | (DT == 0 ? key : (key >> 16));
+      bits[s] = (DT == 1 && wide) ? ((sign << 31) | key) : ((sign << 15) | (DT == 0 ? key : (key >> 16)));
     }
   }
-  evaluate_warp<SLOTS>(sh, k, chunk, idx, bits, io, res);
+  if (DT == 1 && wide) evaluate_warp_q<SLOTS>(sh, k, chunk, idx, bits, io, res);
+  else evaluate_warp<SLOTS>(sh, k, chunk, idx, bits, io, res);
 }
 
 // decode() of Algorithm 2 for one chunk, by one warp: fills res with zeros and
 // the decoded modulus.  A malformed proof (modulus outside [2^15 + 1, 2^16] or a
-// coefficient >= p) is reported without looking at the activations: its result
+// coefficient >= p, >= q for 4-byte coefficients) is reported without looking at the activations: its result
 // is written and false returned.
-__device__ __forceinline__ bool decode_proof(const VerifyIo& io, long long chunk, int k, toploc_chunk_result* res) {
+__device__ __forceinline__ bool decode_proof(const VerifyIo& io, long long chunk, int k, int coef_bytes,
+                                             toploc_chunk_result* res) {
   const int lane = threadIdx.x;
   res->exp_mismatch = 0;
   res->n_match = 0;
@@ -1160,12 +1447,17 @@ __device__ __forceinline__ bool decode_proof(const VerifyIo& io, long long chunk
   res->accept = 0;
   res->status = TOPLOC_CHUNK_OK;
   res->pad[0] = res->pad[1] = 0;
-  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 2 * (size_t)k));
+  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + (size_t)coef_bytes * k));
   uint32_t m = proof[0];
   if (m == 0) m = 65536u;
   res->modulus = m;
   uint32_t bad = (m < kModLow || m > kModHigh);
-  for (int d = lane; d < k; d += kThreads) bad |= proof[1 + d] >= kPrime;
+  if (coef_bytes == 2) {
+    for (int d = lane; d < k; d += kThreads) bad |= proof[1 + d] >= kPrime;
+  } else {
+    for (int d = lane; d < k; d += kThreads)
+      bad |= ((uint32_t)proof[1 + 2 * d] | ((uint32_t)proof[2 + 2 * d] << 16)) >= kPrime32;
+  }
   if (__any_sync(0xFFFFFFFFu, bad != 0)) {
     res->status = TOPLOC_CHUNK_BAD_PROOF;
     if (lane == 0) io.results[chunk] = *res;
@@ -1188,7 +1480,7 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
   const int k = bp.k;
 
   toploc_chunk_result res;
-  if (!decode_proof(io, chunk, k, &res)) return;
+  if (!decode_proof(io, chunk, k, bp.coef_bytes, &res)) return;
   const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
   const long long n_elems = (long long)pl.rows * bp.hidden;
   if (n_elems < k) {
@@ -1203,10 +1495,11 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
   src.vecs_per_row = bp.hidden / ChunkSource<DT, MODE>::kVec;
   select_topk<DT, MODE>(sh, src, (int)n_elems, k);
 
-  if (k <= 32) verify_chunk<DT, 1>(sh, k, chunk, io, res);
-  else if (k <= 64) verify_chunk<DT, 2>(sh, k, chunk, io, res);
-  else if (k <= 128) verify_chunk<DT, 4>(sh, k, chunk, io, res);
-  else verify_chunk<DT, kMaxSlots>(sh, k, chunk, io, res);
+  const bool wide = bp.coef_bytes == 4;
+  if (k <= 32) verify_chunk<DT, 1>(sh, k, wide, chunk, io, res);
+  else if (k <= 64) verify_chunk<DT, 2>(sh, k, wide, chunk, io, res);
+  else if (k <= 128) verify_chunk<DT, 4>(sh, k, wide, chunk, io, res);
+  else verify_chunk<DT, kMaxSlots>(sh, k, wide, chunk, io, res);
 }
 
 // ---------------------------------------------------------------------------
@@ -1221,9 +1514,12 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
 // 2 validation.
 // ---------------------------------------------------------------------------
 template <int DT, int TAIL, int SLOTS>
-__device__ __forceinline__ void finish_merged(SelectShared& sh, int k, long long chunk, const Selection& sel,
-                                              const VerifyIo& io, const toploc_chunk_result& res) {
+__device__ __forceinline__ void finish_merged(SelectShared& sh, const BatchParams& bp, long long chunk,
+                                              const Selection& sel, const VerifyIo& io,
+                                              const toploc_chunk_result& res) {
   const int lane = threadIdx.x;
+  const int k = bp.k;
+  const bool wide = DT == 1 && bp.coef_bytes == 4;
   uint32_t idx[kMaxK / kThreads], bits[SLOTS];
   uint32_t unrepresentable = 0;
 #pragma unroll
@@ -1237,11 +1533,12 @@ __device__ __forceinline__ void finish_merged(SelectShared& sh, int k, long long
       const uint32_t key = (uint32_t)(w >> 33);
       const uint32_t sign = (uint32_t)w & 1u;
       idx[e] = 0xFFFFFFFFu - (uint32_t)(w >> 1);
-      bits[e] = (sign << 15) | (DT == 0 ? key : (key >> 16));
-      unrepresentable |= bits[e] >= kPrime;
+      bits[e] = wide ? ((sign << 31) | key) : ((sign << 15) | (DT == 0 ? key : (key >> 16)));
+      unrepresentable |= bits[e] >= (wide ? kPrime32 : kPrime);
       if (TAIL != 2) {
         sel.idx[chunk * k + j] = idx[e];
-        sel.bits[chunk * k + j] = (uint16_t)bits[e];
+        if (wide) sel.bits32[chunk * k + j] = bits[e];
+        else sel.bits[chunk * k + j] = (uint16_t)bits[e];
         if (sel.indices) {
           int rank = 0;  // position = number of better candidates
           for (int i = 0; i < k; ++i) rank += sh.cand[i] > w;
@@ -1253,11 +1550,11 @@ __device__ __forceinline__ void finish_merged(SelectShared& sh, int k, long long
   if (TAIL == 0) {
     if (lane == 0) sel.status[chunk] = TOPLOC_CHUNK_OK;
   } else if (TAIL == 1) {
-    uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 2 * (size_t)k));
+    uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_stride(bp));
     const int nonfinite = __syncthreads_or(unrepresentable != 0);
-    const uint32_t m = find_injective_modulus(sh, k, idx);
+    const uint32_t m = find_injective_modulus(sh, k, idx, wide);
     if (m == 0) {
-      for (int i = lane; i < k + 1; i += kThreads) proof[i] = 0;
+      for (int i = lane; i < proof_words(bp); i += kThreads) proof[i] = 0;
       if (lane == 0) sel.status[chunk] = TOPLOC_CHUNK_NO_INJECTIVE_MODULUS;
       return;
     }
@@ -1269,7 +1566,8 @@ __device__ __forceinline__ void finish_merged(SelectShared& sh, int k, long long
     uint32_t own[SLOTS];
 #pragma unroll
     for (int e = 0; e < SLOTS; ++e) own[e] = idx[e];
-    evaluate_warp<SLOTS>(sh, k, chunk, own, bits, io, res);
+    if (wide) evaluate_warp_q<SLOTS>(sh, k, chunk, own, bits, io, res);
+    else evaluate_warp<SLOTS>(sh, k, chunk, own, bits, io, res);
   }
 }
 
@@ -1282,7 +1580,7 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
   const long long chunk = blockIdx.x;
   const int k = bp.k;
   toploc_chunk_result res;
-  if (TAIL == 2 && !decode_proof(io, chunk, k, &res)) return;
+  if (TAIL == 2 && !decode_proof(io, chunk, k, bp.coef_bytes, &res)) return;
 
   const ChunkSegments cs = mp.chunks[chunk];
   if (mp.seg_status[cs.first_seg] != TOPLOC_CHUNK_OK) {
@@ -1293,8 +1591,8 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
       return;
     }
     if (TAIL == 1) {
-      uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 2 * (size_t)k));
-      for (int i = lane; i < k + 1; i += kThreads) proof[i] = 0;
+      uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_stride(bp));
+      for (int i = lane; i < proof_words(bp); i += kThreads) proof[i] = 0;
     }
     if (sel.indices)
       for (int i = lane; i < k; i += kThreads) sel.indices[chunk * k + i] = 0;
@@ -1358,10 +1656,10 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
   }
   warp_barrier();
 
-  if (k <= 32) finish_merged<DT, TAIL, 1>(sh, k, chunk, sel, io, res);
-  else if (k <= 64) finish_merged<DT, TAIL, 2>(sh, k, chunk, sel, io, res);
-  else if (k <= 128) finish_merged<DT, TAIL, 4>(sh, k, chunk, sel, io, res);
-  else finish_merged<DT, TAIL, kMaxSlots>(sh, k, chunk, sel, io, res);
+  if (k <= 32) finish_merged<DT, TAIL, 1>(sh, bp, chunk, sel, io, res);
+  else if (k <= 64) finish_merged<DT, TAIL, 2>(sh, bp, chunk, sel, io, res);
+  else if (k <= 128) finish_merged<DT, TAIL, 4>(sh, bp, chunk, sel, io, res);
+  else finish_merged<DT, TAIL, kMaxSlots>(sh, bp, chunk, sel, io, res);
 }
 
 // ---------------------------------------------------------------------------
@@ -1409,8 +1707,9 @@ void count_sequence(const toploc_layout* lay, long long len, long long* chunks, 
 int plan_layout(const toploc_layout* lay, HostPlan* plan) {
   if (lay == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (lay->dtype != TOPLOC_DTYPE_BF16 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
-  if (lay->hidden <= 0 || lay->chunk_len <= 0 || lay->num_seqs <= 0 || lay->reserved != 0)
-    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->hidden <= 0 || lay->chunk_len <= 0 || lay->num_seqs <= 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field != TOPLOC_FIELD_16 && lay->field != TOPLOC_FIELD_32) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field == TOPLOC_FIELD_32 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
   if (lay->k < 1) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (lay->k > TOPLOC_MAX_K) return TOPLOC_ERR_UNSUPPORTED;
   if (lay->row_stride < lay->hidden) return TOPLOC_ERR_INVALID_ARGUMENT;
@@ -1514,6 +1813,9 @@ int pick_mode(const void* act, const toploc_layout* lay) {
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+size_t coef_bytes_of(const toploc_layout* lay) { return lay->field == TOPLOC_FIELD_32 ? 4 : 2; }
+size_t proof_bytes_of(const toploc_layout* lay) { return 2 + coef_bytes_of(lay) * (size_t)lay->k; }
+
 // Scratch of one call: ragged row table, then the selection; with long chunks
 // (segs != chunks) the row table describes segments and is followed by the
 // chunk table, the segments' selections and the merge's words.
@@ -1522,7 +1824,8 @@ struct WorkspacePlan {
   size_t idx_off, bits_off, status_off, total;
 };
 
-WorkspacePlan plan_workspace(bool ragged, long long chunks, int k, long long segs) {
+// pattern_bytes: 2, or 4 for fp32 chunks committed over the 32-bit field.
+WorkspacePlan plan_workspace(bool ragged, long long chunks, int k, long long segs, size_t pattern_bytes) {
   WorkspacePlan w;
   const bool split = segs != chunks;
   size_t off = 0;
@@ -1533,7 +1836,7 @@ WorkspacePlan plan_workspace(bool ragged, long long chunks, int k, long long seg
   w.seg_idx_off = off;
   off += split ? round_up((size_t)segs * k * sizeof(uint32_t), 256) : 0;
   w.seg_bits_off = off;
-  off += split ? round_up((size_t)segs * k * sizeof(uint16_t), 256) : 0;
+  off += split ? round_up((size_t)segs * k * pattern_bytes, 256) : 0;
   w.seg_status_off = off;
   off += split ? round_up((size_t)segs, 256) : 0;
   w.words_off = off;
@@ -1541,7 +1844,7 @@ WorkspacePlan plan_workspace(bool ragged, long long chunks, int k, long long seg
   w.idx_off = off;
   off += round_up((size_t)chunks * k * sizeof(uint32_t), 256);
   w.bits_off = off;
-  off += round_up((size_t)chunks * k * sizeof(uint16_t), 256);
+  off += round_up((size_t)chunks * k * pattern_bytes, 256);
   w.status_off = off;
   off += round_up((size_t)chunks, 256);
   w.total = off;
@@ -1634,7 +1937,7 @@ int prepare_batch(const void* d_act, const toploc_layout* lay, void* d_workspace
                   cudaStream_t stream, const HostPlan* plan, DeviceInfo** dev, PreparedBatch* pb) {
   int rc = device_info(dev);
   if (rc != TOPLOC_OK) return rc;
-  const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k, plan->num_segs);
+  const WorkspacePlan wp = plan_workspace(plan->ragged, plan->num_chunks, lay->k, plan->num_segs, coef_bytes_of(lay));
   if (d_workspace == nullptr || workspace_bytes < wp.total) return TOPLOC_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(d_workspace) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
   char* ws = static_cast<char*>(d_workspace);
@@ -1650,6 +1953,7 @@ int prepare_batch(const void* d_act, const toploc_layout* lay, void* d_workspace
   bp->chunk_len = lay->chunk_len;
   bp->k = lay->k;
   bp->chunks_per_seq = plan->chunks_per_seq;
+  bp->coef_bytes = (int)coef_bytes_of(lay);
   if (plan->ragged || plan->split) {
     if ((rc = upload_spans(lay, *plan, ws + wp.spans_off, ws + wp.chunk_table_off, stream)) != TOPLOC_OK) return rc;
     bp->spans = reinterpret_cast<const ChunkSpan*>(ws + wp.spans_off);
@@ -1657,6 +1961,7 @@ int prepare_batch(const void* d_act, const toploc_layout* lay, void* d_workspace
   if (plan->split) {
     pb->segs.idx = reinterpret_cast<uint32_t*>(ws + wp.seg_idx_off);
     pb->segs.bits = reinterpret_cast<uint16_t*>(ws + wp.seg_bits_off);
+    pb->segs.bits32 = reinterpret_cast<uint32_t*>(ws + wp.seg_bits_off);
     pb->segs.status = reinterpret_cast<uint8_t*>(ws + wp.seg_status_off);
     pb->segs.proofs = nullptr;
     pb->segs.indices = nullptr;
@@ -1681,6 +1986,7 @@ int run_select(const void* d_act, const toploc_layout* lay, void* d_workspace, s
   if (rc != TOPLOC_OK) return rc;
   sel->idx = d_sel_idx_or_null ? d_sel_idx_or_null : reinterpret_cast<uint32_t*>(pb.ws + pb.wp.idx_off);
   sel->bits = d_sel_bits_or_null ? d_sel_bits_or_null : reinterpret_cast<uint16_t*>(pb.ws + pb.wp.bits_off);
+  sel->bits32 = reinterpret_cast<uint32_t*>(pb.ws + pb.wp.bits_off);  // written instead of bits by the 32-bit field
   sel->status = d_status_or_null ? d_status_or_null : reinterpret_cast<uint8_t*>(pb.ws + pb.wp.status_off);
   sel->proofs = d_proofs_or_null;
   sel->indices = d_indices_opt;
@@ -1714,9 +2020,9 @@ StagingPlan carve_staging(const toploc_layout* lay, long long rows, long long ch
   sp.small_off = off;
   off += round_up((size_t)chunks * sizeof(toploc_chunk_result), 256);
   sp.proofs_off = off;
-  off += round_up((size_t)chunks * (2 + 2 * (size_t)lay->k), 256);
+  off += round_up((size_t)chunks * proof_bytes_of(lay), 256);
   sp.work_off = off;
-  sp.work_bytes = plan_workspace(true, chunks, lay->k, segs).total;
+  sp.work_bytes = plan_workspace(true, chunks, lay->k, segs, coef_bytes_of(lay)).total;
   off += sp.work_bytes;
   sp.total = off;
   return sp;
@@ -1750,10 +2056,15 @@ int64_t toploc_num_chunks(const toploc_layout* lay) {
 
 size_t toploc_proof_bytes(int32_t k) { return k > 0 ? 2 + 2 * (size_t)k : 0; }
 
+size_t toploc_layout_proof_bytes(const toploc_layout* lay) {
+  HostPlan plan;
+  return plan_layout(lay, &plan) == TOPLOC_OK ? proof_bytes_of(lay) : 0;
+}
+
 size_t toploc_workspace_bytes(const toploc_layout* lay) {
   HostPlan plan;
   if (plan_layout(lay, &plan) != TOPLOC_OK) return 0;
-  return plan_workspace(plan.ragged, plan.num_chunks, lay->k, plan.num_segs).total;
+  return plan_workspace(plan.ragged, plan.num_chunks, lay->k, plan.num_segs, coef_bytes_of(lay)).total;
 }
 
 size_t toploc_staging_bytes(const toploc_layout* lay) {
@@ -1810,6 +2121,11 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
   rc = run_select(d_act, lay, d_workspace, workspace_bytes, stream, d_status, d_proofs, d_indices_opt, &plan,
                   &sel, &dev);
   if (rc != TOPLOC_OK) return rc;
+  if (lay->field == TOPLOC_FIELD_32) {
+    const long long q_blocks = (plan.num_chunks + kInterpQWarps - 1) / kInterpQWarps;
+    toploc_interpolate_q_kernel<<<(unsigned)q_blocks, kInterpQWarps * 32, 0, stream>>>(sel, lay->k, plan.num_chunks);
+    return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+  }
   const long long per_wave = (long long)kInterpWarps * kInterpChunks;
   long long blocks = (plan.num_chunks + per_wave - 1) / per_wave;
   if (blocks > dev->sms) blocks = dev->sms;
@@ -1870,6 +2186,7 @@ int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_
     return TOPLOC_ERR_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(d_sel_indices) % 4 != 0 || reinterpret_cast<uintptr_t>(d_sel_patterns) % 2 != 0)
     return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field != TOPLOC_FIELD_16) return TOPLOC_ERR_UNSUPPORTED;  // this entry point hands out 16-bit patterns
   if (plan.num_chunks == 0) return TOPLOC_OK;
   Selection sel;
   DeviceInfo* dev = nullptr;
@@ -1883,7 +2200,7 @@ int toploc_build_proofs_builtin_scratch(const void* d_act, const toploc_layout* 
   int rc = plan_layout(lay, &plan);
   if (rc != TOPLOC_OK) return rc;
   if (plan.ragged || plan.split) return TOPLOC_ERR_UNSUPPORTED;  // the row table would have to be built on the heap
-  if (plan_workspace(false, plan.num_chunks, lay->k, plan.num_segs).total > kBuiltinScratchBytes)
+  if (plan_workspace(false, plan.num_chunks, lay->k, plan.num_segs, coef_bytes_of(lay)).total > kBuiltinScratchBytes)
     return TOPLOC_ERR_BUILTIN_SCRATCH;
   DeviceInfo* dev = nullptr;
   if ((rc = device_info(&dev)) != TOPLOC_OK) return rc;
@@ -1909,7 +2226,7 @@ static int run_from_host(bool verify, const void* h_act, const toploc_layout* la
   if (staging_bytes < toploc_staging_bytes(lay)) return TOPLOC_ERR_WORKSPACE;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t esz = lay->dtype == TOPLOC_DTYPE_BF16 ? 2 : 4;
-  const size_t pb = 2 + 2 * (size_t)lay->k;
+  const size_t pb = proof_bytes_of(lay);
   char* stage = static_cast<char*>(d_staging);
   int64_t* rebased = static_cast<int64_t*>(malloc(((size_t)lay->num_seqs + 1) * sizeof(int64_t)));
   if (rebased == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;

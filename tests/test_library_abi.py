@@ -42,7 +42,7 @@ def test_struct_sizes_match_the_header():
 
 def layout(**kw):
     lay = tl.ToplocLayout()
-    base = dict(dtype=0, hidden=4096, chunk_len=32, k=128, num_seqs=2, reserved=0, tokens_per_seq=100,
+    base = dict(dtype=0, hidden=4096, chunk_len=32, k=128, num_seqs=2, field=0, tokens_per_seq=100,
                 row_stride=4096)
     base.update(kw)
     for key, val in base.items():
@@ -71,6 +71,20 @@ def test_chunk_counting():
     assert tl.toploc_staging_bytes(layout()) >= 100 * 4096 * 2 + 4 * 258
 
 
+def test_the_32_bit_field_is_for_fp32_and_doubles_the_coefficients():
+    wide = layout(dtype=1, field=tl.TOPLOC_FIELD_32)
+    narrow = layout(dtype=1)
+    assert tl.toploc_num_chunks(wide) == tl.toploc_num_chunks(narrow) == 8
+    assert tl.toploc_layout_proof_bytes(wide) == 2 + 4 * 128 and tl.toploc_layout_proof_bytes(narrow) == 258
+    assert tl.toploc_layout_proof_bytes(layout(k=0)) == 0
+    grow = tl.toploc_workspace_bytes(wide) - tl.toploc_workspace_bytes(narrow)
+    assert 8 * 128 * 2 <= grow <= 8 * 128 * 2 + 256                 # whole patterns instead of 16 bits
+    assert tl.toploc_staging_bytes(wide) > tl.toploc_staging_bytes(narrow)
+    thr = tl.default_thresholds(128, field=tl.TOPLOC_FIELD_32)
+    assert (thr.t_exp, thr.t_mean, thr.t_median) == (8, 256.0, 128.0)
+    assert tl.TOPLOC_FIELD_32_PRIME == 2 ** 32 - 5
+
+
 def test_long_chunks_are_planned_in_segments():
     """A chunk above 2^19 elements is selected in segments of about 2^18 elements (whole rows) and
     merged: the scratch grows by the segments' selections and the merge's words; the chunk count
@@ -91,7 +105,7 @@ def test_long_chunks_are_planned_in_segments():
 
 @pytest.mark.parametrize("bad", [dict(k=0), dict(k=257), dict(hidden=0), dict(chunk_len=0), dict(num_seqs=0),
                                  dict(dtype=7), dict(row_stride=100), dict(tokens_per_seq=0),
-                                 dict(reserved=1),
+                                 dict(field=1), dict(field=2), dict(dtype=1, field=-1),
                                  dict(hidden=1 << 20, chunk_len=2048, tokens_per_seq=4096, row_stride=1 << 20),
                                  dict(hidden=(1 << 24) + 8, row_stride=(1 << 24) + 8)])
 def test_invalid_layouts_are_refused(bad):
