@@ -715,24 +715,25 @@ static_assert(kGenerator != 0 && mul_mod(kGenerator, kGeneratorInv) == 1u, "gene
 // Algorithm 6 applies as printed).  Returns 0 if there is none.
 // idx[e] is the flat index of point 32 e + lane.  The selection in shared
 // memory is consumed: the tile ring and the candidate buffer become the
-// 65536-bit set of residues seen.
+// 65536-bit set of residues seen.  Run by one warp (the only one of its block
+// that is still at work).
 __device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32_t (&idx)[kMaxK / kThreads],
                                            bool wide_field) {
-  const int tid = threadIdx.x;
+  const int lane = threadIdx.x & 31;
   uint32_t res[kMaxK / kThreads];
 #pragma unroll
   for (int e = 0; e < kMaxK / kThreads; ++e) res[e] = 0;
-  __syncthreads();  // every lane has taken its candidates out of sh.cand
+  warp_barrier();  // every lane has taken its candidates out of sh.cand
   uint32_t* seen = reinterpret_cast<uint32_t*>(sh.ring);  // ring and cand are adjacent: 11 KB
-  for (int i = tid; i < 2048; i += kThreads) seen[i] = 0;
-  __syncthreads();
+  for (int i = lane; i < 2048; i += kThreads) seen[i] = 0;
+  warp_barrier();
   uint32_t found = 0;
 #pragma unroll 1
   for (uint32_t m = kModHigh; m >= kModLow; --m) {
     uint32_t dup = 0;
 #pragma unroll
     for (int e = 0; e < kMaxK / kThreads; ++e) {
-      int j = tid + e * kThreads;
+      int j = lane + e * kThreads;
       if (j < k) {
         uint32_t r = idx[e] % m;
         if (!wide_field && r >= kPrime) r -= kPrime;  // every residue is below q = 2^32 - 5 as it is
@@ -741,13 +742,13 @@ __device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32
         dup |= atomicOr(&seen[r >> 5], bit) & bit;
       }
     }
-    const int clash = __syncthreads_or(dup != 0);
+    const bool clash = __any_sync(0xFFFFFFFFu, dup != 0);  // also orders the set's updates before its clearing
 #pragma unroll
     for (int e = 0; e < kMaxK / kThreads; ++e) {
-      int j = tid + e * kThreads;
+      int j = lane + e * kThreads;
       if (j < k) seen[res[e] >> 5] = 0;
     }
-    __syncthreads();
+    warp_barrier();
     if (!clash) {
       found = m;
       break;
@@ -839,7 +840,7 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
     if (tid == 0) sel.status[chunk] = TOPLOC_CHUNK_OK;
     return;
   }
-  const int nonfinite = __syncthreads_or(unrepresentable != 0);
+  const bool nonfinite = __any_sync(0xFFFFFFFFu, unrepresentable != 0);
   uint32_t picked[kMaxK / kThreads];
 #pragma unroll
   for (int e = 0; e < kMaxK / kThreads; ++e) {
@@ -1002,7 +1003,8 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
   uint16_t* xw = scratch + warp * 2 * kInterpChunks * kMaxK;
   uint16_t* aw = xw + kInterpChunks * kMaxK;
   const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
-  for (long long g = (long long)blockIdx.x * kInterpWarps + warp; g < groups;
+  // group g goes to block g % gridDim.x, so a small batch spreads over the blocks before it fills their warps
+  for (long long g = blockIdx.x + (long long)gridDim.x * warp; g < groups;
        g += (long long)gridDim.x * kInterpWarps) {
     long long chunk[kInterpChunks];
     bool live[kInterpChunks];
@@ -1503,8 +1505,9 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
 }
 
 // ---------------------------------------------------------------------------
-// merge kernel: the top-k of a chunk from the top-k of its segments, one warp
-// per chunk, then the same tails as the select and verify kernels.  Every
+// merge kernel: the top-k of a chunk from the top-k of its segments, one block
+// per chunk (its first warp then runs the same tails as the select and verify
+// kernels).  Every
 // candidate becomes one 64-bit word whose unsigned order is the ranking order
 // over the whole chunk: key << 33 | (2^32 - 1 - flat index) << 1 | sign.  The
 // k-th largest word is found digit by digit (MSB-first radix select, eight
@@ -1551,7 +1554,7 @@ __device__ __forceinline__ void finish_merged(SelectShared& sh, const BatchParam
     if (lane == 0) sel.status[chunk] = TOPLOC_CHUNK_OK;
   } else if (TAIL == 1) {
     uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_stride(bp));
-    const int nonfinite = __syncthreads_or(unrepresentable != 0);
+    const bool nonfinite = __any_sync(0xFFFFFFFFu, unrepresentable != 0);
     const uint32_t m = find_injective_modulus(sh, k, idx, wide);
     if (m == 0) {
       for (int i = lane; i < proof_words(bp); i += kThreads) proof[i] = 0;
@@ -1571,20 +1574,33 @@ __device__ __forceinline__ void finish_merged(SelectShared& sh, const BatchParam
   }
 }
 
+constexpr int kMergeThreads = 256;  // merge kernel: the passes over a chunk's words use the whole block
+
 template <int DT, int TAIL>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kMergeThreads)
 toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) {
   __shared__ SelectShared sh;
-  const int lane = threadIdx.x;
-  const uint32_t below = (1u << lane) - 1u;
+  __shared__ int kept;     // words taken so far
+  __shared__ int proceed;  // decode() found the proof well-formed
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const bool first_warp = tid < 32;  // the warp that goes on to the tail
   const long long chunk = blockIdx.x;
   const int k = bp.k;
   toploc_chunk_result res;
-  if (TAIL == 2 && !decode_proof(io, chunk, k, bp.coef_bytes, &res)) return;
+  if (TAIL == 2) {
+    if (first_warp) {
+      const bool ok = decode_proof(io, chunk, k, bp.coef_bytes, &res);
+      if (lane == 0) proceed = ok;
+    }
+    __syncthreads();
+    if (!proceed) return;
+  }
 
   const ChunkSegments cs = mp.chunks[chunk];
   if (mp.seg_status[cs.first_seg] != TOPLOC_CHUNK_OK) {
     // fewer than k elements: such a chunk is one segment, which said so
+    if (!first_warp) return;
     if (TAIL == 2) {
       res.status = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
       if (lane == 0) io.results[chunk] = res;
@@ -1602,7 +1618,7 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
 
   const int n = cs.n_segs * k;
   unsigned long long* words = mp.words + (size_t)cs.first_seg * k;
-  for (int c = lane; c < n; c += kThreads) {
+  for (int c = tid; c < n; c += kMergeThreads) {
     const int seg = c / k;
     const size_t at = (size_t)(cs.first_seg + seg) * k + (size_t)(c - seg * k);
     const long long seg_row0 = mp.segs[cs.first_seg + seg].row0;
@@ -1614,7 +1630,7 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
       key = pattern & 0x7FFFu;
       sign = pattern >> 15;
     } else {
-      // the segment kept only the upper half of the pattern: read the element again
+      // the segment kept only part of the pattern: read the element again
       const long long row = seg_row0 + local / (uint32_t)bp.hidden;
       const uint32_t col = local % (uint32_t)bp.hidden;
       const uint32_t pattern = static_cast<const uint32_t*>(bp.act)[row * bp.row_stride + col];
@@ -1623,38 +1639,37 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
     }
     words[c] = ((unsigned long long)key << 33) | ((unsigned long long)(0xFFFFFFFFu - flat) << 1) | sign;
   }
-  __syncwarp();
+  if (tid == 0) kept = 0;
+  __syncthreads();
 
   unsigned long long kth = 0;  // the k-th largest word; all of them if the chunk is one segment
   if (n > k) {
     unsigned long long prefix = 0;
     int want = k;
+    // a bf16 key has 15 bits: the two leading digits of its words are zero
 #pragma unroll 1
-    for (int pass = 0; pass < 8; ++pass) {
+    for (int pass = (DT == 0 ? 2 : 0); pass < 8; ++pass) {
       const int shift = 56 - 8 * pass;
-      warp_barrier();
-      for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
-      warp_barrier();
-      for (int c = lane; c < n; c += kThreads) {
+      for (int b = tid; b < 256; b += kMergeThreads) sh.top_hist[b] = 0;
+      __syncthreads();
+      for (int c = tid; c < n; c += kMergeThreads) {
         const unsigned long long w = words[c];
         if (pass == 0 || (w >> (shift + 8)) == prefix) atomicAdd(&sh.top_hist[(uint32_t)(w >> shift) & 255u], 1u);
       }
-      find_from_top<8>(sh, sh.top_hist, want);
+      __syncthreads();
+      if (first_warp) find_from_top<8>(sh, sh.top_hist, want);
+      __syncthreads();
       prefix = (prefix << 8) | sh.digit;
       want = sh.want;
     }
     kth = prefix;
   }
-  int count = 0;
-  for (int c0 = 0; c0 < n; c0 += kThreads) {
-    const int c = c0 + lane;
-    const unsigned long long w = c < n ? words[c] : 0ull;
-    const bool keep = c < n && w >= kth;
-    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, keep);
-    if (keep) sh.cand[count + __popc(votes & below)] = w;  // words are distinct: exactly k are kept
-    count += __popc(votes);
+  for (int c = tid; c < n; c += kMergeThreads) {
+    const unsigned long long w = words[c];
+    if (w >= kth) sh.cand[atomicAdd(&kept, 1)] = w;  // words are distinct: exactly k are taken, in any order
   }
-  warp_barrier();
+  __syncthreads();
+  if (!first_warp) return;
 
   if (k <= 32) finish_merged<DT, TAIL, 1>(sh, bp, chunk, sel, io, res);
   else if (k <= 64) finish_merged<DT, TAIL, 2>(sh, bp, chunk, sel, io, res);
@@ -1916,9 +1931,9 @@ void launch_verify(int mode, unsigned grid, cudaStream_t stream, const BatchPara
 template <int DT>
 void launch_merge(int tail, unsigned grid, cudaStream_t stream, const BatchParams& bp, const MergeParams& mp,
                   const Selection& sel, const VerifyIo& io) {
-  if (tail == 0) toploc_merge_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, mp, sel, io);
-  else if (tail == 1) toploc_merge_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, mp, sel, io);
-  else toploc_merge_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, mp, sel, io);
+  if (tail == 0) toploc_merge_kernel<DT, 0><<<grid, kMergeThreads, 0, stream>>>(bp, mp, sel, io);
+  else if (tail == 1) toploc_merge_kernel<DT, 1><<<grid, kMergeThreads, 0, stream>>>(bp, mp, sel, io);
+  else toploc_merge_kernel<DT, 2><<<grid, kMergeThreads, 0, stream>>>(bp, mp, sel, io);
 }
 
 // A batch as the kernels see it.
@@ -2126,8 +2141,10 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
     toploc_interpolate_q_kernel<<<(unsigned)q_blocks, kInterpQWarps * 32, 0, stream>>>(sel, lay->k, plan.num_chunks);
     return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
   }
-  const long long per_wave = (long long)kInterpWarps * kInterpChunks;
-  long long blocks = (plan.num_chunks + per_wave - 1) / per_wave;
+  // one block per SM; a small batch gets a block for every four of its groups (each block first
+  // builds its table of inverses, so not one per group)
+  const long long groups = (plan.num_chunks + kInterpChunks - 1) / kInterpChunks;
+  long long blocks = (groups + 3) / 4;
   if (blocks > dev->sms) blocks = dev->sms;
   toploc_interpolate_kernel<<<(unsigned)blocks, kInterpWarps * 32, interp_smem_bytes(), stream>>>(
       sel, lay->k, plan.num_chunks);
