@@ -35,8 +35,11 @@ WORKLOADS = {
     "prompt70b": (64, 4096, 8192, 4096, 128, 6),
     # fp32 activations committed whole over the 32-bit field (2 + 4k byte proofs, fp32 thresholds)
     "70b-fp32-wide": (128, 4096, 8192, 32, 128, 7),
+    # small cases of the two above, for profiler captures
+    "prompt8b": (16, 2048, 4096, 2048, 128, 9),
+    "8b-fp32-wide": (64, 2048, 4096, 32, 128, 8),
 }
-WIDE_WORKLOADS = ("70b-fp32-wide",)
+WIDE_WORKLOADS = ("70b-fp32-wide", "8b-fp32-wide")
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one toploc_select_kernel launch on the full
 # batch (ncu, profiles/launch_list_70b_shape.md); None where no capture of the current kernel exists
@@ -164,7 +167,8 @@ def workload_name(key):
     S, T, H, L, k, seed = WORKLOADS[key]
     return "%s-shaped: %d seq x %d tok, H=%d %s, L=%d, k=%d" % (
         {"70b": "Llama-3.1-70B", "8b": "Llama-3.1-8B", "prompt70b": "Llama-3.1-70B prompt chunks",
-         "70b-fp32-wide": "Llama-3.1-70B"}[key], S, T, H,
+         "70b-fp32-wide": "Llama-3.1-70B", "prompt8b": "Llama-3.1-8B prompt chunks",
+         "8b-fp32-wide": "Llama-3.1-8B"}[key], S, T, H,
         "fp32 over the 32-bit field" if key in WIDE_WORKLOADS else "bf16", L, k)
 
 

@@ -26,6 +26,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
+
 namespace {
 
 // ---------------------------------------------------------------------------
@@ -1782,11 +1784,16 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratch
 
 size_t interp_smem_bytes() { return (65536 + (size_t)kInterpWarps * 2 * kInterpChunks * kMaxK) * sizeof(uint16_t); }
 
+// Per-device facts, looked up on a device's first call.  Host threads may call
+// the library concurrently: the table is filled under a lock.
+std::mutex g_device_table_lock;
+
 int device_info(DeviceInfo** out) {
   static DeviceInfo table[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return TOPLOC_ERR_CUDA;
   if (dev < 0 || dev >= 64) return TOPLOC_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> guard(g_device_table_lock);
   DeviceInfo& d = table[dev];
   if (!d.known) {
     if (cudaDeviceGetAttribute(&d.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
@@ -1807,6 +1814,7 @@ int device_info(DeviceInfo** out) {
 
 // Device address of the built-in scratch on the current device (looked up once per device).
 int builtin_scratch_address(DeviceInfo* d, void** out) {
+  std::lock_guard<std::mutex> guard(g_device_table_lock);
   if (d->builtin_scratch == nullptr) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_builtin_scratch) != cudaSuccess || ptr == nullptr) return TOPLOC_ERR_CUDA;
