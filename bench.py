@@ -182,6 +182,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-steps", action="store_true",
+                    help="time incremental proof generation (one row per sequence and step) instead of the main workload")
     ap.add_argument("--sweep", action="store_true",
                     help="time the parameter sweep (k x chunk length x H x dtype) instead of the main workload")
     args = ap.parse_args()
@@ -204,6 +206,10 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
+    if args.decode_steps:
+        if rank == 0:
+            print(json.dumps(decode_steps(tl, synth, dev)), flush=True)
+        return
     if args.sweep:
         if rank == 0:
             print(json.dumps(sweep(tl, synth, dev)), flush=True)
@@ -337,6 +343,58 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def decode_steps(tl, synth, dev, reps=20):
+    """Incremental proof generation as a decoder would drive it: 256 sequences, H = 8192 bf16, one new
+    row per sequence and step, a proof per 32 steps.  Times (CUDA events) of one append, of the finish,
+    and of a whole 32-token interval, beside toploc_build_proofs over the same 256 assembled chunks."""
+    S, L, H, k = 256, 32, 8192, 128
+    act = synth.make_activations(S, L, H, torch.bfloat16, seed=11, device=dev)
+    by_seq = act.view(S, L, H)
+    steps = [by_seq[:, t, :].contiguous() for t in range(L)]     # the decoder's per-step outputs
+    lay, _ = tl.make_layout(steps[0], L, k, S, 1)
+    state = torch.empty(tl.toploc_stream_state_bytes(lay), dtype=torch.uint8, device=dev)
+    ws = torch.empty(tl.toploc_stream_workspace_bytes(lay), dtype=torch.uint8, device=dev)
+    proofs = torch.empty((S, tl.toploc_layout_proof_bytes(lay)), dtype=torch.uint8, device=dev)
+    status = torch.empty((S,), dtype=torch.uint8, device=dev)
+
+    def interval(ev=None):
+        tl.toploc_stream_begin(state, lay)
+        for t in range(L):
+            tl.toploc_stream_append(steps[t], lay, t, state)
+        if ev:
+            ev[0].record()
+        tl.toploc_stream_finish(state, lay, proofs, status, workspace=ws)
+        if ev:
+            ev[1].record()
+
+    for _ in range(3):
+        interval()
+    torch.cuda.synchronize()
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(reps)]
+    for m in marks:
+        m[2].record()
+        interval(m)
+    torch.cuda.synchronize()
+    whole = float(np.mean([m[2].elapsed_time(m[1]) for m in marks]))
+    finish = float(np.mean([m[0].elapsed_time(m[1]) for m in marks]))
+    blay, _ = tl.make_layout(act, L, k, S, L)
+    bws = torch.empty(tl.toploc_workspace_bytes(blay), dtype=torch.uint8, device=dev)
+    ref_proofs = torch.empty_like(proofs)
+    for _ in range(3):
+        tl.toploc_build_proofs(act, blay, ref_proofs, status, workspace=bws)
+    torch.cuda.synchronize()
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b0.record()
+    for _ in range(reps):
+        tl.toploc_build_proofs(act, blay, ref_proofs, status, workspace=bws)
+    b1.record()
+    torch.cuda.synchronize()
+    return {"metric": "incremental_proof_generation", "sequences": S, "hidden": H, "interval_tokens": L, "k": k,
+            "us_per_append": (whole - finish) / L * 1e3, "us_finish": finish * 1e3, "us_per_interval": whole * 1e3,
+            "us_batch_build_of_the_same_chunks": b0.elapsed_time(b1) / reps * 1e3,
+            "bytes_per_append": S * H * 2, "identical_to_batch": bool(torch.equal(proofs, ref_proofs))}
 
 
 def sweep(tl, synth, dev, reps=5):

@@ -271,6 +271,47 @@ int toploc_build_proofs_builtin_scratch(const void* d_act, const toploc_layout* 
                                         uint8_t* d_status, int32_t* d_indices_opt, void* cuda_stream);
 
 /*
+ * Incremental proof generation: Algorithm 1 for a provider that decodes one
+ * token at a time (Section 5.5: a proof per 32 newly generated tokens).  The
+ * rows of the running chunk are handed over as they are produced -- one new
+ * row per sequence and step, still warm in L2 -- and every sequence keeps its
+ * running top-k in d_state between the steps, so the activations of a chunk
+ * never have to be gathered or read again.  The proofs, statuses and indices
+ * are bit-identical to toploc_build_proofs over the assembled chunks (ties go
+ * to the lower flat index = token_in_chunk * hidden + channel either way).
+ *
+ * lay describes the running batch: dtype, field, hidden, k, num_seqs, and
+ * chunk_len = the most tokens a chunk may receive (chunk_len * hidden may not
+ * exceed 2^24); row_stride = elements between the rows of consecutive
+ * sequences in d_rows.  tokens_per_seq and seq_offsets are ignored.
+ *
+ *   toploc_stream_begin    empties the running selections (start of a chunk)
+ *   toploc_stream_append   d_rows DEVICE [num_seqs, hidden]: row token_in_chunk
+ *                          of every sequence's chunk; call with 0, 1, 2, ... in
+ *                          order, on one stream or otherwise ordered
+ *   toploc_stream_finish   modulus, interpolation and encode for the chunks as
+ *                          they stand: d_proofs [num_seqs, proof bytes],
+ *                          d_status [num_seqs], d_indices_opt NULL or
+ *                          [num_seqs, k]; a chunk that received fewer than k
+ *                          elements gets TOPLOC_CHUNK_K_EXCEEDS_CHUNK.  d_state is
+ *                          not modified; begin a new chunk with toploc_stream_begin.
+ *
+ * d_state      DEVICE, toploc_stream_state_bytes(lay) = num_seqs * (16 + 8k) bytes,
+ *              16-byte aligned, owned by the caller, opaque
+ * d_workspace  DEVICE scratch for finish, toploc_stream_workspace_bytes(lay)
+ * All three only enqueue work on cuda_stream; return codes as above.
+ * Validation has no incremental form: a validator sees all tokens at once
+ * (Section 5.1) and uses toploc_verify_proofs.
+ */
+size_t toploc_stream_state_bytes(const toploc_layout* lay);
+size_t toploc_stream_workspace_bytes(const toploc_layout* lay);
+int toploc_stream_begin(void* d_state, const toploc_layout* lay, void* cuda_stream);
+int toploc_stream_append(const void* d_rows, const toploc_layout* lay, int32_t token_in_chunk, void* d_state,
+                         void* cuda_stream);
+int toploc_stream_finish(const void* d_state, const toploc_layout* lay, uint8_t* d_proofs, uint8_t* d_status,
+                         int32_t* d_indices_opt, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The same two operations for callers whose data lives in HOST memory
  * (pinned memory gives asynchronous copies; pageable memory works).  The
  * batch is cut into groups of whole sequences that fit the staging buffer;

@@ -14,7 +14,8 @@ __all__ = [
     "TOPLOC_DTYPE_BF16", "TOPLOC_DTYPE_FP32", "TOPLOC_MAX_K", "RESULT_DTYPE", "ToplocError",
     "ToplocLayout", "ToplocThresholds", "make_layout", "library_path", "load_library",
     "toploc_num_chunks", "toploc_proof_bytes", "toploc_layout_proof_bytes", "toploc_workspace_bytes",
-    "toploc_staging_bytes", "TOPLOC_FIELD_16", "TOPLOC_FIELD_32", "TOPLOC_FIELD_32_PRIME",
+    "toploc_staging_bytes", "toploc_stream_state_bytes", "toploc_stream_workspace_bytes", "toploc_stream_begin",
+    "toploc_stream_append", "toploc_stream_finish", "TOPLOC_FIELD_16", "TOPLOC_FIELD_32", "TOPLOC_FIELD_32_PRIME",
     "toploc_get_constants", "toploc_status_string", "toploc_error_string",
     "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
     "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES", "toploc_select_topk",
@@ -78,6 +79,13 @@ def load_library():
     lib.toploc_num_chunks.restype, lib.toploc_num_chunks.argtypes = i64, [lay_p]
     lib.toploc_proof_bytes.restype, lib.toploc_proof_bytes.argtypes = sz, [i32]
     lib.toploc_layout_proof_bytes.restype = sz
+    lib.toploc_layout_proof_bytes.argtypes = [lay_p]
+    lib.toploc_stream_state_bytes.restype, lib.toploc_stream_state_bytes.argtypes = sz, [lay_p]
+    lib.toploc_stream_workspace_bytes.restype, lib.toploc_stream_workspace_bytes.argtypes = sz, [lay_p]
+    lib.toploc_stream_begin.restype, lib.toploc_stream_begin.argtypes = ctypes.c_int, [vp, lay_p, vp]
+    lib.toploc_stream_append.restype, lib.toploc_stream_append.argtypes = ctypes.c_int, [vp, lay_p, i32, vp, vp]
+    lib.toploc_stream_finish.restype = ctypes.c_int
+    lib.toploc_stream_finish.argtypes = [vp, lay_p, vp, vp, vp, vp, sz, vp]
     lib.toploc_workspace_bytes.restype, lib.toploc_workspace_bytes.argtypes = sz, [lay_p]
     lib.toploc_staging_bytes.restype, lib.toploc_staging_bytes.argtypes = sz, [lay_p]
     lib.toploc_get_constants.restype = None
@@ -331,3 +339,52 @@ def toploc_select_topk(act, lay, sel_indices=None, sel_patterns=None, status=Non
             _dev_ptr(ranked_indices), _dev_ptr(workspace), wbytes, _stream_ptr(stream))
     _check(rc, "toploc_select_topk")
     return sel_indices, sel_patterns, status, ranked_indices
+
+
+def toploc_stream_state_bytes(lay):
+    return int(load_library().toploc_stream_state_bytes(ctypes.byref(lay)))
+
+
+def toploc_stream_workspace_bytes(lay):
+    return int(load_library().toploc_stream_workspace_bytes(ctypes.byref(lay)))
+
+
+def toploc_stream_begin(state, lay, stream=None):
+    """Empties the running selections held in `state` (a CUDA uint8 tensor of
+    toploc_stream_state_bytes(lay) bytes): the start of a chunk for every sequence."""
+    with torch.cuda.device(state.device):
+        rc = load_library().toploc_stream_begin(_dev_ptr(state), ctypes.byref(lay), _stream_ptr(stream))
+    _check(rc, "toploc_stream_begin")
+    return state
+
+
+def toploc_stream_append(rows, lay, token_in_chunk, state, stream=None):
+    """rows: CUDA tensor [num_seqs, hidden], row `token_in_chunk` of every sequence's running chunk."""
+    if not rows.is_cuda:
+        raise ToplocError("toploc_stream_append needs CUDA tensors")
+    with torch.cuda.device(rows.device):
+        rc = load_library().toploc_stream_append(_dev_ptr(rows), ctypes.byref(lay), int(token_in_chunk),
+                                                 _dev_ptr(state), _stream_ptr(stream))
+    _check(rc, "toploc_stream_append")
+
+
+def toploc_stream_finish(state, lay, proofs=None, status=None, indices=None, workspace=None, stream=None,
+                         want_indices=False):
+    """Proofs of the chunks as they stand.  Returns (proofs uint8[num_seqs, proof bytes],
+    status uint8[num_seqs], indices int32[num_seqs, k] or None)."""
+    dev = state.device
+    n, pb = lay.num_seqs, toploc_layout_proof_bytes(lay)
+    if proofs is None:
+        proofs = torch.empty((n, pb), dtype=torch.uint8, device=dev)
+    if status is None:
+        status = torch.empty((n,), dtype=torch.uint8, device=dev)
+    if indices is None and want_indices:
+        indices = torch.empty((n, lay.k), dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(max(16, toploc_stream_workspace_bytes(lay)), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_stream_finish(
+            _dev_ptr(state), ctypes.byref(lay), _dev_ptr(proofs), _dev_ptr(status), _dev_ptr(indices),
+            _dev_ptr(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "toploc_stream_finish")
+    return proofs, status, indices

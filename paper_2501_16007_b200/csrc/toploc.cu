@@ -788,6 +788,10 @@ __device__ __forceinline__ ChunkPlace locate_chunk(const BatchParams& bp, long l
 // select kernel: topk() of Algorithms 1 and 2, one chunk per block; for proof
 // generation (sel.proofs != nullptr) also findInjectiveModulus() of Algorithm 1.
 // ---------------------------------------------------------------------------
+template <int DT>
+__device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchParams& bp, long long chunk,
+                                                  const Selection& sel);
+
 template <int DT, int MODE>
 __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_select_kernel(BatchParams bp, Selection sel) {
   __shared__ SelectShared sh;
@@ -795,7 +799,6 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
   const long long chunk = blockIdx.x;
   const int k = bp.k;
   uint16_t* proof = sel.proofs ? reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_stride(bp)) : nullptr;
-  const bool wide = DT == 1 && bp.coef_bytes == 4;
   int32_t* indices = sel.indices ? sel.indices + chunk * k : nullptr;
 
   const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
@@ -814,8 +817,20 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
   src.hidden = bp.hidden;
   src.vecs_per_row = bp.hidden / ChunkSource<DT, MODE>::kVec;
   select_topk<DT, MODE>(sh, src, (int)n_elems, k);
+  publish_selection<DT>(sh, bp, chunk, sel);
+}
 
-  // hand the selection to the interpolation kernel; rank order only where the caller asked for indices
+// The chunk's selection (sh.cand[0..k)) goes to the interpolation kernel: indices
+// and patterns to scratch, rank order where the caller asked for indices, and
+// for proof generation the modulus (Algorithm 6) and the chunk's status.
+template <int DT>
+__device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchParams& bp, long long chunk,
+                                                  const Selection& sel) {
+  const int tid = threadIdx.x;
+  const int k = bp.k;
+  uint16_t* proof = sel.proofs ? reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_stride(bp)) : nullptr;
+  const bool wide = DT == 1 && bp.coef_bytes == 4;
+  int32_t* indices = sel.indices ? sel.indices + chunk * k : nullptr;
   uint32_t unrepresentable = 0;
   for (int j = tid; j < k; j += kThreads) {
     const unsigned long long cj = sh.cand[j];
@@ -1680,6 +1695,88 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
 }
 
 // ---------------------------------------------------------------------------
+// Incremental proof generation (the provider's side during decoding, Section
+// 5.5: a proof per 32 new tokens): the rows of a chunk arrive one token at a
+// time, while they are still warm in L2, and each sequence keeps its running
+// top-k between the steps.  Streaming a chunk in index order and keeping the
+// best k so far (ties to the lower index) yields the chunk's top-k, so the
+// result equals toploc_build_proofs over the assembled chunk.
+// ---------------------------------------------------------------------------
+struct StreamHeader {  // per sequence, followed by kMaxK-independent room for k candidates
+  uint32_t count;      // candidates held (at most k between steps)
+  uint32_t thr;        // an element is a candidate iff its key is >= thr
+  uint32_t pad[2];
+};
+
+__host__ __device__ inline size_t stream_state_stride(int k) { return sizeof(StreamHeader) + 8 * (size_t)k; }
+
+// One new row per sequence: token t of the running chunk.  One warp per sequence.
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kThreads)
+toploc_stream_append_kernel(const char* rows, long long row_stride, int hidden, int k, int token,
+                            unsigned char* state) {
+  constexpr int VEC = ChunkSource<DT, MODE>::kVec;
+  constexpr int kElem = DT == 0 ? 2 : 4;
+  __shared__ SelectShared sh;
+  const int lane = threadIdx.x;
+  const long long seq = blockIdx.x;
+  StreamHeader* head = reinterpret_cast<StreamHeader*>(state + seq * stream_state_stride(k));
+  unsigned long long* held = reinterpret_cast<unsigned long long*>(head + 1);
+  WarpState st;
+  st.count = (int)head->count;
+  st.thr = head->thr;
+  st.nhits = 0;
+  for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
+  if (lane == 0) sh.top_bin = kNoBin;
+  warp_barrier();
+  for (int e = lane; e < st.count; e += kThreads) {
+    const unsigned long long c = held[e];
+    sh.cand[e] = c;
+    atomicAdd(&sh.top_hist[coarse_key<DT>(c) >> 7], 1u);
+  }
+  warp_barrier();
+  // the row stands at flat indices token * hidden ..: a source whose vector token * (hidden / VEC) is the row's first
+  ChunkSource<DT, MODE> src;
+  src.base = rows + seq * row_stride * kElem - (long long)token * hidden * kElem;
+  src.row_stride = hidden;
+  src.hidden = hidden;
+  src.vecs_per_row = hidden / VEC;
+  const int per_row = hidden / VEC;
+  st = select_carefully<DT, MODE>(sh, src, token * per_row, (token + 1) * per_row, k, st);
+  st = compact_candidates<DT>(sh, k, st, true);  // at most k are carried to the next step
+  warp_barrier();
+  for (int e = lane; e < st.count; e += kThreads) held[e] = sh.cand[e];
+  if (lane == 0) {
+    head->count = (uint32_t)st.count;
+    head->thr = st.thr;
+  }
+}
+
+// The running selections become the chunks' selections: what the select kernel
+// leaves behind, for the interpolation kernel to finish.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) toploc_stream_finish_kernel(BatchParams bp, Selection sel,
+                                                                        const unsigned char* state) {
+  __shared__ SelectShared sh;
+  const int lane = threadIdx.x;
+  const long long seq = blockIdx.x;
+  const int k = bp.k;
+  const StreamHeader* head = reinterpret_cast<const StreamHeader*>(state + seq * stream_state_stride(k));
+  const unsigned long long* held = reinterpret_cast<const unsigned long long*>(head + 1);
+  if ((int)head->count < k) {
+    uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + seq * proof_stride(bp));
+    for (int i = lane; i < proof_words(bp); i += kThreads) proof[i] = 0;
+    if (sel.indices)
+      for (int i = lane; i < k; i += kThreads) sel.indices[seq * k + i] = 0;
+    if (lane == 0) sel.status[seq] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+    return;
+  }
+  for (int e = lane; e < k; e += kThreads) sh.cand[e] = held[e];
+  warp_barrier();
+  publish_selection<DT>(sh, bp, seq, sel);
+}
+
+// ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
 struct HostPlan {
@@ -2064,6 +2161,51 @@ StagingPlan carve_staging_for(const toploc_layout* lay, int s0, int s1) {
   return carve_staging(lay, seq_begin(lay, s1) - seq_begin(lay, s0), chunks, segs);
 }
 
+// What the incremental entry points accept: one chunk per sequence, short enough
+// for the 24-bit index field of a candidate.
+int plan_stream(const toploc_layout* lay) {
+  if (lay == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->dtype != TOPLOC_DTYPE_BF16 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
+  if (lay->hidden <= 0 || lay->chunk_len <= 0 || lay->num_seqs <= 0 || lay->k < 1 || lay->row_stride < lay->hidden)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field != TOPLOC_FIELD_16 && lay->field != TOPLOC_FIELD_32) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field == TOPLOC_FIELD_32 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
+  if (lay->k > TOPLOC_MAX_K) return TOPLOC_ERR_UNSUPPORTED;
+  if ((long long)lay->hidden * lay->chunk_len > kMaxSegmentElems) return TOPLOC_ERR_UNSUPPORTED;
+  return TOPLOC_OK;
+}
+
+template <int DT>
+void launch_stream_append(int mode, const toploc_layout* lay, const void* d_rows, int token, void* d_state,
+                                 cudaStream_t stream) {
+  const char* rows = static_cast<const char*>(d_rows);
+  unsigned char* state = static_cast<unsigned char*>(d_state);
+  const unsigned grid = (unsigned)lay->num_seqs;
+  if (mode == 0)
+    toploc_stream_append_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(rows, lay->row_stride, lay->hidden, lay->k,
+                                                                      token, state);
+  else
+    toploc_stream_append_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(rows, lay->row_stride, lay->hidden, lay->k,
+                                                                      token, state);
+}
+
+// Algorithm 3 and encode() for the chunks whose selection and modulus are in place.
+void launch_interpolation(const toploc_layout* lay, const DeviceInfo* dev, const Selection& sel, long long num_chunks,
+                          cudaStream_t stream) {
+  if (lay->field == TOPLOC_FIELD_32) {
+    const long long q_blocks = (num_chunks + kInterpQWarps - 1) / kInterpQWarps;
+    toploc_interpolate_q_kernel<<<(unsigned)q_blocks, kInterpQWarps * 32, 0, stream>>>(sel, lay->k, num_chunks);
+    return;
+  }
+  // one block per SM; a small batch gets a block for every four of its groups (each block first
+  // builds its table of inverses, so not one per group)
+  const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
+  long long blocks = (groups + 3) / 4;
+  if (blocks > dev->sms) blocks = dev->sms;
+  toploc_interpolate_kernel<<<(unsigned)blocks, kInterpWarps * 32, interp_smem_bytes(), stream>>>(sel, lay->k,
+                                                                                                 num_chunks);
+}
+
 }  // namespace
 
 // ===========================================================================
@@ -2144,18 +2286,7 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
   rc = run_select(d_act, lay, d_workspace, workspace_bytes, stream, d_status, d_proofs, d_indices_opt, &plan,
                   &sel, &dev);
   if (rc != TOPLOC_OK) return rc;
-  if (lay->field == TOPLOC_FIELD_32) {
-    const long long q_blocks = (plan.num_chunks + kInterpQWarps - 1) / kInterpQWarps;
-    toploc_interpolate_q_kernel<<<(unsigned)q_blocks, kInterpQWarps * 32, 0, stream>>>(sel, lay->k, plan.num_chunks);
-    return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
-  }
-  // one block per SM; a small batch gets a block for every four of its groups (each block first
-  // builds its table of inverses, so not one per group)
-  const long long groups = (plan.num_chunks + kInterpChunks - 1) / kInterpChunks;
-  long long blocks = (groups + 3) / 4;
-  if (blocks > dev->sms) blocks = dev->sms;
-  toploc_interpolate_kernel<<<(unsigned)blocks, kInterpWarps * 32, interp_smem_bytes(), stream>>>(
-      sel, lay->k, plan.num_chunks);
+  launch_interpolation(lay, dev, sel, plan.num_chunks, stream);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
@@ -2235,6 +2366,80 @@ int toploc_build_proofs_builtin_scratch(const void* d_act, const toploc_layout* 
   // selection and status entry that the interpolation kernel goes on to read.
   return toploc_build_proofs(d_act, lay, d_proofs, d_status, d_indices_opt, scratch, kBuiltinScratchBytes,
                              cuda_stream);
+}
+
+// ---- incremental proof generation -------------------------------------------
+
+size_t toploc_stream_state_bytes(const toploc_layout* lay) {
+  return plan_stream(lay) == TOPLOC_OK ? (size_t)lay->num_seqs * stream_state_stride(lay->k) : 0;
+}
+
+size_t toploc_stream_workspace_bytes(const toploc_layout* lay) {
+  if (plan_stream(lay) != TOPLOC_OK) return 0;
+  return plan_workspace(false, lay->num_seqs, lay->k, lay->num_seqs, coef_bytes_of(lay)).total;
+}
+
+int toploc_stream_begin(void* d_state, const toploc_layout* lay, void* cuda_stream) {
+  int rc = plan_stream(lay);
+  if (rc != TOPLOC_OK) return rc;
+  if (d_state == nullptr || reinterpret_cast<uintptr_t>(d_state) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  // empty running selections: nothing held, every element is a candidate
+  return cudaMemsetAsync(d_state, 0, toploc_stream_state_bytes(lay), static_cast<cudaStream_t>(cuda_stream)) ==
+                 cudaSuccess
+             ? TOPLOC_OK
+             : TOPLOC_ERR_CUDA;
+}
+
+int toploc_stream_append(const void* d_rows, const toploc_layout* lay, int32_t token_in_chunk, void* d_state,
+                         void* cuda_stream) {
+  int rc = plan_stream(lay);
+  if (rc != TOPLOC_OK) return rc;
+  if (d_rows == nullptr || d_state == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (token_in_chunk < 0 || token_in_chunk >= lay->chunk_len) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(d_state) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  DeviceInfo* dev = nullptr;
+  if ((rc = device_info(&dev)) != TOPLOC_OK) return rc;
+  // rows that are 16-byte aligned are read as vectors, others element by element
+  const int mode = pick_mode(d_rows, lay) == 2 ? 2 : 0;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (lay->dtype == TOPLOC_DTYPE_BF16) launch_stream_append<0>(mode, lay, d_rows, token_in_chunk, d_state, stream);
+  else launch_stream_append<1>(mode, lay, d_rows, token_in_chunk, d_state, stream);
+  return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+}
+
+int toploc_stream_finish(const void* d_state, const toploc_layout* lay, uint8_t* d_proofs, uint8_t* d_status,
+                         int32_t* d_indices_opt, void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = plan_stream(lay);
+  if (rc != TOPLOC_OK) return rc;
+  if (d_state == nullptr || d_proofs == nullptr || d_status == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (reinterpret_cast<uintptr_t>(d_proofs) % 2 != 0 || reinterpret_cast<uintptr_t>(d_state) % 16 != 0)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  const WorkspacePlan wp = plan_workspace(false, lay->num_seqs, lay->k, lay->num_seqs, coef_bytes_of(lay));
+  if (d_workspace == nullptr || workspace_bytes < wp.total) return TOPLOC_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(d_workspace) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  DeviceInfo* dev = nullptr;
+  if ((rc = device_info(&dev)) != TOPLOC_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(d_workspace);
+  BatchParams bp = {};
+  bp.hidden = lay->hidden;
+  bp.chunk_len = lay->chunk_len;
+  bp.k = lay->k;
+  bp.coef_bytes = (int)coef_bytes_of(lay);
+  Selection sel;
+  sel.idx = reinterpret_cast<uint32_t*>(ws + wp.idx_off);
+  sel.bits = reinterpret_cast<uint16_t*>(ws + wp.bits_off);
+  sel.bits32 = reinterpret_cast<uint32_t*>(ws + wp.bits_off);
+  sel.status = d_status;
+  sel.proofs = d_proofs;
+  sel.indices = d_indices_opt;
+  const unsigned char* state = static_cast<const unsigned char*>(d_state);
+  const long long n = lay->num_seqs;
+  if (lay->dtype == TOPLOC_DTYPE_BF16) toploc_stream_finish_kernel<0><<<(unsigned)n, kThreads, 0, stream>>>(bp, sel, state);
+  else toploc_stream_finish_kernel<1><<<(unsigned)n, kThreads, 0, stream>>>(bp, sel, state);
+  if (cudaGetLastError() != cudaSuccess) return TOPLOC_ERR_CUDA;
+  launch_interpolation(lay, dev, sel, n, stream);
+  return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
 // Shared driver of the two host-memory entry points: groups of whole sequences
