@@ -685,7 +685,11 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
 // ---------------------------------------------------------------------------
 __host__ __device__ constexpr uint32_t mul_mod(uint32_t a, uint32_t b) { return (a * b) % kPrime; }
 __device__ __forceinline__ uint32_t mad_mod(uint32_t a, uint32_t b, uint32_t c) { return (a * b + c) % kPrime; }
-__device__ __forceinline__ uint32_t sub_mod(uint32_t a, uint32_t b) { return a >= b ? a - b : a + kPrime - b; }
+// a - b in Z_p, given neg_b = p - b (in (0, p]).
+__device__ __forceinline__ uint32_t diff_mod(uint32_t a, uint32_t neg_b) {
+  const uint32_t d = a + neg_b;   // in (0, 2p)
+  return min(d, d - kPrime);      // d - p wraps to a huge value when d < p
+}
 
 __host__ __device__ constexpr uint32_t pow_mod(uint32_t a, uint32_t e) {
   uint32_t r = 1;
@@ -883,8 +887,9 @@ __device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchP
 
 // Algorithm 3 for NCH chunks of one warp at a time (their dependency chains are
 // independent, which keeps the issue slots filled).  inv[] is the table of
-// inverses in Z_p; xw / aw are this warp's scratch rows (NCH x kMaxK entries
-// each).  A chunk that is not live is carried along with zeros and not written.
+// inverses in Z_p; xa is this warp's scratch (NCH rows of kMaxK words: x_j in the
+// lower half of word j, the Newton coefficient a_j in the upper half).  A chunk
+// that is not live is carried along with zeros and not written.
 //
 // Divided differences are taken point by point instead of level by level (the
 // same table, visited row-wise): with a_0 = y_0, step i lets every later point j
@@ -897,10 +902,10 @@ __device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchP
 // with coefficient d in lane d / SLOTS, slot d % SLOTS, so that the shift by one
 // degree stays inside a lane except for one value per lane and step.
 template <int SLOTS, int NCH>
-__device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t* xw, uint16_t* aw, int k,
-                                                   const Selection& sel, const long long (&chunk)[NCH],
-                                                   const bool (&live)[NCH]) {
+__device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t* xa, int k, const Selection& sel,
+                                                   const long long (&chunk)[NCH], const bool (&live)[NCH]) {
   const int lane = threadIdx.x & 31;
+  uint16_t* a_half = reinterpret_cast<uint16_t*>(xa) + 1;  // the upper half of word j: a_j
   const size_t proof_bytes = 2 + 2 * (size_t)k;
   uint32_t x[NCH][SLOTS], t[NCH][SLOTS];
 #pragma unroll
@@ -925,33 +930,42 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t
         }
         x[c][s] = r;
         t[c][s] = y;
-        xw[c * kMaxK + j] = (uint16_t)r;
-        if (j == 0) aw[c * kMaxK] = (uint16_t)y;
+        xa[c * kMaxK + j] = r | (j == 0 ? y << 16 : 0u);  // x_j below, a_j above (a_0 = y_0; the others follow)
       }
     }
   }
+  // Steps i = 32 b + ii: the points of slot b in lanes above ii and every point of the later
+  // slots take part (no per-slot tests inside the loop); x_i and a_i come as one word.
+#pragma unroll
+  for (int b = 0; b < SLOTS; ++b) {
+    const int steps = min(32, k - 1 - 32 * b);
 #pragma unroll 1
-  for (int i = 0; i + 1 < k; ++i) {
-    __syncwarp();  // a_i has been stored
-    uint32_t a_i[NCH], x_i[NCH];
+    for (int ii = 0; ii < steps; ++ii) {
+      const int i = 32 * b + ii;
+      __syncwarp();  // a_i has been stored
+      uint32_t neg_a[NCH], neg_x[NCH];
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      a_i[c] = aw[c * kMaxK + i];
-      x_i[c] = xw[c * kMaxK + i];
-    }
-    const int s_lo = (i + 1) >> 5;
+      for (int c = 0; c < NCH; ++c) {
+        const uint32_t pair = xa[c * kMaxK + i];
+        neg_x[c] = kPrime - (pair & 0xFFFFu);
+        neg_a[c] = kPrime - (pair >> 16);
+      }
 #pragma unroll
-    for (int s = 0; s < SLOTS; ++s) {
-      if (s >= s_lo) {
-        const int j = s * 32 + lane;
-        const bool active = j > i && j < k;
+      for (int c = 0; c < NCH; ++c) {
+        // a point at or before i computes a value that is dropped (its span indexes the table all the same)
+        const uint32_t next = mul_mod(diff_mod(t[c][b], neg_a[c]), inv[diff_mod(x[c][b], neg_x[c])]);
+        t[c][b] = lane > ii ? next : t[c][b];
+        if (lane == ii + 1) a_half[2 * (c * kMaxK + i + 1)] = (uint16_t)next;
+      }
 #pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-          const uint32_t span = active ? sub_mod(x[c][s], x_i[c]) : 0u;
-          const uint32_t next = mul_mod(sub_mod(t[c][s], a_i[c]), inv[span]);
-          t[c][s] = active ? next : t[c][s];
-          if (s == s_lo && j == i + 1) aw[c * kMaxK + j] = (uint16_t)next;
-        }
+      for (int s = b + 1; s < SLOTS; ++s) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c)
+          t[c][s] = mul_mod(diff_mod(t[c][s], neg_a[c]), inv[diff_mod(x[c][s], neg_x[c])]);
+      }
+      if (b + 1 < SLOTS && ii == 31 && lane == 0) {  // the next coefficient belongs to the next slot
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) a_half[2 * (c * kMaxK + i + 1)] = (uint16_t)t[c][b + 1 < SLOTS ? b + 1 : b];
       }
     }
   }
@@ -961,18 +975,17 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint16_t
   for (int c = 0; c < NCH; ++c) {
 #pragma unroll
     for (int b = 0; b < SLOTS; ++b) co[c][b] = 0;
-    if (lane == 0) co[c][0] = aw[c * kMaxK + k - 1];
+    if (lane == 0) co[c][0] = xa[c * kMaxK + k - 1] >> 16;
   }
 #pragma unroll 1
   for (int i = k - 2; i >= 0; --i) {
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
-      const uint32_t xi = xw[c * kMaxK + i];
-      const uint32_t neg_x = xi ? kPrime - xi : 0u;
-      const uint32_t a_i = aw[c * kMaxK + i];
+      const uint32_t pair = xa[c * kMaxK + i];
+      const uint32_t neg_x = kPrime - (pair & 0xFFFFu);  // p for x_i = 0, which multiplies like 0
       // coefficient d takes  c[d-1] + (-x_i) c[d];  entries above the current degree are 0 and stay 0
       uint32_t carry = __shfl_up_sync(0xFFFFFFFFu, co[c][SLOTS - 1], 1);
-      if (lane == 0) carry = a_i;
+      if (lane == 0) carry = pair >> 16;  // a_i
 #pragma unroll
       for (int b = SLOTS - 1; b >= 1; --b) co[c][b] = mad_mod(co[c][b], neg_x, co[c][b - 1]);
       co[c][0] = mad_mod(co[c][0], neg_x, carry);
@@ -1017,8 +1030,7 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
     }
   }
   __syncthreads();
-  uint16_t* xw = scratch + warp * 2 * kInterpChunks * kMaxK;
-  uint16_t* aw = xw + kInterpChunks * kMaxK;
+  uint32_t* xa = reinterpret_cast<uint32_t*>(scratch) + warp * kInterpChunks * kMaxK;
   const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
   // group g goes to block g % gridDim.x, so a small batch spreads over the blocks before it fills their warps
   for (long long g = blockIdx.x + (long long)gridDim.x * warp; g < groups;
@@ -1037,10 +1049,10 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
       any |= live[c];
     }
     if (!any) continue;
-    if (k <= 32) interpolate_chunks<1, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
-    else if (k <= 64) interpolate_chunks<2, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
-    else if (k <= 128) interpolate_chunks<4, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
-    else interpolate_chunks<kMaxSlots, kInterpChunks>(inv, xw, aw, k, sel, chunk, live);
+    if (k <= 32) interpolate_chunks<1, kInterpChunks>(inv, xa, k, sel, chunk, live);
+    else if (k <= 64) interpolate_chunks<2, kInterpChunks>(inv, xa, k, sel, chunk, live);
+    else if (k <= 128) interpolate_chunks<4, kInterpChunks>(inv, xa, k, sel, chunk, live);
+    else interpolate_chunks<kMaxSlots, kInterpChunks>(inv, xa, k, sel, chunk, live);
   }
 }
 
