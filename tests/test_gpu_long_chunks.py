@@ -78,6 +78,13 @@ def test_chunk_beyond_two_to_the_24_elements():
     parity_case(act, 4100, 128, 1, 4100, recomputed=rec, where="33M")
 
 
+def test_very_wide_rows_become_one_segment_each():
+    """hidden = 2^20: 24 rows are 25 M elements; no segment may hold more than 2^24 of them, and none can
+    split a row, so every row is a segment of its own (k = 64, fp32 committed as 16 bits)."""
+    act = synth.make_activations(1, 24, 1 << 20, torch.float32, seed=43, device=DEV, outliers="none")
+    parity_case(act, 24, 64, 1, 24, where="wide rows")
+
+
 def test_host_buffer_entry_points_with_a_long_chunk():
     lens = [650, 64]
     offs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)

@@ -98,6 +98,10 @@ def test_long_chunks_are_planned_in_segments():
     assert tl.toploc_workspace_bytes(direct) < 2 * 1024           # 2^19 elements: selected directly
     huge_len = layout(hidden=8192, row_stride=8192, chunk_len=1 << 30, tokens_per_seq=5000, num_seqs=2, k=128)
     assert tl.toploc_num_chunks(huge_len) == 2                    # 5000 x 8192 = 41 M elements each
+    # the 24-bit index field of a candidate can force more than 64 segments: 1100 rows of 2^20
+    # elements, at most 16 rows per segment -> 69 segments
+    forced = layout(hidden=1 << 20, row_stride=1 << 20, chunk_len=1100, tokens_per_seq=1100, num_seqs=1, k=128)
+    assert 69 * per_seg <= tl.toploc_workspace_bytes(forced) - 128 * 6 <= 69 * per_seg + 8 * 256
     lib = tl.load_library()
     assert lib.toploc_build_proofs_builtin_scratch(ctypes.c_void_p(16), ctypes.byref(long_one), ctypes.c_void_p(16),
                                                    ctypes.c_void_p(16), None, None) == -2
