@@ -6,18 +6,26 @@
 //                 topk()), then runs the injective-modulus search (Algorithm 6).
 //                 The k (index, pattern) pairs go to scratch memory.
 //   interpolate   one warp per chunk does the arithmetic over Z_p: Newton
-//                 interpolation and packing (Algorithm 3).
+//                 interpolation and packing (Algorithm 3).  fp32 chunks that
+//                 commit whole patterns use a second interpolation kernel over
+//                 Z_q, q = 2^32 - 5.
 // Validation, one kernel per call:
 //   verify        the same selection (Algorithm 2, topk()), after which the same
 //                 warp evaluates the committed polynomial at its k points
 //                 (Algorithm 5), compares bit fields, and writes statistics and
 //                 verdict.  Nothing goes through scratch memory.
+// Around these:
+//   merge         a chunk too long for one warp (a prompt as one chunk) is
+//                 selected in segments by the select kernel; the merge kernel
+//                 joins the segments' winners and runs the tail of its call.
+//   stream        incremental proof generation: one new row per sequence and
+//                 decode step updates a running selection kept in device memory.
 //
 // The path is a selection over data read once plus integer modular arithmetic:
 // HBM bandwidth is the roofline, there is no dense contraction and therefore no
 // tensor-core work.  The selection keeps its loads in flight as asynchronous
 // copies into a small shared-memory ring per warp (many independent warps per
-// SM, none waits on another) and spends about one instruction per five
+// SM, none waits on another) and spends about one instruction per seven
 // elements on the elements that lose.
 #include "toploc.h"
 
