@@ -162,12 +162,12 @@ def decode32(proof):
     return st, k.value, m.value, c[:k.value]
 
 
-def _batch_dtype_code(act, wide):
+def _batch_dtype_code(act, wide, padded=False):
     code = _dtype_code(act)
-    if wide:
+    if wide or padded:
         if code != 1:
-            raise TypeError("the 32-bit field variant commits fp32 activations")
-        return 2
+            raise TypeError("the 32-bit field variant and the padded comparison are for fp32 activations")
+        return 3 if padded else 2
     return code
 
 
@@ -202,8 +202,10 @@ def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None
 
 def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None,
                   t_exp=38, t_mean=10.0, t_median=8.0, sign_in_exponent=True, gen_indices=None,
-                  first_chunk=0, last_chunk=-1, threads=None, wide=False):
-    """Returns a structured array (RESULT_DTYPE) with one entry per chunk."""
+                  first_chunk=0, last_chunk=-1, threads=None, wide=False, padded=False):
+    """Returns a structured array (RESULT_DTYPE) with one entry per chunk.
+    padded: fp32 activations against 16-bit field proofs, the committed patterns padded with 16 zero
+    bits and compared as fp32 (Section 5.6)."""
     assert act.ndim == 2 and act.strides[1] == act.itemsize
     hidden = act.shape[1]
     row_stride = act.strides[0] // act.itemsize
@@ -214,7 +216,7 @@ def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_off
     gi = None if gen_indices is None else np.ascontiguousarray(gen_indices, np.int32)
     results = np.zeros(n, RESULT_DTYPE)
     lib().oracle_verify_proofs(
-        _ptr(act), _batch_dtype_code(act, wide), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
+        _ptr(act), _batch_dtype_code(act, wide, padded), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
         None if so is None else _ptr(so), ctypes.c_int64(row_stride), ctypes.c_int64(first_chunk),
         ctypes.c_int64(last_chunk), _ptr(proofs), int(t_exp), ctypes.c_double(t_mean),
         ctypes.c_double(t_median), int(bool(sign_in_exponent)), None if gi is None else _ptr(gi),

@@ -20,7 +20,8 @@
  *   - fp32 activations rank on the 31-bit magnitude and commit the upper 16
  *     bits of the pattern (Section 5.6, mantissa scaled to bf16), or, in the
  *     32-bit field variant further down (dtype code 2 of the batch drivers),
- *     the whole pattern over Z_q, q = 2^32 - 5.
+ *     the whole pattern over Z_q, q = 2^32 - 5; dtype code 3 validates fp32
+ *     activations against a 16-bit field proof padded with 16 zero bits.
  *
  * Pins (tests/test_oracle_*.py): worked examples and the paper's printed
  * values under tests/golden/, brute force on tiny inputs, P(x_j) = y_j with
@@ -690,6 +691,77 @@ void oracle_verify_chunk32(const void* chunk, int rows, int hidden, int64_t row_
   free(diffs);
 }
 
+/* Algorithm 2 for an fp32 validator against the proof of a bf16 generator
+ * (Section 5.6: "when validating a bf16 decode model with fp32, we padded 16
+ * zero bits to the bf16 representation").  The proof is an ordinary 16-bit
+ * field proof; the validator ranks its fp32 chunk on the full magnitude,
+ * evaluates the polynomial over Z_p, pads the committed 16-bit pattern with 16
+ * zero bits and compares fp32 bit fields (23-bit mantissas), which is what the
+ * fp32 thresholds of Section 5.2 apply to. */
+void oracle_verify_chunk_padded(const void* chunk, int rows, int hidden, int64_t row_stride, int k,
+                                const uint8_t* proof, int t_exp, double t_mean, double t_median,
+                                int sign_in_exponent, const int32_t* gen_indices_opt, oracle_result* out) {
+  memset(out, 0, sizeof(*out));
+  out->topk_mismatch = -1;
+  uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* pattern = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* coef = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  uint32_t* diffs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  int kk = 0;
+  uint32_t m = 0;
+  int status = oracle_decode(proof, 2 + 2 * (int64_t)k, &kk, &m, coef);
+  out->modulus = m;
+  if (status == ST_OK) status = topk_patterns32(chunk, rows, hidden, row_stride, k, idx, pattern);
+  if (status == ST_OK) {
+    uint32_t err_e = 0, n = 0;
+    uint64_t sum = 0;
+    for (int j = 0; j < k; ++j) {
+      uint32_t committed = oracle_horner(coef, k, (idx[j] % m) % P_FIELD) << 16; /* padded with 16 zero bits */
+      uint32_t seen = pattern[j];
+      uint32_t e_p = committed >> 23, e_v = seen >> 23;
+      if (!sign_in_exponent) {
+        e_p &= 0xFFu;
+        e_v &= 0xFFu;
+      }
+      uint32_t m_p = committed & 0x7FFFFFu, m_v = seen & 0x7FFFFFu;
+      if (e_p == e_v) {
+        uint32_t d = m_p > m_v ? m_p - m_v : m_v - m_p;
+        diffs[n++] = d;
+        sum += d;
+      } else {
+        ++err_e;
+      }
+    }
+    out->exp_mismatch = err_e;
+    out->n_match = n;
+    out->mant_diff_sum = (uint32_t)sum;
+    if (n > 0) {
+      out->mant_mean = (double)sum / (double)n;
+      qsort(diffs, n, sizeof(uint32_t), ascending_u32);
+      out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
+    }
+    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    if (n == 0) reject = 1;
+    out->accept = reject ? 0 : 1;
+    if (gen_indices_opt) {
+      int common = 0;
+      for (int a = 0; a < k; ++a)
+        for (int b = 0; b < k; ++b)
+          if ((uint32_t)gen_indices_opt[a] == idx[b]) {
+            ++common;
+            break;
+          }
+      out->topk_mismatch = k - common;
+    }
+  }
+  out->status = (uint8_t)status;
+  if (status != ST_OK) out->accept = 0;
+  free(idx);
+  free(pattern);
+  free(coef);
+  free(diffs);
+}
+
 /* ------------------------------------------------------------------ */
 /* Batch drivers: chunks of chunk_len rows per sequence (Section 5.5:   */
 /* one proof per 32 new tokens), the last chunk of a sequence may be    */
@@ -751,6 +823,11 @@ static void* worker(void* arg) {
       jb->status[c] = (uint8_t)oracle_build_chunk32(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
                                                     jb->proofs + (size_t)c * pbytes,
                                                     jb->indices ? jb->indices + (size_t)c * jb->k : NULL);
+    } else if (jb->verify && jb->dtype == 3) {
+      oracle_verify_chunk_padded(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
+                                 jb->proofs_in + (size_t)c * pbytes, jb->t_exp, jb->t_mean, jb->t_median,
+                                 jb->sign_in_exponent,
+                                 jb->gen_indices ? jb->gen_indices + (size_t)c * jb->k : NULL, &jb->results[c]);
     } else if (wide) {
       oracle_verify_chunk32(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
                             jb->proofs_in + (size_t)c * pbytes, jb->t_exp, jb->t_mean, jb->t_median,

@@ -200,3 +200,35 @@ def test_wide_and_narrow_proofs_of_an_fp32_chunk_share_selection_and_modulus():
     narrow, _, ni = oracle.build_proofs(act, 32, 128, 1, 32)
     assert wi.tolist() == ni.tolist() and wide[0, :2].tolist() == narrow[0, :2].tolist()
     assert wide.shape[1] == 2 + 4 * 128 and narrow.shape[1] == 2 + 2 * 128
+
+
+def test_padded_validation_of_a_bf16_proof_against_fp32_activations():
+    """Section 5.6: the committed 16-bit pattern is padded with 16 zero bits and compared with the fp32
+    validator's pattern.  fp32 values whose upper halves are the generator's bf16 patterns differ from
+    the padded commitment by exactly their lower 16 bits."""
+    upper = np.zeros((4, 64), np.uint16)
+    upper[0, :8] = [0x4480, 0xC400, 0x4380, 0x4300, 0x4280, 0x4200, 0x4180, 0x4100]    # 1024, -512, 256 .. 8
+    low = np.zeros((4, 64), np.uint32)
+    deltas = [0, 1, 77, 300, 20000, 0x7FFF, 5, 5]
+    low[0, :8] = deltas
+    fp32 = (upper.astype(np.uint32) << 16) | low
+    proofs, status, idx = oracle.build_proofs(upper, 4, 8, 1, 4)                       # the bf16 generator
+    assert status.tolist() == [0] and proofs.shape == (1, 2 + 2 * 8)
+    res = oracle.verify_proofs(fp32.view(np.float32), proofs, 4, 8, 1, 4, t_exp=8, t_mean=1e9, t_median=1e9,
+                               gen_indices=idx, padded=True)[0]
+    assert res["exp_mismatch"] == 0 and res["n_match"] == 8 and res["topk_mismatch"] == 0
+    assert res["mant_diff_sum"] == sum(deltas) and res["mant_mean"] == sum(deltas) / 8
+    assert res["mant_median"] == (5 + 77) / 2 and res["accept"] == 1                   # 0 1 5 5 | 77 300 20000 32767
+    strict = oracle.verify_proofs(fp32.view(np.float32), proofs, 4, 8, 1, 4, t_exp=8, t_mean=256.0,
+                                  t_median=128.0, padded=True)[0]
+    assert strict["accept"] == 0                                                       # the mean is far above 256
+    exact = oracle.verify_proofs((upper.astype(np.uint32) << 16).view(np.float32), proofs, 4, 8, 1, 4, t_exp=8,
+                                 t_mean=256.0, t_median=128.0, padded=True)[0]
+    assert exact["accept"] == 1 and exact["mant_diff_sum"] == 0
+    # an exponent change in the validator's value is an exponent mismatch, not a mantissa difference
+    bumped = fp32.copy()
+    bumped[0, 4] += 1 << 23
+    assert oracle.verify_proofs(bumped.view(np.float32), proofs, 4, 8, 1, 4, t_exp=8, t_mean=1e9, t_median=1e9,
+                                padded=True)[0]["exp_mismatch"] == 1
+    with pytest.raises(TypeError):
+        oracle.verify_proofs(upper, proofs, 4, 8, 1, 4, padded=True)
