@@ -51,6 +51,14 @@ extern "C" {
 #define TOPLOC_FIELD_16 0
 #define TOPLOC_FIELD_32 1
 #define TOPLOC_FIELD_32_PRIME 4294967291u
+/* Validation only (toploc_verify_proofs and its _host variant), fp32 chunks
+ * only: the proofs are TOPLOC_FIELD_16 proofs of a bf16 generator; the
+ * polynomial is evaluated over Z_p, every committed 16-bit pattern is padded
+ * with 16 zero bits and compared with the validator's whole fp32 pattern
+ * (23-bit mantissas, the fp32 thresholds) -- the "bf16 model validated with
+ * fp32" case of Section 5.6.  Proofs keep 2 + 2k bytes.  The generating entry
+ * points return TOPLOC_ERR_UNSUPPORTED for it. */
+#define TOPLOC_FIELD_16_PADDED 2
 
 /* Largest k the kernels are built for and largest chunk (elements; only chunks
  * the layout really contains count, so chunk_len may exceed every sequence).
@@ -96,7 +104,7 @@ typedef struct {
   int32_t chunk_len;          /* L > 0 tokens per chunk (32 in Section 5.5) */
   int32_t k;                  /* 1..TOPLOC_MAX_K (128 in the paper) */
   int32_t num_seqs;           /* > 0 */
-  int32_t field;              /* TOPLOC_FIELD_* (0 = 16-bit field, the default) */
+  int32_t field;              /* TOPLOC_FIELD_* (0 = 16-bit field, the default); fp32 only for the others */
   int64_t tokens_per_seq;     /* uniform sequence length; used when seq_offsets == NULL */
   const int64_t* seq_offsets; /* HOST, optional: num_seqs + 1 ascending row offsets (ragged batch);
                                  read before the call returns */

@@ -15,7 +15,7 @@ __all__ = [
     "ToplocLayout", "ToplocThresholds", "make_layout", "library_path", "load_library",
     "toploc_num_chunks", "toploc_proof_bytes", "toploc_layout_proof_bytes", "toploc_workspace_bytes",
     "toploc_staging_bytes", "toploc_stream_state_bytes", "toploc_stream_workspace_bytes", "toploc_stream_begin",
-    "toploc_stream_append", "toploc_stream_finish", "TOPLOC_FIELD_16", "TOPLOC_FIELD_32", "TOPLOC_FIELD_32_PRIME",
+    "toploc_stream_append", "toploc_stream_finish", "TOPLOC_FIELD_16", "TOPLOC_FIELD_32", "TOPLOC_FIELD_16_PADDED", "TOPLOC_FIELD_32_PRIME",
     "toploc_get_constants", "toploc_status_string", "toploc_error_string",
     "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
     "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES", "toploc_select_topk",
@@ -24,6 +24,7 @@ __all__ = [
 TOPLOC_DTYPE_BF16 = 0
 TOPLOC_FIELD_16 = 0
 TOPLOC_FIELD_32 = 1
+TOPLOC_FIELD_16_PADDED = 2   # validation only: fp32 activations against 16-bit field proofs
 TOPLOC_FIELD_32_PRIME = 4294967291
 TOPLOC_DTYPE_FP32 = 1
 TOPLOC_MAX_K = 256
@@ -262,7 +263,7 @@ def default_thresholds(k=128, sign_in_exponent=True, field=TOPLOC_FIELD_16):
     for fp32 inference (TOPLOC_FIELD_32, 23-bit mantissas); the exponent threshold scales with k for
     other proof sizes."""
     thr = ToplocThresholds()
-    wide = field == TOPLOC_FIELD_32
+    wide = field in (TOPLOC_FIELD_32, TOPLOC_FIELD_16_PADDED)
     thr.t_exp = ((8 if wide else 38) * k) // 128
     thr.sign_in_exponent = 1 if sign_in_exponent else 0
     thr.t_mean = 256.0 if wide else 10.0

@@ -107,6 +107,7 @@ struct BatchParams {
   int k;
   int chunks_per_seq;
   int coef_bytes;              // 2: coefficients in Z_p; 4: fp32 chunks over Z_q, q = 2^32 - 5
+  int padded;                  // validation only: fp32 chunks against Z_p proofs, commitments padded to 32 bits
 };
 
 __device__ __forceinline__ size_t proof_stride(const BatchParams& bp) { return 2 + (size_t)bp.coef_bytes * bp.k; }
@@ -1342,19 +1343,24 @@ toploc_interpolate_q_kernel(Selection sel, int k, long long num_chunks) {
 // (Algorithm 5), extractBits() (bit 31 sign, bits 30..23 exponent, bits 22..0
 // mantissa), error accumulation, verdict.  The median of up to k 23-bit
 // differences is found by rank counting (no histogram fits).
-template <int SLOTS>
+// PADDED: the proof is a 16-bit field proof (a bf16 generator's); the polynomial is evaluated
+// over Z_p and the committed 16-bit pattern padded with 16 zero bits before the comparison
+// (Section 5.6, fp32 validator of a bf16 model).
+template <int SLOTS, bool PADDED>
 __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long long chunk, const uint32_t (&idx)[SLOTS],
                                                 const uint32_t (&pattern)[SLOTS], const VerifyIo& io,
                                                 toploc_chunk_result res) {
   const int lane = threadIdx.x;
-  const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 4 * (size_t)k));
+  const uint16_t* proof =
+      reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + (PADDED ? 2 : 4) * (size_t)k));
   // the selection has left shared memory, so the ring is free: three rows of kMaxK words
   uint32_t* coef = reinterpret_cast<uint32_t*>(sh.ring);
   uint32_t* gen = coef + kMaxK;
   uint32_t* diffs = gen + kMaxK;
   constexpr uint32_t kNoMatch = 0xFFFFFFFFu;  // larger than any 23-bit difference
   warp_barrier();
-  for (int d = lane; d < k; d += 32) coef[d] = (uint32_t)proof[1 + 2 * d] | ((uint32_t)proof[2 + 2 * d] << 16);
+  for (int d = lane; d < k; d += 32)
+    coef[d] = PADDED ? (uint32_t)proof[1 + d] : ((uint32_t)proof[1 + 2 * d] | ((uint32_t)proof[2 + 2 * d] << 16));
   if (io.gen_indices)
     for (int j = lane; j < k; j += 32) gen[j] = (uint32_t)io.gen_indices[chunk * k + j];
   warp_barrier();
@@ -1364,13 +1370,18 @@ __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long lo
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
     x[s] = idx[s] % m;
+    if (PADDED && x[s] >= kPrime) x[s] -= kPrime;
     acc[s] = coef[k - 1];  // Horner, highest degree first
   }
 #pragma unroll 2
   for (int d = k - 2; d >= 0; --d) {
     const uint32_t cd = coef[d];
 #pragma unroll
-    for (int s = 0; s < SLOTS; ++s) acc[s] = mad_q(acc[s], x[s], cd);
+    for (int s = 0; s < SLOTS; ++s) acc[s] = PADDED ? mad_mod(acc[s], x[s], cd) : mad_q(acc[s], x[s], cd);
+  }
+  if (PADDED) {
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) acc[s] <<= 16;  // the committed 16-bit pattern, 16 zero bits below it
   }
   uint32_t err_e = 0, diff_sum = 0, common = 0;
 #pragma unroll
@@ -1449,8 +1460,8 @@ __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long lo
 }
 
 template <int DT, int SLOTS>
-__device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, bool wide, long long chunk, const VerifyIo& io,
-                                             const toploc_chunk_result& res) {
+__device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, bool wide, bool padded, long long chunk,
+                                             const VerifyIo& io, const toploc_chunk_result& res) {
   const int lane = threadIdx.x;
   uint32_t idx[SLOTS], bits[SLOTS];
 #pragma unroll
@@ -1466,7 +1477,8 @@ __device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, bool wide,
       bits[s] = (DT == 1 && wide) ? ((sign << 31) | key) : ((sign << 15) | (DT == 0 ? key : (key >> 16)));
     }
   }
-  if (DT == 1 && wide) evaluate_warp_q<SLOTS>(sh, k, chunk, idx, bits, io, res);
+  if (DT == 1 && wide && padded) evaluate_warp_q<SLOTS, true>(sh, k, chunk, idx, bits, io, res);
+  else if (DT == 1 && wide) evaluate_warp_q<SLOTS, false>(sh, k, chunk, idx, bits, io, res);
   else evaluate_warp<SLOTS>(sh, k, chunk, idx, bits, io, res);
 }
 
@@ -1534,11 +1546,12 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
   src.vecs_per_row = bp.hidden / ChunkSource<DT, MODE>::kVec;
   select_topk<DT, MODE>(sh, src, (int)n_elems, k);
 
-  const bool wide = bp.coef_bytes == 4;
-  if (k <= 32) verify_chunk<DT, 1>(sh, k, wide, chunk, io, res);
-  else if (k <= 64) verify_chunk<DT, 2>(sh, k, wide, chunk, io, res);
-  else if (k <= 128) verify_chunk<DT, 4>(sh, k, wide, chunk, io, res);
-  else verify_chunk<DT, kMaxSlots>(sh, k, wide, chunk, io, res);
+  const bool padded = bp.padded != 0;
+  const bool wide = bp.coef_bytes == 4 || padded;  // whole patterns are compared
+  if (k <= 32) verify_chunk<DT, 1>(sh, k, wide, padded, chunk, io, res);
+  else if (k <= 64) verify_chunk<DT, 2>(sh, k, wide, padded, chunk, io, res);
+  else if (k <= 128) verify_chunk<DT, 4>(sh, k, wide, padded, chunk, io, res);
+  else verify_chunk<DT, kMaxSlots>(sh, k, wide, padded, chunk, io, res);
 }
 
 // ---------------------------------------------------------------------------
@@ -1559,7 +1572,8 @@ __device__ __forceinline__ void finish_merged(SelectShared& sh, const BatchParam
                                               const toploc_chunk_result& res) {
   const int lane = threadIdx.x;
   const int k = bp.k;
-  const bool wide = DT == 1 && bp.coef_bytes == 4;
+  const bool padded = DT == 1 && TAIL == 2 && bp.padded != 0;
+  const bool wide = DT == 1 && (bp.coef_bytes == 4 || padded);
   uint32_t idx[kMaxK / kThreads], bits[SLOTS];
   uint32_t unrepresentable = 0;
 #pragma unroll
@@ -1606,7 +1620,8 @@ __device__ __forceinline__ void finish_merged(SelectShared& sh, const BatchParam
     uint32_t own[SLOTS];
 #pragma unroll
     for (int e = 0; e < SLOTS; ++e) own[e] = idx[e];
-    if (wide) evaluate_warp_q<SLOTS>(sh, k, chunk, own, bits, io, res);
+    if (padded) evaluate_warp_q<SLOTS, true>(sh, k, chunk, own, bits, io, res);
+    else if (wide) evaluate_warp_q<SLOTS, false>(sh, k, chunk, own, bits, io, res);
     else evaluate_warp<SLOTS>(sh, k, chunk, own, bits, io, res);
   }
 }
@@ -1842,8 +1857,9 @@ int plan_layout(const toploc_layout* lay, HostPlan* plan) {
   if (lay == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (lay->dtype != TOPLOC_DTYPE_BF16 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
   if (lay->hidden <= 0 || lay->chunk_len <= 0 || lay->num_seqs <= 0) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (lay->field != TOPLOC_FIELD_16 && lay->field != TOPLOC_FIELD_32) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (lay->field == TOPLOC_FIELD_32 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
+  if (lay->field != TOPLOC_FIELD_16 && lay->field != TOPLOC_FIELD_32 && lay->field != TOPLOC_FIELD_16_PADDED)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field != TOPLOC_FIELD_16 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
   if (lay->k < 1) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (lay->k > TOPLOC_MAX_K) return TOPLOC_ERR_UNSUPPORTED;
   if (lay->row_stride < lay->hidden) return TOPLOC_ERR_INVALID_ARGUMENT;
@@ -2094,6 +2110,7 @@ int prepare_batch(const void* d_act, const toploc_layout* lay, void* d_workspace
   bp->k = lay->k;
   bp->chunks_per_seq = plan->chunks_per_seq;
   bp->coef_bytes = (int)coef_bytes_of(lay);
+  bp->padded = lay->field == TOPLOC_FIELD_16_PADDED;
   if (plan->ragged || plan->split) {
     if ((rc = upload_spans(lay, *plan, ws + wp.spans_off, ws + wp.chunk_table_off, stream)) != TOPLOC_OK) return rc;
     bp->spans = reinterpret_cast<const ChunkSpan*>(ws + wp.spans_off);
@@ -2299,6 +2316,7 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
   if (rc != TOPLOC_OK) return rc;
   if (d_act == nullptr || d_proofs == nullptr || d_status == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (reinterpret_cast<uintptr_t>(d_proofs) % 2 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field == TOPLOC_FIELD_16_PADDED) return TOPLOC_ERR_UNSUPPORTED;  // a way to validate, not to commit
   if (plan.num_chunks == 0) return TOPLOC_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   Selection sel;

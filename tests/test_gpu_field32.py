@@ -121,3 +121,35 @@ def test_host_entry_points_and_refusals():
     bf = act.to(torch.bfloat16)
     with pytest.raises(tl.ToplocError):
         tl.make_layout(bf, 32, 128, 3, 64, field=WIDE) and tl.toploc_num_chunks(tl.make_layout(bf, 32, 128, 3, 64, field=WIDE)[0])
+
+
+def test_fp32_validator_of_a_bf16_model_pads_the_commitments():
+    """Section 5.6: proofs generated from bf16 activations, validated against the fp32 activations they
+    were rounded from, the committed patterns padded with 16 zero bits: exponents agree, the mantissas
+    differ by what the rounding removed (thousands of fp32 units), so the fp32 thresholds reject."""
+    PAD = tl.TOPLOC_FIELD_16_PADDED
+    full = synth.make_activations(3, 64, 2048, torch.float32, seed=21, device=DEV, outliers="none")
+    model = full.to(torch.bfloat16)                           # what the bf16 generator computed with
+    g = gpu_build(model, 32, 128, 3, 64)
+    r = oracle.build_proofs(synth.host_patterns(model), 32, 128, 3, 64)
+    assert_build_equal(g, r, "bf16 generator")
+    kw = oracle_thresholds(128, wide=True)
+    for name, seen in (("fp32 original", full), ("bf16 values as fp32", model.to(torch.float32))):
+        gv = gpu_verify(seen, g[0], 32, 128, 3, 64, gen_indices=g[2], field=PAD)
+        rv = oracle.verify_proofs(synth.host_patterns(seen), r[0], 32, 128, 3, 64, gen_indices=r[2], padded=True, **kw)
+        assert_results_equal(gv, rv, "padded " + name)
+        if name.startswith("bf16"):
+            assert rv["accept"].all() and not rv["mant_diff_sum"].any()
+        else:
+            assert not rv["accept"].any() and (rv["mant_mean"] > 256.0).all()
+    # a long chunk and the host entry point take the same path
+    long_full = synth.make_activations(1, 300, 4096, torch.float32, seed=22, device=DEV, outliers="none")
+    long_model = long_full.to(torch.bfloat16)
+    lg = gpu_build(long_model, 300, 128, 1, 300)
+    lr = oracle.build_proofs(synth.host_patterns(long_model), 300, 128, 1, 300)
+    gv = gpu_verify(long_full, lg[0], 300, 128, 1, 300, gen_indices=lg[2], field=PAD)
+    rv = oracle.verify_proofs(synth.host_patterns(long_full), lr[0], 300, 128, 1, 300, gen_indices=lr[2], padded=True, **kw)
+    assert_results_equal(gv, rv, "padded long chunk")
+    lay, _ = tl.make_layout(full, 32, 128, 3, 64, field=PAD)
+    with pytest.raises(tl.ToplocError, match="unsupported"):
+        tl.toploc_build_proofs(full, lay)

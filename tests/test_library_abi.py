@@ -83,6 +83,12 @@ def test_the_32_bit_field_is_for_fp32_and_doubles_the_coefficients():
     thr = tl.default_thresholds(128, field=tl.TOPLOC_FIELD_32)
     assert (thr.t_exp, thr.t_mean, thr.t_median) == (8, 256.0, 128.0)
     assert tl.TOPLOC_FIELD_32_PRIME == 2 ** 32 - 5
+    padded = layout(dtype=1, field=tl.TOPLOC_FIELD_16_PADDED)       # validating a bf16 model's proofs with fp32
+    assert tl.toploc_layout_proof_bytes(padded) == 258
+    assert tl.toploc_workspace_bytes(padded) == tl.toploc_workspace_bytes(narrow)
+    lib = tl.load_library()
+    assert lib.toploc_build_proofs(ctypes.c_void_p(16), ctypes.byref(padded), ctypes.c_void_p(16),
+                                   ctypes.c_void_p(16), None, None, 0, None) == -2
 
 
 def test_long_chunks_are_planned_in_segments():
@@ -109,7 +115,7 @@ def test_long_chunks_are_planned_in_segments():
 
 @pytest.mark.parametrize("bad", [dict(k=0), dict(k=257), dict(hidden=0), dict(chunk_len=0), dict(num_seqs=0),
                                  dict(dtype=7), dict(row_stride=100), dict(tokens_per_seq=0),
-                                 dict(field=1), dict(field=2), dict(dtype=1, field=-1),
+                                 dict(field=1), dict(field=2), dict(dtype=1, field=3), dict(dtype=1, field=-1),
                                  dict(hidden=1 << 20, chunk_len=2048, tokens_per_seq=4096, row_stride=1 << 20),
                                  dict(hidden=(1 << 24) + 8, row_stride=(1 << 24) + 8)])
 def test_invalid_layouts_are_refused(bad):
