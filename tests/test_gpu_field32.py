@@ -153,3 +153,40 @@ def test_fp32_validator_of_a_bf16_model_pads_the_commitments():
     lay, _ = tl.make_layout(full, 32, 128, 3, 64, field=PAD)
     with pytest.raises(tl.ToplocError, match="unsupported"):
         tl.toploc_build_proofs(full, lay)
+
+
+def test_the_four_generation_validation_precision_pairs():
+    """The pairs of the precision table in Section 5.6 on synthetic activations: an fp32 model passes both
+    validators, a bf16 model only the bf16 one."""
+    S, T, H, L, k = 2, 64, 4096, 32, 128
+    full = synth.make_activations(S, T, H, torch.float32, seed=23, device=DEV, outliers="none")
+    half = full.to(torch.bfloat16)
+    recomputed_full = noise(full, 24, 2.0 ** -22)             # each validator recomputes with its own rounding noise
+    recomputed_half = synth.honest_noise(half, seed=25)
+    outcomes = {}
+    # fp32 model, fp32 validator: whole patterns, fp32 thresholds
+    _, out = parity_case(full, L, k, S, T, recomputed={"v": recomputed_full}, where="fp32-fp32", wide=True)
+    outcomes["fp32-fp32"] = out["v"]["accept"].all()
+    # fp32 model, bf16 validator: 16-bit commitments of the fp32 values, bf16 thresholds
+    g = gpu_build(full, L, k, S, T)
+    r = oracle.build_proofs(synth.host_patterns(full), L, k, S, T)
+    assert_build_equal(g, r, "fp32 model, 16-bit field")
+    gv = gpu_verify(recomputed_half, g[0], L, k, S, T, gen_indices=g[2])
+    rv = oracle.verify_proofs(synth.host_patterns(recomputed_half), r[0], L, k, S, T, gen_indices=r[2],
+                              **oracle_thresholds(k))
+    assert_results_equal(gv, rv, "fp32-bf16")
+    outcomes["fp32-bf16"] = rv["accept"].all()
+    # bf16 model: bf16 validator, then fp32 validator with padded commitments
+    g = gpu_build(half, L, k, S, T)
+    r = oracle.build_proofs(synth.host_patterns(half), L, k, S, T)
+    gv = gpu_verify(recomputed_half, g[0], L, k, S, T, gen_indices=g[2])
+    rv = oracle.verify_proofs(synth.host_patterns(recomputed_half), r[0], L, k, S, T, gen_indices=r[2],
+                              **oracle_thresholds(k))
+    assert_results_equal(gv, rv, "bf16-bf16")
+    outcomes["bf16-bf16"] = rv["accept"].all()
+    gv = gpu_verify(recomputed_full, g[0], L, k, S, T, gen_indices=g[2], field=tl.TOPLOC_FIELD_16_PADDED)
+    rv = oracle.verify_proofs(synth.host_patterns(recomputed_full), r[0], L, k, S, T, gen_indices=r[2], padded=True,
+                              **oracle_thresholds(k, wide=True))
+    assert_results_equal(gv, rv, "bf16-fp32")
+    outcomes["bf16-fp32"] = rv["accept"].any()
+    assert outcomes == {"fp32-fp32": True, "fp32-bf16": True, "bf16-bf16": True, "bf16-fp32": False}
