@@ -650,6 +650,14 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
         copy_async_wait<kStages - 1>();  // this lane's copies of `tile` have landed
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) w[u] = sh.ring[(stage * kUnroll + u) * kThreads + lane];
+        // Refill the stage as soon as the tile is in registers instead of after its tests.  The
+        // instructions below read one register of every load, so they issue only once all of
+        // them have returned; the copies are issued after them and cannot overwrite a slot
+        // that is still being read.
+        uint32_t landed = 0;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) asm volatile("or.b32 %0, %0, %1;" : "+r"(landed) : "r"(w[u].x));
+        request_tile(tile + kStages, stage);
       } else {
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) w[u] = src.load(v0 + u * kThreads + lane);
@@ -677,7 +685,7 @@ __device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, 
           st.nhits += __popc(votes[u]);
         }
       }
-      request_tile(tile + kStages, stage);  // refill the stage just consumed
+      if (!kRing) request_tile(tile + kStages, stage);  // (keeps the commit-group count in step; no copies)
       // a tile parks at most kTileVecs vectors, so the buffer cannot overflow
       if (st.nhits >= kHitTrigger) st = drain_hits<DT, MODE>(sh, src, k, st);
     }
