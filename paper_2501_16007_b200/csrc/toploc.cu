@@ -248,6 +248,15 @@ struct ChunkSource {
 // its top bit exactly when key >= thr (no carry leaves a lane).
 __device__ __forceinline__ uint32_t bf16_lane_add(uint32_t thr) { return (0x8000u - thr) * 0x00010001u; }
 
+// Per 16-bit lane the larger magnitude of two bf16 values (the sign bit of the result is not
+// meaningful); a NaN in either gives the all-ones magnitude, which every threshold lets through
+// to the exact unpacking.
+__device__ __forceinline__ uint32_t max_magnitude_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.NaN.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+
 template <int DT, int VEC>
 __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uint32_t add) {
   if (VEC == 1) {
@@ -255,9 +264,8 @@ __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uin
   } else if (DT == 0) {
     // largest key of each 16-bit lane over the four words (three-input packed maximum), then
     // the add-and-test-top-bit comparison once
-    const uint32_t m = __vimax3_u16x2(__vimax3_u16x2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu, w.z & 0x7FFF7FFFu),
-                                      w.w & 0x7FFF7FFFu, 0u);
-    return ((m + add) & 0x80008000u) != 0;
+    const uint32_t m = max_magnitude_bf16x2(max_magnitude_bf16x2(w.x, w.y), max_magnitude_bf16x2(w.z, w.w));
+    return (((m & 0x7FFF7FFFu) + add) & 0x80008000u) != 0;
   } else {
     return max(max(w.x & 0x7FFFFFFFu, w.y & 0x7FFFFFFFu), max(w.z & 0x7FFFFFFFu, w.w & 0x7FFFFFFFu)) >= thr;
   }
