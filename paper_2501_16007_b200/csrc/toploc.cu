@@ -262,8 +262,8 @@ __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uin
   if (VEC == 1) {
     return (DT == 0 ? (w.x & 0x7FFFu) : (w.x & 0x7FFFFFFFu)) >= thr;
   } else if (DT == 0) {
-    // largest key of each 16-bit lane over the four words (three-input packed maximum), then
-    // the add-and-test-top-bit comparison once
+    // largest magnitude of each 16-bit lane over the four words (three packed maxima, no sign
+    // masking of the inputs), then the add-and-test-top-bit comparison once
     const uint32_t m = max_magnitude_bf16x2(max_magnitude_bf16x2(w.x, w.y), max_magnitude_bf16x2(w.z, w.w));
     return (((m & 0x7FFF7FFFu) + add) & 0x80008000u) != 0;
   } else {
