@@ -43,7 +43,7 @@ WIDE_WORKLOADS = ("70b-fp32-wide", "8b-fp32-wide")
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one toploc_select_kernel launch on the full
 # batch (ncu, profiles/launch_list_70b_shape.md); None where no capture of the current kernel exists
-SELECT_DRAM_BYTES_PER_LAUNCH = {"70b": 17478986982 + 25839590}
+SELECT_DRAM_BYTES_PER_LAUNCH = {"70b": 17474558106 + 25958630}
 
 
 def measured_hbm_peak():
