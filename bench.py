@@ -117,15 +117,18 @@ def reference_arm(args, rank):
     import oracle
     from paper_2501_16007_b200 import synth
     S, T, H, L, k, seed = WORKLOADS[args.workload]
-    act = synth.make_activations(1, T, H, torch.bfloat16, seed=seed, device="cpu")
-    noisy = synth.honest_noise(act, seed=seed + 1)
+    wide = args.workload in WIDE_WORKLOADS
+    act = synth.make_activations(1, T, H, torch.float32 if wide else torch.bfloat16, seed=seed, device="cpu",
+                                 outliers="jitter" if wide else "fixed")
+    noisy = act.clone() if L * H > (1 << 19) else synth.honest_noise(act, seed=seed + 1, rel=2.0 ** (-22 if wide else -8))
     host, host_noisy = synth.host_patterns(act), synth.host_patterns(noisy)
     chunks = T // L
     cores = oracle.default_threads()
+    thr = {"t_exp": 8 * k // 128, "t_mean": 256.0, "t_median": 128.0} if wide else {}
 
     def step():
-        proofs, status, idx = oracle.build_proofs(host, L, k, 1, T, threads=cores)
-        oracle.verify_proofs(host_noisy, proofs, L, k, 1, T, gen_indices=idx, threads=cores)
+        proofs, status, idx = oracle.build_proofs(host, L, k, 1, T, threads=cores, wide=wide)
+        oracle.verify_proofs(host_noisy, proofs, L, k, 1, T, gen_indices=idx, threads=cores, wide=wide, **thr)
 
     for _ in range(args.warmup):
         step()
@@ -141,7 +144,8 @@ def reference_arm(args, rank):
         "dtype": "u32", "data": "synthetic",
         "config": {"workload": workload_name(args.workload), "sample": "first sequence (%d chunks) per step" % chunks},
         "cpu_baseline": {"value": value, "unit": "chunks/s", "cores": cores, "kind": "oracle",
-                         "sample": "first sequence: %d chunks of %d x %d bf16, build + verify" % (chunks, L, H)},
+                         "sample": "first sequence: %d chunks of %d x %d %s, build + verify" % (
+                             chunks, L, H, "fp32 (32-bit field)" if wide else "bf16")},
         "e2e": {"value": value, "unit": "chunks/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
