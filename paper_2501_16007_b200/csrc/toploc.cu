@@ -257,6 +257,13 @@ __device__ __forceinline__ uint32_t max_magnitude_bf16x2(uint32_t a, uint32_t b)
   return d;
 }
 
+// The same for two fp32 values.
+__device__ __forceinline__ uint32_t max_magnitude_f32(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.NaN.xorsign.abs.f32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+
 template <int DT, int VEC>
 __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uint32_t add) {
   if (VEC == 1) {
@@ -267,7 +274,8 @@ __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uin
     const uint32_t m = max_magnitude_bf16x2(max_magnitude_bf16x2(w.x, w.y), max_magnitude_bf16x2(w.z, w.w));
     return (((m & 0x7FFF7FFFu) + add) & 0x80008000u) != 0;
   } else {
-    return max(max(w.x & 0x7FFFFFFFu, w.y & 0x7FFFFFFFu), max(w.z & 0x7FFFFFFFu, w.w & 0x7FFFFFFFu)) >= thr;
+    const uint32_t m = max_magnitude_f32(max_magnitude_f32(w.x, w.y), max_magnitude_f32(w.z, w.w));
+    return (m & 0x7FFFFFFFu) >= thr;
   }
 }
 
