@@ -1769,6 +1769,44 @@ struct StreamHeader {  // per sequence, followed by kMaxK-independent room for k
 
 __host__ __device__ inline size_t stream_state_stride(int k) { return sizeof(StreamHeader) + 8 * (size_t)k; }
 
+// Vectors [vb, ve) against a threshold that is already meaningful: the filter of the select kernel's
+// streaming loop (test, park the vectors that reach the threshold, unpack them by the warp), with
+// plain loads instead of the ring.
+template <int DT, int MODE>
+__device__ __forceinline__ WarpState filter_vectors(SelectShared& sh, const ChunkSource<DT, MODE>& src, int vb, int ve,
+                                                    int k, WarpState st) {
+  constexpr int VEC = ChunkSource<DT, MODE>::kVec;
+  const int lane = threadIdx.x;
+  const uint32_t below = (1u << lane) - 1u;
+  for (int v0 = vb; v0 < ve; v0 += kThreads * kUnroll) {
+    uint4 w[kUnroll];
+    bool hit[kUnroll];
+    uint32_t votes[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int v = v0 + u * kThreads + lane;
+      w[u] = v < ve ? src.load(v) : make_uint4(0, 0, 0, 0);
+    }
+    const uint32_t add = bf16_lane_add(st.thr);
+    uint32_t any_votes = 0;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      hit[u] = (v0 + u * kThreads + lane < ve) && vector_reaches<DT, VEC>(w[u], st.thr, add);
+      votes[u] = __ballot_sync(0xFFFFFFFFu, hit[u]);
+      any_votes |= votes[u];
+    }
+    if (any_votes) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (hit[u]) sh.hit_idx[st.nhits + __popc(votes[u] & below)] = (uint32_t)(v0 + u * kThreads + lane);
+        st.nhits += __popc(votes[u]);
+      }
+      if (st.nhits >= kHitTrigger) st = drain_hits<DT, MODE>(sh, src, k, st);
+    }
+  }
+  return drain_hits<DT, MODE>(sh, src, k, st);
+}
+
 // One new row per sequence: token t of the running chunk.  One warp per sequence.
 template <int DT, int MODE>
 __global__ void __launch_bounds__(kThreads)
@@ -1801,7 +1839,9 @@ toploc_stream_append_kernel(const char* rows, long long row_stride, int hidden, 
   src.hidden = hidden;
   src.vecs_per_row = hidden / VEC;
   const int per_row = hidden / VEC;
-  st = select_carefully<DT, MODE>(sh, src, token * per_row, (token + 1) * per_row, k, st);
+  // once k candidates are held the threshold does the work; before that every element is a candidate
+  if (st.count >= k) st = filter_vectors<DT, MODE>(sh, src, token * per_row, (token + 1) * per_row, k, st);
+  else st = select_carefully<DT, MODE>(sh, src, token * per_row, (token + 1) * per_row, k, st);
   st = compact_candidates<DT>(sh, k, st, true);  // at most k are carried to the next step
   warp_barrier();
   for (int e = lane; e < st.count; e += kThreads) held[e] = sh.cand[e];
