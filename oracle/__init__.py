@@ -222,3 +222,48 @@ def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_off
         ctypes.c_double(t_median), int(bool(sign_in_exponent)), None if gi is None else _ptr(gi),
         _ptr(results), threads or default_threads())
     return results
+
+
+def _chunk_spans(num_seqs, tokens_per_seq, chunk_len, seq_offsets):
+    spans = []
+    for s in range(num_seqs):
+        begin = int(seq_offsets[s]) if seq_offsets is not None else s * tokens_per_seq
+        end = int(seq_offsets[s + 1]) if seq_offsets is not None else begin + tokens_per_seq
+        for r in range(begin, end, chunk_len):
+            spans.append((r, min(chunk_len, end - r)))
+    return spans
+
+
+def commit_direct(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None):
+    """Direct commitments (Section 4: index and value stored as they are, 6 bytes per point).
+
+    Returns (commits uint8[n, 6k], status uint8[n])."""
+    assert act.ndim == 2 and act.strides[1] == act.itemsize
+    hidden, row_stride, code = act.shape[1], act.strides[0] // act.itemsize, _dtype_code(act)
+    spans = _chunk_spans(num_seqs, tokens_per_seq, chunk_len, seq_offsets)
+    commits = np.zeros((len(spans), 6 * k), np.uint8)
+    status = np.zeros(len(spans), np.uint8)
+    for c, (row0, rows) in enumerate(spans):
+        status[c] = lib().oracle_commit_direct_chunk(_ptr(act[row0:]), code, rows, hidden,
+                                                     ctypes.c_int64(row_stride), k, _ptr(commits[c]))
+    return commits, status
+
+
+def verify_direct(act, commits, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None,
+                  t_exp=38, t_mean=10.0, t_median=8.0, sign_in_exponent=True):
+    """Algorithm 2 against direct commitments.  Returns (results RESULT_DTYPE[n], exp_dev uint32[n, 9]):
+    exp_dev counts, over the indices both sides selected, the exponent deviations 0, -1, +1, -2, +2,
+    -10..-3, 3..10, 11..99 and >= 100 in absolute value (the columns of the table in Section 3)."""
+    assert act.ndim == 2 and act.strides[1] == act.itemsize
+    hidden, row_stride, code = act.shape[1], act.strides[0] // act.itemsize, _dtype_code(act)
+    spans = _chunk_spans(num_seqs, tokens_per_seq, chunk_len, seq_offsets)
+    commits = np.ascontiguousarray(commits, np.uint8)
+    assert commits.shape == (len(spans), 6 * k)
+    results = np.zeros(len(spans), RESULT_DTYPE)
+    exp_dev = np.zeros((len(spans), 9), np.uint32)
+    for c, (row0, rows) in enumerate(spans):
+        lib().oracle_verify_direct_chunk(
+            _ptr(act[row0:]), code, rows, hidden, ctypes.c_int64(row_stride), k, _ptr(commits[c]), int(t_exp),
+            ctypes.c_double(t_mean), ctypes.c_double(t_median), int(bool(sign_in_exponent)),
+            _ptr(results[c:c + 1]), _ptr(exp_dev[c]))
+    return results, exp_dev

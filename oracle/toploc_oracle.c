@@ -21,7 +21,10 @@
  *     bits of the pattern (Section 5.6, mantissa scaled to bf16), or, in the
  *     32-bit field variant further down (dtype code 2 of the batch drivers),
  *     the whole pattern over Z_q, q = 2^32 - 5; dtype code 3 validates fp32
- *     activations against a 16-bit field proof padded with 16 zero bits.
+ *     activations against a 16-bit field proof padded with 16 zero bits;
+ *   - direct commitments (Section 4's 6 bytes per point, for k beyond what
+ *     Algorithm 6 can serve): records in ascending index order, an index
+ *     that was not committed counts as an exponent mismatch.
  *
  * Pins (tests/test_oracle_*.py): worked examples and the paper's printed
  * values under tests/golden/, brute force on tiny inputs, P(x_j) = y_j with
@@ -759,6 +762,160 @@ void oracle_verify_chunk_padded(const void* chunk, int rows, int hidden, int64_t
   free(idx);
   free(pattern);
   free(coef);
+  free(diffs);
+}
+
+/* ================================================================== */
+/* Direct commitments: Section 4 opens with the plain alternative to   */
+/* the polynomial, "storing top-k indices and values directly", at 6   */
+/* bytes per point (4 for the index, 2 for the value).  It is the only */
+/* form that exists for the larger k of the exponent-error table in    */
+/* Section 3 (k up to 4096): k indices below 2^16 residues collide for */
+/* every candidate modulus once k reaches the thousands, so Algorithm  */
+/* 6 has nothing to return there.  Readings used here:                 */
+/*   - a commitment is k records of 6 bytes, record j = flat index     */
+/*     (4 bytes little-endian) then the 16-bit pattern (2 bytes        */
+/*     little-endian), records in ascending index order (the paper     */
+/*     fixes no order; this one makes the bytes unique);               */
+/*   - validation is Algorithm 2 with "evaluate the polynomial at the  */
+/*     index" replaced by "look the index up": a recomputed top-k      */
+/*     index that was not committed has nothing to agree with and      */
+/*     counts as an exponent mismatch;                                 */
+/*   - a commitment whose indices are not strictly ascending or reach  */
+/*     beyond the chunk is malformed (ST_BAD_PROOF);                   */
+/*   - exponent deviation (the columns of the table in Section 3):     */
+/*     d = exponent field seen - exponent field committed, for every   */
+/*     index both sides selected, counted in nine bins: 0, -1, +1, -2, */
+/*     +2, -10..-3, 3..10, 11 <= |d| <= 99, |d| >= 100.                */
+/* ================================================================== */
+
+static int by_flat_index(const void* a, const void* b) {
+  const ranked* p = (const ranked*)a;
+  const ranked* q = (const ranked*)b;
+  return p->flat < q->flat ? -1 : (p->flat > q->flat ? 1 : 0);
+}
+
+/* commit: 6k bytes.  Returns ST_OK or ST_K_EXCEEDS (commit zero-filled). */
+int oracle_commit_direct_chunk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
+                               uint8_t* commit) {
+  memset(commit, 0, 6 * (size_t)k);
+  uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* bits = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  int status = oracle_topk(chunk, dtype, rows, hidden, row_stride, k, idx, bits);
+  if (status == ST_OK) {
+    ranked* pts = (ranked*)malloc((size_t)k * sizeof(ranked));
+    for (int j = 0; j < k; ++j) {
+      pts[j].key = 0;
+      pts[j].flat = idx[j];
+      pts[j].bits = bits[j];
+    }
+    qsort(pts, (size_t)k, sizeof(ranked), by_flat_index);
+    for (int j = 0; j < k; ++j) {
+      uint8_t* rec = commit + 6 * (size_t)j;
+      rec[0] = (uint8_t)(pts[j].flat & 0xFFu);
+      rec[1] = (uint8_t)((pts[j].flat >> 8) & 0xFFu);
+      rec[2] = (uint8_t)((pts[j].flat >> 16) & 0xFFu);
+      rec[3] = (uint8_t)(pts[j].flat >> 24);
+      rec[4] = (uint8_t)(pts[j].bits & 0xFFu);
+      rec[5] = (uint8_t)(pts[j].bits >> 8);
+    }
+    free(pts);
+  }
+  free(idx);
+  free(bits);
+  return status;
+}
+
+/* exp_dev: 9 counters (see above), may be NULL.  out->modulus stays 0 and
+ * out->topk_mismatch is always filled (the commitment carries the indices). */
+void oracle_verify_direct_chunk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
+                                const uint8_t* commit, int t_exp, double t_mean, double t_median,
+                                int sign_in_exponent, oracle_result* out, uint32_t* exp_dev) {
+  memset(out, 0, sizeof(*out));
+  if (exp_dev) memset(exp_dev, 0, 9 * sizeof(uint32_t));
+  uint32_t* c_idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* c_bits = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* bits = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  uint32_t* diffs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  int64_t n_elems = (int64_t)rows * hidden;
+  int status = ST_OK;
+  for (int j = 0; j < k; ++j) {
+    const uint8_t* rec = commit + 6 * (size_t)j;
+    c_idx[j] = (uint32_t)rec[0] | ((uint32_t)rec[1] << 8) | ((uint32_t)rec[2] << 16) | ((uint32_t)rec[3] << 24);
+    c_bits[j] = (uint16_t)(rec[4] | (rec[5] << 8));
+  }
+  if (k > n_elems) status = ST_K_EXCEEDS;
+  if (status == ST_OK) {
+    for (int j = 0; j < k; ++j) {
+      if ((int64_t)c_idx[j] >= n_elems) status = ST_BAD_PROOF;
+      if (j > 0 && c_idx[j] <= c_idx[j - 1]) status = ST_BAD_PROOF;
+    }
+  }
+  if (status == ST_OK) status = oracle_topk(chunk, dtype, rows, hidden, row_stride, k, idx, bits);
+  if (status == ST_OK) {
+    uint32_t err_e = 0, n = 0, sum = 0;
+    int common = 0;
+    for (int j = 0; j < k; ++j) {
+      int at = -1;
+      for (int a = 0; a < k; ++a)
+        if (c_idx[a] == idx[j]) at = a;
+      if (at < 0) {
+        ++err_e; /* nothing was committed for this index */
+        continue;
+      }
+      ++common;
+      uint32_t committed = c_bits[at], seen = bits[j];
+      uint32_t e_p, e_v;
+      if (sign_in_exponent) {
+        e_p = committed >> 7;
+        e_v = seen >> 7;
+      } else {
+        e_p = (committed >> 7) & 0xFFu;
+        e_v = (seen >> 7) & 0xFFu;
+      }
+      uint32_t m_p = committed & 0x7Fu, m_v = seen & 0x7Fu;
+      if (e_p == e_v) {
+        uint32_t d = m_p > m_v ? m_p - m_v : m_v - m_p;
+        diffs[n++] = d;
+        sum += d;
+      } else {
+        ++err_e;
+      }
+      if (exp_dev) {
+        int d = (int)((seen >> 7) & 0xFFu) - (int)((committed >> 7) & 0xFFu);
+        int a = d < 0 ? -d : d;
+        int bin;
+        if (d == 0) bin = 0;
+        else if (a == 1) bin = d < 0 ? 1 : 2;
+        else if (a == 2) bin = d < 0 ? 3 : 4;
+        else if (a <= 10) bin = d < 0 ? 5 : 6;
+        else if (a <= 99) bin = 7;
+        else bin = 8;
+        ++exp_dev[bin];
+      }
+    }
+    out->exp_mismatch = err_e;
+    out->n_match = n;
+    out->mant_diff_sum = sum;
+    out->topk_mismatch = k - common;
+    if (n > 0) {
+      out->mant_mean = (double)sum / (double)n;
+      qsort(diffs, n, sizeof(uint32_t), ascending_u32);
+      out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
+    }
+    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    if (n == 0) reject = 1;
+    out->accept = reject ? 0 : 1;
+  } else {
+    out->topk_mismatch = -1;
+  }
+  out->status = (uint8_t)status;
+  if (status != ST_OK) out->accept = 0;
+  free(c_idx);
+  free(c_bits);
+  free(idx);
+  free(bits);
   free(diffs);
 }
 
