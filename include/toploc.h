@@ -68,6 +68,9 @@ extern "C" {
  * exceed 2^24. */
 #define TOPLOC_MAX_K 256
 #define TOPLOC_MAX_CHUNK_ELEMS 0x7FFFFFFF
+/* Largest k of a direct commitment (toploc_commit_direct): the largest top-k
+ * the paper looks at (the exponent-error table of Section 3). */
+#define TOPLOC_MAX_K_DIRECT 4096
 
 /* Host-side return codes (0 = success, negative = nothing was enqueued). */
 #define TOPLOC_OK 0
@@ -245,6 +248,51 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
 int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_sel_indices,
                        uint16_t* d_sel_patterns, uint8_t* d_status, int32_t* d_ranked_indices_opt,
                        void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Direct commitments.  Section 4 starts from the plain way of committing to a
+ * chunk -- "storing top-k indices and values directly", 6 bytes per point: 4
+ * for the index and 2 for the value -- before replacing it by the polynomial.
+ * These two entry points are that plain form.  It is three times the size,
+ * but it exists for every k: with thousands of indices (the exponent-error
+ * table of Section 3 goes up to k = 4096) no modulus below 2^16 separates
+ * them, so Algorithm 6 has nothing to return and a polynomial proof cannot be
+ * made.  Same top-k as everywhere else (magnitude key, ties to the lower flat
+ * index), 16-bit patterns (fp32 chunks commit their upper 16 bits).
+ *
+ * A commitment is k records of 6 bytes in ascending index order (the paper
+ * fixes no order; this one makes the bytes unique): flat index, 4 bytes
+ * little-endian, then the pattern, 2 bytes little-endian.
+ *
+ * Validation is Algorithm 2 with the polynomial evaluation replaced by a
+ * look-up: for every index of the recomputed top-k, the committed pattern at
+ * that index is compared as in toploc_verify_proofs; an index that was not
+ * committed counts as an exponent mismatch.  topk_mismatch is always filled
+ * (the commitment carries the indices), modulus is 0.  A commitment whose
+ * indices do not ascend strictly or reach beyond the chunk gets
+ * TOPLOC_CHUNK_BAD_PROOF.  Thresholds as in toploc_thresholds (Section 5.2
+ * gives them for k = 128; the exponent threshold scales with k).
+ *
+ * d_commits      DEVICE  [num_chunks, 6k] bytes, 2-byte aligned; zero-filled by
+ *                        toploc_commit_direct for a chunk with fewer than k elements
+ * d_status       DEVICE  out, [num_chunks]: TOPLOC_CHUNK_OK or K_EXCEEDS_CHUNK
+ * d_results      DEVICE  out, [num_chunks]
+ * d_exp_dev_opt  DEVICE  out, optional: [num_chunks, 9] u32 counts of the exponent
+ *                        deviation (exponent field seen - committed, sign bit left
+ *                        out) over the indices both sides selected, in the columns of
+ *                        the table in Section 3: 0, -1, +1, -2, +2, -10..-3, 3..10,
+ *                        11 <= |d| <= 99, |d| >= 100
+ *
+ * Limits: lay->k up to TOPLOC_MAX_K_DIRECT, TOPLOC_FIELD_16, uniform batches
+ * (seq_offsets == NULL), chunks of at most 2^24 elements; otherwise
+ * TOPLOC_ERR_UNSUPPORTED.  No scratch memory is needed.  Asynchronous.
+ */
+size_t toploc_direct_commit_bytes(int32_t k); /* 6k */
+int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d_commits, uint8_t* d_status,
+                         void* cuda_stream);
+int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
+                         const toploc_thresholds* thr, toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt,
+                         void* cuda_stream);
 
 /*
  * toploc_build_proofs for callers that have no way to hand over scratch

@@ -19,6 +19,7 @@ __all__ = [
     "toploc_get_constants", "toploc_status_string", "toploc_error_string",
     "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
     "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES", "toploc_select_topk",
+    "TOPLOC_MAX_K_DIRECT", "toploc_direct_commit_bytes", "toploc_commit_direct", "toploc_verify_direct",
 ]
 
 TOPLOC_DTYPE_BF16 = 0
@@ -28,6 +29,7 @@ TOPLOC_FIELD_16_PADDED = 2   # validation only: fp32 activations against 16-bit 
 TOPLOC_FIELD_32_PRIME = 4294967291
 TOPLOC_DTYPE_FP32 = 1
 TOPLOC_MAX_K = 256
+TOPLOC_MAX_K_DIRECT = 4096
 TOPLOC_BUILTIN_SCRATCH_BYTES = 8 << 20
 
 RESULT_DTYPE = np.dtype([
@@ -105,6 +107,11 @@ def load_library():
     lib.toploc_select_topk.argtypes = [vp, lay_p, vp, vp, vp, vp, vp, sz, vp]
     lib.toploc_build_proofs_builtin_scratch.restype = ctypes.c_int
     lib.toploc_build_proofs_builtin_scratch.argtypes = [vp, lay_p, vp, vp, vp, vp]
+    lib.toploc_direct_commit_bytes.restype, lib.toploc_direct_commit_bytes.argtypes = sz, [i32]
+    lib.toploc_commit_direct.restype = ctypes.c_int
+    lib.toploc_commit_direct.argtypes = [vp, lay_p, vp, vp, vp]
+    lib.toploc_verify_direct.restype = ctypes.c_int
+    lib.toploc_verify_direct.argtypes = [vp, lay_p, vp, thr_p, vp, vp, vp]
     _LIB = lib
     return lib
 
@@ -389,3 +396,52 @@ def toploc_stream_finish(state, lay, proofs=None, status=None, indices=None, wor
             _dev_ptr(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "toploc_stream_finish")
     return proofs, status, indices
+
+
+def toploc_direct_commit_bytes(k):
+    return int(load_library().toploc_direct_commit_bytes(k))
+
+
+def _direct_chunks(lay):
+    # uniform batches only (the entry points refuse the others)
+    return lay.num_seqs * ((lay.tokens_per_seq + lay.chunk_len - 1) // lay.chunk_len)
+
+
+def toploc_commit_direct(act, lay, commits=None, status=None, stream=None):
+    """Direct commitments (Section 4: index and value as they are, 6 bytes per point), k up to
+    TOPLOC_MAX_K_DIRECT.  Returns (commits uint8 [n, 6k], status uint8 [n])."""
+    if not act.is_cuda:
+        raise ToplocError("toploc_commit_direct needs a CUDA tensor")
+    n, dev = _direct_chunks(lay), act.device
+    if commits is None:
+        commits = torch.empty((n, 6 * lay.k), dtype=torch.uint8, device=dev)
+    if status is None:
+        status = torch.empty((n,), dtype=torch.uint8, device=dev)
+    assert commits.is_contiguous() and commits.numel() == n * 6 * lay.k and status.numel() == n
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_commit_direct(_dev_ptr(act), ctypes.byref(lay), _dev_ptr(commits),
+                                                 _dev_ptr(status), _stream_ptr(stream))
+    _check(rc, "toploc_commit_direct")
+    return commits, status
+
+
+def toploc_verify_direct(act, lay, commits, thresholds=None, results=None, exp_dev=None, want_exp_dev=True,
+                         stream=None):
+    """Validation against direct commitments.  Returns (results uint8 [n, 40] -- view with
+    RESULT_DTYPE --, exp_dev int32 [n, 9] or None)."""
+    if not act.is_cuda:
+        raise ToplocError("toploc_verify_direct needs a CUDA tensor")
+    n, dev = _direct_chunks(lay), act.device
+    thr = thresholds if thresholds is not None else default_thresholds(lay.k)
+    if results is None:
+        results = torch.empty((n, RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    if exp_dev is None and want_exp_dev:
+        exp_dev = torch.empty((n, 9), dtype=torch.int32, device=dev)
+    assert commits.is_contiguous() and commits.numel() == n * 6 * lay.k
+    assert results.is_contiguous() and results.numel() == n * RESULT_DTYPE.itemsize
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_verify_direct(_dev_ptr(act), ctypes.byref(lay), _dev_ptr(commits),
+                                                 ctypes.byref(thr), _dev_ptr(results), _dev_ptr(exp_dev),
+                                                 _stream_ptr(stream))
+    _check(rc, "toploc_verify_direct")
+    return results, exp_dev

@@ -1,0 +1,574 @@
+// toploc_direct.cu -- direct commitments for sm_100a: the top-k indices and values of a
+// chunk stored as they are (Section 4: 6 bytes per point), for k up to 4096 (the range of
+// the exponent-error table in Section 3), and their validation (Algorithm 2 with the
+// polynomial evaluation replaced by an index look-up).
+//
+// Kernels:
+//   toploc_direct_commit_kernel<dtype, vector>   one 1024-thread block per chunk
+//   toploc_direct_verify_kernel<dtype, vector>   the same selection, then the comparison
+//
+// Selection of a chunk (both kernels): a radix select on the magnitude key with the whole
+// first digit -- 15 bits, i.e. every bf16 key -- histogrammed in shared memory.  The first
+// eighth of the chunk is counted in full; the k-th largest key of that part is a sound lower
+// bound for the chunk's k-th largest key, so the rest of the chunk only counts elements that
+// reach it (few shared-memory atomics).  fp32 keys take two more 8-bit digits over the
+// elements that match the digits found so far.  A last pass in index order takes every key
+// above the k-th largest and the first elements equal to it (ties go to the lower index) and
+// places them, by a block-wide prefix sum, in ascending index order.  The chunk is read from
+// HBM by the first pass; the later passes find it in L2 (one block per SM: 148 chunks in flight).
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "toploc.h"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kTopBits = 15;                 // width of the first digit
+constexpr int kBins = 1 << kTopBits;
+constexpr int kUnroll = 4;                   // 16-byte loads in flight per thread
+constexpr int kMaxChunkElems = 1 << 24;
+
+struct DirectParams {
+  const void* act;
+  long long row_stride;      // elements
+  long long tokens_per_seq;
+  int hidden;
+  int chunk_len;
+  int k;
+  int chunks_per_seq;
+};
+
+struct DirectVerify {
+  const uint8_t* commits;
+  toploc_chunk_result* results;
+  uint32_t* exp_dev;         // optional [num_chunks, 9]
+  int t_exp;
+  int sign_in_exponent;
+  double t_mean;
+  double t_median;
+};
+
+struct DirectShared {
+  uint32_t hist[kBins];
+  unsigned long long warp_sums[2][kWarps];
+  uint32_t picked_bin;
+  uint32_t picked_remaining;
+  uint32_t bad;
+  uint32_t counters[4];      // exponent mismatches, matches, mantissa difference sum, common indices
+  uint32_t dev[9];
+};
+
+// A group is VEC consecutive elements of one row (one 16-byte vector, or one element when
+// the layout does not allow aligned vectors).
+template <int DT, bool VECTOR>
+struct Reader {
+  static constexpr int ESZ = DT == 0 ? 2 : 4;
+  static constexpr int VEC = VECTOR ? 16 / ESZ : 1;
+  const char* base;
+  long long row_stride_bytes;
+  int groups_per_row;
+  int n_groups;
+
+  __device__ __forceinline__ void load(int g, uint32_t (&w)[4]) const {
+    const int row = g / groups_per_row;
+    const int col = g - row * groups_per_row;
+    const char* p = base + row * row_stride_bytes + (long long)col * (VEC * ESZ);
+    if (VECTOR) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+      w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else if (DT == 0) {
+      w[0] = *reinterpret_cast<const uint16_t*>(p);
+    } else {
+      w[0] = *reinterpret_cast<const uint32_t*>(p);
+    }
+  }
+  // whole pattern of element j of a loaded group
+  __device__ __forceinline__ static uint32_t pattern(const uint32_t (&w)[4], int j) {
+    if (DT == 0) return VECTOR ? (w[j >> 1] >> ((j & 1) * 16)) & 0xFFFFu : w[0];
+    return w[VECTOR ? j : 0];
+  }
+  __device__ __forceinline__ static uint32_t key(uint32_t pat) { return DT == 0 ? pat & 0x7FFFu : pat & 0x7FFFFFFFu; }
+  __device__ __forceinline__ static uint32_t committed(uint32_t pat) { return DT == 0 ? pat : pat >> 16; }
+};
+
+__host__ __device__ constexpr int key_bits(int dt) { return dt == 0 ? 15 : 31; }
+
+// Exclusive prefix sum over the block of a 64-bit value (callers pack several small counters
+// into it); *total receives the block's sum.  `slot` alternates between calls so that one
+// barrier per call is enough.
+__device__ __forceinline__ unsigned long long block_scan_exclusive(DirectShared& sh, unsigned long long v, int slot,
+                                                                   unsigned long long* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned long long inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+    if (lane >= d) inc += o;
+  }
+  if (lane == 31) sh.warp_sums[slot][warp] = inc;
+  __syncthreads();
+  unsigned long long mine = sh.warp_sums[slot][lane];  // kWarps == 32: lane w holds warp w's sum
+  unsigned long long winc = mine;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+    if (lane >= d) winc += o;
+  }
+  *total = __shfl_sync(0xFFFFFFFFu, winc, 31);
+  const unsigned long long before_warp = __shfl_sync(0xFFFFFFFFu, winc - mine, warp);
+  return before_warp + inc - v;
+}
+static_assert(kWarps == 32, "the second level of the block scan is one warp wide");
+static_assert((kBins / kThreads & (kBins / kThreads - 1)) == 0, "bins per thread: a power of two");
+
+// The bin, counted from the top, in which the want-th largest counted element lies
+// (1 <= want <= number of counted elements): sh.picked_bin, and sh.picked_remaining = want
+// minus the elements in higher bins.  All threads call; ends with a barrier.
+__device__ __forceinline__ void find_bin_from_top(DirectShared& sh, int nbins, uint32_t want, int slot) {
+  const int per = nbins >= kThreads ? nbins / kThreads : 1;
+  const int top = nbins - 1 - (int)threadIdx.x * per;  // this thread owns bins top, top-1, ..., top-per+1
+  uint32_t s = 0;
+  if (top >= 0)  // each lane starts at another offset: its bins are `per` words apart from its neighbour's
+    for (int b = 0; b < per; ++b) s += sh.hist[top - ((b + (int)threadIdx.x) & (per - 1))];
+  unsigned long long total;
+  const uint32_t before = (uint32_t)block_scan_exclusive(sh, s, slot, &total);
+  if (top >= 0 && before < want && want <= before + s) {
+    uint32_t c = before;
+    for (int b = 0; b < per; ++b) {
+      const uint32_t h = sh.hist[top - b];
+      if (c + h >= want) {
+        sh.picked_bin = (uint32_t)(top - b);
+        sh.picked_remaining = want - c;
+        break;
+      }
+      c += h;
+    }
+  }
+  __syncthreads();
+}
+
+// Counts, over groups [g_begin, g_end), digit (key >> shift) & dmask of every element with
+// (key & mask) == prefix and key >= floor_key.
+template <int DT, bool VECTOR>
+__device__ __forceinline__ void histogram_pass(DirectShared& sh, const Reader<DT, VECTOR>& rd, int g_begin, int g_end,
+                                               uint32_t mask, uint32_t prefix, uint32_t floor_key, int shift,
+                                               uint32_t dmask) {
+  using R = Reader<DT, VECTOR>;
+  for (int g0 = g_begin + (int)threadIdx.x; g0 < g_end; g0 += kUnroll * kThreads) {
+    uint32_t w[kUnroll][4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = g0 + u * kThreads;
+      if (g < g_end) rd.load(g, w[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = g0 + u * kThreads;
+      if (g < g_end) {
+#pragma unroll
+        for (int j = 0; j < R::VEC; ++j) {
+          const uint32_t key = R::key(R::pattern(w[u], j));
+          if ((key & mask) == prefix && key >= floor_key) atomicAdd(&sh.hist[(key >> shift) & dmask], 1u);
+        }
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void clear_bins(DirectShared& sh, int nbins) {  // nbins: a multiple of 4
+  uint4* h = reinterpret_cast<uint4*>(sh.hist);
+  for (int b = threadIdx.x; b < nbins / 4; b += kThreads) h[b] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+}
+
+// The k-th largest key of the chunk (*kth) and how many elements equal to it belong to the
+// top-k (*take >= 1; the k - *take others have larger keys).  Requires k <= elements.
+template <int DT, bool VECTOR>
+__device__ void find_kth_key(DirectShared& sh, const Reader<DT, VECTOR>& rd, int k, uint32_t* kth, uint32_t* take) {
+  using R = Reader<DT, VECTOR>;
+  constexpr int BITS = key_bits(DT);
+  constexpr int SHIFT0 = BITS - kTopBits;
+  clear_bins(sh, kBins);
+  // first part of the chunk in full; its k-th largest bounds the chunk's from below
+  int g_part = rd.n_groups / 8;
+  const int g_need = (2 * k + R::VEC - 1) / R::VEC;
+  if (g_part < g_need) g_part = g_need;
+  if (g_part > rd.n_groups) g_part = rd.n_groups;
+  histogram_pass<DT, VECTOR>(sh, rd, 0, g_part, 0u, 0u, 0u, SHIFT0, kBins - 1);
+  __syncthreads();
+  if (g_part < rd.n_groups) {
+    find_bin_from_top(sh, kBins, (uint32_t)k, 0);
+    const uint32_t floor_key = sh.picked_bin << SHIFT0;
+    histogram_pass<DT, VECTOR>(sh, rd, g_part, rd.n_groups, 0u, 0u, floor_key, SHIFT0, kBins - 1);
+    __syncthreads();
+  }
+  find_bin_from_top(sh, kBins, (uint32_t)k, 1);
+  uint32_t prefix = sh.picked_bin << SHIFT0;
+  uint32_t remaining = sh.picked_remaining;
+  uint32_t mask = (uint32_t)(kBins - 1) << SHIFT0;
+  // fp32: the 16 bits below the first digit, 8 at a time
+  int slot = 0;
+  for (int shift = SHIFT0 - 8; shift >= 0; shift -= 8) {
+    __syncthreads();
+    clear_bins(sh, 256);
+    histogram_pass<DT, VECTOR>(sh, rd, 0, rd.n_groups, mask, prefix, 0u, shift, 255u);
+    __syncthreads();
+    find_bin_from_top(sh, 256, remaining, slot);
+    slot ^= 1;
+    prefix |= sh.picked_bin << shift;
+    remaining = sh.picked_remaining;
+    mask |= 255u << shift;
+  }
+  *kth = prefix;
+  *take = remaining;
+  __syncthreads();
+}
+static_assert((key_bits(1) - kTopBits) % 8 == 0 && key_bits(0) == kTopBits, "digits cover the key exactly");
+
+// Visits the chunk's top-k in ascending index order: emit(position, flat index, pattern).
+template <int DT, bool VECTOR, class Emit>
+__device__ void collect_in_index_order(DirectShared& sh, const Reader<DT, VECTOR>& rd, int k, uint32_t kth,
+                                       uint32_t take, Emit emit) {
+  using R = Reader<DT, VECTOR>;
+  const uint32_t n_above = (uint32_t)k - take;
+  uint32_t base_above = 0, base_equal = 0;
+  int slot = 0;
+  for (int t0 = 0; t0 < rd.n_groups; t0 += kUnroll * kThreads) {
+    uint32_t w[kUnroll][4];
+    unsigned long long above = 0, equal = 0;  // 16 bits per sub-tile
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = t0 + u * kThreads + (int)threadIdx.x;
+      if (g < rd.n_groups) rd.load(g, w[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = t0 + u * kThreads + (int)threadIdx.x;
+      if (g < rd.n_groups) {
+        uint32_t a = 0, e = 0;
+#pragma unroll
+        for (int j = 0; j < R::VEC; ++j) {
+          const uint32_t key = R::key(R::pattern(w[u], j));
+          a += key > kth;
+          e += key == kth;
+        }
+        above |= (unsigned long long)a << (16 * u);
+        equal |= (unsigned long long)e << (16 * u);
+      }
+    }
+    unsigned long long total_above, total_equal;
+    const unsigned long long ex_above = block_scan_exclusive(sh, above, slot, &total_above);
+    const unsigned long long ex_equal = block_scan_exclusive(sh, equal, slot ^ 1, &total_equal);
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = t0 + u * kThreads + (int)threadIdx.x;
+      uint32_t above_before = base_above + (uint32_t)((ex_above >> (16 * u)) & 0xFFFFu);
+      uint32_t equal_before = base_equal + (uint32_t)((ex_equal >> (16 * u)) & 0xFFFFu);
+      if (g < rd.n_groups && (((above | equal) >> (16 * u)) & 0xFFFFu) != 0) {
+#pragma unroll
+        for (int j = 0; j < R::VEC; ++j) {
+          const uint32_t pat = R::pattern(w[u], j);
+          const uint32_t key = R::key(pat);
+          if (key > kth) {
+            emit(above_before + (equal_before < take ? equal_before : take), (uint32_t)g * R::VEC + j, R::committed(pat));
+            ++above_before;
+          } else if (key == kth) {
+            if (equal_before < take) emit(above_before + equal_before, (uint32_t)g * R::VEC + j, R::committed(pat));
+            ++equal_before;
+          }
+        }
+      }
+      base_above += (uint32_t)((total_above >> (16 * u)) & 0xFFFFu);
+      base_equal += (uint32_t)((total_equal >> (16 * u)) & 0xFFFFu);
+    }
+    if (base_above == n_above && base_equal >= take) break;  // the same for every thread
+  }
+}
+
+template <int DT, bool VECTOR>
+__device__ __forceinline__ Reader<DT, VECTOR> locate_chunk(const DirectParams& p, long long chunk) {
+  using R = Reader<DT, VECTOR>;
+  const long long seq = chunk / p.chunks_per_seq;
+  const long long j = chunk - seq * p.chunks_per_seq;
+  const long long row0 = seq * p.tokens_per_seq + j * p.chunk_len;
+  const long long left = p.tokens_per_seq - j * p.chunk_len;
+  const int rows = (int)(left < p.chunk_len ? left : p.chunk_len);
+  R rd;
+  rd.base = static_cast<const char*>(p.act) + row0 * p.row_stride * R::ESZ;
+  rd.row_stride_bytes = p.row_stride * R::ESZ;
+  rd.groups_per_row = p.hidden / R::VEC;
+  rd.n_groups = rows * rd.groups_per_row;
+  return rd;
+}
+
+template <int DT, bool VECTOR>
+__global__ void __launch_bounds__(kThreads, 1)
+toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw);
+  using R = Reader<DT, VECTOR>;
+  const long long chunk = blockIdx.x;
+  const R rd = locate_chunk<DT, VECTOR>(p, chunk);
+  uint16_t* rec = reinterpret_cast<uint16_t*>(commits + (size_t)chunk * 6u * (size_t)p.k);
+  if ((long long)rd.n_groups * R::VEC < p.k) {
+    for (int i = threadIdx.x; i < 3 * p.k; i += kThreads) rec[i] = 0;
+    if (threadIdx.x == 0) status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+    return;
+  }
+  uint32_t kth, take;
+  find_kth_key<DT, VECTOR>(sh, rd, p.k, &kth, &take);
+  collect_in_index_order<DT, VECTOR>(sh, rd, p.k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+    if (pos >= (uint32_t)p.k) return;
+    rec[3 * pos] = (uint16_t)(flat & 0xFFFFu);
+    rec[3 * pos + 1] = (uint16_t)(flat >> 16);
+    rec[3 * pos + 2] = (uint16_t)pat;
+  });
+  if (threadIdx.x == 0) status[chunk] = TOPLOC_CHUNK_OK;
+}
+
+template <int DT, bool VECTOR>
+__global__ void __launch_bounds__(kThreads, 1)
+toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw);
+  uint32_t* sel_idx = reinterpret_cast<uint32_t*>(smem_raw + sizeof(DirectShared));
+  uint32_t* com_idx = sel_idx + p.k;
+  uint16_t* sel_pat = reinterpret_cast<uint16_t*>(com_idx + p.k);
+  uint16_t* com_pat = sel_pat + p.k;
+  using R = Reader<DT, VECTOR>;
+  const long long chunk = blockIdx.x;
+  const int k = p.k;
+  const R rd = locate_chunk<DT, VECTOR>(p, chunk);
+  const uint32_t n_elems = (uint32_t)rd.n_groups * R::VEC;
+
+  // decode the commitment; its indices must ascend strictly and lie inside the chunk
+  const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
+  if (threadIdx.x == 0) sh.bad = 0;
+  if (threadIdx.x < 4) sh.counters[threadIdx.x] = 0;
+  if (threadIdx.x < 9) sh.dev[threadIdx.x] = 0;
+  for (int j = threadIdx.x; j < k; j += kThreads) {
+    com_idx[j] = (uint32_t)rec[3 * j] | ((uint32_t)rec[3 * j + 1] << 16);
+    com_pat[j] = rec[3 * j + 2];
+  }
+  __syncthreads();
+  int status = TOPLOC_CHUNK_OK;
+  if (n_elems < (uint32_t)k) {
+    status = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+  } else {
+    uint32_t bad = 0;
+    for (int j = threadIdx.x; j < k; j += kThreads)
+      bad |= (com_idx[j] >= n_elems) | (j > 0 && com_idx[j] <= com_idx[j - 1]);
+    if (bad) sh.bad = 1;
+    __syncthreads();
+    if (sh.bad) status = TOPLOC_CHUNK_BAD_PROOF;
+  }
+  if (status != TOPLOC_CHUNK_OK) {
+    if (threadIdx.x == 0) {
+      toploc_chunk_result r = {};
+      r.topk_mismatch = -1;
+      r.status = (uint8_t)status;
+      io.results[chunk] = r;
+    }
+    if (io.exp_dev != nullptr && threadIdx.x < 9) io.exp_dev[(size_t)chunk * 9 + threadIdx.x] = 0;
+    return;
+  }
+
+  uint32_t kth, take;
+  find_kth_key<DT, VECTOR>(sh, rd, k, &kth, &take);
+  collect_in_index_order<DT, VECTOR>(sh, rd, k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+    if (pos >= (uint32_t)k) return;
+    sel_idx[pos] = flat;
+    sel_pat[pos] = (uint16_t)pat;
+  });
+  __syncthreads();
+  for (int b = threadIdx.x; b < 128; b += kThreads) sh.hist[b] = 0;  // mantissa differences 0..127
+  __syncthreads();
+
+  // Algorithm 2 with a look-up in place of the polynomial
+  uint32_t err_e = 0, n_match = 0, sum = 0, common = 0, dev[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  for (int j = threadIdx.x; j < k; j += kThreads) {
+    const uint32_t want = sel_idx[j];
+    int lo = 0, hi = k;  // first committed index >= want
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (com_idx[mid] < want) lo = mid + 1; else hi = mid;
+    }
+    if (lo == k || com_idx[lo] != want) {
+      ++err_e;  // nothing was committed for this index
+      continue;
+    }
+    ++common;
+    const uint32_t committed = com_pat[lo], seen = sel_pat[j];
+    const uint32_t field = io.sign_in_exponent ? 0x1FFu : 0xFFu;
+    if (((committed >> 7) & field) == ((seen >> 7) & field)) {
+      const uint32_t mp = committed & 0x7Fu, mv = seen & 0x7Fu;
+      const uint32_t d = mp > mv ? mp - mv : mv - mp;
+      ++n_match;
+      sum += d;
+      atomicAdd(&sh.hist[d], 1u);
+    } else {
+      ++err_e;
+    }
+    const int d = (int)((seen >> 7) & 0xFFu) - (int)((committed >> 7) & 0xFFu);
+    const int a = d < 0 ? -d : d;
+    const int bin = d == 0 ? 0 : a == 1 ? (d < 0 ? 1 : 2) : a == 2 ? (d < 0 ? 3 : 4) : a <= 10 ? (d < 0 ? 5 : 6) : a <= 99 ? 7 : 8;
+#pragma unroll
+    for (int b = 0; b < 9; ++b) dev[b] += bin == b;
+  }
+  err_e = __reduce_add_sync(0xFFFFFFFFu, err_e);
+  n_match = __reduce_add_sync(0xFFFFFFFFu, n_match);
+  sum = __reduce_add_sync(0xFFFFFFFFu, sum);
+  common = __reduce_add_sync(0xFFFFFFFFu, common);
+#pragma unroll
+  for (int b = 0; b < 9; ++b) dev[b] = __reduce_add_sync(0xFFFFFFFFu, dev[b]);
+  if ((threadIdx.x & 31) == 0) {
+    atomicAdd(&sh.counters[0], err_e);
+    atomicAdd(&sh.counters[1], n_match);
+    atomicAdd(&sh.counters[2], sum);
+    atomicAdd(&sh.counters[3], common);
+#pragma unroll
+    for (int b = 0; b < 9; ++b)
+      if (dev[b]) atomicAdd(&sh.dev[b], dev[b]);
+  }
+  __syncthreads();
+  if (io.exp_dev != nullptr && threadIdx.x < 9) io.exp_dev[(size_t)chunk * 9 + threadIdx.x] = sh.dev[threadIdx.x];
+  if (threadIdx.x == 0) {
+    toploc_chunk_result r = {};
+    r.exp_mismatch = sh.counters[0];
+    r.n_match = sh.counters[1];
+    r.mant_diff_sum = sh.counters[2];
+    r.topk_mismatch = k - (int)sh.counters[3];
+    bool reject = r.exp_mismatch > (uint32_t)io.t_exp;
+    if (r.n_match > 0) {
+      r.mant_mean = (double)r.mant_diff_sum / (double)r.n_match;
+      // values at sorted positions (n - 1) / 2 and n / 2
+      const uint32_t lo_rank = (r.n_match - 1) / 2, hi_rank = r.n_match / 2;
+      uint32_t seen = 0;
+      int lo_val = -1, hi_val = -1;
+      for (int b = 0; b < 128 && hi_val < 0; ++b) {
+        seen += sh.hist[b];
+        if (lo_val < 0 && seen > lo_rank) lo_val = b;
+        if (seen > hi_rank) hi_val = b;
+      }
+      r.mant_median = ((double)lo_val + (double)hi_val) / 2.0;
+      reject = reject || r.mant_mean > io.t_mean || r.mant_median > io.t_median;
+    } else {
+      reject = true;  // nothing matched: no statistic to accept on
+    }
+    r.accept = reject ? 0 : 1;
+    r.status = TOPLOC_CHUNK_OK;
+    io.results[chunk] = r;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+
+struct DirectPlan {
+  DirectParams params;
+  long long num_chunks;
+  bool vector;
+};
+
+int plan_direct(const void* d_act, const toploc_layout* lay, DirectPlan* plan) {
+  if (lay == nullptr || d_act == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->dtype != TOPLOC_DTYPE_BF16 && lay->dtype != TOPLOC_DTYPE_FP32) return TOPLOC_ERR_UNSUPPORTED;
+  if (lay->hidden <= 0 || lay->chunk_len <= 0 || lay->num_seqs <= 0 || lay->tokens_per_seq <= 0 || lay->k < 1 ||
+      lay->row_stride < lay->hidden)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (lay->field != TOPLOC_FIELD_16 || lay->seq_offsets != nullptr || lay->k > TOPLOC_MAX_K_DIRECT)
+    return TOPLOC_ERR_UNSUPPORTED;
+  const long long rows = lay->tokens_per_seq < lay->chunk_len ? lay->tokens_per_seq : lay->chunk_len;
+  if (rows * lay->hidden > kMaxChunkElems) return TOPLOC_ERR_UNSUPPORTED;
+  const long long cps = (lay->tokens_per_seq + lay->chunk_len - 1) / lay->chunk_len;
+  const long long n = cps * lay->num_seqs;
+  if (cps > 0x7FFFFFFFll || n > 0x7FFFFFFFll) return TOPLOC_ERR_UNSUPPORTED;
+  const int esz = lay->dtype == TOPLOC_DTYPE_BF16 ? 2 : 4;
+  const int vec = 16 / esz;
+  plan->vector = lay->hidden % vec == 0 && lay->row_stride % vec == 0 && (reinterpret_cast<uintptr_t>(d_act) & 15u) == 0;
+  if (!plan->vector && (reinterpret_cast<uintptr_t>(d_act) & (uintptr_t)(esz - 1)) != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  plan->params.act = d_act;
+  plan->params.row_stride = lay->row_stride;
+  plan->params.tokens_per_seq = lay->tokens_per_seq;
+  plan->params.hidden = lay->hidden;
+  plan->params.chunk_len = lay->chunk_len;
+  plan->params.k = lay->k;
+  plan->params.chunks_per_seq = (int)cps;
+  plan->num_chunks = n;
+  return TOPLOC_OK;
+}
+
+int check_device() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TOPLOC_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TOPLOC_ERR_CUDA;
+  return major == 10 ? TOPLOC_OK : TOPLOC_ERR_ARCH;
+}
+
+template <class Kernel, class... Args>
+int launch_direct(Kernel kernel, long long num_chunks, size_t smem, cudaStream_t stream, Args... args) {
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return TOPLOC_ERR_CUDA;
+  }
+  kernel<<<(unsigned)num_chunks, kThreads, smem, stream>>>(args...);
+  return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t toploc_direct_commit_bytes(int32_t k) { return k > 0 ? 6 * (size_t)k : 0; }
+
+int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d_commits, uint8_t* d_status,
+                         void* cuda_stream) {
+  DirectPlan plan;
+  int rc = plan_direct(d_act, lay, &plan);
+  if (rc != TOPLOC_OK) return rc;
+  if (d_commits == nullptr || d_status == nullptr || (reinterpret_cast<uintptr_t>(d_commits) & 1u) != 0)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if ((rc = check_device()) != TOPLOC_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t smem = sizeof(DirectShared);
+  const DirectParams& p = plan.params;
+  if (lay->dtype == TOPLOC_DTYPE_BF16)
+    return plan.vector ? launch_direct(toploc_direct_commit_kernel<0, true>, plan.num_chunks, smem, stream, p, d_commits, d_status)
+                       : launch_direct(toploc_direct_commit_kernel<0, false>, plan.num_chunks, smem, stream, p, d_commits, d_status);
+  return plan.vector ? launch_direct(toploc_direct_commit_kernel<1, true>, plan.num_chunks, smem, stream, p, d_commits, d_status)
+                     : launch_direct(toploc_direct_commit_kernel<1, false>, plan.num_chunks, smem, stream, p, d_commits, d_status);
+}
+
+int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
+                         const toploc_thresholds* thr, toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt,
+                         void* cuda_stream) {
+  DirectPlan plan;
+  int rc = plan_direct(d_act, lay, &plan);
+  if (rc != TOPLOC_OK) return rc;
+  if (d_commits == nullptr || thr == nullptr || d_results == nullptr ||
+      (reinterpret_cast<uintptr_t>(d_commits) & 1u) != 0 || (reinterpret_cast<uintptr_t>(d_results) & 7u) != 0 ||
+      (reinterpret_cast<uintptr_t>(d_exp_dev_opt) & 3u) != 0)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  if ((rc = check_device()) != TOPLOC_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  DirectVerify io;
+  io.commits = d_commits;
+  io.results = d_results;
+  io.exp_dev = d_exp_dev_opt;
+  io.t_exp = thr->t_exp;
+  io.sign_in_exponent = thr->sign_in_exponent;
+  io.t_mean = thr->t_mean;
+  io.t_median = thr->t_median;
+  const size_t smem = sizeof(DirectShared) + 12 * (size_t)lay->k;
+  const DirectParams& p = plan.params;
+  if (lay->dtype == TOPLOC_DTYPE_BF16)
+    return plan.vector ? launch_direct(toploc_direct_verify_kernel<0, true>, plan.num_chunks, smem, stream, p, io)
+                       : launch_direct(toploc_direct_verify_kernel<0, false>, plan.num_chunks, smem, stream, p, io);
+  return plan.vector ? launch_direct(toploc_direct_verify_kernel<1, true>, plan.num_chunks, smem, stream, p, io)
+                     : launch_direct(toploc_direct_verify_kernel<1, false>, plan.num_chunks, smem, stream, p, io);
+}
+
+}  // extern "C"

@@ -1,0 +1,150 @@
+"""GPU parity of the direct commitments (index and value stored as they are, Section 4) with
+the oracle: commitment bytes, statuses, every integer statistic and the exponent-deviation
+counts are compared for equality, fp64 mean / median within 1e-9."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2501_16007_b200 as tl
+from paper_2501_16007_b200 import synth
+
+from helpers import assert_results_equal, oracle_thresholds
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def host_of(act):
+    return synth.host_patterns(act) if act.is_contiguous() else synth.host_patterns(act._base)[:, :act.shape[1]]
+
+
+def direct_case(act, chunk_len, k, num_seqs, tokens_per_seq, recomputed=None, where=""):
+    lay, _ = tl.make_layout(act, chunk_len, k, num_seqs, tokens_per_seq)
+    commits, status = tl.toploc_commit_direct(act, lay)
+    torch.cuda.synchronize()
+    ref_commits, ref_status = oracle.commit_direct(host_of(act), chunk_len, k, num_seqs, tokens_per_seq)
+    assert np.array_equal(status.cpu().numpy(), ref_status), where + " status"
+    bad = np.nonzero((commits.cpu().numpy() != ref_commits).any(axis=1))[0]
+    assert bad.size == 0, "%s commitment bytes differ at chunks %s" % (where, bad[:8])
+    cases = {"same": act}
+    cases.update(recomputed or {})
+    out = {}
+    for name, rec in cases.items():
+        res, dev = tl.toploc_verify_direct(rec, lay, commits, tl.default_thresholds(k))
+        torch.cuda.synchronize()
+        got = res.cpu().numpy().view(tl.RESULT_DTYPE).reshape(-1)
+        ref, ref_dev = oracle.verify_direct(host_of(rec), ref_commits, chunk_len, k, num_seqs, tokens_per_seq,
+                                            **oracle_thresholds(k))
+        assert_results_equal(got, ref, "%s verify[%s]" % (where, name))
+        assert np.array_equal(dev.cpu().numpy().astype(np.uint32), ref_dev), "%s deviation bins [%s]" % (where, name)
+        out[name] = ref
+    return out
+
+
+@pytest.mark.parametrize("k", [1, 128, 1000, 4096])
+@pytest.mark.parametrize("outliers", ["fixed", "none"])
+def test_bf16_chunks(k, outliers):
+    S, T, H, L = 3, 96, 4096, 32
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=40 + k, device=DEV, outliers=outliers)
+    rec = {"noise": synth.honest_noise(act, seed=7), "ulp": synth.plus_one_ulp(act, seed=8),
+           "other": synth.make_activations(S, T, H, torch.bfloat16, seed=900 + k, device=DEV, outliers=outliers)}
+    out = direct_case(act, L, k, S, T, rec, "bf16 k=%d %s" % (k, outliers))
+    assert (out["same"]["accept"] == 1).all() and (out["same"]["exp_mismatch"] == 0).all()
+    if outliers == "none" and k >= 128:
+        assert (out["other"]["accept"] == 0).all()
+
+
+@pytest.mark.parametrize("k", [64, 2048])
+def test_fp32_chunks(k):
+    S, T, H, L = 2, 64, 2048, 32
+    act = synth.make_activations(S, T, H, torch.float32, seed=50 + k, device=DEV, outliers="jitter")
+    rec = {"noise": synth.honest_noise(act, seed=9, rel=2.0 ** -10)}
+    direct_case(act, L, k, S, T, rec, "fp32 k=%d" % k)
+
+
+def test_70b_shaped_chunks_and_ragged_tail():
+    # 8192-wide rows, 100 tokens per sequence: three chunks of 32 rows and one of 4
+    S, T, H, L, k = 2, 100, 8192, 32, 4096
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=61, device=DEV)
+    direct_case(act, L, k, S, T, {"noise": synth.honest_noise(act, seed=3)}, "70B-shaped")
+
+
+def test_ties_decide_the_selection():
+    # all equal; two values only; ascending magnitudes
+    H, L = 1024, 16
+    same = torch.full((L, H), 1.5, dtype=torch.bfloat16, device=DEV)
+    direct_case(same, L, 300, 1, L, None, "all equal")
+    two = torch.where(torch.arange(L * H, device=DEV).reshape(L, H) % 3 == 0, 2.0, -2.0).to(torch.bfloat16)
+    direct_case(two, L, 777, 1, L, None, "two signs")
+    asc = (torch.arange(L * H, device=DEV, dtype=torch.float32).reshape(L, H) / 64).to(torch.bfloat16)
+    direct_case(asc, L, 512, 1, L, None, "ascending")
+
+
+def test_special_patterns():
+    H, L, k = 512, 8, 200
+    bits = torch.randint(0, 65536, (L, H), dtype=torch.int32, device=DEV).to(torch.int16)  # NaN, Inf, subnormals
+    act = bits.view(torch.bfloat16)
+    direct_case(act, L, k, 1, L, None, "random patterns")
+
+
+def test_odd_shapes_take_the_scalar_path():
+    # hidden not a multiple of the vector width, and a strided view
+    S, T, H, L, k = 2, 24, 1003, 8, 333
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=71, device=DEV, outliers="none")
+    direct_case(act, L, k, S, T, None, "H=1003")
+    wide = synth.make_activations(S, T, 1024 + 64, torch.bfloat16, seed=72, device=DEV, outliers="none")
+    view = wide[:, :1024]
+    direct_case(view, L, k, S, T, None, "strided rows")
+    f = synth.make_activations(S, T, 1001, torch.float32, seed=73, device=DEV, outliers="none")
+    direct_case(f, L, 100, S, T, None, "fp32 H=1001")
+
+
+def test_chunk_smaller_than_k_and_malformed_commitments():
+    S, T, H, L, k = 1, 10, 64, 4, 200      # chunks of 256, 256 and 128 elements
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=81, device=DEV, outliers="none")
+    out = direct_case(act, L, k, S, T, None, "short last chunk")
+    assert out["same"]["status"].tolist() == [0, 0, 2]   # the last one: TOPLOC_CHUNK_K_EXCEEDS_CHUNK
+    lay, _ = tl.make_layout(act, L, k, S, T)
+    commits, _ = tl.toploc_commit_direct(act, lay)
+    host = commits.cpu().numpy().copy()
+    host[0, 6:12], host[0, 12:18] = host[0, 12:18].copy(), host[0, 6:12].copy()   # two records swapped
+    host[1, 6 * (k - 1) + 2] = 0xFF                                                  # an index beyond the chunk
+    bad = torch.from_numpy(host).to(DEV)
+    res, dev = tl.toploc_verify_direct(act, lay, bad)
+    torch.cuda.synchronize()
+    got = res.cpu().numpy().view(tl.RESULT_DTYPE).reshape(-1)
+    ref, ref_dev = oracle.verify_direct(synth.host_patterns(act), host, L, k, S, T, **oracle_thresholds(k))
+    assert ref["status"].tolist() == [3, 3, 2]
+    assert_results_equal(got, ref, "malformed")
+    assert np.array_equal(dev.cpu().numpy().astype(np.uint32), ref_dev)
+
+
+def test_argument_errors_come_back_before_any_launch():
+    act = torch.zeros((64, 256), dtype=torch.bfloat16, device=DEV)
+    lay, _ = tl.make_layout(act, 32, tl.TOPLOC_MAX_K_DIRECT + 1, 1, 64)
+    with pytest.raises(tl.ToplocError, match="unsupported"):
+        tl.toploc_commit_direct(act, lay)
+    offs = np.array([0, 64], np.int64)
+    lay, keep = tl.make_layout(act, 32, 16, 1, 0, seq_offsets=offs)
+    lay.tokens_per_seq = 64
+    with pytest.raises(tl.ToplocError, match="unsupported"):
+        tl.toploc_commit_direct(act, lay)
+    lay, _ = tl.make_layout(act, 32, 16, 1, 64)
+    lib = tl.load_library()
+    assert lib.toploc_commit_direct(None, ctypes.byref(lay), None, None, None) == -1
+
+
+def test_agrees_with_the_proof_path_selection():
+    """Same top-k as toploc_build_proofs (its optional index output, as a set)."""
+    S, T, H, L, k = 4, 64, 4096, 32, 256
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=91, device=DEV, outliers="jitter")
+    lay, _ = tl.make_layout(act, L, k, S, T)
+    _, _, indices = tl.toploc_build_proofs(act, lay, want_indices=True)
+    commits, _ = tl.toploc_commit_direct(act, lay)
+    torch.cuda.synchronize()
+    rec = commits.cpu().numpy().reshape(-1, k, 6).astype(np.int64)
+    idx = rec[..., 0] | (rec[..., 1] << 8) | (rec[..., 2] << 16) | (rec[..., 3] << 24)
+    assert np.array_equal(idx, np.sort(indices.cpu().numpy().astype(np.int64), axis=1))
