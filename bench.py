@@ -11,6 +11,9 @@ Rank 0 prints one JSON line.  `value` counts chunks generated-and-validated per 
 the activations resident in HBM; `e2e` is the same through the host-buffer entry points
 (pinned host memory, copies inside the timed region).  With N > 1 (torchrun) every rank
 processes its own full batch: weak scaling, no collective on the data path.
+
+Other modes (each prints its own JSON line): --decode-steps (incremental generation), --sweep
+(k x chunk length x H x dtype), --direct (direct commitments, k = 128 .. 4096).
 """
 import argparse
 import json
@@ -188,6 +191,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-steps", action="store_true",
                     help="time incremental proof generation (one row per sequence and step) instead of the main workload")
+    ap.add_argument("--direct", action="store_true",
+                    help="time direct commitments (index and value stored as they are) for k = 128 .. 4096 "
+                         "instead of the main workload")
     ap.add_argument("--sweep", action="store_true",
                     help="time the parameter sweep (k x chunk length x H x dtype) instead of the main workload")
     args = ap.parse_args()
@@ -213,6 +219,10 @@ def main():
     if args.decode_steps:
         if rank == 0:
             print(json.dumps(decode_steps(tl, synth, dev)), flush=True)
+        return
+    if args.direct:
+        if rank == 0:
+            print(json.dumps(direct_commitments(tl, synth, dev, args.workload)), flush=True)
         return
     if args.sweep:
         if rank == 0:
@@ -399,6 +409,49 @@ def decode_steps(tl, synth, dev, reps=20):
             "us_per_append": (whole - finish) / L * 1e3, "us_finish": finish * 1e3, "us_per_interval": whole * 1e3,
             "us_batch_build_of_the_same_chunks": b0.elapsed_time(b1) / reps * 1e3,
             "bytes_per_append": S * H * 2, "identical_to_batch": bool(torch.equal(proofs, ref_proofs))}
+
+
+def direct_commitments(tl, synth, dev, workload, reps=10):
+    """toploc_commit_direct / toploc_verify_direct over the workload's batch for k = 128 .. 4096:
+    CUDA-event time per call, activation GB/s (the batch's bytes, once) and its fraction of the
+    measured copy peak."""
+    S, T, H, L, _, seed = WORKLOADS[workload]
+    dtype = torch.float32 if workload in WIDE_WORKLOADS else torch.bfloat16
+    act = synth.make_activations(S, T, H, dtype, seed=seed, device=dev)
+    rec = synth.honest_noise(act, seed=seed + 100)
+    peak, peak_kind = measured_hbm_peak()
+    nbytes = act.numel() * act.element_size()
+    points = []
+    for k in (128, 512, 1024, 4096):
+        lay, _ = tl.make_layout(act, L, k, S, T)
+        commits, status = tl.toploc_commit_direct(act, lay)
+        results, dev_bins = tl.toploc_verify_direct(rec, lay, commits)
+        thr = tl.default_thresholds(k)
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        t_commit = timed(lambda: tl.toploc_commit_direct(act, lay, commits, status))
+        t_verify = timed(lambda: tl.toploc_verify_direct(rec, lay, commits, thr, results, dev_bins))
+        got = results.cpu().numpy().view(tl.RESULT_DTYPE).reshape(-1)
+        points.append({"k": k, "commit_bytes": 6 * k, "commit_ms": t_commit, "verify_ms": t_verify,
+                       "commit_GB_per_s": nbytes / t_commit / 1e6, "verify_GB_per_s": nbytes / t_verify / 1e6,
+                       "commit_frac_of_peak": nbytes / t_commit / 1e6 / peak,
+                       "verify_frac_of_peak": nbytes / t_verify / 1e6 / peak,
+                       "accepted": int(got["accept"].sum()), "chunks": int(got.size),
+                       "mean_topk_mismatch": float(got["topk_mismatch"].mean())})
+    return {"metric": "direct_commitments", "workload": workload_name(workload), "activation_bytes": nbytes,
+            "peak_GB_per_s": peak, "peak_kind": peak_kind, "recomputed": "honest reorder noise, relative 2^-8",
+            "points": points}
 
 
 def sweep(tl, synth, dev, reps=5):

@@ -8,8 +8,8 @@
 //   toploc_direct_verify_kernel<dtype, vector>   the same selection, then the comparison
 //
 // Selection of a chunk (both kernels): a radix select on the magnitude key with the whole
-// first digit -- 15 bits, i.e. every bf16 key -- histogrammed in shared memory.  The first
-// eighth of the chunk is counted in full; the k-th largest key of that part is a sound lower
+// first digit -- 15 bits, i.e. every bf16 key -- histogrammed in shared memory.  A first part
+// of the chunk is counted in full; the k-th largest key of that part is a sound lower
 // bound for the chunk's k-th largest key, so the rest of the chunk only counts elements that
 // reach it (few shared-memory atomics).  fp32 keys take two more 8-bit digits over the
 // elements that match the digits found so far.  A last pass in index order takes every key
@@ -29,6 +29,8 @@ constexpr int kTopBits = 15;                 // width of the first digit
 constexpr int kBins = 1 << kTopBits;
 constexpr int kUnroll = 4;                   // 16-byte loads in flight per thread
 constexpr int kMaxChunkElems = 1 << 24;
+constexpr int kListOffset = 256;             // verify: words of the histogram kept for the mantissa differences
+constexpr size_t kRingBytes = (size_t)kUnroll * kThreads * 16;
 
 struct DirectParams {
   const void* act;
@@ -70,24 +72,99 @@ struct Reader {
   long long row_stride_bytes;
   int groups_per_row;
   int n_groups;
+  bool flat;
 
-  __device__ __forceinline__ void load(int g, uint32_t (&w)[4]) const {
+  __device__ __forceinline__ const char* address(int g) const {
+    if (flat) return base + (long long)g * (VEC * ESZ);  // rows follow one another without a gap
     const int row = g / groups_per_row;
     const int col = g - row * groups_per_row;
-    const char* p = base + row * row_stride_bytes + (long long)col * (VEC * ESZ);
-    if (VECTOR) {
-      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
-      w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-    } else if (DT == 0) {
-      w[0] = *reinterpret_cast<const uint16_t*>(p);
-    } else {
-      w[0] = *reinterpret_cast<const uint32_t*>(p);
+    return base + row * row_stride_bytes + (long long)col * (VEC * ESZ);
+  }
+
+  // A batch is this thread's groups first + u * kThreads, u < kUnroll, below g_end.  Vector
+  // layouts move a batch through the thread's own kUnroll 16-byte slots of the ring in shared
+  // memory with asynchronous copies: request() starts the copies, take() waits for them and
+  // moves the slots to registers, after which the next batch may be requested -- so a batch is
+  // in flight while the previous one is worked on, barriers included.  Nothing waits on
+  // another thread.  Other layouts load directly in take().
+  __device__ __forceinline__ void request(uint4* ring, int first, int g_end) const {
+    if constexpr (VECTOR) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int g = first + u * kThreads;
+        if (g < g_end) {
+          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(ring + u * kThreads + threadIdx.x);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(address(g)) : "memory");
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
   }
-  // whole pattern of element j of a loaded group
-  __device__ __forceinline__ static uint32_t pattern(const uint32_t (&w)[4], int j) {
-    if (DT == 0) return VECTOR ? (w[j >> 1] >> ((j & 1) * 16)) & 0xFFFFu : w[0];
-    return w[VECTOR ? j : 0];
+  // The same, for the batch after one whose registers are w: each copy's destination is made
+  // to depend on the register that was read from it, so the copy cannot overtake the read.
+  __device__ __forceinline__ void request_after(uint4* ring, int first, int g_end, const uint32_t (&w)[kUnroll][4],
+                                                int prev_first, int prev_end) const {
+    if constexpr (VECTOR) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int g = first + u * kThreads;
+        if (g < g_end) {
+          uint32_t dst = (uint32_t)__cvta_generic_to_shared(ring + u * kThreads + threadIdx.x);
+          if (prev_first + u * kThreads < prev_end) {
+            uint32_t zero;
+            asm volatile("and.b32 %0, %1, 0;" : "=r"(zero) : "r"(w[u][3]));
+            dst += zero;
+          }
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(address(g)) : "memory");
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+  }
+  __device__ __forceinline__ void take(const uint4* ring, int first, int g_end, uint32_t (&w)[kUnroll][4]) const {
+    if (VECTOR) asm volatile("cp.async.wait_group 0;" ::: "memory");
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = first + u * kThreads;
+      if (g < g_end) {
+        if (VECTOR) {
+          const uint4 v = ring[u * kThreads + threadIdx.x];
+          w[u][0] = v.x; w[u][1] = v.y; w[u][2] = v.z; w[u][3] = v.w;
+        } else if (DT == 0) {
+          w[u][0] = *reinterpret_cast<const uint16_t*>(address(g));
+        } else {
+          w[u][0] = *reinterpret_cast<const uint32_t*>(address(g));
+        }
+      }
+    }
+  }
+  // whole pattern of element j of a loaded group, j known at run time (no indexed registers)
+  __device__ __forceinline__ static uint32_t pattern_at(const uint32_t (&w)[4], uint32_t j) {
+    if (!VECTOR) return w[0];
+    if (DT == 0) {
+      const uint32_t lo = (j & 2u) ? w[1] : w[0], hi = (j & 2u) ? w[3] : w[2];
+      const uint32_t word = (j & 4u) ? hi : lo;
+      return (j & 1u) ? word >> 16 : word & 0xFFFFu;
+    }
+    const uint32_t lo = (j & 1u) ? w[1] : w[0], hi = (j & 1u) ? w[3] : w[2];
+    return (j & 2u) ? hi : lo;
+  }
+  // Bit j is set iff the key of element j is >= thr; thr may be one past the largest key
+  // (no bit set).  bf16 vectors: per word, (keys + (2^15 - thr)) carries into bits 15 and 31
+  // exactly for the keys that reach thr (keys have 15 bits, so nothing crosses the halves).
+  __device__ __forceinline__ static uint32_t reach_mask(const uint32_t (&w)[4], uint32_t thr) {
+    if (!VECTOR) return key(w[0]) >= thr ? 1u : 0u;
+    if (DT == 0) {
+      const uint32_t add = (0x8000u - thr) * 0x00010001u;
+      const uint32_t m0 = ((w[0] & 0x7FFF7FFFu) + add) & 0x80008000u;
+      const uint32_t m1 = ((w[1] & 0x7FFF7FFFu) + add) & 0x80008000u;
+      const uint32_t m2 = ((w[2] & 0x7FFF7FFFu) + add) & 0x80008000u;
+      const uint32_t m3 = ((w[3] & 0x7FFF7FFFu) + add) & 0x80008000u;
+      const uint32_t m = (m0 >> 15) | (m1 >> 13) | (m2 >> 11) | (m3 >> 9);  // even elements at bits 0..6, odd at 16..22
+      return (m | (m >> 15)) & 0xFFu;
+    }
+    return ((w[0] & 0x7FFFFFFFu) >= thr ? 1u : 0u) | ((w[1] & 0x7FFFFFFFu) >= thr ? 2u : 0u) |
+           ((w[2] & 0x7FFFFFFFu) >= thr ? 4u : 0u) | ((w[3] & 0x7FFFFFFFu) >= thr ? 8u : 0u);
   }
   __device__ __forceinline__ static uint32_t key(uint32_t pat) { return DT == 0 ? pat & 0x7FFFu : pat & 0x7FFFFFFFu; }
   __device__ __forceinline__ static uint32_t committed(uint32_t pat) { return DT == 0 ? pat : pat >> 16; }
@@ -121,6 +198,8 @@ __device__ __forceinline__ unsigned long long block_scan_exclusive(DirectShared&
   return before_warp + inc - v;
 }
 static_assert(kWarps == 32, "the second level of the block scan is one warp wide");
+static_assert(kListOffset * 4 + 12 * TOPLOC_MAX_K_DIRECT <= kBins * 4, "the verify lists fit where the histogram was");
+static_assert(sizeof(DirectShared) % 16 == 0 && sizeof(DirectShared) + kRingBytes <= 227 * 1024, "shared memory budget");
 static_assert((kBins / kThreads & (kBins / kThreads - 1)) == 0, "bins per thread: a power of two");
 
 // The bin, counted from the top, in which the want-th largest counted element lies
@@ -150,27 +229,29 @@ __device__ __forceinline__ void find_bin_from_top(DirectShared& sh, int nbins, u
 }
 
 // Counts, over groups [g_begin, g_end), digit (key >> shift) & dmask of every element with
-// (key & mask) == prefix and key >= floor_key.
+// lo_key <= key < hi_key.  A group is tested as a whole; only the elements that pass are
+// looked at one by one.
 template <int DT, bool VECTOR>
-__device__ __forceinline__ void histogram_pass(DirectShared& sh, const Reader<DT, VECTOR>& rd, int g_begin, int g_end,
-                                               uint32_t mask, uint32_t prefix, uint32_t floor_key, int shift,
-                                               uint32_t dmask) {
+__device__ __forceinline__ void histogram_pass(DirectShared& sh, uint4* ring, const Reader<DT, VECTOR>& rd, int g_begin, int g_end,
+                                               uint32_t lo_key, uint32_t hi_key, int shift, uint32_t dmask) {
   using R = Reader<DT, VECTOR>;
-  for (int g0 = g_begin + (int)threadIdx.x; g0 < g_end; g0 += kUnroll * kThreads) {
+  constexpr uint32_t kLargestKey = DT == 0 ? 0x7FFFu : 0x7FFFFFFFu;
+  rd.request(ring, g_begin + (int)threadIdx.x, g_end);
+  for (int base = g_begin; base < g_end; base += kUnroll * kThreads) {
+    const int g0 = base + (int)threadIdx.x;
     uint32_t w[kUnroll][4];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int g = g0 + u * kThreads;
-      if (g < g_end) rd.load(g, w[u]);
-    }
+    rd.take(ring, g0, g_end, w);
+    if (base + kUnroll * kThreads < g_end) rd.request_after(ring, g0 + kUnroll * kThreads, g_end, w, g0, g_end);
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int g = g0 + u * kThreads;
       if (g < g_end) {
-#pragma unroll
-        for (int j = 0; j < R::VEC; ++j) {
-          const uint32_t key = R::key(R::pattern(w[u], j));
-          if ((key & mask) == prefix && key >= floor_key) atomicAdd(&sh.hist[(key >> shift) & dmask], 1u);
+        uint32_t m = R::reach_mask(w[u], lo_key);
+        if (hi_key <= kLargestKey) m &= ~R::reach_mask(w[u], hi_key);
+        while (m) {
+          const uint32_t j = (uint32_t)__ffs((int)m) - 1u;
+          m &= m - 1u;
+          atomicAdd(&sh.hist[(R::key(R::pattern_at(w[u], j)) >> shift) & dmask], 1u);
         }
       }
     }
@@ -186,40 +267,42 @@ __device__ __forceinline__ void clear_bins(DirectShared& sh, int nbins) {  // nb
 // The k-th largest key of the chunk (*kth) and how many elements equal to it belong to the
 // top-k (*take >= 1; the k - *take others have larger keys).  Requires k <= elements.
 template <int DT, bool VECTOR>
-__device__ void find_kth_key(DirectShared& sh, const Reader<DT, VECTOR>& rd, int k, uint32_t* kth, uint32_t* take) {
+__device__ void find_kth_key(DirectShared& sh, uint4* ring, const Reader<DT, VECTOR>& rd, int k, uint32_t* kth,
+                             uint32_t* take) {
   using R = Reader<DT, VECTOR>;
   constexpr int BITS = key_bits(DT);
   constexpr int SHIFT0 = BITS - kTopBits;
   clear_bins(sh, kBins);
-  // first part of the chunk in full; its k-th largest bounds the chunk's from below
-  int g_part = rd.n_groups / 8;
-  const int g_need = (2 * k + R::VEC - 1) / R::VEC;
-  if (g_part < g_need) g_part = g_need;
+  // First part of the chunk in full; its k-th largest bounds the chunk's from below.  A part of
+  // a elements costs a atomics and lets about (n - a) k / a of the others through, least for
+  // a = sqrt(n k): the smallest power-of-two multiple of 2k elements that reaches it.
+  int g_part = (2 * k + R::VEC - 1) / R::VEC;
+  while ((long long)g_part * g_part * R::VEC < (long long)rd.n_groups * k) g_part *= 2;
   if (g_part > rd.n_groups) g_part = rd.n_groups;
-  histogram_pass<DT, VECTOR>(sh, rd, 0, g_part, 0u, 0u, 0u, SHIFT0, kBins - 1);
+  constexpr uint32_t kPastLargest = DT == 0 ? 0x8000u : 0x80000000u;
+  histogram_pass<DT, VECTOR>(sh, ring, rd, 0, g_part, 0u, kPastLargest, SHIFT0, kBins - 1);
   __syncthreads();
   if (g_part < rd.n_groups) {
     find_bin_from_top(sh, kBins, (uint32_t)k, 0);
     const uint32_t floor_key = sh.picked_bin << SHIFT0;
-    histogram_pass<DT, VECTOR>(sh, rd, g_part, rd.n_groups, 0u, 0u, floor_key, SHIFT0, kBins - 1);
+    histogram_pass<DT, VECTOR>(sh, ring, rd, g_part, rd.n_groups, floor_key, kPastLargest, SHIFT0, kBins - 1);
     __syncthreads();
   }
   find_bin_from_top(sh, kBins, (uint32_t)k, 1);
   uint32_t prefix = sh.picked_bin << SHIFT0;
   uint32_t remaining = sh.picked_remaining;
-  uint32_t mask = (uint32_t)(kBins - 1) << SHIFT0;
   // fp32: the 16 bits below the first digit, 8 at a time
   int slot = 0;
   for (int shift = SHIFT0 - 8; shift >= 0; shift -= 8) {
     __syncthreads();
     clear_bins(sh, 256);
-    histogram_pass<DT, VECTOR>(sh, rd, 0, rd.n_groups, mask, prefix, 0u, shift, 255u);
+    // the keys that start with the digits found so far: prefix .. prefix + 2^(shift + 8) - 1
+    histogram_pass<DT, VECTOR>(sh, ring, rd, 0, rd.n_groups, prefix, prefix + (1u << (shift + 8)), shift, 255u);
     __syncthreads();
     find_bin_from_top(sh, 256, remaining, slot);
     slot ^= 1;
     prefix |= sh.picked_bin << shift;
     remaining = sh.picked_remaining;
-    mask |= 255u << shift;
   }
   *kth = prefix;
   *take = remaining;
@@ -229,33 +312,31 @@ static_assert((key_bits(1) - kTopBits) % 8 == 0 && key_bits(0) == kTopBits, "dig
 
 // Visits the chunk's top-k in ascending index order: emit(position, flat index, pattern).
 template <int DT, bool VECTOR, class Emit>
-__device__ void collect_in_index_order(DirectShared& sh, const Reader<DT, VECTOR>& rd, int k, uint32_t kth,
+__device__ void collect_in_index_order(DirectShared& sh, uint4* ring, const Reader<DT, VECTOR>& rd, int k, uint32_t kth,
                                        uint32_t take, Emit emit) {
   using R = Reader<DT, VECTOR>;
   const uint32_t n_above = (uint32_t)k - take;
   uint32_t base_above = 0, base_equal = 0;
   int slot = 0;
+  rd.request(ring, (int)threadIdx.x, rd.n_groups);
   for (int t0 = 0; t0 < rd.n_groups; t0 += kUnroll * kThreads) {
     uint32_t w[kUnroll][4];
     unsigned long long above = 0, equal = 0;  // 16 bits per sub-tile
+    rd.take(ring, t0 + (int)threadIdx.x, rd.n_groups, w);
+    if (t0 + kUnroll * kThreads < rd.n_groups)
+      rd.request_after(ring, t0 + kUnroll * kThreads + (int)threadIdx.x, rd.n_groups, w, t0 + (int)threadIdx.x,
+                       rd.n_groups);
+    uint32_t reach[kUnroll];  // per sub-tile: elements >= kth in bits 0..7, elements > kth in bits 8..15
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int g = t0 + u * kThreads + (int)threadIdx.x;
-      if (g < rd.n_groups) rd.load(g, w[u]);
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int g = t0 + u * kThreads + (int)threadIdx.x;
+      reach[u] = 0;
       if (g < rd.n_groups) {
-        uint32_t a = 0, e = 0;
-#pragma unroll
-        for (int j = 0; j < R::VEC; ++j) {
-          const uint32_t key = R::key(R::pattern(w[u], j));
-          a += key > kth;
-          e += key == kth;
-        }
+        const uint32_t ge = R::reach_mask(w[u], kth), gt = R::reach_mask(w[u], kth + 1u);
+        reach[u] = ge | (gt << 8);
+        const uint32_t a = (uint32_t)__popc(gt);
         above |= (unsigned long long)a << (16 * u);
-        equal |= (unsigned long long)e << (16 * u);
+        equal |= (unsigned long long)((uint32_t)__popc(ge) - a) << (16 * u);
       }
     }
     unsigned long long total_above, total_equal;
@@ -266,18 +347,17 @@ __device__ void collect_in_index_order(DirectShared& sh, const Reader<DT, VECTOR
       const int g = t0 + u * kThreads + (int)threadIdx.x;
       uint32_t above_before = base_above + (uint32_t)((ex_above >> (16 * u)) & 0xFFFFu);
       uint32_t equal_before = base_equal + (uint32_t)((ex_equal >> (16 * u)) & 0xFFFFu);
-      if (g < rd.n_groups && (((above | equal) >> (16 * u)) & 0xFFFFu) != 0) {
-#pragma unroll
-        for (int j = 0; j < R::VEC; ++j) {
-          const uint32_t pat = R::pattern(w[u], j);
-          const uint32_t key = R::key(pat);
-          if (key > kth) {
-            emit(above_before + (equal_before < take ? equal_before : take), (uint32_t)g * R::VEC + j, R::committed(pat));
-            ++above_before;
-          } else if (key == kth) {
-            if (equal_before < take) emit(above_before + equal_before, (uint32_t)g * R::VEC + j, R::committed(pat));
-            ++equal_before;
-          }
+      uint32_t m = reach[u] & 0xFFu;
+      while (m) {  // in index order
+        const uint32_t j = (uint32_t)__ffs((int)m) - 1u;
+        m &= m - 1u;
+        const uint32_t pat = R::pattern_at(w[u], j);
+        if ((reach[u] >> (8 + j)) & 1u) {
+          emit(above_before + (equal_before < take ? equal_before : take), (uint32_t)g * R::VEC + j, R::committed(pat));
+          ++above_before;
+        } else {
+          if (equal_before < take) emit(above_before + equal_before, (uint32_t)g * R::VEC + j, R::committed(pat));
+          ++equal_before;
         }
       }
       base_above += (uint32_t)((total_above >> (16 * u)) & 0xFFFFu);
@@ -285,6 +365,7 @@ __device__ void collect_in_index_order(DirectShared& sh, const Reader<DT, VECTOR
     }
     if (base_above == n_above && base_equal >= take) break;  // the same for every thread
   }
+  if (VECTOR) asm volatile("cp.async.wait_group 0;" ::: "memory");  // a batch requested before the break
 }
 
 template <int DT, bool VECTOR>
@@ -299,6 +380,7 @@ __device__ __forceinline__ Reader<DT, VECTOR> locate_chunk(const DirectParams& p
   rd.base = static_cast<const char*>(p.act) + row0 * p.row_stride * R::ESZ;
   rd.row_stride_bytes = p.row_stride * R::ESZ;
   rd.groups_per_row = p.hidden / R::VEC;
+  rd.flat = p.row_stride == p.hidden;
   rd.n_groups = rows * rd.groups_per_row;
   return rd;
 }
@@ -308,6 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw);
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw + sizeof(DirectShared));
   using R = Reader<DT, VECTOR>;
   const long long chunk = blockIdx.x;
   const R rd = locate_chunk<DT, VECTOR>(p, chunk);
@@ -318,8 +401,8 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
     return;
   }
   uint32_t kth, take;
-  find_kth_key<DT, VECTOR>(sh, rd, p.k, &kth, &take);
-  collect_in_index_order<DT, VECTOR>(sh, rd, p.k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+  find_kth_key<DT, VECTOR>(sh, ring, rd, p.k, &kth, &take);
+  collect_in_index_order<DT, VECTOR>(sh, ring, rd, p.k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
     if (pos >= (uint32_t)p.k) return;
     rec[3 * pos] = (uint16_t)(flat & 0xFFFFu);
     rec[3 * pos + 1] = (uint16_t)(flat >> 16);
@@ -333,7 +416,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw);
-  uint32_t* sel_idx = reinterpret_cast<uint32_t*>(smem_raw + sizeof(DirectShared));
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw + sizeof(DirectShared));
+  // the two selections live where the key histogram was (it is done with once the k-th key is known)
+  uint32_t* sel_idx = sh.hist + kListOffset;
   uint32_t* com_idx = sel_idx + p.k;
   uint16_t* sel_pat = reinterpret_cast<uint16_t*>(com_idx + p.k);
   uint16_t* com_pat = sel_pat + p.k;
@@ -343,28 +428,10 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
   const R rd = locate_chunk<DT, VECTOR>(p, chunk);
   const uint32_t n_elems = (uint32_t)rd.n_groups * R::VEC;
 
-  // decode the commitment; its indices must ascend strictly and lie inside the chunk
-  const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
   if (threadIdx.x == 0) sh.bad = 0;
   if (threadIdx.x < 4) sh.counters[threadIdx.x] = 0;
   if (threadIdx.x < 9) sh.dev[threadIdx.x] = 0;
-  for (int j = threadIdx.x; j < k; j += kThreads) {
-    com_idx[j] = (uint32_t)rec[3 * j] | ((uint32_t)rec[3 * j + 1] << 16);
-    com_pat[j] = rec[3 * j + 2];
-  }
-  __syncthreads();
-  int status = TOPLOC_CHUNK_OK;
-  if (n_elems < (uint32_t)k) {
-    status = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
-  } else {
-    uint32_t bad = 0;
-    for (int j = threadIdx.x; j < k; j += kThreads)
-      bad |= (com_idx[j] >= n_elems) | (j > 0 && com_idx[j] <= com_idx[j - 1]);
-    if (bad) sh.bad = 1;
-    __syncthreads();
-    if (sh.bad) status = TOPLOC_CHUNK_BAD_PROOF;
-  }
-  if (status != TOPLOC_CHUNK_OK) {
+  auto refuse = [&](int status) {  // every thread takes the same way out
     if (threadIdx.x == 0) {
       toploc_chunk_result r = {};
       r.topk_mismatch = -1;
@@ -372,19 +439,39 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
       io.results[chunk] = r;
     }
     if (io.exp_dev != nullptr && threadIdx.x < 9) io.exp_dev[(size_t)chunk * 9 + threadIdx.x] = 0;
+  };
+  if (n_elems < (uint32_t)k) {
+    refuse(TOPLOC_CHUNK_K_EXCEEDS_CHUNK);
     return;
   }
 
   uint32_t kth, take;
-  find_kth_key<DT, VECTOR>(sh, rd, k, &kth, &take);
-  collect_in_index_order<DT, VECTOR>(sh, rd, k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+  find_kth_key<DT, VECTOR>(sh, ring, rd, k, &kth, &take);
+  collect_in_index_order<DT, VECTOR>(sh, ring, rd, k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
     if (pos >= (uint32_t)k) return;
     sel_idx[pos] = flat;
     sel_pat[pos] = (uint16_t)pat;
   });
-  __syncthreads();
+
+  // decode the commitment; its indices must ascend strictly and lie inside the chunk
+  const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
+  for (int j = threadIdx.x; j < k; j += kThreads) {
+    com_idx[j] = (uint32_t)rec[3 * j] | ((uint32_t)rec[3 * j + 1] << 16);
+    com_pat[j] = rec[3 * j + 2];
+  }
   for (int b = threadIdx.x; b < 128; b += kThreads) sh.hist[b] = 0;  // mantissa differences 0..127
   __syncthreads();
+  {
+    uint32_t bad = 0;
+    for (int j = threadIdx.x; j < k; j += kThreads)
+      bad |= (com_idx[j] >= n_elems) | (j > 0 && com_idx[j] <= com_idx[j - 1]);
+    if (bad) sh.bad = 1;
+    __syncthreads();
+    if (sh.bad) {
+      refuse(TOPLOC_CHUNK_BAD_PROOF);
+      return;
+    }
+  }
 
   // Algorithm 2 with a look-up in place of the polynomial
   uint32_t err_e = 0, n_match = 0, sum = 0, common = 0, dev[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
@@ -533,7 +620,7 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
     return TOPLOC_ERR_INVALID_ARGUMENT;
   if ((rc = check_device()) != TOPLOC_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const size_t smem = sizeof(DirectShared);
+  const size_t smem = sizeof(DirectShared) + kRingBytes;
   const DirectParams& p = plan.params;
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_commit_kernel<0, true>, plan.num_chunks, smem, stream, p, d_commits, d_status)
@@ -562,7 +649,7 @@ int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint
   io.sign_in_exponent = thr->sign_in_exponent;
   io.t_mean = thr->t_mean;
   io.t_median = thr->t_median;
-  const size_t smem = sizeof(DirectShared) + 12 * (size_t)lay->k;
+  const size_t smem = sizeof(DirectShared) + kRingBytes;
   const DirectParams& p = plan.params;
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_verify_kernel<0, true>, plan.num_chunks, smem, stream, p, io)
