@@ -17,6 +17,7 @@
 // places them, by a block-wide prefix sum, in ascending index order.  The chunk is read from
 // HBM by the first pass; the later passes find it in L2 (one block per SM: 148 chunks in flight).
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include "toploc.h"
@@ -52,15 +53,29 @@ struct DirectVerify {
   double t_median;
 };
 
+// Dynamic shared memory of a block: the copy ring, this struct, and kSpareBytes that continue
+// its last member (the one-pass selection keeps its candidates in hist and the spare together).
 struct DirectShared {
-  uint32_t hist[kBins];
   unsigned long long warp_sums[2][kWarps];
   uint32_t picked_bin;
   uint32_t picked_remaining;
   uint32_t bad;
   uint32_t counters[4];      // exponent mismatches, matches, mantissa difference sum, common indices
   uint32_t dev[9];
+  uint32_t hist[kBins];
 };
+constexpr size_t kSpareBytes = 35264;
+constexpr size_t kSharedBytes = kRingBytes + sizeof(DirectShared) + kSpareBytes;
+// One-pass selection (bf16 vector layouts, k <= kStreamMaxK): a histogram of the upper 11 key
+// bits and up to kCandCap candidates (flat index, pattern) in index order.
+constexpr int kCoarseBins = 2048;
+constexpr int kCoarseShift = 4;
+constexpr int kCandCap = 26112;
+constexpr int kStreamMaxK = 2048;
+static_assert(kSharedBytes <= 227 * 1024 && sizeof(DirectShared) % 16 == 0 && kSpareBytes % 16 == 0, "shared memory budget");
+static_assert(offsetof(DirectShared, hist) + sizeof(uint32_t) * kBins == sizeof(DirectShared), "hist is the last member");
+static_assert((size_t)kCoarseBins * 4 + (size_t)kCandCap * 6 <= (size_t)kBins * 4 + kSpareBytes, "candidates fit");
+static_assert(12 * TOPLOC_MAX_K_DIRECT <= kRingBytes, "the verify lists fit the idle ring");
 
 // A group is VEC consecutive elements of one row (one 16-byte vector, or one element when
 // the layout does not allow aligned vectors).
@@ -199,7 +214,6 @@ __device__ __forceinline__ unsigned long long block_scan_exclusive(DirectShared&
 }
 static_assert(kWarps == 32, "the second level of the block scan is one warp wide");
 static_assert(kListOffset * 4 + 12 * TOPLOC_MAX_K_DIRECT <= kBins * 4, "the verify lists fit where the histogram was");
-static_assert(sizeof(DirectShared) % 16 == 0 && sizeof(DirectShared) + kRingBytes <= 227 * 1024, "shared memory budget");
 static_assert((kBins / kThreads & (kBins / kThreads - 1)) == 0, "bins per thread: a power of two");
 
 // The bin, counted from the top, in which the want-th largest counted element lies
@@ -368,6 +382,133 @@ __device__ void collect_in_index_order(DirectShared& sh, uint4* ring, const Read
   if (VECTOR) asm volatile("cp.async.wait_group 0;" ::: "memory");  // a batch requested before the break
 }
 
+// One-pass selection for bf16 vector layouts.  The chunk is streamed once, in batches of
+// kUnroll * kThreads vectors; every element whose key reaches the running threshold is kept as a
+// candidate (flat index, pattern), in index order (a block-wide prefix sum per batch places
+// them), and counted in a histogram of its upper 11 key bits.  Whenever enough candidates have
+// arrived, the threshold is raised to the lowest key of the bin that holds the k-th largest
+// candidate so far -- a lower bound of the chunk's k-th largest key, so nothing of the top-k is
+// ever dropped.  The first batch (about 4k elements, threshold 0) seeds the histogram.  At the
+// end the exact k-th key is found among the candidates (two digits of 8 and 7 bits) and the
+// top-k leaves in index order, ties to the lower index.  Returns false, having emitted nothing,
+// when the candidates outgrow their buffer (data sorted upwards, say): the caller then takes
+// the two-pass selection.
+template <class Emit>
+__device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<0, true>& rd, int k, Emit emit) {
+  using R = Reader<0, true>;
+  uint32_t* coarse = sh.hist;
+  uint32_t* cand_flat = sh.hist + kCoarseBins;
+  uint16_t* cand_pat = reinterpret_cast<uint16_t*>(cand_flat + kCandCap);
+  clear_bins(sh, kCoarseBins);
+  int seed_groups = (4 * k > 8192 ? 4 * k : 8192) / R::VEC;
+  if (seed_groups > rd.n_groups) seed_groups = rd.n_groups;
+  const uint32_t raise_step = (uint32_t)(k / 4 > 64 ? k / 4 : 64);
+  uint32_t thr = 0, count = 0, last_raise = 0;
+  int begin = 0, end = seed_groups, slot = 0;
+  bool overflow = false;
+  rd.request(ring, (int)threadIdx.x, end);
+  while (begin < rd.n_groups) {
+    uint32_t w[kUnroll][4];
+    rd.take(ring, begin + (int)threadIdx.x, end, w);
+    const int next_begin = end;
+    int next_end = next_begin + kUnroll * kThreads;
+    if (next_end > rd.n_groups) next_end = rd.n_groups;
+    if (next_begin < rd.n_groups)
+      rd.request_after(ring, next_begin + (int)threadIdx.x, next_end, w, begin + (int)threadIdx.x, end);
+    uint32_t reach[kUnroll];
+    unsigned long long hits = 0;  // 16 bits per sub-tile
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = begin + u * kThreads + (int)threadIdx.x;
+      reach[u] = g < end ? R::reach_mask(w[u], thr) : 0u;
+      hits |= (unsigned long long)__popc(reach[u]) << (16 * u);
+    }
+    unsigned long long total;
+    const unsigned long long before = block_scan_exclusive(sh, hits, slot, &total);
+    slot ^= 1;
+    uint32_t batch_total = 0;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) batch_total += (uint32_t)((total >> (16 * u)) & 0xFFFFu);
+    if (count + batch_total > (uint32_t)kCandCap) {  // the same for every thread
+      overflow = true;
+      break;
+    }
+    uint32_t tile_base = count;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = begin + u * kThreads + (int)threadIdx.x;
+      uint32_t at = tile_base + (uint32_t)((before >> (16 * u)) & 0xFFFFu);
+      uint32_t m = reach[u];
+      while (m) {  // in index order
+        const uint32_t j = (uint32_t)__ffs((int)m) - 1u;
+        m &= m - 1u;
+        const uint32_t pat = R::pattern_at(w[u], j);
+        cand_flat[at] = (uint32_t)g * R::VEC + j;
+        cand_pat[at] = (uint16_t)pat;
+        atomicAdd(&coarse[(pat & 0x7FFFu) >> kCoarseShift], 1u);
+        ++at;
+      }
+      tile_base += (uint32_t)((total >> (16 * u)) & 0xFFFFu);
+    }
+    count += batch_total;
+    if (count - last_raise >= raise_step && next_begin < rd.n_groups) {  // the same for every thread
+      __syncthreads();  // this batch's counts are in
+      find_bin_from_top(sh, kCoarseBins, (uint32_t)k, slot);
+      slot ^= 1;
+      const uint32_t floor_key = sh.picked_bin << kCoarseShift;
+      if (floor_key > thr) thr = floor_key;
+      last_raise = count;
+    }
+    begin = next_begin;
+    end = next_end;
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");  // a batch requested before leaving the loop
+  __syncthreads();
+  if (overflow) return false;
+
+  // the exact k-th key among the candidates: upper 8 bits, then lower 7
+  clear_bins(sh, 256);
+  for (uint32_t i = threadIdx.x; i < count; i += kThreads) atomicAdd(&sh.hist[(cand_pat[i] & 0x7FFFu) >> 7], 1u);
+  __syncthreads();
+  find_bin_from_top(sh, 256, (uint32_t)k, 0);
+  const uint32_t upper = sh.picked_bin, within = sh.picked_remaining;
+  __syncthreads();
+  clear_bins(sh, 128);
+  for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+    const uint32_t key = cand_pat[i] & 0x7FFFu;
+    if ((key >> 7) == upper) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
+  }
+  __syncthreads();
+  find_bin_from_top(sh, 128, within, 1);
+  const uint32_t kth = (upper << 7) | sh.picked_bin, take = sh.picked_remaining;
+
+  // the top-k in index order: every thread takes a run of consecutive candidates
+  const uint32_t per = ((count + kThreads - 1) / kThreads) | 1u;  // odd: the runs start in different banks
+  const uint32_t lo = threadIdx.x * per < count ? threadIdx.x * per : count;
+  const uint32_t hi = lo + per < count ? lo + per : count;
+  uint32_t above = 0, equal = 0;
+  for (uint32_t i = lo; i < hi; ++i) {
+    const uint32_t key = cand_pat[i] & 0x7FFFu;
+    above += key > kth;
+    equal += key == kth;
+  }
+  unsigned long long total;
+  const unsigned long long before = block_scan_exclusive(sh, above | ((unsigned long long)equal << 32), 0, &total);
+  uint32_t above_before = (uint32_t)before, equal_before = (uint32_t)(before >> 32);
+  for (uint32_t i = lo; i < hi; ++i) {
+    const uint32_t pat = cand_pat[i], key = pat & 0x7FFFu;
+    if (key > kth) {
+      emit(above_before + (equal_before < take ? equal_before : take), cand_flat[i], pat);
+      ++above_before;
+    } else if (key == kth) {
+      if (equal_before < take) emit(above_before + equal_before, cand_flat[i], pat);
+      ++equal_before;
+    }
+  }
+  __syncthreads();
+  return true;
+}
+
 template <int DT, bool VECTOR>
 __device__ __forceinline__ Reader<DT, VECTOR> locate_chunk(const DirectParams& p, long long chunk) {
   using R = Reader<DT, VECTOR>;
@@ -389,8 +530,8 @@ template <int DT, bool VECTOR>
 __global__ void __launch_bounds__(kThreads, 1)
 toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw);
-  uint4* ring = reinterpret_cast<uint4*>(smem_raw + sizeof(DirectShared));
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw);
+  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw + kRingBytes);
   using R = Reader<DT, VECTOR>;
   const long long chunk = blockIdx.x;
   const R rd = locate_chunk<DT, VECTOR>(p, chunk);
@@ -400,28 +541,74 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
     if (threadIdx.x == 0) status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
     return;
   }
-  uint32_t kth, take;
-  find_kth_key<DT, VECTOR>(sh, ring, rd, p.k, &kth, &take);
-  collect_in_index_order<DT, VECTOR>(sh, ring, rd, p.k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+  auto emit = [&](uint32_t pos, uint32_t flat, uint32_t pat) {
     if (pos >= (uint32_t)p.k) return;
     rec[3 * pos] = (uint16_t)(flat & 0xFFFFu);
     rec[3 * pos + 1] = (uint16_t)(flat >> 16);
     rec[3 * pos + 2] = (uint16_t)pat;
-  });
+  };
+  bool done = false;
+  if constexpr (DT == 0 && VECTOR) {
+    if (p.k <= kStreamMaxK) done = select_in_one_pass(sh, ring, rd, p.k, emit);
+  }
+  if (!done) {
+    uint32_t kth, take;
+    find_kth_key<DT, VECTOR>(sh, ring, rd, p.k, &kth, &take);
+    collect_in_index_order<DT, VECTOR>(sh, ring, rd, p.k, kth, take, emit);
+  }
   if (threadIdx.x == 0) status[chunk] = TOPLOC_CHUNK_OK;
+}
+
+// The double nearest to s / n (ties to even; n > 0) by long division in integers -- the
+// same value as the fp64 division, which, issued by one thread at the end of a block that
+// has the SM to itself, was measured at 5 us per chunk.
+__device__ __forceinline__ double nearest_ratio(uint32_t s, uint32_t n) {
+  if (s == 0) return 0.0;
+  const uint32_t whole = s / n;
+  unsigned long long r = s - whole * n, m;
+  int e, have;
+  if (whole) {
+    e = 31 - __clz(whole);
+    m = whole;
+    have = e + 1;
+  } else {  // the leading zeros of the fraction
+    e = 0;
+    do {
+      --e;
+      r <<= 1;
+    } while (r < n);
+    r -= n;
+    m = 1;
+    have = 1;
+  }
+  for (; have < 54; ++have) {  // 53 bits and a guard bit
+    r <<= 1;
+    m <<= 1;
+    if (r >= n) {
+      r -= n;
+      m |= 1;
+    }
+  }
+  const bool guard = m & 1ull;
+  m >>= 1;
+  if (guard && (r != 0 || (m & 1ull))) ++m;
+  if (m >> 53) {
+    m >>= 1;
+    ++e;
+  }
+  return __longlong_as_double(((long long)(1023 + e) << 52) | (long long)(m & ((1ull << 52) - 1ull)));
 }
 
 template <int DT, bool VECTOR>
 __global__ void __launch_bounds__(kThreads, 1)
 toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw);
-  uint4* ring = reinterpret_cast<uint4*>(smem_raw + sizeof(DirectShared));
-  // the two selections live where the key histogram was (it is done with once the k-th key is known)
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw);
+  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw + kRingBytes);
+  // The two selections live where the key histogram was (it is done with once the k-th key is
+  // known), or, after the one-pass selection, in the ring (idle by then).
   uint32_t* sel_idx = sh.hist + kListOffset;
-  uint32_t* com_idx = sel_idx + p.k;
-  uint16_t* sel_pat = reinterpret_cast<uint16_t*>(com_idx + p.k);
-  uint16_t* com_pat = sel_pat + p.k;
+  uint16_t* sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * p.k);
   using R = Reader<DT, VECTOR>;
   const long long chunk = blockIdx.x;
   const int k = p.k;
@@ -445,13 +632,28 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
     return;
   }
 
-  uint32_t kth, take;
-  find_kth_key<DT, VECTOR>(sh, ring, rd, k, &kth, &take);
-  collect_in_index_order<DT, VECTOR>(sh, ring, rd, k, kth, take, [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+  auto emit = [&](uint32_t pos, uint32_t flat, uint32_t pat) {
     if (pos >= (uint32_t)k) return;
     sel_idx[pos] = flat;
     sel_pat[pos] = (uint16_t)pat;
-  });
+  };
+  bool done = false;
+  if constexpr (DT == 0 && VECTOR) {
+    if (k <= kStreamMaxK) {
+      sel_idx = reinterpret_cast<uint32_t*>(ring);
+      sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
+      done = select_in_one_pass(sh, ring, rd, k, emit);
+    }
+  }
+  if (!done) {
+    sel_idx = sh.hist + kListOffset;
+    sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
+    uint32_t kth, take;
+    find_kth_key<DT, VECTOR>(sh, ring, rd, k, &kth, &take);
+    collect_in_index_order<DT, VECTOR>(sh, ring, rd, k, kth, take, emit);
+  }
+  uint32_t* com_idx = sel_idx + k;
+  uint16_t* com_pat = sel_pat + k;
 
   // decode the commitment; its indices must ascend strictly and lie inside the chunk
   const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
@@ -529,7 +731,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
     r.topk_mismatch = k - (int)sh.counters[3];
     bool reject = r.exp_mismatch > (uint32_t)io.t_exp;
     if (r.n_match > 0) {
-      r.mant_mean = (double)r.mant_diff_sum / (double)r.n_match;
+      r.mant_mean = nearest_ratio(r.mant_diff_sum, r.n_match);
       // values at sorted positions (n - 1) / 2 and n / 2
       const uint32_t lo_rank = (r.n_match - 1) / 2, hi_rank = r.n_match / 2;
       uint32_t seen = 0;
@@ -539,7 +741,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
         if (lo_val < 0 && seen > lo_rank) lo_val = b;
         if (seen > hi_rank) hi_val = b;
       }
-      r.mant_median = ((double)lo_val + (double)hi_val) / 2.0;
+      r.mant_median = ((double)lo_val + (double)hi_val) * 0.5;
       reject = reject || r.mant_mean > io.t_mean || r.mant_median > io.t_median;
     } else {
       reject = true;  // nothing matched: no statistic to accept on
@@ -620,7 +822,7 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
     return TOPLOC_ERR_INVALID_ARGUMENT;
   if ((rc = check_device()) != TOPLOC_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const size_t smem = sizeof(DirectShared) + kRingBytes;
+  const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_commit_kernel<0, true>, plan.num_chunks, smem, stream, p, d_commits, d_status)
@@ -649,7 +851,7 @@ int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint
   io.sign_in_exponent = thr->sign_in_exponent;
   io.t_mean = thr->t_mean;
   io.t_median = thr->t_median;
-  const size_t smem = sizeof(DirectShared) + kRingBytes;
+  const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_verify_kernel<0, true>, plan.num_chunks, smem, stream, p, io)
