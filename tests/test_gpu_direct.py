@@ -83,6 +83,16 @@ def test_ties_decide_the_selection():
     direct_case(asc, L, 512, 1, L, None, "ascending")
 
 
+def test_rising_magnitudes_outgrow_the_candidate_buffer():
+    # every element reaches the running threshold: the one-pass selection gives up and the
+    # two-pass selection takes the chunk; a second, ordinary chunk rides along
+    H, L, k = 4096, 32, 512
+    rising = (torch.arange(L * H, device=DEV, dtype=torch.float32).reshape(L, H) / 256 + 1).to(torch.bfloat16)
+    usual = synth.make_activations(1, L, H, torch.bfloat16, seed=77, device=DEV, outliers="none")
+    act = torch.cat([rising, usual]).contiguous()
+    direct_case(act, L, k, 2, L, {"falling": torch.cat([rising.flip(0).flip(1), usual]).contiguous()}, "rising")
+
+
 def test_special_patterns():
     H, L, k = 512, 8, 200
     bits = torch.randint(0, 65536, (L, H), dtype=torch.int32, device=DEV).to(torch.int16)  # NaN, Inf, subnormals
