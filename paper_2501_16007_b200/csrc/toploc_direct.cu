@@ -7,15 +7,21 @@
 //   toploc_direct_commit_kernel<dtype, vector>   one 1024-thread block per chunk
 //   toploc_direct_verify_kernel<dtype, vector>   the same selection, then the comparison
 //
-// Selection of a chunk (both kernels): a radix select on the magnitude key with the whole
-// first digit -- 15 bits, i.e. every bf16 key -- histogrammed in shared memory.  A first part
-// of the chunk is counted in full; the k-th largest key of that part is a sound lower
-// bound for the chunk's k-th largest key, so the rest of the chunk only counts elements that
-// reach it (few shared-memory atomics).  fp32 keys take two more 8-bit digits over the
-// elements that match the digits found so far.  A last pass in index order takes every key
-// above the k-th largest and the first elements equal to it (ties go to the lower index) and
-// places them, by a block-wide prefix sum, in ascending index order.  The chunk is read from
-// HBM by the first pass; the later passes find it in L2 (one block per SM: 148 chunks in flight).
+// Selection of a chunk (both kernels), one of two ways:
+//   one pass (bf16 vector layouts, k <= 2048): the chunk is streamed once; elements that reach a
+//   running threshold are kept as candidates in shared memory, in index order, and counted in a
+//   histogram of their upper 11 key bits, from which the threshold is raised as candidates
+//   arrive; the exact k-th key is then found among the candidates (select_in_one_pass);
+//   two passes (everything else, and chunks whose candidates outgrow their buffer): a radix
+//   select on the magnitude key with the whole first digit -- 15 bits, i.e. every bf16 key --
+//   histogrammed in shared memory.  A first part of the chunk is counted in full; the k-th
+//   largest key of that part is a sound lower bound for the chunk's k-th largest key, so the
+//   rest of the chunk only counts elements that reach it.  fp32 keys take two more 8-bit digits
+//   over the elements that match the digits found so far.  A last pass in index order takes
+//   every key above the k-th largest and the first elements equal to it (ties go to the lower
+//   index) and places them, by a block-wide prefix sum, in ascending index order.  The chunk is
+//   read from HBM by the first pass; the second finds it in L2 (one block per SM: 148 chunks
+//   in flight).
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -400,7 +406,7 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<0
   uint32_t* cand_flat = sh.hist + kCoarseBins;
   uint16_t* cand_pat = reinterpret_cast<uint16_t*>(cand_flat + kCandCap);
   clear_bins(sh, kCoarseBins);
-  int seed_groups = (4 * k > 8192 ? 4 * k : 8192) / R::VEC;
+  int seed_groups = (4 * k > 2048 ? 4 * k : 2048) / R::VEC;
   if (seed_groups > rd.n_groups) seed_groups = rd.n_groups;
   const uint32_t raise_step = (uint32_t)(k / 4 > 64 ? k / 4 : 64);
   uint32_t thr = 0, count = 0, last_raise = 0;
