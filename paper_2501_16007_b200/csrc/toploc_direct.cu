@@ -26,6 +26,7 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include "nearest_ratio.cuh"
 #include "toploc.h"
 
 namespace {
@@ -563,46 +564,6 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
     collect_in_index_order<DT, VECTOR>(sh, ring, rd, p.k, kth, take, emit);
   }
   if (threadIdx.x == 0) status[chunk] = TOPLOC_CHUNK_OK;
-}
-
-// The double nearest to s / n (ties to even; n > 0) by long division in integers -- the
-// same value as the fp64 division, which, issued by one thread at the end of a block that
-// has the SM to itself, was measured at 5 us per chunk.
-__device__ __forceinline__ double nearest_ratio(uint32_t s, uint32_t n) {
-  if (s == 0) return 0.0;
-  const uint32_t whole = s / n;
-  unsigned long long r = s - whole * n, m;
-  int e, have;
-  if (whole) {
-    e = 31 - __clz(whole);
-    m = whole;
-    have = e + 1;
-  } else {  // the leading zeros of the fraction
-    e = 0;
-    do {
-      --e;
-      r <<= 1;
-    } while (r < n);
-    r -= n;
-    m = 1;
-    have = 1;
-  }
-  for (; have < 54; ++have) {  // 53 bits and a guard bit
-    r <<= 1;
-    m <<= 1;
-    if (r >= n) {
-      r -= n;
-      m |= 1;
-    }
-  }
-  const bool guard = m & 1ull;
-  m >>= 1;
-  if (guard && (r != 0 || (m & 1ull))) ++m;
-  if (m >> 53) {
-    m >>= 1;
-    ++e;
-  }
-  return __longlong_as_double(((long long)(1023 + e) << 52) | (long long)(m & ((1ull << 52) - 1ull)));
 }
 
 template <int DT, bool VECTOR>
