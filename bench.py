@@ -450,6 +450,7 @@ def direct_commitments(tl, synth, dev, workload, reps=10):
                        "accepted": int(got["accept"].sum()), "chunks": int(got.size),
                        "mean_topk_mismatch": float(got["topk_mismatch"].mean())})
     return {"metric": "direct_commitments", "workload": workload_name(workload), "activation_bytes": nbytes,
+            "activations": "fp32, upper 16 bits of a pattern committed" if dtype == torch.float32 else "bf16",
             "peak_GB_per_s": peak, "peak_kind": peak_kind, "recomputed": "honest reorder noise, relative 2^-8",
             "points": points}
 

@@ -8,7 +8,7 @@
 //   toploc_direct_verify_kernel<dtype, vector>   the same selection, then the comparison
 //
 // Selection of a chunk (both kernels), one of two ways:
-//   one pass (bf16 vector layouts, k <= 2048): the chunk is streamed once; elements that reach a
+//   one pass (vector layouts; k <= 2048 for bf16, 1024 for fp32): the chunk is streamed once; elements that reach a
 //   running threshold are kept as candidates in shared memory, in index order, and counted in a
 //   histogram of their upper 11 key bits, from which the threshold is raised as candidates
 //   arrive; the exact k-th key is then found among the candidates (select_in_one_pass);
@@ -73,15 +73,16 @@ struct DirectShared {
 };
 constexpr size_t kSpareBytes = 35264;
 constexpr size_t kSharedBytes = kRingBytes + sizeof(DirectShared) + kSpareBytes;
-// One-pass selection (bf16 vector layouts, k <= kStreamMaxK): a histogram of the upper 11 key
-// bits and up to kCandCap candidates (flat index, pattern) in index order.
+// One-pass selection (vector layouts, k <= stream_max_k): a histogram of the upper 11 key bits
+// and up to cand_cap candidates (flat index, whole pattern) in index order.
 constexpr int kCoarseBins = 2048;
-constexpr int kCoarseShift = 4;
-constexpr int kCandCap = 26112;
-constexpr int kStreamMaxK = 2048;
+__host__ __device__ constexpr int cand_cap(int dt) { return dt == 0 ? 26112 : 19712; }       // 6 / 8 bytes each
+__host__ __device__ constexpr int stream_max_k(int dt) { return dt == 0 ? 2048 : 1024; }
 static_assert(kSharedBytes <= 227 * 1024 && sizeof(DirectShared) % 16 == 0 && kSpareBytes % 16 == 0, "shared memory budget");
 static_assert(offsetof(DirectShared, hist) + sizeof(uint32_t) * kBins == sizeof(DirectShared), "hist is the last member");
-static_assert((size_t)kCoarseBins * 4 + (size_t)kCandCap * 6 <= (size_t)kBins * 4 + kSpareBytes, "candidates fit");
+static_assert((size_t)kCoarseBins * 4 + (size_t)cand_cap(0) * 6 <= (size_t)kBins * 4 + kSpareBytes &&
+                  (size_t)kCoarseBins * 4 + (size_t)cand_cap(1) * 8 <= (size_t)kBins * 4 + kSpareBytes,
+              "candidates fit");
 static_assert(12 * TOPLOC_MAX_K_DIRECT <= kRingBytes, "the verify lists fit the idle ring");
 
 // A group is VEC consecutive elements of one row (one 16-byte vector, or one element when
@@ -389,23 +390,29 @@ __device__ void collect_in_index_order(DirectShared& sh, uint4* ring, const Read
   if (VECTOR) asm volatile("cp.async.wait_group 0;" ::: "memory");  // a batch requested before the break
 }
 
-// One-pass selection for bf16 vector layouts.  The chunk is streamed once, in batches of
+// One-pass selection for vector layouts.  The chunk is streamed once, in batches of
 // kUnroll * kThreads vectors; every element whose key reaches the running threshold is kept as a
 // candidate (flat index, pattern), in index order (a block-wide prefix sum per batch places
 // them), and counted in a histogram of its upper 11 key bits.  Whenever enough candidates have
 // arrived, the threshold is raised to the lowest key of the bin that holds the k-th largest
 // candidate so far -- a lower bound of the chunk's k-th largest key, so nothing of the top-k is
 // ever dropped.  The first batch (about 4k elements, threshold 0) seeds the histogram.  At the
-// end the exact k-th key is found among the candidates (two digits of 8 and 7 bits) and the
+// end the exact k-th key is found among the candidates (digits of 8 bits, the last of 7) and the
 // top-k leaves in index order, ties to the lower index.  Returns false, having emitted nothing,
 // when the candidates outgrow their buffer (data sorted upwards, say): the caller then takes
 // the two-pass selection.
-template <class Emit>
-__device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<0, true>& rd, int k, Emit emit) {
-  using R = Reader<0, true>;
+template <int DT> struct StoredPattern { typedef uint16_t type; };
+template <> struct StoredPattern<1> { typedef uint32_t type; };
+
+template <int DT, class Emit>
+__device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit) {
+  using R = Reader<DT, true>;
+  using Pat = typename StoredPattern<DT>::type;
+  constexpr int kCandCap = cand_cap(DT);
+  constexpr int kCoarseShift = key_bits(DT) - 11;
   uint32_t* coarse = sh.hist;
   uint32_t* cand_flat = sh.hist + kCoarseBins;
-  uint16_t* cand_pat = reinterpret_cast<uint16_t*>(cand_flat + kCandCap);
+  Pat* cand_pat = reinterpret_cast<Pat*>(cand_flat + kCandCap);
   clear_bins(sh, kCoarseBins);
   int seed_groups = (4 * k > 2048 ? 4 * k : 2048) / R::VEC;
   if (seed_groups > rd.n_groups) seed_groups = rd.n_groups;
@@ -451,8 +458,8 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<0
         m &= m - 1u;
         const uint32_t pat = R::pattern_at(w[u], j);
         cand_flat[at] = (uint32_t)g * R::VEC + j;
-        cand_pat[at] = (uint16_t)pat;
-        atomicAdd(&coarse[(pat & 0x7FFFu) >> kCoarseShift], 1u);
+        cand_pat[at] = (Pat)pat;
+        atomicAdd(&coarse[R::key(pat) >> kCoarseShift], 1u);
         ++at;
       }
       tile_base += (uint32_t)((total >> (16 * u)) & 0xFFFFu);
@@ -473,21 +480,22 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<0
   __syncthreads();
   if (overflow) return false;
 
-  // the exact k-th key among the candidates: upper 8 bits, then lower 7
-  clear_bins(sh, 256);
-  for (uint32_t i = threadIdx.x; i < count; i += kThreads) atomicAdd(&sh.hist[(cand_pat[i] & 0x7FFFu) >> 7], 1u);
-  __syncthreads();
-  find_bin_from_top(sh, 256, (uint32_t)k, 0);
-  const uint32_t upper = sh.picked_bin, within = sh.picked_remaining;
-  __syncthreads();
-  clear_bins(sh, 128);
-  for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
-    const uint32_t key = cand_pat[i] & 0x7FFFu;
-    if ((key >> 7) == upper) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
+  // the exact k-th key among the candidates, 8 bits at a time from the top (the last digit has 7)
+  uint32_t kth = 0, known = 0, take = (uint32_t)k;
+  for (int shift = key_bits(DT) - 8, round = 0; shift > -8; shift -= 8, ++round) {
+    const int low = shift < 0 ? 0 : shift, width = shift < 0 ? 8 + shift : 8;
+    clear_bins(sh, 256);
+    for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+      const uint32_t key = R::key(cand_pat[i]);
+      if ((key & known) == kth) atomicAdd(&sh.hist[(key >> low) & ((1u << width) - 1u)], 1u);
+    }
+    __syncthreads();
+    find_bin_from_top(sh, 1 << width, take, round & 1);
+    kth |= sh.picked_bin << low;
+    known |= ((1u << width) - 1u) << low;
+    take = sh.picked_remaining;
+    __syncthreads();
   }
-  __syncthreads();
-  find_bin_from_top(sh, 128, within, 1);
-  const uint32_t kth = (upper << 7) | sh.picked_bin, take = sh.picked_remaining;
 
   // the top-k in index order: every thread takes a run of consecutive candidates
   const uint32_t per = ((count + kThreads - 1) / kThreads) | 1u;  // odd: the runs start in different banks
@@ -495,7 +503,7 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<0
   const uint32_t hi = lo + per < count ? lo + per : count;
   uint32_t above = 0, equal = 0;
   for (uint32_t i = lo; i < hi; ++i) {
-    const uint32_t key = cand_pat[i] & 0x7FFFu;
+    const uint32_t key = R::key(cand_pat[i]);
     above += key > kth;
     equal += key == kth;
   }
@@ -503,12 +511,12 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<0
   const unsigned long long before = block_scan_exclusive(sh, above | ((unsigned long long)equal << 32), 0, &total);
   uint32_t above_before = (uint32_t)before, equal_before = (uint32_t)(before >> 32);
   for (uint32_t i = lo; i < hi; ++i) {
-    const uint32_t pat = cand_pat[i], key = pat & 0x7FFFu;
+    const uint32_t pat = cand_pat[i], key = R::key(pat);
     if (key > kth) {
-      emit(above_before + (equal_before < take ? equal_before : take), cand_flat[i], pat);
+      emit(above_before + (equal_before < take ? equal_before : take), cand_flat[i], R::committed(pat));
       ++above_before;
     } else if (key == kth) {
-      if (equal_before < take) emit(above_before + equal_before, cand_flat[i], pat);
+      if (equal_before < take) emit(above_before + equal_before, cand_flat[i], R::committed(pat));
       ++equal_before;
     }
   }
@@ -555,8 +563,8 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
     rec[3 * pos + 2] = (uint16_t)pat;
   };
   bool done = false;
-  if constexpr (DT == 0 && VECTOR) {
-    if (p.k <= kStreamMaxK) done = select_in_one_pass(sh, ring, rd, p.k, emit);
+  if constexpr (VECTOR) {
+    if (p.k <= stream_max_k(DT)) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
   }
   if (!done) {
     uint32_t kth, take;
@@ -605,11 +613,11 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
     sel_pat[pos] = (uint16_t)pat;
   };
   bool done = false;
-  if constexpr (DT == 0 && VECTOR) {
-    if (k <= kStreamMaxK) {
+  if constexpr (VECTOR) {
+    if (k <= stream_max_k(DT)) {
       sel_idx = reinterpret_cast<uint32_t*>(ring);
       sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
-      done = select_in_one_pass(sh, ring, rd, k, emit);
+      done = select_in_one_pass<DT>(sh, ring, rd, k, emit);
     }
   }
   if (!done) {

@@ -57,7 +57,7 @@ def test_bf16_chunks(k, outliers):
         assert (out["other"]["accept"] == 0).all()
 
 
-@pytest.mark.parametrize("k", [64, 2048])
+@pytest.mark.parametrize("k", [64, 1000, 2048])
 def test_fp32_chunks(k):
     S, T, H, L = 2, 64, 2048, 32
     act = synth.make_activations(S, T, H, torch.float32, seed=50 + k, device=DEV, outliers="jitter")
