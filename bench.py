@@ -422,7 +422,7 @@ def direct_commitments(tl, synth, dev, workload, reps=10):
     peak, peak_kind = measured_hbm_peak()
     nbytes = act.numel() * act.element_size()
     points = []
-    for k in (128, 512, 1024, 4096):
+    for k in (128, 512, 1024, 2048, 4096):
         lay, _ = tl.make_layout(act, L, k, S, T)
         commits, status = tl.toploc_commit_direct(act, lay)
         results, dev_bins = tl.toploc_verify_direct(rec, lay, commits)

@@ -8,7 +8,7 @@
 //   toploc_direct_verify_kernel<dtype, vector>   the same selection, then the comparison
 //
 // Selection of a chunk (both kernels), one of two ways:
-//   one pass (vector layouts; k <= 2048 for bf16, 1024 for fp32): the chunk is streamed once; elements that reach a
+//   one pass (vector layouts, k <= 2048): the chunk is streamed once; elements that reach a
 //   running threshold are kept as candidates in shared memory, in index order, and counted in a
 //   histogram of their upper 11 key bits, from which the threshold is raised as candidates
 //   arrive; the exact k-th key is then found among the candidates (select_in_one_pass);
@@ -73,11 +73,11 @@ struct DirectShared {
 };
 constexpr size_t kSpareBytes = 35264;
 constexpr size_t kSharedBytes = kRingBytes + sizeof(DirectShared) + kSpareBytes;
-// One-pass selection (vector layouts, k <= stream_max_k): a histogram of the upper 11 key bits
+// One-pass selection (vector layouts, k <= kStreamMaxK): a histogram of the upper 11 key bits
 // and up to cand_cap candidates (flat index, whole pattern) in index order.
 constexpr int kCoarseBins = 2048;
 __host__ __device__ constexpr int cand_cap(int dt) { return dt == 0 ? 26112 : 19712; }       // 6 / 8 bytes each
-__host__ __device__ constexpr int stream_max_k(int dt) { return dt == 0 ? 2048 : 1024; }
+constexpr int kStreamMaxK = 2048;   // beyond it the candidates of a 2^18-element chunk no longer fit
 static_assert(kSharedBytes <= 227 * 1024 && sizeof(DirectShared) % 16 == 0 && kSpareBytes % 16 == 0, "shared memory budget");
 static_assert(offsetof(DirectShared, hist) + sizeof(uint32_t) * kBins == sizeof(DirectShared), "hist is the last member");
 static_assert((size_t)kCoarseBins * 4 + (size_t)cand_cap(0) * 6 <= (size_t)kBins * 4 + kSpareBytes &&
@@ -564,7 +564,7 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
   };
   bool done = false;
   if constexpr (VECTOR) {
-    if (p.k <= stream_max_k(DT)) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
+    if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
   }
   if (!done) {
     uint32_t kth, take;
@@ -614,7 +614,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
   };
   bool done = false;
   if constexpr (VECTOR) {
-    if (k <= stream_max_k(DT)) {
+    if (k <= kStreamMaxK) {
       sel_idx = reinterpret_cast<uint32_t*>(ring);
       sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
       done = select_in_one_pass<DT>(sh, ring, rd, k, emit);
