@@ -397,7 +397,7 @@ __device__ void collect_in_index_order(DirectShared& sh, uint4* ring, const Read
 // arrived, the threshold is raised to the lowest key of the bin that holds the k-th largest
 // candidate so far -- a lower bound of the chunk's k-th largest key, so nothing of the top-k is
 // ever dropped.  The first batch (about 4k elements, threshold 0) seeds the histogram.  At the
-// end the exact k-th key is found among the candidates (digits of 8 bits, the last of 7) and the
+// end the exact k-th key is found among the candidates (the histogram, then the bits below) and the
 // top-k leaves in index order, ties to the lower index.  Returns false, having emitted nothing,
 // when the candidates outgrow their buffer (data sorted upwards, say): the caller then takes
 // the two-pass selection.
@@ -480,9 +480,13 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<D
   __syncthreads();
   if (overflow) return false;
 
-  // the exact k-th key among the candidates, 8 bits at a time from the top (the last digit has 7)
-  uint32_t kth = 0, known = 0, take = (uint32_t)k;
-  for (int shift = key_bits(DT) - 8, round = 0; shift > -8; shift -= 8, ++round) {
+  // The exact k-th key among the candidates: its upper 11 bits from the histogram that the
+  // stream kept (it counts every candidate), the bits below 8 at a time (the last digit has 4).
+  find_bin_from_top(sh, kCoarseBins, (uint32_t)k, 0);
+  uint32_t kth = sh.picked_bin << kCoarseShift, known = (uint32_t)(kCoarseBins - 1) << kCoarseShift;
+  uint32_t take = sh.picked_remaining;
+  __syncthreads();
+  for (int shift = kCoarseShift - 8, round = 1; shift > -8; shift -= 8, ++round) {
     const int low = shift < 0 ? 0 : shift, width = shift < 0 ? 8 + shift : 8;
     clear_bins(sh, 256);
     for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
