@@ -416,7 +416,7 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<D
   clear_bins(sh, kCoarseBins);
   int seed_groups = (4 * k > 2048 ? 4 * k : 2048) / R::VEC;
   if (seed_groups > rd.n_groups) seed_groups = rd.n_groups;
-  const uint32_t raise_step = (uint32_t)(k / 4 > 64 ? k / 4 : 64);
+  const uint32_t raise_step = (uint32_t)(k / 2 > 64 ? k / 2 : 64);
   uint32_t thr = 0, count = 0, last_raise = 0;
   int begin = 0, end = seed_groups, slot = 0;
   bool overflow = false;
