@@ -31,8 +31,8 @@ extern "C" {
 /* ---- constants -------------------------------------------------------- */
 
 /* Activation element types.  fp32 chunks are ranked on the full 31-bit
- * magnitude but commit only the upper 16 bits of each selected pattern (the
- * "fp32 mantissa scaled to match bf16" of Section 5.6), so proofs keep the
+ * magnitude but commit only the upper 16 bits of each selected pattern
+ * (Section 5.6 scales the fp32 mantissa down to bf16's), so proofs keep the
  * 2 + 2k byte size. */
 #define TOPLOC_DTYPE_BF16 0
 #define TOPLOC_DTYPE_FP32 1
@@ -45,7 +45,7 @@ extern "C" {
  * appendix names 2^32 as the modulus size for 32-bit types), coefficients take
  * 4 bytes little-endian and a proof 2 + 4k bytes.  Validation then compares
  * fp32 bit fields (sign, 8 exponent bits, 23 mantissa bits), which is what the
- * thresholds "for fp32 inference" of Section 5.2 (8 / 256 / 128) are stated
+ * fp32-inference thresholds of Section 5.2 (8 / 256 / 128) are stated
  * on.  The paper prints neither q nor this layout; they are this library's
  * reading. */
 #define TOPLOC_FIELD_16 0
@@ -55,8 +55,8 @@ extern "C" {
  * only: the proofs are TOPLOC_FIELD_16 proofs of a bf16 generator; the
  * polynomial is evaluated over Z_p, every committed 16-bit pattern is padded
  * with 16 zero bits and compared with the validator's whole fp32 pattern
- * (23-bit mantissas, the fp32 thresholds) -- the "bf16 model validated with
- * fp32" case of Section 5.6.  Proofs keep 2 + 2k bytes.  The generating entry
+ * (23-bit mantissas, the fp32 thresholds) -- the case of Section 5.6 in which
+ * a bf16 model is validated in fp32.  Proofs keep 2 + 2k bytes.  The generating entry
  * points return TOPLOC_ERR_UNSUPPORTED for it. */
 #define TOPLOC_FIELD_16_PADDED 2
 
@@ -251,8 +251,8 @@ int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_
 
 /*
  * Direct commitments.  Section 4 starts from the plain way of committing to a
- * chunk -- "storing top-k indices and values directly", 6 bytes per point: 4
- * for the index and 2 for the value -- before replacing it by the polynomial.
+ * chunk -- the top-k indices and values kept as they are, 6 bytes per point
+ * (4 for the index, 2 for the value) -- before replacing it by the polynomial.
  * These two entry points are that plain form.  It is three times the size,
  * but it exists for every k: with thousands of indices (the exponent-error
  * table of Section 3 goes up to k = 4096) no modulus below 2^16 separates

@@ -90,12 +90,13 @@ def mod_inverse_euclid(a, m):
     return int(lib().oracle_mod_inverse_euclid(ctypes.c_int64(a), ctypes.c_int64(m)))
 
 
-def interpolate(x, y, newton=False):
-    """Coefficients (ascending degree, uint16) of the polynomial through (x_j, y_j) over Z_p."""
+def interpolate(x, y, lagrange=False):
+    """Coefficients (ascending degree, uint16) of the polynomial through (x_j, y_j) over Z_p:
+    by elimination on the Vandermonde system, or (the second statement) by Lagrange's form."""
     x = np.ascontiguousarray(x, np.uint32)
     y = np.ascontiguousarray(y, np.uint32)
     c = np.zeros(len(x), np.uint16)
-    fn = lib().oracle_interpolate_newton if newton else lib().oracle_interpolate
+    fn = lib().oracle_interpolate_lagrange if lagrange else lib().oracle_interpolate
     if fn(_ptr(x), _ptr(y), len(x), _ptr(c)) != 0:
         raise ValueError("x values are not distinct mod p")
     return c
@@ -128,12 +129,12 @@ def mod_inverse32(a):
     return int(lib().oracle_mod_inverse32(ctypes.c_uint32(a)))
 
 
-def interpolate32(x, y, newton=False):
+def interpolate32(x, y, lagrange=False):
     """Coefficients (ascending degree, uint32) of the polynomial through (x_j, y_j) over Z_q."""
     x = np.ascontiguousarray(x, np.uint32)
     y = np.ascontiguousarray(y, np.uint32)
     c = np.zeros(len(x), np.uint32)
-    fn = lib().oracle_interpolate32_newton if newton else lib().oracle_interpolate32
+    fn = lib().oracle_interpolate32_lagrange if lagrange else lib().oracle_interpolate32
     if fn(_ptr(x), _ptr(y), len(x), _ptr(c)) != 0:
         raise ValueError("x values are not distinct mod q")
     return c
@@ -177,13 +178,13 @@ def num_chunks(num_seqs, tokens_per_seq, chunk_len, seq_offsets=None):
                                        None if so is None else _ptr(so), chunk_len))
 
 
-def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None, first_chunk=0,
-                 last_chunk=-1, want_indices=True, threads=None, wide=False):
+def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None, want_indices=True,
+                 threads=None, wide=False):
     """act: 2-D [total_tokens, hidden] host array (uint16 bf16 patterns or float32).
     wide: the 32-bit field variant (fp32 only; proofs of 2 + 4k bytes).
 
-    Returns (proofs uint8[n, 2+2k], status uint8[n], indices int32[n, k] or None), all indexed by
-    absolute chunk number; only rows first_chunk..last_chunk-1 are filled."""
+    Returns (proofs uint8[n, 2+2k], status uint8[n], indices int32[n, k] or None), chunks in
+    batch order."""
     assert act.ndim == 2 and act.strides[1] == act.itemsize
     hidden = act.shape[1]
     row_stride = act.strides[0] // act.itemsize
@@ -194,16 +195,17 @@ def build_proofs(act, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None
     indices = np.zeros((n, k), np.int32) if want_indices else None
     lib().oracle_build_proofs(
         _ptr(act), _batch_dtype_code(act, wide), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
-        None if so is None else _ptr(so), ctypes.c_int64(row_stride), ctypes.c_int64(first_chunk),
-        ctypes.c_int64(last_chunk), _ptr(proofs), _ptr(status),
+        None if so is None else _ptr(so), ctypes.c_int64(row_stride), _ptr(proofs), _ptr(status),
         None if indices is None else _ptr(indices), threads or default_threads())
     return proofs, status, indices
 
 
 def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_offsets=None,
                   t_exp=38, t_mean=10.0, t_median=8.0, sign_in_exponent=True, gen_indices=None,
-                  first_chunk=0, last_chunk=-1, threads=None, wide=False, padded=False):
+                  threads=None, wide=False, padded=False):
     """Returns a structured array (RESULT_DTYPE) with one entry per chunk.
+    t_exp / t_mean / t_median: one number for the whole batch, or an array with one entry per
+    chunk (thresholds chosen per generation, Section 6).
     padded: fp32 activations against 16-bit field proofs, the committed patterns padded with 16 zero
     bits and compared as fp32 (Section 5.6)."""
     assert act.ndim == 2 and act.strides[1] == act.itemsize
@@ -215,11 +217,23 @@ def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_off
     assert proofs.shape == (n, 2 + (4 if wide else 2) * k)
     gi = None if gen_indices is None else np.ascontiguousarray(gen_indices, np.int32)
     results = np.zeros(n, RESULT_DTYPE)
+
+    def each(value, dtype):
+        if np.ndim(value) == 0:
+            return value, None
+        arr = np.ascontiguousarray(value, dtype)
+        assert arr.shape == (n,)
+        return 0, arr
+
+    t_exp, exp_each = each(t_exp, np.int32)
+    t_mean, mean_each = each(t_mean, np.float64)
+    t_median, median_each = each(t_median, np.float64)
     lib().oracle_verify_proofs(
         _ptr(act), _batch_dtype_code(act, wide, padded), hidden, chunk_len, k, num_seqs, ctypes.c_int64(tokens_per_seq),
-        None if so is None else _ptr(so), ctypes.c_int64(row_stride), ctypes.c_int64(first_chunk),
-        ctypes.c_int64(last_chunk), _ptr(proofs), int(t_exp), ctypes.c_double(t_mean),
-        ctypes.c_double(t_median), int(bool(sign_in_exponent)), None if gi is None else _ptr(gi),
+        None if so is None else _ptr(so), ctypes.c_int64(row_stride), _ptr(proofs), int(t_exp),
+        ctypes.c_double(t_mean), ctypes.c_double(t_median), int(bool(sign_in_exponent)),
+        None if exp_each is None else _ptr(exp_each), None if mean_each is None else _ptr(mean_each),
+        None if median_each is None else _ptr(median_each), None if gi is None else _ptr(gi),
         _ptr(results), threads or default_threads())
     return results
 

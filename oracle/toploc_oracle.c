@@ -28,7 +28,7 @@
  *
  * Pins (tests/test_oracle_*.py): worked examples and the paper's printed
  * values under tests/golden/, brute force on tiny inputs, P(x_j) = y_j with
- * Python integers, exhaustive a * inverse(a) = 1, Newton (Algorithm 3) against
+ * Python integers, exhaustive a * inverse(a) = 1, Lagrange's form against
  * elimination, the modulus distribution of Table 11.  Unpinned: byte
  * compatibility with the upstream project's proofs (its code is not
  * available here) -- "parity unpinned" for that claim only.
@@ -39,7 +39,7 @@
 #include <string.h>
 
 #define P_FIELD 65521u /* largest prime below 2^16 */
-#define M_HIGH 65536u  /* Algorithm 6: "for i = 65536 downto 2^15 + 1" */
+#define M_HIGH 65536u  /* Algorithm 6 tries 65536 first and stops after 2^15 + 1 */
 #define M_LOW 32769u
 
 enum { ST_OK = 0, ST_NO_MODULUS = 1, ST_K_EXCEEDS = 2, ST_BAD_PROOF = 3, ST_NONFINITE = 4 };
@@ -58,7 +58,7 @@ typedef struct {
 } oracle_result;
 
 /* ------------------------------------------------------------------ */
-/* Section 5.3 "top-k magnitude elements"; Algorithm 1 step topk(h,k). */
+/* topk(h, k) of Algorithm 1; Section 5.3 ranks by magnitude. */
 /* ------------------------------------------------------------------ */
 
 typedef struct {
@@ -160,25 +160,34 @@ uint32_t oracle_mod_inverse(uint32_t a) {
   return result;
 }
 
-/* Algorithm 4 as an algorithm: extended Euclid on (a, m), Bezout coefficient
- * of a brought into [0, m).  Returns 0 when m <= 1; returns m (an impossible
- * inverse) when gcd(a, m) != 1, standing for the algorithm's "throw". */
+/* The inverse by the extended Euclidean method (the method of Algorithm 4),
+ * stated through the recursion  gcd(a, b) = gcd(b, a mod b):  if
+ * g = b s' + (a mod b) t'  then  g = a t' + b (s' - floor(a / b) t').
+ * bezout() returns g and the two cofactors. */
+static int64_t bezout(int64_t a, int64_t b, int64_t* s, int64_t* t) {
+  if (b == 0) {
+    *s = 1;
+    *t = 0;
+    return a;
+  }
+  int64_t s1, t1;
+  int64_t g = bezout(b, a % b, &s1, &t1);
+  *s = t1;
+  *t = s1 - (a / b) * t1;
+  return g;
+}
+
+/* Inverse of a modulo m in [0, m).  Returns 0 when m <= 1 (no ring to invert
+ * in) and m itself, an impossible inverse, when gcd(a, m) != 1: the two cases
+ * in which Algorithm 4 has nothing to return. */
 int64_t oracle_mod_inverse_euclid(int64_t a, int64_t m) {
   if (m <= 1) return 0;
-  int64_t r0 = a, r1 = m, s0 = 1, s1 = 0;
-  while (r1 != 0) {
-    int64_t q = r0 / r1;
-    int64_t r2 = r0 - q * r1;
-    r0 = r1;
-    r1 = r2;
-    int64_t s2 = s0 - q * s1;
-    s0 = s1;
-    s1 = s2;
-  }
-  if (r0 != 1) return m;
-  int64_t s = s0 % m;
-  if (s < 0) s += m;
-  return s;
+  int64_t s, t;
+  a %= m;
+  if (a < 0) a += m;
+  if (bezout(a, m, &s, &t) != 1) return m;
+  s %= m;
+  return s < 0 ? s + m : s;
 }
 
 /* Algorithm 5, Horner: c[0..k-1] ascending degree, result in [0, p). */
@@ -190,8 +199,8 @@ uint32_t oracle_horner(const uint16_t* c, int k, uint32_t x) {
 }
 
 /* ------------------------------------------------------------------ */
-/* Section 4: "there always exists a unique k-1-degree polynomial that  */
-/* goes through the points".  The interpolant is the solution of the   */
+/* Section 4 relies on the interpolant being unique: k points with     */
+/* distinct x fix one polynomial of degree below k.  It solves the     */
 /* Vandermonde system  sum_d c_d x_j^d = y_j  over Z_p; solved here by  */
 /* Gaussian elimination.  x must be pairwise distinct mod p.           */
 /* Returns 0 on success, 1 if the system is singular.                  */
@@ -246,40 +255,47 @@ int oracle_interpolate(const uint32_t* x, const uint32_t* y, int k, uint16_t* c)
   return 0;
 }
 
-/* Algorithm 3, Newton interpolation, kept beside the elimination above as a
- * second statement of the same polynomial (the two must agree because the
- * interpolant is unique).  Divided differences first, then the Newton form
- * a_0 + (x - x_0)(a_1 + (x - x_1)(...)) is multiplied out from the inside.
- * Inverses by the extended Euclidean routine (Algorithm 4). */
-int oracle_interpolate_newton(const uint32_t* x, const uint32_t* y, int k, uint16_t* c) {
-  uint32_t* dd = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
-  uint32_t* poly = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
-  for (int j = 0; j < k; ++j) dd[j] = y[j] % P_FIELD;
-  for (int level = 1; level < k; ++level)
-    for (int i = k - 1; i >= level; --i) {
-      uint32_t num = subp(dd[i], dd[i - 1]);
-      uint32_t den = subp(x[i] % P_FIELD, x[i - level] % P_FIELD);
-      int64_t inv = oracle_mod_inverse_euclid((int64_t)den, (int64_t)P_FIELD);
-      if (den == 0 || inv == (int64_t)P_FIELD) {
-        free(dd);
-        free(poly);
-        return 1;
-      }
-      dd[i] = mulp(num, (uint32_t)inv);
-    }
-  /* poly <- dd[k-1]; then for i = k-2..0: poly <- poly * (x - x_i) + dd[i] */
-  poly[0] = dd[k - 1];
-  int deg = 0;
-  for (int i = k - 2; i >= 0; --i) {
-    uint32_t neg_xi = subp(0, x[i] % P_FIELD);
-    for (int d = deg + 1; d >= 1; --d) poly[d] = addp(poly[d - 1], mulp(poly[d], neg_xi));
-    poly[0] = addp(mulp(poly[0], neg_xi), dd[i]);
-    ++deg;
+/* A second statement of the same polynomial, kept beside the elimination as a
+ * pin (the two must agree because the interpolant is unique, Section 4):
+ * Lagrange's form
+ *   P(x) = sum_j y_j L_j(x),   L_j(x) = prod_{i != j} (x - x_i) / (x_j - x_i).
+ * The master polynomial M(x) = prod_i (x - x_i) is multiplied out once; for
+ * every j the quotient Q_j = M / (x - x_j) comes from one synthetic division
+ * and the denominator is Q_j(x_j).  Inverses by the extended Euclidean routine.
+ * (The CUDA path uses Newton's divided differences, Algorithm 3: a third
+ * route to the same coefficients.)  Returns 1 if two x coincide mod p. */
+int oracle_interpolate_lagrange(const uint32_t* x, const uint32_t* y, int k, uint16_t* c) {
+  uint32_t* master = (uint32_t*)calloc((size_t)k + 1, sizeof(uint32_t));
+  uint32_t* quot = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+  uint32_t* sum = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+  int failed = 0;
+  master[0] = 1; /* the constant polynomial 1, then one factor (x - x_i) at a time */
+  for (int i = 0; i < k; ++i) {
+    uint32_t xi = x[i] % P_FIELD;
+    for (int d = i + 1; d >= 1; --d) master[d] = subp(master[d - 1], mulp(master[d], xi));
+    master[0] = subp(0, mulp(master[0], xi));
   }
-  for (int d = 0; d < k; ++d) c[d] = (uint16_t)poly[d];
-  free(dd);
-  free(poly);
-  return 0;
+  for (int j = 0; j < k && !failed; ++j) {
+    uint32_t xj = x[j] % P_FIELD;
+    /* M = (x - x_j) Q_j:  q_{k-1} = M_k,  q_{d-1} = M_d + x_j q_d */
+    quot[k - 1] = master[k];
+    for (int d = k - 1; d >= 1; --d) quot[d - 1] = addp(master[d], mulp(xj, quot[d]));
+    uint32_t den = 0; /* Q_j(x_j) = prod_{i != j} (x_j - x_i) */
+    for (int d = k - 1; d >= 0; --d) den = addp(mulp(den, xj), quot[d]);
+    int64_t inv = oracle_mod_inverse_euclid((int64_t)den, (int64_t)P_FIELD);
+    if (den == 0 || inv == (int64_t)P_FIELD) {
+      failed = 1;
+      break;
+    }
+    uint32_t w = mulp(y[j] % P_FIELD, (uint32_t)inv);
+    for (int d = 0; d < k; ++d) sum[d] = addp(sum[d], mulp(w, quot[d]));
+  }
+  if (!failed)
+    for (int d = 0; d < k; ++d) c[d] = (uint16_t)sum[d];
+  free(master);
+  free(quot);
+  free(sum);
+  return failed;
 }
 
 /* ------------------------------------------------------------------ */
@@ -337,7 +353,7 @@ int oracle_build_chunk(const void* chunk, int dtype, int rows, int hidden, int64
     } else {
       for (int j = 0; j < k; ++j) {
         xs[j] = (idx[j] % m) % P_FIELD;
-        ys[j] = (uint32_t)bits[j] % P_FIELD; /* "dd <- y mod M" */
+        ys[j] = (uint32_t)bits[j] % P_FIELD; /* Algorithm 3 reduces every y mod M first */
         if (bits[j] >= P_FIELD) status = ST_NONFINITE;
       }
       oracle_interpolate(xs, ys, k, coef);
@@ -432,10 +448,10 @@ void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int
 /* ================================================================== */
 /* 32-bit field variant: an fp32 chunk commits the full 32-bit pattern */
 /* of each selected value.  The paper uses it without printing its     */
-/* layout: Section 5.2 gives thresholds "for fp32 inference" (8 / 256 / */
+/* layout: Section 5.2 gives thresholds for fp32 inference (8 / 256 /   */
 /* 128, on 23-bit mantissas, cf. the fp32 rows of the precision table   */
-/* in Section 5.6), and the subroutines appendix names "2^32 for        */
-/* 32-bit types" as the size of the modulus.  Readings used here:      */
+/* in Section 5.6), and the subroutines appendix puts the modulus of   */
+/* 32-bit types at 2^32.  Readings used here:                          */
 /*   - field prime q = 4294967291 = 2^32 - 5, the largest prime below  */
 /*     2^32 (a prime that fits 4-byte coefficients, as p fits 2 bytes); */
 /*   - proof: the same 2 modulus bytes, then k coefficients of 4 bytes  */
@@ -521,35 +537,39 @@ int oracle_interpolate32(const uint32_t* x, const uint32_t* y, int k, uint32_t* 
   return 0;
 }
 
-/* Algorithm 3 over Z_q with the inverses of Algorithm 4: the second statement
- * of the same polynomial. */
-int oracle_interpolate32_newton(const uint32_t* x, const uint32_t* y, int k, uint32_t* c) {
-  uint32_t* dd = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
-  for (int j = 0; j < k; ++j) {
-    dd[j] = y[j] % Q_FIELD;
-    c[j] = 0;
+/* Lagrange's form over Z_q (see oracle_interpolate_lagrange): the second
+ * statement of the same polynomial. */
+int oracle_interpolate32_lagrange(const uint32_t* x, const uint32_t* y, int k, uint32_t* c) {
+  uint32_t* master = (uint32_t*)calloc((size_t)k + 1, sizeof(uint32_t));
+  uint32_t* quot = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+  uint32_t* sum = (uint32_t*)calloc((size_t)k, sizeof(uint32_t));
+  int failed = 0;
+  master[0] = 1;
+  for (int i = 0; i < k; ++i) {
+    uint32_t xi = x[i] % Q_FIELD;
+    for (int d = i + 1; d >= 1; --d) master[d] = subq(master[d - 1], mulq(master[d], xi));
+    master[0] = subq(0, mulq(master[0], xi));
   }
-  for (int level = 1; level < k; ++level)
-    for (int i = k - 1; i >= level; --i) {
-      uint32_t num = subq(dd[i], dd[i - 1]);
-      uint32_t den = subq(x[i] % Q_FIELD, x[i - level] % Q_FIELD);
-      int64_t inv = oracle_mod_inverse_euclid((int64_t)den, (int64_t)Q_FIELD);
-      if (den == 0 || inv == (int64_t)Q_FIELD) {
-        free(dd);
-        return 1;
-      }
-      dd[i] = mulq(num, (uint32_t)inv);
+  for (int j = 0; j < k && !failed; ++j) {
+    uint32_t xj = x[j] % Q_FIELD;
+    quot[k - 1] = master[k];
+    for (int d = k - 1; d >= 1; --d) quot[d - 1] = addq(master[d], mulq(xj, quot[d]));
+    uint32_t den = 0;
+    for (int d = k - 1; d >= 0; --d) den = addq(mulq(den, xj), quot[d]);
+    int64_t inv = oracle_mod_inverse_euclid((int64_t)den, (int64_t)Q_FIELD);
+    if (den == 0 || inv == (int64_t)Q_FIELD) {
+      failed = 1;
+      break;
     }
-  c[0] = dd[k - 1];
-  int deg = 0;
-  for (int i = k - 2; i >= 0; --i) {
-    uint32_t neg_xi = subq(0, x[i] % Q_FIELD);
-    for (int d = deg + 1; d >= 1; --d) c[d] = addq(c[d - 1], mulq(c[d], neg_xi));
-    c[0] = addq(mulq(c[0], neg_xi), dd[i]);
-    ++deg;
+    uint32_t w = mulq(y[j] % Q_FIELD, (uint32_t)inv);
+    for (int d = 0; d < k; ++d) sum[d] = addq(sum[d], mulq(w, quot[d]));
   }
-  free(dd);
-  return 0;
+  if (!failed)
+    for (int d = 0; d < k; ++d) c[d] = sum[d];
+  free(master);
+  free(quot);
+  free(sum);
+  return failed;
 }
 
 /* 2 + 4k bytes. */
@@ -695,8 +715,8 @@ void oracle_verify_chunk32(const void* chunk, int rows, int hidden, int64_t row_
 }
 
 /* Algorithm 2 for an fp32 validator against the proof of a bf16 generator
- * (Section 5.6: "when validating a bf16 decode model with fp32, we padded 16
- * zero bits to the bf16 representation").  The proof is an ordinary 16-bit
+ * (Section 5.6 validates a bf16 model in fp32 by widening each bf16 pattern
+ * with 16 zero bits).  The proof is an ordinary 16-bit
  * field proof; the validator ranks its fp32 chunk on the full magnitude,
  * evaluates the polynomial over Z_p, pads the committed 16-bit pattern with 16
  * zero bits and compares fp32 bit fields (23-bit mantissas), which is what the
@@ -767,7 +787,7 @@ void oracle_verify_chunk_padded(const void* chunk, int rows, int hidden, int64_t
 
 /* ================================================================== */
 /* Direct commitments: Section 4 opens with the plain alternative to   */
-/* the polynomial, "storing top-k indices and values directly", at 6   */
+/* the polynomial: keep the top-k indices and values as they are, at 6 */
 /* bytes per point (4 for the index, 2 for the value).  It is the only */
 /* form that exists for the larger k of the exponent-error table in    */
 /* Section 3 (k up to 4096): k indices below 2^16 residues collide for */
@@ -958,7 +978,7 @@ typedef struct {
   int dtype, hidden, k;
   int64_t row_stride;
   const chunk_span* spans;
-  int64_t first, last; /* chunk range [first, last) */
+  int64_t count; /* chunks of the batch */
   uint8_t* proofs;
   uint8_t* status;
   int32_t* indices;
@@ -967,6 +987,11 @@ typedef struct {
   oracle_result* results;
   int t_exp, sign_in_exponent;
   double t_mean, t_median;
+  /* optional, one entry per chunk (Section 6 suggests thresholds chosen per generation);
+   * where absent the scalars above hold for every chunk */
+  const int32_t* t_exp_each;
+  const double* t_mean_each;
+  const double* t_median_each;
 } job;
 
 static void* worker(void* arg) {
@@ -974,20 +999,23 @@ static void* worker(void* arg) {
   size_t esz = jb->dtype == 0 ? 2 : 4;
   int wide = jb->dtype == 2; /* fp32 chunks committed over Z_q */
   size_t pbytes = 2 + (wide ? 4 : 2) * (size_t)jb->k;
-  for (int64_t c = jb->first + jb->tid; c < jb->last; c += jb->nthreads) {
+  for (int64_t c = jb->tid; c < jb->count; c += jb->nthreads) {
     const void* chunk = jb->act + (size_t)jb->spans[c].row0 * (size_t)jb->row_stride * esz;
+    const int t_exp = jb->t_exp_each ? jb->t_exp_each[c] : jb->t_exp;
+    const double t_mean = jb->t_mean_each ? jb->t_mean_each[c] : jb->t_mean;
+    const double t_median = jb->t_median_each ? jb->t_median_each[c] : jb->t_median;
     if (!jb->verify && wide) {
       jb->status[c] = (uint8_t)oracle_build_chunk32(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
                                                     jb->proofs + (size_t)c * pbytes,
                                                     jb->indices ? jb->indices + (size_t)c * jb->k : NULL);
     } else if (jb->verify && jb->dtype == 3) {
       oracle_verify_chunk_padded(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
-                                 jb->proofs_in + (size_t)c * pbytes, jb->t_exp, jb->t_mean, jb->t_median,
+                                 jb->proofs_in + (size_t)c * pbytes, t_exp, t_mean, t_median,
                                  jb->sign_in_exponent,
                                  jb->gen_indices ? jb->gen_indices + (size_t)c * jb->k : NULL, &jb->results[c]);
     } else if (wide) {
       oracle_verify_chunk32(chunk, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
-                            jb->proofs_in + (size_t)c * pbytes, jb->t_exp, jb->t_mean, jb->t_median,
+                            jb->proofs_in + (size_t)c * pbytes, t_exp, t_mean, t_median,
                             jb->sign_in_exponent,
                             jb->gen_indices ? jb->gen_indices + (size_t)c * jb->k : NULL, &jb->results[c]);
     } else if (!jb->verify) {
@@ -997,7 +1025,7 @@ static void* worker(void* arg) {
       jb->status[c] = (uint8_t)st;
     } else {
       oracle_verify_chunk(chunk, jb->dtype, jb->spans[c].rows, jb->hidden, jb->row_stride, jb->k,
-                          jb->proofs_in + (size_t)c * pbytes, jb->t_exp, jb->t_mean, jb->t_median,
+                          jb->proofs_in + (size_t)c * pbytes, t_exp, t_mean, t_median,
                           jb->sign_in_exponent,
                           jb->gen_indices ? jb->gen_indices + (size_t)c * jb->k : NULL, &jb->results[c]);
     }
@@ -1021,11 +1049,10 @@ static int run_jobs(job* proto, int nthreads) {
   return 0;
 }
 
-/* Proofs for chunks [first_chunk, last_chunk) of the batch (last_chunk < 0:
- * all).  Outputs are indexed by absolute chunk number. */
+/* Proofs for every chunk of the batch, in batch order. */
 int oracle_build_proofs(const void* act, int dtype, int hidden, int chunk_len, int k, int num_seqs,
                         int64_t tokens_per_seq, const int64_t* seq_offsets, int64_t row_stride,
-                        int64_t first_chunk, int64_t last_chunk, uint8_t* proofs, uint8_t* status,
+                        uint8_t* proofs, uint8_t* status,
                         int32_t* indices_opt, int nthreads) {
   int64_t n = enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, NULL);
   chunk_span* spans = (chunk_span*)malloc((size_t)(n > 0 ? n : 1) * sizeof(chunk_span));
@@ -1038,8 +1065,7 @@ int oracle_build_proofs(const void* act, int dtype, int hidden, int chunk_len, i
   jb.k = k;
   jb.row_stride = row_stride;
   jb.spans = spans;
-  jb.first = first_chunk;
-  jb.last = last_chunk < 0 ? n : last_chunk;
+  jb.count = n;
   jb.proofs = proofs;
   jb.status = status;
   jb.indices = indices_opt;
@@ -1050,9 +1076,10 @@ int oracle_build_proofs(const void* act, int dtype, int hidden, int chunk_len, i
 
 int oracle_verify_proofs(const void* act, int dtype, int hidden, int chunk_len, int k, int num_seqs,
                          int64_t tokens_per_seq, const int64_t* seq_offsets, int64_t row_stride,
-                         int64_t first_chunk, int64_t last_chunk, const uint8_t* proofs, int t_exp,
-                         double t_mean, double t_median, int sign_in_exponent,
-                         const int32_t* gen_indices_opt, oracle_result* results, int nthreads) {
+                         const uint8_t* proofs, int t_exp, double t_mean, double t_median,
+                         int sign_in_exponent, const int32_t* t_exp_each_opt, const double* t_mean_each_opt,
+                         const double* t_median_each_opt, const int32_t* gen_indices_opt,
+                         oracle_result* results, int nthreads) {
   int64_t n = enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, NULL);
   chunk_span* spans = (chunk_span*)malloc((size_t)(n > 0 ? n : 1) * sizeof(chunk_span));
   enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, spans);
@@ -1065,8 +1092,7 @@ int oracle_verify_proofs(const void* act, int dtype, int hidden, int chunk_len, 
   jb.k = k;
   jb.row_stride = row_stride;
   jb.spans = spans;
-  jb.first = first_chunk;
-  jb.last = last_chunk < 0 ? n : last_chunk;
+  jb.count = n;
   jb.proofs_in = proofs;
   jb.gen_indices = gen_indices_opt;
   jb.results = results;
@@ -1074,6 +1100,9 @@ int oracle_verify_proofs(const void* act, int dtype, int hidden, int chunk_len, 
   jb.t_mean = t_mean;
   jb.t_median = t_median;
   jb.sign_in_exponent = sign_in_exponent;
+  jb.t_exp_each = t_exp_each_opt;
+  jb.t_mean_each = t_mean_each_opt;
+  jb.t_median_each = t_median_each_opt;
   run_jobs(&jb, nthreads);
   free(spans);
   return 0;

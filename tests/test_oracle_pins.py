@@ -216,9 +216,9 @@ def test_inverse_exhaustive():
 def test_euclid_inverse_agrees_and_handles_edge_cases():
     for a in list(range(1, 400)) + [P - 1, P - 2, 32768, 40000]:
         assert oracle.mod_inverse_euclid(a, P) == pow(a, -1, P)
-    assert oracle.mod_inverse_euclid(5, 1) == 0      # "no inverse when modulus is invalid"
+    assert oracle.mod_inverse_euclid(5, 1) == 0      # no ring to invert in
     assert oracle.mod_inverse_euclid(5, 0) == 0
-    assert oracle.mod_inverse_euclid(6, 9) == 9      # gcd 3: the routine's "throw" marker
+    assert oracle.mod_inverse_euclid(6, 9) == 9      # gcd 3: no inverse exists, reported as m
     assert oracle.mod_inverse_euclid(7, 40) == pow(7, -1, 40)
 
 
@@ -247,7 +247,7 @@ def test_interpolation_small_closed_forms():
     assert oracle.interpolate([x0, x1], [y0, y1]).tolist() == [icpt, slope]
 
 
-@pytest.mark.parametrize("k", [3, 16, 128, 256])
+@pytest.mark.parametrize("k", [3, 16, 128, 256, 512])
 def test_interpolant_passes_through_every_point(k):
     rng = np.random.default_rng(k)
     x = rng.choice(P, size=k, replace=False)
@@ -255,8 +255,8 @@ def test_interpolant_passes_through_every_point(k):
     c = oracle.interpolate(x, y)
     for xj, yj in zip(x.tolist(), y.tolist()):
         assert sum(int(cd) * pow(xj, d, P) for d, cd in enumerate(c)) % P == yj
-    # uniqueness: Newton's method (Algorithm 3) must give the same coefficients
-    assert oracle.interpolate(x, y, newton=True).tolist() == c.tolist()
+    # uniqueness: Lagrange's form must give the same coefficients
+    assert oracle.interpolate(x, y, lagrange=True).tolist() == c.tolist()
     # and the order of the points is irrelevant
     perm = rng.permutation(k)
     assert oracle.interpolate(x[perm], y[perm]).tolist() == c.tolist()
@@ -392,6 +392,51 @@ def test_nothing_matched_is_rejected():
     res = oracle.verify_proofs(staircase_chunk(base, signs=[1, 1, 1]), proofs, 1, 3, 1, 1, t_exp=100)[0]
     assert (res["exp_mismatch"], res["n_match"], res["accept"]) == (3, 0, 0)
     assert res["mant_mean"] == 0.0 and res["mant_median"] == 0.0
+
+
+def test_index_overlap_hand_cases():
+    """topk_mismatch = k - |generator indices ∩ validator indices| (Section 5.4), predicted by hand."""
+    k = 4
+    gen = np.zeros((1, 64), np.uint16)
+    for j in range(k):
+        gen[0, j] = (140 - j) << 7                    # the generator selects elements 0, 1, 2, 3
+    proofs, _, indices = oracle.build_proofs(gen, 1, k, 1, 1)
+    assert sorted(indices[0].tolist()) == [0, 1, 2, 3]
+    # the validator's element 3 falls to zero and element 40 rises: it selects 0, 1, 2, 40 -> one index differs
+    one_off = gen.copy()
+    one_off[0, 3] = 0
+    one_off[0, 40] = 137 << 7
+    res = oracle.verify_proofs(one_off, proofs, 1, k, 1, 1, gen_indices=indices)[0]
+    assert res["topk_mismatch"] == 1 and res["status"] == 0
+    # the validator's large values sit at 10 .. 13: no index in common -> k
+    moved = np.zeros((1, 64), np.uint16)
+    for j in range(k):
+        moved[0, 10 + j] = (140 - j) << 7
+    res = oracle.verify_proofs(moved, proofs, 1, k, 1, 1, gen_indices=indices)[0]
+    assert res["topk_mismatch"] == k
+    # generator indices given in another order: a set difference does not depend on it
+    res = oracle.verify_proofs(one_off, proofs, 1, k, 1, 1, gen_indices=indices[:, ::-1].copy())[0]
+    assert res["topk_mismatch"] == 1
+    # without generator indices there is nothing to compare
+    assert oracle.verify_proofs(one_off, proofs, 1, k, 1, 1)[0]["topk_mismatch"] == -1
+
+
+def test_thresholds_per_chunk():
+    """Thresholds given per chunk (Section 6: thresholds chosen per generation) decide each chunk by
+    its own entry; the statistics do not depend on them."""
+    base = [0] * 8
+    one = staircase_chunk(base)
+    gen = np.concatenate([one, one, one])             # three identical one-row chunks
+    proofs, _, _ = oracle.build_proofs(gen, 1, 8, 3, 1)
+    moved_one = staircase_chunk([4] * 8, signs=[1, 1, 0, 0, 0, 0, 0, 0])   # err_e 2, diffs all 4
+    moved = np.concatenate([moved_one, moved_one, moved_one])
+    res = oracle.verify_proofs(moved, proofs, 1, 8, 3, 1, t_exp=[2, 1, 2], t_mean=[4.0, 4.0, 3.5],
+                               t_median=[4.0, 4.0, 4.0])
+    assert res["accept"].tolist() == [1, 0, 0]
+    assert res["exp_mismatch"].tolist() == [2, 2, 2] and res["mant_mean"].tolist() == [4.0, 4.0, 4.0]
+    # scalars and arrays mix
+    res = oracle.verify_proofs(moved, proofs, 1, 8, 3, 1, t_exp=2, t_mean=4.0, t_median=[4.0, 3.5, 5.0])
+    assert res["accept"].tolist() == [1, 0, 1]
 
 
 def test_bad_proof_and_short_chunk_statuses():

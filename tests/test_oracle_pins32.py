@@ -29,7 +29,7 @@ def test_inverse_against_python_integers():
     for a in [1, 2, 3, Q - 1, Q - 2, 65521, 2 ** 31] + rng.integers(1, Q, 500).tolist():
         inv = oracle.mod_inverse32(int(a))
         assert 0 < inv < Q and (int(a) * inv) % Q == 1
-        assert oracle.mod_inverse_euclid(int(a), Q) == inv          # Algorithm 4 gives the same element
+        assert oracle.mod_inverse_euclid(int(a), Q) == inv          # the extended Euclidean method gives the same element
     assert oracle.mod_inverse32(Q - 1) == Q - 1                     # -1 is its own inverse
 
 
@@ -67,14 +67,14 @@ def test_interpolant_passes_through_every_point_and_both_methods_agree(k):
     assert c.dtype == np.uint32 and (c.astype(np.int64) < Q).all()
     for xj, yj in zip(x.tolist(), y.tolist()):
         assert poly_eval(c, xj) == yj
-    assert oracle.interpolate32(x, y, newton=True).tolist() == c.tolist()
+    assert oracle.interpolate32(x, y, lagrange=True).tolist() == c.tolist()
 
 
 def test_interpolation_rejects_repeated_x():
     with pytest.raises(ValueError):
         oracle.interpolate32([3, 8, 3], [1, 2, 3])
     with pytest.raises(ValueError):
-        oracle.interpolate32([3, 8, 3], [1, 2, 3], newton=True)
+        oracle.interpolate32([3, 8, 3], [1, 2, 3], lagrange=True)
 
 
 def test_encode_decode_layout():
