@@ -80,6 +80,8 @@ extern "C" {
 #define TOPLOC_ERR_CUDA (-4)              /* a CUDA runtime call or a launch failed */
 #define TOPLOC_ERR_ARCH (-5)              /* current device is not compute capability 10.x */
 #define TOPLOC_ERR_BUILTIN_SCRATCH (-6)   /* batch too large for toploc_build_proofs_builtin_scratch */
+#define TOPLOC_ERR_HOST_MEMORY (-7)       /* the host heap could not supply a row table (ragged batches,
+                                             long chunks) or the offsets of a *_host call */
 
 /* Size of the scratch buffer built into the library's device image (8 MiB):
  * enough for 10905 chunks at k = 128 (769 bytes each). */
@@ -201,8 +203,20 @@ const char* toploc_error_string(int return_code);
  *                       16-byte aligned; contents are undefined afterwards
  * cuda_stream   a cudaStream_t (NULL = default stream)
  *
+ * Alignment: d_act a multiple of the element size (2 or 4 bytes; 16-byte
+ * aligned rows take the vector path), d_proofs of 2, d_indices_opt of 4, else
+ * TOPLOC_ERR_INVALID_ARGUMENT -- nothing is launched with a pointer a kernel
+ * could not dereference.
+ *
  * Asynchronous: returns after enqueueing; results are valid once the stream
  * has been synchronised.  Returns TOPLOC_OK or a negative TOPLOC_ERR_*.
+ * Uniform batches of ordinary chunks do no other host work.  A ragged batch
+ * (seq_offsets != NULL) or one with a long chunk (more than 2^19 elements)
+ * needs a row table: the call builds it on the host heap -- work and memory
+ * proportional to the number of chunks (16 bytes per chunk or segment) --
+ * and hands it to the device with a copy from pageable memory, which blocks
+ * the calling thread until the bytes are staged; such a call cannot be
+ * captured into a CUDA graph.  TOPLOC_ERR_HOST_MEMORY if the heap is exhausted.
  */
 int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_proofs,
                         uint8_t* d_status, int32_t* d_indices_opt, void* d_workspace,
@@ -223,12 +237,43 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
  * d_results         DEVICE  out, [num_chunks] toploc_chunk_result
  * d_gen_indices_opt DEVICE  optional: the generator's [num_chunks, k] indices
  *                           (d_indices_opt of build) for topk_mismatch
- * other arguments as for toploc_build_proofs.
+ * other arguments as for toploc_build_proofs (d_results 8-byte aligned;
+ * thr->t_exp < 0 is refused).
  */
 int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint8_t* d_proofs,
                          const toploc_thresholds* thr, toploc_chunk_result* d_results,
                          const int32_t* d_gen_indices_opt, void* d_workspace,
                          size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same validation with one toploc_thresholds entry per chunk.  Section 6
+ * proposes acceptance thresholds chosen for the generation at hand (model,
+ * precision, sampling settings) instead of one global set; a batch that mixes
+ * generations then needs a threshold per chunk.  The statistics do not depend
+ * on the thresholds; only accept does (and the exponent comparison, through
+ * sign_in_exponent).
+ *
+ * d_thr_per_chunk  DEVICE  [num_chunks] toploc_thresholds, 8-byte aligned, read
+ *                          by the kernels (keep it alive until the stream has
+ *                          passed the call).  An entry with a negative t_exp
+ *                          rejects its chunk.
+ */
+int toploc_verify_proofs_per_chunk_thresholds(const void* d_act, const toploc_layout* lay,
+                                              const uint8_t* d_proofs,
+                                              const toploc_thresholds* d_thr_per_chunk,
+                                              toploc_chunk_result* d_results,
+                                              const int32_t* d_gen_indices_opt, void* d_workspace,
+                                              size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Thresholds of Section 5.2 for a proof of k points: 38 / 10 / 8 at k = 128
+ * for the 16-bit field (bf16, or fp32 scaled to 16 bits), 8 / 256 / 128 for
+ * fp32 bit fields (TOPLOC_FIELD_32, TOPLOC_FIELD_16_PADDED).  The paper states
+ * them at k = 128 only: the exponent threshold counts points and is scaled to
+ * floor(t * k / 128); mean and median are per-point statistics and stay.
+ * sign_in_exponent is set to 1.  thr HOST, out.  Host only, no CUDA calls.
+ */
+int toploc_default_thresholds(int32_t k, int32_t field, toploc_thresholds* thr);
 
 /*
  * The selection step on its own: topk(h, k) of Algorithms 1 and 2 for every
@@ -293,6 +338,12 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
 int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
                          const toploc_thresholds* thr, toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt,
                          void* cuda_stream);
+/* With one thresholds entry per chunk (DEVICE, [num_chunks]), as
+ * toploc_verify_proofs_per_chunk_thresholds. */
+int toploc_verify_direct_per_chunk_thresholds(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
+                                              const toploc_thresholds* d_thr_per_chunk,
+                                              toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt,
+                                              void* cuda_stream);
 
 /*
  * toploc_build_proofs for callers that have no way to hand over scratch

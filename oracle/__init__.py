@@ -267,7 +267,8 @@ def verify_direct(act, commits, chunk_len, k, num_seqs, tokens_per_seq=0, seq_of
                   t_exp=38, t_mean=10.0, t_median=8.0, sign_in_exponent=True):
     """Algorithm 2 against direct commitments.  Returns (results RESULT_DTYPE[n], exp_dev uint32[n, 9]):
     exp_dev counts, over the indices both sides selected, the exponent deviations 0, -1, +1, -2, +2,
-    -10..-3, 3..10, 11..99 and >= 100 in absolute value (the columns of the table in Section 3)."""
+    -10..-3, 3..10, 11..99 and >= 100 in absolute value (the columns of the table in Section 3).
+    t_exp / t_mean / t_median: one number for the batch or one entry per chunk."""
     assert act.ndim == 2 and act.strides[1] == act.itemsize
     hidden, row_stride, code = act.shape[1], act.strides[0] // act.itemsize, _dtype_code(act)
     spans = _chunk_spans(num_seqs, tokens_per_seq, chunk_len, seq_offsets)
@@ -275,9 +276,11 @@ def verify_direct(act, commits, chunk_len, k, num_seqs, tokens_per_seq=0, seq_of
     assert commits.shape == (len(spans), 6 * k)
     results = np.zeros(len(spans), RESULT_DTYPE)
     exp_dev = np.zeros((len(spans), 9), np.uint32)
+    pick = lambda v, c: v if np.ndim(v) == 0 else v[c]
     for c, (row0, rows) in enumerate(spans):
         lib().oracle_verify_direct_chunk(
-            _ptr(act[row0:]), code, rows, hidden, ctypes.c_int64(row_stride), k, _ptr(commits[c]), int(t_exp),
-            ctypes.c_double(t_mean), ctypes.c_double(t_median), int(bool(sign_in_exponent)),
+            _ptr(act[row0:]), code, rows, hidden, ctypes.c_int64(row_stride), k, _ptr(commits[c]),
+            int(pick(t_exp, c)), ctypes.c_double(pick(t_mean, c)), ctypes.c_double(pick(t_median, c)),
+            int(bool(sign_in_exponent)),
             _ptr(results[c:c + 1]), _ptr(exp_dev[c]))
     return results, exp_dev

@@ -423,7 +423,7 @@ void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int
       qsort(diffs, n, sizeof(uint32_t), ascending_u32);
       out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
     }
-    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    int reject = ((int64_t)err_e > (int64_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
     if (n == 0) reject = 1; /* nothing matched: no statistic to accept on */
     out->accept = reject ? 0 : 1;
     if (gen_indices_opt) {
@@ -692,7 +692,7 @@ void oracle_verify_chunk32(const void* chunk, int rows, int hidden, int64_t row_
       qsort(diffs, n, sizeof(uint32_t), ascending_u32);
       out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
     }
-    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    int reject = ((int64_t)err_e > (int64_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
     if (n == 0) reject = 1;
     out->accept = reject ? 0 : 1;
     if (gen_indices_opt) {
@@ -763,7 +763,7 @@ void oracle_verify_chunk_padded(const void* chunk, int rows, int hidden, int64_t
       qsort(diffs, n, sizeof(uint32_t), ascending_u32);
       out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
     }
-    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    int reject = ((int64_t)err_e > (int64_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
     if (n == 0) reject = 1;
     out->accept = reject ? 0 : 1;
     if (gen_indices_opt) {
@@ -924,7 +924,7 @@ void oracle_verify_direct_chunk(const void* chunk, int dtype, int rows, int hidd
       qsort(diffs, n, sizeof(uint32_t), ascending_u32);
       out->mant_median = (n & 1u) ? (double)diffs[n / 2] : ((double)diffs[n / 2 - 1] + (double)diffs[n / 2]) / 2.0;
     }
-    int reject = (err_e > (uint32_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
+    int reject = ((int64_t)err_e > (int64_t)t_exp) || (out->mant_mean > t_mean) || (out->mant_median > t_median);
     if (n == 0) reject = 1;
     out->accept = reject ? 0 : 1;
   } else {

@@ -20,6 +20,8 @@ __all__ = [
     "toploc_build_proofs", "toploc_verify_proofs", "toploc_build_proofs_host",
     "toploc_verify_proofs_host", "toploc_build_proofs_builtin_scratch", "TOPLOC_BUILTIN_SCRATCH_BYTES", "toploc_select_topk",
     "TOPLOC_MAX_K_DIRECT", "toploc_direct_commit_bytes", "toploc_commit_direct", "toploc_verify_direct",
+    "toploc_default_thresholds", "toploc_verify_proofs_per_chunk_thresholds",
+    "toploc_verify_direct_per_chunk_thresholds", "THRESHOLDS_DTYPE", "thresholds_tensor",
 ]
 
 TOPLOC_DTYPE_BF16 = 0
@@ -37,6 +39,10 @@ RESULT_DTYPE = np.dtype([
     ("mant_mean", "<f8"), ("mant_median", "<f8"), ("modulus", "<u4"),
     ("accept", "u1"), ("status", "u1"), ("pad", "u1", (2,)),
 ])
+
+
+# toploc_thresholds as a numpy record: the layout of one entry of a per-chunk threshold array
+THRESHOLDS_DTYPE = np.dtype([("t_exp", "<i4"), ("sign_in_exponent", "<i4"), ("t_mean", "<f8"), ("t_median", "<f8")])
 
 
 class ToplocError(RuntimeError):
@@ -112,6 +118,12 @@ def load_library():
     lib.toploc_commit_direct.argtypes = [vp, lay_p, vp, vp, vp]
     lib.toploc_verify_direct.restype = ctypes.c_int
     lib.toploc_verify_direct.argtypes = [vp, lay_p, vp, thr_p, vp, vp, vp]
+    lib.toploc_verify_proofs_per_chunk_thresholds.restype = ctypes.c_int
+    lib.toploc_verify_proofs_per_chunk_thresholds.argtypes = [vp, lay_p, vp, vp, vp, vp, vp, sz, vp]
+    lib.toploc_verify_direct_per_chunk_thresholds.restype = ctypes.c_int
+    lib.toploc_verify_direct_per_chunk_thresholds.argtypes = [vp, lay_p, vp, vp, vp, vp, vp]
+    lib.toploc_default_thresholds.restype = ctypes.c_int
+    lib.toploc_default_thresholds.argtypes = [i32, i32, thr_p]
     _LIB = lib
     return lib
 
@@ -265,20 +277,53 @@ def toploc_verify_proofs(act, lay, proofs, thresholds=None, results=None, gen_in
     return results
 
 
-def default_thresholds(k=128, sign_in_exponent=True, field=TOPLOC_FIELD_16):
-    """Section 5.2 thresholds: 38 / 10 / 8 at k = 128 for bf16 (and fp32 scaled to 16 bits), 8 / 256 / 128
-    for fp32 inference (TOPLOC_FIELD_32, 23-bit mantissas); the exponent threshold scales with k for
-    other proof sizes."""
+def toploc_default_thresholds(k=128, field=TOPLOC_FIELD_16):
+    """The library's default thresholds for a proof of k points (Section 5.2; see the header)."""
     thr = ToplocThresholds()
-    wide = field in (TOPLOC_FIELD_32, TOPLOC_FIELD_16_PADDED)
-    thr.t_exp = ((8 if wide else 38) * k) // 128
+    _check(load_library().toploc_default_thresholds(int(k), int(field), ctypes.byref(thr)), "toploc_default_thresholds")
+    return thr
+
+
+def default_thresholds(k=128, sign_in_exponent=True, field=TOPLOC_FIELD_16):
+    """toploc_default_thresholds with the sign-bit reading chosen by the caller."""
+    thr = toploc_default_thresholds(k, field)
     thr.sign_in_exponent = 1 if sign_in_exponent else 0
-    thr.t_mean = 256.0 if wide else 10.0
-    thr.t_median = 128.0 if wide else 8.0
     return thr
 
 
 __all__.append("default_thresholds")
+
+
+def thresholds_tensor(t_exp, t_mean, t_median, sign_in_exponent, device):
+    """Packs per-chunk thresholds (equal-length sequences) into a CUDA uint8 tensor laid out as
+    toploc_thresholds[n], for the *_per_chunk_thresholds entry points."""
+    n = len(t_exp)
+    rec = np.zeros(n, THRESHOLDS_DTYPE)
+    rec["t_exp"], rec["t_mean"], rec["t_median"] = t_exp, t_mean, t_median
+    rec["sign_in_exponent"] = sign_in_exponent
+    return torch.from_numpy(rec.view(np.uint8).reshape(n, THRESHOLDS_DTYPE.itemsize)).to(device)
+
+
+def toploc_verify_proofs_per_chunk_thresholds(act, lay, proofs, thresholds, results=None, gen_indices=None,
+                                              workspace=None, stream=None):
+    """toploc_verify_proofs with one toploc_thresholds entry per chunk: `thresholds` is a CUDA uint8
+    tensor [n, 24] (see thresholds_tensor).  Returns the results tensor [n, 40]."""
+    if not act.is_cuda or not thresholds.is_cuda:
+        raise ToplocError("toploc_verify_proofs_per_chunk_thresholds needs CUDA tensors")
+    n = toploc_num_chunks(lay)
+    dev = act.device
+    if results is None:
+        results = torch.empty((n, RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    assert proofs.is_contiguous() and proofs.numel() == n * toploc_layout_proof_bytes(lay)
+    assert thresholds.is_contiguous() and thresholds.numel() * thresholds.element_size() == n * THRESHOLDS_DTYPE.itemsize
+    assert results.is_contiguous() and results.numel() == n * RESULT_DTYPE.itemsize
+    workspace, wbytes = _workspace(lay, workspace, dev)
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_verify_proofs_per_chunk_thresholds(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(proofs), _dev_ptr(thresholds), _dev_ptr(results),
+            _dev_ptr(gen_indices), _dev_ptr(workspace), wbytes, _stream_ptr(stream))
+    _check(rc, "toploc_verify_proofs_per_chunk_thresholds")
+    return results
 
 
 def toploc_build_proofs_host(act, lay, proofs, status, staging, stream=None):
@@ -444,4 +489,24 @@ def toploc_verify_direct(act, lay, commits, thresholds=None, results=None, exp_d
                                                  ctypes.byref(thr), _dev_ptr(results), _dev_ptr(exp_dev),
                                                  _stream_ptr(stream))
     _check(rc, "toploc_verify_direct")
+    return results, exp_dev
+
+
+def toploc_verify_direct_per_chunk_thresholds(act, lay, commits, thresholds, results=None, exp_dev=None,
+                                              want_exp_dev=True, stream=None):
+    """toploc_verify_direct with one toploc_thresholds entry per chunk (CUDA uint8 tensor [n, 24])."""
+    if not act.is_cuda or not thresholds.is_cuda:
+        raise ToplocError("toploc_verify_direct_per_chunk_thresholds needs CUDA tensors")
+    n, dev = _direct_chunks(lay), act.device
+    if results is None:
+        results = torch.empty((n, RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    if exp_dev is None and want_exp_dev:
+        exp_dev = torch.empty((n, 9), dtype=torch.int32, device=dev)
+    assert commits.is_contiguous() and commits.numel() == n * 6 * lay.k
+    assert thresholds.is_contiguous() and thresholds.numel() * thresholds.element_size() == n * THRESHOLDS_DTYPE.itemsize
+    with torch.cuda.device(dev):
+        rc = load_library().toploc_verify_direct_per_chunk_thresholds(
+            _dev_ptr(act), ctypes.byref(lay), _dev_ptr(commits), _dev_ptr(thresholds), _dev_ptr(results),
+            _dev_ptr(exp_dev), _stream_ptr(stream))
+    _check(rc, "toploc_verify_direct_per_chunk_thresholds")
     return results, exp_dev

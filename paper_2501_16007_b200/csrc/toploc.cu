@@ -137,11 +137,21 @@ struct VerifyIo {
   const uint8_t* proofs;
   toploc_chunk_result* results;
   const int32_t* gen_indices;  // optional
-  int t_exp;
-  int sign_in_exponent;
-  double t_mean;
-  double t_median;
+  toploc_thresholds thr;              // thresholds of the call ...
+  const toploc_thresholds* thr_each;  // ... or, when not null, one entry per chunk (device memory)
 };
+
+// The thresholds chunk `chunk` is judged by.
+__device__ __forceinline__ toploc_thresholds thresholds_of(const VerifyIo& io, long long chunk) {
+  return io.thr_each ? io.thr_each[chunk] : io.thr;
+}
+
+// Algorithm 2's verdict: reject iff a statistic exceeds its threshold (strictly), or nothing matched.
+__device__ __forceinline__ bool rejects(const toploc_thresholds& t, const toploc_chunk_result& res) {
+  if (res.n_match == 0) return true;  // nothing matched: nothing to accept on
+  return ((long long)res.exp_mismatch > (long long)t.t_exp) || (res.mant_mean > t.t_mean) ||
+         (res.mant_median > t.t_median);
+}
 
 // A candidate is one 64-bit word whose unsigned order is the ranking order:
 // magnitude key (bit pattern without sign) descending, then flat index
@@ -1102,6 +1112,7 @@ __device__ __forceinline__ void evaluate_warp(SelectShared& sh, int k, long long
   uint32_t* coef = reinterpret_cast<uint32_t*>(sh.ring);  // kMaxK words
   uint32_t* gen = coef + kMaxK;                           // kMaxK words
   uint32_t* hist = sh.top_hist;                           // a 7-bit mantissa difference is at most 127
+  const toploc_thresholds thr = thresholds_of(io, chunk);
   warp_barrier();
   for (int d = lane; d < k; d += 32) coef[d] = proof[1 + d];
   if (io.gen_indices)
@@ -1130,7 +1141,7 @@ __device__ __forceinline__ void evaluate_warp(SelectShared& sh, int k, long long
     if (s * 32 + lane >= k) continue;
     const uint32_t seen = bits[s];
     uint32_t e_p = acc[s] >> 7, e_v = seen >> 7;  // sign + 8 exponent bits
-    if (!io.sign_in_exponent) {
+    if (!thr.sign_in_exponent) {
       e_p &= 0xFFu;
       e_v &= 0xFFu;
     }
@@ -1191,14 +1202,11 @@ __device__ __forceinline__ void evaluate_warp(SelectShared& sh, int k, long long
     res.n_match = n;
     res.mant_diff_sum = diff_sum;
     if (io.gen_indices) res.topk_mismatch = k - (int)common;
-    bool reject = true;  // nothing matched: nothing to accept on
     if (n > 0) {
       res.mant_mean = (double)diff_sum / (double)n;
       res.mant_median = ((double)lo_val + (double)hi_val) * 0.5;
-      reject = (res.exp_mismatch > (uint32_t)io.t_exp) || (res.mant_mean > io.t_mean) ||
-               (res.mant_median > io.t_median);
     }
-    res.accept = reject ? 0 : 1;
+    res.accept = rejects(thr, res) ? 0 : 1;
     io.results[chunk] = res;
   }
 }
@@ -1382,6 +1390,7 @@ __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long lo
   uint32_t* gen = coef + kMaxK;
   uint32_t* diffs = gen + kMaxK;
   constexpr uint32_t kNoMatch = 0xFFFFFFFFu;  // larger than any 23-bit difference
+  const toploc_thresholds thr = thresholds_of(io, chunk);
   warp_barrier();
   for (int d = lane; d < k; d += 32)
     coef[d] = PADDED ? (uint32_t)proof[1 + d] : ((uint32_t)proof[1 + 2 * d] | ((uint32_t)proof[2 + 2 * d] << 16));
@@ -1414,7 +1423,7 @@ __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long lo
     if (j >= k) continue;
     const uint32_t seen = pattern[s];
     uint32_t e_p = acc[s] >> 23, e_v = seen >> 23;  // sign + 8 exponent bits
-    if (!io.sign_in_exponent) {
+    if (!thr.sign_in_exponent) {
       e_p &= 0xFFu;
       e_v &= 0xFFu;
     }
@@ -1471,14 +1480,11 @@ __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long lo
     res.n_match = n;
     res.mant_diff_sum = diff_sum;
     if (io.gen_indices) res.topk_mismatch = k - (int)common;
-    bool reject = true;  // nothing matched: nothing to accept on
     if (n > 0) {
       res.mant_mean = (double)diff_sum / (double)n;
       res.mant_median = ((double)lo_val + (double)hi_val) * 0.5;
-      reject = (res.exp_mismatch > (uint32_t)io.t_exp) || (res.mant_mean > io.t_mean) ||
-               (res.mant_median > io.t_median);
     }
-    res.accept = reject ? 0 : 1;
+    res.accept = rejects(thr, res) ? 0 : 1;
     io.results[chunk] = res;
   }
 }
@@ -2033,6 +2039,11 @@ int pick_mode(const void* act, const toploc_layout* lay) {
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Pointers the kernels read or write with loads of their element size: an address that is not
+// a multiple of it would fault on the device, so it is refused on the host.
+bool misaligned(const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; }
+size_t element_bytes(const toploc_layout* lay) { return lay->dtype == TOPLOC_DTYPE_BF16 ? 2 : 4; }
+
 size_t coef_bytes_of(const toploc_layout* lay) { return lay->field == TOPLOC_FIELD_32 ? 4 : 2; }
 size_t proof_bytes_of(const toploc_layout* lay) { return 2 + coef_bytes_of(lay) * (size_t)lay->k; }
 
@@ -2086,7 +2097,7 @@ int upload_spans(const toploc_layout* lay, const HostPlan& plan, void* d_spans, 
   if (spans == nullptr || (plan.split && table == nullptr)) {
     free(spans);
     free(table);
-    return TOPLOC_ERR_INVALID_ARGUMENT;
+    return TOPLOC_ERR_HOST_MEMORY;
   }
   long long c = 0, g = 0;
   for (int s = 0; s < lay->num_seqs; ++s) {
@@ -2366,6 +2377,7 @@ const char* toploc_error_string(int rc) {
     case TOPLOC_ERR_WORKSPACE: return "workspace or staging buffer too small";
     case TOPLOC_ERR_CUDA: return "CUDA runtime error";
     case TOPLOC_ERR_ARCH: return "device is not compute capability 10.x";
+    case TOPLOC_ERR_HOST_MEMORY: return "out of host memory";
     case TOPLOC_ERR_BUILTIN_SCRATCH:
       return "batch needs more scratch than the library's built-in buffer holds (TOPLOC_BUILTIN_SCRATCH_BYTES)";
     default: return "unknown error";
@@ -2379,7 +2391,8 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
   int rc = plan_layout(lay, &plan);
   if (rc != TOPLOC_OK) return rc;
   if (d_act == nullptr || d_proofs == nullptr || d_status == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (reinterpret_cast<uintptr_t>(d_proofs) % 2 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (misaligned(d_proofs, 2) || misaligned(d_act, element_bytes(lay)) || misaligned(d_indices_opt, 4))
+    return TOPLOC_ERR_INVALID_ARGUMENT;
   if (lay->field == TOPLOC_FIELD_16_PADDED) return TOPLOC_ERR_UNSUPPORTED;  // a way to validate, not to commit
   if (plan.num_chunks == 0) return TOPLOC_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -2392,18 +2405,21 @@ int toploc_build_proofs(const void* d_act, const toploc_layout* lay, uint8_t* d_
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
-int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint8_t* d_proofs,
-                         const toploc_thresholds* thr, toploc_chunk_result* d_results,
-                         const int32_t* d_gen_indices_opt, void* d_workspace, size_t workspace_bytes,
-                         void* cuda_stream) {
+// Validation with the thresholds of the call (thr, host memory) or one entry per chunk
+// (d_thr_each, device memory); exactly one of the two is given.
+static int verify_proofs_with(const void* d_act, const toploc_layout* lay, const uint8_t* d_proofs,
+                              const toploc_thresholds* thr, const toploc_thresholds* d_thr_each,
+                              toploc_chunk_result* d_results, const int32_t* d_gen_indices_opt,
+                              void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
   HostPlan plan;
   int rc = plan_layout(lay, &plan);
   if (rc != TOPLOC_OK) return rc;
-  if (d_act == nullptr || d_proofs == nullptr || thr == nullptr || d_results == nullptr)
+  if (d_act == nullptr || d_proofs == nullptr || (thr == nullptr && d_thr_each == nullptr) || d_results == nullptr)
     return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (reinterpret_cast<uintptr_t>(d_proofs) % 2 != 0 || reinterpret_cast<uintptr_t>(d_results) % 8 != 0)
+  if (misaligned(d_proofs, 2) || misaligned(d_results, 8) || misaligned(d_act, element_bytes(lay)) ||
+      misaligned(d_gen_indices_opt, 4) || misaligned(d_thr_each, 8))
     return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (thr->t_exp < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (thr != nullptr && thr->t_exp < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (plan.num_chunks == 0) return TOPLOC_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   DeviceInfo* dev = nullptr;
@@ -2414,10 +2430,8 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   io.proofs = d_proofs;
   io.results = d_results;
   io.gen_indices = d_gen_indices_opt;
-  io.t_exp = thr->t_exp;
-  io.sign_in_exponent = thr->sign_in_exponent;
-  io.t_mean = thr->t_mean;
-  io.t_median = thr->t_median;
+  io.thr = thr ? *thr : toploc_thresholds{};
+  io.thr_each = d_thr_each;
   const int mode = pick_mode(d_act, lay);
   const bool bf16 = lay->dtype == TOPLOC_DTYPE_BF16;
   if (!plan.split) {
@@ -2434,6 +2448,38 @@ int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
+int toploc_verify_proofs(const void* d_act, const toploc_layout* lay, const uint8_t* d_proofs,
+                         const toploc_thresholds* thr, toploc_chunk_result* d_results,
+                         const int32_t* d_gen_indices_opt, void* d_workspace, size_t workspace_bytes,
+                         void* cuda_stream) {
+  if (thr == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  return verify_proofs_with(d_act, lay, d_proofs, thr, nullptr, d_results, d_gen_indices_opt, d_workspace,
+                            workspace_bytes, cuda_stream);
+}
+
+int toploc_verify_proofs_per_chunk_thresholds(const void* d_act, const toploc_layout* lay, const uint8_t* d_proofs,
+                                              const toploc_thresholds* d_thr_per_chunk,
+                                              toploc_chunk_result* d_results, const int32_t* d_gen_indices_opt,
+                                              void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (d_thr_per_chunk == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  return verify_proofs_with(d_act, lay, d_proofs, nullptr, d_thr_per_chunk, d_results, d_gen_indices_opt,
+                            d_workspace, workspace_bytes, cuda_stream);
+}
+
+int toploc_default_thresholds(int32_t k, int32_t field, toploc_thresholds* thr) {
+  if (thr == nullptr || k < 1) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (field != TOPLOC_FIELD_16 && field != TOPLOC_FIELD_32 && field != TOPLOC_FIELD_16_PADDED)
+    return TOPLOC_ERR_INVALID_ARGUMENT;
+  // Section 5.2 states 38 / 10 / 8 (bf16) and 8 / 256 / 128 (fp32) at k = 128.  The exponent
+  // threshold counts points and scales with k; mean and median are per-point statistics.
+  const bool fp32_fields = field != TOPLOC_FIELD_16;
+  thr->t_exp = (int32_t)(((long long)(fp32_fields ? 8 : 38) * k) / 128);
+  thr->sign_in_exponent = 1;
+  thr->t_mean = fp32_fields ? 256.0 : 10.0;
+  thr->t_median = fp32_fields ? 128.0 : 8.0;
+  return TOPLOC_OK;
+}
+
 int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_sel_indices,
                        uint16_t* d_sel_patterns, uint8_t* d_status, int32_t* d_ranked_indices_opt,
                        void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
@@ -2442,7 +2488,8 @@ int toploc_select_topk(const void* d_act, const toploc_layout* lay, uint32_t* d_
   if (rc != TOPLOC_OK) return rc;
   if (d_act == nullptr || d_sel_indices == nullptr || d_sel_patterns == nullptr || d_status == nullptr)
     return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (reinterpret_cast<uintptr_t>(d_sel_indices) % 4 != 0 || reinterpret_cast<uintptr_t>(d_sel_patterns) % 2 != 0)
+  if (misaligned(d_sel_indices, 4) || misaligned(d_sel_patterns, 2) || misaligned(d_act, element_bytes(lay)) ||
+      misaligned(d_ranked_indices_opt, 4))
     return TOPLOC_ERR_INVALID_ARGUMENT;
   if (lay->field != TOPLOC_FIELD_16) return TOPLOC_ERR_UNSUPPORTED;  // this entry point hands out 16-bit patterns
   if (plan.num_chunks == 0) return TOPLOC_OK;
@@ -2498,7 +2545,7 @@ int toploc_stream_append(const void* d_rows, const toploc_layout* lay, int32_t t
   if (rc != TOPLOC_OK) return rc;
   if (d_rows == nullptr || d_state == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
   if (token_in_chunk < 0 || token_in_chunk >= lay->chunk_len) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (reinterpret_cast<uintptr_t>(d_state) % 16 != 0) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (misaligned(d_state, 16) || misaligned(d_rows, element_bytes(lay))) return TOPLOC_ERR_INVALID_ARGUMENT;
   DeviceInfo* dev = nullptr;
   if ((rc = device_info(&dev)) != TOPLOC_OK) return rc;
   // rows that are 16-byte aligned are read as vectors, others element by element
@@ -2514,7 +2561,7 @@ int toploc_stream_finish(const void* d_state, const toploc_layout* lay, uint8_t*
   int rc = plan_stream(lay);
   if (rc != TOPLOC_OK) return rc;
   if (d_state == nullptr || d_proofs == nullptr || d_status == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if (reinterpret_cast<uintptr_t>(d_proofs) % 2 != 0 || reinterpret_cast<uintptr_t>(d_state) % 16 != 0)
+  if (misaligned(d_proofs, 2) || misaligned(d_state, 16) || misaligned(d_indices_opt, 4))
     return TOPLOC_ERR_INVALID_ARGUMENT;
   const WorkspacePlan wp = plan_workspace(false, lay->num_seqs, lay->k, lay->num_seqs, coef_bytes_of(lay));
   if (d_workspace == nullptr || workspace_bytes < wp.total) return TOPLOC_ERR_WORKSPACE;
@@ -2561,7 +2608,7 @@ static int run_from_host(bool verify, const void* h_act, const toploc_layout* la
   const size_t pb = proof_bytes_of(lay);
   char* stage = static_cast<char*>(d_staging);
   int64_t* rebased = static_cast<int64_t*>(malloc(((size_t)lay->num_seqs + 1) * sizeof(int64_t)));
-  if (rebased == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (rebased == nullptr) return TOPLOC_ERR_HOST_MEMORY;
   long long chunk0 = 0;
   int s0 = 0;
   while (s0 < lay->num_seqs && rc == TOPLOC_OK) {

@@ -54,10 +54,8 @@ struct DirectVerify {
   const uint8_t* commits;
   toploc_chunk_result* results;
   uint32_t* exp_dev;         // optional [num_chunks, 9]
-  int t_exp;
-  int sign_in_exponent;
-  double t_mean;
-  double t_median;
+  toploc_thresholds thr;              // thresholds of the call ...
+  const toploc_thresholds* thr_each;  // ... or, when not null, one entry per chunk (device memory)
 };
 
 // Dynamic shared memory of a block: the copy ring, this struct, and kSpareBytes that continue
@@ -656,6 +654,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
 
   // Algorithm 2 with a look-up in place of the polynomial
   uint32_t err_e = 0, n_match = 0, sum = 0, common = 0, dev[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  const int sign_in_exponent = io.thr_each ? io.thr_each[chunk].sign_in_exponent : io.thr.sign_in_exponent;
   for (int j = threadIdx.x; j < k; j += kThreads) {
     const uint32_t want = sel_idx[j];
     int lo = 0, hi = k;  // first committed index >= want
@@ -669,7 +668,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
     }
     ++common;
     const uint32_t committed = com_pat[lo], seen = sel_pat[j];
-    const uint32_t field = io.sign_in_exponent ? 0x1FFu : 0xFFu;
+    const uint32_t field = sign_in_exponent ? 0x1FFu : 0xFFu;
     if (((committed >> 7) & field) == ((seen >> 7) & field)) {
       const uint32_t mp = committed & 0x7Fu, mv = seen & 0x7Fu;
       const uint32_t d = mp > mv ? mp - mv : mv - mp;
@@ -708,7 +707,8 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
     r.n_match = sh.counters[1];
     r.mant_diff_sum = sh.counters[2];
     r.topk_mismatch = k - (int)sh.counters[3];
-    bool reject = r.exp_mismatch > (uint32_t)io.t_exp;
+    const toploc_thresholds thr = io.thr_each ? io.thr_each[chunk] : io.thr;
+    bool reject = (long long)r.exp_mismatch > (long long)thr.t_exp;
     if (r.n_match > 0) {
       r.mant_mean = nearest_ratio(r.mant_diff_sum, r.n_match);
       // values at sorted positions (n - 1) / 2 and n / 2
@@ -721,7 +721,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
         if (seen > hi_rank) hi_val = b;
       }
       r.mant_median = ((double)lo_val + (double)hi_val) * 0.5;
-      reject = reject || r.mant_mean > io.t_mean || r.mant_median > io.t_median;
+      reject = reject || r.mant_mean > thr.t_mean || r.mant_median > thr.t_median;
     } else {
       reject = true;  // nothing matched: no statistic to accept on
     }
@@ -810,26 +810,29 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
                      : launch_direct(toploc_direct_commit_kernel<1, false>, plan.num_chunks, smem, stream, p, d_commits, d_status);
 }
 
-int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
-                         const toploc_thresholds* thr, toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt,
-                         void* cuda_stream) {
+}  // extern "C"
+
+// Validation with the thresholds of the call (thr, host memory) or one entry per chunk
+// (d_thr_each, device memory); exactly one of the two is given.
+static int verify_direct_with(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
+                              const toploc_thresholds* thr, const toploc_thresholds* d_thr_each,
+                              toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt, void* cuda_stream) {
   DirectPlan plan;
   int rc = plan_direct(d_act, lay, &plan);
   if (rc != TOPLOC_OK) return rc;
-  if (d_commits == nullptr || thr == nullptr || d_results == nullptr ||
+  if (d_commits == nullptr || (thr == nullptr && d_thr_each == nullptr) || d_results == nullptr ||
       (reinterpret_cast<uintptr_t>(d_commits) & 1u) != 0 || (reinterpret_cast<uintptr_t>(d_results) & 7u) != 0 ||
-      (reinterpret_cast<uintptr_t>(d_exp_dev_opt) & 3u) != 0)
+      (reinterpret_cast<uintptr_t>(d_exp_dev_opt) & 3u) != 0 || (reinterpret_cast<uintptr_t>(d_thr_each) & 7u) != 0)
     return TOPLOC_ERR_INVALID_ARGUMENT;
+  if (thr != nullptr && thr->t_exp < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
   if ((rc = check_device()) != TOPLOC_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   DirectVerify io;
   io.commits = d_commits;
   io.results = d_results;
   io.exp_dev = d_exp_dev_opt;
-  io.t_exp = thr->t_exp;
-  io.sign_in_exponent = thr->sign_in_exponent;
-  io.t_mean = thr->t_mean;
-  io.t_median = thr->t_median;
+  io.thr = thr ? *thr : toploc_thresholds{};
+  io.thr_each = d_thr_each;
   const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
   if (lay->dtype == TOPLOC_DTYPE_BF16)
@@ -837,6 +840,23 @@ int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint
                        : launch_direct(toploc_direct_verify_kernel<0, false>, plan.num_chunks, smem, stream, p, io);
   return plan.vector ? launch_direct(toploc_direct_verify_kernel<1, true>, plan.num_chunks, smem, stream, p, io)
                      : launch_direct(toploc_direct_verify_kernel<1, false>, plan.num_chunks, smem, stream, p, io);
+}
+
+extern "C" {
+
+int toploc_verify_direct(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
+                         const toploc_thresholds* thr, toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt,
+                         void* cuda_stream) {
+  if (thr == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  return verify_direct_with(d_act, lay, d_commits, thr, nullptr, d_results, d_exp_dev_opt, cuda_stream);
+}
+
+int toploc_verify_direct_per_chunk_thresholds(const void* d_act, const toploc_layout* lay, const uint8_t* d_commits,
+                                              const toploc_thresholds* d_thr_per_chunk,
+                                              toploc_chunk_result* d_results, uint32_t* d_exp_dev_opt,
+                                              void* cuda_stream) {
+  if (d_thr_per_chunk == nullptr) return TOPLOC_ERR_INVALID_ARGUMENT;
+  return verify_direct_with(d_act, lay, d_commits, nullptr, d_thr_per_chunk, d_results, d_exp_dev_opt, cuda_stream);
 }
 
 }  // extern "C"

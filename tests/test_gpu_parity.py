@@ -265,54 +265,118 @@ def test_config_8b_decode_and_validation_sweep():
     assert not v["other_seed"]["accept"].any() and not v["prefix_shift"]["accept"].any()
 
 
-def test_config_70b_full_size_sampled():
-    """256 sequences x 4096 tokens, H = 8192 (~17 GB): generate and validate at full size in the
-    launch configuration the benchmark times; the oracle checks whole sampled sequences, and
-    properties that hold for every chunk are checked on all 32768."""
-    S, T, H = 256, 4096, 8192
+def full_size_70b_case(recipe, seed, sequences):
+    """Generates and validates the 70B-shaped batch (256 sequences x 4096 tokens, H = 8192, ~17 GB) in
+    one call each -- the launch configuration the benchmark times -- and compares the sequences
+    listed with the oracle chunk by chunk: proof bytes, statuses and indices of the build, every
+    statistic and verdict of the validation against an honest-noise copy.  The oracle receives
+    one sequence (64 MiB) at a time."""
+    S, T, H, L, k = 256, 4096, 8192, 32, 128
     free, _ = torch.cuda.mem_get_info()
     if free < 40 * 2 ** 30:
         pytest.skip("needs 40 GB of free device memory")
-    act = synth.make_activations(S, T, H, torch.bfloat16, seed=4, device=DEV)
-    g = gpu_build(act, 32, 128, S, T)
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=seed, device=DEV, outliers=recipe)
+    g = gpu_build(act, L, k, S, T)
     assert not g[1].any().item()
-    same = gpu_verify(act, g[0], 32, 128, S, T, gen_indices=g[2])
+    same = gpu_verify(act, g[0], L, k, S, T, gen_indices=g[2])
     assert same["accept"].all() and not same["exp_mismatch"].any() and not same["mant_diff_sum"].any()
-    assert (same["n_match"] == 128).all() and not same["topk_mismatch"].any()
+    assert (same["n_match"] == k).all() and not same["topk_mismatch"].any()
     assert ((same["modulus"] >= 32769) & (same["modulus"] <= 65536)).all()
-    noisy = synth.honest_noise(act, seed=5)
-    honest = gpu_verify(noisy, g[0], 32, 128, S, T, gen_indices=g[2])
-    cps = T // 32
-    for s in (0, 77, 255):
+    noisy = synth.honest_noise(act, seed=seed + 1)
+    honest = gpu_verify(noisy, g[0], L, k, S, T, gen_indices=g[2])
+    cps = T // L
+    for s in sequences:
         rows = slice(s * T, (s + 1) * T)
-        host = synth.host_patterns(act[rows])
-        r = oracle.build_proofs(host, 32, 128, 1, T)
-        sub = (g[0][s * cps:(s + 1) * cps], g[1][s * cps:(s + 1) * cps], g[2][s * cps:(s + 1) * cps])
-        assert_build_equal(sub, r, "70B seq %d" % s)
-        rv = oracle.verify_proofs(synth.host_patterns(noisy[rows]), r[0], 32, 128, 1, T, gen_indices=r[2],
-                                  **oracle_thresholds(128))
-        assert_results_equal(honest[s * cps:(s + 1) * cps], rv, "70B honest seq %d" % s)
+        r = oracle.build_proofs(synth.host_patterns(act[rows]), L, k, 1, T)
+        sub = tuple(t[s * cps:(s + 1) * cps] for t in g)
+        assert_build_equal(sub, r, "70B %s seq %d" % (recipe, s))
+        rv = oracle.verify_proofs(synth.host_patterns(noisy[rows]), r[0], L, k, 1, T, gen_indices=r[2],
+                                  **oracle_thresholds(k))
+        assert_results_equal(honest[s * cps:(s + 1) * cps], rv, "70B %s honest seq %d" % (recipe, s))
+    return g, honest
+
+
+def test_config_70b_full_size_every_chunk():
+    """The literal recipe (+-80 on eight fixed channels): all 32768 chunks against the oracle."""
+    full_size_70b_case("fixed", 4, range(256))
+
+
+@pytest.mark.parametrize("recipe", ["jitter", "none"])
+def test_config_70b_full_size_varied_selections(recipe):
+    """With +-80 outliers every chunk selects the same index set (the first 128 outliers); jittered
+    outlier magnitudes and plain heavy-tailed data make the selected set, the modulus and the
+    statistics differ from chunk to chunk.  Same full-size launches; sixteen whole sequences
+    (2048 chunks) against the oracle."""
+    g, honest = full_size_70b_case(recipe, 40 if recipe == "jitter" else 41, range(7, 256, 16))
+    distinct = {tuple(row) for row in g[2][:4096:64].cpu().numpy().tolist()}
+    assert len(distinct) > 32, "the selected index sets should vary from chunk to chunk"
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("hidden", [2048, 4096, 8192])
 def test_config_sweep(hidden, dtype):
-    """k in {32, 64, 128, 256} x chunk length in {16, 32, 64} at 128 sequences x 1024 tokens;
-    the GPU runs the full point, the oracle checks two whole sequences of it."""
+    """k in {32, 64, 128, 256} x chunk length in {16, 32, 64} at 128 sequences x 1024 tokens.  The
+    GPU runs every point in full.  The oracle checks every chunk of the corner points -- smallest
+    and largest k on the smallest and the largest chunk of each dtype -- and eight whole
+    sequences of every other point."""
     S, T = 128, 1024
     act = synth.make_activations(S, T, hidden, dtype, seed=50 + hidden // 1024, device=DEV)
     noisy = synth.honest_noise(act, seed=9)
+    host, host_noisy = synth.host_patterns(act), synth.host_patterns(noisy)
     for chunk_len in (16, 32, 64):
         cps = T // chunk_len
         for k in (32, 64, 128, 256):
             g = gpu_build(act, chunk_len, k, S, T)
             gv = gpu_verify(noisy, g[0], chunk_len, k, S, T, gen_indices=g[2])
-            for s in (1, 126):
-                rows = slice(s * T, (s + 1) * T)
-                r = oracle.build_proofs(synth.host_patterns(act[rows]), chunk_len, k, 1, T)
-                sub = tuple(t[s * cps:(s + 1) * cps] for t in g)
-                where = "sweep H%d L%d k%d %s seq %d" % (hidden, chunk_len, k, dtype, s)
-                assert_build_equal(sub, r, where)
-                rv = oracle.verify_proofs(synth.host_patterns(noisy[rows]), r[0], chunk_len, k, 1, T,
-                                          gen_indices=r[2], **oracle_thresholds(k))
-                assert_results_equal(gv[s * cps:(s + 1) * cps], rv, where)
+            corner = k in (32, 256) and (hidden, chunk_len) in ((2048, 16), (8192, 64))
+            seqs = list(range(S)) if corner else [1, 18, 35, 52, 69, 86, 103, 126]
+            # consecutive runs of sequences go to the oracle in one call
+            runs, start = [], seqs[0]
+            for a, b in zip(seqs, seqs[1:] + [None]):
+                if b != a + 1:
+                    runs.append((start, a + 1))
+                    start = b
+            for s0, s1 in runs:
+                rows, chunks = slice(s0 * T, s1 * T), slice(s0 * cps, s1 * cps)
+                r = oracle.build_proofs(host[rows], chunk_len, k, s1 - s0, T)
+                where = "sweep H%d L%d k%d %s seqs %d..%d" % (hidden, chunk_len, k, dtype, s0, s1 - 1)
+                assert_build_equal(tuple(t[chunks] for t in g), r, where)
+                rv = oracle.verify_proofs(host_noisy[rows], r[0], chunk_len, k, s1 - s0, T, gen_indices=r[2],
+                                          **oracle_thresholds(k))
+                assert_results_equal(gv[chunks], rv, where)
+
+
+def test_thresholds_per_chunk_decide_each_chunk_by_its_own_entry():
+    """Section 6: thresholds chosen per generation.  One call, a thresholds entry per chunk; the
+    statistics equal those of the single-threshold call, the verdicts follow each chunk's entry,
+    and both agree with the oracle given the same per-chunk thresholds."""
+    S, T, H, L, k = 4, 128, 2048, 32, 64
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=61, device=DEV, outliers="none")
+    noisy = synth.honest_noise(act, seed=62, rel=2.0 ** -6)          # coarse noise: statistics well above zero
+    lay, _ = tl.make_layout(act, L, k, S, T)
+    n = tl.toploc_num_chunks(lay)
+    g = gpu_build(act, L, k, S, T)
+    plain = gpu_verify(noisy, g[0], L, k, S, T, gen_indices=g[2])
+    assert plain["exp_mismatch"].max() > 0 and plain["mant_mean"].max() > 0
+    # chunk c is judged by: exponent threshold = its own mismatch count minus (c % 2), generous otherwise
+    t_exp = (plain["exp_mismatch"].astype(np.int64) - (np.arange(n) % 2)).astype(np.int32)
+    t_mean = np.where(np.arange(n) % 3 == 0, plain["mant_mean"] * 0.5, 1e9)
+    t_median = np.full(n, 1e9)
+    thr = tl.thresholds_tensor(t_exp, t_mean, t_median, 1, DEV)
+    res = tl.toploc_verify_proofs_per_chunk_thresholds(noisy, lay, g[0], thr, gen_indices=g[2])
+    torch.cuda.synchronize()
+    got = res.cpu().numpy().view(tl.RESULT_DTYPE).reshape(-1)
+    ref = oracle.verify_proofs(synth.host_patterns(noisy), g[0].cpu().numpy(), L, k, S, T, gen_indices=g[2].cpu().numpy(),
+                               t_exp=t_exp, t_mean=t_mean, t_median=t_median)
+    assert_results_equal(got, ref, "per-chunk thresholds")
+    for f in ("exp_mismatch", "n_match", "mant_diff_sum", "topk_mismatch"):
+        assert np.array_equal(got[f], plain[f])
+    assert 0 < got["accept"].sum() < n                                 # both verdicts occur in the one call
+    # the direct form takes the same array
+    commits, _ = tl.toploc_commit_direct(act, lay)
+    dres, _ = tl.toploc_verify_direct_per_chunk_thresholds(noisy, lay, commits, thr)
+    torch.cuda.synchronize()
+    dgot = dres.cpu().numpy().view(tl.RESULT_DTYPE).reshape(-1)
+    dref, _ = oracle.verify_direct(synth.host_patterns(noisy), commits.cpu().numpy(), L, k, S, T, t_exp=t_exp,
+                                   t_mean=t_mean, t_median=t_median)
+    assert_results_equal(dgot, dref, "per-chunk thresholds, direct")

@@ -138,3 +138,64 @@ def test_null_pointers_are_refused_before_any_cuda_call():
     assert lib.toploc_verify_proofs(None, ctypes.byref(lay), None, ctypes.byref(thr), None, None, None, 0,
                                     None) == -1
     assert lib.toploc_build_proofs_host(None, ctypes.byref(lay), None, None, None, 0, None) == -1
+
+
+def test_misaligned_pointers_are_refused_before_any_cuda_call():
+    """A pointer a kernel would dereference with 2- or 4-byte loads must be a multiple of that size;
+    the entry points say so with a return code instead of launching a kernel that would fault."""
+    lib = tl.load_library()
+    vp = ctypes.c_void_p
+    ok = 1 << 20                                        # a 16-byte aligned address (never dereferenced here)
+    bf16, fp32 = layout(), layout(dtype=1)
+    thr = tl.default_thresholds()
+
+    def build(act, lay, indices=None):
+        return lib.toploc_build_proofs(vp(act), ctypes.byref(lay), vp(ok), vp(ok), indices, vp(ok), 1 << 30, None)
+
+    def verify(act, lay, gen=None, results=ok):
+        return lib.toploc_verify_proofs(vp(act), ctypes.byref(lay), vp(ok), ctypes.byref(thr), vp(results), gen,
+                                        vp(ok), 1 << 30, None)
+
+    assert build(ok + 1, bf16) == -1 and build(ok + 2, fp32) == -1 and build(ok + 3, fp32) == -1
+    assert build(ok, bf16, vp(ok + 2)) == -1            # int32 indices at a 2-byte offset
+    assert verify(ok + 1, bf16) == -1 and verify(ok + 2, fp32) == -1
+    assert verify(ok, bf16, gen=vp(ok + 1)) == -1 and verify(ok, bf16, results=ok + 4) == -1
+    assert lib.toploc_select_topk(vp(ok + 1), ctypes.byref(bf16), vp(ok), vp(ok), vp(ok), None, vp(ok), 1 << 30,
+                                  None) == -1
+    assert lib.toploc_select_topk(vp(ok), ctypes.byref(bf16), vp(ok), vp(ok), vp(ok), vp(ok + 2), vp(ok), 1 << 30,
+                                  None) == -1
+    assert lib.toploc_stream_append(vp(ok + 1), ctypes.byref(bf16), 0, vp(ok), None) == -1
+    assert lib.toploc_stream_append(vp(ok + 2), ctypes.byref(fp32), 0, vp(ok), None) == -1
+    assert lib.toploc_stream_finish(vp(ok), ctypes.byref(bf16), vp(ok), vp(ok), vp(ok + 2), vp(ok), 1 << 30,
+                                    None) == -1
+    assert lib.toploc_verify_proofs_per_chunk_thresholds(vp(ok), ctypes.byref(bf16), vp(ok), vp(ok + 4), vp(ok),
+                                                         None, vp(ok), 1 << 30, None) == -1
+    assert lib.toploc_commit_direct(vp(ok + 1), ctypes.byref(layout(hidden=1001, row_stride=1001)), vp(ok), vp(ok),
+                                    None) == -1
+
+
+def test_default_thresholds_come_from_the_library():
+    t = tl.toploc_default_thresholds()
+    assert (t.t_exp, t.sign_in_exponent, t.t_mean, t.t_median) == (38, 1, 10.0, 8.0)      # Section 5.2, k = 128
+    assert [tl.toploc_default_thresholds(k).t_exp for k in (32, 64, 256, 512)] == [9, 19, 76, 152]
+    w = tl.toploc_default_thresholds(128, tl.TOPLOC_FIELD_32)
+    assert (w.t_exp, w.t_mean, w.t_median) == (8, 256.0, 128.0)
+    assert tl.toploc_default_thresholds(64, tl.TOPLOC_FIELD_16_PADDED).t_exp == 4
+    lib = tl.load_library()
+    assert lib.toploc_default_thresholds(0, 0, ctypes.byref(t)) == -1
+    assert lib.toploc_default_thresholds(128, 9, ctypes.byref(t)) == -1
+    assert lib.toploc_default_thresholds(128, 0, None) == -1
+    assert tl.THRESHOLDS_DTYPE.itemsize == ctypes.sizeof(tl.ToplocThresholds)
+
+
+def test_negative_exponent_threshold_is_refused_by_both_validators():
+    lib = tl.load_library()
+    vp = ctypes.c_void_p
+    ok = 1 << 20
+    lay = layout()
+    thr = tl.default_thresholds()
+    thr.t_exp = -1
+    assert lib.toploc_verify_proofs(vp(ok), ctypes.byref(lay), vp(ok), ctypes.byref(thr), vp(ok), None, vp(ok),
+                                    1 << 30, None) == -1
+    assert lib.toploc_verify_direct(vp(ok), ctypes.byref(lay), vp(ok), ctypes.byref(thr), vp(ok), None, None) == -1
+    assert "host memory" in tl.toploc_error_string(-7)

@@ -434,6 +434,9 @@ def test_thresholds_per_chunk():
                                t_median=[4.0, 4.0, 4.0])
     assert res["accept"].tolist() == [1, 0, 0]
     assert res["exp_mismatch"].tolist() == [2, 2, 2] and res["mant_mean"].tolist() == [4.0, 4.0, 4.0]
+    # the comparison is over the integers: a negative exponent threshold is exceeded by zero mismatches
+    res = oracle.verify_proofs(gen, proofs, 1, 8, 3, 1, t_exp=[-1, 0, 5])
+    assert res["exp_mismatch"].tolist() == [0, 0, 0] and res["accept"].tolist() == [0, 1, 1]
     # scalars and arrays mix
     res = oracle.verify_proofs(moved, proofs, 1, 8, 3, 1, t_exp=2, t_mean=4.0, t_median=[4.0, 3.5, 5.0])
     assert res["accept"].tolist() == [1, 0, 1]
