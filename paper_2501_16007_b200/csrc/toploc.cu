@@ -209,6 +209,14 @@ __device__ __forceinline__ uint4 load_streaming(const uint4* p) {
 __device__ __forceinline__ void copy_async_16(uint32_t smem_dst, const void* gmem_src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
+// Programmatic dependent launch.  A kernel that is followed in its stream by the interpolation
+// kernel lets that grid be scheduled early (its blocks need an SM almost to themselves, so they
+// only land where this grid has drained); the interpolation kernel builds its table of inverses
+// and then waits here until the whole grid before it has finished and its writes are visible.
+// Without a dependent launch behind it (or before it) both are no-ops.
+__device__ __forceinline__ void allow_dependent_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void wait_for_previous_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void copy_async_wait() {
@@ -847,6 +855,7 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
   const int k = bp.k;
   uint16_t* proof = sel.proofs ? reinterpret_cast<uint16_t*>(sel.proofs + chunk * proof_stride(bp)) : nullptr;
   int32_t* indices = sel.indices ? sel.indices + chunk * k : nullptr;
+  allow_dependent_launch();
 
   const ChunkPlace pl = locate_chunk<DT>(bp, chunk);
   const long long n_elems = (long long)pl.rows * bp.hidden;
@@ -930,27 +939,32 @@ __device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchP
 
 // Algorithm 3 for NCH chunks of one warp at a time (their dependency chains are
 // independent, which keeps the issue slots filled).  inv[] is the table of
-// inverses in Z_p; xa is this warp's scratch (NCH rows of kMaxK words: x_j in the
-// lower half of word j, the Newton coefficient a_j in the upper half).  A chunk
+// inverses in Z_p; xa is this warp's scratch (NCH rows of kMaxK words: x_i in the
+// lower half of word i, the Newton coefficient a_i in the upper half).  A chunk
 // that is not live is carried along with zeros and not written.
 //
-// Divided differences are taken point by point instead of level by level (the
-// same table, visited row-wise): with a_0 = y_0, step i lets every later point j
-// do  t_j <- (t_j - a_i) / (x_j - x_i), after which t_{i+1} is the Newton
-// coefficient a_{i+1}.  All points advance together and only a_i and x_i are
-// broadcast, so no value has to travel between neighbouring entries.  Point j
-// lives in lane j % 32, slot j / 32.
+// The Newton coefficients are the divided differences of Algorithm 3, reached
+// without a division per pair of points: with P_{i-1} the interpolant of the
+// first i points and N_i(x) = prod_{l < i} (x - x_l),
+//   a_i = (y_i - P_{i-1}(x_i)) / N_i(x_i).
+// Every point j carries t_j = y_j - P_{i-1}(x_j) and n_j = N_i(x_j); step i takes
+// a_i = t_i / n_i from point i (ONE look-up in the table of inverses, at an
+// address the whole warp shares, so it is a broadcast and not a gather) and
+// every later point does  t_j <- t_j - a_i n_j,  n_j <- n_j (x_j - x_i).  Point j
+// lives in lane j % 32, slot j / 32; only a_i and x_i travel between lanes.
+// (One division per pair, t_j <- (t_j - a_i) / (x_j - x_i), costs the same
+// arithmetic but k^2 / 2 gathers from the table per chunk; their bank conflicts
+// made shared memory the bottleneck: 0.47 ms per launch on the 70B-shaped batch
+// against 0.39 ms this way, which is bound by the integer-multiply pipe.)
 // The Newton form is then multiplied out from the inside,
-//   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0,
-// with coefficient d in lane d / SLOTS, slot d % SLOTS, so that the shift by one
-// degree stays inside a lane except for one value per lane and step.
+//   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0.
 template <int SLOTS, int NCH>
 __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t* xa, int k, const Selection& sel,
                                                    const long long (&chunk)[NCH], const bool (&live)[NCH]) {
   const int lane = threadIdx.x & 31;
-  uint16_t* a_half = reinterpret_cast<uint16_t*>(xa) + 1;  // the upper half of word j: a_j
+  constexpr uint32_t kFull = 0xFFFFFFFFu;
   const size_t proof_bytes = 2 + 2 * (size_t)k;
-  uint32_t x[NCH][SLOTS], t[NCH][SLOTS];
+  uint32_t x[NCH][SLOTS], t[NCH][SLOTS], n[NCH][SLOTS];
 #pragma unroll
   for (int c = 0; c < NCH; ++c) {
     uint32_t m = 65536u;
@@ -963,56 +977,60 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t
       const int j = s * 32 + lane;
       x[c][s] = 0;
       t[c][s] = 0;
-      if (j < k) {
-        uint32_t r = 0, y = 0;
-        if (live[c]) {
-          r = sel.idx[chunk[c] * k + j] % m;  // i_m = i mod m, then into Z_p
-          if (r >= kPrime) r -= kPrime;
-          y = sel.bits[chunk[c] * k + j];     // "dd <- y mod M"
-          if (y >= kPrime) y -= kPrime;
-        }
+      n[c][s] = 1;
+      if (j < k && live[c]) {
+        uint32_t r = sel.idx[chunk[c] * k + j] % m;  // i_m = i mod m, then into Z_p
+        if (r >= kPrime) r -= kPrime;
+        uint32_t y = sel.bits[chunk[c] * k + j];     // Algorithm 3 starts from y mod M
+        if (y >= kPrime) y -= kPrime;
         x[c][s] = r;
         t[c][s] = y;
-        xa[c * kMaxK + j] = r | (j == 0 ? y << 16 : 0u);  // x_j below, a_j above (a_0 = y_0; the others follow)
       }
     }
   }
   // Steps i = 32 b + ii: the points of slot b in lanes above ii and every point of the later
-  // slots take part (no per-slot tests inside the loop); x_i and a_i come as one word.
+  // slots take part (no per-slot tests inside the loop).
 #pragma unroll
   for (int b = 0; b < SLOTS; ++b) {
-    const int steps = min(32, k - 1 - 32 * b);
+    const int steps = min(32, k - 32 * b);  // the last point only yields its coefficient
 #pragma unroll 1
     for (int ii = 0; ii < steps; ++ii) {
       const int i = 32 * b + ii;
-      __syncwarp();  // a_i has been stored
       uint32_t neg_a[NCH], neg_x[NCH];
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
-        const uint32_t pair = xa[c * kMaxK + i];
-        neg_x[c] = kPrime - (pair & 0xFFFFu);
-        neg_a[c] = kPrime - (pair >> 16);
+        const uint32_t ni = __shfl_sync(kFull, n[c][b], ii);
+        const uint32_t ti = __shfl_sync(kFull, t[c][b], ii);
+        const uint32_t xi = __shfl_sync(kFull, x[c][b], ii);
+        const uint32_t a = mul_mod(ti, inv[ni]);  // n_i != 0: the x are distinct (Algorithm 6)
+        if (lane == 0) xa[c * kMaxK + i] = xi | (a << 16);
+        neg_a[c] = kPrime - a;
+        neg_x[c] = kPrime - xi;
       }
+      const bool later = lane > ii;
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
-        // a point at or before i computes a value that is dropped (its span indexes the table all the same)
-        const uint32_t next = mul_mod(diff_mod(t[c][b], neg_a[c]), inv[diff_mod(x[c][b], neg_x[c])]);
-        t[c][b] = lane > ii ? next : t[c][b];
-        if (lane == ii + 1) a_half[2 * (c * kMaxK + i + 1)] = (uint16_t)next;
+        // a point at or before i computes values that are dropped
+        const uint32_t tb = mad_mod(neg_a[c], n[c][b], t[c][b]);
+        const uint32_t nb = mul_mod(n[c][b], diff_mod(x[c][b], neg_x[c]));
+        t[c][b] = later ? tb : t[c][b];
+        n[c][b] = later ? nb : n[c][b];
       }
 #pragma unroll
       for (int s = b + 1; s < SLOTS; ++s) {
 #pragma unroll
-        for (int c = 0; c < NCH; ++c)
-          t[c][s] = mul_mod(diff_mod(t[c][s], neg_a[c]), inv[diff_mod(x[c][s], neg_x[c])]);
-      }
-      if (b + 1 < SLOTS && ii == 31 && lane == 0) {  // the next coefficient belongs to the next slot
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) a_half[2 * (c * kMaxK + i + 1)] = (uint16_t)t[c][b + 1 < SLOTS ? b + 1 : b];
+        for (int c = 0; c < NCH; ++c) {
+          t[c][s] = mad_mod(neg_a[c], n[c][s], t[c][s]);
+          n[c][s] = mul_mod(n[c][s], diff_mod(x[c][s], neg_x[c]));
+        }
       }
     }
   }
   __syncwarp();
+  // The Newton form multiplied out from the inside; after the step for x_i the polynomial has
+  // degree D = k - 1 - i.  Coefficient d lives in lane d % 32, slot d / 32: slots above D / 32
+  // hold zeros and are skipped, and the shift by one degree is a rotation of every live slot by
+  // one lane (lane 0 of a slot takes lane 31 of the slot below, lane 0 of slot 0 takes a_i).
   uint32_t co[NCH][SLOTS];
 #pragma unroll
   for (int c = 0; c < NCH; ++c) {
@@ -1020,18 +1038,25 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t
     for (int b = 0; b < SLOTS; ++b) co[c][b] = 0;
     if (lane == 0) co[c][0] = xa[c * kMaxK + k - 1] >> 16;
   }
+  const int from = (lane + 31) & 31;
+#pragma unroll
+  for (int top = 0; top < SLOTS; ++top) {  // the slot that holds the leading coefficient
+    const int d_first = max(32 * top, 1), d_last = min(32 * top + 31, k - 1);
 #pragma unroll 1
-  for (int i = k - 2; i >= 0; --i) {
+    for (int D = d_first; D <= d_last; ++D) {
+      const int i = k - 1 - D;
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      const uint32_t pair = xa[c * kMaxK + i];
-      const uint32_t neg_x = kPrime - (pair & 0xFFFFu);  // p for x_i = 0, which multiplies like 0
-      // coefficient d takes  c[d-1] + (-x_i) c[d];  entries above the current degree are 0 and stay 0
-      uint32_t carry = __shfl_up_sync(0xFFFFFFFFu, co[c][SLOTS - 1], 1);
-      if (lane == 0) carry = pair >> 16;  // a_i
+      for (int c = 0; c < NCH; ++c) {
+        const uint32_t pair = xa[c * kMaxK + i];
+        const uint32_t neg_x = kPrime - (pair & 0xFFFFu);  // p for x_i = 0, which multiplies like 0
+        uint32_t below[SLOTS];  // coefficient d - 1, as seen from the owner of coefficient d
 #pragma unroll
-      for (int b = SLOTS - 1; b >= 1; --b) co[c][b] = mad_mod(co[c][b], neg_x, co[c][b - 1]);
-      co[c][0] = mad_mod(co[c][0], neg_x, carry);
+        for (int b = 0; b <= top; ++b) below[b] = __shfl_sync(kFull, co[c][b], from);
+        // coefficient d takes  c[d-1] + (-x_i) c[d]
+#pragma unroll
+        for (int b = top; b >= 1; --b) co[c][b] = mad_mod(co[c][b], neg_x, lane == 0 ? below[b - 1] : below[b]);
+        co[c][0] = mad_mod(co[c][0], neg_x, lane == 0 ? (pair >> 16) : below[0]);
+      }
     }
   }
   // proof bytes 2 + 2d, 3 + 2d: coefficient of degree d, little-endian
@@ -1041,7 +1066,7 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t
     uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk[c] * proof_bytes);
 #pragma unroll
     for (int b = 0; b < SLOTS; ++b) {
-      const int d = lane * SLOTS + b;
+      const int d = b * 32 + lane;
       if (d < k) proof[1 + d] = (uint16_t)co[c][b];
     }
   }
@@ -1073,6 +1098,7 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
     }
   }
   __syncthreads();
+  wait_for_previous_grid();  // the selections and moduli are in place
   uint32_t* xa = reinterpret_cast<uint32_t*>(scratch) + warp * kInterpChunks * kMaxK;
   const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
   // group g goes to block g % gridDim.x, so a small batch spreads over the blocks before it fills their warps
@@ -1095,7 +1121,15 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
     if (k <= 32) interpolate_chunks<1, kInterpChunks>(inv, xa, k, sel, chunk, live);
     else if (k <= 64) interpolate_chunks<2, kInterpChunks>(inv, xa, k, sel, chunk, live);
     else if (k <= 128) interpolate_chunks<4, kInterpChunks>(inv, xa, k, sel, chunk, live);
-    else interpolate_chunks<kMaxSlots, kInterpChunks>(inv, xa, k, sel, chunk, live);
+    else {
+      // eight slots per lane: one chunk at a time keeps the state in registers
+#pragma unroll
+      for (int c = 0; c < kInterpChunks; ++c) {
+        const long long one_chunk[1] = {chunk[c]};
+        const bool one_live[1] = {live[c]};
+        if (live[c]) interpolate_chunks<kMaxSlots, 1>(inv, xa, k, sel, one_chunk, one_live);
+      }
+    }
   }
 }
 
@@ -2314,8 +2348,17 @@ void launch_interpolation(const toploc_layout* lay, const DeviceInfo* dev, const
   const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
   long long blocks = (groups + 3) / 4;
   if (blocks > dev->sms) blocks = dev->sms;
-  toploc_interpolate_kernel<<<(unsigned)blocks, kInterpWarps * 32, interp_smem_bytes(), stream>>>(sel, lay->k,
-                                                                                                 num_chunks);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks);
+  cfg.blockDim = dim3(kInterpWarps * 32);
+  cfg.dynamicSmemBytes = interp_smem_bytes();
+  cfg.stream = stream;
+  cudaLaunchAttribute early[1];
+  early[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see wait_for_previous_grid()
+  early[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = early;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, toploc_interpolate_kernel, sel, lay->k, num_chunks);
 }
 
 }  // namespace
