@@ -405,10 +405,43 @@ def decode_steps(tl, synth, dev, reps=20):
         tl.toploc_build_proofs(act, blay, ref_proofs, status, workspace=bws)
     b1.record()
     torch.cuda.synchronize()
+    # The producer-side hook: the final RMSNorm of the decode step, alone, and with the commitment
+    # taken from its output tile while that is still in shared memory (toploc_rmsnorm_append).
+    weight = torch.ones(H, dtype=torch.bfloat16, device=dev)
+    y = torch.empty_like(steps[0])
+
+    def timed_steps(fn):
+        """Mean time of one decode step over whole 32-token intervals (each starts an empty chunk)."""
+        def interval_of(fn):
+            tl.toploc_stream_begin(state, lay)
+            for t in range(L):
+                fn(t)
+        interval_of(fn)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            interval_of(fn)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / (reps * L) * 1e3
+
+    norm_alone = timed_steps(lambda t: tl.toploc_rmsnorm_append(steps[t], weight, 1e-5, lay, t, y, None))
+    norm_fused = timed_steps(lambda t: tl.toploc_rmsnorm_append(steps[t], weight, 1e-5, lay, t, y, state))
+
+    def norm_then_append(t):
+        tl.toploc_rmsnorm_append(steps[t], weight, 1e-5, lay, t, y, None)
+        tl.toploc_stream_append(y, lay, t, state)
+
+    norm_separate = timed_steps(norm_then_append)
     return {"metric": "incremental_proof_generation", "sequences": S, "hidden": H, "interval_tokens": L, "k": k,
             "us_per_append": (whole - finish) / L * 1e3, "us_finish": finish * 1e3, "us_per_interval": whole * 1e3,
             "us_batch_build_of_the_same_chunks": b0.elapsed_time(b1) / reps * 1e3,
-            "bytes_per_append": S * H * 2, "identical_to_batch": bool(torch.equal(proofs, ref_proofs))}
+            "bytes_per_append": S * H * 2, "identical_to_batch": bool(torch.equal(proofs, ref_proofs)),
+            "final_norm": {"us_norm_alone": norm_alone, "us_norm_with_fused_commit": norm_fused,
+                           "us_norm_then_separate_append": norm_separate,
+                           "us_added_by_fused_commit": norm_fused - norm_alone,
+                           "us_added_by_separate_append": norm_separate - norm_alone}}
 
 
 def direct_commitments(tl, synth, dev, workload, reps=10):

@@ -419,6 +419,37 @@ int toploc_stream_finish(const void* d_state, const toploc_layout* lay, uint8_t*
                          int32_t* d_indices_opt, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The engine-side hook of Section 5.5 fused into the kernel that produces the
+ * last hidden states: a final RMSNorm (the last operation before a Llama-style
+ * model's language-model head) that commits to its output while writing it.
+ *   y = x * rsqrt(mean(x^2) + eps) * weight     per row, fp32 arithmetic,
+ *                                               bf16 in and out (round to nearest even)
+ * One block per sequence normalises the sequence's new row, keeps it in shared
+ * memory, writes it to d_y, and offers the same tile to the sequence's running
+ * top-k as token token_in_chunk of its chunk -- the proof never reads the row
+ * from HBM.  Use it in place of toploc_stream_append: toploc_stream_begin
+ * before token 0, this call once per decode step with 0, 1, 2, ..., and
+ * toploc_stream_finish for the proofs, which are bit-identical to
+ * toploc_build_proofs over the rows written to d_y.  The device routines it is
+ * built from are public (include/toploc_device.cuh) for engines that want the
+ * same hook in a kernel of their own.
+ *
+ * d_x          DEVICE  [num_seqs, hidden] bf16, x_row_stride elements between rows
+ * d_weight     DEVICE  [hidden] bf16
+ * lay          HOST    as for toploc_stream_append (dtype bf16, TOPLOC_FIELD_16;
+ *                      row_stride = elements between the rows of d_y)
+ * d_y          DEVICE  out, [num_seqs, hidden] bf16
+ * d_state_opt  DEVICE  the running selections (toploc_stream_state_bytes), or
+ *                      NULL for the normalisation alone
+ * hidden and both strides must be multiples of 8 and every pointer 16-byte
+ * aligned (rows move as 16-byte vectors), hidden at most 81920; else
+ * TOPLOC_ERR_UNSUPPORTED / TOPLOC_ERR_INVALID_ARGUMENT.  Asynchronous.
+ */
+int toploc_rmsnorm_append(const void* d_x, int64_t x_row_stride, const void* d_weight, float eps,
+                          const toploc_layout* lay, int32_t token_in_chunk, void* d_y, void* d_state_opt,
+                          void* cuda_stream);
+
+/*
  * The same two operations for callers whose data lives in HOST memory
  * (pinned memory gives asynchronous copies; pageable memory works).  The
  * batch is cut into groups of whole sequences that fit the staging buffer;

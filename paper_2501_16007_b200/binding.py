@@ -22,6 +22,7 @@ __all__ = [
     "TOPLOC_MAX_K_DIRECT", "toploc_direct_commit_bytes", "toploc_commit_direct", "toploc_verify_direct",
     "toploc_default_thresholds", "toploc_verify_proofs_per_chunk_thresholds",
     "toploc_verify_direct_per_chunk_thresholds", "THRESHOLDS_DTYPE", "thresholds_tensor",
+    "toploc_rmsnorm_append",
 ]
 
 TOPLOC_DTYPE_BF16 = 0
@@ -122,6 +123,8 @@ def load_library():
     lib.toploc_verify_proofs_per_chunk_thresholds.argtypes = [vp, lay_p, vp, vp, vp, vp, vp, sz, vp]
     lib.toploc_verify_direct_per_chunk_thresholds.restype = ctypes.c_int
     lib.toploc_verify_direct_per_chunk_thresholds.argtypes = [vp, lay_p, vp, vp, vp, vp, vp]
+    lib.toploc_rmsnorm_append.restype = ctypes.c_int
+    lib.toploc_rmsnorm_append.argtypes = [vp, i64, vp, ctypes.c_float, lay_p, i32, vp, vp, vp]
     lib.toploc_default_thresholds.restype = ctypes.c_int
     lib.toploc_default_thresholds.argtypes = [i32, i32, thr_p]
     _LIB = lib
@@ -510,3 +513,21 @@ def toploc_verify_direct_per_chunk_thresholds(act, lay, commits, thresholds, res
             _dev_ptr(exp_dev), _stream_ptr(stream))
     _check(rc, "toploc_verify_direct_per_chunk_thresholds")
     return results, exp_dev
+
+
+def toploc_rmsnorm_append(x, weight, eps, lay, token_in_chunk, y, state=None, stream=None):
+    """Final RMSNorm of one new row per sequence (x, y: CUDA bf16 [num_seqs, hidden]; weight: bf16
+    [hidden]) that offers the normalised rows to the running selections in `state` (None: the
+    normalisation alone).  See toploc_rmsnorm_append in the header."""
+    if not (x.is_cuda and y.is_cuda and weight.is_cuda):
+        raise ToplocError("toploc_rmsnorm_append needs CUDA tensors")
+    if x.dtype != torch.bfloat16 or y.dtype != torch.bfloat16 or weight.dtype != torch.bfloat16:
+        raise ToplocError("toploc_rmsnorm_append works on bfloat16 tensors")
+    if x.dim() != 2 or x.stride(1) != 1 or y.stride(1) != 1 or not weight.is_contiguous():
+        raise ToplocError("rows must be contiguous")
+    with torch.cuda.device(x.device):
+        rc = load_library().toploc_rmsnorm_append(
+            _dev_ptr(x), x.stride(0) if x.shape[0] > 1 else x.shape[1], _dev_ptr(weight), float(eps),
+            ctypes.byref(lay), int(token_in_chunk), _dev_ptr(y), _dev_ptr(state), _stream_ptr(stream))
+    _check(rc, "toploc_rmsnorm_append")
+    return y

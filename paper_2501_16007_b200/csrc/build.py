@@ -8,8 +8,10 @@ import sys
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(os.path.dirname(_HERE))
-SOURCES = [os.path.join(_HERE, "toploc.cu"), os.path.join(_HERE, "toploc_direct.cu")]
-HEADERS = [os.path.join(_ROOT, "include", "toploc.h"), os.path.join(_HERE, "nearest_ratio.cuh")]
+SOURCES = [os.path.join(_HERE, "toploc.cu"), os.path.join(_HERE, "toploc_direct.cu"),
+           os.path.join(_HERE, "toploc_producer.cu")]
+HEADERS = [os.path.join(_ROOT, "include", "toploc.h"), os.path.join(_ROOT, "include", "toploc_device.cuh"),
+           os.path.join(_HERE, "nearest_ratio.cuh")]
 LIBRARY = os.path.join(_HERE, "libtoploc.so")
 
 
