@@ -2,6 +2,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 70b|8b] [--impl ours|reference]
 
+With --gpus N > 1 and no torchrun environment the script starts N ranks of itself
+(torch.distributed.run, one per GPU); under torchrun it is one of the ranks.
+
 One step = proof generation for every chunk of the batch followed by validation of every
 proof against recomputed activations (honest-noise copy), i.e. one pass of the whole path.
 The default workload is the Llama-3.1-70B-shaped batch: 256 sequences x 4096 tokens,
@@ -38,15 +41,21 @@ WORKLOADS = {
     "prompt70b": (64, 4096, 8192, 4096, 128, 6),
     # fp32 activations committed whole over the 32-bit field (2 + 4k byte proofs, fp32 thresholds)
     "70b-fp32-wide": (128, 4096, 8192, 32, 128, 7),
-    # small cases of the two above, for profiler captures
+    # small cases of the two above: sized for profiler captures, not benchmark workloads
     "prompt8b": (16, 2048, 4096, 2048, 128, 9),
     "8b-fp32-wide": (64, 2048, 4096, 32, 128, 8),
 }
 WIDE_WORKLOADS = ("70b-fp32-wide", "8b-fp32-wide")
+CAPTURE_ONLY_WORKLOADS = ("prompt8b", "8b-fp32-wide")
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one toploc_select_kernel launch on the full
-# batch (ncu, profiles/launch_list_70b_shape.md); None where no capture of the current kernel exists
-SELECT_DRAM_BYTES_PER_LAUNCH = {"70b": 17474558106 + 25958630}
+# DRAM traffic of one toploc_select_kernel launch, from a profiler capture (not measured by this
+# run): dram__bytes_read.sum + dram__bytes_write.sum of one launch on the 8B-shaped batch divided
+# by that batch's activation bytes.  The kernel reads every chunk once whatever the batch, so the
+# ratio carries over to the other bf16 batches.  None: no capture of the current kernel exists.
+SELECT_DRAM_TRAFFIC = {
+    "ratio_to_activation_bytes": None,
+    "source": None,
+}
 
 
 def measured_hbm_peak():
@@ -142,7 +151,8 @@ def reference_arm(args, rank):
     value = chunks / dt
     line = {
         "impl": "reference", "metric": "proof_chunks_per_s_generate_plus_verify", "value": value,
-        "unit": "chunks/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "unit": "chunks/s", "n_gpus": args.gpus, "ranks_started": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u32", "data": "synthetic",
         "config": {"workload": workload_name(args.workload), "sample": "first sequence (%d chunks) per step" % chunks},
@@ -179,16 +189,29 @@ def workload_name(key):
         "fp32 over the 32-bit field" if key in WIDE_WORKLOADS else "bf16", L, k)
 
 
+def start_ranks(n):
+    """Replaces this process by `n` ranks of the same command line under torch.distributed.run."""
+    port = os.environ.get("MASTER_PORT", str(29500 + os.getpid() % 2000))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", port, os.path.abspath(__file__)] + sys.argv[1:]
+    sys.stdout.flush()
+    os.execv(sys.executable, cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="70b")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="70b",
+                    help="70b is the headline batch; %s are small cases for profiler captures only"
+                         % " and ".join(CAPTURE_ONLY_WORKLOADS))
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-recipes", action="store_true",
+                    help="skip the extra timings of the 70B-shaped batch with jittered and without outlier channels")
     ap.add_argument("--decode-steps", action="store_true",
                     help="time incremental proof generation (one row per sequence and step) instead of the main workload")
     ap.add_argument("--direct", action="store_true",
@@ -199,6 +222,8 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        start_ranks(args.gpus)  # does not return
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -214,6 +239,8 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("NCCL_DEBUG", "INFO")        # the communicator's rank count shows in the log
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
         dist.init_process_group("nccl", device_id=dev)
 
     if args.decode_steps:
@@ -261,19 +288,21 @@ def main():
         if ev:
             ev[2].record()
 
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
         gpu_id = str(local_rank)
+    # the sampler runs from before the warm-up (the same steps as the timed ones) to the end of the
+    # timed region, so that a short timed region still sees the clock under this load
     sampler = ClockSampler(gpu_id)
+    sampler.start()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    sampler.start()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
     for i in range(args.steps):
@@ -342,7 +371,9 @@ def main():
                      "achieved": select_gbs, "peak": peak, "peak_kind": peak_kind + " (torch copy, burst)",
                      "unit": "GB/s", "frac": select_gbs / peak, "ms_per_launch": select_ms,
                      "algorithmic_bytes_per_launch": act_bytes,
-                     "traffic": SELECT_DRAM_BYTES_PER_LAUNCH.get(args.workload),
+                     "traffic": (None if wide or SELECT_DRAM_TRAFFIC["ratio_to_activation_bytes"] is None
+                                 else int(act_bytes * SELECT_DRAM_TRAFFIC["ratio_to_activation_bytes"])),
+                     "traffic_source": None if wide else SELECT_DRAM_TRAFFIC["source"],
                      "frac_of_8TBs_nominal": select_gbs / 8000.0},
         "roofline_calls": {"generate_frac_of_peak": build_gbs / peak, "verify_frac_of_peak": verify_gbs / peak,
                            "note": "whole calls: generate = select + interpolate kernels, verify = one kernel"},
@@ -354,9 +385,42 @@ def main():
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(act, recomputed, S, T, H, L, k, wide)
+    if args.workload == "70b" and world == 1 and not args.no_recipes:
+        # The literal +-80 recipe is the streaming filter's best case (every chunk's top-128 is its
+        # first 128 outliers, known after the first rows).  The same batch shape with jittered
+        # outlier magnitudes and with no outlier channels, regenerated in place and timed the same way.
+        line["other_recipes"] = {
+            name: time_recipe(tl, synth, name, act, recomputed, lay, proofs, status, results, thr, workspace,
+                              S, T, H, seed, min(args.steps, 20), n)
+            for name in ("jitter", "none")}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_recipe(tl, synth, outliers, act, recomputed, lay, proofs, status, results, thr, workspace, S, T, H, seed,
+                steps, n):
+    """Regenerates the batch in place with another outlier recipe and times generate and verify calls
+    (CUDA events, mean over `steps` steps after three warm-ups)."""
+    synth.make_activations(S, T, H, act.dtype, seed=seed + 500, device=act.device, outliers=outliers, out=act)
+    recomputed.copy_(synth.honest_noise(act, seed=seed + 501))
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    for i in range(-3, steps):
+        if i >= 0:
+            ev[i][0].record()
+        tl.toploc_build_proofs(act, lay, proofs, status, workspace=workspace)
+        if i >= 0:
+            ev[i][1].record()
+        tl.toploc_verify_proofs(recomputed, lay, proofs, thr, results, workspace=workspace)
+        if i >= 0:
+            ev[i][2].record()
+    torch.cuda.synchronize()
+    g = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    v = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    nbytes = act.numel() * act.element_size()
+    return {"generate_ms": g, "verify_ms": v, "generate_frac_of_8TBs_nominal": nbytes / g / 1e6 / 8000.0,
+            "verify_frac_of_8TBs_nominal": nbytes / v / 1e6 / 8000.0,
+            "accepted_chunks": int(results.cpu().numpy().view(tl.RESULT_DTYPE)["accept"].sum()), "chunks": n}
 
 
 def decode_steps(tl, synth, dev, reps=20):
@@ -568,21 +632,25 @@ def measure_e2e(tl, act, lay, n, k, thr, dev, steps, world):
 
 
 def cpu_baseline(act, recomputed, S, T, H, L, k, wide=False):
+    """The oracle, as it stands, on a bounded sample of the same batch: whole sequences from the
+    front, at least 1024 chunks where the batch has them (about 5 to 30 s on the host cores)."""
     import oracle
     from paper_2501_16007_b200 import synth
-    host = synth.host_patterns(act[:T])
-    host_rec = synth.host_patterns(recomputed[:T])
+    per_seq = (T + L - 1) // L
+    seqs = max(1, min(S, -(-1024 // per_seq))) if L * H <= (1 << 19) else 1   # a prompt-sized chunk takes seconds
+    host = synth.host_patterns(act[:seqs * T])
+    host_rec = synth.host_patterns(recomputed[:seqs * T])
     cores = oracle.default_threads()
-    chunks = T // L
+    chunks = seqs * per_seq
     t0 = time.perf_counter()
-    proofs, status, idx = oracle.build_proofs(host, L, k, 1, T, threads=cores, wide=wide)
+    proofs, status, idx = oracle.build_proofs(host, L, k, seqs, T, threads=cores, wide=wide)
     t1 = time.perf_counter()
-    oracle.verify_proofs(host_rec, proofs, L, k, 1, T, gen_indices=idx, threads=cores, wide=wide,
+    oracle.verify_proofs(host_rec, proofs, L, k, seqs, T, gen_indices=idx, threads=cores, wide=wide,
                          **({"t_exp": 8 * k // 128, "t_mean": 256.0, "t_median": 128.0} if wide else {}))
     t2 = time.perf_counter()
     return {"value": chunks / (t2 - t0), "unit": "chunks/s", "cores": cores, "kind": "oracle",
-            "sample": "first sequence: %d chunks of %d x %d %s, build + verify" % (
-            chunks, L, H, "fp32 (32-bit field)" if wide else "bf16"),
+            "sample": "first %d sequence(s): %d chunks of %d x %d %s, build + verify" % (
+            seqs, chunks, L, H, "fp32 (32-bit field)" if wide else "bf16"),
             "generate_chunks_per_s": chunks / (t1 - t0), "verify_chunks_per_s": chunks / (t2 - t1)}
 
 

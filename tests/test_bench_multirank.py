@@ -48,3 +48,19 @@ def test_reference_arm_prints_one_json_line():
     res = json.loads(out.stdout.strip().splitlines()[-1])
     assert res["impl"] == "reference" and res["unit"] == "chunks/s" and res["value"] > 0
     assert res["cpu_baseline"]["kind"] == "oracle" and res["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` without a torchrun environment starts two ranks of itself (here on the
+    reference arm, which needs no GPU: rank 0 measures and prints, rank 1 exits)."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    env["MASTER_PORT"] = "29547"
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--workload", "8b", "--steps", "1", "--warmup", "0"], capture_output=True, text=True,
+                         timeout=600, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    import json
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                              # one rank prints
+    res = json.loads(lines[0])
+    assert res["impl"] == "reference" and res["n_gpus"] == 2 and res["ranks_started"] == 2
