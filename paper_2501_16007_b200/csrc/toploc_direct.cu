@@ -28,6 +28,7 @@
 
 #include "nearest_ratio.cuh"
 #include "toploc.h"
+#include "toploc_device.cuh"
 
 namespace {
 
@@ -67,9 +68,17 @@ struct DirectShared {
   uint32_t bad;
   uint32_t counters[4];      // exponent mismatches, matches, mantissa difference sum, common indices
   uint32_t dev[9];
+  // the free-running one-pass selection (select_unordered)
+  uint32_t cand_count;       // candidates handed out so far (may run past the buffer: then overflow is set)
+  uint32_t thr;              // an element is a candidate iff its key is >= thr; only ever raised
+  uint32_t last_raise;       // cand_count when thr was last raised
+  uint32_t raise_lock;       // 1 while a warp is raising thr
+  uint32_t overflow;
+  uint32_t emitted;
+  uint32_t pad[2];
   uint32_t hist[kBins];
 };
-constexpr size_t kSpareBytes = 35264;
+constexpr size_t kSpareBytes = 35232;
 constexpr size_t kSharedBytes = kRingBytes + sizeof(DirectShared) + kSpareBytes;
 // One-pass selection (vector layouts, k <= kStreamMaxK): a histogram of the upper 11 key bits
 // and up to cand_cap candidates (flat index, whole pattern) in index order.
@@ -82,6 +91,17 @@ static_assert((size_t)kCoarseBins * 4 + (size_t)cand_cap(0) * 6 <= (size_t)kBins
                   (size_t)kCoarseBins * 4 + (size_t)cand_cap(1) * 8 <= (size_t)kBins * 4 + kSpareBytes,
               "candidates fit");
 static_assert(12 * TOPLOC_MAX_K_DIRECT <= kRingBytes, "the verify lists fit the idle ring");
+// The free-running one-pass selection parks, per warp, the vectors that passed the quick test
+// until there are enough of them to unpack with every lane busy; its candidates are unordered.
+constexpr int kParkCap = 32 + kUnroll * 32;   // a batch parks at most kUnroll vectors per lane
+constexpr int kParkTrigger = 32;
+constexpr size_t kParkBytes = (size_t)kWarps * kParkCap * 4;
+__host__ __device__ constexpr int loose_cap(int dt) {
+  return (int)(((size_t)kBins * 4 + kSpareBytes - (size_t)kCoarseBins * 4 - kParkBytes) / (dt == 0 ? 6 : 8)) / 64 * 64;
+}
+constexpr int kLooseMaxElems = 1 << 19;       // its index-order bitmap must fit the ring
+static_assert((size_t)kLooseMaxElems / 8 <= kRingBytes, "one bit per element of the chunk");
+static_assert(loose_cap(0) >= 5 * 4096 && loose_cap(1) >= 4 * 4096, "room for the candidates of k = 4096");
 
 // A group is VEC consecutive elements of one row (one 16-byte vector, or one element when
 // the layout does not allow aligned vectors).
@@ -526,6 +546,286 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<D
   return true;
 }
 
+
+// One-pass selection without a barrier in the streaming loop (vector layouts, chunks of at most
+// kLooseMaxElems elements).  Every warp streams its share of the chunk on its own: a vector is
+// tested as a whole against the block's running threshold; vectors that pass are parked per
+// warp and, 32 at a time, unpacked by the whole warp into the block's candidate buffer
+// (slots handed out by one atomic per round) and counted in a histogram of their upper 11 key
+// bits.  The threshold only ever rises: whenever enough new candidates have arrived, one warp
+// (whoever gets the lock) walks the histogram from the top to the bin that holds the k-th
+// largest candidate so far and publishes that bin's lowest key -- at least k candidates reach
+// it, so nothing below it can belong to the top-k, whatever the other warps add meanwhile (the
+// counts only grow).  Warps that still test against an older threshold only admit more.
+// Candidates arrive in no particular order; the exact k-th key, the ties that belong to the
+// top-k (lowest flat indices) and the position of every selected element in index order are
+// settled at the end.  ORDERED: emit(position in ascending index order, ...), by ranking the
+// selected indices in a bitmap of the chunk; otherwise positions are handed out as they come.
+// Returns false, having emitted nothing, when the candidates outgrow their buffer.
+template <int DT, bool ORDERED, class Emit>
+__device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit) {
+  using R = Reader<DT, true>;
+  using Pat = typename StoredPattern<DT>::type;
+  constexpr int VEC = R::VEC;
+  constexpr int kCap = loose_cap(DT);
+  constexpr int kCoarseShift = key_bits(DT) - 11;
+  constexpr uint32_t kFull = 0xFFFFFFFFu;
+  constexpr int kBatch = kUnroll * kThreads;
+  uint32_t* coarse = sh.hist;
+  uint32_t* cand_flat = sh.hist + kCoarseBins;
+  Pat* cand_pat = reinterpret_cast<Pat*>(cand_flat + kCap);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* park = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(sh.hist) + (size_t)kBins * 4 +
+                                               kSpareBytes - kParkBytes) + warp * kParkCap;
+  volatile uint32_t* shared_thr = &sh.thr;
+  volatile uint32_t* shared_overflow = &sh.overflow;
+  volatile uint32_t* shared_last_raise = &sh.last_raise;
+  if (threadIdx.x == 0) {
+    sh.cand_count = 0;
+    sh.thr = 0;
+    sh.last_raise = 0;
+    sh.raise_lock = 0;
+    sh.overflow = 0;
+    sh.emitted = 0;
+  }
+  clear_bins(sh, kCoarseBins);  // ends with a barrier
+
+  // One vector per lane: its elements that reach thr become candidates.  Returns the number of
+  // candidates handed out so far (0 if the round added none).
+  auto admit = [&](bool valid, uint32_t g, uint32_t thr) -> uint32_t {
+    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+    if (valid) w = toploc_device::load_streaming(reinterpret_cast<const uint4*>(rd.address((int)g)));
+    uint32_t mask = valid ? toploc_device::passing_mask<DT, VEC>(w, thr) : 0u;
+    const int mine = __popc(mask);
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int other = __shfl_up_sync(kFull, incl, off);
+      if (lane >= off) incl += other;
+    }
+    const int total = __shfl_sync(kFull, incl, 31);
+    if (total == 0) return 0u;
+    uint32_t base = 0;
+    if (lane == 0) base = atomicAdd(&sh.cand_count, (uint32_t)total);
+    base = __shfl_sync(kFull, base, 0);
+    if (base + (uint32_t)total > (uint32_t)kCap) {
+      if (lane == 0) *shared_overflow = 1u;
+      return base + (uint32_t)total;
+    }
+    uint32_t at = base + (uint32_t)(incl - mine);
+    while (mask) {
+      const uint32_t e = (uint32_t)__ffs((int)mask) - 1u;
+      mask &= mask - 1u;
+      uint32_t key, sign;
+      toploc_device::pick_element<DT, VEC>(w, e, &key, &sign);
+      cand_flat[at] = g * VEC + e;
+      cand_pat[at] = (Pat)((sign << (DT == 0 ? 15 : 31)) | key);
+      atomicAdd(&coarse[key >> kCoarseShift], 1u);
+      ++at;
+    }
+    return base + (uint32_t)total;
+  };
+
+  // A sound first threshold from the chunk's first vectors: the k-th largest of their per-vector
+  // maxima (each maximum is a different element, so at least k elements reach it).  Those vectors
+  // are then streamed like the rest.  A chunk of fewer than k vectors starts from 0.
+  {
+    const int first_end = kBatch < rd.n_groups ? kBatch : rd.n_groups;
+    rd.request(ring, (int)threadIdx.x, first_end);  // in flight meanwhile
+  }
+  const int seed_groups = 4 * k < rd.n_groups ? 4 * k : rd.n_groups;
+  if (seed_groups >= k) {
+    for (int g = threadIdx.x; g < seed_groups; g += kThreads) {
+      const uint4 w = toploc_device::load_streaming(reinterpret_cast<const uint4*>(rd.address(g)));
+      atomicAdd(&coarse[toploc_device::vector_max_coarse_key<DT, VEC>(w) >> 4], 1u);  // upper 11 of 15 bits
+    }
+    __syncthreads();
+    find_bin_from_top(sh, kCoarseBins, (uint32_t)k, 0);
+    const uint32_t first = sh.picked_bin << kCoarseShift;
+    __syncthreads();
+    if (threadIdx.x == 0) sh.thr = first;
+    clear_bins(sh, kCoarseBins);
+  }
+
+  const uint32_t raise_step = (uint32_t)(k / 2 > 256 ? k / 2 : 256);
+  uint32_t thr = *shared_thr;
+  int nparked = 0;
+  auto drain = [&]() {
+    __syncwarp();
+    uint32_t handed_out = 0;
+    for (int b = 0; b < nparked; b += 32) {
+      const bool valid = b + lane < nparked;
+      const uint32_t g = valid ? park[b + lane] : 0u;
+      const uint32_t after = admit(valid, g, thr);
+      handed_out = after > handed_out ? after : handed_out;
+    }
+    nparked = 0;
+    __syncwarp();
+    // raise the threshold if enough candidates have arrived since the last time and nobody else is at it
+    uint32_t go = 0;
+    if (lane == 0 && handed_out >= (uint32_t)k && handed_out <= (uint32_t)kCap &&
+        handed_out - *shared_last_raise >= raise_step)
+      go = atomicCAS(&sh.raise_lock, 0u, 1u) == 0u ? 1u : 0u;
+    go = __shfl_sync(kFull, go, 0);
+    if (go) {
+      // lane l owns bins top, top - 1, ..., top - 63 (lane 0 the highest keys)
+      constexpr int kPerLane = kCoarseBins / 32;
+      const int top = kCoarseBins - 1 - lane * kPerLane;
+      volatile uint32_t* bins = coarse;
+      uint32_t sum = 0;
+      for (int b = 0; b < kPerLane; ++b) sum += bins[top - ((b + lane) & (kPerLane - 1))];
+      uint32_t upto = sum;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t other = __shfl_up_sync(kFull, upto, off);
+        if (lane >= off) upto += other;
+      }
+      const uint32_t before = upto - sum;
+      if (before < (uint32_t)k && (uint32_t)k <= upto) {
+        uint32_t c = before;
+        for (int b = 0; b < kPerLane; ++b) {
+          c += bins[top - b];
+          if (c >= (uint32_t)k) {  // (counts read a second time are no smaller than the first time)
+            atomicMax(&sh.thr, (uint32_t)(top - b) << kCoarseShift);
+            break;
+          }
+        }
+      }
+      if (lane == 0) *shared_last_raise = handed_out;
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence_block();
+        atomicExch(&sh.raise_lock, 0u);
+      }
+    }
+  };
+
+  for (int begin = 0; begin < rd.n_groups; begin += kBatch) {
+    const int end = begin + kBatch < rd.n_groups ? begin + kBatch : rd.n_groups;
+    uint32_t w[kUnroll][4];
+    rd.take(ring, begin + (int)threadIdx.x, end, w);
+    if (end < rd.n_groups) {
+      const int next_end = end + kBatch < rd.n_groups ? end + kBatch : rd.n_groups;
+      rd.request_after(ring, end + (int)threadIdx.x, next_end, w, begin + (int)threadIdx.x, end);
+    }
+    const uint32_t add = toploc_device::bf16_lane_add(thr);
+    bool hit[kUnroll];
+    uint32_t votes[kUnroll], any_votes = 0;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int g = begin + u * kThreads + (int)threadIdx.x;
+      hit[u] = g < end && toploc_device::vector_reaches<DT, VEC>(make_uint4(w[u][0], w[u][1], w[u][2], w[u][3]), thr, add);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      votes[u] = __ballot_sync(kFull, hit[u]);
+      any_votes |= votes[u];
+    }
+    if (any_votes) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (hit[u]) park[nparked + __popc(votes[u] & ((1u << lane) - 1u))] = (uint32_t)(begin + u * kThreads) + threadIdx.x;
+        nparked += __popc(votes[u]);
+      }
+      if (nparked >= kParkTrigger) drain();
+    }
+    thr = *shared_thr;
+    if (*shared_overflow) break;
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");  // a batch requested before leaving the loop
+  if (!*shared_overflow) drain();
+  __syncthreads();
+  if (sh.overflow) return false;
+  const uint32_t count = sh.cand_count;
+
+  // The exact k-th key among the candidates: its upper 11 bits from the histogram (it counts
+  // every candidate), the bits below 8 at a time (the last digit has 4).
+  find_bin_from_top(sh, kCoarseBins, (uint32_t)k, 0);
+  uint32_t kth = sh.picked_bin << kCoarseShift, known = (uint32_t)(kCoarseBins - 1) << kCoarseShift;
+  uint32_t take = sh.picked_remaining, ties = 0;
+  __syncthreads();
+  for (int shift = kCoarseShift - 8, round = 1; shift > -8; shift -= 8, ++round) {
+    const int low = shift < 0 ? 0 : shift, width = shift < 0 ? 8 + shift : 8;
+    clear_bins(sh, 256);
+    for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+      const uint32_t key = R::key(cand_pat[i]);
+      if ((key & known) == kth) atomicAdd(&sh.hist[(key >> low) & ((1u << width) - 1u)], 1u);
+    }
+    __syncthreads();
+    find_bin_from_top(sh, 1 << width, take, round & 1);
+    kth |= sh.picked_bin << low;
+    known |= ((1u << width) - 1u) << low;
+    take = sh.picked_remaining;
+    ties = sh.hist[sh.picked_bin];  // after the last digit: the candidates equal to the k-th key
+    __syncthreads();
+  }
+  // Of the candidates equal to the k-th key the `take` lowest flat indices belong to the top-k:
+  // the take-th largest of (2^24 - 1 - flat index) among them, digit by digit (nothing to find
+  // when all of them belong).
+  uint32_t cut = 0, cut_known = 0;
+  for (int shift = 16, round = 0; shift >= 0 && ties != take; shift -= 8, ++round) {
+    clear_bins(sh, 256);
+    for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+      if (R::key(cand_pat[i]) != kth) continue;
+      const uint32_t inv = 0xFFFFFFu - cand_flat[i];
+      if ((inv & cut_known) == cut) atomicAdd(&sh.hist[(inv >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    find_bin_from_top(sh, 256, take, round & 1);
+    cut |= sh.picked_bin << shift;
+    cut_known |= 255u << shift;
+    take = sh.picked_remaining;
+    __syncthreads();
+  }
+  auto selected = [&](uint32_t i) {
+    const uint32_t key = R::key(cand_pat[i]);
+    return key > kth || (key == kth && 0xFFFFFFu - cand_flat[i] >= cut);
+  };
+
+  if (!ORDERED) {
+    for (uint32_t i0 = 0; i0 < count; i0 += kThreads) {
+      const uint32_t i = i0 + threadIdx.x;
+      const bool mine = i < count && selected(i);
+      const uint32_t votes = __ballot_sync(kFull, mine);
+      uint32_t base = 0;
+      if (lane == 0 && votes) base = atomicAdd(&sh.emitted, (uint32_t)__popc(votes));
+      base = __shfl_sync(kFull, base, 0);
+      if (mine) emit(base + (uint32_t)__popc(votes & ((1u << lane) - 1u)), cand_flat[i], R::committed(cand_pat[i]));
+    }
+    __syncthreads();
+    return true;
+  }
+  // Index order: one bit per element of the chunk for the selected ones; an element's position is
+  // the number of set bits before its own.
+  uint32_t* bitmap = reinterpret_cast<uint32_t*>(ring);
+  const uint32_t n_words = ((uint32_t)rd.n_groups * VEC + 31u) / 32u;
+  const uint32_t per_thread = (n_words + kThreads - 1) / kThreads;  // consecutive words a thread counts
+  for (uint32_t wd = threadIdx.x; wd < n_words; wd += kThreads) bitmap[wd] = 0u;
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < count; i += kThreads)
+    if (selected(i)) atomicOr(&bitmap[cand_flat[i] >> 5], 1u << (cand_flat[i] & 31u));
+  __syncthreads();
+  {
+    const uint32_t lo = threadIdx.x * per_thread < n_words ? threadIdx.x * per_thread : n_words;
+    const uint32_t hi = lo + per_thread < n_words ? lo + per_thread : n_words;
+    uint32_t ones = 0;
+    for (uint32_t wd = lo; wd < hi; ++wd) ones += (uint32_t)__popc(bitmap[wd]);
+    unsigned long long total;
+    sh.hist[threadIdx.x] = (uint32_t)block_scan_exclusive(sh, ones, 0, &total);  // set bits before this thread's words
+  }
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+    if (!selected(i)) continue;
+    const uint32_t flat = cand_flat[i], wd = flat >> 5, owner = wd / per_thread;
+    uint32_t pos = sh.hist[owner];
+    for (uint32_t v = owner * per_thread; v < wd; ++v) pos += (uint32_t)__popc(bitmap[v]);
+    pos += (uint32_t)__popc(bitmap[wd] & ((1u << (flat & 31u)) - 1u));
+    emit(pos, flat, R::committed(cand_pat[i]));
+  }
+  __syncthreads();
+  return true;
+}
+
 template <int DT, bool VECTOR>
 __device__ __forceinline__ Reader<DT, VECTOR> locate_chunk(const DirectParams& p, long long chunk) {
   using R = Reader<DT, VECTOR>;
@@ -566,7 +866,8 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
   };
   bool done = false;
   if constexpr (VECTOR) {
-    if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
+    if ((long long)rd.n_groups * R::VEC <= kLooseMaxElems) done = select_unordered<DT, true>(sh, ring, rd, p.k, emit);
+    else if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
   }
   if (!done) {
     uint32_t kth, take;
@@ -616,10 +917,11 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
   };
   bool done = false;
   if constexpr (VECTOR) {
-    if (k <= kStreamMaxK) {
+    const bool loose = n_elems <= (uint32_t)kLooseMaxElems;  // the comparison below needs no particular order
+    if (loose || k <= kStreamMaxK) {
       sel_idx = reinterpret_cast<uint32_t*>(ring);
       sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
-      done = select_in_one_pass<DT>(sh, ring, rd, k, emit);
+      done = loose ? select_unordered<DT, false>(sh, ring, rd, k, emit) : select_in_one_pass<DT>(sh, ring, rd, k, emit);
     }
   }
   if (!done) {
@@ -731,6 +1033,247 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
   }
 }
 
+
+// ---------------------------------------------------------------------------
+// Small k (k <= TOPLOC_MAX_K, chunks of at most 2^19 elements): one warp per chunk, the
+// selection of the proof path (toploc_device::select_topk: the chunk streams once through the
+// warp's ring, the exact top-k ends up in shared memory), sixteen chunks per SM in flight and
+// nothing that waits on another warp.  The commitment is the selection sorted by index; the
+// validation looks every selected index up in the commitment.
+// ---------------------------------------------------------------------------
+namespace small_k {
+using namespace toploc_device;
+
+constexpr int kSlots = TOPLOC_MAX_K / 32;
+constexpr long long kMaxElems = 1ll << 19;
+
+template <int DT, int MODE>
+__device__ __forceinline__ ChunkSource<DT, MODE> source_of(const DirectParams& p, long long chunk, long long* n_elems) {
+  const long long seq = chunk / p.chunks_per_seq;
+  const long long j = chunk - seq * p.chunks_per_seq;
+  const long long row0 = seq * p.tokens_per_seq + j * p.chunk_len;
+  const long long left = p.tokens_per_seq - j * p.chunk_len;
+  const long long rows = left < p.chunk_len ? left : p.chunk_len;
+  ChunkSource<DT, MODE> src;
+  src.base = static_cast<const char*>(p.act) + row0 * p.row_stride * (DT == 0 ? 2 : 4);
+  src.row_stride = p.row_stride;
+  src.hidden = p.hidden;
+  src.vecs_per_row = p.hidden / ChunkSource<DT, MODE>::kVec;
+  *n_elems = rows * p.hidden;
+  return src;
+}
+
+// flat index and committed 16-bit pattern of a candidate word
+template <int DT>
+__device__ __forceinline__ void unpack(unsigned long long c, uint32_t* flat, uint32_t* pattern) {
+  const uint32_t key = (uint32_t)(c >> (kIdxBits + 1)), sign = (uint32_t)c & 1u;
+  *flat = kIdxMask - ((uint32_t)(c >> 1) & kIdxMask);
+  *pattern = (sign << 15) | (DT == 0 ? key : key >> 16);
+}
+
+template <int DT, int MODE>
+__global__ void __launch_bounds__(32, 15) toploc_direct_commit_warp_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
+  __shared__ SelectShared sh;
+  const int lane = threadIdx.x;
+  const long long chunk = blockIdx.x;
+  const int k = p.k;
+  uint16_t* rec = reinterpret_cast<uint16_t*>(commits + (size_t)chunk * 6u * (size_t)k);
+  long long n_elems;
+  const ChunkSource<DT, MODE> src = source_of<DT, MODE>(p, chunk, &n_elems);
+  if (n_elems < k) {
+    for (int i = lane; i < 3 * k; i += 32) rec[i] = 0;
+    if (lane == 0) status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+    return;
+  }
+  select_topk<DT, MODE>(sh, src, (int)n_elems, k);
+  // ascending index order: a point's record number is the number of selected indices below its own
+  for (int j = lane; j < k; j += 32) {
+    uint32_t flat, pattern;
+    unpack<DT>(sh.cand[j], &flat, &pattern);
+    const uint32_t mine = kIdxMask - flat;  // the index field as stored: larger means a lower index
+    int pos = 0;
+    for (int i = 0; i < k; ++i) pos += (((uint32_t)(sh.cand[i] >> 1)) & kIdxMask) > mine;
+    rec[3 * pos] = (uint16_t)(flat & 0xFFFFu);
+    rec[3 * pos + 1] = (uint16_t)(flat >> 16);
+    rec[3 * pos + 2] = (uint16_t)pattern;
+  }
+  if (lane == 0) status[chunk] = TOPLOC_CHUNK_OK;
+}
+
+template <int DT, int MODE>
+__global__ void __launch_bounds__(32, 15) toploc_direct_verify_warp_kernel(DirectParams p, DirectVerify io) {
+  __shared__ SelectShared sh;
+  const int lane = threadIdx.x;
+  const long long chunk = blockIdx.x;
+  const int k = p.k;
+  long long n_elems;
+  const ChunkSource<DT, MODE> src = source_of<DT, MODE>(p, chunk, &n_elems);
+  auto refuse = [&](int status) {
+    if (lane == 0) {
+      toploc_chunk_result r = {};
+      r.topk_mismatch = -1;
+      r.status = (uint8_t)status;
+      io.results[chunk] = r;
+    }
+    if (io.exp_dev != nullptr && lane < 9) io.exp_dev[(size_t)chunk * 9 + lane] = 0;
+  };
+  if (n_elems < k) {
+    refuse(TOPLOC_CHUNK_K_EXCEEDS_CHUNK);
+    return;
+  }
+  select_topk<DT, MODE>(sh, src, (int)n_elems, k);
+  uint32_t sel_flat[kSlots], sel_pat[kSlots];
+#pragma unroll
+  for (int s = 0; s < kSlots; ++s) {
+    sel_flat[s] = 0;
+    sel_pat[s] = 0;
+    if (s * 32 + lane < k) unpack<DT>(sh.cand[s * 32 + lane], &sel_flat[s], &sel_pat[s]);
+  }
+  // the selection is in registers: the ring holds the commitment, the histograms the statistics
+  uint32_t* com_idx = reinterpret_cast<uint32_t*>(sh.ring);
+  uint32_t* com_pat = com_idx + TOPLOC_MAX_K;
+  uint32_t* hist = sh.top_hist;  // a 7-bit mantissa difference is at most 127
+  warp_barrier();
+  const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
+  for (int j = lane; j < k; j += 32) {
+    com_idx[j] = (uint32_t)rec[3 * j] | ((uint32_t)rec[3 * j + 1] << 16);
+    com_pat[j] = rec[3 * j + 2];
+  }
+  for (int b = lane; b < 128; b += 32) hist[b] = 0;
+  warp_barrier();
+  uint32_t bad = 0;  // indices must ascend strictly and lie inside the chunk
+  for (int j = lane; j < k; j += 32) bad |= (com_idx[j] >= (uint32_t)n_elems) | (j > 0 && com_idx[j] <= com_idx[j - 1]);
+  if (__any_sync(0xFFFFFFFFu, bad != 0)) {
+    refuse(TOPLOC_CHUNK_BAD_PROOF);
+    return;
+  }
+  const toploc_thresholds thr = io.thr_each ? io.thr_each[chunk] : io.thr;
+  const uint32_t field = thr.sign_in_exponent ? 0x1FFu : 0xFFu;
+  uint32_t err_e = 0, n_match = 0, sum = 0, common = 0, dev[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+  for (int s = 0; s < kSlots; ++s) {
+    if (s * 32 + lane >= k) continue;
+    const uint32_t want = sel_flat[s];
+    int lo = 0, hi = k;  // first committed index >= want
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (com_idx[mid] < want) lo = mid + 1; else hi = mid;
+    }
+    if (lo == k || com_idx[lo] != want) {
+      ++err_e;  // nothing was committed for this index
+      continue;
+    }
+    ++common;
+    const uint32_t committed = com_pat[lo], seen = sel_pat[s];
+    if (((committed >> 7) & field) == ((seen >> 7) & field)) {
+      const uint32_t mp = committed & 0x7Fu, mv = seen & 0x7Fu;
+      const uint32_t d = mp > mv ? mp - mv : mv - mp;
+      ++n_match;
+      sum += d;
+      atomicAdd(&hist[d], 1u);
+    } else {
+      ++err_e;
+    }
+    const int d = (int)((seen >> 7) & 0xFFu) - (int)((committed >> 7) & 0xFFu);
+    const int a = d < 0 ? -d : d;
+    const int bin = d == 0 ? 0 : a == 1 ? (d < 0 ? 1 : 2) : a == 2 ? (d < 0 ? 3 : 4) : a <= 10 ? (d < 0 ? 5 : 6) : a <= 99 ? 7 : 8;
+#pragma unroll
+    for (int b = 0; b < 9; ++b) dev[b] += bin == b;
+  }
+  err_e = __reduce_add_sync(0xFFFFFFFFu, err_e);
+  n_match = __reduce_add_sync(0xFFFFFFFFu, n_match);
+  sum = __reduce_add_sync(0xFFFFFFFFu, sum);
+  common = __reduce_add_sync(0xFFFFFFFFu, common);
+#pragma unroll
+  for (int b = 0; b < 9; ++b) dev[b] = __reduce_add_sync(0xFFFFFFFFu, dev[b]);
+  warp_barrier();
+  if (io.exp_dev != nullptr && lane < 9) {
+    uint32_t mine = 0;
+#pragma unroll
+    for (int b = 0; b < 9; ++b) mine = lane == b ? dev[b] : mine;
+    io.exp_dev[(size_t)chunk * 9 + lane] = mine;
+  }
+  // median from the histogram: sorted positions (n - 1) / 2 and n / 2; lane l owns bins 4l .. 4l + 3
+  uint32_t local[4], mine = 0;
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    local[b] = hist[lane * 4 + b];
+    mine += local[b];
+  }
+  uint32_t incl = mine;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t other = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    if (lane >= off) incl += other;
+  }
+  int lo_val = -1, hi_val = -1;
+  if (n_match > 0) {
+    const uint32_t lo_pos = (n_match - 1) / 2, hi_pos = n_match / 2;
+    uint32_t below = incl - mine;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const uint32_t upto = below + local[b];
+      if (below <= lo_pos && lo_pos < upto) lo_val = lane * 4 + b;
+      if (below <= hi_pos && hi_pos < upto) hi_val = lane * 4 + b;
+      below = upto;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    lo_val = max(lo_val, __shfl_xor_sync(0xFFFFFFFFu, lo_val, off));
+    hi_val = max(hi_val, __shfl_xor_sync(0xFFFFFFFFu, hi_val, off));
+  }
+  if (lane == 0) {
+    toploc_chunk_result r = {};
+    r.exp_mismatch = err_e;
+    r.n_match = n_match;
+    r.mant_diff_sum = sum;
+    r.topk_mismatch = k - (int)common;
+    bool reject = (long long)err_e > (long long)thr.t_exp;
+    if (n_match > 0) {
+      r.mant_mean = nearest_ratio(sum, n_match);
+      r.mant_median = ((double)lo_val + (double)hi_val) * 0.5;
+      reject = reject || r.mant_mean > thr.t_mean || r.mant_median > thr.t_median;
+    } else {
+      reject = true;  // nothing matched: no statistic to accept on
+    }
+    r.accept = reject ? 0 : 1;
+    r.status = TOPLOC_CHUNK_OK;
+    io.results[chunk] = r;
+  }
+}
+
+// 0: flat vectors, 1: aligned rows with padding, 2: element-wise (as in the proof path)
+inline int layout_mode(const void* act, const toploc_layout* lay) {
+  const int esz = lay->dtype == TOPLOC_DTYPE_BF16 ? 2 : 4;
+  const int vec = 16 / esz;
+  const bool aligned = (reinterpret_cast<uintptr_t>(act) % 16 == 0) && (lay->hidden % vec == 0) && (lay->row_stride % vec == 0);
+  if (!aligned) return 2;
+  return lay->row_stride == lay->hidden ? 0 : 1;
+}
+
+inline bool applies(const toploc_layout* lay) {
+  const long long rows = lay->tokens_per_seq < lay->chunk_len ? lay->tokens_per_seq : lay->chunk_len;
+  return lay->k <= TOPLOC_MAX_K && rows * lay->hidden <= kMaxElems;
+}
+
+template <int DT>
+int launch_commit(int mode, long long n, cudaStream_t stream, const DirectParams& p, uint8_t* commits, uint8_t* status) {
+  if (mode == 0) toploc_direct_commit_warp_kernel<DT, 0><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
+  else if (mode == 1) toploc_direct_commit_warp_kernel<DT, 1><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
+  else toploc_direct_commit_warp_kernel<DT, 2><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
+  return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+}
+
+template <int DT>
+int launch_verify(int mode, long long n, cudaStream_t stream, const DirectParams& p, const DirectVerify& io) {
+  if (mode == 0) toploc_direct_verify_warp_kernel<DT, 0><<<(unsigned)n, 32, 0, stream>>>(p, io);
+  else if (mode == 1) toploc_direct_verify_warp_kernel<DT, 1><<<(unsigned)n, 32, 0, stream>>>(p, io);
+  else toploc_direct_verify_warp_kernel<DT, 2><<<(unsigned)n, 32, 0, stream>>>(p, io);
+  return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+}
+}  // namespace small_k
+
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
@@ -803,6 +1346,11 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
+  if (small_k::applies(lay)) {
+    const int mode = small_k::layout_mode(d_act, lay);
+    return lay->dtype == TOPLOC_DTYPE_BF16 ? small_k::launch_commit<0>(mode, plan.num_chunks, stream, p, d_commits, d_status)
+                                           : small_k::launch_commit<1>(mode, plan.num_chunks, stream, p, d_commits, d_status);
+  }
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_commit_kernel<0, true>, plan.num_chunks, smem, stream, p, d_commits, d_status)
                        : launch_direct(toploc_direct_commit_kernel<0, false>, plan.num_chunks, smem, stream, p, d_commits, d_status);
@@ -835,6 +1383,11 @@ static int verify_direct_with(const void* d_act, const toploc_layout* lay, const
   io.thr_each = d_thr_each;
   const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
+  if (small_k::applies(lay)) {
+    const int mode = small_k::layout_mode(d_act, lay);
+    return lay->dtype == TOPLOC_DTYPE_BF16 ? small_k::launch_verify<0>(mode, plan.num_chunks, stream, p, io)
+                                           : small_k::launch_verify<1>(mode, plan.num_chunks, stream, p, io);
+  }
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_verify_kernel<0, true>, plan.num_chunks, smem, stream, p, io)
                        : launch_direct(toploc_direct_verify_kernel<0, false>, plan.num_chunks, smem, stream, p, io);
