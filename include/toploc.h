@@ -60,13 +60,17 @@ extern "C" {
  * points return TOPLOC_ERR_UNSUPPORTED for it. */
 #define TOPLOC_FIELD_16_PADDED 2
 
-/* Largest k the kernels are built for and largest chunk (elements; only chunks
+/* Largest k of a polynomial proof and largest chunk (elements; only chunks
  * the layout really contains count, so chunk_len may exceed every sequence).
  * A chunk of more than 2^19 elements -- a prompt committed as one chunk,
  * Section 5.5 -- is selected in segments of whole rows, one warp each, whose
  * winners are merged; the result is the same top-k.  hidden itself may not
- * exceed 2^24. */
-#define TOPLOC_MAX_K 256
+ * exceed 2^24.  k = 512 is about as far as Algorithm 6 reaches: a candidate
+ * modulus m separates k indices with probability near exp(-k^2 / 2m), 0.13 at
+ * k = 512 and below 1e-3 at k = 1024, so larger k are served by the direct
+ * commitments below.  Proofs of k <= 256 take the smaller of two per-warp
+ * scratch sizes (sixteen chunks in flight per SM instead of thirteen). */
+#define TOPLOC_MAX_K 512
 #define TOPLOC_MAX_CHUNK_ELEMS 0x7FFFFFFF
 /* Largest k of a direct commitment (toploc_commit_direct): the largest top-k
  * the paper looks at (the exponent-error table of Section 3). */

@@ -30,7 +30,8 @@
  * toploc_verify_kernel and toploc_stream_append_kernel run.
  *
  * Rules: one full warp (32 converged lanes) drives a selection; a SelectShared
- * object (13.4 KB of shared memory) belongs to that warp from open to close;
+ * object (13.4 KB of shared memory; SelectSharedBig, 16.5 KB, for k above 256) belongs to that warp
+ * from open to close;
  * tiles are 16-byte aligned, hold a multiple of 8 bf16 (4 fp32) values and are
  * offered in ascending flat-index order (flat index = token_in_chunk * hidden +
  * channel, at most 2^24 per chunk); k <= TOPLOC_MAX_K.
@@ -60,18 +61,13 @@ constexpr int kStages = TOPLOC_SELECT_STAGES;
 #ifndef TOPLOC_CAND_CAP
 #define TOPLOC_CAND_CAP 640
 #endif
-constexpr int kCandCap = TOPLOC_CAND_CAP;  // select: candidate buffer entries (8 bytes each)
 #ifndef TOPLOC_HIT_TRIGGER
 #define TOPLOC_HIT_TRIGGER 32
 #endif
 constexpr int kHitCap = TOPLOC_HIT_TRIGGER + 128;  // select: vectors that can be parked between drains
 constexpr int kHitTrigger = TOPLOC_HIT_TRIGGER;    // select: drain once this many are parked
-constexpr int kMaxK = TOPLOC_MAX_K;
-constexpr int kMaxSlots = kMaxK / 32;    // tail: entries a lane owns at most
 constexpr int kIdxBits = 24;             // flat index field of a candidate
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
-static_assert(kCandCap * 8 >= 8 * kMaxK * 2, "the candidate buffer holds the maxima of the first vectors");
-static_assert(kCandCap >= kMaxK + kThreads * 8, "a round of appends must fit after a compaction");
 static_assert(kHitCap >= kHitTrigger - 1 + kThreads * kUnroll, "a tile's hits must fit below the drain trigger");
 
 // A candidate is one 64-bit word whose unsigned order is the ranking order:
@@ -81,9 +77,21 @@ __device__ __forceinline__ unsigned long long make_candidate(uint32_t key, uint3
   return ((unsigned long long)key << (kIdxBits + 1)) | ((unsigned long long)(kIdxMask - flat) << 1) | sign;
 }
 
-struct __align__(16) SelectShared {
+// Shared memory of one selecting warp.  CAP: candidate buffer entries (8 bytes each); KMAX: the
+// largest k it serves.  Two sizes are in use: SelectShared (k <= 256, 13.4 KB: sixteen warps per
+// SM) and SelectSharedBig (k <= TOPLOC_MAX_K = 512, 16.5 KB: thirteen).
+template <int CAP, int KMAX>
+struct __align__(16) SelectSharedT {
+  static constexpr int kCap = CAP;
+  static constexpr int kMaxK = KMAX;
+  static constexpr int kMaxSlots = KMAX / 32;  // tail: entries a lane owns at most
+  static_assert(CAP * 8 >= 8 * KMAX * 2, "the candidate buffer holds the maxima of the first vectors");
+  static_assert(CAP >= KMAX + kThreads * 8, "a round of appends must fit after a compaction");
+  static_assert(sizeof(uint4) * kStages * kUnroll * kThreads + 8 * CAP >= 8192,
+                "ring + candidates double as the 65536-bit residue set");
+  static_assert(sizeof(uint4) * kStages * kUnroll * kThreads >= 12 * KMAX, "the ring holds three rows of KMAX words");
   uint4 ring[kStages * kUnroll * kThreads];  // tiles on their way from HBM (asynchronous copies)
-  unsigned long long cand[kCandCap];  // candidates held; ring + cand later serve as the residue set
+  unsigned long long cand[CAP];       // candidates held; ring + cand later serve as the residue set
   uint32_t hit_idx[kHitCap];          // vectors that passed the streaming filter, not yet unpacked
                                       // (index within the chunk; they are fetched again when unpacked)
   uint32_t top_hist[256];             // held candidates by the upper 8 bits of their 15-bit key; a
@@ -94,9 +102,10 @@ struct __align__(16) SelectShared {
   uint32_t bin;
   int want;
 };
+using SelectShared = SelectSharedT<TOPLOC_CAND_CAP, 256>;
+using SelectSharedBig = SelectSharedT<1024, TOPLOC_MAX_K>;
+static_assert(TOPLOC_MAX_K == 512, "SelectSharedBig is sized for k up to 512");
 constexpr uint32_t kNoBin = 0xFFFFFFFFu;
-static_assert(sizeof(uint4) * kStages * kUnroll * kThreads + 8 * kCandCap >= 8192,
-              "ring + candidates double as the 65536-bit residue set");
 
 // What the warp knows about its chunk so far.  Every lane holds the same
 // values: appends are agreed on by ballot, so the counters need no atomics.
@@ -219,8 +228,8 @@ __device__ __forceinline__ bool vector_reaches(const uint4& w, uint32_t thr, uin
 // PER_LANE * l .. PER_LANE * l + PER_LANE - 1.  Writes sh.digit (the bin, or
 // kNoBin when the histogram holds fewer than want entries), sh.bin (its
 // population) and sh.want (the rank wanted inside it).
-template <int PER_LANE>
-__device__ __forceinline__ void find_from_top(SelectShared& sh, const uint32_t* hist, int want) {
+template <int PER_LANE, class SH>
+__device__ __forceinline__ void find_from_top(SH& sh, const uint32_t* hist, int want) {
   const int lane = threadIdx.x & 31;
   warp_barrier();  // histogram updates are in; results of an earlier call have been read
   uint32_t local[PER_LANE];
@@ -261,8 +270,8 @@ __device__ __forceinline__ void find_from_top(SelectShared& sh, const uint32_t* 
 // has a higher flat index, later elements must beat it strictly.  For fp32 the
 // 15 bits are only the upper half of the key, so later elements need only
 // reach it.
-template <int DT>
-__device__ __noinline__ uint32_t raise_threshold(SelectShared& sh, int k, uint32_t thr, int count) {
+template <int DT, class SH>
+__device__ __noinline__ uint32_t raise_threshold(SH& sh, int k, uint32_t thr, int count) {
   const int lane = threadIdx.x & 31;
   if (count < k) return thr;
   find_from_top<8>(sh, sh.top_hist, k);
@@ -292,8 +301,8 @@ __device__ __noinline__ uint32_t raise_threshold(SelectShared& sh, int k, uint32
 // whole -- because exactly k candidates remain, or, for a compaction in
 // mid-stream (exact == false), because at most kMaxK remain; only the last
 // compaction of a chunk must leave exactly k.  Returns the new state.
-template <int DT>
-__device__ __noinline__ WarpState compact_candidates(SelectShared& sh, int k, WarpState st, bool exact) {
+template <int DT, class SH>
+__device__ __noinline__ WarpState compact_candidates(SH& sh, int k, WarpState st, bool exact) {
   const int lane = threadIdx.x & 31;
   const int n = st.count;
   if (n <= k) return st;
@@ -315,7 +324,7 @@ __device__ __noinline__ WarpState compact_candidates(SelectShared& sh, int k, Wa
     want = sh.want;
     const int kept = k - want + (int)sh.bin;
     // lower bits of the pivot stay 0: the boundary bin is kept whole
-    if (shift <= 24 && (kept == k || (!exact && kept <= kMaxK))) break;
+    if (shift <= 24 && (kept == k || (!exact && kept <= SH::kMaxK))) break;
   }
   const unsigned long long pivot = prefix;  // everything >= pivot is kept
   // in place, in order: a slot is overwritten only after it has been read
@@ -334,7 +343,7 @@ __device__ __noinline__ WarpState compact_candidates(SelectShared& sh, int k, Wa
   // Distinct candidates leave at most kMaxK here (exactly k when exact).  Equal candidates -- a
   // caller of the incremental entry points offering a flat index twice -- could leave more at the
   // cut; the buffer's arithmetic relies on the bound, so it is enforced.
-  out = min(out, exact ? k : kMaxK);
+  out = min(out, exact ? k : SH::kMaxK);
   // the key histograms describe the survivors only
   for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
   if (lane == 0) sh.top_bin = kNoBin;
@@ -392,8 +401,8 @@ __device__ __forceinline__ void pick_element(const uint4& w, uint32_t e, uint32_
 // lane counts its passing elements, a warp prefix sum hands out the slots (the
 // counter is warp-uniform, no atomic), then every lane stores its own few.
 // Makes room first (a mid-stream compaction) if the round would not fit.
-template <int DT, int VEC>
-__device__ __forceinline__ void append_round(SelectShared& sh, int k, WarpState& st, const uint4& w, bool valid,
+template <int DT, int VEC, class SH>
+__device__ __forceinline__ void append_round(SH& sh, int k, WarpState& st, const uint4& w, bool valid,
                                              uint32_t flat0) {
   const int lane = threadIdx.x & 31;
   uint32_t mask = 0;
@@ -408,8 +417,8 @@ __device__ __forceinline__ void append_round(SelectShared& sh, int k, WarpState&
       if (lane >= off) incl += other;
     }
     total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-    if (st.count + total <= kCandCap) break;
-    // leaves at most kMaxK and may raise the threshold; a round adds at most 32 * VEC
+    if (st.count + total <= SH::kCap) break;
+    // leaves at most SH::kMaxK and may raise the threshold; a round adds at most 32 * VEC
     st = compact_candidates<DT>(sh, k, st, false);
   }
   int pos = st.count + incl - __popc(mask);
@@ -431,8 +440,8 @@ __device__ __forceinline__ void append_round(SelectShared& sh, int k, WarpState&
 
 // Processes vectors [vb, ve) one vector per lane at a time, raising the
 // threshold after every round.
-template <int DT, int MODE>
-__device__ __noinline__ WarpState select_carefully(SelectShared& sh, const ChunkSource<DT, MODE> src, int vb,
+template <int DT, int MODE, class SH>
+__device__ __noinline__ WarpState select_carefully(SH& sh, const ChunkSource<DT, MODE> src, int vb,
                                                    int ve, int k, WarpState st) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x & 31;
@@ -454,8 +463,8 @@ __device__ __noinline__ WarpState select_carefully(SelectShared& sh, const Chunk
 // possibly higher, threshold), one vector per lane and round, then raises the
 // threshold.  Only the vector's index was parked: the 16 bytes are fetched
 // again (they were read moments ago, so this rarely reaches DRAM).
-template <int DT, int MODE>
-__device__ __noinline__ WarpState drain_hits(SelectShared& sh, const ChunkSource<DT, MODE> src, int k,
+template <int DT, int MODE, class SH>
+__device__ __noinline__ WarpState drain_hits(SH& sh, const ChunkSource<DT, MODE> src, int k,
                                              WarpState st) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x & 31;
@@ -495,8 +504,8 @@ __device__ __forceinline__ uint32_t vector_max_coarse_key(const uint4& w) {
 // element, so at least k elements of the chunk reach it and the k-th largest
 // element cannot lie below it.  Uses the candidate buffer to hold the maxima
 // and leaves the histograms empty again.
-template <int DT, int MODE>
-__device__ __noinline__ uint32_t sound_first_threshold(SelectShared& sh, const ChunkSource<DT, MODE> src,
+template <int DT, int MODE, class SH>
+__device__ __noinline__ uint32_t sound_first_threshold(SH& sh, const ChunkSource<DT, MODE> src,
                                                        int n_first, int k) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x & 31;
@@ -536,8 +545,8 @@ __device__ __noinline__ uint32_t sound_first_threshold(SelectShared& sh, const C
 // once, so the rare slow work is done with every lane busy.  Nothing here
 // waits on another warp: a chunk's serial steps only delay that chunk, while
 // the other warps of the SM keep their own loads in flight.
-template <int DT, int MODE>
-__device__ void select_topk(SelectShared& sh, const ChunkSource<DT, MODE>& src, int n_elems, int k) {
+template <int DT, int MODE, class SH>
+__device__ void select_topk(SH& sh, const ChunkSource<DT, MODE>& src, int n_elems, int k) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   constexpr int kTileVecs = kThreads * kUnroll;
   const int lane = threadIdx.x & 31;
@@ -664,8 +673,8 @@ __host__ __device__ inline size_t stream_state_stride(int k) { return sizeof(Str
 // Vectors [vb, ve) against a threshold that is already meaningful: the filter of the select kernel's
 // streaming loop (test, park the vectors that reach the threshold, unpack them by the warp), with
 // plain loads instead of the ring.
-template <int DT, int MODE>
-__device__ __forceinline__ WarpState filter_vectors(SelectShared& sh, const ChunkSource<DT, MODE>& src, int vb, int ve,
+template <int DT, int MODE, class SH>
+__device__ __forceinline__ WarpState filter_vectors(SH& sh, const ChunkSource<DT, MODE>& src, int vb, int ve,
                                                     int k, WarpState st) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x & 31;
@@ -707,8 +716,8 @@ __device__ __forceinline__ WarpState filter_vectors(SelectShared& sh, const Chun
 // ---------------------------------------------------------------------------
 __host__ __device__ inline size_t running_selection_bytes(int k) { return stream_state_stride(k); }
 
-template <int DT>
-__device__ __forceinline__ WarpState running_selection_open(SelectShared& sh, const unsigned char* state, int k) {
+template <int DT, class SH>
+__device__ __forceinline__ WarpState running_selection_open(SH& sh, const unsigned char* state, int k) {
   const int lane = threadIdx.x & 31;
   const StreamHeader* head = reinterpret_cast<const StreamHeader*>(state);
   const unsigned long long* held = reinterpret_cast<const unsigned long long*>(head + 1);
@@ -730,16 +739,16 @@ __device__ __forceinline__ WarpState running_selection_open(SelectShared& sh, co
 
 // Vectors [vb, ve) of a source against the running selection: once k candidates are held the
 // threshold does the work; before that every element is a candidate.
-template <int DT, int MODE>
-__device__ __forceinline__ WarpState running_selection_take(SelectShared& sh, WarpState st,
+template <int DT, int MODE, class SH>
+__device__ __forceinline__ WarpState running_selection_take(SH& sh, WarpState st,
                                                             const ChunkSource<DT, MODE>& src, int vb, int ve, int k) {
   if (st.count >= k) return filter_vectors<DT, MODE>(sh, src, vb, ve, k, st);
   return select_carefully<DT, MODE>(sh, src, vb, ve, k, st);
 }
 
 // tile: n_elems values whose first one has flat index flat_base within the chunk.
-template <int DT>
-__device__ __forceinline__ WarpState running_selection_offer(SelectShared& sh, WarpState st, const void* tile,
+template <int DT, class SH>
+__device__ __forceinline__ WarpState running_selection_offer(SH& sh, WarpState st, const void* tile,
                                                              int n_elems, uint32_t flat_base, int k) {
   constexpr int VEC = ChunkSource<DT, 3>::kVec;
   constexpr int kElem = ChunkSource<DT, 3>::kElemBytes;
@@ -753,8 +762,8 @@ __device__ __forceinline__ WarpState running_selection_offer(SelectShared& sh, W
   return running_selection_take<DT, 3>(sh, st, src, vb, vb + n_elems / VEC, k);
 }
 
-template <int DT>
-__device__ __forceinline__ void running_selection_close(SelectShared& sh, WarpState st, unsigned char* state, int k) {
+template <int DT, class SH>
+__device__ __forceinline__ void running_selection_close(SH& sh, WarpState st, unsigned char* state, int k) {
   const int lane = threadIdx.x & 31;
   StreamHeader* head = reinterpret_cast<StreamHeader*>(state);
   unsigned long long* held = reinterpret_cast<unsigned long long*>(head + 1);

@@ -31,7 +31,7 @@ TOPLOC_FIELD_32 = 1
 TOPLOC_FIELD_16_PADDED = 2   # validation only: fp32 activations against 16-bit field proofs
 TOPLOC_FIELD_32_PRIME = 4294967291
 TOPLOC_DTYPE_FP32 = 1
-TOPLOC_MAX_K = 256
+TOPLOC_MAX_K = 512
 TOPLOC_MAX_K_DIRECT = 4096
 TOPLOC_BUILTIN_SCRATCH_BYTES = 8 << 20
 

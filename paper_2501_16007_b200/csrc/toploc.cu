@@ -41,6 +41,9 @@ namespace {
 
 using namespace toploc_device;
 
+constexpr int kMaxK = TOPLOC_MAX_K;                 // polynomial proofs: largest k
+constexpr int kSmallMaxK = SelectShared::kMaxK;     // up to here the smaller per-warp scratch serves
+
 // ---------------------------------------------------------------------------
 // constants of the method
 // ---------------------------------------------------------------------------
@@ -62,7 +65,11 @@ constexpr int kInterpWarps = 32;         // interpolation kernel: warps per bloc
 #define TOPLOC_INTERP_CHUNKS 2
 #endif
 constexpr int kInterpChunks = TOPLOC_INTERP_CHUNKS;  // interpolation kernel: chunks a warp works on at once
-static_assert((65536 + kInterpWarps * 2 * kInterpChunks * TOPLOC_MAX_K) * 2 <= 227 * 1024,
+// k above 256: sixteen slots per lane need more registers than a 1024-thread block has, so those
+// chunks go to 512-thread blocks, one chunk per warp at a time.
+constexpr int kInterpWarpsBig = 16;
+static_assert((65536 + kInterpWarps * 2 * kInterpChunks * kSmallMaxK) * 2 <= 227 * 1024 &&
+                  (65536 + kInterpWarpsBig * 2 * kMaxK) * 2 <= 227 * 1024,
               "table of inverses + per-warp rows must fit the shared memory of one block");
 
 struct ChunkSpan {   // one per chunk of a ragged batch, built on the host
@@ -178,12 +185,14 @@ static_assert(kGenerator != 0 && mul_mod(kGenerator, kGeneratorInv) == 1u, "gene
 // memory is consumed: the tile ring and the candidate buffer become the
 // 65536-bit set of residues seen.  Run by one warp (the only one of its block
 // that is still at work).
-__device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32_t (&idx)[kMaxK / kThreads],
+template <class SH>
+__device__ uint32_t find_injective_modulus(SH& sh, int k, const uint32_t (&idx)[SH::kMaxK / kThreads],
                                            bool wide_field) {
+  constexpr int kOwned = SH::kMaxK / kThreads;
   const int lane = threadIdx.x & 31;
-  uint32_t res[kMaxK / kThreads];
+  uint32_t res[kOwned];
 #pragma unroll
-  for (int e = 0; e < kMaxK / kThreads; ++e) res[e] = 0;
+  for (int e = 0; e < kOwned; ++e) res[e] = 0;
   warp_barrier();  // every lane has taken its candidates out of sh.cand
   uint32_t* seen = reinterpret_cast<uint32_t*>(sh.ring);  // ring and cand are adjacent: 11 KB
   for (int i = lane; i < 2048; i += kThreads) seen[i] = 0;
@@ -193,7 +202,7 @@ __device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32
   for (uint32_t m = kModHigh; m >= kModLow; --m) {
     uint32_t dup = 0;
 #pragma unroll
-    for (int e = 0; e < kMaxK / kThreads; ++e) {
+    for (int e = 0; e < kOwned; ++e) {
       int j = lane + e * kThreads;
       if (j < k) {
         uint32_t r = idx[e] % m;
@@ -205,7 +214,7 @@ __device__ uint32_t find_injective_modulus(SelectShared& sh, int k, const uint32
     }
     const bool clash = __any_sync(0xFFFFFFFFu, dup != 0);  // also orders the set's updates before its clearing
 #pragma unroll
-    for (int e = 0; e < kMaxK / kThreads; ++e) {
+    for (int e = 0; e < kOwned; ++e) {
       int j = lane + e * kThreads;
       if (j < k) seen[res[e] >> 5] = 0;
     }
@@ -247,13 +256,17 @@ __device__ __forceinline__ ChunkPlace locate_chunk(const BatchParams& bp, long l
 // select kernel: topk() of Algorithms 1 and 2, one chunk per block; for proof
 // generation (sel.proofs != nullptr) also findInjectiveModulus() of Algorithm 1.
 // ---------------------------------------------------------------------------
-template <int DT>
-__device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchParams& bp, long long chunk,
+template <int DT, class SH>
+__device__ __forceinline__ void publish_selection(SH& sh, const BatchParams& bp, long long chunk,
                                                   const Selection& sel);
 
-template <int DT, int MODE>
-__global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_select_kernel(BatchParams bp, Selection sel) {
-  __shared__ SelectShared sh;
+// one-warp blocks per SM the launch bound asks for (shared memory allows one or two more)
+template <class SH>
+constexpr int select_min_blocks() { return SH::kMaxK > 256 ? 13 : TOPLOC_SELECT_MIN_BLOCKS; }
+
+template <int DT, int MODE, class SH>
+__global__ void __launch_bounds__(kThreads, select_min_blocks<SH>()) toploc_select_kernel(BatchParams bp, Selection sel) {
+  __shared__ SH sh;
   const int tid = threadIdx.x;
   const long long chunk = blockIdx.x;
   const int k = bp.k;
@@ -283,8 +296,8 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_sel
 // The chunk's selection (sh.cand[0..k)) goes to the interpolation kernel: indices
 // and patterns to scratch, rank order where the caller asked for indices, and
 // for proof generation the modulus (Algorithm 6) and the chunk's status.
-template <int DT>
-__device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchParams& bp, long long chunk,
+template <int DT, class SH>
+__device__ __forceinline__ void publish_selection(SH& sh, const BatchParams& bp, long long chunk,
                                                   const Selection& sel) {
   const int tid = threadIdx.x;
   const int k = bp.k;
@@ -318,9 +331,9 @@ __device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchP
     return;
   }
   const bool nonfinite = __any_sync(0xFFFFFFFFu, unrepresentable != 0);
-  uint32_t picked[kMaxK / kThreads];
+  uint32_t picked[SH::kMaxK / kThreads];
 #pragma unroll
-  for (int e = 0; e < kMaxK / kThreads; ++e) {
+  for (int e = 0; e < SH::kMaxK / kThreads; ++e) {
     const int j = tid + e * kThreads;
     picked[e] = j < k ? kIdxMask - ((uint32_t)(sh.cand[j] >> 1) & kIdxMask) : 0u;
   }
@@ -343,7 +356,7 @@ __device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchP
 
 // Algorithm 3 for NCH chunks of one warp at a time (their dependency chains are
 // independent, which keeps the issue slots filled).  inv[] is the table of
-// inverses in Z_p; xa is this warp's scratch (NCH rows of kMaxK words: x_i in the
+// inverses in Z_p; xa is this warp's scratch (NCH rows of ROW words: x_i in the
 // lower half of word i, the Newton coefficient a_i in the upper half).  A chunk
 // that is not live is carried along with zeros and not written.
 //
@@ -362,7 +375,7 @@ __device__ __forceinline__ void publish_selection(SelectShared& sh, const BatchP
 // against 0.39 ms this way, which is bound by the integer-multiply pipe.)
 // The Newton form is then multiplied out from the inside,
 //   P <- a_{k-1};  P <- P * (x - x_i) + a_i  for i = k-2 .. 0.
-template <int SLOTS, int NCH>
+template <int SLOTS, int NCH, int ROW>
 __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t* xa, int k, const Selection& sel,
                                                    const long long (&chunk)[NCH], const bool (&live)[NCH]) {
   const int lane = threadIdx.x & 31;
@@ -407,7 +420,7 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t
         const uint32_t ti = __shfl_sync(kFull, t[c][b], ii);
         const uint32_t xi = __shfl_sync(kFull, x[c][b], ii);
         const uint32_t a = mul_mod(ti, inv[ni]);  // n_i != 0: the x are distinct (Algorithm 6)
-        if (lane == 0) xa[c * kMaxK + i] = xi | (a << 16);
+        if (lane == 0) xa[c * ROW + i] = xi | (a << 16);
         neg_a[c] = kPrime - a;
         neg_x[c] = kPrime - xi;
       }
@@ -440,7 +453,7 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t
   for (int c = 0; c < NCH; ++c) {
 #pragma unroll
     for (int b = 0; b < SLOTS; ++b) co[c][b] = 0;
-    if (lane == 0) co[c][0] = xa[c * kMaxK + k - 1] >> 16;
+    if (lane == 0) co[c][0] = xa[c * ROW + k - 1] >> 16;
   }
   const int from = (lane + 31) & 31;
 #pragma unroll
@@ -451,7 +464,7 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t
       const int i = k - 1 - D;
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
-        const uint32_t pair = xa[c * kMaxK + i];
+        const uint32_t pair = xa[c * ROW + i];
         const uint32_t neg_x = kPrime - (pair & 0xFFFFu);  // p for x_i = 0, which multiplies like 0
         uint32_t below[SLOTS];  // coefficient d - 1, as seen from the owner of coefficient d
 #pragma unroll
@@ -481,21 +494,26 @@ __device__ __forceinline__ void interpolate_chunks(const uint16_t* inv, uint32_t
 // select kernel finished.  Each block first fills a table of all inverses in
 // Z_p (walking the powers of a generator forwards and backwards), then every
 // warp takes chunks in turn, kInterpChunks at a time.
-__global__ void __launch_bounds__(kInterpWarps * 32, 1)
+// WARPS x 32 threads per block, ROW = the largest k of the instantiation: 32 warps and 256 for
+// k <= 256 (two chunks per warp at a time up to k = 128), 16 warps and 512 above.
+template <int WARPS, int ROW>
+__global__ void __launch_bounds__(WARPS * 32, 1)
 toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
+  constexpr int NCH = ROW > 256 ? 1 : kInterpChunks;  // chunks a warp works on at once
   extern __shared__ __align__(16) uint16_t dyn_smem[];
   uint16_t* inv = dyn_smem;                               // 65536 entries
-  uint16_t* scratch = dyn_smem + 65536;                   // 2 * kInterpChunks rows of kMaxK per warp
+  uint16_t* scratch = dyn_smem + 65536;                   // NCH rows of ROW words per warp
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   {
-    // thread t owns exponents 64t .. 64t + 63 of the generator
-    const uint32_t e0 = (uint32_t)tid * 64u;
+    // thread t owns a run of consecutive exponents of the generator
+    constexpr uint32_t kRun = 65536u / (WARPS * 32);
+    const uint32_t e0 = (uint32_t)tid * kRun;
     uint32_t a = pow_mod(kGenerator, e0);
     uint32_t b = pow_mod(kGeneratorInv, e0);
     if (tid == 0) inv[0] = 0;
 #pragma unroll 4
-    for (int i = 0; i < 64; ++i) {
+    for (uint32_t i = 0; i < kRun; ++i) {
       if (e0 + i < kPrime - 1) inv[a] = (uint16_t)b;
       a = mul_mod(a, kGenerator);
       b = mul_mod(b, kGeneratorInv);
@@ -503,17 +521,16 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
   }
   __syncthreads();
   wait_for_previous_grid();  // the selections and moduli are in place
-  uint32_t* xa = reinterpret_cast<uint32_t*>(scratch) + warp * kInterpChunks * kMaxK;
-  const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
+  uint32_t* xa = reinterpret_cast<uint32_t*>(scratch) + warp * NCH * ROW;
+  const long long groups = (num_chunks + NCH - 1) / NCH;
   // group g goes to block g % gridDim.x, so a small batch spreads over the blocks before it fills their warps
-  for (long long g = blockIdx.x + (long long)gridDim.x * warp; g < groups;
-       g += (long long)gridDim.x * kInterpWarps) {
-    long long chunk[kInterpChunks];
-    bool live[kInterpChunks];
+  for (long long g = blockIdx.x + (long long)gridDim.x * warp; g < groups; g += (long long)gridDim.x * WARPS) {
+    long long chunk[NCH];
+    bool live[NCH];
     bool any = false;
 #pragma unroll
-    for (int c = 0; c < kInterpChunks; ++c) {
-      chunk[c] = g * kInterpChunks + c;
+    for (int c = 0; c < NCH; ++c) {
+      chunk[c] = g * NCH + c;
       live[c] = false;
       if (chunk[c] < num_chunks) {
         const uint8_t st = sel.status[chunk[c]];
@@ -522,16 +539,20 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
       any |= live[c];
     }
     if (!any) continue;
-    if (k <= 32) interpolate_chunks<1, kInterpChunks>(inv, xa, k, sel, chunk, live);
-    else if (k <= 64) interpolate_chunks<2, kInterpChunks>(inv, xa, k, sel, chunk, live);
-    else if (k <= 128) interpolate_chunks<4, kInterpChunks>(inv, xa, k, sel, chunk, live);
-    else {
-      // eight slots per lane: one chunk at a time keeps the state in registers
+    if constexpr (ROW > 256) {
+      interpolate_chunks<ROW / 32, 1, ROW>(inv, xa, k, sel, chunk, live);
+    } else {
+      if (k <= 32) interpolate_chunks<1, NCH, ROW>(inv, xa, k, sel, chunk, live);
+      else if (k <= 64) interpolate_chunks<2, NCH, ROW>(inv, xa, k, sel, chunk, live);
+      else if (k <= 128) interpolate_chunks<4, NCH, ROW>(inv, xa, k, sel, chunk, live);
+      else {
+        // eight slots per lane: one chunk at a time keeps the state in registers
 #pragma unroll
-      for (int c = 0; c < kInterpChunks; ++c) {
-        const long long one_chunk[1] = {chunk[c]};
-        const bool one_live[1] = {live[c]};
-        if (live[c]) interpolate_chunks<kMaxSlots, 1>(inv, xa, k, sel, one_chunk, one_live);
+        for (int c = 0; c < NCH; ++c) {
+          const long long one_chunk[1] = {chunk[c]};
+          const bool one_live[1] = {live[c]};
+          if (live[c]) interpolate_chunks<8, 1, ROW>(inv, xa, k, sel, one_chunk, one_live);
+        }
       }
     }
   }
@@ -540,15 +561,15 @@ toploc_interpolate_kernel(Selection sel, int k, long long num_chunks) {
 // decode(), Horner evaluation (Algorithm 5), extractBits(), the error
 // accumulation and the verdict of Algorithm 2 for one chunk, by the warp that
 // selected it.  res arrives initialised and with the decoded modulus.
-template <int SLOTS>
-__device__ __forceinline__ void evaluate_warp(SelectShared& sh, int k, long long chunk, const uint32_t (&idx)[SLOTS],
+template <int SLOTS, class SH>
+__device__ __forceinline__ void evaluate_warp(SH& sh, int k, long long chunk, const uint32_t (&idx)[SLOTS],
                                               const uint32_t (&bits)[SLOTS], const VerifyIo& io,
                                               toploc_chunk_result res) {
   const int lane = threadIdx.x;
   const uint16_t* proof = reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + 2 * (size_t)k));
   // the selection has left shared memory (it is in idx / bits), so the ring is free
-  uint32_t* coef = reinterpret_cast<uint32_t*>(sh.ring);  // kMaxK words
-  uint32_t* gen = coef + kMaxK;                           // kMaxK words
+  uint32_t* coef = reinterpret_cast<uint32_t*>(sh.ring);  // SH::kMaxK words
+  uint32_t* gen = coef + SH::kMaxK;                       // SH::kMaxK words
   uint32_t* hist = sh.top_hist;                           // a 7-bit mantissa difference is at most 127
   const toploc_thresholds thr = thresholds_of(io, chunk);
   warp_barrier();
@@ -805,7 +826,8 @@ toploc_interpolate_q_kernel(Selection sel, int k, long long num_chunks) {
   if (k <= 32) interpolate_chunk_q<1>(sel, k, chunk, rows[warp]);
   else if (k <= 64) interpolate_chunk_q<2>(sel, k, chunk, rows[warp]);
   else if (k <= 128) interpolate_chunk_q<4>(sel, k, chunk, rows[warp]);
-  else interpolate_chunk_q<kMaxSlots>(sel, k, chunk, rows[warp]);
+  else if (k <= 256) interpolate_chunk_q<8>(sel, k, chunk, rows[warp]);
+  else interpolate_chunk_q<kMaxK / 32>(sel, k, chunk, rows[warp]);
 }
 
 // Algorithm 2 after the selection, over Z_q, for one chunk whose selected
@@ -816,8 +838,8 @@ toploc_interpolate_q_kernel(Selection sel, int k, long long num_chunks) {
 // PADDED: the proof is a 16-bit field proof (a bf16 generator's); the polynomial is evaluated
 // over Z_p and the committed 16-bit pattern padded with 16 zero bits before the comparison
 // (Section 5.6, fp32 validator of a bf16 model).
-template <int SLOTS, bool PADDED>
-__device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long long chunk, const uint32_t (&idx)[SLOTS],
+template <int SLOTS, bool PADDED, class SH>
+__device__ __forceinline__ void evaluate_warp_q(SH& sh, int k, long long chunk, const uint32_t (&idx)[SLOTS],
                                                 const uint32_t (&pattern)[SLOTS], const VerifyIo& io,
                                                 toploc_chunk_result res) {
   const int lane = threadIdx.x;
@@ -825,8 +847,8 @@ __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long lo
       reinterpret_cast<const uint16_t*>(io.proofs + chunk * (2 + (PADDED ? 2 : 4) * (size_t)k));
   // the selection has left shared memory, so the ring is free: three rows of kMaxK words
   uint32_t* coef = reinterpret_cast<uint32_t*>(sh.ring);
-  uint32_t* gen = coef + kMaxK;
-  uint32_t* diffs = gen + kMaxK;
+  uint32_t* gen = coef + SH::kMaxK;
+  uint32_t* diffs = gen + SH::kMaxK;
   constexpr uint32_t kNoMatch = 0xFFFFFFFFu;  // larger than any 23-bit difference
   const toploc_thresholds thr = thresholds_of(io, chunk);
   warp_barrier();
@@ -927,8 +949,8 @@ __device__ __forceinline__ void evaluate_warp_q(SelectShared& sh, int k, long lo
   }
 }
 
-template <int DT, int SLOTS>
-__device__ __forceinline__ void verify_chunk(SelectShared& sh, int k, bool wide, bool padded, long long chunk,
+template <int DT, int SLOTS, class SH>
+__device__ __forceinline__ void verify_chunk(SH& sh, int k, bool wide, bool padded, long long chunk,
                                              const VerifyIo& io, const toploc_chunk_result& res) {
   const int lane = threadIdx.x;
   uint32_t idx[SLOTS], bits[SLOTS];
@@ -991,9 +1013,9 @@ __device__ __forceinline__ bool decode_proof(const VerifyIo& io, long long chunk
 // verdict by the same warp.  Validation needs no scratch memory beyond the row
 // table of a ragged batch.
 // ---------------------------------------------------------------------------
-template <int DT, int MODE>
-__global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_verify_kernel(BatchParams bp, VerifyIo io) {
-  __shared__ SelectShared sh;
+template <int DT, int MODE, class SH>
+__global__ void __launch_bounds__(kThreads, select_min_blocks<SH>()) toploc_verify_kernel(BatchParams bp, VerifyIo io) {
+  __shared__ SH sh;
   const int tid = threadIdx.x;
   const long long chunk = blockIdx.x;
   const int k = bp.k;
@@ -1016,10 +1038,14 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
 
   const bool padded = bp.padded != 0;
   const bool wide = bp.coef_bytes == 4 || padded;  // whole patterns are compared
-  if (k <= 32) verify_chunk<DT, 1>(sh, k, wide, padded, chunk, io, res);
-  else if (k <= 64) verify_chunk<DT, 2>(sh, k, wide, padded, chunk, io, res);
-  else if (k <= 128) verify_chunk<DT, 4>(sh, k, wide, padded, chunk, io, res);
-  else verify_chunk<DT, kMaxSlots>(sh, k, wide, padded, chunk, io, res);
+  if constexpr (SH::kMaxK > 256) {
+    verify_chunk<DT, SH::kMaxSlots>(sh, k, wide, padded, chunk, io, res);  // launched for k above 256 only
+  } else {
+    if (k <= 32) verify_chunk<DT, 1>(sh, k, wide, padded, chunk, io, res);
+    else if (k <= 64) verify_chunk<DT, 2>(sh, k, wide, padded, chunk, io, res);
+    else if (k <= 128) verify_chunk<DT, 4>(sh, k, wide, padded, chunk, io, res);
+    else verify_chunk<DT, 8>(sh, k, wide, padded, chunk, io, res);
+  }
 }
 
 // ---------------------------------------------------------------------------
@@ -1034,18 +1060,18 @@ __global__ void __launch_bounds__(kThreads, TOPLOC_SELECT_MIN_BLOCKS) toploc_ver
 // TAIL: 0 hand the selection out, 1 proof generation (also the modulus),
 // 2 validation.
 // ---------------------------------------------------------------------------
-template <int DT, int TAIL, int SLOTS>
-__device__ __forceinline__ void finish_merged(SelectShared& sh, const BatchParams& bp, long long chunk,
+template <int DT, int TAIL, int SLOTS, class SH>
+__device__ __forceinline__ void finish_merged(SH& sh, const BatchParams& bp, long long chunk,
                                               const Selection& sel, const VerifyIo& io,
                                               const toploc_chunk_result& res) {
   const int lane = threadIdx.x;
   const int k = bp.k;
   const bool padded = DT == 1 && TAIL == 2 && bp.padded != 0;
   const bool wide = DT == 1 && (bp.coef_bytes == 4 || padded);
-  uint32_t idx[kMaxK / kThreads], bits[SLOTS];
+  uint32_t idx[SH::kMaxK / kThreads], bits[SLOTS];
   uint32_t unrepresentable = 0;
 #pragma unroll
-  for (int e = 0; e < kMaxK / kThreads; ++e) idx[e] = 0;
+  for (int e = 0; e < SH::kMaxK / kThreads; ++e) idx[e] = 0;
 #pragma unroll
   for (int e = 0; e < SLOTS; ++e) {
     const int j = e * 32 + lane;
@@ -1099,7 +1125,7 @@ constexpr int kMergeThreads = 256;  // merge kernel: the passes over a chunk's w
 template <int DT, int TAIL>
 __global__ void __launch_bounds__(kMergeThreads)
 toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) {
-  __shared__ SelectShared sh;
+  __shared__ SelectSharedBig sh;  // (one block per chunk: the larger scratch costs nothing here)
   __shared__ int kept;     // words taken so far
   __shared__ int proceed;  // decode() found the proof well-formed
   const int tid = threadIdx.x;
@@ -1194,7 +1220,8 @@ toploc_merge_kernel(BatchParams bp, MergeParams mp, Selection sel, VerifyIo io) 
   if (k <= 32) finish_merged<DT, TAIL, 1>(sh, bp, chunk, sel, io, res);
   else if (k <= 64) finish_merged<DT, TAIL, 2>(sh, bp, chunk, sel, io, res);
   else if (k <= 128) finish_merged<DT, TAIL, 4>(sh, bp, chunk, sel, io, res);
-  else finish_merged<DT, TAIL, kMaxSlots>(sh, bp, chunk, sel, io, res);
+  else if (k <= 256) finish_merged<DT, TAIL, 8>(sh, bp, chunk, sel, io, res);
+  else finish_merged<DT, TAIL, kMaxK / 32>(sh, bp, chunk, sel, io, res);
 }
 
 // ---------------------------------------------------------------------------
@@ -1212,7 +1239,7 @@ toploc_stream_append_kernel(const char* rows, long long row_stride, int hidden, 
                             unsigned char* state) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   constexpr int kElem = DT == 0 ? 2 : 4;
-  __shared__ SelectShared sh;
+  __shared__ SelectSharedBig sh;
   const long long seq = blockIdx.x;
   unsigned char* mine = state + seq * stream_state_stride(k);
   WarpState st = running_selection_open<DT>(sh, mine, k);
@@ -1232,7 +1259,7 @@ toploc_stream_append_kernel(const char* rows, long long row_stride, int hidden, 
 template <int DT>
 __global__ void __launch_bounds__(kThreads) toploc_stream_finish_kernel(BatchParams bp, Selection sel,
                                                                         const unsigned char* state) {
-  __shared__ SelectShared sh;
+  __shared__ SelectSharedBig sh;
   const int lane = threadIdx.x;
   const long long seq = blockIdx.x;
   const int k = bp.k;
@@ -1355,7 +1382,11 @@ struct DeviceInfo {
 constexpr size_t kBuiltinScratchBytes = TOPLOC_BUILTIN_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
 
-size_t interp_smem_bytes() { return (65536 + (size_t)kInterpWarps * 2 * kInterpChunks * kMaxK) * sizeof(uint16_t); }
+// table of inverses + the warps' rows (x_i and a_i as one 32-bit word per point)
+size_t interp_smem_bytes(bool big) {
+  const size_t row_words = big ? (size_t)kInterpWarpsBig * kMaxK : (size_t)kInterpWarps * kInterpChunks * kSmallMaxK;
+  return (65536 + 2 * row_words) * sizeof(uint16_t);
+}
 
 // Per-device facts, looked up on a device's first call.  Host threads may call
 // the library concurrently: the table is filled under a lock.
@@ -1376,8 +1407,10 @@ int device_info(DeviceInfo** out) {
   }
   if (d.major != 10) return TOPLOC_ERR_ARCH;
   if (!d.interp_smem_set) {
-    if (cudaFuncSetAttribute(toploc_interpolate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)interp_smem_bytes()) != cudaSuccess)
+    if (cudaFuncSetAttribute(toploc_interpolate_kernel<kInterpWarps, kSmallMaxK>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)interp_smem_bytes(false)) != cudaSuccess ||
+        cudaFuncSetAttribute(toploc_interpolate_kernel<kInterpWarpsBig, kMaxK>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)interp_smem_bytes(true)) != cudaSuccess)
       return TOPLOC_ERR_CUDA;
     d.interp_smem_set = true;
   }
@@ -1500,18 +1533,31 @@ int upload_spans(const toploc_layout* lay, const HostPlan& plan, void* d_spans, 
   return err == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
+// k above 256 takes the kernels built around the larger per-warp scratch.
+template <int DT, class SH>
+void launch_select_sized(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const Selection& sel) {
+  if (mode == 0) toploc_select_kernel<DT, 0, SH><<<grid, kThreads, 0, stream>>>(bp, sel);
+  else if (mode == 1) toploc_select_kernel<DT, 1, SH><<<grid, kThreads, 0, stream>>>(bp, sel);
+  else toploc_select_kernel<DT, 2, SH><<<grid, kThreads, 0, stream>>>(bp, sel);
+}
+
 template <int DT>
 void launch_select(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const Selection& sel) {
-  if (mode == 0) toploc_select_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, sel);
-  else if (mode == 1) toploc_select_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, sel);
-  else toploc_select_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, sel);
+  if (bp.k > kSmallMaxK) launch_select_sized<DT, SelectSharedBig>(mode, grid, stream, bp, sel);
+  else launch_select_sized<DT, SelectShared>(mode, grid, stream, bp, sel);
+}
+
+template <int DT, class SH>
+void launch_verify_sized(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const VerifyIo& io) {
+  if (mode == 0) toploc_verify_kernel<DT, 0, SH><<<grid, kThreads, 0, stream>>>(bp, io);
+  else if (mode == 1) toploc_verify_kernel<DT, 1, SH><<<grid, kThreads, 0, stream>>>(bp, io);
+  else toploc_verify_kernel<DT, 2, SH><<<grid, kThreads, 0, stream>>>(bp, io);
 }
 
 template <int DT>
 void launch_verify(int mode, unsigned grid, cudaStream_t stream, const BatchParams& bp, const VerifyIo& io) {
-  if (mode == 0) toploc_verify_kernel<DT, 0><<<grid, kThreads, 0, stream>>>(bp, io);
-  else if (mode == 1) toploc_verify_kernel<DT, 1><<<grid, kThreads, 0, stream>>>(bp, io);
-  else toploc_verify_kernel<DT, 2><<<grid, kThreads, 0, stream>>>(bp, io);
+  if (bp.k > kSmallMaxK) launch_verify_sized<DT, SelectSharedBig>(mode, grid, stream, bp, io);
+  else launch_verify_sized<DT, SelectShared>(mode, grid, stream, bp, io);
 }
 
 template <int DT>
@@ -1681,20 +1727,22 @@ void launch_interpolation(const toploc_layout* lay, const DeviceInfo* dev, const
   }
   // one block per SM; a small batch gets a block for every four of its groups (each block first
   // builds its table of inverses, so not one per group)
-  const long long groups = (num_chunks + kInterpChunks - 1) / kInterpChunks;
+  const bool big = lay->k > kSmallMaxK;
+  const long long groups = big ? num_chunks : (num_chunks + kInterpChunks - 1) / kInterpChunks;
   long long blocks = (groups + 3) / 4;
   if (blocks > dev->sms) blocks = dev->sms;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)blocks);
-  cfg.blockDim = dim3(kInterpWarps * 32);
-  cfg.dynamicSmemBytes = interp_smem_bytes();
+  cfg.blockDim = dim3((big ? kInterpWarpsBig : kInterpWarps) * 32);
+  cfg.dynamicSmemBytes = interp_smem_bytes(big);
   cfg.stream = stream;
   cudaLaunchAttribute early[1];
   early[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see wait_for_previous_grid()
   early[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = early;
   cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, toploc_interpolate_kernel, sel, lay->k, num_chunks);
+  if (big) cudaLaunchKernelEx(&cfg, toploc_interpolate_kernel<kInterpWarpsBig, kMaxK>, sel, lay->k, num_chunks);
+  else cudaLaunchKernelEx(&cfg, toploc_interpolate_kernel<kInterpWarps, kSmallMaxK>, sel, lay->k, num_chunks);
 }
 
 }  // namespace

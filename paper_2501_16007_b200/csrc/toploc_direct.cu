@@ -1035,7 +1035,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
 
 
 // ---------------------------------------------------------------------------
-// Small k (k <= TOPLOC_MAX_K, chunks of at most 2^19 elements): one warp per chunk, the
+// Small k (k <= 256, chunks of at most 2^19 elements): one warp per chunk, the
 // selection of the proof path (toploc_device::select_topk: the chunk streams once through the
 // warp's ring, the exact top-k ends up in shared memory), sixteen chunks per SM in flight and
 // nothing that waits on another warp.  The commitment is the selection sorted by index; the
@@ -1044,7 +1044,8 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
 namespace small_k {
 using namespace toploc_device;
 
-constexpr int kSlots = TOPLOC_MAX_K / 32;
+constexpr int kSmallK = SelectShared::kMaxK;   // 256: the per-warp scratch of sixteen warps per SM
+constexpr int kSlots = kSmallK / 32;
 constexpr long long kMaxElems = 1ll << 19;
 
 template <int DT, int MODE>
@@ -1131,7 +1132,7 @@ __global__ void __launch_bounds__(32, 15) toploc_direct_verify_warp_kernel(Direc
   }
   // the selection is in registers: the ring holds the commitment, the histograms the statistics
   uint32_t* com_idx = reinterpret_cast<uint32_t*>(sh.ring);
-  uint32_t* com_pat = com_idx + TOPLOC_MAX_K;
+  uint32_t* com_pat = com_idx + kSmallK;
   uint32_t* hist = sh.top_hist;  // a 7-bit mantissa difference is at most 127
   warp_barrier();
   const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
@@ -1254,7 +1255,7 @@ inline int layout_mode(const void* act, const toploc_layout* lay) {
 
 inline bool applies(const toploc_layout* lay) {
   const long long rows = lay->tokens_per_seq < lay->chunk_len ? lay->tokens_per_seq : lay->chunk_len;
-  return lay->k <= TOPLOC_MAX_K && rows * lay->hidden <= kMaxElems;
+  return lay->k <= kSmallK && rows * lay->hidden <= kMaxElems;
 }
 
 template <int DT>

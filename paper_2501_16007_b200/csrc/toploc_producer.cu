@@ -42,7 +42,7 @@ toploc_rmsnorm_append_kernel(const uint4* x, long long x_row_vecs, const uint4* 
                              long long y_row_vecs, int hidden, int k, int token, unsigned char* state) {
   extern __shared__ __align__(16) unsigned char dyn[];
   uint4* tile = reinterpret_cast<uint4*>(dyn);  // the row: x first, then y in place
-  __shared__ SelectShared sh;
+  __shared__ SelectSharedBig sh;  // serves every k up to TOPLOC_MAX_K
   __shared__ float partial[kNormThreads / 32];
   const int tid = threadIdx.x;
   const long long seq = blockIdx.x;

@@ -56,6 +56,13 @@ def test_long_chunk_with_padded_rows_and_with_unaligned_rows():
     parity_case(odd, 6000, 256, 1, 6000, where="unaligned")
 
 
+def test_long_chunk_with_the_largest_k():
+    """A prompt-sized chunk (selected in segments, merged) at k = 512: the segments and the merge
+    take the larger scratch and sixteen points per lane."""
+    act = synth.make_activations(1, 300, 4096, torch.bfloat16, seed=44, device=DEV, outliers="none")
+    parity_case(act, 300, 512, 1, 300, where="long k512")
+
+
 def test_selection_entry_point_on_a_long_chunk():
     act = synth.make_activations(1, 520, 4096, torch.float32, seed=39, device=DEV, outliers="none")
     lay, _ = tl.make_layout(act, 520, 128, 1, 520)

@@ -41,6 +41,24 @@ def test_small_shapes(hidden, rows, chunk_len, k, dtype):
                 where="H%d L%d k%d %s" % (hidden, chunk_len, k, dtype))
 
 
+@pytest.mark.parametrize("dtype,wide", [(torch.bfloat16, False), (torch.float32, False), (torch.float32, True)])
+def test_k_512(dtype, wide):
+    """The largest k of the polynomial proofs: Algorithm 6 still finds a modulus for 512 indices (a
+    given candidate separates them with probability about exp(-k^2 / 2m) = 0.13), the kernels take
+    their larger per-warp scratch and sixteen points per lane.  Proofs of 2 + 2k = 1026 bytes."""
+    S, T, H, L, k = 2, 96, 4096, 32, 512
+    act = synth.make_activations(S, T, H, dtype, seed=77, device=DEV, outliers="jitter")
+    noisy = synth.honest_noise(act, seed=78, rel=2.0 ** (-22 if wide else -8))
+    other = synth.make_activations(S, T, H, dtype, seed=79, device=DEV, outliers="jitter")
+    r, v = parity_case(act, L, k, S, T, recomputed={"honest": noisy, "other": other}, where="k512 %s" % dtype,
+                       wide=wide)
+    assert r[0].shape == (6, 2 + (4 if wide else 2) * k) and not r[1].any()
+    assert v["same"]["accept"].all() and not v["other"]["accept"].any()
+    # ragged tail, padded rows and a k between the two scratch sizes' limits
+    wide_rows = synth.make_activations(1, 70, 2048 + 64, dtype, seed=80, device=DEV, outliers="none")
+    parity_case(wide_rows[:, :2048], 32, 300, 1, 70, where="k300 strided %s" % dtype, wide=wide)
+
+
 @pytest.mark.parametrize("outliers", ["fixed", "none"])
 def test_outlier_recipes(outliers):
     act = synth.make_activations(3, 64, 4096, torch.bfloat16, seed=3, device=DEV, outliers=outliers)

@@ -39,7 +39,8 @@ def decode_with_fused_commit(x, weight, eps, num_seqs, tokens, k, pad=0):
 @pytest.mark.parametrize("hidden,tokens,k,pad,outliers", [
     (4096, 32, 128, 0, "fixed"),      # the paper's interval at the 8B hidden size
     (8192, 32, 128, 0, "jitter"),     # 70B hidden size
-    (2048, 32, 256, 8, "none"),       # padded step buffers, the largest k
+    (2048, 32, 256, 8, "none"),       # padded step buffers
+    (4096, 16, 512, 0, "jitter"),     # the largest k
     (1000, 5, 64, 0, "none"),         # rows that are not a multiple of 32 vectors
     (64, 3, 256, 0, "none"),          # fewer than k elements in the whole chunk: status, zero proof
 ])

@@ -40,6 +40,7 @@ def stream_chunks(act, num_seqs, tokens, k, field=0, pad=0):
     (torch.float32, 0, 2048, 32, 128, "jitter"),
     (torch.float32, 1, 2048, 32, 128, "jitter"),     # whole patterns over the 32-bit field
     (torch.bfloat16, 0, 64, 3, 256, "none"),         # fewer than k elements: status, zero proof
+    (torch.bfloat16, 0, 2048, 32, 512, "jitter"),    # the largest k
 ])
 def test_streamed_chunks_equal_the_batch_path_and_the_oracle(dtype, field, hidden, tokens, k, outliers):
     S = 5

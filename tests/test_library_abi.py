@@ -113,7 +113,7 @@ def test_long_chunks_are_planned_in_segments():
                                                    ctypes.c_void_p(16), None, None) == -2
 
 
-@pytest.mark.parametrize("bad", [dict(k=0), dict(k=257), dict(hidden=0), dict(chunk_len=0), dict(num_seqs=0),
+@pytest.mark.parametrize("bad", [dict(k=0), dict(k=513), dict(hidden=0), dict(chunk_len=0), dict(num_seqs=0),
                                  dict(dtype=7), dict(row_stride=100), dict(tokens_per_seq=0),
                                  dict(field=1), dict(field=2), dict(dtype=1, field=3), dict(dtype=1, field=-1),
                                  dict(hidden=1 << 20, chunk_len=2048, tokens_per_seq=4096, row_stride=1 << 20),
