@@ -1035,18 +1035,20 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
 
 
 // ---------------------------------------------------------------------------
-// Small k (k <= 256, chunks of at most 2^19 elements): one warp per chunk, the
+// Small k (k <= TOPLOC_MAX_K = 512, chunks of at most 2^19 elements): one warp per chunk, the
 // selection of the proof path (toploc_device::select_topk: the chunk streams once through the
 // warp's ring, the exact top-k ends up in shared memory), sixteen chunks per SM in flight and
-// nothing that waits on another warp.  The commitment is the selection sorted by index; the
-// validation looks every selected index up in the commitment.
+// nothing that waits on another warp (thirteen with the larger scratch of k > 256).  The
+// commitment is the selection sorted by index; the validation looks every selected index up in
+// the commitment.
 // ---------------------------------------------------------------------------
 namespace small_k {
 using namespace toploc_device;
 
-constexpr int kSmallK = SelectShared::kMaxK;   // 256: the per-warp scratch of sixteen warps per SM
-constexpr int kSlots = kSmallK / 32;
+constexpr int kSmallK = SelectSharedBig::kMaxK;  // 512; k <= 256 takes the smaller scratch (sixteen warps per SM)
 constexpr long long kMaxElems = 1ll << 19;
+template <class SH>
+constexpr int min_blocks() { return SH::kMaxK > 256 ? 13 : 15; }
 
 template <int DT, int MODE>
 __device__ __forceinline__ ChunkSource<DT, MODE> source_of(const DirectParams& p, long long chunk, long long* n_elems) {
@@ -1072,9 +1074,10 @@ __device__ __forceinline__ void unpack(unsigned long long c, uint32_t* flat, uin
   *pattern = (sign << 15) | (DT == 0 ? key : key >> 16);
 }
 
-template <int DT, int MODE>
-__global__ void __launch_bounds__(32, 15) toploc_direct_commit_warp_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
-  __shared__ SelectShared sh;
+template <int DT, int MODE, class SH>
+__global__ void __launch_bounds__(32, min_blocks<SH>()) toploc_direct_commit_warp_kernel(DirectParams p, uint8_t* commits,
+                                                                                         uint8_t* status) {
+  __shared__ SH sh;
   const int lane = threadIdx.x;
   const long long chunk = blockIdx.x;
   const int k = p.k;
@@ -1087,13 +1090,41 @@ __global__ void __launch_bounds__(32, 15) toploc_direct_commit_warp_kernel(Direc
     return;
   }
   select_topk<DT, MODE>(sh, src, (int)n_elems, k);
-  // ascending index order: a point's record number is the number of selected indices below its own
-  for (int j = lane; j < k; j += 32) {
-    uint32_t flat, pattern;
-    unpack<DT>(sh.cand[j], &flat, &pattern);
-    const uint32_t mine = kIdxMask - flat;  // the index field as stored: larger means a lower index
-    int pos = 0;
-    for (int i = 0; i < k; ++i) pos += (((uint32_t)(sh.cand[i] >> 1)) & kIdxMask) > mine;
+  // Ascending index order.  The candidate words are re-keyed by their index field (stored
+  // complemented: larger means a lower index) and sorted downwards by a bitonic network over the
+  // next power of two (padding words are 0 and sink to the end).
+  int padded = 32;
+  while (padded < k) padded <<= 1;
+  for (int j = lane; j < padded; j += 32) {
+    unsigned long long c = 0ull;
+    if (j < k) {
+      c = sh.cand[j];
+      // index field on top, then key and sign: still one distinct word per candidate
+      c = ((unsigned long long)(((uint32_t)(c >> 1)) & kIdxMask) << 40) | ((c >> (kIdxBits + 1)) << 1) | (c & 1ull) | (1ull << 39);
+    }
+    sh.cand[j] = c;
+  }
+  warp_barrier();
+  for (int size = 2; size <= padded; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = lane; t < padded / 2; t += 32) {
+        const int i = 2 * t - (t & (stride - 1));  // lower partner of pair t
+        const int j = i + stride;
+        const bool descending = (i & size) == 0;
+        const unsigned long long a = sh.cand[i], b = sh.cand[j];
+        if ((a < b) == descending) {
+          sh.cand[i] = b;
+          sh.cand[j] = a;
+        }
+      }
+      warp_barrier();
+    }
+  }
+  for (int pos = lane; pos < k; pos += 32) {
+    const unsigned long long c = sh.cand[pos];
+    const uint32_t flat = kIdxMask - (uint32_t)(c >> 40);
+    const uint32_t key = (uint32_t)(c >> 1) & 0x7FFFFFFFu, sign = (uint32_t)c & 1u;
+    const uint32_t pattern = (sign << 15) | (DT == 0 ? key : key >> 16);
     rec[3 * pos] = (uint16_t)(flat & 0xFFFFu);
     rec[3 * pos + 1] = (uint16_t)(flat >> 16);
     rec[3 * pos + 2] = (uint16_t)pattern;
@@ -1101,9 +1132,10 @@ __global__ void __launch_bounds__(32, 15) toploc_direct_commit_warp_kernel(Direc
   if (lane == 0) status[chunk] = TOPLOC_CHUNK_OK;
 }
 
-template <int DT, int MODE>
-__global__ void __launch_bounds__(32, 15) toploc_direct_verify_warp_kernel(DirectParams p, DirectVerify io) {
-  __shared__ SelectShared sh;
+template <int DT, int MODE, class SH>
+__global__ void __launch_bounds__(32, min_blocks<SH>()) toploc_direct_verify_warp_kernel(DirectParams p, DirectVerify io) {
+  constexpr int kSlots = SH::kMaxSlots;
+  __shared__ SH sh;
   const int lane = threadIdx.x;
   const long long chunk = blockIdx.x;
   const int k = p.k;
@@ -1132,7 +1164,7 @@ __global__ void __launch_bounds__(32, 15) toploc_direct_verify_warp_kernel(Direc
   }
   // the selection is in registers: the ring holds the commitment, the histograms the statistics
   uint32_t* com_idx = reinterpret_cast<uint32_t*>(sh.ring);
-  uint32_t* com_pat = com_idx + kSmallK;
+  uint32_t* com_pat = com_idx + SH::kMaxK;
   uint32_t* hist = sh.top_hist;  // a 7-bit mantissa difference is at most 127
   warp_barrier();
   const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
@@ -1258,19 +1290,31 @@ inline bool applies(const toploc_layout* lay) {
   return lay->k <= kSmallK && rows * lay->hidden <= kMaxElems;
 }
 
+template <int DT, class SH>
+void launch_commit_sized(int mode, long long n, cudaStream_t stream, const DirectParams& p, uint8_t* commits, uint8_t* status) {
+  if (mode == 0) toploc_direct_commit_warp_kernel<DT, 0, SH><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
+  else if (mode == 1) toploc_direct_commit_warp_kernel<DT, 1, SH><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
+  else toploc_direct_commit_warp_kernel<DT, 2, SH><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
+}
+
 template <int DT>
 int launch_commit(int mode, long long n, cudaStream_t stream, const DirectParams& p, uint8_t* commits, uint8_t* status) {
-  if (mode == 0) toploc_direct_commit_warp_kernel<DT, 0><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
-  else if (mode == 1) toploc_direct_commit_warp_kernel<DT, 1><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
-  else toploc_direct_commit_warp_kernel<DT, 2><<<(unsigned)n, 32, 0, stream>>>(p, commits, status);
+  if (p.k > SelectShared::kMaxK) launch_commit_sized<DT, SelectSharedBig>(mode, n, stream, p, commits, status);
+  else launch_commit_sized<DT, SelectShared>(mode, n, stream, p, commits, status);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
+}
+
+template <int DT, class SH>
+void launch_verify_sized(int mode, long long n, cudaStream_t stream, const DirectParams& p, const DirectVerify& io) {
+  if (mode == 0) toploc_direct_verify_warp_kernel<DT, 0, SH><<<(unsigned)n, 32, 0, stream>>>(p, io);
+  else if (mode == 1) toploc_direct_verify_warp_kernel<DT, 1, SH><<<(unsigned)n, 32, 0, stream>>>(p, io);
+  else toploc_direct_verify_warp_kernel<DT, 2, SH><<<(unsigned)n, 32, 0, stream>>>(p, io);
 }
 
 template <int DT>
 int launch_verify(int mode, long long n, cudaStream_t stream, const DirectParams& p, const DirectVerify& io) {
-  if (mode == 0) toploc_direct_verify_warp_kernel<DT, 0><<<(unsigned)n, 32, 0, stream>>>(p, io);
-  else if (mode == 1) toploc_direct_verify_warp_kernel<DT, 1><<<(unsigned)n, 32, 0, stream>>>(p, io);
-  else toploc_direct_verify_warp_kernel<DT, 2><<<(unsigned)n, 32, 0, stream>>>(p, io);
+  if (p.k > SelectShared::kMaxK) launch_verify_sized<DT, SelectSharedBig>(mode, n, stream, p, io);
+  else launch_verify_sized<DT, SelectShared>(mode, n, stream, p, io);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 }  // namespace small_k
