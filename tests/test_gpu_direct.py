@@ -44,7 +44,7 @@ def direct_case(act, chunk_len, k, num_seqs, tokens_per_seq, recomputed=None, wh
     return out
 
 
-@pytest.mark.parametrize("k", [1, 128, 1000, 4096])
+@pytest.mark.parametrize("k", [1, 128, 256, 257, 512, 1000, 4096])
 @pytest.mark.parametrize("outliers", ["fixed", "none"])
 def test_bf16_chunks(k, outliers):
     S, T, H, L = 3, 96, 4096, 32
@@ -70,6 +70,39 @@ def test_70b_shaped_chunks_and_ragged_tail():
     S, T, H, L, k = 2, 100, 8192, 32, 4096
     act = synth.make_activations(S, T, H, torch.bfloat16, seed=61, device=DEV)
     direct_case(act, L, k, S, T, {"noise": synth.honest_noise(act, seed=3)}, "70B-shaped")
+
+
+@pytest.mark.parametrize("k", [128, 1024])
+def test_full_size_launch_sampled(k):
+    """The 70B-shaped batch (256 sequences x 4096 tokens, H = 8192) committed and validated in one call
+    each, the launch configuration `bench.py --direct` times (k = 128: a warp per chunk; k = 1024: a
+    block per chunk); whole sampled sequences against the oracle, properties of an exact copy on all
+    32768 chunks."""
+    S, T, H, L = 256, 4096, 8192, 32
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2 ** 30:
+        pytest.skip("needs 40 GB of free device memory")
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=4, device=DEV)
+    noisy = synth.honest_noise(act, seed=5)
+    lay, _ = tl.make_layout(act, L, k, S, T)
+    commits, status = tl.toploc_commit_direct(act, lay)
+    same, _ = tl.toploc_verify_direct(act, lay, commits, tl.default_thresholds(k))
+    honest, dev = tl.toploc_verify_direct(noisy, lay, commits, tl.default_thresholds(k))
+    torch.cuda.synchronize()
+    assert not status.any().item()
+    same = same.cpu().numpy().view(tl.RESULT_DTYPE).reshape(-1)
+    assert same["accept"].all() and not same["exp_mismatch"].any() and not same["topk_mismatch"].any()
+    assert (same["n_match"] == k).all() and not same["mant_diff_sum"].any()
+    honest = honest.cpu().numpy().view(tl.RESULT_DTYPE).reshape(-1)
+    cps = T // L
+    for s in (3, 200):
+        rows, chunks = slice(s * T, (s + 1) * T), slice(s * cps, (s + 1) * cps)
+        ref_commits, ref_status = oracle.commit_direct(synth.host_patterns(act[rows]), L, k, 1, T)
+        assert np.array_equal(commits[chunks].cpu().numpy(), ref_commits), "commitments of sequence %d" % s
+        ref, ref_dev = oracle.verify_direct(synth.host_patterns(noisy[rows]), ref_commits, L, k, 1, T,
+                                            **oracle_thresholds(k))
+        assert_results_equal(honest[chunks], ref, "70B direct k=%d seq %d" % (k, s))
+        assert np.array_equal(dev[chunks].cpu().numpy().astype(np.uint32), ref_dev)
 
 
 def test_ties_decide_the_selection():
