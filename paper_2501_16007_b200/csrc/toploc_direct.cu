@@ -626,21 +626,40 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
     return base + (uint32_t)total;
   };
 
-  // A sound first threshold from the chunk's first vectors: the k-th largest of their per-vector
-  // maxima (each maximum is a different element, so at least k elements reach it).  Those vectors
-  // are then streamed like the rest.  A chunk of fewer than k vectors starts from 0.
+  // A sound and tight threshold before anything is collected: a first pass streams the whole chunk
+  // and counts every vector's largest key in the histogram; the k-th largest of these maxima is
+  // reached by at least k elements (each maximum is a different element), so the chunk's k-th key
+  // cannot lie below it, and by little more than k (k vectors reach it, few of them twice).  The
+  // second pass finds the chunk in L2 (one chunk per SM in flight).  A chunk of fewer than k
+  // vectors starts from 0 and is streamed once.
   {
     const int first_end = kBatch < rd.n_groups ? kBatch : rd.n_groups;
     rd.request(ring, (int)threadIdx.x, first_end);  // in flight meanwhile
   }
-  const int seed_groups = 4 * k < rd.n_groups ? 4 * k : rd.n_groups;
-  if (seed_groups >= k) {
-    for (int g = threadIdx.x; g < seed_groups; g += kThreads) {
-      const uint4 w = toploc_device::load_streaming(reinterpret_cast<const uint4*>(rd.address(g)));
-      atomicAdd(&coarse[toploc_device::vector_max_coarse_key<DT, VEC>(w) >> 4], 1u);  // upper 11 of 15 bits
+  if (rd.n_groups >= k) {
+    for (int begin = 0; begin < rd.n_groups; begin += kBatch) {
+      const int end = begin + kBatch < rd.n_groups ? begin + kBatch : rd.n_groups;
+      uint32_t w[kUnroll][4];
+      rd.take(ring, begin + (int)threadIdx.x, end, w);
+      if (end < rd.n_groups) {
+        const int next_end = end + kBatch < rd.n_groups ? end + kBatch : rd.n_groups;
+        rd.request_after(ring, end + (int)threadIdx.x, next_end, w, begin + (int)threadIdx.x, end);
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (begin + u * kThreads + (int)threadIdx.x < end) {
+          const uint32_t m = toploc_device::vector_max_coarse_key<DT, VEC>(make_uint4(w[u][0], w[u][1], w[u][2], w[u][3]));
+          atomicAdd(&coarse[m >> 4], 1u);  // upper 11 of the 15 bits
+        }
+      }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    {
+      const int first_end = kBatch < rd.n_groups ? kBatch : rd.n_groups;
+      rd.request(ring, (int)threadIdx.x, first_end);  // the second pass's first batch
     }
     __syncthreads();
-    find_bin_from_top(sh, kCoarseBins, (uint32_t)k, 0);
+    find_bin_from_top(sh, kCoarseBins, (uint32_t)k, 1);
     const uint32_t first = sh.picked_bin << kCoarseShift;
     __syncthreads();
     if (threadIdx.x == 0) sh.thr = first;
@@ -759,23 +778,45 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
     ties = sh.hist[sh.picked_bin];  // after the last digit: the candidates equal to the k-th key
     __syncthreads();
   }
-  // Of the candidates equal to the k-th key the `take` lowest flat indices belong to the top-k:
-  // the take-th largest of (2^24 - 1 - flat index) among them, digit by digit (nothing to find
-  // when all of them belong).
-  uint32_t cut = 0, cut_known = 0;
-  for (int shift = 16, round = 0; shift >= 0 && ties != take; shift -= 8, ++round) {
-    clear_bins(sh, 256);
-    for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
-      if (R::key(cand_pat[i]) != kth) continue;
-      const uint32_t inv = 0xFFFFFFu - cand_flat[i];
-      if ((inv & cut_known) == cut) atomicAdd(&sh.hist[(inv >> shift) & 255u], 1u);
+  // Of the candidates equal to the k-th key the `take` lowest flat indices belong to the top-k.
+  // Usually there are a handful: they are listed and the take-th lowest index is found by counting.
+  // A long list (a chunk of many equal values) takes the take-th largest of (2^24 - 1 - flat
+  // index) digit by digit instead.  Nothing to find when all of them belong.
+  uint32_t cut = 0;
+  constexpr uint32_t kShortList = 1024;
+  if (ties != take && ties <= kShortList) {
+    uint32_t* list = sh.hist;  // (the histogram is done with)
+    if (threadIdx.x == 0) sh.emitted = 0;
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < count; i += kThreads)
+      if (R::key(cand_pat[i]) == kth) list[atomicAdd(&sh.emitted, 1u)] = cand_flat[i];
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < ties; i += kThreads) {
+      const uint32_t mine = list[i];
+      uint32_t lower = 0;
+      for (uint32_t j = 0; j < ties; ++j) lower += list[j] < mine;
+      if (lower == take - 1) sh.picked_bin = 0xFFFFFFu - mine;  // exactly one index has take - 1 below it
     }
     __syncthreads();
-    find_bin_from_top(sh, 256, take, round & 1);
-    cut |= sh.picked_bin << shift;
-    cut_known |= 255u << shift;
-    take = sh.picked_remaining;
+    cut = sh.picked_bin;
+    if (threadIdx.x == 0) sh.emitted = 0;
     __syncthreads();
+  } else if (ties != take) {
+    uint32_t cut_known = 0;
+    for (int shift = 16, round = 0; shift >= 0; shift -= 8, ++round) {
+      clear_bins(sh, 256);
+      for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+        if (R::key(cand_pat[i]) != kth) continue;
+        const uint32_t inv = 0xFFFFFFu - cand_flat[i];
+        if ((inv & cut_known) == cut) atomicAdd(&sh.hist[(inv >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      find_bin_from_top(sh, 256, take, round & 1);
+      cut |= sh.picked_bin << shift;
+      cut_known |= 255u << shift;
+      take = sh.picked_remaining;
+      __syncthreads();
+    }
   }
   auto selected = [&](uint32_t i) {
     const uint32_t key = R::key(cand_pat[i]);
