@@ -59,6 +59,21 @@ def test_k_512(dtype, wide):
     parity_case(wide_rows[:, :2048], 32, 300, 1, 70, where="k300 strided %s" % dtype, wide=wide)
 
 
+def test_no_injective_modulus_is_a_status_not_a_proof():
+    """Algorithm 6 ends without a modulus when the differences of the selected indices cover its
+    whole search range: 512 indices (0..255 and the multiples of 256 up to 65536) do.  The chunk
+    gets its status and a zero proof on both sides; its neighbour in the batch is unaffected; the
+    zero proofs validate the same way on both sides."""
+    idx = list(range(256)) + [256 * j for j in range(1, 257)]
+    pat = np.full((64, 4096), 0x3C00, np.uint16)
+    pat[:32].reshape(-1)[idx] = 0x4500                               # first chunk: no modulus exists
+    rng = np.random.default_rng(3)
+    pat[32:] = rng.integers(0x3000, 0x4400, size=(32, 4096)).astype(np.uint16)   # second chunk: ordinary
+    act = from_patterns(pat)
+    r, v = parity_case(act, 32, 512, 1, 64, where="no modulus")
+    assert r[1].tolist() == [oracle.ST_NO_MODULUS, oracle.ST_OK] and not r[0][0].any() and r[0][1].any()
+
+
 @pytest.mark.parametrize("outliers", ["fixed", "none"])
 def test_outlier_recipes(outliers):
     act = synth.make_activations(3, 64, 4096, torch.bfloat16, seed=3, device=DEV, outliers=outliers)

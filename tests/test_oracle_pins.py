@@ -12,6 +12,7 @@ import oracle
 from paper_2501_16007_b200 import synth
 
 P = 65521
+M_LOW, M_HIGH = 2 ** 15 + 1, 2 ** 16      # Algorithm 6 search range, inclusive
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
@@ -179,6 +180,30 @@ def test_modulus_none_exists():
     # 65537 values in 65536 residue classes can never be injective; a much smaller clash:
     # indices that agree modulo every candidate do not exist, so use duplicates.
     assert oracle.find_injective_modulus([5, 5, 9]) == 0
+
+
+def covering_index_set():
+    """512 distinct indices whose pairwise differences take every value from 1 to 65536: the residues
+    0..255 and the multiples 256, 512, ..., 65536 (256 j - r covers [256 j - 255, 256 j]).  Every
+    candidate modulus of Algorithm 6 equals one of the differences, so none is injective."""
+    return list(range(256)) + [256 * j for j in range(1, 257)]
+
+
+def test_modulus_none_exists_for_a_covering_set():
+    idx = covering_index_set()
+    assert len(set(idx)) == 512
+    diffs = {b - a for a in idx for b in idx if b > a}
+    assert all(m in diffs for m in range(M_LOW, M_HIGH + 1))       # the reason, checked directly
+    assert oracle.find_injective_modulus(idx) == 0
+    assert oracle.find_injective_modulus(idx, field_distinct=False) == 0
+    # a chunk whose 512 largest magnitudes sit exactly there: Algorithm 6 has nothing to return,
+    # the chunk gets its status and a zero proof
+    pat = np.full((32, 4096), 0x3C00, np.uint16)
+    flat = pat.reshape(-1)
+    flat[idx] = 0x4500
+    proofs, status, indices = oracle.build_proofs(pat, 32, 512, 1, 32)
+    assert status.tolist() == [oracle.ST_NO_MODULUS] and not proofs.any()
+    assert sorted(indices[0].tolist()) == sorted(idx)
 
 
 def test_modulus_distribution_matches_table_11():
