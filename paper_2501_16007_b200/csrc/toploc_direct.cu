@@ -61,6 +61,19 @@ struct DirectVerify {
 
 // Dynamic shared memory of a block: the copy ring, this struct, and kSpareBytes that continue
 // its last member (the one-pass selection keeps its candidates in hist and the spare together).
+// Scalars of the two-pass selection without barriers (select_unordered), in shared memory.
+struct LooseControl {
+  unsigned long long warp_sums[2][32];
+  uint32_t picked_bin;
+  uint32_t picked_remaining;
+  uint32_t cand_count;       // candidates handed out so far (may run past the buffer: then overflow is set)
+  uint32_t thr;              // an element is a candidate iff its key is >= thr; only ever raised
+  uint32_t last_raise;       // cand_count when thr was last raised
+  uint32_t raise_lock;       // 1 while a warp is raising thr
+  uint32_t overflow;
+  uint32_t emitted;
+};
+
 struct DirectShared {
   unsigned long long warp_sums[2][kWarps];
   uint32_t picked_bin;
@@ -68,22 +81,16 @@ struct DirectShared {
   uint32_t bad;
   uint32_t counters[4];      // exponent mismatches, matches, mantissa difference sum, common indices
   uint32_t dev[9];
-  // the free-running one-pass selection (select_unordered)
-  uint32_t cand_count;       // candidates handed out so far (may run past the buffer: then overflow is set)
-  uint32_t thr;              // an element is a candidate iff its key is >= thr; only ever raised
-  uint32_t last_raise;       // cand_count when thr was last raised
-  uint32_t raise_lock;       // 1 while a warp is raising thr
-  uint32_t overflow;
-  uint32_t emitted;
-  uint32_t pad[2];
+  uint32_t pad[4];
+  LooseControl loose;
   uint32_t hist[kBins];
 };
-constexpr size_t kSpareBytes = 35232;
+constexpr size_t kSpareBytes = 34704;
 constexpr size_t kSharedBytes = kRingBytes + sizeof(DirectShared) + kSpareBytes;
 // One-pass selection (vector layouts, k <= kStreamMaxK): a histogram of the upper 11 key bits
 // and up to cand_cap candidates (flat index, whole pattern) in index order.
 constexpr int kCoarseBins = 2048;
-__host__ __device__ constexpr int cand_cap(int dt) { return dt == 0 ? 26112 : 19712; }       // 6 / 8 bytes each
+__host__ __device__ constexpr int cand_cap(int dt) { return dt == 0 ? 25984 : 19584; }       // 6 / 8 bytes each
 constexpr int kStreamMaxK = 2048;   // beyond it the candidates of a 2^18-element chunk no longer fit
 static_assert(kSharedBytes <= 227 * 1024 && sizeof(DirectShared) % 16 == 0 && kSpareBytes % 16 == 0, "shared memory budget");
 static_assert(offsetof(DirectShared, hist) + sizeof(uint32_t) * kBins == sizeof(DirectShared), "hist is the last member");
@@ -128,13 +135,14 @@ struct Reader {
   // moves the slots to registers, after which the next batch may be requested -- so a batch is
   // in flight while the previous one is worked on, barriers included.  Nothing waits on
   // another thread.  Other layouts load directly in take().
+  template <int T = kThreads>
   __device__ __forceinline__ void request(uint4* ring, int first, int g_end) const {
     if constexpr (VECTOR) {
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        const int g = first + u * kThreads;
+        const int g = first + u * T;
         if (g < g_end) {
-          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(ring + u * kThreads + threadIdx.x);
+          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(ring + u * T + threadIdx.x);
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(address(g)) : "memory");
         }
       }
@@ -143,15 +151,16 @@ struct Reader {
   }
   // The same, for the batch after one whose registers are w: each copy's destination is made
   // to depend on the register that was read from it, so the copy cannot overtake the read.
+  template <int T = kThreads>
   __device__ __forceinline__ void request_after(uint4* ring, int first, int g_end, const uint32_t (&w)[kUnroll][4],
                                                 int prev_first, int prev_end) const {
     if constexpr (VECTOR) {
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        const int g = first + u * kThreads;
+        const int g = first + u * T;
         if (g < g_end) {
-          uint32_t dst = (uint32_t)__cvta_generic_to_shared(ring + u * kThreads + threadIdx.x);
-          if (prev_first + u * kThreads < prev_end) {
+          uint32_t dst = (uint32_t)__cvta_generic_to_shared(ring + u * T + threadIdx.x);
+          if (prev_first + u * T < prev_end) {
             uint32_t zero;
             asm volatile("and.b32 %0, %1, 0;" : "=r"(zero) : "r"(w[u][3]));
             dst += zero;
@@ -162,14 +171,15 @@ struct Reader {
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
   }
+  template <int T = kThreads>
   __device__ __forceinline__ void take(const uint4* ring, int first, int g_end, uint32_t (&w)[kUnroll][4]) const {
     if (VECTOR) asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      const int g = first + u * kThreads;
+      const int g = first + u * T;
       if (g < g_end) {
         if (VECTOR) {
-          const uint4 v = ring[u * kThreads + threadIdx.x];
+          const uint4 v = ring[u * T + threadIdx.x];
           w[u][0] = v.x; w[u][1] = v.y; w[u][2] = v.z; w[u][3] = v.w;
         } else if (DT == 0) {
           w[u][0] = *reinterpret_cast<const uint16_t*>(address(g));
@@ -562,21 +572,94 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<D
 // settled at the end.  ORDERED: emit(position in ascending index order, ...), by ranking the
 // selected indices in a bitmap of the chunk; otherwise positions are handed out as they come.
 // Returns false, having emitted nothing, when the candidates outgrow their buffer.
-template <int DT, bool ORDERED, class Emit>
-__device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit) {
+// Where the two-pass selection without barriers keeps its state; the two kernels that use it
+// (a 1024-thread block per SM, or two 512-thread blocks) carve it from their shared memory.
+template <int DT>
+struct LooseWorkspace {
+  LooseControl* ctl;
+  uint32_t* coarse;      // kCoarseBins words: the histogram; later digit histograms, the tie list, per-thread prefixes
+  uint32_t* cand_flat;   // cap candidates: flat index ...
+  typename StoredPattern<DT>::type* cand_pat;  // ... and whole pattern
+  uint32_t* park;        // kParkCap words per warp
+  int cap;
+};
+
+template <int T>
+__device__ __forceinline__ void clear_words(uint32_t* words, int n) {  // n: a multiple of 4; ends with a barrier
+  uint4* q = reinterpret_cast<uint4*>(words);
+  for (int b = threadIdx.x; b < n / 4; b += T) q[b] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+}
+
+// Exclusive prefix sum over a block of T threads (T / 32 <= 32 warps) of a 64-bit value; *total
+// receives the block's sum.  `slot` alternates between calls so that one barrier per call is enough.
+template <int T>
+__device__ __forceinline__ unsigned long long scan_exclusive(LooseControl& sh, unsigned long long v, int slot,
+                                                             unsigned long long* total) {
+  constexpr int kW = T / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned long long inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+    if (lane >= d) inc += o;
+  }
+  if (lane == 31) sh.warp_sums[slot][warp] = inc;
+  __syncthreads();
+  unsigned long long mine = lane < kW ? sh.warp_sums[slot][lane] : 0ull;
+  unsigned long long winc = mine;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+    if (lane >= d) winc += o;
+  }
+  *total = __shfl_sync(0xFFFFFFFFu, winc, 31);
+  const unsigned long long before_warp = __shfl_sync(0xFFFFFFFFu, winc - mine, warp);
+  return before_warp + inc - v;
+}
+
+// The bin of hist[0 .. nbins), counted from the top, in which the want-th largest counted element
+// lies (1 <= want <= number counted): sh.picked_bin, and sh.picked_remaining = want minus the
+// elements in higher bins.  All T threads call; ends with a barrier.
+template <int T>
+__device__ __forceinline__ void find_from_top(LooseControl& sh, const uint32_t* hist, int nbins, uint32_t want, int slot) {
+  const int per = nbins >= T ? nbins / T : 1;  // nbins and T are powers of two
+  const int top = nbins - 1 - (int)threadIdx.x * per;  // this thread owns bins top, top-1, ..., top-per+1
+  uint32_t s = 0;
+  if (top >= 0)  // each lane starts at another offset: its bins are `per` words apart from its neighbour's
+    for (int b = 0; b < per; ++b) s += hist[top - ((b + (int)threadIdx.x) & (per - 1))];
+  unsigned long long total;
+  const uint32_t before = (uint32_t)scan_exclusive<T>(sh, s, slot, &total);
+  if (top >= 0 && before < want && want <= before + s) {
+    uint32_t c = before;
+    for (int b = 0; b < per; ++b) {
+      const uint32_t h = hist[top - b];
+      if (c + h >= want) {
+        sh.picked_bin = (uint32_t)(top - b);
+        sh.picked_remaining = want - c;
+        break;
+      }
+      c += h;
+    }
+  }
+  __syncthreads();
+}
+
+template <int DT, bool ORDERED, int T, class Emit>
+__device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit) {
   using R = Reader<DT, true>;
   using Pat = typename StoredPattern<DT>::type;
   constexpr int VEC = R::VEC;
-  constexpr int kCap = loose_cap(DT);
   constexpr int kCoarseShift = key_bits(DT) - 11;
   constexpr uint32_t kFull = 0xFFFFFFFFu;
-  constexpr int kBatch = kUnroll * kThreads;
-  uint32_t* coarse = sh.hist;
-  uint32_t* cand_flat = sh.hist + kCoarseBins;
-  Pat* cand_pat = reinterpret_cast<Pat*>(cand_flat + kCap);
+  constexpr int kBatch = kUnroll * T;
+  LooseControl& sh = *ws.ctl;
+  const int kCap = ws.cap;
+  uint32_t* coarse = ws.coarse;
+  uint32_t* cand_flat = ws.cand_flat;
+  Pat* cand_pat = ws.cand_pat;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t* park = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(sh.hist) + (size_t)kBins * 4 +
-                                               kSpareBytes - kParkBytes) + warp * kParkCap;
+  uint32_t* park = ws.park + warp * kParkCap;
   volatile uint32_t* shared_thr = &sh.thr;
   volatile uint32_t* shared_overflow = &sh.overflow;
   volatile uint32_t* shared_last_raise = &sh.last_raise;
@@ -588,7 +671,7 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
     sh.overflow = 0;
     sh.emitted = 0;
   }
-  clear_bins(sh, kCoarseBins);  // ends with a barrier
+  clear_words<T>(coarse, kCoarseBins);  // ends with a barrier
 
   // One vector per lane: its elements that reach thr become candidates.  Returns the number of
   // candidates handed out so far (0 if the round added none).
@@ -634,20 +717,20 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
   // vectors starts from 0 and is streamed once.
   {
     const int first_end = kBatch < rd.n_groups ? kBatch : rd.n_groups;
-    rd.request(ring, (int)threadIdx.x, first_end);  // in flight meanwhile
+    rd.template request<T>(ring, (int)threadIdx.x, first_end);  // in flight meanwhile
   }
   if (rd.n_groups >= k) {
     for (int begin = 0; begin < rd.n_groups; begin += kBatch) {
       const int end = begin + kBatch < rd.n_groups ? begin + kBatch : rd.n_groups;
       uint32_t w[kUnroll][4];
-      rd.take(ring, begin + (int)threadIdx.x, end, w);
+      rd.template take<T>(ring, begin + (int)threadIdx.x, end, w);
       if (end < rd.n_groups) {
         const int next_end = end + kBatch < rd.n_groups ? end + kBatch : rd.n_groups;
-        rd.request_after(ring, end + (int)threadIdx.x, next_end, w, begin + (int)threadIdx.x, end);
+        rd.template request_after<T>(ring, end + (int)threadIdx.x, next_end, w, begin + (int)threadIdx.x, end);
       }
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        if (begin + u * kThreads + (int)threadIdx.x < end) {
+        if (begin + u * T + (int)threadIdx.x < end) {
           const uint32_t m = toploc_device::vector_max_coarse_key<DT, VEC>(make_uint4(w[u][0], w[u][1], w[u][2], w[u][3]));
           atomicAdd(&coarse[m >> 4], 1u);  // upper 11 of the 15 bits
         }
@@ -656,14 +739,14 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     {
       const int first_end = kBatch < rd.n_groups ? kBatch : rd.n_groups;
-      rd.request(ring, (int)threadIdx.x, first_end);  // the second pass's first batch
+      rd.template request<T>(ring, (int)threadIdx.x, first_end);  // the second pass's first batch
     }
     __syncthreads();
-    find_bin_from_top(sh, kCoarseBins, (uint32_t)k, 1);
+    find_from_top<T>(sh, coarse, kCoarseBins, (uint32_t)k, 1);
     const uint32_t first = sh.picked_bin << kCoarseShift;
     __syncthreads();
     if (threadIdx.x == 0) sh.thr = first;
-    clear_bins(sh, kCoarseBins);
+    clear_words<T>(coarse, kCoarseBins);
   }
 
   const uint32_t raise_step = (uint32_t)(k / 2 > 256 ? k / 2 : 256);
@@ -722,17 +805,17 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
   for (int begin = 0; begin < rd.n_groups; begin += kBatch) {
     const int end = begin + kBatch < rd.n_groups ? begin + kBatch : rd.n_groups;
     uint32_t w[kUnroll][4];
-    rd.take(ring, begin + (int)threadIdx.x, end, w);
+    rd.template take<T>(ring, begin + (int)threadIdx.x, end, w);
     if (end < rd.n_groups) {
       const int next_end = end + kBatch < rd.n_groups ? end + kBatch : rd.n_groups;
-      rd.request_after(ring, end + (int)threadIdx.x, next_end, w, begin + (int)threadIdx.x, end);
+      rd.template request_after<T>(ring, end + (int)threadIdx.x, next_end, w, begin + (int)threadIdx.x, end);
     }
     const uint32_t add = toploc_device::bf16_lane_add(thr);
     bool hit[kUnroll];
     uint32_t votes[kUnroll], any_votes = 0;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      const int g = begin + u * kThreads + (int)threadIdx.x;
+      const int g = begin + u * T + (int)threadIdx.x;
       hit[u] = g < end && toploc_device::vector_reaches<DT, VEC>(make_uint4(w[u][0], w[u][1], w[u][2], w[u][3]), thr, add);
     }
 #pragma unroll
@@ -743,7 +826,7 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
     if (any_votes) {
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        if (hit[u]) park[nparked + __popc(votes[u] & ((1u << lane) - 1u))] = (uint32_t)(begin + u * kThreads) + threadIdx.x;
+        if (hit[u]) park[nparked + __popc(votes[u] & ((1u << lane) - 1u))] = (uint32_t)(begin + u * T) + threadIdx.x;
         nparked += __popc(votes[u]);
       }
       if (nparked >= kParkTrigger) drain();
@@ -759,23 +842,23 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
 
   // The exact k-th key among the candidates: its upper 11 bits from the histogram (it counts
   // every candidate), the bits below 8 at a time (the last digit has 4).
-  find_bin_from_top(sh, kCoarseBins, (uint32_t)k, 0);
+  find_from_top<T>(sh, coarse, kCoarseBins, (uint32_t)k, 0);
   uint32_t kth = sh.picked_bin << kCoarseShift, known = (uint32_t)(kCoarseBins - 1) << kCoarseShift;
   uint32_t take = sh.picked_remaining, ties = 0;
   __syncthreads();
   for (int shift = kCoarseShift - 8, round = 1; shift > -8; shift -= 8, ++round) {
     const int low = shift < 0 ? 0 : shift, width = shift < 0 ? 8 + shift : 8;
-    clear_bins(sh, 256);
-    for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+    clear_words<T>(coarse, 256);
+    for (uint32_t i = threadIdx.x; i < count; i += T) {
       const uint32_t key = R::key(cand_pat[i]);
-      if ((key & known) == kth) atomicAdd(&sh.hist[(key >> low) & ((1u << width) - 1u)], 1u);
+      if ((key & known) == kth) atomicAdd(&coarse[(key >> low) & ((1u << width) - 1u)], 1u);
     }
     __syncthreads();
-    find_bin_from_top(sh, 1 << width, take, round & 1);
+    find_from_top<T>(sh, coarse, 1 << width, take, round & 1);
     kth |= sh.picked_bin << low;
     known |= ((1u << width) - 1u) << low;
     take = sh.picked_remaining;
-    ties = sh.hist[sh.picked_bin];  // after the last digit: the candidates equal to the k-th key
+    ties = coarse[sh.picked_bin];  // after the last digit: the candidates equal to the k-th key
     __syncthreads();
   }
   // Of the candidates equal to the k-th key the `take` lowest flat indices belong to the top-k.
@@ -785,13 +868,13 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
   uint32_t cut = 0;
   constexpr uint32_t kShortList = 1024;
   if (ties != take && ties <= kShortList) {
-    uint32_t* list = sh.hist;  // (the histogram is done with)
+    uint32_t* list = coarse;  // (the histogram is done with)
     if (threadIdx.x == 0) sh.emitted = 0;
     __syncthreads();
-    for (uint32_t i = threadIdx.x; i < count; i += kThreads)
+    for (uint32_t i = threadIdx.x; i < count; i += T)
       if (R::key(cand_pat[i]) == kth) list[atomicAdd(&sh.emitted, 1u)] = cand_flat[i];
     __syncthreads();
-    for (uint32_t i = threadIdx.x; i < ties; i += kThreads) {
+    for (uint32_t i = threadIdx.x; i < ties; i += T) {
       const uint32_t mine = list[i];
       uint32_t lower = 0;
       for (uint32_t j = 0; j < ties; ++j) lower += list[j] < mine;
@@ -804,14 +887,14 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
   } else if (ties != take) {
     uint32_t cut_known = 0;
     for (int shift = 16, round = 0; shift >= 0; shift -= 8, ++round) {
-      clear_bins(sh, 256);
-      for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+      clear_words<T>(coarse, 256);
+      for (uint32_t i = threadIdx.x; i < count; i += T) {
         if (R::key(cand_pat[i]) != kth) continue;
         const uint32_t inv = 0xFFFFFFu - cand_flat[i];
-        if ((inv & cut_known) == cut) atomicAdd(&sh.hist[(inv >> shift) & 255u], 1u);
+        if ((inv & cut_known) == cut) atomicAdd(&coarse[(inv >> shift) & 255u], 1u);
       }
       __syncthreads();
-      find_bin_from_top(sh, 256, take, round & 1);
+      find_from_top<T>(sh, coarse, 256, take, round & 1);
       cut |= sh.picked_bin << shift;
       cut_known |= 255u << shift;
       take = sh.picked_remaining;
@@ -824,7 +907,7 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
   };
 
   if (!ORDERED) {
-    for (uint32_t i0 = 0; i0 < count; i0 += kThreads) {
+    for (uint32_t i0 = 0; i0 < count; i0 += T) {
       const uint32_t i = i0 + threadIdx.x;
       const bool mine = i < count && selected(i);
       const uint32_t votes = __ballot_sync(kFull, mine);
@@ -838,12 +921,12 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
   }
   // Index order: one bit per element of the chunk for the selected ones; an element's position is
   // the number of set bits before its own.
-  uint32_t* bitmap = reinterpret_cast<uint32_t*>(ring);
+  uint32_t* bitmap = reinterpret_cast<uint32_t*>(ring);  // (the caller made sure one bit per element fits)
   const uint32_t n_words = ((uint32_t)rd.n_groups * VEC + 31u) / 32u;
-  const uint32_t per_thread = (n_words + kThreads - 1) / kThreads;  // consecutive words a thread counts
-  for (uint32_t wd = threadIdx.x; wd < n_words; wd += kThreads) bitmap[wd] = 0u;
+  const uint32_t per_thread = (n_words + T - 1) / T;  // consecutive words a thread counts
+  for (uint32_t wd = threadIdx.x; wd < n_words; wd += T) bitmap[wd] = 0u;
   __syncthreads();
-  for (uint32_t i = threadIdx.x; i < count; i += kThreads)
+  for (uint32_t i = threadIdx.x; i < count; i += T)
     if (selected(i)) atomicOr(&bitmap[cand_flat[i] >> 5], 1u << (cand_flat[i] & 31u));
   __syncthreads();
   {
@@ -852,19 +935,34 @@ __device__ bool select_unordered(DirectShared& sh, uint4* ring, const Reader<DT,
     uint32_t ones = 0;
     for (uint32_t wd = lo; wd < hi; ++wd) ones += (uint32_t)__popc(bitmap[wd]);
     unsigned long long total;
-    sh.hist[threadIdx.x] = (uint32_t)block_scan_exclusive(sh, ones, 0, &total);  // set bits before this thread's words
+    coarse[threadIdx.x] = (uint32_t)scan_exclusive<T>(sh, ones, 0, &total);  // set bits before this thread's words
   }
   __syncthreads();
-  for (uint32_t i = threadIdx.x; i < count; i += kThreads) {
+  for (uint32_t i = threadIdx.x; i < count; i += T) {
     if (!selected(i)) continue;
     const uint32_t flat = cand_flat[i], wd = flat >> 5, owner = wd / per_thread;
-    uint32_t pos = sh.hist[owner];
+    uint32_t pos = coarse[owner];
     for (uint32_t v = owner * per_thread; v < wd; ++v) pos += (uint32_t)__popc(bitmap[v]);
     pos += (uint32_t)__popc(bitmap[wd] & ((1u << (flat & 31u)) - 1u));
     emit(pos, flat, R::committed(cand_pat[i]));
   }
   __syncthreads();
   return true;
+}
+
+// The workspace of select_unordered inside the 1024-thread block's shared memory: histogram and
+// candidates where the key histogram of the other selections lives, the parked vectors at the
+// end of the spare bytes.
+template <int DT>
+__device__ __forceinline__ LooseWorkspace<DT> loose_workspace(DirectShared& sh) {
+  LooseWorkspace<DT> ws;
+  ws.ctl = &sh.loose;
+  ws.coarse = sh.hist;
+  ws.cand_flat = sh.hist + kCoarseBins;
+  ws.cap = loose_cap(DT);
+  ws.cand_pat = reinterpret_cast<typename StoredPattern<DT>::type*>(ws.cand_flat + ws.cap);
+  ws.park = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(sh.hist) + (size_t)kBins * 4 + kSpareBytes - kParkBytes);
+  return ws;
 }
 
 template <int DT, bool VECTOR>
@@ -884,14 +982,17 @@ __device__ __forceinline__ Reader<DT, VECTOR> locate_chunk(const DirectParams& p
   return rd;
 }
 
+// Per-chunk status an intermediate kernel leaves for the chunks it hands on to the rescue launch
+// (never seen by the caller: the rescue launch follows in the same call).
+constexpr uint8_t kRetry = 0xFF;
+
+// One chunk's commitment by a 1024-thread block.  loose_failed: the two-pass selection without
+// barriers has already outgrown its buffer on this chunk (the rescue launch): go straight to the
+// radix select.
 template <int DT, bool VECTOR>
-__global__ void __launch_bounds__(kThreads, 1)
-toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint4* ring = reinterpret_cast<uint4*>(smem_raw);
-  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw + kRingBytes);
+__device__ void commit_one_chunk(DirectShared& sh, uint4* ring, const DirectParams& p, long long chunk, uint8_t* commits,
+                                 uint8_t* status, bool loose_failed) {
   using R = Reader<DT, VECTOR>;
-  const long long chunk = blockIdx.x;
   const R rd = locate_chunk<DT, VECTOR>(p, chunk);
   uint16_t* rec = reinterpret_cast<uint16_t*>(commits + (size_t)chunk * 6u * (size_t)p.k);
   if ((long long)rd.n_groups * R::VEC < p.k) {
@@ -907,8 +1008,11 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
   };
   bool done = false;
   if constexpr (VECTOR) {
-    if ((long long)rd.n_groups * R::VEC <= kLooseMaxElems) done = select_unordered<DT, true>(sh, ring, rd, p.k, emit);
-    else if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
+    if (!loose_failed) {
+      if ((long long)rd.n_groups * R::VEC <= kLooseMaxElems)
+        done = select_unordered<DT, true, kThreads>(loose_workspace<DT>(sh), ring, rd, p.k, emit);
+      else if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
+    }
   }
   if (!done) {
     uint32_t kth, take;
@@ -920,85 +1024,64 @@ toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
 
 template <int DT, bool VECTOR>
 __global__ void __launch_bounds__(kThreads, 1)
-toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
+toploc_direct_commit_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* ring = reinterpret_cast<uint4*>(smem_raw);
   DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw + kRingBytes);
-  // The two selections live where the key histogram was (it is done with once the k-th key is
-  // known), or, after the one-pass selection, in the ring (idle by then).
-  uint32_t* sel_idx = sh.hist + kListOffset;
-  uint16_t* sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * p.k);
-  using R = Reader<DT, VECTOR>;
-  const long long chunk = blockIdx.x;
-  const int k = p.k;
-  const R rd = locate_chunk<DT, VECTOR>(p, chunk);
-  const uint32_t n_elems = (uint32_t)rd.n_groups * R::VEC;
+  commit_one_chunk<DT, VECTOR>(sh, ring, p, blockIdx.x, commits, status, false);
+}
 
-  if (threadIdx.x == 0) sh.bad = 0;
-  if (threadIdx.x < 4) sh.counters[threadIdx.x] = 0;
-  if (threadIdx.x < 9) sh.dev[threadIdx.x] = 0;
-  auto refuse = [&](int status) {  // every thread takes the same way out
-    if (threadIdx.x == 0) {
-      toploc_chunk_result r = {};
-      r.topk_mismatch = -1;
-      r.status = (uint8_t)status;
-      io.results[chunk] = r;
-    }
-    if (io.exp_dev != nullptr && threadIdx.x < 9) io.exp_dev[(size_t)chunk * 9 + threadIdx.x] = 0;
-  };
-  if (n_elems < (uint32_t)k) {
-    refuse(TOPLOC_CHUNK_K_EXCEEDS_CHUNK);
-    return;
-  }
+// What the comparison against a commitment needs besides the two lists.
+struct CompareScratch {
+  uint32_t bad;
+  uint32_t counters[4];  // exponent mismatches, matches, mantissa difference sum, common indices
+  uint32_t dev[9];
+  uint32_t pad[2];
+  uint32_t hist[128];    // mantissa differences 0..127
+};
 
-  auto emit = [&](uint32_t pos, uint32_t flat, uint32_t pat) {
-    if (pos >= (uint32_t)k) return;
-    sel_idx[pos] = flat;
-    sel_pat[pos] = (uint16_t)pat;
-  };
-  bool done = false;
-  if constexpr (VECTOR) {
-    const bool loose = n_elems <= (uint32_t)kLooseMaxElems;  // the comparison below needs no particular order
-    if (loose || k <= kStreamMaxK) {
-      sel_idx = reinterpret_cast<uint32_t*>(ring);
-      sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
-      done = loose ? select_unordered<DT, false>(sh, ring, rd, k, emit) : select_in_one_pass<DT>(sh, ring, rd, k, emit);
-    }
+// A chunk that cannot be validated: zero result with its status.
+__device__ __forceinline__ void refuse_chunk(const DirectVerify& io, long long chunk, int status) {
+  if (threadIdx.x == 0) {
+    toploc_chunk_result r = {};
+    r.topk_mismatch = -1;
+    r.status = (uint8_t)status;
+    io.results[chunk] = r;
   }
-  if (!done) {
-    sel_idx = sh.hist + kListOffset;
-    sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
-    uint32_t kth, take;
-    find_kth_key<DT, VECTOR>(sh, ring, rd, k, &kth, &take);
-    collect_in_index_order<DT, VECTOR>(sh, ring, rd, k, kth, take, emit);
-  }
-  uint32_t* com_idx = sel_idx + k;
-  uint16_t* com_pat = sel_pat + k;
+  if (io.exp_dev != nullptr && threadIdx.x < 9) io.exp_dev[(size_t)chunk * 9 + threadIdx.x] = 0;
+}
 
-  // decode the commitment; its indices must ascend strictly and lie inside the chunk
+// Algorithm 2 with a look-up in place of the polynomial, by a block of T threads: the k selected
+// (index, pattern) pairs are in sel_idx / sel_pat (any order, all written and visible); the
+// commitment is decoded into com_idx / com_pat, checked (indices ascend strictly, lie inside the
+// chunk), and every selected index is looked up in it.  Writes the chunk's result.
+template <int T>
+__device__ void compare_with_commitment(CompareScratch& cs, const DirectVerify& io, long long chunk, int k, uint32_t n_elems,
+                                        const uint32_t* sel_idx, const uint16_t* sel_pat, uint32_t* com_idx,
+                                        uint16_t* com_pat) {
+  if (threadIdx.x == 0) cs.bad = 0;
+  if (threadIdx.x < 4) cs.counters[threadIdx.x] = 0;
+  if (threadIdx.x < 9) cs.dev[threadIdx.x] = 0;
   const uint16_t* rec = reinterpret_cast<const uint16_t*>(io.commits + (size_t)chunk * 6u * (size_t)k);
-  for (int j = threadIdx.x; j < k; j += kThreads) {
+  for (int j = threadIdx.x; j < k; j += T) {
     com_idx[j] = (uint32_t)rec[3 * j] | ((uint32_t)rec[3 * j + 1] << 16);
     com_pat[j] = rec[3 * j + 2];
   }
-  for (int b = threadIdx.x; b < 128; b += kThreads) sh.hist[b] = 0;  // mantissa differences 0..127
+  for (int b = threadIdx.x; b < 128; b += T) cs.hist[b] = 0;
   __syncthreads();
   {
     uint32_t bad = 0;
-    for (int j = threadIdx.x; j < k; j += kThreads)
-      bad |= (com_idx[j] >= n_elems) | (j > 0 && com_idx[j] <= com_idx[j - 1]);
-    if (bad) sh.bad = 1;
+    for (int j = threadIdx.x; j < k; j += T) bad |= (com_idx[j] >= n_elems) | (j > 0 && com_idx[j] <= com_idx[j - 1]);
+    if (bad) cs.bad = 1;
     __syncthreads();
-    if (sh.bad) {
-      refuse(TOPLOC_CHUNK_BAD_PROOF);
+    if (cs.bad) {
+      refuse_chunk(io, chunk, TOPLOC_CHUNK_BAD_PROOF);
       return;
     }
   }
-
-  // Algorithm 2 with a look-up in place of the polynomial
   uint32_t err_e = 0, n_match = 0, sum = 0, common = 0, dev[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
   const int sign_in_exponent = io.thr_each ? io.thr_each[chunk].sign_in_exponent : io.thr.sign_in_exponent;
-  for (int j = threadIdx.x; j < k; j += kThreads) {
+  for (int j = threadIdx.x; j < k; j += T) {
     const uint32_t want = sel_idx[j];
     int lo = 0, hi = k;  // first committed index >= want
     while (lo < hi) {
@@ -1017,7 +1100,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
       const uint32_t d = mp > mv ? mp - mv : mv - mp;
       ++n_match;
       sum += d;
-      atomicAdd(&sh.hist[d], 1u);
+      atomicAdd(&cs.hist[d], 1u);
     } else {
       ++err_e;
     }
@@ -1034,22 +1117,22 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
 #pragma unroll
   for (int b = 0; b < 9; ++b) dev[b] = __reduce_add_sync(0xFFFFFFFFu, dev[b]);
   if ((threadIdx.x & 31) == 0) {
-    atomicAdd(&sh.counters[0], err_e);
-    atomicAdd(&sh.counters[1], n_match);
-    atomicAdd(&sh.counters[2], sum);
-    atomicAdd(&sh.counters[3], common);
+    atomicAdd(&cs.counters[0], err_e);
+    atomicAdd(&cs.counters[1], n_match);
+    atomicAdd(&cs.counters[2], sum);
+    atomicAdd(&cs.counters[3], common);
 #pragma unroll
     for (int b = 0; b < 9; ++b)
-      if (dev[b]) atomicAdd(&sh.dev[b], dev[b]);
+      if (dev[b]) atomicAdd(&cs.dev[b], dev[b]);
   }
   __syncthreads();
-  if (io.exp_dev != nullptr && threadIdx.x < 9) io.exp_dev[(size_t)chunk * 9 + threadIdx.x] = sh.dev[threadIdx.x];
+  if (io.exp_dev != nullptr && threadIdx.x < 9) io.exp_dev[(size_t)chunk * 9 + threadIdx.x] = cs.dev[threadIdx.x];
   if (threadIdx.x == 0) {
     toploc_chunk_result r = {};
-    r.exp_mismatch = sh.counters[0];
-    r.n_match = sh.counters[1];
-    r.mant_diff_sum = sh.counters[2];
-    r.topk_mismatch = k - (int)sh.counters[3];
+    r.exp_mismatch = cs.counters[0];
+    r.n_match = cs.counters[1];
+    r.mant_diff_sum = cs.counters[2];
+    r.topk_mismatch = k - (int)cs.counters[3];
     const toploc_thresholds thr = io.thr_each ? io.thr_each[chunk] : io.thr;
     bool reject = (long long)r.exp_mismatch > (long long)thr.t_exp;
     if (r.n_match > 0) {
@@ -1059,7 +1142,7 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
       uint32_t seen = 0;
       int lo_val = -1, hi_val = -1;
       for (int b = 0; b < 128 && hi_val < 0; ++b) {
-        seen += sh.hist[b];
+        seen += cs.hist[b];
         if (lo_val < 0 && seen > lo_rank) lo_val = b;
         if (seen > hi_rank) hi_val = b;
       }
@@ -1073,7 +1156,200 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
     io.results[chunk] = r;
   }
 }
+static_assert(sizeof(CompareScratch) <= 4 * kListOffset, "the comparison's scratch sits below the verify lists");
 
+// One chunk's validation by a 1024-thread block (see commit_one_chunk for loose_failed).
+template <int DT, bool VECTOR>
+__device__ void verify_one_chunk(DirectShared& sh, uint4* ring, const DirectParams& p, long long chunk, const DirectVerify& io,
+                                 bool loose_failed) {
+  // The two selections live where the key histogram was (it is done with once the k-th key is
+  // known), or, after a one-pass selection, in the ring (idle by then).
+  uint32_t* sel_idx = sh.hist + kListOffset;
+  uint16_t* sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * p.k);
+  using R = Reader<DT, VECTOR>;
+  const int k = p.k;
+  const R rd = locate_chunk<DT, VECTOR>(p, chunk);
+  const uint32_t n_elems = (uint32_t)rd.n_groups * R::VEC;
+  if (n_elems < (uint32_t)k) {
+    refuse_chunk(io, chunk, TOPLOC_CHUNK_K_EXCEEDS_CHUNK);
+    return;
+  }
+  auto emit = [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+    if (pos >= (uint32_t)k) return;
+    sel_idx[pos] = flat;
+    sel_pat[pos] = (uint16_t)pat;
+  };
+  bool done = false;
+  if constexpr (VECTOR) {
+    const bool loose = n_elems <= (uint32_t)kLooseMaxElems;  // the comparison needs no particular order
+    if (!loose_failed && (loose || k <= kStreamMaxK)) {
+      sel_idx = reinterpret_cast<uint32_t*>(ring);
+      sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
+      done = loose ? select_unordered<DT, false, kThreads>(loose_workspace<DT>(sh), ring, rd, k, emit)
+                   : select_in_one_pass<DT>(sh, ring, rd, k, emit);
+    }
+  }
+  if (!done) {
+    sel_idx = sh.hist + kListOffset;
+    sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
+    uint32_t kth, take;
+    find_kth_key<DT, VECTOR>(sh, ring, rd, k, &kth, &take);
+    collect_in_index_order<DT, VECTOR>(sh, ring, rd, k, kth, take, emit);
+  }
+  __syncthreads();
+  CompareScratch& cs = *reinterpret_cast<CompareScratch*>(sh.hist);  // (below kListOffset words: free in either case)
+  compare_with_commitment<kThreads>(cs, io, chunk, k, n_elems, sel_idx, sel_pat, sel_idx + k, sel_pat + k);
+}
+
+template <int DT, bool VECTOR>
+__global__ void __launch_bounds__(kThreads, 1)
+toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw);
+  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw + kRingBytes);
+  verify_one_chunk<DT, VECTOR>(sh, ring, p, blockIdx.x, io, false);
+}
+
+// ---------------------------------------------------------------------------
+// 512 < k, vector layouts, chunks of at most 2^18 elements: the two-pass selection without
+// barriers needs little more than k candidate slots, so two 512-thread blocks share an SM (113 KB
+// each) and one chunk's serial phases -- threshold, exact key, ties, ranking -- run under the
+// other's loads.  A chunk whose candidates outgrow the smaller buffer (many equal values) is
+// marked and taken by the rescue launch that follows in the same call: a few 1024-thread blocks
+// that look at every chunk's mark and run the radix select on the marked ones.
+// ---------------------------------------------------------------------------
+namespace half_block {
+constexpr int kT = 512;
+constexpr int kW = kT / 32;
+constexpr size_t kRing = (size_t)kUnroll * kT * 16;         // 32 KB; later one bit per element of the chunk
+constexpr long long kMaxElems = (long long)kRing * 8;       // 2^18
+constexpr size_t kPark = (size_t)kW * kParkCap * 4;
+constexpr size_t kFixed = kRing + sizeof(LooseControl) + sizeof(CompareScratch) + (size_t)kCoarseBins * 4 + kPark;
+constexpr size_t kBlockBytes = (227 * 1024) / 2 - 1024;      // two blocks per SM, 1 KB reserved for each
+__host__ __device__ constexpr int cap(int dt) { return (int)((kBlockBytes - kFixed) / (dt == 0 ? 6 : 8)) / 64 * 64; }
+static_assert(kFixed % 16 == 0 && cap(0) >= 2 * 4096 && cap(1) >= 4096 + 2048, "room for the candidates of k = 4096");
+static_assert(6 * TOPLOC_MAX_K_DIRECT <= kRing && 6 * TOPLOC_MAX_K_DIRECT <= 6 * 4096,
+              "the selection fits the ring, the decoded commitment the candidates' place");
+
+struct Carve {
+  uint4* ring;
+  CompareScratch* cs;
+};
+
+template <int DT>
+__device__ __forceinline__ LooseWorkspace<DT> carve(unsigned char* smem, Carve* out) {
+  LooseWorkspace<DT> ws;
+  out->ring = reinterpret_cast<uint4*>(smem);
+  unsigned char* at = smem + kRing;
+  ws.ctl = reinterpret_cast<LooseControl*>(at);
+  at += sizeof(LooseControl);
+  out->cs = reinterpret_cast<CompareScratch*>(at);
+  at += sizeof(CompareScratch);
+  ws.coarse = reinterpret_cast<uint32_t*>(at);
+  at += (size_t)kCoarseBins * 4;
+  ws.park = reinterpret_cast<uint32_t*>(at);
+  at += kPark;
+  ws.cap = cap(DT);
+  ws.cand_flat = reinterpret_cast<uint32_t*>(at);
+  ws.cand_pat = reinterpret_cast<typename StoredPattern<DT>::type*>(ws.cand_flat + ws.cap);
+  return ws;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kT, 2) toploc_direct_commit_half_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Carve cv;
+  const LooseWorkspace<DT> ws = carve<DT>(smem_raw, &cv);
+  using R = Reader<DT, true>;
+  const long long chunk = blockIdx.x;
+  const R rd = locate_chunk<DT, true>(p, chunk);
+  uint16_t* rec = reinterpret_cast<uint16_t*>(commits + (size_t)chunk * 6u * (size_t)p.k);
+  if ((long long)rd.n_groups * R::VEC < p.k) {
+    for (int i = threadIdx.x; i < 3 * p.k; i += kT) rec[i] = 0;
+    if (threadIdx.x == 0) status[chunk] = TOPLOC_CHUNK_K_EXCEEDS_CHUNK;
+    return;
+  }
+  auto emit = [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+    if (pos >= (uint32_t)p.k) return;
+    rec[3 * pos] = (uint16_t)(flat & 0xFFFFu);
+    rec[3 * pos + 1] = (uint16_t)(flat >> 16);
+    rec[3 * pos + 2] = (uint16_t)pat;
+  };
+  const bool done = select_unordered<DT, true, kT>(ws, cv.ring, rd, p.k, emit);
+  if (threadIdx.x == 0) status[chunk] = done ? TOPLOC_CHUNK_OK : kRetry;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kT, 2) toploc_direct_verify_half_kernel(DirectParams p, DirectVerify io) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Carve cv;
+  const LooseWorkspace<DT> ws = carve<DT>(smem_raw, &cv);
+  using R = Reader<DT, true>;
+  const long long chunk = blockIdx.x;
+  const int k = p.k;
+  const R rd = locate_chunk<DT, true>(p, chunk);
+  const uint32_t n_elems = (uint32_t)rd.n_groups * R::VEC;
+  if (n_elems < (uint32_t)k) {
+    refuse_chunk(io, chunk, TOPLOC_CHUNK_K_EXCEEDS_CHUNK);
+    return;
+  }
+  // the selection goes to the ring (idle once the chunk has streamed), the decoded commitment where
+  // the candidates were (done with once the selection has been written out)
+  uint32_t* sel_idx = reinterpret_cast<uint32_t*>(cv.ring);
+  uint16_t* sel_pat = reinterpret_cast<uint16_t*>(sel_idx + k);
+  auto emit = [&](uint32_t pos, uint32_t flat, uint32_t pat) {
+    if (pos >= (uint32_t)k) return;
+    sel_idx[pos] = flat;
+    sel_pat[pos] = (uint16_t)pat;
+  };
+  if (!select_unordered<DT, false, kT>(ws, cv.ring, rd, k, emit)) {
+    if (threadIdx.x == 0) {
+      toploc_chunk_result r = {};
+      r.status = kRetry;
+      io.results[chunk] = r;
+    }
+    return;
+  }
+  __syncthreads();
+  uint32_t* com_idx = ws.cand_flat;
+  uint16_t* com_pat = reinterpret_cast<uint16_t*>(com_idx + k);
+  compare_with_commitment<kT>(*cv.cs, io, chunk, k, n_elems, sel_idx, sel_pat, com_idx, com_pat);
+}
+
+// The rescue launch: 1024-thread blocks, one per SM at most, look at every chunk's mark.
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 1) toploc_direct_commit_rescue_kernel(DirectParams p, long long num_chunks,
+                                                                                  uint8_t* commits, uint8_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw);
+  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw + kRingBytes);
+  for (long long chunk = blockIdx.x; chunk < num_chunks; chunk += gridDim.x) {
+    if (status[chunk] != kRetry) continue;  // (the same for every thread: the mark is only rewritten below, after barriers)
+    __syncthreads();
+    commit_one_chunk<DT, true>(sh, ring, p, chunk, commits, status, true);
+    __syncthreads();
+  }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 1) toploc_direct_verify_rescue_kernel(DirectParams p, long long num_chunks,
+                                                                                  DirectVerify io) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw);
+  DirectShared& sh = *reinterpret_cast<DirectShared*>(smem_raw + kRingBytes);
+  for (long long chunk = blockIdx.x; chunk < num_chunks; chunk += gridDim.x) {
+    if (io.results[chunk].status != kRetry) continue;
+    __syncthreads();
+    verify_one_chunk<DT, true>(sh, ring, p, chunk, io, true);
+    __syncthreads();
+  }
+}
+
+inline bool applies(const toploc_layout* lay, bool vector) {
+  const long long rows = lay->tokens_per_seq < lay->chunk_len ? lay->tokens_per_seq : lay->chunk_len;
+  return vector && rows * lay->hidden <= kMaxElems;
+}
+}  // namespace half_block
 
 // ---------------------------------------------------------------------------
 // Small k (k <= TOPLOC_MAX_K = 512, chunks of at most 2^19 elements): one warp per chunk, the
@@ -1368,6 +1644,7 @@ struct DirectPlan {
   DirectParams params;
   long long num_chunks;
   bool vector;
+  int device;  // filled by check_device
 };
 
 int plan_direct(const void* d_act, const toploc_layout* lay, DirectPlan* plan) {
@@ -1398,20 +1675,21 @@ int plan_direct(const void* d_act, const toploc_layout* lay, DirectPlan* plan) {
   return TOPLOC_OK;
 }
 
-int check_device() {
+int check_device(DirectPlan* plan) {
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return TOPLOC_ERR_CUDA;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TOPLOC_ERR_CUDA;
+  plan->device = dev;
   return major == 10 ? TOPLOC_OK : TOPLOC_ERR_ARCH;
 }
 
-template <class Kernel, class... Args>
-int launch_direct(Kernel kernel, long long num_chunks, size_t smem, cudaStream_t stream, Args... args) {
+template <int T = kThreads, class Kernel, class... Args>
+int launch_direct(Kernel kernel, long long num_blocks, size_t smem, cudaStream_t stream, Args... args) {
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     cudaGetLastError();
     return TOPLOC_ERR_CUDA;
   }
-  kernel<<<(unsigned)num_chunks, kThreads, smem, stream>>>(args...);
+  kernel<<<(unsigned)num_blocks, T, smem, stream>>>(args...);
   return cudaGetLastError() == cudaSuccess ? TOPLOC_OK : TOPLOC_ERR_CUDA;
 }
 
@@ -1428,7 +1706,7 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
   if (rc != TOPLOC_OK) return rc;
   if (d_commits == nullptr || d_status == nullptr || (reinterpret_cast<uintptr_t>(d_commits) & 1u) != 0)
     return TOPLOC_ERR_INVALID_ARGUMENT;
-  if ((rc = check_device()) != TOPLOC_OK) return rc;
+  if ((rc = check_device(&plan)) != TOPLOC_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
@@ -1436,6 +1714,25 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
     const int mode = small_k::layout_mode(d_act, lay);
     return lay->dtype == TOPLOC_DTYPE_BF16 ? small_k::launch_commit<0>(mode, plan.num_chunks, stream, p, d_commits, d_status)
                                            : small_k::launch_commit<1>(mode, plan.num_chunks, stream, p, d_commits, d_status);
+  }
+  if (half_block::applies(lay, plan.vector)) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, plan.device) != cudaSuccess) return TOPLOC_ERR_CUDA;
+    const long long rescuers = plan.num_chunks < sms ? plan.num_chunks : sms;
+    if (lay->dtype == TOPLOC_DTYPE_BF16) {
+      rc = launch_direct<half_block::kT>(half_block::toploc_direct_commit_half_kernel<0>, plan.num_chunks,
+                                         half_block::kBlockBytes, stream, p, d_commits, d_status);
+      if (rc == TOPLOC_OK)
+        rc = launch_direct(half_block::toploc_direct_commit_rescue_kernel<0>, rescuers, smem, stream, p, plan.num_chunks,
+                           d_commits, d_status);
+    } else {
+      rc = launch_direct<half_block::kT>(half_block::toploc_direct_commit_half_kernel<1>, plan.num_chunks,
+                                         half_block::kBlockBytes, stream, p, d_commits, d_status);
+      if (rc == TOPLOC_OK)
+        rc = launch_direct(half_block::toploc_direct_commit_rescue_kernel<1>, rescuers, smem, stream, p, plan.num_chunks,
+                           d_commits, d_status);
+    }
+    return rc;
   }
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_commit_kernel<0, true>, plan.num_chunks, smem, stream, p, d_commits, d_status)
@@ -1459,7 +1756,7 @@ static int verify_direct_with(const void* d_act, const toploc_layout* lay, const
       (reinterpret_cast<uintptr_t>(d_exp_dev_opt) & 3u) != 0 || (reinterpret_cast<uintptr_t>(d_thr_each) & 7u) != 0)
     return TOPLOC_ERR_INVALID_ARGUMENT;
   if (thr != nullptr && thr->t_exp < 0) return TOPLOC_ERR_INVALID_ARGUMENT;
-  if ((rc = check_device()) != TOPLOC_OK) return rc;
+  if ((rc = check_device(&plan)) != TOPLOC_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   DirectVerify io;
   io.commits = d_commits;
@@ -1473,6 +1770,23 @@ static int verify_direct_with(const void* d_act, const toploc_layout* lay, const
     const int mode = small_k::layout_mode(d_act, lay);
     return lay->dtype == TOPLOC_DTYPE_BF16 ? small_k::launch_verify<0>(mode, plan.num_chunks, stream, p, io)
                                            : small_k::launch_verify<1>(mode, plan.num_chunks, stream, p, io);
+  }
+  if (half_block::applies(lay, plan.vector)) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, plan.device) != cudaSuccess) return TOPLOC_ERR_CUDA;
+    const long long rescuers = plan.num_chunks < sms ? plan.num_chunks : sms;
+    if (lay->dtype == TOPLOC_DTYPE_BF16) {
+      rc = launch_direct<half_block::kT>(half_block::toploc_direct_verify_half_kernel<0>, plan.num_chunks,
+                                         half_block::kBlockBytes, stream, p, io);
+      if (rc == TOPLOC_OK)
+        rc = launch_direct(half_block::toploc_direct_verify_rescue_kernel<0>, rescuers, smem, stream, p, plan.num_chunks, io);
+    } else {
+      rc = launch_direct<half_block::kT>(half_block::toploc_direct_verify_half_kernel<1>, plan.num_chunks,
+                                         half_block::kBlockBytes, stream, p, io);
+      if (rc == TOPLOC_OK)
+        rc = launch_direct(half_block::toploc_direct_verify_rescue_kernel<1>, rescuers, smem, stream, p, plan.num_chunks, io);
+    }
+    return rc;
   }
   if (lay->dtype == TOPLOC_DTYPE_BF16)
     return plan.vector ? launch_direct(toploc_direct_verify_kernel<0, true>, plan.num_chunks, smem, stream, p, io)
