@@ -506,14 +506,25 @@ __device__ __forceinline__ uint32_t vector_max_coarse_key(const uint4& w) {
 // and leaves the histograms empty again.
 template <int DT, int MODE, class SH>
 __device__ __noinline__ uint32_t sound_first_threshold(SH& sh, const ChunkSource<DT, MODE> src,
-                                                       int n_first, int k) {
+                                                       int n_first, int k, int ring_vecs) {
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x & 31;
   uint16_t* maxima = reinterpret_cast<uint16_t*>(sh.cand);
   warp_barrier();
+  // The first ring_vecs vectors are on their way into the ring already (vector v in slot v,
+  // copied by the lane that reads it here): the vectors beyond them are loaded first, then the
+  // ring's are taken from shared memory once they have landed -- one round trip to memory for
+  // the whole look-ahead of the common case instead of one per four vectors of a lane.
+  if (ring_vecs > n_first) ring_vecs = n_first;
 #pragma unroll 4
-  for (int v = lane; v < n_first; v += kThreads) {
+  for (int v = ring_vecs + lane; v < n_first; v += kThreads) {
     const uint32_t key = vector_max_coarse_key<DT, VEC>(src.load(v));
+    maxima[v] = (uint16_t)key;
+    atomicAdd(&sh.top_hist[key >> 7], 1u);
+  }
+  if (ring_vecs > 0) copy_async_wait<0>();
+  for (int v = lane; v < ring_vecs; v += kThreads) {
+    const uint32_t key = vector_max_coarse_key<DT, VEC>(sh.ring[v]);
     maxima[v] = (uint16_t)key;
     atomicAdd(&sh.top_hist[key >> 7], 1u);
   }
@@ -601,7 +612,7 @@ __device__ void select_topk(SH& sh, const ChunkSource<DT, MODE>& src, int n_elem
   for (int t = 0; t < kStages; ++t) request_tile(t, t);
   warp_barrier();
 
-  if (look_ahead) st.thr = sound_first_threshold<DT, MODE>(sh, src, first, k);
+  if (look_ahead) st.thr = sound_first_threshold<DT, MODE>(sh, src, first, k, kRing ? min(n_tiles, kStages) * kTileVecs : 0);
   else st = select_carefully<DT, MODE>(sh, src, 0, warm, k, st);
 
   for (int tile0 = 0; tile0 < n_tiles; tile0 += kStages) {
