@@ -126,6 +126,21 @@ def test_rising_magnitudes_outgrow_the_candidate_buffer():
     direct_case(act, L, k, 2, L, {"falling": torch.cat([rising.flip(0).flip(1), usual]).contiguous()}, "rising")
 
 
+def test_many_equal_values_go_to_the_rescue_launch():
+    """k above 512 on chunks of the 70B shape: a chunk of equal magnitudes makes every element a
+    candidate, which outgrows the half-block kernel's buffer; that chunk is marked and taken by
+    the rescue launch of the same call, its ordinary neighbours are not."""
+    H, L, k = 8192, 32, 1024
+    usual = synth.make_activations(2, L, H, torch.bfloat16, seed=78, device=DEV, outliers="none")
+    flat = torch.where(torch.arange(L * H, device=DEV).reshape(L, H) % 5 == 0, -3.0, 3.0).to(torch.bfloat16)
+    act = torch.cat([usual[:L], flat, usual[L:]]).contiguous()
+    out = direct_case(act, L, k, 3, L, {"noise": synth.honest_noise(act, seed=4)}, "equal values, k=1024")
+    assert out["same"]["status"].tolist() == [0, 0, 0] and (out["same"]["accept"] == 1).all()
+    direct_case(act, L, 4096, 3, L, None, "equal values, k=4096")
+    f = act.float()
+    direct_case(f, L, 2048, 3, L, None, "equal values, fp32")
+
+
 def test_special_patterns():
     H, L, k = 512, 8, 200
     bits = torch.randint(0, 65536, (L, H), dtype=torch.int32, device=DEV).to(torch.int16)  # NaN, Inf, subnormals
