@@ -690,17 +690,38 @@ __device__ __forceinline__ void evaluate_warp(SH& sh, int k, long long chunk, co
 // ---------------------------------------------------------------------------
 // The 32-bit field: fp32 chunks that commit whole patterns work in Z_q,
 // q = 2^32 - 5 (products are 64 bits wide and 2^32 = 5 folds them back).  A
-// table of inverses is out of reach, so Algorithm 3 is arranged around k
-// inversions per chunk instead of k^2 / 2.
+// table of inverses is out of reach, so Algorithm 3 is arranged around ONE
+// inversion per chunk.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t reduce_q(unsigned long long t) {
-  unsigned long long s = (t & 0xFFFFFFFFull) + 5ull * (t >> 32);  // < 6 * 2^32
-  s = (s & 0xFFFFFFFFull) + 5ull * (s >> 32);                     // < 2^32 + 25 < 2q
-  return (uint32_t)(s >= kPrime32 ? s - kPrime32 : s);
+
+// hi * 2^32 + lo reduced into [0, q): 2^32 == 5, so the value is 5 hi + lo; that sum has at most
+// three bits above the 32nd, which fold the same way; a last wrap of 2^32 adds 5 to a small rest.
+__device__ __forceinline__ uint32_t fold_q(uint32_t hi, uint32_t lo) {
+  uint32_t s, above, r, wrapped;
+  asm("{\n\t"
+      ".reg .u32 l5, h5;\n\t"
+      "mul.lo.u32 l5, %2, 5;\n\t"
+      "mul.hi.u32 h5, %2, 5;\n\t"
+      "add.cc.u32 %0, %3, l5;\n\t"
+      "addc.u32 %1, h5, 0;\n\t"
+      "}"
+      : "=r"(s), "=r"(above)
+      : "r"(hi), "r"(lo));
+  asm("mad.lo.cc.u32 %0, %2, 5, %3;\n\t"
+      "addc.u32 %1, 0, 0;"
+      : "=r"(r), "=r"(wrapped)
+      : "r"(above), "r"(s));
+  r += 5u * wrapped;              // above <= 5: after a wrap the rest is below 25
+  return min(r, r - kPrime32);    // r - q wraps to a huge value when r < q
 }
-__device__ __forceinline__ uint32_t mul_q(uint32_t a, uint32_t b) { return reduce_q((unsigned long long)a * b); }
+__device__ __forceinline__ uint32_t mul_q(uint32_t a, uint32_t b) { return fold_q(__umulhi(a, b), a * b); }
 __device__ __forceinline__ uint32_t mad_q(uint32_t a, uint32_t b, uint32_t c) {
-  return reduce_q((unsigned long long)a * b + c);
+  uint32_t lo, hi;
+  asm("mad.lo.cc.u32 %0, %2, %3, %4;\n\t"
+      "madc.hi.u32 %1, %2, %3, 0;"
+      : "=r"(lo), "=r"(hi)
+      : "r"(a), "r"(b), "r"(c));
+  return fold_q(hi, lo);
 }
 __device__ __forceinline__ uint32_t sub_q(uint32_t a, uint32_t b) { return a >= b ? a - b : a + (kPrime32 - b); }
 
@@ -719,87 +740,111 @@ __device__ __forceinline__ uint32_t inv_q(uint32_t a) {
 // Algorithm 3 (InterpolateModPolynomial) over Z_q for one chunk, by one warp.
 // Point j lives in lane j % 32, slot j / 32.  The Newton coefficient of point i is
 //   a_i = (y_i - P_{i-1}(x_i)) / N_i(x_i),   N_i(x) = prod_{l < i} (x - x_l),
-// where P_{i-1} interpolates the first i points.  A first sweep forms every
-// denominator N_j(x_j) (they do not depend on y) and inverts the k of them; a
-// second sweep carries, for every later point j, the partial sum
-// S_j = P_{i-1}(x_j) and the partial product N_i(x_j); only a_i and x_i are
-// broadcast per step.  The Newton form is then multiplied out from the inside,
+// where P_{i-1} interpolates the first i points.  Every point j carries
+// n_j = N_i(x_j) and, instead of t_j = y_j - P_{i-1}(x_j), the multiple
+// T_j = s_i t_j with s_i = n_0 n_1 ... n_{i-1} (the pivots' n so far), because
+//   t_j <- t_j - (t_i / n_i) n_j      becomes      T_j <- n_i T_j - T_i n_j
+// without any division; then a_i = T_i / s_{i+1}.  The divisors are prefix
+// products of the pivots' n_i, so ONE inversion of the last one and a suffix
+// product per point give them all:  1 / s_{i+1} = (1 / s_k) n_{i+1} ... n_{k-1}.
+// The Newton form is then multiplied out from the inside,
 //   P <- P * (x - x_i) + a_i  for i = k-2 .. 0,
-// with coefficient d in lane d / SLOTS, slot d % SLOTS, so the shift by one
-// degree stays inside a lane except for one value per lane and step.
-// row_x / row_a: this warp's scratch rows of kMaxK words in shared memory.
+// with coefficient d in lane d % 32, slot d / 32: slots above the current degree hold zeros and
+// are skipped, the shift by one degree is a rotation of every live slot by one lane.
+// row_x / row_t / row_n: this warp's scratch rows in shared memory (x_i; T_i, later a_i; n_i).
 template <int SLOTS>
 __device__ __forceinline__ void interpolate_warp_q(int k, const uint32_t (&x)[SLOTS], const uint32_t (&y)[SLOTS],
-                                                   uint32_t* row_x, uint32_t* row_a, uint16_t* proof) {
+                                                   uint16_t* row_x, uint32_t* row_t, uint32_t* row_n, uint16_t* proof) {
   const int lane = threadIdx.x & 31;
   constexpr uint32_t kFull = 0xFFFFFFFFu;
-  uint32_t den[SLOTS];
-#pragma unroll
-  for (int s = 0; s < SLOTS; ++s) den[s] = 1u;
-#pragma unroll
-  for (int b = 0; b < SLOTS; ++b) {
-    const int steps = min(32, k - 1 - 32 * b);  // points i = 32b + ii with i + 1 < k
-#pragma unroll 1
-    for (int ii = 0; ii < steps; ++ii) {
-      const uint32_t xi = __shfl_sync(kFull, x[b], ii);
-      den[b] = mul_q(den[b], lane > ii ? sub_q(x[b], xi) : 1u);
-#pragma unroll
-      for (int s = b + 1; s < SLOTS; ++s) den[s] = mul_q(den[s], sub_q(x[s], xi));
-    }
-  }
-  uint32_t inv_den[SLOTS];
-#pragma unroll
-  for (int s = 0; s < SLOTS; ++s) inv_den[s] = inv_q(den[s]);
-
-  uint32_t part[SLOTS], prod[SLOTS];  // S_j and N_i(x_j)
+  uint32_t T[SLOTS], N[SLOTS];
 #pragma unroll
   for (int s = 0; s < SLOTS; ++s) {
-    part[s] = 0u;
-    prod[s] = 1u;
-    if (s * 32 + lane < k) row_x[s * 32 + lane] = x[s];
+    T[s] = y[s];
+    N[s] = 1u;
   }
+  uint32_t scale = 1u;  // s_i, the same in every lane
 #pragma unroll
   for (int b = 0; b < SLOTS; ++b) {
-    const int steps = min(32, k - 32 * b);  // includes the last point, which only yields its a
+    const int steps = min(32, k - 32 * b);  // the last point only hands out its T and n
 #pragma unroll 1
     for (int ii = 0; ii < steps; ++ii) {
-      // every lane forms the quotient of its own slot-b point; lane ii's is a_i
-      const uint32_t quot = mul_q(sub_q(y[b], part[b]), inv_den[b]);
-      const uint32_t a_i = __shfl_sync(kFull, quot, ii);
+      const uint32_t ni = __shfl_sync(kFull, N[b], ii);
+      const uint32_t ti = __shfl_sync(kFull, T[b], ii);
       const uint32_t xi = __shfl_sync(kFull, x[b], ii);
-      if (lane == ii) row_a[32 * b + ii] = a_i;
+      scale = mul_q(scale, ni);
+      if (lane == 0) {
+        row_x[32 * b + ii] = (uint16_t)xi;  // x = index mod m is below 2^16
+        row_t[32 * b + ii] = ti;
+        row_n[32 * b + ii] = ni;
+      }
       const bool later = lane > ii;
-      const uint32_t part_b = mad_q(a_i, prod[b], part[b]);
-      const uint32_t prod_b = mul_q(prod[b], sub_q(x[b], xi));
-      part[b] = later ? part_b : part[b];
-      prod[b] = later ? prod_b : prod[b];
+      const uint32_t tb = sub_q(mul_q(ni, T[b]), mul_q(ti, N[b]));
+      const uint32_t nb = mul_q(N[b], sub_q(x[b], xi));
+      T[b] = later ? tb : T[b];
+      N[b] = later ? nb : N[b];
 #pragma unroll
       for (int s = b + 1; s < SLOTS; ++s) {
-        part[s] = mad_q(a_i, prod[s], part[s]);
-        prod[s] = mul_q(prod[s], sub_q(x[s], xi));
+        T[s] = sub_q(mul_q(ni, T[s]), mul_q(ti, N[s]));
+        N[s] = mul_q(N[s], sub_q(x[s], xi));
       }
+    }
+  }
+  __syncwarp();
+  // a_i = T_i / s_{i+1}: lane l owns i = l * SLOTS .. l * SLOTS + SLOTS - 1
+  {
+    const uint32_t inv_last = inv_q(scale);  // 1 / s_k
+    uint32_t own[SLOTS], after[SLOTS];       // n_i, and the product of the n beyond i inside this lane
+#pragma unroll
+    for (int e = 0; e < SLOTS; ++e) {
+      const int i = lane * SLOTS + e;
+      own[e] = i < k ? row_n[i] : 1u;
+    }
+    after[SLOTS - 1] = 1u;
+#pragma unroll
+    for (int e = SLOTS - 2; e >= 0; --e) after[e] = mul_q(after[e + 1], own[e + 1]);
+    uint32_t from_here = mul_q(after[0], own[0]);  // product over this lane's i, then over the lanes above too
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t other = __shfl_down_sync(kFull, from_here, off);
+      if (lane + off < 32) from_here = mul_q(from_here, other);
+    }
+    uint32_t beyond = __shfl_down_sync(kFull, from_here, 1);  // the lanes above this one
+    if (lane == 31) beyond = 1u;
+    const uint32_t base = mul_q(inv_last, beyond);
+#pragma unroll
+    for (int e = 0; e < SLOTS; ++e) {
+      const int i = lane * SLOTS + e;
+      if (i < k) row_t[i] = mul_q(row_t[i], mul_q(base, after[e]));
     }
   }
   __syncwarp();
   uint32_t co[SLOTS];
 #pragma unroll
   for (int b = 0; b < SLOTS; ++b) co[b] = 0u;
-  if (lane == 0) co[0] = row_a[k - 1];
-#pragma unroll 1
-  for (int i = k - 2; i >= 0; --i) {
-    const uint32_t neg_x = sub_q(0u, row_x[i]);
-    const uint32_t a_i = row_a[i];
-    // coefficient d takes  c[d-1] + (-x_i) c[d];  entries above the current degree are 0 and stay 0
-    uint32_t carry = __shfl_up_sync(kFull, co[SLOTS - 1], 1);
-    if (lane == 0) carry = a_i;
+  if (lane == 0) co[0] = row_t[k - 1];
+  const int from = (lane + 31) & 31;
 #pragma unroll
-    for (int b = SLOTS - 1; b >= 1; --b) co[b] = mad_q(co[b], neg_x, co[b - 1]);
-    co[0] = mad_q(co[0], neg_x, carry);
+  for (int top = 0; top < SLOTS; ++top) {  // the slot that holds the leading coefficient
+    const int d_first = max(32 * top, 1), d_last = min(32 * top + 31, k - 1);
+#pragma unroll 1
+    for (int D = d_first; D <= d_last; ++D) {
+      const int i = k - 1 - D;
+      const uint32_t neg_x = sub_q(0u, (uint32_t)row_x[i]);
+      const uint32_t a_i = row_t[i];
+      uint32_t below[SLOTS];  // coefficient d - 1, as seen from the owner of coefficient d
+#pragma unroll
+      for (int b = 0; b <= top; ++b) below[b] = __shfl_sync(kFull, co[b], from);
+      // coefficient d takes  c[d-1] + (-x_i) c[d]
+#pragma unroll
+      for (int b = top; b >= 1; --b) co[b] = mad_q(co[b], neg_x, lane == 0 ? below[b - 1] : below[b]);
+      co[0] = mad_q(co[0], neg_x, lane == 0 ? a_i : below[0]);
+    }
   }
   // proof bytes 2 + 4d .. 5 + 4d: coefficient of degree d, little-endian (the proof is 2-byte aligned)
 #pragma unroll
   for (int b = 0; b < SLOTS; ++b) {
-    const int d = lane * SLOTS + b;
+    const int d = b * 32 + lane;
     if (d < k) {
       proof[1 + 2 * d] = (uint16_t)(co[b] & 0xFFFFu);
       proof[2 + 2 * d] = (uint16_t)(co[b] >> 16);
@@ -812,7 +857,8 @@ constexpr int kInterpQWarps = 8;  // 32-bit field interpolation: warps (chunks) 
 // InterpolateModPolynomial() and encode() of Algorithm 1 over Z_q for every
 // chunk the select (or merge) kernel finished, one warp per chunk.
 template <int SLOTS>
-__device__ __forceinline__ void interpolate_chunk_q(const Selection& sel, int k, long long chunk, uint32_t* rows) {
+__device__ __forceinline__ void interpolate_chunk_q(const Selection& sel, int k, long long chunk, uint32_t* rows,
+                                                    uint16_t* row_x) {
   const int lane = threadIdx.x & 31;
   uint16_t* proof = reinterpret_cast<uint16_t*>(sel.proofs + chunk * (2 + 4 * (size_t)k));
   uint32_t m = proof[0];
@@ -829,22 +875,23 @@ __device__ __forceinline__ void interpolate_chunk_q(const Selection& sel, int k,
       y[s] = pattern >= kPrime32 ? pattern - kPrime32 : pattern;  // "dd <- y mod M"
     }
   }
-  interpolate_warp_q<SLOTS>(k, x, y, rows, rows + kMaxK, proof);
+  interpolate_warp_q<SLOTS>(k, x, y, row_x, rows, rows + kMaxK, proof);
 }
 
 __global__ void __launch_bounds__(kInterpQWarps * 32)
 toploc_interpolate_q_kernel(Selection sel, int k, long long num_chunks) {
   __shared__ uint32_t rows[kInterpQWarps][2 * kMaxK];
+  __shared__ uint16_t rows_x[kInterpQWarps][kMaxK];
   const int warp = threadIdx.x >> 5;
   const long long chunk = (long long)blockIdx.x * kInterpQWarps + warp;
   if (chunk >= num_chunks) return;
   const uint8_t st = sel.status[chunk];
   if (st == TOPLOC_CHUNK_NO_INJECTIVE_MODULUS || st == TOPLOC_CHUNK_K_EXCEEDS_CHUNK) return;
-  if (k <= 32) interpolate_chunk_q<1>(sel, k, chunk, rows[warp]);
-  else if (k <= 64) interpolate_chunk_q<2>(sel, k, chunk, rows[warp]);
-  else if (k <= 128) interpolate_chunk_q<4>(sel, k, chunk, rows[warp]);
-  else if (k <= 256) interpolate_chunk_q<8>(sel, k, chunk, rows[warp]);
-  else interpolate_chunk_q<kMaxK / 32>(sel, k, chunk, rows[warp]);
+  if (k <= 32) interpolate_chunk_q<1>(sel, k, chunk, rows[warp], rows_x[warp]);
+  else if (k <= 64) interpolate_chunk_q<2>(sel, k, chunk, rows[warp], rows_x[warp]);
+  else if (k <= 128) interpolate_chunk_q<4>(sel, k, chunk, rows[warp], rows_x[warp]);
+  else if (k <= 256) interpolate_chunk_q<8>(sel, k, chunk, rows[warp], rows_x[warp]);
+  else interpolate_chunk_q<kMaxK / 32>(sel, k, chunk, rows[warp], rows_x[warp]);
 }
 
 // Algorithm 2 after the selection, over Z_q, for one chunk whose selected
