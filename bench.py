@@ -212,7 +212,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-recipes", action="store_true",
-                    help="skip the extra timings of the 70B-shaped batch with jittered and without outlier channels")
+                    help="skip the extra timings of the 70B-shaped batch with the other input recipes (jittered "
+                         "outliers, no outlier channels, magnitudes rising through every chunk)")
     ap.add_argument("--decode-steps", action="store_true",
                     help="time incremental proof generation (one row per sequence and step) instead of the main workload")
     ap.add_argument("--direct", action="store_true",
@@ -389,11 +390,12 @@ def main():
     if args.workload == "70b" and world == 1 and not args.no_recipes:
         # The literal +-80 recipe is the streaming filter's best case (every chunk's top-128 is its
         # first 128 outliers, known after the first rows).  The same batch shape with jittered
-        # outlier magnitudes and with no outlier channels, regenerated in place and timed the same way.
+        # outlier magnitudes, with no outlier channels, and with magnitudes that grow fourfold over every
+        # chunk (the running threshold rises to the end), regenerated in place and timed the same way.
         line["other_recipes"] = {
             name: time_recipe(tl, synth, name, act, recomputed, lay, proofs, status, results, thr, workspace,
                               S, T, H, seed, min(args.steps, 20), n)
-            for name in ("jitter", "none")}
+            for name in ("jitter", "none", "rising")}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

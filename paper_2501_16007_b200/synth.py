@@ -46,7 +46,10 @@ def make_activations(num_seqs, tokens_per_seq, hidden, dtype=torch.bfloat16, see
 
     outliers: "fixed"  -> +-80 on the outlier channels (the literal recipe),
               "jitter" -> 80 * (1 + 0.25 u), u ~ U(-1, 1), so the top-k varies per chunk,
-              "none"   -> no outlier channels (pure heavy-tailed data).
+              "none"   -> no outlier channels (pure heavy-tailed data),
+              "rising" -> jittered outliers, and token t of a sequence scaled by 4 ** ((t mod 32) / 31):
+                          magnitudes grow fourfold over every 32-token interval, so a running top-k
+                          keeps admitting new elements to the end of a chunk.
     Each sequence draws from its own generator seeded with seed * 1000003 + sequence, so a
     sequence's bytes do not depend on the batch around it (on a given device type).
     """
@@ -65,10 +68,13 @@ def make_activations(num_seqs, tokens_per_seq, hidden, dtype=torch.bfloat16, see
             shape = (tokens_per_seq, len(outlier_channels))
             sign = torch.randint(0, 2, shape, generator=g, device=device).to(torch.float32) * 2.0 - 1.0
             mag = torch.full(shape, 80.0, device=device, dtype=torch.float32)
-            if outliers == "jitter":
+            if outliers in ("jitter", "rising"):
                 u = torch.rand(shape, generator=g, device=device, dtype=torch.float32) * 2.0 - 1.0
                 mag = mag * (1.0 + 0.25 * u)
             x[:, ch] = sign * mag
+        if outliers == "rising":
+            t = torch.arange(tokens_per_seq, device=device, dtype=torch.float32)
+            x *= torch.pow(torch.tensor(4.0, device=device), (t % 32) / 31.0).unsqueeze(1)
         out[s * tokens_per_seq:(s + 1) * tokens_per_seq].copy_(x.to(dtype))
         del x
     return out

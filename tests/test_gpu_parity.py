@@ -334,13 +334,13 @@ def test_config_70b_full_size_every_chunk():
     full_size_70b_case("fixed", 4, range(256))
 
 
-@pytest.mark.parametrize("recipe", ["jitter", "none"])
+@pytest.mark.parametrize("recipe", ["jitter", "none", "rising"])
 def test_config_70b_full_size_varied_selections(recipe):
     """With +-80 outliers every chunk selects the same index set (the first 128 outliers); jittered
-    outlier magnitudes and plain heavy-tailed data make the selected set, the modulus and the
-    statistics differ from chunk to chunk.  Same full-size launches; sixteen whole sequences
+    outlier magnitudes, plain heavy-tailed data and magnitudes that grow through every chunk make
+    the selected set, the modulus and the statistics differ from chunk to chunk.  Same full-size launches; sixteen whole sequences
     (2048 chunks) against the oracle."""
-    g, honest = full_size_70b_case(recipe, 40 if recipe == "jitter" else 41, range(7, 256, 16))
+    g, honest = full_size_70b_case(recipe, {"jitter": 40, "none": 41, "rising": 42}[recipe], range(7, 256, 16))
     distinct = {tuple(row) for row in g[2][:4096:64].cpu().numpy().tolist()}
     assert len(distinct) > 32, "the selected index sets should vary from chunk to chunk"
 
