@@ -64,11 +64,18 @@ constexpr int kStages = TOPLOC_SELECT_STAGES;
 #ifndef TOPLOC_HIT_TRIGGER
 #define TOPLOC_HIT_TRIGGER 32
 #endif
-constexpr int kHitCap = TOPLOC_HIT_TRIGGER + 128;  // select: vectors that can be parked between drains
-constexpr int kHitTrigger = TOPLOC_HIT_TRIGGER;    // select: drain once this many are parked
+#ifndef TOPLOC_HIT_TRIGGER_DIV
+#define TOPLOC_HIT_TRIGGER_DIV 4
+#endif
+#ifndef TOPLOC_HIT_CAP
+#define TOPLOC_HIT_CAP 184
+#endif
+#ifndef TOPLOC_HIT_CAP_BIG
+#define TOPLOC_HIT_CAP_BIG 256
+#endif
+constexpr int kHitTrigger = TOPLOC_HIT_TRIGGER;    // select: drain once this many are parked (more for large k)
 constexpr int kIdxBits = 24;             // flat index field of a candidate
 constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
-static_assert(kHitCap >= kHitTrigger - 1 + kThreads * kUnroll, "a tile's hits must fit below the drain trigger");
 
 // A candidate is one 64-bit word whose unsigned order is the ranking order:
 // magnitude key (bit pattern without sign) descending, then flat index
@@ -80,10 +87,14 @@ __device__ __forceinline__ unsigned long long make_candidate(uint32_t key, uint3
 // Shared memory of one selecting warp.  CAP: candidate buffer entries (8 bytes each); KMAX: the
 // largest k it serves.  Two sizes are in use: SelectShared (k <= 256, 13.4 KB: sixteen warps per
 // SM) and SelectSharedBig (k <= TOPLOC_MAX_K = 512, 16.5 KB: thirteen).
-template <int CAP, int KMAX>
+template <int CAP, int KMAX, int HITCAP>
 struct __align__(16) SelectSharedT {
   static constexpr int kCap = CAP;
   static constexpr int kMaxK = KMAX;
+  static constexpr int kHitCap = HITCAP;  // vectors that can be parked between drains
+  static constexpr int kLooseKeep = CAP - 8 * kThreads;  // a mid-stream compaction may leave this many:
+                                                         // a round appends at most 8 per lane
+  static_assert(HITCAP >= kHitTrigger - 1 + kThreads * kUnroll, "a tile's hits must fit below the drain trigger");
   static constexpr int kMaxSlots = KMAX / 32;  // tail: entries a lane owns at most
   static_assert(CAP * 8 >= 8 * KMAX * 2, "the candidate buffer holds the maxima of the first vectors");
   static_assert(CAP >= KMAX + kThreads * 8, "a round of appends must fit after a compaction");
@@ -92,7 +103,7 @@ struct __align__(16) SelectSharedT {
   static_assert(sizeof(uint4) * kStages * kUnroll * kThreads >= 12 * KMAX, "the ring holds three rows of KMAX words");
   uint4 ring[kStages * kUnroll * kThreads];  // tiles on their way from HBM (asynchronous copies)
   unsigned long long cand[CAP];       // candidates held; ring + cand later serve as the residue set
-  uint32_t hit_idx[kHitCap];          // vectors that passed the streaming filter, not yet unpacked
+  uint32_t hit_idx[HITCAP];           // vectors that passed the streaming filter, not yet unpacked
                                       // (index within the chunk; they are fetched again when unpacked)
   uint32_t top_hist[256];             // held candidates by the upper 8 bits of their 15-bit key; a
                                       // compaction borrows it for its digit histograms
@@ -102,8 +113,8 @@ struct __align__(16) SelectSharedT {
   uint32_t bin;
   int want;
 };
-using SelectShared = SelectSharedT<TOPLOC_CAND_CAP, 256>;
-using SelectSharedBig = SelectSharedT<1024, TOPLOC_MAX_K>;
+using SelectShared = SelectSharedT<TOPLOC_CAND_CAP, 256, TOPLOC_HIT_CAP>;
+using SelectSharedBig = SelectSharedT<1024, TOPLOC_MAX_K, TOPLOC_HIT_CAP_BIG>;
 static_assert(TOPLOC_MAX_K == 512, "SelectSharedBig is sized for k up to 512");
 constexpr uint32_t kNoBin = 0xFFFFFFFFu;
 
@@ -299,8 +310,9 @@ __device__ __noinline__ uint32_t raise_threshold(SH& sh, int k, uint32_t thr, in
 // the k-th".  Ties on the key are only broken by index when it matters: once
 // the key digits are settled the scan stops if the boundary bin can be kept
 // whole -- because exactly k candidates remain, or, for a compaction in
-// mid-stream (exact == false), because at most kMaxK remain; only the last
-// compaction of a chunk must leave exactly k.  Returns the new state.
+// mid-stream (exact == false), because a round of appends still fits behind
+// what remains; only the last compaction of a chunk must leave exactly k.
+// Returns the new state.
 template <int DT, class SH>
 __device__ __noinline__ WarpState compact_candidates(SH& sh, int k, WarpState st, bool exact) {
   const int lane = threadIdx.x & 31;
@@ -324,7 +336,7 @@ __device__ __noinline__ WarpState compact_candidates(SH& sh, int k, WarpState st
     want = sh.want;
     const int kept = k - want + (int)sh.bin;
     // lower bits of the pivot stay 0: the boundary bin is kept whole
-    if (shift <= 24 && (kept == k || (!exact && kept <= SH::kMaxK))) break;
+    if (shift <= 24 && (kept == k || (!exact && kept <= SH::kLooseKeep))) break;
   }
   const unsigned long long pivot = prefix;  // everything >= pivot is kept
   // in place, in order: a slot is overwritten only after it has been read
@@ -340,10 +352,10 @@ __device__ __noinline__ WarpState compact_candidates(SH& sh, int k, WarpState st
     if (keep) sh.cand[pos] = c;
     out += __popc(votes);
   }
-  // Distinct candidates leave at most kMaxK here (exactly k when exact).  Equal candidates -- a
+  // Distinct candidates leave at most kLooseKeep here (exactly k when exact).  Equal candidates -- a
   // caller of the incremental entry points offering a flat index twice -- could leave more at the
   // cut; the buffer's arithmetic relies on the bound, so it is enforced.
-  out = min(out, exact ? k : SH::kMaxK);
+  out = min(out, exact ? k : SH::kLooseKeep);
   // the key histograms describe the survivors only
   for (int b = lane; b < 256; b += kThreads) sh.top_hist[b] = 0;
   if (lane == 0) sh.top_bin = kNoBin;
@@ -352,6 +364,47 @@ __device__ __noinline__ WarpState compact_candidates(SH& sh, int k, WarpState st
   warp_barrier();
   st.count = out;
   st.thr = max(st.thr, (uint32_t)(pivot >> (kIdxBits + 1)) + 1u);
+  return st;
+}
+
+// The cheap way to make room in mid-stream: the key histograms already know the k-th largest
+// 15-bit key among the held candidates, so everything below it is dropped in one pass and the
+// histograms are trimmed to match.  What remains is k plus the rest of the boundary key's bin --
+// a handful on ordinary data; the caller falls back on compact_candidates when that is still too
+// many (long runs of equal magnitudes).
+template <int DT, class SH>
+__device__ __noinline__ WarpState shed_below_kth(SH& sh, int k, WarpState st) {
+  const int lane = threadIdx.x & 31;
+  const int n = st.count;
+  if (n <= k) return st;
+  st.thr = raise_threshold<DT>(sh, k, st.thr, n);  // leaves top_bin and digit describing the k-th key
+  const uint32_t top = sh.top_bin, low = sh.digit;
+  const uint32_t kth = (top << 7) | low;
+  int out = 0;
+  warp_barrier();
+  for (int base = 0; base < n; base += kThreads) {
+    const int e = base + lane;
+    const unsigned long long c = e < n ? sh.cand[e] : 0ull;
+    const bool keep = e < n && coarse_key<DT>(c) >= kth;
+    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, keep);
+    const int pos = out + __popc(votes & ((1u << lane) - 1u));
+    warp_barrier();
+    if (keep) sh.cand[pos] = c;
+    out += __popc(votes);
+  }
+  uint32_t in_top = 0;
+  for (int b = lane; b < 128; b += kThreads) {
+    if ((uint32_t)b < low) sh.low_hist[b] = 0;
+    else in_top += sh.low_hist[b];
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) in_top += __shfl_xor_sync(0xFFFFFFFFu, in_top, off);
+  for (int b = lane; b < 256; b += kThreads) {
+    if ((uint32_t)b < top) sh.top_hist[b] = 0;
+    else if ((uint32_t)b == top) sh.top_hist[b] = in_top;
+  }
+  warp_barrier();
+  st.count = out;
   return st;
 }
 
@@ -418,8 +471,9 @@ __device__ __forceinline__ void append_round(SH& sh, int k, WarpState& st, const
     }
     total = __shfl_sync(0xFFFFFFFFu, incl, 31);
     if (st.count + total <= SH::kCap) break;
-    // leaves at most SH::kMaxK and may raise the threshold; a round adds at most 32 * VEC
-    st = compact_candidates<DT>(sh, k, st, false);
+    // Both leave at most SH::kLooseKeep (a round adds at most 32 * VEC) and may raise the threshold.
+    st = shed_below_kth<DT>(sh, k, st);
+    if (st.count > SH::kLooseKeep) st = compact_candidates<DT>(sh, k, st, false);
   }
   int pos = st.count + incl - __popc(mask);
   const uint32_t top_bin = sh.top_bin;
@@ -483,6 +537,14 @@ __device__ __noinline__ WarpState drain_hits(SH& sh, const ChunkSource<DT, MODE>
   st.nhits = 0;
   st.thr = raise_threshold<DT>(sh, k, st.thr, st.count);
   return st;
+}
+
+// Parked vectors are unpacked once this many of them wait.  A larger k admits more of them and
+// every drain ends with a look at the key histograms, so the trigger grows with k as far as the
+// parking space allows (one tile can park kThreads * kUnroll more).
+template <class SH>
+__device__ __forceinline__ int drain_trigger(int k) {
+  return min(max(kHitTrigger, k / TOPLOC_HIT_TRIGGER_DIV), SH::kHitCap - kThreads * kUnroll + 1);
 }
 
 // Largest key in one vector, as the 15-bit key the threshold is kept in.
@@ -575,6 +637,7 @@ __device__ void select_topk(SH& sh, const ChunkSource<DT, MODE>& src, int n_elem
   // aligned chunks get it from a look at the maxima of their first vectors
   // (which are then streamed like everything else); otherwise the first vectors
   // are selected from directly.
+  const int trigger = drain_trigger<SH>(k);
   const int first = (32 / VEC) * max(k, 128);
   const bool look_ahead = (MODE != 2) && n_vecs >= first;
   const int warm = look_ahead ? 0 : min(n_vecs, first);
@@ -663,7 +726,7 @@ __device__ void select_topk(SH& sh, const ChunkSource<DT, MODE>& src, int n_elem
       }
       if (!kRing) request_tile(tile + kStages, stage);  // (keeps the commit-group count in step; no copies)
       // a tile parks at most kTileVecs vectors, so the buffer cannot overflow
-      if (st.nhits >= kHitTrigger) st = drain_hits<DT, MODE>(sh, src, k, st);
+      if (st.nhits >= trigger) st = drain_hits<DT, MODE>(sh, src, k, st);
     }
   }
   if (kRing) copy_async_wait<0>();
@@ -690,6 +753,7 @@ __device__ __forceinline__ WarpState filter_vectors(SH& sh, const ChunkSource<DT
   constexpr int VEC = ChunkSource<DT, MODE>::kVec;
   const int lane = threadIdx.x & 31;
   const uint32_t below = (1u << lane) - 1u;
+  const int trigger = drain_trigger<SH>(k);
   for (int v0 = vb; v0 < ve; v0 += kThreads * kUnroll) {
     uint4 w[kUnroll];
     bool hit[kUnroll];
@@ -713,7 +777,7 @@ __device__ __forceinline__ WarpState filter_vectors(SH& sh, const ChunkSource<DT
         if (hit[u]) sh.hit_idx[st.nhits + __popc(votes[u] & below)] = (uint32_t)(v0 + u * kThreads + lane);
         st.nhits += __popc(votes[u]);
       }
-      if (st.nhits >= kHitTrigger) st = drain_hits<DT, MODE>(sh, src, k, st);
+      if (st.nhits >= trigger) st = drain_hits<DT, MODE>(sh, src, k, st);
     }
   }
   return drain_hits<DT, MODE>(sh, src, k, st);
