@@ -645,8 +645,38 @@ __device__ __forceinline__ void find_from_top(LooseControl& sh, const uint32_t* 
   __syncthreads();
 }
 
+// The commitment of one chunk from its k (index, committed value) pairs in index order, held in
+// shared memory: 6 bytes per pair (index low half, index high half, value).  Whole 16-byte words
+// where the record's place and k allow it, coalesced 2-byte words otherwise.
+template <int T>
+__device__ __forceinline__ void write_commitment(uint16_t* rec, const uint32_t* flat, const uint16_t* pat, int k) {
+  if ((k & 7) == 0 && (reinterpret_cast<uintptr_t>(rec) & 15u) == 0) {
+    uint4* out = reinterpret_cast<uint4*>(rec);
+    for (int g = threadIdx.x; g < k / 8; g += T) {
+      uint32_t h[12];  // 24 half words: 8 records
+#pragma unroll
+      for (int r = 0; r < 8; r += 2) {
+        const uint32_t f0 = flat[8 * g + r], f1 = flat[8 * g + r + 1];
+        const uint32_t p0 = pat[8 * g + r], p1 = pat[8 * g + r + 1];
+        h[3 * (r / 2)] = f0;                                   // low, high of the first index
+        h[3 * (r / 2) + 1] = p0 | (f1 << 16);                  // its value, low half of the second
+        h[3 * (r / 2) + 2] = (f1 >> 16) | (p1 << 16);          // high half of the second, its value
+      }
+      out[3 * g] = make_uint4(h[0], h[1], h[2], h[3]);
+      out[3 * g + 1] = make_uint4(h[4], h[5], h[6], h[7]);
+      out[3 * g + 2] = make_uint4(h[8], h[9], h[10], h[11]);
+    }
+  } else {
+    for (int w = threadIdx.x; w < 3 * k; w += T) {
+      const int r = w / 3, part = w - 3 * r;
+      rec[w] = part == 2 ? pat[r] : (uint16_t)(part == 0 ? flat[r] & 0xFFFFu : flat[r] >> 16);
+    }
+  }
+}
+
 template <int DT, bool ORDERED, int T, class Emit>
-__device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit) {
+__device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit,
+                                 uint16_t* rec = nullptr) {
   using R = Reader<DT, true>;
   using Pat = typename StoredPattern<DT>::type;
   constexpr int VEC = R::VEC;
@@ -752,16 +782,23 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   const uint32_t raise_step = (uint32_t)(k / 2 > 256 ? k / 2 : 256);
   uint32_t thr = *shared_thr;
   int nparked = 0;
-  auto drain = [&]() {
+  // Unpacks the parked vectors a full round (32 of them) at a time; what is left over waits for
+  // the next drain unless this is the last one.
+  auto drain = [&](bool all) {
     __syncwarp();
     uint32_t handed_out = 0;
-    for (int b = 0; b < nparked; b += 32) {
+    const int upto = all ? nparked : (nparked & ~31);
+    for (int b = 0; b < upto; b += 32) {
       const bool valid = b + lane < nparked;
       const uint32_t g = valid ? park[b + lane] : 0u;
       const uint32_t after = admit(valid, g, thr);
       handed_out = after > handed_out ? after : handed_out;
     }
-    nparked = 0;
+    const int left = all ? 0 : nparked - upto;  // < 32
+    const uint32_t moved = lane < left ? park[upto + lane] : 0u;
+    __syncwarp();
+    if (lane < left) park[lane] = moved;
+    nparked = left;
     __syncwarp();
     // raise the threshold if enough candidates have arrived since the last time and nobody else is at it
     uint32_t go = 0;
@@ -829,13 +866,13 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
         if (hit[u]) park[nparked + __popc(votes[u] & ((1u << lane) - 1u))] = (uint32_t)(begin + u * T) + threadIdx.x;
         nparked += __popc(votes[u]);
       }
-      if (nparked >= kParkTrigger) drain();
+      if (nparked >= kParkTrigger) drain(false);
     }
     thr = *shared_thr;
     if (*shared_overflow) break;
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");  // a batch requested before leaving the loop
-  if (!*shared_overflow) drain();
+  if (!*shared_overflow) drain(true);
   __syncthreads();
   if (sh.overflow) return false;
   const uint32_t count = sh.cand_count;
@@ -921,32 +958,67 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   }
   // Index order: one bit per element of the chunk for the selected ones; an element's position is
   // the number of set bits before its own.
+  // The number of set bits before every group of kGroup words is kept (16 bits each, in the
+  // histogram's place), so a position costs at most kGroup word counts.
   uint32_t* bitmap = reinterpret_cast<uint32_t*>(ring);  // (the caller made sure one bit per element fits)
+  uint16_t* before_group = reinterpret_cast<uint16_t*>(coarse);
   const uint32_t n_words = ((uint32_t)rd.n_groups * VEC + 31u) / 32u;
-  const uint32_t per_thread = (n_words + T - 1) / T;  // consecutive words a thread counts
-  for (uint32_t wd = threadIdx.x; wd < n_words; wd += T) bitmap[wd] = 0u;
+  constexpr uint32_t kGroups = 2u * kCoarseBins;       // 16-bit entries the histogram's place holds
+  uint32_t group_shift = 0;                             // words per group: the smallest power of two that fits
+  while (((n_words + (1u << group_shift) - 1u) >> group_shift) > kGroups) ++group_shift;
+  const uint32_t n_groups = (n_words + (1u << group_shift) - 1u) >> group_shift;
+  const uint32_t per_thread = (n_groups + T - 1) / T;   // consecutive groups a thread counts
+  {
+    uint4* q = reinterpret_cast<uint4*>(bitmap);         // (the ring is a whole number of 16-byte words)
+    for (uint32_t wd = threadIdx.x; wd < (n_words + 3u) / 4u; wd += T) q[wd] = make_uint4(0u, 0u, 0u, 0u);
+  }
   __syncthreads();
   for (uint32_t i = threadIdx.x; i < count; i += T)
     if (selected(i)) atomicOr(&bitmap[cand_flat[i] >> 5], 1u << (cand_flat[i] & 31u));
   __syncthreads();
   {
-    const uint32_t lo = threadIdx.x * per_thread < n_words ? threadIdx.x * per_thread : n_words;
-    const uint32_t hi = lo + per_thread < n_words ? lo + per_thread : n_words;
+    const uint32_t lo = threadIdx.x * per_thread < n_groups ? threadIdx.x * per_thread : n_groups;
+    const uint32_t hi = lo + per_thread < n_groups ? lo + per_thread : n_groups;
     uint32_t ones = 0;
-    for (uint32_t wd = lo; wd < hi; ++wd) ones += (uint32_t)__popc(bitmap[wd]);
+    for (uint32_t g = lo; g < hi; ++g) {
+      const uint32_t w0 = g << group_shift, w1 = w0 + (1u << group_shift) < n_words ? w0 + (1u << group_shift) : n_words;
+      for (uint32_t wd = w0; wd < w1; ++wd) ones += (uint32_t)__popc(bitmap[wd]);
+    }
     unsigned long long total;
-    coarse[threadIdx.x] = (uint32_t)scan_exclusive<T>(sh, ones, 0, &total);  // set bits before this thread's words
+    uint32_t running = (uint32_t)scan_exclusive<T>(sh, ones, 0, &total);  // set bits before this thread's groups
+    // (scan_exclusive's barrier lies between the histogram's last use and these stores)
+    for (uint32_t g = lo; g < hi; ++g) {
+      before_group[g] = (uint16_t)running;
+      const uint32_t w0 = g << group_shift, w1 = w0 + (1u << group_shift) < n_words ? w0 + (1u << group_shift) : n_words;
+      for (uint32_t wd = w0; wd < w1; ++wd) running += (uint32_t)__popc(bitmap[wd]);
+    }
   }
   __syncthreads();
+  // With room behind the candidates the pairs are first put in order in shared memory and the
+  // commitment is written in whole words; otherwise every pair goes out on its own.
+  const bool staged = rec != nullptr && count + (uint32_t)k <= (uint32_t)kCap;
+  uint32_t* sorted_flat = cand_flat + count;
+  uint16_t* sorted_pat = reinterpret_cast<uint16_t*>(cand_pat + count);
   for (uint32_t i = threadIdx.x; i < count; i += T) {
     if (!selected(i)) continue;
-    const uint32_t flat = cand_flat[i], wd = flat >> 5, owner = wd / per_thread;
-    uint32_t pos = coarse[owner];
-    for (uint32_t v = owner * per_thread; v < wd; ++v) pos += (uint32_t)__popc(bitmap[v]);
+    const uint32_t flat = cand_flat[i], wd = flat >> 5;
+    uint32_t pos = before_group[wd >> group_shift];
+    for (uint32_t v = (wd >> group_shift) << group_shift; v < wd; ++v) pos += (uint32_t)__popc(bitmap[v]);
     pos += (uint32_t)__popc(bitmap[wd] & ((1u << (flat & 31u)) - 1u));
-    emit(pos, flat, R::committed(cand_pat[i]));
+    if (staged) {
+      if (pos < (uint32_t)k) {
+        sorted_flat[pos] = flat;
+        sorted_pat[pos] = (uint16_t)R::committed(cand_pat[i]);
+      }
+    } else {
+      emit(pos, flat, R::committed(cand_pat[i]));
+    }
   }
   __syncthreads();
+  if (staged) {
+    write_commitment<T>(rec, sorted_flat, sorted_pat, k);
+    __syncthreads();
+  }
   return true;
 }
 
@@ -1010,7 +1082,7 @@ __device__ void commit_one_chunk(DirectShared& sh, uint4* ring, const DirectPara
   if constexpr (VECTOR) {
     if (!loose_failed) {
       if ((long long)rd.n_groups * R::VEC <= kLooseMaxElems)
-        done = select_unordered<DT, true, kThreads>(loose_workspace<DT>(sh), ring, rd, p.k, emit);
+        done = select_unordered<DT, true, kThreads>(loose_workspace<DT>(sh), ring, rd, p.k, emit, rec);
       else if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
     }
   }
@@ -1275,7 +1347,7 @@ __global__ void __launch_bounds__(kT, 2) toploc_direct_commit_half_kernel(Direct
     rec[3 * pos + 1] = (uint16_t)(flat >> 16);
     rec[3 * pos + 2] = (uint16_t)pat;
   };
-  const bool done = select_unordered<DT, true, kT>(ws, cv.ring, rd, p.k, emit);
+  const bool done = select_unordered<DT, true, kT>(ws, cv.ring, rd, p.k, emit, rec);
   if (threadIdx.x == 0) status[chunk] = done ? TOPLOC_CHUNK_OK : kRetry;
 }
 
