@@ -582,7 +582,20 @@ struct LooseWorkspace {
   typename StoredPattern<DT>::type* cand_pat;  // ... and whole pattern
   uint32_t* park;        // kParkCap words per warp
   int cap;
+  uint8_t* seen_max;     // MAP only: one byte per 8 elements (their largest key, coarsely), written by the first pass
+  uint32_t* bitmap;      // ORDERED only: one bit per element for the ranking in index order
 };
+
+// The byte the first pass leaves for every 8 consecutive elements: the upper 11 bits of their
+// largest key (exponent and three mantissa bits) counted from 2^-20, 0 for anything smaller, 255
+// for 2^11.75 and above -- 32 binades around the magnitudes activations have.  A group whose byte
+// reaches the threshold's byte may hold an element that reaches the threshold; a group below it
+// cannot (magnitudes beyond either end of the window only make the second pass look at groups
+// it need not have looked at).
+constexpr uint32_t kSeenBase = (127u - 20u) << 3;
+__device__ __forceinline__ uint32_t seen_byte(uint32_t bin11) {
+  return bin11 < kSeenBase ? 0u : (bin11 - kSeenBase + 1u < 255u ? bin11 - kSeenBase + 1u : 255u);
+}
 
 template <int T>
 __device__ __forceinline__ void clear_words(uint32_t* words, int n) {  // n: a multiple of 4; ends with a barrier
@@ -674,7 +687,7 @@ __device__ __forceinline__ void write_commitment(uint16_t* rec, const uint32_t* 
   }
 }
 
-template <int DT, bool ORDERED, int T, class Emit>
+template <int DT, bool ORDERED, int T, bool MAP, class Emit>
 __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit,
                                  uint16_t* rec = nullptr) {
   using R = Reader<DT, true>;
@@ -745,7 +758,11 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   // cannot lie below it, and by little more than k (k vectors reach it, few of them twice).  The
   // second pass finds the chunk in L2 (one chunk per SM in flight).  A chunk of fewer than k
   // vectors starts from 0 and is streamed once.
-  {
+  // MAP: the first pass also leaves seen_max, and the second pass is a scan of those bytes that
+  // fetches only the groups which can hold a candidate (about k of them, from L2) -- the chunk is
+  // streamed once, and the candidates may use the ring's place.
+  constexpr int kPerByte = 8 / VEC;  // vectors per byte of seen_max
+  if (!MAP || rd.n_groups >= k) {
     const int first_end = kBatch < rd.n_groups ? kBatch : rd.n_groups;
     rd.template request<T>(ring, (int)threadIdx.x, first_end);  // in flight meanwhile
   }
@@ -760,14 +777,24 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
       }
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        if (begin + u * T + (int)threadIdx.x < end) {
+        const int g = begin + u * T + (int)threadIdx.x;
+        uint32_t bin = 0;
+        if (g < end) {
           const uint32_t m = toploc_device::vector_max_coarse_key<DT, VEC>(make_uint4(w[u][0], w[u][1], w[u][2], w[u][3]));
-          atomicAdd(&coarse[m >> 4], 1u);  // upper 11 of the 15 bits
+          bin = m >> 4;  // upper 11 of the 15 bits
+          atomicAdd(&coarse[bin], 1u);
+        }
+        if (MAP) {
+          if (kPerByte == 2) {  // neighbouring lanes hold the two vectors of a byte (begin and T are even)
+            const uint32_t other = __shfl_xor_sync(kFull, bin, 1);
+            bin = bin > other ? bin : other;
+          }
+          if (g < end && (kPerByte == 1 || (g & 1) == 0)) ws.seen_max[g / kPerByte] = (uint8_t)seen_byte(bin);
         }
       }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    {
+    if (!MAP) {
       const int first_end = kBatch < rd.n_groups ? kBatch : rd.n_groups;
       rd.template request<T>(ring, (int)threadIdx.x, first_end);  // the second pass's first batch
     }
@@ -791,8 +818,17 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
     for (int b = 0; b < upto; b += 32) {
       const bool valid = b + lane < nparked;
       const uint32_t g = valid ? park[b + lane] : 0u;
-      const uint32_t after = admit(valid, g, thr);
-      handed_out = after > handed_out ? after : handed_out;
+      if (MAP) {  // a parked entry stands for 8 elements: one or two vectors
+#pragma unroll
+        for (int h = 0; h < kPerByte; ++h) {
+          const uint32_t v = g * kPerByte + h;
+          const uint32_t after = admit(valid && v < (uint32_t)rd.n_groups, v, thr);
+          handed_out = after > handed_out ? after : handed_out;
+        }
+      } else {
+        const uint32_t after = admit(valid, g, thr);
+        handed_out = after > handed_out ? after : handed_out;
+      }
     }
     const int left = all ? 0 : nparked - upto;  // < 32
     const uint32_t moved = lane < left ? park[upto + lane] : 0u;
@@ -802,7 +838,7 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
     __syncwarp();
     // raise the threshold if enough candidates have arrived since the last time and nobody else is at it
     uint32_t go = 0;
-    if (lane == 0 && handed_out >= (uint32_t)k && handed_out <= (uint32_t)kCap &&
+    if (!MAP && lane == 0 && handed_out >= (uint32_t)k && handed_out <= (uint32_t)kCap &&
         handed_out - *shared_last_raise >= raise_step)
       go = atomicCAS(&sh.raise_lock, 0u, 1u) == 0u ? 1u : 0u;
     go = __shfl_sync(kFull, go, 0);
@@ -839,7 +875,35 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
     }
   };
 
-  for (int begin = 0; begin < rd.n_groups; begin += kBatch) {
+  if (MAP) {
+    // The threshold is a bin's lowest key (or 0 for a chunk of fewer than k vectors, whose bytes
+    // were never written: every byte reaches 0).  Four bytes per lane and step.
+    const uint32_t bin = thr >> kCoarseShift;
+    const uint32_t want = seen_byte(bin) * 0x01010101u;
+    const int n_bytes = (rd.n_groups + kPerByte - 1) / kPerByte;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(ws.seen_max);
+    const uint32_t below = (1u << lane) - 1u;
+    for (int w0 = 0; w0 * 4 < n_bytes; w0 += T) {
+      const int wi = w0 + (int)threadIdx.x;
+      const uint32_t reach = wi * 4 < n_bytes ? __vcmpgeu4(words[wi], want) : 0u;  // 0xFF per byte that reaches
+      uint32_t votes[4], any_votes = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        votes[j] = __ballot_sync(kFull, ((reach >> (8 * j)) & 1u) != 0 && wi * 4 + j < n_bytes);
+        any_votes |= votes[j];
+      }
+      if (any_votes) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if ((votes[j] >> lane) & 1u) park[nparked + __popc(votes[j] & below)] = (uint32_t)(wi * 4 + j);
+          nparked += __popc(votes[j]);
+        }
+        if (nparked >= kParkTrigger) drain(false);
+      }
+      if (*shared_overflow) break;
+    }
+  }
+  for (int begin = 0; !MAP && begin < rd.n_groups; begin += kBatch) {
     const int end = begin + kBatch < rd.n_groups ? begin + kBatch : rd.n_groups;
     uint32_t w[kUnroll][4];
     rd.template take<T>(ring, begin + (int)threadIdx.x, end, w);
@@ -960,7 +1024,7 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   // the number of set bits before its own.
   // The number of set bits before every group of kGroup words is kept (16 bits each, in the
   // histogram's place), so a position costs at most kGroup word counts.
-  uint32_t* bitmap = reinterpret_cast<uint32_t*>(ring);  // (the caller made sure one bit per element fits)
+  uint32_t* bitmap = ws.bitmap;  // (the caller made sure one bit per element fits)
   uint16_t* before_group = reinterpret_cast<uint16_t*>(coarse);
   const uint32_t n_words = ((uint32_t)rd.n_groups * VEC + 31u) / 32u;
   constexpr uint32_t kGroups = 2u * kCoarseBins;       // 16-bit entries the histogram's place holds
@@ -1026,8 +1090,10 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
 // candidates where the key histogram of the other selections lives, the parked vectors at the
 // end of the spare bytes.
 template <int DT>
-__device__ __forceinline__ LooseWorkspace<DT> loose_workspace(DirectShared& sh) {
+__device__ __forceinline__ LooseWorkspace<DT> loose_workspace(DirectShared& sh, uint4* ring) {
   LooseWorkspace<DT> ws;
+  ws.seen_max = nullptr;
+  ws.bitmap = reinterpret_cast<uint32_t*>(ring);
   ws.ctl = &sh.loose;
   ws.coarse = sh.hist;
   ws.cand_flat = sh.hist + kCoarseBins;
@@ -1082,7 +1148,7 @@ __device__ void commit_one_chunk(DirectShared& sh, uint4* ring, const DirectPara
   if constexpr (VECTOR) {
     if (!loose_failed) {
       if ((long long)rd.n_groups * R::VEC <= kLooseMaxElems)
-        done = select_unordered<DT, true, kThreads>(loose_workspace<DT>(sh), ring, rd, p.k, emit, rec);
+        done = select_unordered<DT, true, kThreads, false>(loose_workspace<DT>(sh, ring), ring, rd, p.k, emit, rec);
       else if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
     }
   }
@@ -1257,7 +1323,7 @@ __device__ void verify_one_chunk(DirectShared& sh, uint4* ring, const DirectPara
     if (!loose_failed && (loose || k <= kStreamMaxK)) {
       sel_idx = reinterpret_cast<uint32_t*>(ring);
       sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
-      done = loose ? select_unordered<DT, false, kThreads>(loose_workspace<DT>(sh), ring, rd, k, emit)
+      done = loose ? select_unordered<DT, false, kThreads, false>(loose_workspace<DT>(sh, ring), ring, rd, k, emit)
                    : select_in_one_pass<DT>(sh, ring, rd, k, emit);
     }
   }
@@ -1293,26 +1359,39 @@ toploc_direct_verify_kernel(DirectParams p, DirectVerify io) {
 namespace half_block {
 constexpr int kT = 512;
 constexpr int kW = kT / 32;
-constexpr size_t kRing = (size_t)kUnroll * kT * 16;         // 32 KB; later one bit per element of the chunk
-constexpr long long kMaxElems = (long long)kRing * 8;       // 2^18
+constexpr size_t kRing = (size_t)kUnroll * kT * 16;         // 32 KB; the candidates start here once the chunk has streamed
+constexpr size_t kSeen = 32 * 1024;                         // a byte per 8 elements; later a bit per element, or the selection
+constexpr long long kMaxElems = (long long)kSeen * 8;       // 2^18
 constexpr size_t kPark = (size_t)kW * kParkCap * 4;
-constexpr size_t kFixed = kRing + sizeof(LooseControl) + sizeof(CompareScratch) + (size_t)kCoarseBins * 4 + kPark;
+constexpr size_t kFixed = kSeen + sizeof(LooseControl) + sizeof(CompareScratch) + (size_t)kCoarseBins * 4 + kPark;
 constexpr size_t kBlockBytes = (227 * 1024) / 2 - 1024;      // two blocks per SM, 1 KB reserved for each
 __host__ __device__ constexpr int cap(int dt) { return (int)((kBlockBytes - kFixed) / (dt == 0 ? 6 : 8)) / 64 * 64; }
 static_assert(kFixed % 16 == 0 && cap(0) >= 2 * 4096 && cap(1) >= 4096 + 2048, "room for the candidates of k = 4096");
-static_assert(6 * TOPLOC_MAX_K_DIRECT <= kRing && 6 * TOPLOC_MAX_K_DIRECT <= 6 * 4096,
-              "the selection fits the ring, the decoded commitment the candidates' place");
+static_assert((size_t)cap(0) * 6 >= kRing && (size_t)cap(1) * 8 >= kRing, "the candidates' place contains the ring");
+static_assert(6 * TOPLOC_MAX_K_DIRECT <= kSeen && 6 * TOPLOC_MAX_K_DIRECT <= 6 * 4096,
+              "the selection fits the bytes' place, the decoded commitment the candidates' place");
 
 struct Carve {
   uint4* ring;
   CompareScratch* cs;
+  unsigned char* seen;  // kSeen bytes
 };
 
 template <int DT>
 __device__ __forceinline__ LooseWorkspace<DT> carve(unsigned char* smem, Carve* out) {
+  // from the end: control, comparison scratch, histogram, parked groups, the bytes of the first
+  // pass; everything before them is the candidates' (flat indices, then patterns), whose first
+  // 32 KB are the ring while the chunk streams
   LooseWorkspace<DT> ws;
   out->ring = reinterpret_cast<uint4*>(smem);
-  unsigned char* at = smem + kRing;
+  ws.cap = cap(DT);
+  ws.cand_flat = reinterpret_cast<uint32_t*>(smem);
+  ws.cand_pat = reinterpret_cast<typename StoredPattern<DT>::type*>(ws.cand_flat + ws.cap);
+  unsigned char* at = smem + kBlockBytes - kFixed;
+  out->seen = at;
+  ws.seen_max = at;
+  ws.bitmap = reinterpret_cast<uint32_t*>(at);
+  at += kSeen;
   ws.ctl = reinterpret_cast<LooseControl*>(at);
   at += sizeof(LooseControl);
   out->cs = reinterpret_cast<CompareScratch*>(at);
@@ -1320,10 +1399,6 @@ __device__ __forceinline__ LooseWorkspace<DT> carve(unsigned char* smem, Carve* 
   ws.coarse = reinterpret_cast<uint32_t*>(at);
   at += (size_t)kCoarseBins * 4;
   ws.park = reinterpret_cast<uint32_t*>(at);
-  at += kPark;
-  ws.cap = cap(DT);
-  ws.cand_flat = reinterpret_cast<uint32_t*>(at);
-  ws.cand_pat = reinterpret_cast<typename StoredPattern<DT>::type*>(ws.cand_flat + ws.cap);
   return ws;
 }
 
@@ -1347,7 +1422,7 @@ __global__ void __launch_bounds__(kT, 2) toploc_direct_commit_half_kernel(Direct
     rec[3 * pos + 1] = (uint16_t)(flat >> 16);
     rec[3 * pos + 2] = (uint16_t)pat;
   };
-  const bool done = select_unordered<DT, true, kT>(ws, cv.ring, rd, p.k, emit, rec);
+  const bool done = select_unordered<DT, true, kT, true>(ws, cv.ring, rd, p.k, emit, rec);
   if (threadIdx.x == 0) status[chunk] = done ? TOPLOC_CHUNK_OK : kRetry;
 }
 
@@ -1365,16 +1440,16 @@ __global__ void __launch_bounds__(kT, 2) toploc_direct_verify_half_kernel(Direct
     refuse_chunk(io, chunk, TOPLOC_CHUNK_K_EXCEEDS_CHUNK);
     return;
   }
-  // the selection goes to the ring (idle once the chunk has streamed), the decoded commitment where
-  // the candidates were (done with once the selection has been written out)
-  uint32_t* sel_idx = reinterpret_cast<uint32_t*>(cv.ring);
+  // the selection goes where the first pass's bytes were (done with once the candidates are in),
+  // the decoded commitment where the candidates were (done with once the selection has been written out)
+  uint32_t* sel_idx = reinterpret_cast<uint32_t*>(cv.seen);
   uint16_t* sel_pat = reinterpret_cast<uint16_t*>(sel_idx + k);
   auto emit = [&](uint32_t pos, uint32_t flat, uint32_t pat) {
     if (pos >= (uint32_t)k) return;
     sel_idx[pos] = flat;
     sel_pat[pos] = (uint16_t)pat;
   };
-  if (!select_unordered<DT, false, kT>(ws, cv.ring, rd, k, emit)) {
+  if (!select_unordered<DT, false, kT, true>(ws, cv.ring, rd, k, emit)) {
     if (threadIdx.x == 0) {
       toploc_chunk_result r = {};
       r.status = kRetry;
