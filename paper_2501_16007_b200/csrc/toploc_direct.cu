@@ -718,9 +718,16 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
 
   // One vector per lane: its elements that reach thr become candidates.  Returns the number of
   // candidates handed out so far (0 if the round added none).
-  auto admit = [&](bool valid, uint32_t g, uint32_t thr) -> uint32_t {
-    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-    if (valid) w = toploc_device::load_streaming(reinterpret_cast<const uint4*>(rd.address((int)g)));
+  // MAP: the threshold no longer moves once candidates arrive, so they are counted by their
+  // distance above it in steps of one 15-bit key (the last bin takes everything further up):
+  // the candidates spread over hundreds of bins instead of a few, and the k-th key's upper 15 bits
+  // come out of one walk.
+  constexpr int kFineShift = key_bits(DT) - 15;
+  auto fetch = [&](bool valid, uint32_t g) -> uint4 {
+    return valid ? toploc_device::load_streaming(reinterpret_cast<const uint4*>(rd.address((int)g)))
+                 : make_uint4(0u, 0u, 0u, 0u);
+  };
+  auto admit = [&](bool valid, uint32_t g, const uint4& w, uint32_t thr) -> uint32_t {
     uint32_t mask = valid ? toploc_device::passing_mask<DT, VEC>(w, thr) : 0u;
     const int mine = __popc(mask);
     int incl = mine;
@@ -746,7 +753,12 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
       toploc_device::pick_element<DT, VEC>(w, e, &key, &sign);
       cand_flat[at] = g * VEC + e;
       cand_pat[at] = (Pat)((sign << (DT == 0 ? 15 : 31)) | key);
-      atomicAdd(&coarse[key >> kCoarseShift], 1u);
+      if (MAP) {
+        const uint32_t above = (key - thr) >> kFineShift;
+        atomicAdd(&coarse[above < (uint32_t)kCoarseBins - 1u ? above : (uint32_t)kCoarseBins - 1u], 1u);
+      } else {
+        atomicAdd(&coarse[key >> kCoarseShift], 1u);
+      }
       ++at;
     }
     return base + (uint32_t)total;
@@ -815,20 +827,32 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
     __syncwarp();
     uint32_t handed_out = 0;
     const int upto = all ? nparked : (nparked & ~31);
-    for (int b = 0; b < upto; b += 32) {
-      const bool valid = b + lane < nparked;
-      const uint32_t g = valid ? park[b + lane] : 0u;
-      if (MAP) {  // a parked entry stands for 8 elements: one or two vectors
+    // a parked entry is a vector, or (MAP) 8 elements: one or two vectors; the next round's
+    // vectors are requested before this round's are unpacked
+    constexpr int kVecs = MAP ? kPerByte : 1;
+    uint4 cur[kVecs], nxt[kVecs];
+    uint32_t g_cur = 0, g_nxt = 0;
+    bool ok_cur[kVecs], ok_nxt[kVecs];
+    auto fetch_round = [&](int b, uint32_t* g, uint4 (&w)[kVecs], bool (&ok)[kVecs]) {
+      const bool valid = b < upto && b + lane < nparked;
+      *g = valid ? park[b + lane] : 0u;
 #pragma unroll
-        for (int h = 0; h < kPerByte; ++h) {
-          const uint32_t v = g * kPerByte + h;
-          const uint32_t after = admit(valid && v < (uint32_t)rd.n_groups, v, thr);
-          handed_out = after > handed_out ? after : handed_out;
-        }
-      } else {
-        const uint32_t after = admit(valid, g, thr);
-        handed_out = after > handed_out ? after : handed_out;
+      for (int h = 0; h < kVecs; ++h) {
+        ok[h] = valid && *g * kVecs + h < (uint32_t)rd.n_groups;
+        w[h] = fetch(ok[h], *g * kVecs + h);
       }
+    };
+    fetch_round(0, &g_cur, cur, ok_cur);
+    for (int b = 0; b < upto; b += 32) {
+      fetch_round(b + 32, &g_nxt, nxt, ok_nxt);
+#pragma unroll
+      for (int h = 0; h < kVecs; ++h) {
+        const uint32_t after = admit(ok_cur[h], g_cur * kVecs + h, cur[h], thr);
+        handed_out = after > handed_out ? after : handed_out;
+        cur[h] = nxt[h];
+        ok_cur[h] = ok_nxt[h];
+      }
+      g_cur = g_nxt;
     }
     const int left = all ? 0 : nparked - upto;  // < 32
     const uint32_t moved = lane < left ? park[upto + lane] : 0u;
@@ -943,11 +967,23 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
 
   // The exact k-th key among the candidates: its upper 11 bits from the histogram (it counts
   // every candidate), the bits below 8 at a time (the last digit has 4).
+  // (MAP: the histogram is in single 15-bit keys above the threshold, so the walk gives the upper
+  // 15 bits at once -- unless the k-th key lies in the last bin, which holds everything beyond the
+  // histogram's reach: then the candidates are counted again by their upper 11 bits.)
   find_from_top<T>(sh, coarse, kCoarseBins, (uint32_t)k, 0);
-  uint32_t kth = sh.picked_bin << kCoarseShift, known = (uint32_t)(kCoarseBins - 1) << kCoarseShift;
-  uint32_t take = sh.picked_remaining, ties = 0;
+  bool fine = MAP && sh.picked_bin < (uint32_t)kCoarseBins - 1u;
+  if (MAP && !fine) {
+    __syncthreads();
+    clear_words<T>(coarse, kCoarseBins);
+    for (uint32_t i = threadIdx.x; i < count; i += T) atomicAdd(&coarse[R::key(cand_pat[i]) >> kCoarseShift], 1u);
+    __syncthreads();
+    find_from_top<T>(sh, coarse, kCoarseBins, (uint32_t)k, 0);
+  }
+  uint32_t kth = fine ? thr + (sh.picked_bin << kFineShift) : sh.picked_bin << kCoarseShift;
+  uint32_t known = fine ? 0x7FFFu << kFineShift : (uint32_t)(kCoarseBins - 1) << kCoarseShift;
+  uint32_t take = sh.picked_remaining, ties = coarse[sh.picked_bin];
   __syncthreads();
-  for (int shift = kCoarseShift - 8, round = 1; shift > -8; shift -= 8, ++round) {
+  for (int shift = (fine ? kFineShift : kCoarseShift) - 8, round = 1; shift > -8; shift -= 8, ++round) {
     const int low = shift < 0 ? 0 : shift, width = shift < 0 ? 8 + shift : 8;
     clear_words<T>(coarse, 256);
     for (uint32_t i = threadIdx.x; i < count; i += T) {
@@ -1031,30 +1067,51 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   uint32_t group_shift = 0;                             // words per group: the smallest power of two that fits
   while (((n_words + (1u << group_shift) - 1u) >> group_shift) > kGroups) ++group_shift;
   const uint32_t n_groups = (n_words + (1u << group_shift) - 1u) >> group_shift;
-  const uint32_t per_thread = (n_groups + T - 1) / T;   // consecutive groups a thread counts
-  {
-    uint4* q = reinterpret_cast<uint4*>(bitmap);         // (the ring is a whole number of 16-byte words)
-    for (uint32_t wd = threadIdx.x; wd < (n_words + 3u) / 4u; wd += T) q[wd] = make_uint4(0u, 0u, 0u, 0u);
-  }
+  const uint32_t n_quads = (n_words + 3u) / 4u;          // 16-byte words (the bitmap's place is a whole number of them)
+  uint4* quads = reinterpret_cast<uint4*>(bitmap);
+  for (uint32_t q = threadIdx.x; q < n_quads; q += T) quads[q] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   for (uint32_t i = threadIdx.x; i < count; i += T)
     if (selected(i)) atomicOr(&bitmap[cand_flat[i] >> 5], 1u << (cand_flat[i] & 31u));
   __syncthreads();
   {
-    const uint32_t lo = threadIdx.x * per_thread < n_groups ? threadIdx.x * per_thread : n_groups;
-    const uint32_t hi = lo + per_thread < n_groups ? lo + per_thread : n_groups;
-    uint32_t ones = 0;
-    for (uint32_t g = lo; g < hi; ++g) {
-      const uint32_t w0 = g << group_shift, w1 = w0 + (1u << group_shift) < n_words ? w0 + (1u << group_shift) : n_words;
-      for (uint32_t wd = w0; wd < w1; ++wd) ones += (uint32_t)__popc(bitmap[wd]);
+    // A warp counts a contiguous stretch of the bitmap, 32 quads (one per lane) at a time, so its
+    // loads and stores touch every bank once; a prefix sum over the lanes puts the counts in
+    // index order.  First the stretches' totals, then the stores with the warps before added.
+    constexpr int kW = T / 32;
+    const uint32_t quads_per_warp = ((n_quads + kW - 1) / kW + 31u) / 32u * 32u;
+    const uint32_t q_begin = (uint32_t)warp * quads_per_warp;
+    uint32_t stretch = 0;
+    for (uint32_t q0 = q_begin; q0 < q_begin + quads_per_warp && q0 < n_quads; q0 += 32) {
+      const uint32_t q = q0 + (uint32_t)lane;
+      const uint4 v = q < n_quads ? quads[q] : make_uint4(0u, 0u, 0u, 0u);
+      stretch += (uint32_t)(__popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w));
     }
+    stretch = __reduce_add_sync(kFull, stretch);
     unsigned long long total;
-    uint32_t running = (uint32_t)scan_exclusive<T>(sh, ones, 0, &total);  // set bits before this thread's groups
+    // (every lane of a warp passes the same value: the scan is over warps, read from lane 0's result)
+    uint32_t running = (uint32_t)scan_exclusive<T>(sh, lane == 0 ? stretch : 0u, 0, &total);
+    running = __shfl_sync(kFull, running, 0);
     // (scan_exclusive's barrier lies between the histogram's last use and these stores)
-    for (uint32_t g = lo; g < hi; ++g) {
-      before_group[g] = (uint16_t)running;
-      const uint32_t w0 = g << group_shift, w1 = w0 + (1u << group_shift) < n_words ? w0 + (1u << group_shift) : n_words;
-      for (uint32_t wd = w0; wd < w1; ++wd) running += (uint32_t)__popc(bitmap[wd]);
+    for (uint32_t q0 = q_begin; q0 < q_begin + quads_per_warp && q0 < n_quads; q0 += 32) {
+      const uint32_t q = q0 + (uint32_t)lane;
+      const uint4 v = q < n_quads ? quads[q] : make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t c[4] = {(uint32_t)__popc(v.x), (uint32_t)__popc(v.y), (uint32_t)__popc(v.z), (uint32_t)__popc(v.w)};
+      const uint32_t mine = c[0] + c[1] + c[2] + c[3];
+      uint32_t incl = mine;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t other = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += other;
+      }
+      uint32_t before = running + incl - mine;
+      running += __shfl_sync(kFull, incl, 31);
+#pragma unroll
+      for (uint32_t j = 0; j < 4; ++j) {
+        const uint32_t wd = 4u * q + j;
+        if (q < n_quads && wd < n_words && (wd & ((1u << group_shift) - 1u)) == 0) before_group[wd >> group_shift] = (uint16_t)before;
+        before += c[j];
+      }
     }
   }
   __syncthreads();
