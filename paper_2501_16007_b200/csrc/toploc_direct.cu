@@ -1567,6 +1567,7 @@ namespace small_k {
 using namespace toploc_device;
 
 constexpr int kSmallK = SelectSharedBig::kMaxK;  // 512; k <= 256 takes the smaller scratch (sixteen warps per SM)
+constexpr int kWarpsBestUpTo = SelectShared::kMaxK;  // 256: beyond it the half-block kernels are preferred where they apply
 constexpr long long kMaxElems = 1ll << 19;
 template <class SH>
 constexpr int min_blocks() { return SH::kMaxK > 256 ? 13 : 15; }
@@ -1914,12 +1915,15 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
-  if (small_k::applies(lay)) {
+  // k <= 256: a warp per chunk; above, two half-blocks per SM where they apply (they are level with
+  // the warps on chunks of 2^18 elements and well ahead on smaller ones), else the warps up to k = 512
+  const bool halves = half_block::applies(lay, plan.vector);
+  if (small_k::applies(lay) && !(halves && lay->k > small_k::kWarpsBestUpTo)) {
     const int mode = small_k::layout_mode(d_act, lay);
     return lay->dtype == TOPLOC_DTYPE_BF16 ? small_k::launch_commit<0>(mode, plan.num_chunks, stream, p, d_commits, d_status)
                                            : small_k::launch_commit<1>(mode, plan.num_chunks, stream, p, d_commits, d_status);
   }
-  if (half_block::applies(lay, plan.vector)) {
+  if (halves) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, plan.device) != cudaSuccess) return TOPLOC_ERR_CUDA;
     const long long rescuers = plan.num_chunks < sms ? plan.num_chunks : sms;
@@ -1970,12 +1974,13 @@ static int verify_direct_with(const void* d_act, const toploc_layout* lay, const
   io.thr_each = d_thr_each;
   const size_t smem = kSharedBytes;
   const DirectParams& p = plan.params;
-  if (small_k::applies(lay)) {
+  const bool halves = half_block::applies(lay, plan.vector);
+  if (small_k::applies(lay) && !(halves && lay->k > small_k::kWarpsBestUpTo)) {
     const int mode = small_k::layout_mode(d_act, lay);
     return lay->dtype == TOPLOC_DTYPE_BF16 ? small_k::launch_verify<0>(mode, plan.num_chunks, stream, p, io)
                                            : small_k::launch_verify<1>(mode, plan.num_chunks, stream, p, io);
   }
-  if (half_block::applies(lay, plan.vector)) {
+  if (halves) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, plan.device) != cudaSuccess) return TOPLOC_ERR_CUDA;
     const long long rescuers = plan.num_chunks < sms ? plan.num_chunks : sms;

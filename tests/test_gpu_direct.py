@@ -72,6 +72,15 @@ def test_70b_shaped_chunks_and_ragged_tail():
     direct_case(act, L, k, S, T, {"noise": synth.honest_noise(act, seed=3)}, "70B-shaped")
 
 
+def test_k_above_256_on_chunks_too_long_for_two_blocks_per_sm():
+    # 2^19 elements per chunk: beyond the 512-thread kernels' reach, so k = 300 and 512 stay with the
+    # warp-per-chunk kernels (which they leave for chunks of up to 2^18 elements)
+    S, T, H, L = 2, 64, 8192, 64
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=63, device=DEV, outliers="jitter")
+    for k in (300, 512):
+        direct_case(act, L, k, S, T, {"noise": synth.honest_noise(act, seed=5)}, "2^19-element chunks k=%d" % k)
+
+
 @pytest.mark.parametrize("k", [128, 1024])
 def test_full_size_launch_sampled(k):
     """The 70B-shaped batch (256 sequences x 4096 tokens, H = 8192) committed and validated in one call
