@@ -71,7 +71,7 @@ constexpr int kStages = TOPLOC_SELECT_STAGES;
 #define TOPLOC_HIT_CAP 184
 #endif
 #ifndef TOPLOC_HIT_CAP_BIG
-#define TOPLOC_HIT_CAP_BIG 256
+#define TOPLOC_HIT_CAP_BIG 188
 #endif
 constexpr int kHitTrigger = TOPLOC_HIT_TRIGGER;    // select: drain once this many are parked (more for large k)
 constexpr int kIdxBits = 24;             // flat index field of a candidate
@@ -115,6 +115,9 @@ struct __align__(16) SelectSharedT {
 };
 using SelectShared = SelectSharedT<TOPLOC_CAND_CAP, 256, TOPLOC_HIT_CAP>;
 using SelectSharedBig = SelectSharedT<1024, TOPLOC_MAX_K, TOPLOC_HIT_CAP_BIG>;
+// Shared memory is handed out in units of 256 bytes plus 1 KB per block, 228 KB per SM: these sizes
+// are what keeps sixteen (thirteen) one-warp blocks resident.
+static_assert(sizeof(SelectShared) <= 13568 && sizeof(SelectSharedBig) <= 16640, "resident blocks per SM");
 static_assert(TOPLOC_MAX_K == 512, "SelectSharedBig is sized for k up to 512");
 constexpr uint32_t kNoBin = 0xFFFFFFFFu;
 
