@@ -238,6 +238,63 @@ def verify_proofs(act, proofs, chunk_len, k, num_seqs, tokens_per_seq=0, seq_off
     return results
 
 
+def _pointer_array(arrays):
+    """A C array of pointers to the given numpy arrays (None entries become NULL)."""
+    out = (ctypes.c_void_p * len(arrays))()
+    for i, a in enumerate(arrays):
+        out[i] = None if a is None else a.ctypes.data
+    return out
+
+
+def build_proofs_ks(act, chunk_len, ks, num_seqs, tokens_per_seq=0, seq_offsets=None, threads=None):
+    """build_proofs for several k over the same batch: each chunk is ranked once, for the largest
+    k, and every k takes its prefix of that ranking (topk(h, k) is the first k of the sorted
+    chunk).  16-bit field.  Returns {k: (proofs, status, indices)}."""
+    assert act.ndim == 2 and act.strides[1] == act.itemsize
+    hidden = act.shape[1]
+    row_stride = act.strides[0] // act.itemsize
+    so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
+    n = num_chunks(num_seqs, tokens_per_seq, chunk_len, so)
+    ks = [int(k) for k in ks]
+    karr = np.asarray(ks, np.int32)
+    proofs = [np.zeros((n, 2 + 2 * k), np.uint8) for k in ks]
+    status = [np.zeros(n, np.uint8) for _ in ks]
+    indices = [np.zeros((n, k), np.int32) for k in ks]
+    rc = lib().oracle_build_proofs_ks(
+        _ptr(act), _dtype_code(act), hidden, chunk_len, _ptr(karr), len(ks), num_seqs, ctypes.c_int64(tokens_per_seq),
+        None if so is None else _ptr(so), ctypes.c_int64(row_stride), _pointer_array(proofs), _pointer_array(status),
+        _pointer_array(indices), threads or default_threads())
+    assert rc == 0
+    return {k: (proofs[i], status[i], indices[i]) for i, k in enumerate(ks)}
+
+
+def verify_proofs_ks(act, proofs_by_k, chunk_len, num_seqs, tokens_per_seq=0, seq_offsets=None, t_exp_by_k=None,
+                     t_mean=10.0, t_median=8.0, sign_in_exponent=True, gen_indices_by_k=None, threads=None):
+    """verify_proofs for several k over the same batch (proofs_by_k: {k: uint8[n, 2+2k]}), each
+    chunk ranked once.  t_exp_by_k: {k: exponent threshold}.  Returns {k: results}."""
+    assert act.ndim == 2 and act.strides[1] == act.itemsize
+    hidden = act.shape[1]
+    row_stride = act.strides[0] // act.itemsize
+    so = None if seq_offsets is None else np.ascontiguousarray(seq_offsets, np.int64)
+    n = num_chunks(num_seqs, tokens_per_seq, chunk_len, so)
+    ks = [int(k) for k in proofs_by_k]
+    karr = np.asarray(ks, np.int32)
+    proofs = [np.ascontiguousarray(proofs_by_k[k], np.uint8) for k in ks]
+    for k, pr in zip(ks, proofs):
+        assert pr.shape == (n, 2 + 2 * k)
+    texp = np.asarray([38 if t_exp_by_k is None else int(t_exp_by_k[k]) for k in ks], np.int32)
+    gens = [None if gen_indices_by_k is None or gen_indices_by_k.get(k) is None
+            else np.ascontiguousarray(gen_indices_by_k[k], np.int32) for k in ks]
+    results = [np.zeros(n, RESULT_DTYPE) for _ in ks]
+    rc = lib().oracle_verify_proofs_ks(
+        _ptr(act), _dtype_code(act), hidden, chunk_len, _ptr(karr), len(ks), num_seqs, ctypes.c_int64(tokens_per_seq),
+        None if so is None else _ptr(so), ctypes.c_int64(row_stride), _pointer_array(proofs), _ptr(texp),
+        ctypes.c_double(t_mean), ctypes.c_double(t_median), int(bool(sign_in_exponent)), _pointer_array(gens),
+        _pointer_array(results), threads or default_threads())
+    assert rc == 0
+    return {k: results[i] for i, k in enumerate(ks)}
+
+
 def _chunk_spans(num_seqs, tokens_per_seq, chunk_len, seq_offsets):
     spans = []
     for s in range(num_seqs):

@@ -333,6 +333,33 @@ int oracle_decode(const uint8_t* proof, int64_t len, int* k_out, uint32_t* m_out
 /* ------------------------------------------------------------------ */
 /* Algorithm 1 for one chunk.                                          */
 /* ------------------------------------------------------------------ */
+/* Algorithm 1 after its topk line: idx / bits are the k selected elements in rank order. */
+static int build_from_selection(const uint32_t* idx, const uint16_t* bits, int k, uint8_t* proof,
+                                int32_t* indices_opt) {
+  uint32_t* xs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint32_t* ys = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
+  uint16_t* coef = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
+  int status = ST_OK;
+  if (indices_opt)
+    for (int j = 0; j < k; ++j) indices_opt[j] = (int32_t)idx[j];
+  uint32_t m = oracle_find_injective_modulus(idx, k, 1);
+  if (m == 0) {
+    status = ST_NO_MODULUS;
+  } else {
+    for (int j = 0; j < k; ++j) {
+      xs[j] = (idx[j] % m) % P_FIELD;
+      ys[j] = (uint32_t)bits[j] % P_FIELD; /* Algorithm 3 reduces every y mod M first */
+      if (bits[j] >= P_FIELD) status = ST_NONFINITE;
+    }
+    oracle_interpolate(xs, ys, k, coef);
+    oracle_encode(m, coef, k, proof);
+  }
+  free(xs);
+  free(ys);
+  free(coef);
+  return status;
+}
+
 int oracle_build_chunk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
                        uint8_t* proof, int32_t* indices_opt) {
   size_t nbytes = 2 + 2 * (size_t)k;
@@ -340,31 +367,10 @@ int oracle_build_chunk(const void* chunk, int dtype, int rows, int hidden, int64
   if (indices_opt) memset(indices_opt, 0, (size_t)k * sizeof(int32_t));
   uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
   uint16_t* bits = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
-  uint32_t* xs = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
-  uint32_t* ys = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
-  uint16_t* coef = (uint16_t*)malloc((size_t)k * sizeof(uint16_t));
   int status = oracle_topk(chunk, dtype, rows, hidden, row_stride, k, idx, bits);
-  if (status == ST_OK) {
-    if (indices_opt)
-      for (int j = 0; j < k; ++j) indices_opt[j] = (int32_t)idx[j];
-    uint32_t m = oracle_find_injective_modulus(idx, k, 1);
-    if (m == 0) {
-      status = ST_NO_MODULUS;
-    } else {
-      for (int j = 0; j < k; ++j) {
-        xs[j] = (idx[j] % m) % P_FIELD;
-        ys[j] = (uint32_t)bits[j] % P_FIELD; /* Algorithm 3 reduces every y mod M first */
-        if (bits[j] >= P_FIELD) status = ST_NONFINITE;
-      }
-      oracle_interpolate(xs, ys, k, coef);
-      oracle_encode(m, coef, k, proof);
-    }
-  }
+  if (status == ST_OK) status = build_from_selection(idx, bits, k, proof, indices_opt);
   free(idx);
   free(bits);
-  free(xs);
-  free(ys);
-  free(coef);
   return status;
 }
 
@@ -378,9 +384,14 @@ static int ascending_u32(const void* a, const void* b) {
 /* 16-bit pattern: bit 15 sign, bits 14..7 exponent, bits 6..0         */
 /* mantissa (bf16 has 7 mantissa bits, Section 5.2).                   */
 /* ------------------------------------------------------------------ */
-void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
-                         const uint8_t* proof, int t_exp, double t_mean, double t_median,
-                         int sign_in_exponent, const int32_t* gen_indices_opt, oracle_result* out) {
+/* Algorithm 2 from its second line on.  select: the topk line -- either sorts the chunk (chunk
+ * != NULL) or, when the caller has already ranked the chunk's elements, takes the first k of that
+ * ranking (ranked_idx / ranked_bits hold at least k entries, or n_ranked < k of them when the
+ * chunk has fewer than k elements). */
+static void verify_with_selection(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride,
+                                  const uint32_t* ranked_idx, const uint16_t* ranked_bits, int64_t n_ranked, int k,
+                                  const uint8_t* proof, int t_exp, double t_mean, double t_median,
+                                  int sign_in_exponent, const int32_t* gen_indices_opt, oracle_result* out) {
   memset(out, 0, sizeof(*out));
   out->topk_mismatch = -1;
   uint32_t* idx = (uint32_t*)malloc((size_t)k * sizeof(uint32_t));
@@ -391,7 +402,16 @@ void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int
   uint32_t m = 0;
   int status = oracle_decode(proof, 2 + 2 * (int64_t)k, &kk, &m, coef);
   out->modulus = m;
-  if (status == ST_OK) status = oracle_topk(chunk, dtype, rows, hidden, row_stride, k, idx, bits);
+  if (status == ST_OK) {
+    if (chunk != NULL) {
+      status = oracle_topk(chunk, dtype, rows, hidden, row_stride, k, idx, bits);
+    } else if (n_ranked < k) {
+      status = ST_K_EXCEEDS;
+    } else {
+      memcpy(idx, ranked_idx, (size_t)k * sizeof(uint32_t));
+      memcpy(bits, ranked_bits, (size_t)k * sizeof(uint16_t));
+    }
+  }
   if (status == ST_OK) {
     uint32_t err_e = 0, n = 0, sum = 0;
     for (int j = 0; j < k; ++j) {
@@ -443,6 +463,13 @@ void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int
   free(bits);
   free(coef);
   free(diffs);
+}
+
+void oracle_verify_chunk(const void* chunk, int dtype, int rows, int hidden, int64_t row_stride, int k,
+                         const uint8_t* proof, int t_exp, double t_mean, double t_median,
+                         int sign_in_exponent, const int32_t* gen_indices_opt, oracle_result* out) {
+  verify_with_selection(chunk, dtype, rows, hidden, row_stride, NULL, NULL, 0, k, proof, t_exp, t_mean, t_median,
+                        sign_in_exponent, gen_indices_opt, out);
 }
 
 /* ================================================================== */
@@ -1106,4 +1133,133 @@ int oracle_verify_proofs(const void* act, int dtype, int hidden, int chunk_len, 
   run_jobs(&jb, nthreads);
   free(spans);
   return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* Several k over the same batch (a parameter sweep).  topk(h, k) is    */
+/* the first k of the chunk's elements in rank order, so the selections */
+/* of all the k are prefixes of one ranking: each chunk is sorted once, */
+/* for the largest k, and Algorithm 1 or 2 then runs once per k on its  */
+/* prefix.  16-bit field only (dtype 0 or 1).  Arrays indexed by the    */
+/* position of k in ks; a chunk with fewer than k elements gets         */
+/* ST_K_EXCEEDS for that k, as in the single-k drivers.                 */
+/* ------------------------------------------------------------------ */
+typedef struct {
+  int tid, nthreads, verify;
+  const uint8_t* act;
+  int dtype, hidden, nk;
+  const int32_t* ks;
+  int64_t row_stride;
+  const chunk_span* spans;
+  int64_t count;
+  uint8_t* const* proofs;
+  uint8_t* const* status;
+  int32_t* const* indices;
+  const uint8_t* const* proofs_in;
+  const int32_t* const* gen_indices;
+  oracle_result* const* results;
+  const int32_t* t_exp; /* one per k */
+  double t_mean, t_median;
+  int sign_in_exponent;
+} sweep_job;
+
+static void* sweep_worker(void* arg) {
+  sweep_job* jb = (sweep_job*)arg;
+  size_t esz = jb->dtype == 0 ? 2 : 4;
+  int kmax = 0;
+  for (int i = 0; i < jb->nk; ++i)
+    if (jb->ks[i] > kmax) kmax = jb->ks[i];
+  uint32_t* idx = (uint32_t*)malloc((size_t)kmax * sizeof(uint32_t));
+  uint16_t* bits = (uint16_t*)malloc((size_t)kmax * sizeof(uint16_t));
+  for (int64_t c = jb->tid; c < jb->count; c += jb->nthreads) {
+    const void* chunk = jb->act + (size_t)jb->spans[c].row0 * (size_t)jb->row_stride * esz;
+    int64_t n = (int64_t)jb->spans[c].rows * jb->hidden;
+    int ranked = (int)(n < kmax ? n : kmax); /* the whole (short) chunk, or the largest k */
+    oracle_topk(chunk, jb->dtype, jb->spans[c].rows, jb->hidden, jb->row_stride, ranked, idx, bits);
+    for (int i = 0; i < jb->nk; ++i) {
+      int k = jb->ks[i];
+      size_t pbytes = 2 + 2 * (size_t)k;
+      if (!jb->verify) {
+        uint8_t* proof = jb->proofs[i] + (size_t)c * pbytes;
+        int32_t* ind = (jb->indices && jb->indices[i]) ? jb->indices[i] + (size_t)c * k : NULL;
+        memset(proof, 0, pbytes);
+        if (ind) memset(ind, 0, (size_t)k * sizeof(int32_t));
+        jb->status[i][c] = (uint8_t)(k > n ? ST_K_EXCEEDS : build_from_selection(idx, bits, k, proof, ind));
+      } else {
+        const int32_t* gen = (jb->gen_indices && jb->gen_indices[i]) ? jb->gen_indices[i] + (size_t)c * k : NULL;
+        verify_with_selection(NULL, jb->dtype, jb->spans[c].rows, jb->hidden, jb->row_stride, idx, bits, ranked, k,
+                              jb->proofs_in[i] + (size_t)c * pbytes, jb->t_exp[i], jb->t_mean, jb->t_median,
+                              jb->sign_in_exponent, gen, &jb->results[i][c]);
+      }
+    }
+  }
+  free(idx);
+  free(bits);
+  return NULL;
+}
+
+static int run_sweep(sweep_job* proto, int num_seqs, int64_t tokens_per_seq, const int64_t* seq_offsets,
+                     int chunk_len, int nthreads) {
+  if (proto->dtype != 0 && proto->dtype != 1) return -1;
+  int64_t n = enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, NULL);
+  chunk_span* spans = (chunk_span*)malloc((size_t)(n > 0 ? n : 1) * sizeof(chunk_span));
+  enumerate_chunks(num_seqs, tokens_per_seq, seq_offsets, chunk_len, spans);
+  proto->spans = spans;
+  proto->count = n;
+  if (nthreads < 1) nthreads = 1;
+  pthread_t* th = (pthread_t*)malloc((size_t)nthreads * sizeof(pthread_t));
+  sweep_job* jobs = (sweep_job*)malloc((size_t)nthreads * sizeof(sweep_job));
+  for (int t = 0; t < nthreads; ++t) {
+    jobs[t] = *proto;
+    jobs[t].tid = t;
+    jobs[t].nthreads = nthreads;
+    pthread_create(&th[t], NULL, sweep_worker, &jobs[t]);
+  }
+  for (int t = 0; t < nthreads; ++t) pthread_join(th[t], NULL);
+  free(jobs);
+  free(th);
+  free(spans);
+  return 0;
+}
+
+int oracle_build_proofs_ks(const void* act, int dtype, int hidden, int chunk_len, const int32_t* ks, int nk,
+                           int num_seqs, int64_t tokens_per_seq, const int64_t* seq_offsets, int64_t row_stride,
+                           uint8_t* const* proofs, uint8_t* const* status, int32_t* const* indices_opt,
+                           int nthreads) {
+  sweep_job jb;
+  memset(&jb, 0, sizeof(jb));
+  jb.act = (const uint8_t*)act;
+  jb.dtype = dtype;
+  jb.hidden = hidden;
+  jb.ks = ks;
+  jb.nk = nk;
+  jb.row_stride = row_stride;
+  jb.proofs = proofs;
+  jb.status = status;
+  jb.indices = indices_opt;
+  return run_sweep(&jb, num_seqs, tokens_per_seq, seq_offsets, chunk_len, nthreads);
+}
+
+int oracle_verify_proofs_ks(const void* act, int dtype, int hidden, int chunk_len, const int32_t* ks, int nk,
+                            int num_seqs, int64_t tokens_per_seq, const int64_t* seq_offsets, int64_t row_stride,
+                            const uint8_t* const* proofs, const int32_t* t_exp_per_k, double t_mean,
+                            double t_median, int sign_in_exponent, const int32_t* const* gen_indices_opt,
+                            oracle_result* const* results, int nthreads) {
+  sweep_job jb;
+  memset(&jb, 0, sizeof(jb));
+  jb.verify = 1;
+  jb.act = (const uint8_t*)act;
+  jb.dtype = dtype;
+  jb.hidden = hidden;
+  jb.ks = ks;
+  jb.nk = nk;
+  jb.row_stride = row_stride;
+  jb.proofs_in = proofs;
+  jb.gen_indices = gen_indices_opt;
+  jb.results = results;
+  jb.t_exp = t_exp_per_k;
+  jb.t_mean = t_mean;
+  jb.t_median = t_median;
+  jb.sign_in_exponent = sign_in_exponent;
+  return run_sweep(&jb, num_seqs, tokens_per_seq, seq_offsets, chunk_len, nthreads);
 }

@@ -338,8 +338,8 @@ def test_config_70b_full_size_every_chunk():
 def test_config_70b_full_size_varied_selections(recipe):
     """With +-80 outliers every chunk selects the same index set (the first 128 outliers); jittered
     outlier magnitudes, plain heavy-tailed data and magnitudes that grow through every chunk make
-    the selected set, the modulus and the statistics differ from chunk to chunk.  Same full-size launches; sixteen whole sequences
-    (2048 chunks) against the oracle."""
+    the selected set, the modulus and the statistics differ from chunk to chunk.  Same full-size
+    launches; sixteen whole sequences (2048 chunks) against the oracle."""
     g, honest = full_size_70b_case(recipe, {"jitter": 40, "none": 41, "rising": 42}[recipe], range(7, 256, 16))
     distinct = {tuple(row) for row in g[2][:4096:64].cpu().numpy().tolist()}
     assert len(distinct) > 32, "the selected index sets should vary from chunk to chunk"
@@ -348,35 +348,26 @@ def test_config_70b_full_size_varied_selections(recipe):
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("hidden", [2048, 4096, 8192])
 def test_config_sweep(hidden, dtype):
-    """k in {32, 64, 128, 256} x chunk length in {16, 32, 64} at 128 sequences x 1024 tokens.  The
-    GPU runs every point in full.  The oracle checks every chunk of the corner points -- smallest
-    and largest k on the smallest and the largest chunk of each dtype -- and eight whole
-    sequences of every other point."""
+    """k in {32, 64, 128, 256} x chunk length in {16, 32, 64} at 128 sequences x 1024 tokens.
+    Every chunk of every point is compared with the oracle: proof bytes, statuses and indices of
+    the build, every statistic and verdict of the validation against an honest-noise copy.  The
+    oracle ranks a chunk once per chunk length and gives each k its prefix of that ranking."""
     S, T = 128, 1024
+    ks = (32, 64, 128, 256)
     act = synth.make_activations(S, T, hidden, dtype, seed=50 + hidden // 1024, device=DEV)
     noisy = synth.honest_noise(act, seed=9)
     host, host_noisy = synth.host_patterns(act), synth.host_patterns(noisy)
     for chunk_len in (16, 32, 64):
-        cps = T // chunk_len
-        for k in (32, 64, 128, 256):
+        built = oracle.build_proofs_ks(host, chunk_len, ks, S, T)
+        judged = oracle.verify_proofs_ks(host_noisy, {k: built[k][0] for k in ks}, chunk_len, S, T,
+                                         t_exp_by_k={k: oracle_thresholds(k)["t_exp"] for k in ks},
+                                         gen_indices_by_k={k: built[k][2] for k in ks})
+        for k in ks:
+            where = "sweep H%d L%d k%d %s" % (hidden, chunk_len, k, dtype)
             g = gpu_build(act, chunk_len, k, S, T)
+            assert_build_equal(g, built[k], where)
             gv = gpu_verify(noisy, g[0], chunk_len, k, S, T, gen_indices=g[2])
-            corner = k in (32, 256) and (hidden, chunk_len) in ((2048, 16), (8192, 64))
-            seqs = list(range(S)) if corner else [1, 18, 35, 52, 69, 86, 103, 126]
-            # consecutive runs of sequences go to the oracle in one call
-            runs, start = [], seqs[0]
-            for a, b in zip(seqs, seqs[1:] + [None]):
-                if b != a + 1:
-                    runs.append((start, a + 1))
-                    start = b
-            for s0, s1 in runs:
-                rows, chunks = slice(s0 * T, s1 * T), slice(s0 * cps, s1 * cps)
-                r = oracle.build_proofs(host[rows], chunk_len, k, s1 - s0, T)
-                where = "sweep H%d L%d k%d %s seqs %d..%d" % (hidden, chunk_len, k, dtype, s0, s1 - 1)
-                assert_build_equal(tuple(t[chunks] for t in g), r, where)
-                rv = oracle.verify_proofs(host_noisy[rows], r[0], chunk_len, k, s1 - s0, T, gen_indices=r[2],
-                                          **oracle_thresholds(k))
-                assert_results_equal(gv[chunks], rv, where)
+            assert_results_equal(gv, judged[k], where)
 
 
 def test_thresholds_per_chunk_decide_each_chunk_by_its_own_entry():

@@ -502,6 +502,31 @@ def test_ragged_batches_and_row_stride():
     assert res["accept"].tolist() == [1] * 7
 
 
+def test_several_k_over_one_ranking_equal_the_single_k_drivers():
+    """The sweep drivers rank a chunk once and give every k its prefix: same bytes, statuses,
+    indices and results as one call per k -- on a ragged batch whose last chunks are shorter than
+    the largest k, with fp32 values as well, and with a proof built from other data."""
+    rng = np.random.default_rng(34)
+    for make in (lambda: random_chunk(rng, 23, 64), lambda: rng.standard_normal((23, 64)).astype(np.float32)):
+        act, other = make(), make()
+        offsets = [0, 9, 9, 23]                 # chunk_len 4: chunks of 4,4,1 and 4,4,4,2 rows (64..256 elements)
+        ks = [200, 3, 64, 128]
+        built = oracle.build_proofs_ks(act, 4, ks, 3, seq_offsets=offsets)
+        foreign = oracle.build_proofs_ks(other, 4, ks, 3, seq_offsets=offsets)
+        for k in ks:
+            p1, s1, i1 = oracle.build_proofs(act, 4, k, 3, seq_offsets=offsets)
+            assert np.array_equal(built[k][0], p1) and np.array_equal(built[k][1], s1) and np.array_equal(built[k][2], i1)
+        assert oracle.ST_K_EXCEEDS in built[200][1].tolist() and oracle.ST_OK in built[200][1].tolist()
+        thr = {k: (38 * k) // 128 for k in ks}
+        for proofs, gen in ((built, True), (foreign, False)):
+            many = oracle.verify_proofs_ks(act, {k: proofs[k][0] for k in ks}, 4, 3, seq_offsets=offsets, t_exp_by_k=thr,
+                                           gen_indices_by_k={k: proofs[k][2] for k in ks} if gen else None)
+            for k in ks:
+                one = oracle.verify_proofs(act, proofs[k][0], 4, k, 3, seq_offsets=offsets, t_exp=thr[k],
+                                           gen_indices=proofs[k][2] if gen else None)
+                assert many[k].tobytes() == one.tobytes(), (k, gen)
+
+
 # ---------------------------------------------------------------- seeded configurations
 
 def tiny_config(seed=0, outliers="fixed", hidden=4096, chunks=4):
