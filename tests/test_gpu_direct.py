@@ -150,11 +150,25 @@ def test_many_equal_values_go_to_the_rescue_launch():
     direct_case(f, L, 2048, 3, L, None, "equal values, fp32")
 
 
-def test_special_patterns():
-    H, L, k = 512, 8, 200
+@pytest.mark.parametrize("k", [200, 300, 1000])
+def test_special_patterns(k):
+    H, L = 512, 8
     bits = torch.randint(0, 65536, (L, H), dtype=torch.int32, device=DEV).to(torch.int16)  # NaN, Inf, subnormals
     act = bits.view(torch.bfloat16)
-    direct_case(act, L, k, 1, L, None, "random patterns")
+    direct_case(act, L, k, 1, L, None, "random patterns k=%d" % k)
+
+
+@pytest.mark.parametrize("scale", [2.0 ** -40, 2.0 ** -18, 2.0 ** 9, 2.0 ** 30])
+def test_magnitudes_far_from_one(scale):
+    # the one-pass selection for k > 256 keeps a coarse byte per 8 elements that covers 2^-20 .. 2^12:
+    # chunks that lie below, across the lower edge, across the upper edge and above the window
+    S, T, H, L = 2, 64, 2048, 32
+    base = synth.make_activations(S, T, H, torch.bfloat16, seed=97, device=DEV, outliers="jitter")
+    act = (base.to(torch.float32) * scale).to(torch.bfloat16)
+    for k in (300, 1024):
+        direct_case(act, L, k, S, T, {"noise": synth.honest_noise(act, seed=6)}, "scale %g k=%d" % (scale, k))
+    f = (synth.make_activations(S, T, H, torch.float32, seed=98, device=DEV, outliers="none") * scale).contiguous()
+    direct_case(f, L, 600, S, T, None, "fp32 scale %g" % scale)
 
 
 def test_odd_shapes_take_the_scalar_path():
