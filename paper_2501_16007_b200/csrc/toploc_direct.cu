@@ -3,11 +3,20 @@
 // the exponent-error table in Section 3), and their validation (Algorithm 2 with the
 // polynomial evaluation replaced by an index look-up).
 //
-// Kernels:
-//   toploc_direct_commit_kernel<dtype, vector>   one 1024-thread block per chunk
-//   toploc_direct_verify_kernel<dtype, vector>   the same selection, then the comparison
+// Kernels, by the shape of the call:
+//   k <= 256 (k <= 512 where the next pair does not apply), chunks of at most 2^19 elements:
+//     toploc_direct_commit_warp_kernel / toploc_direct_verify_warp_kernel -- one warp per chunk,
+//     the selection of the proof path (toploc_device::select_topk);
+//   k > 256, 16-byte aligned rows, chunks of at most 2^18 elements:
+//     toploc_direct_commit_half_kernel / toploc_direct_verify_half_kernel -- one 512-thread block
+//     per chunk, two per SM; the chunk is streamed once (select_unordered with the bytes of its
+//     first pass); chunks whose candidates outgrow the buffer go to toploc_direct_*_rescue_kernel;
+//   everything else:
+//     toploc_direct_commit_kernel / toploc_direct_verify_kernel<dtype, vector> -- one 1024-thread
+//     block per chunk: select_unordered with a second streaming pass (aligned rows, at most 2^19
+//     elements), else one of the two selections below.
 //
-// Selection of a chunk (both kernels), one of two ways:
+// The two older selections of the 1024-thread kernels:
 //   one pass (vector layouts, k <= 2048): the chunk is streamed once; elements that reach a
 //   running threshold are kept as candidates in shared memory, in index order, and counted in a
 //   histogram of their upper 11 key bits, from which the threshold is raised as candidates
@@ -557,22 +566,28 @@ __device__ bool select_in_one_pass(DirectShared& sh, uint4* ring, const Reader<D
 }
 
 
-// One-pass selection without a barrier in the streaming loop (vector layouts, chunks of at most
-// kLooseMaxElems elements).  Every warp streams its share of the chunk on its own: a vector is
-// tested as a whole against the block's running threshold; vectors that pass are parked per
-// warp and, 32 at a time, unpacked by the whole warp into the block's candidate buffer
-// (slots handed out by one atomic per round) and counted in a histogram of their upper 11 key
-// bits.  The threshold only ever rises: whenever enough new candidates have arrived, one warp
-// (whoever gets the lock) walks the histogram from the top to the bin that holds the k-th
-// largest candidate so far and publishes that bin's lowest key -- at least k candidates reach
-// it, so nothing below it can belong to the top-k, whatever the other warps add meanwhile (the
-// counts only grow).  Warps that still test against an older threshold only admit more.
-// Candidates arrive in no particular order; the exact k-th key, the ties that belong to the
+// select_unordered: selection without a barrier in its streaming loops (vector layouts).
+// A first pass streams the chunk and counts every vector's largest key in a histogram of the
+// upper 11 key bits: the k-th largest of these maxima is reached by at least k elements, so it
+// is a sound threshold, and by few more than k, so the candidates fit a small buffer.  Then
+// the elements that reach the threshold are collected, in no particular order:
+//   MAP (two 512-thread blocks per SM): the first pass also left one byte per 8 elements -- the
+//   11 bits of the group's largest key, counted from 2^-20 -- and the collection is a scan of
+//   those bytes that parks the groups which reach the threshold's byte and fetches only them:
+//   the chunk is streamed once;
+//   otherwise (1024-thread block): a second streaming pass (from L2) tests every vector as a
+//   whole and parks those that pass; while it runs the threshold can still rise -- whenever
+//   enough new candidates have arrived, one warp (whoever gets the lock) walks the histogram of
+//   the candidates' upper 11 key bits to the bin that holds the k-th largest so far and
+//   publishes that bin's lowest key; at least k candidates reach it, so nothing below it can
+//   belong to the top-k, whatever the other warps add meanwhile (the counts only grow).
+// Parked groups are unpacked by a whole warp, 32 at a time, into the block's candidate buffer
+// (slots handed out by one atomic per round).  The exact k-th key, the ties that belong to the
 // top-k (lowest flat indices) and the position of every selected element in index order are
-// settled at the end.  ORDERED: emit(position in ascending index order, ...), by ranking the
-// selected indices in a bitmap of the chunk; otherwise positions are handed out as they come.
+// settled at the end.  ORDERED: positions in ascending index order, by ranking the selected
+// indices in a bitmap of the chunk; otherwise positions are handed out as they come.
 // Returns false, having emitted nothing, when the candidates outgrow their buffer.
-// Where the two-pass selection without barriers keeps its state; the two kernels that use it
+// Where select_unordered keeps its state; the two kernels that use it
 // (a 1024-thread block per SM, or two 512-thread blocks) carve it from their shared memory.
 template <int DT>
 struct LooseWorkspace {
