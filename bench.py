@@ -53,9 +53,9 @@ FALLBACK_HBM_GBS = 6650.0
 # by that batch's activation bytes.  The kernel reads every chunk once whatever the batch, so the
 # ratio carries over to the other bf16 batches.  None: no capture of the current kernel exists.
 SELECT_DRAM_TRAFFIC = {
-    "ratio_to_activation_bytes": 1.0143,   # (1083.140 MB read + 5.932 MB written) / 1073.742 MB
+    "ratio_to_activation_bytes": 1.0148,   # (1083.005 MB read + 6.613 MB written) / 1073.742 MB
     "source": "ncu capture of one toploc_select_kernel launch on the 8B-shaped batch, scaled by activation bytes "
-              "(profiles/select_kernel_8b_shape_ncu.md; selection code as of commit 62e0eac); not measured by this run",
+              "(profiles/select_kernel_8b_shape_ncu.md; selection code as of commit a7c3af5); not measured by this run",
 }
 
 
