@@ -109,8 +109,8 @@ static_assert((size_t)kCoarseBins * 4 + (size_t)cand_cap(0) * 6 <= (size_t)kBins
 static_assert(12 * TOPLOC_MAX_K_DIRECT <= kRingBytes, "the verify lists fit the idle ring");
 // The free-running one-pass selection parks, per warp, the vectors that passed the quick test
 // until there are enough of them to unpack with every lane busy; its candidates are unordered.
-constexpr int kParkCap = 32 + kUnroll * 32;   // a batch parks at most kUnroll vectors per lane
-constexpr int kParkTrigger = 32;
+constexpr int kParkCap = 64 + kUnroll * 32;   // a batch parks at most kUnroll vectors per lane
+constexpr int kParkTrigger = 64;              // at most: a round of unpacking takes two vectors per lane
 constexpr size_t kParkBytes = (size_t)kWarps * kParkCap * 4;
 __host__ __device__ constexpr int loose_cap(int dt) {
   return (int)(((size_t)kBins * 4 + kSpareBytes - (size_t)kCoarseBins * 4 - kParkBytes) / (dt == 0 ? 6 : 8)) / 64 * 64;
@@ -702,7 +702,7 @@ __device__ __forceinline__ void write_commitment(uint16_t* rec, const uint32_t* 
   }
 }
 
-template <int DT, bool ORDERED, int T, bool MAP, class Emit>
+template <int DT, bool ORDERED, int T, bool MAP, bool TWO, class Emit>
 __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, const Reader<DT, true>& rd, int k, Emit emit,
                                  uint16_t* rec = nullptr) {
   using R = Reader<DT, true>;
@@ -738,12 +738,24 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   // the candidates spread over hundreds of bins instead of a few, and the k-th key's upper 15 bits
   // come out of one walk.
   constexpr int kFineShift = key_bits(DT) - 15;
+  // A parked entry is a vector, or (MAP) 8 elements: one or two vectors.  A round of unpacking
+  // takes one entry per lane, or (TWO) two where an entry is one vector: one prefix sum and one
+  // atomic for twice the entries, which is worth 7 % of the call at k = 4096; at k = 1024 the
+  // rounds fill too slowly and it costs 2 %, so the caller asks for it from k = 2048 on.
+  constexpr int kVecs = MAP ? 8 / VEC : 1;                       // vectors per parked entry
+  constexpr int kEntriesPerLane = kVecs == 2 ? 1 : (TWO ? 2 : 1);  // entries a lane takes per round
+  constexpr int kLaneVecs = kVecs * kEntriesPerLane;              // 1 or 2
+  constexpr int kRound = 32 * kEntriesPerLane;
   auto fetch = [&](bool valid, uint32_t g) -> uint4 {
     return valid ? toploc_device::load_streaming(reinterpret_cast<const uint4*>(rd.address((int)g)))
                  : make_uint4(0u, 0u, 0u, 0u);
   };
-  auto admit = [&](bool valid, uint32_t g, const uint4& w, uint32_t thr) -> uint32_t {
-    uint32_t mask = valid ? toploc_device::passing_mask<DT, VEC>(w, thr) : 0u;
+  // Two vectors per lane: their elements that reach thr become candidates (one prefix sum and one
+  // atomic for both).  Returns the number of candidates handed out so far (0 if the round added none).
+  auto admit = [&](bool valid_a, uint32_t g_a, const uint4& w_a, bool valid_b, uint32_t g_b, const uint4& w_b,
+                   uint32_t thr) -> uint32_t {
+    uint32_t mask = valid_a ? toploc_device::passing_mask<DT, VEC>(w_a, thr) : 0u;
+    if (kLaneVecs == 2) mask |= (valid_b ? toploc_device::passing_mask<DT, VEC>(w_b, thr) : 0u) << VEC;
     const int mine = __popc(mask);
     int incl = mine;
 #pragma unroll
@@ -762,11 +774,14 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
     }
     uint32_t at = base + (uint32_t)(incl - mine);
     while (mask) {
-      const uint32_t e = (uint32_t)__ffs((int)mask) - 1u;
+      const uint32_t bit = (uint32_t)__ffs((int)mask) - 1u;
       mask &= mask - 1u;
+      const bool second = kLaneVecs == 2 && bit >= (uint32_t)VEC;
+      const uint32_t e = second ? bit - (uint32_t)VEC : bit;
+      const uint4 w = second ? w_b : w_a;
       uint32_t key, sign;
       toploc_device::pick_element<DT, VEC>(w, e, &key, &sign);
-      cand_flat[at] = g * VEC + e;
+      cand_flat[at] = (second ? g_b : g_a) * VEC + e;
       cand_pat[at] = (Pat)((sign << (DT == 0 ? 15 : 31)) | key);
       if (MAP) {
         const uint32_t above = (key - thr) >> kFineShift;
@@ -838,41 +853,51 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   int nparked = 0;
   // Unpacks the parked vectors a full round (32 of them) at a time; what is left over waits for
   // the next drain unless this is the last one.
+  static_assert(kRound <= kParkTrigger && kParkCap >= kParkTrigger - 1 + kUnroll * 32, "parking space");
   auto drain = [&](bool all) {
     __syncwarp();
     uint32_t handed_out = 0;
-    const int upto = all ? nparked : (nparked & ~31);
-    // a parked entry is a vector, or (MAP) 8 elements: one or two vectors; the next round's
-    // vectors are requested before this round's are unpacked
-    constexpr int kVecs = MAP ? kPerByte : 1;
-    uint4 cur[kVecs], nxt[kVecs];
-    uint32_t g_cur = 0, g_nxt = 0;
-    bool ok_cur[kVecs], ok_nxt[kVecs];
-    auto fetch_round = [&](int b, uint32_t* g, uint4 (&w)[kVecs], bool (&ok)[kVecs]) {
-      const bool valid = b < upto && b + lane < nparked;
-      *g = valid ? park[b + lane] : 0u;
+    const int upto = all ? nparked : nparked / kRound * kRound;
+    // the next round's vectors are requested before this round's are unpacked
+    uint4 cur[kLaneVecs], nxt[kLaneVecs];
+    uint32_t g_cur[kLaneVecs], g_nxt[kLaneVecs];
+    bool ok_cur[kLaneVecs], ok_nxt[kLaneVecs];
+    auto fetch_round = [&](int b, uint32_t (&g)[kLaneVecs], uint4 (&w)[kLaneVecs], bool (&ok)[kLaneVecs]) {
 #pragma unroll
-      for (int h = 0; h < kVecs; ++h) {
-        ok[h] = valid && *g * kVecs + h < (uint32_t)rd.n_groups;
-        w[h] = fetch(ok[h], *g * kVecs + h);
+      for (int i = 0; i < kEntriesPerLane; ++i) {
+        const int at = b + i * 32 + lane;
+        const bool valid = at < upto;
+        const uint32_t entry = valid ? park[at] : 0u;
+#pragma unroll
+        for (int h = 0; h < kVecs; ++h) {
+          const int s = i * kVecs + h;
+          g[s] = entry * kVecs + h;
+          ok[s] = valid && g[s] < (uint32_t)rd.n_groups;
+          w[s] = fetch(ok[s], g[s]);
+        }
       }
     };
-    fetch_round(0, &g_cur, cur, ok_cur);
-    for (int b = 0; b < upto; b += 32) {
-      fetch_round(b + 32, &g_nxt, nxt, ok_nxt);
+    fetch_round(0, g_cur, cur, ok_cur);
+    for (int b = 0; b < upto; b += kRound) {
+      fetch_round(b + kRound, g_nxt, nxt, ok_nxt);
+      constexpr int kLast = kLaneVecs - 1;  // (one vector per lane: the second operand is never looked at)
+      const uint32_t after = admit(ok_cur[0], g_cur[0], cur[0], kLaneVecs == 2 && ok_cur[kLast], g_cur[kLast], cur[kLast], thr);
+      handed_out = after > handed_out ? after : handed_out;
 #pragma unroll
-      for (int h = 0; h < kVecs; ++h) {
-        const uint32_t after = admit(ok_cur[h], g_cur * kVecs + h, cur[h], thr);
-        handed_out = after > handed_out ? after : handed_out;
-        cur[h] = nxt[h];
-        ok_cur[h] = ok_nxt[h];
+      for (int s = 0; s < kLaneVecs; ++s) {
+        cur[s] = nxt[s];
+        ok_cur[s] = ok_nxt[s];
+        g_cur[s] = g_nxt[s];
       }
-      g_cur = g_nxt;
     }
-    const int left = all ? 0 : nparked - upto;  // < 32
-    const uint32_t moved = lane < left ? park[upto + lane] : 0u;
+    const int left = all ? 0 : nparked - upto;  // < kRound
+    uint32_t moved[kEntriesPerLane];
+#pragma unroll
+    for (int i = 0; i < kEntriesPerLane; ++i) moved[i] = i * 32 + lane < left ? park[upto + i * 32 + lane] : 0u;
     __syncwarp();
-    if (lane < left) park[lane] = moved;
+#pragma unroll
+    for (int i = 0; i < kEntriesPerLane; ++i)
+      if (i * 32 + lane < left) park[i * 32 + lane] = moved[i];
     nparked = left;
     __syncwarp();
     // raise the threshold if enough candidates have arrived since the last time and nobody else is at it
@@ -937,7 +962,7 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
           if ((votes[j] >> lane) & 1u) park[nparked + __popc(votes[j] & below)] = (uint32_t)(wi * 4 + j);
           nparked += __popc(votes[j]);
         }
-        if (nparked >= kParkTrigger) drain(false);
+        if (nparked >= kRound) drain(false);
       }
       if (*shared_overflow) break;
     }
@@ -969,7 +994,7 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
         if (hit[u]) park[nparked + __popc(votes[u] & ((1u << lane) - 1u))] = (uint32_t)(begin + u * T) + threadIdx.x;
         nparked += __popc(votes[u]);
       }
-      if (nparked >= kParkTrigger) drain(false);
+      if (nparked >= kRound) drain(false);
     }
     thr = *shared_thr;
     if (*shared_overflow) break;
@@ -1220,7 +1245,7 @@ __device__ void commit_one_chunk(DirectShared& sh, uint4* ring, const DirectPara
   if constexpr (VECTOR) {
     if (!loose_failed) {
       if ((long long)rd.n_groups * R::VEC <= kLooseMaxElems)
-        done = select_unordered<DT, true, kThreads, false>(loose_workspace<DT>(sh, ring), ring, rd, p.k, emit, rec);
+        done = select_unordered<DT, true, kThreads, false, false>(loose_workspace<DT>(sh, ring), ring, rd, p.k, emit, rec);
       else if (p.k <= kStreamMaxK) done = select_in_one_pass<DT>(sh, ring, rd, p.k, emit);
     }
   }
@@ -1395,7 +1420,7 @@ __device__ void verify_one_chunk(DirectShared& sh, uint4* ring, const DirectPara
     if (!loose_failed && (loose || k <= kStreamMaxK)) {
       sel_idx = reinterpret_cast<uint32_t*>(ring);
       sel_pat = reinterpret_cast<uint16_t*>(sel_idx + 2 * k);
-      done = loose ? select_unordered<DT, false, kThreads, false>(loose_workspace<DT>(sh, ring), ring, rd, k, emit)
+      done = loose ? select_unordered<DT, false, kThreads, false, false>(loose_workspace<DT>(sh, ring), ring, rd, k, emit)
                    : select_in_one_pass<DT>(sh, ring, rd, k, emit);
     }
   }
@@ -1474,7 +1499,9 @@ __device__ __forceinline__ LooseWorkspace<DT> carve(unsigned char* smem, Carve* 
   return ws;
 }
 
-template <int DT>
+// TWO: two parked vectors per lane and round of unpacking (bf16, k >= kTwoFrom).
+constexpr int kTwoFrom = 2048;
+template <int DT, bool TWO>
 __global__ void __launch_bounds__(kT, 2) toploc_direct_commit_half_kernel(DirectParams p, uint8_t* commits, uint8_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Carve cv;
@@ -1494,11 +1521,11 @@ __global__ void __launch_bounds__(kT, 2) toploc_direct_commit_half_kernel(Direct
     rec[3 * pos + 1] = (uint16_t)(flat >> 16);
     rec[3 * pos + 2] = (uint16_t)pat;
   };
-  const bool done = select_unordered<DT, true, kT, true>(ws, cv.ring, rd, p.k, emit, rec);
+  const bool done = select_unordered<DT, true, kT, true, TWO>(ws, cv.ring, rd, p.k, emit, rec);
   if (threadIdx.x == 0) status[chunk] = done ? TOPLOC_CHUNK_OK : kRetry;
 }
 
-template <int DT>
+template <int DT, bool TWO>
 __global__ void __launch_bounds__(kT, 2) toploc_direct_verify_half_kernel(DirectParams p, DirectVerify io) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Carve cv;
@@ -1521,7 +1548,7 @@ __global__ void __launch_bounds__(kT, 2) toploc_direct_verify_half_kernel(Direct
     sel_idx[pos] = flat;
     sel_pat[pos] = (uint16_t)pat;
   };
-  if (!select_unordered<DT, false, kT, true>(ws, cv.ring, rd, k, emit)) {
+  if (!select_unordered<DT, false, kT, true, TWO>(ws, cv.ring, rd, k, emit)) {
     if (threadIdx.x == 0) {
       toploc_chunk_result r = {};
       r.status = kRetry;
@@ -1943,13 +1970,16 @@ int toploc_commit_direct(const void* d_act, const toploc_layout* lay, uint8_t* d
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, plan.device) != cudaSuccess) return TOPLOC_ERR_CUDA;
     const long long rescuers = plan.num_chunks < sms ? plan.num_chunks : sms;
     if (lay->dtype == TOPLOC_DTYPE_BF16) {
-      rc = launch_direct<half_block::kT>(half_block::toploc_direct_commit_half_kernel<0>, plan.num_chunks,
-                                         half_block::kBlockBytes, stream, p, d_commits, d_status);
+      rc = lay->k >= half_block::kTwoFrom
+               ? launch_direct<half_block::kT>(half_block::toploc_direct_commit_half_kernel<0, true>, plan.num_chunks,
+                                               half_block::kBlockBytes, stream, p, d_commits, d_status)
+               : launch_direct<half_block::kT>(half_block::toploc_direct_commit_half_kernel<0, false>, plan.num_chunks,
+                                               half_block::kBlockBytes, stream, p, d_commits, d_status);
       if (rc == TOPLOC_OK)
         rc = launch_direct(half_block::toploc_direct_commit_rescue_kernel<0>, rescuers, smem, stream, p, plan.num_chunks,
                            d_commits, d_status);
     } else {
-      rc = launch_direct<half_block::kT>(half_block::toploc_direct_commit_half_kernel<1>, plan.num_chunks,
+      rc = launch_direct<half_block::kT>(half_block::toploc_direct_commit_half_kernel<1, false>, plan.num_chunks,
                                          half_block::kBlockBytes, stream, p, d_commits, d_status);
       if (rc == TOPLOC_OK)
         rc = launch_direct(half_block::toploc_direct_commit_rescue_kernel<1>, rescuers, smem, stream, p, plan.num_chunks,
@@ -2000,12 +2030,15 @@ static int verify_direct_with(const void* d_act, const toploc_layout* lay, const
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, plan.device) != cudaSuccess) return TOPLOC_ERR_CUDA;
     const long long rescuers = plan.num_chunks < sms ? plan.num_chunks : sms;
     if (lay->dtype == TOPLOC_DTYPE_BF16) {
-      rc = launch_direct<half_block::kT>(half_block::toploc_direct_verify_half_kernel<0>, plan.num_chunks,
-                                         half_block::kBlockBytes, stream, p, io);
+      rc = lay->k >= half_block::kTwoFrom
+               ? launch_direct<half_block::kT>(half_block::toploc_direct_verify_half_kernel<0, true>, plan.num_chunks,
+                                               half_block::kBlockBytes, stream, p, io)
+               : launch_direct<half_block::kT>(half_block::toploc_direct_verify_half_kernel<0, false>, plan.num_chunks,
+                                               half_block::kBlockBytes, stream, p, io);
       if (rc == TOPLOC_OK)
         rc = launch_direct(half_block::toploc_direct_verify_rescue_kernel<0>, rescuers, smem, stream, p, plan.num_chunks, io);
     } else {
-      rc = launch_direct<half_block::kT>(half_block::toploc_direct_verify_half_kernel<1>, plan.num_chunks,
+      rc = launch_direct<half_block::kT>(half_block::toploc_direct_verify_half_kernel<1, false>, plan.num_chunks,
                                          half_block::kBlockBytes, stream, p, io);
       if (rc == TOPLOC_OK)
         rc = launch_direct(half_block::toploc_direct_verify_rescue_kernel<1>, rescuers, smem, stream, p, plan.num_chunks, io);
