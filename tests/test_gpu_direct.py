@@ -183,6 +183,17 @@ def test_odd_shapes_take_the_scalar_path():
     direct_case(f, L, 100, S, T, None, "fp32 H=1001")
 
 
+def test_fewer_vectors_than_k():
+    # 512 elements per chunk = 64 vectors of eight: k = 300 and k = 512 (every element) exceed the
+    # number of vectors, so no threshold can come from the vectors' maxima
+    S, T, H, L = 2, 16, 64, 8
+    act = synth.make_activations(S, T, H, torch.bfloat16, seed=83, device=DEV, outliers="none")
+    for k in (300, 512):
+        direct_case(act, L, k, S, T, {"noise": synth.honest_noise(act, seed=4)}, "64 vectors, k=%d" % k)
+    f = synth.make_activations(S, T, 128, torch.float32, seed=84, device=DEV, outliers="none")
+    direct_case(f, 4, 400, S, T, None, "fp32: 128 vectors, k=400")
+
+
 def test_chunk_smaller_than_k_and_malformed_commitments():
     S, T, H, L, k = 1, 10, 64, 4, 200      # chunks of 256, 256 and 128 elements
     act = synth.make_activations(S, T, H, torch.bfloat16, seed=81, device=DEV, outliers="none")
