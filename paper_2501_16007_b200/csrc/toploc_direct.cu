@@ -809,7 +809,43 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
     rd.template request<T>(ring, (int)threadIdx.x, first_end);  // in flight meanwhile
   }
   if (rd.n_groups >= k) {
-    for (int begin = 0; begin < rd.n_groups; begin += kBatch) {
+    int begin = 0;
+    if (rd.flat) {
+      // Rows without gaps: while this batch and the next are whole, nothing needs a bound and a
+      // thread's vectors lie kBatch * 16 bytes apart from batch to batch.
+      const char* mine = rd.base + (size_t)threadIdx.x * 16u;
+      const uint32_t slot = (uint32_t)__cvta_generic_to_shared(ring + threadIdx.x);
+      for (; begin + 2 * kBatch <= rd.n_groups; begin += kBatch) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v[u] = ring[u * T + threadIdx.x];
+        const char* next = mine + (size_t)(begin + kBatch) * 16u;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {  // (each copy's destination depends on the register read from it)
+          uint32_t zero;
+          asm volatile("and.b32 %0, %1, 0;" : "=r"(zero) : "r"(v[u].w));
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot + (uint32_t)(u * T * 16) + zero),
+                       "l"(next + (size_t)u * T * 16u)
+                       : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+          const int g = begin + u * T + (int)threadIdx.x;
+          uint32_t bin = toploc_device::vector_max_coarse_key<DT, VEC>(v[u]) >> 4;  // upper 11 of the 15 bits
+          atomicAdd(&coarse[bin], 1u);
+          if (MAP) {
+            if (kPerByte == 2) {
+              const uint32_t other = __shfl_xor_sync(kFull, bin, 1);
+              bin = bin > other ? bin : other;
+            }
+            if (kPerByte == 1 || (g & 1) == 0) ws.seen_max[g / kPerByte] = (uint8_t)seen_byte(bin);
+          }
+        }
+      }
+    }
+    for (; begin < rd.n_groups; begin += kBatch) {
       const int end = begin + kBatch < rd.n_groups ? begin + kBatch : rd.n_groups;
       uint32_t w[kUnroll][4];
       rd.template take<T>(ring, begin + (int)threadIdx.x, end, w);
