@@ -598,6 +598,7 @@ struct LooseWorkspace {
   uint32_t* park;        // kParkCap words per warp
   int cap;
   uint8_t* seen_max;     // MAP only: one byte per 8 elements (their largest key, coarsely), written by the first pass
+  uint4* second_stage;   // MAP only: kUnroll * T more 16-byte slots that are idle during the first pass
   uint32_t* bitmap;      // ORDERED only: one bit per element for the ranking in index order
 };
 
@@ -810,7 +811,66 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   }
   if (rd.n_groups >= k) {
     int begin = 0;
-    if (rd.flat) {
+    // One whole batch of a gap-free chunk in the first pass: its histogram entries and (MAP) bytes.
+    auto count_whole_batch = [&](int first, const uint4 (&v)[kUnroll]) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int g = first + u * T + (int)threadIdx.x;
+        uint32_t bin = toploc_device::vector_max_coarse_key<DT, VEC>(v[u]) >> 4;  // upper 11 of the 15 bits
+        atomicAdd(&coarse[bin], 1u);
+        if (MAP) {
+          if (kPerByte == 2) {
+            const uint32_t other = __shfl_xor_sync(kFull, bin, 1);
+            bin = bin > other ? bin : other;
+          }
+          if (kPerByte == 1 || (g & 1) == 0) ws.seen_max[g / kPerByte] = (uint8_t)seen_byte(bin);
+        }
+      }
+    };
+    if (MAP && rd.flat && rd.n_groups >= 2 * kBatch) {
+      // Rows without gaps, and room for a second batch in flight: the memory behind the ring is
+      // idle until candidates arrive (ws.second_stage), so two batches are on their way while one
+      // is counted -- a block that streams while its neighbour on the SM is busy with a chunk's
+      // later phases then draws more than one ring's worth of bandwidth.  Whole batches only: no
+      // bounds, plain pointer steps; a ragged last batch is left to the loop below.
+      const int n_whole = rd.n_groups / kBatch;
+      const char* mine = rd.base + (size_t)threadIdx.x * 16u;
+      const uint4* stage0 = ring + threadIdx.x;
+      const uint4* stage1 = ws.second_stage + threadIdx.x;
+      const uint32_t slot0 = (uint32_t)__cvta_generic_to_shared(stage0), slot1 = (uint32_t)__cvta_generic_to_shared(stage1);
+      // batch 0 is on its way to the ring already; batch 1 goes to the second stage
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot1 + (uint32_t)(u * T * 16)),
+                     "l"(mine + ((size_t)kBatch + (size_t)u * T) * 16u)
+                     : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      for (int b = 0; b < n_whole; ++b) {
+        // groups complete in order: all but the latest one have landed, batch b among them
+        if (b + 1 < n_whole) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        const uint4* stage = (b & 1) ? stage1 : stage0;
+        const uint32_t slot = (b & 1) ? slot1 : slot0;
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v[u] = stage[u * T];
+        if (b + 2 < n_whole) {
+          const char* next = mine + (size_t)(b + 2) * kBatch * 16u;
+#pragma unroll
+          for (int u = 0; u < kUnroll; ++u) {  // (each copy's destination depends on the register read from it)
+            uint32_t zero;
+            asm volatile("and.b32 %0, %1, 0;" : "=r"(zero) : "r"(v[u].w));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot + (uint32_t)(u * T * 16) + zero),
+                         "l"(next + (size_t)u * T * 16u)
+                         : "memory");
+          }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");  // (an empty group keeps the count in step)
+        count_whole_batch(b * kBatch, v);
+      }
+      begin = n_whole * kBatch;
+      if (begin < rd.n_groups) rd.template request<T>(ring, begin + (int)threadIdx.x, rd.n_groups);  // the ragged rest
+    } else if (rd.flat) {
       // Rows without gaps: while this batch and the next are whole, nothing needs a bound and a
       // thread's vectors lie kBatch * 16 bytes apart from batch to batch.
       const char* mine = rd.base + (size_t)threadIdx.x * 16u;
@@ -830,19 +890,7 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
                        : "memory");
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          const int g = begin + u * T + (int)threadIdx.x;
-          uint32_t bin = toploc_device::vector_max_coarse_key<DT, VEC>(v[u]) >> 4;  // upper 11 of the 15 bits
-          atomicAdd(&coarse[bin], 1u);
-          if (MAP) {
-            if (kPerByte == 2) {
-              const uint32_t other = __shfl_xor_sync(kFull, bin, 1);
-              bin = bin > other ? bin : other;
-            }
-            if (kPerByte == 1 || (g & 1) == 0) ws.seen_max[g / kPerByte] = (uint8_t)seen_byte(bin);
-          }
-        }
+        count_whole_batch(begin, v);
       }
     }
     for (; begin < rd.n_groups; begin += kBatch) {
@@ -1226,6 +1274,7 @@ template <int DT>
 __device__ __forceinline__ LooseWorkspace<DT> loose_workspace(DirectShared& sh, uint4* ring) {
   LooseWorkspace<DT> ws;
   ws.seen_max = nullptr;
+  ws.second_stage = nullptr;
   ws.bitmap = reinterpret_cast<uint32_t*>(ring);
   ws.ctl = &sh.loose;
   ws.coarse = sh.hist;
@@ -1501,6 +1550,7 @@ constexpr size_t kBlockBytes = (227 * 1024) / 2 - 1024;      // two blocks per S
 __host__ __device__ constexpr int cap(int dt) { return (int)((kBlockBytes - kFixed) / (dt == 0 ? 6 : 8)) / 64 * 64; }
 static_assert(kFixed % 16 == 0 && cap(0) >= 2 * 4096 && cap(1) >= 4096 + 2048, "room for the candidates of k = 4096");
 static_assert((size_t)cap(0) * 6 >= kRing && (size_t)cap(1) * 8 >= kRing, "the candidates' place contains the ring");
+static_assert(kBlockBytes - kFixed + kPark >= 2 * kRing, "candidates and parked groups make room for the second stage");
 static_assert(6 * TOPLOC_MAX_K_DIRECT <= kSeen && 6 * TOPLOC_MAX_K_DIRECT <= 6 * 4096,
               "the selection fits the bytes' place, the decoded commitment the candidates' place");
 
@@ -1512,15 +1562,20 @@ struct Carve {
 
 template <int DT>
 __device__ __forceinline__ LooseWorkspace<DT> carve(unsigned char* smem, Carve* out) {
-  // from the end: control, comparison scratch, histogram, parked groups, the bytes of the first
-  // pass; everything before them is the candidates' (flat indices, then patterns), whose first
-  // 32 KB are the ring while the chunk streams
+  // from the end: histogram, comparison scratch, control, the bytes of the first pass, parked
+  // groups; everything before them is the candidates' (flat indices, then patterns).  While the
+  // chunk streams the first 32 KB are the ring and the next 32 KB -- the rest of the candidates'
+  // place and the beginning of the parked groups', both idle until the second pass -- a second
+  // stage of it.
   LooseWorkspace<DT> ws;
   out->ring = reinterpret_cast<uint4*>(smem);
   ws.cap = cap(DT);
   ws.cand_flat = reinterpret_cast<uint32_t*>(smem);
   ws.cand_pat = reinterpret_cast<typename StoredPattern<DT>::type*>(ws.cand_flat + ws.cap);
+  ws.second_stage = out->ring + kRing / sizeof(uint4);
   unsigned char* at = smem + kBlockBytes - kFixed;
+  ws.park = reinterpret_cast<uint32_t*>(at);
+  at += kPark;
   out->seen = at;
   ws.seen_max = at;
   ws.bitmap = reinterpret_cast<uint32_t*>(at);
@@ -1530,8 +1585,6 @@ __device__ __forceinline__ LooseWorkspace<DT> carve(unsigned char* smem, Carve* 
   out->cs = reinterpret_cast<CompareScratch*>(at);
   at += sizeof(CompareScratch);
   ws.coarse = reinterpret_cast<uint32_t*>(at);
-  at += (size_t)kCoarseBins * 4;
-  ws.park = reinterpret_cast<uint32_t*>(at);
   return ws;
 }
 
