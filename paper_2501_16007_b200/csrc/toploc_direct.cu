@@ -1025,29 +1025,70 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
 
   if (MAP) {
     // The threshold is a bin's lowest key (or 0 for a chunk of fewer than k vectors, whose bytes
-    // were never written: every byte reaches 0).  Four bytes per lane and step.
+    // were never written: every byte reaches 0).
     const uint32_t bin = thr >> kCoarseShift;
     const uint32_t want = seen_byte(bin) * 0x01010101u;
     const int n_bytes = (rd.n_groups + kPerByte - 1) / kPerByte;
-    const uint32_t* words = reinterpret_cast<const uint32_t*>(ws.seen_max);
-    const uint32_t below = (1u << lane) - 1u;
-    for (int w0 = 0; w0 * 4 < n_bytes; w0 += T) {
-      const int wi = w0 + (int)threadIdx.x;
-      const uint32_t reach = wi * 4 < n_bytes ? __vcmpgeu4(words[wi], want) : 0u;  // 0xFF per byte that reaches
-      uint32_t votes[4], any_votes = 0;
+    const uint4* quads = reinterpret_cast<const uint4*>(ws.seen_max);  // (its place is a whole number of 16-byte words)
+    // Sixteen bytes per lane and step.  The bytes that reach the threshold's are counted per lane,
+    // one prefix sum over the lanes hands out the places, and every lane parks its own few.
+    // A step that would not fit the parking space (dense data, or the threshold 0) is taken a word
+    // (four bytes per lane) at a time with drains in between.
+    auto exclusive = [&](int mine, int* total) {
+      int incl = mine;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        votes[j] = __ballot_sync(kFull, ((reach >> (8 * j)) & 1u) != 0 && wi * 4 + j < n_bytes);
-        any_votes |= votes[j];
+      for (int off = 1; off < 32; off <<= 1) {
+        const int other = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += other;
       }
-      if (any_votes) {
+      *total = __shfl_sync(kFull, incl, 31);
+      return incl - mine;
+    };
+    auto park_word = [&](uint32_t bits, int first_index, int at) {  // bits: bit 0 of byte j set = entry first_index + j
+      while (bits) {
+        const int j = (__ffs((int)bits) - 1) >> 3;
+        bits &= bits - 1u;
+        park[at++] = (uint32_t)(first_index + j);
+      }
+      return at;
+    };
+    for (int q0 = 0; q0 * 16 < n_bytes; q0 += T) {
+      const int qi = q0 + (int)threadIdx.x;
+      uint32_t reach[4] = {0u, 0u, 0u, 0u};
+      if (qi * 16 < n_bytes) {
+        const uint4 b = quads[qi];
+        reach[0] = __vcmpgeu4(b.x, want) & 0x01010101u;
+        reach[1] = __vcmpgeu4(b.y, want) & 0x01010101u;
+        reach[2] = __vcmpgeu4(b.z, want) & 0x01010101u;
+        reach[3] = __vcmpgeu4(b.w, want) & 0x01010101u;
+        if (qi * 16 + 16 > n_bytes) {  // the last, partial quad: entries beyond the chunk do not count
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          if ((votes[j] >> lane) & 1u) park[nparked + __popc(votes[j] & below)] = (uint32_t)(wi * 4 + j);
-          nparked += __popc(votes[j]);
+          for (int wd = 0; wd < 4; ++wd)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (qi * 16 + wd * 4 + j >= n_bytes) reach[wd] &= ~(1u << (8 * j));
         }
-        if (nparked >= kRound) drain(false);
       }
+      const int mine = __popc(reach[0]) + __popc(reach[1]) + __popc(reach[2]) + __popc(reach[3]);
+      int total;
+      const int before = exclusive(mine, &total);
+      if (total == 0) continue;
+      if (nparked + total <= kParkCap) {
+        int at = nparked + before;
+#pragma unroll
+        for (int wd = 0; wd < 4; ++wd) at = park_word(reach[wd], qi * 16 + wd * 4, at);
+        nparked += total;
+      } else {
+#pragma unroll
+        for (int wd = 0; wd < 4; ++wd) {
+          int word_total;
+          const int word_before = exclusive(__popc(reach[wd]), &word_total);
+          if (nparked + word_total > kParkCap) drain(false);  // leaves fewer than kRound; a word adds at most 128
+          park_word(reach[wd], qi * 16 + wd * 4, nparked + word_before);
+          nparked += word_total;
+        }
+      }
+      if (nparked >= kRound) drain(false);
       if (*shared_overflow) break;
     }
   }
