@@ -712,6 +712,19 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   constexpr int kCoarseShift = key_bits(DT) - 11;
   constexpr uint32_t kFull = 0xFFFFFFFFu;
   constexpr int kBatch = kUnroll * T;
+  // every pointer of the workspace is shared memory: said once, so that loads, stores and atomics
+  // through them compile to shared-memory instructions instead of generic ones
+  __builtin_assume(__isShared(ws.ctl));
+  __builtin_assume(__isShared(ws.coarse));
+  __builtin_assume(__isShared(ws.cand_flat));
+  __builtin_assume(__isShared(ws.cand_pat));
+  __builtin_assume(__isShared(ws.park));
+  __builtin_assume(__isShared(ws.bitmap));
+  __builtin_assume(__isShared(ring));
+  if (MAP) {
+    __builtin_assume(__isShared(ws.seen_max));
+    __builtin_assume(__isShared(ws.second_stage));
+  }
   LooseControl& sh = *ws.ctl;
   const int kCap = ws.cap;
   uint32_t* coarse = ws.coarse;
@@ -812,18 +825,23 @@ __device__ bool select_unordered(const LooseWorkspace<DT>& ws, uint4* ring, cons
   if (rd.n_groups >= k) {
     int begin = 0;
     // One whole batch of a gap-free chunk in the first pass: its histogram entries and (MAP) bytes.
+    // (shared-memory addresses taken once: the histogram and the bytes are reached through pointers
+    // in a struct, and plain shared-memory instructions are cheaper than generic ones)
+    const uint32_t coarse_at = (uint32_t)__cvta_generic_to_shared(coarse);
+    const uint32_t seen_at = MAP ? (uint32_t)__cvta_generic_to_shared(ws.seen_max) : 0u;
     auto count_whole_batch = [&](int first, const uint4 (&v)[kUnroll]) {
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const int g = first + u * T + (int)threadIdx.x;
         uint32_t bin = toploc_device::vector_max_coarse_key<DT, VEC>(v[u]) >> 4;  // upper 11 of the 15 bits
-        atomicAdd(&coarse[bin], 1u);
+        asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(coarse_at + 4u * bin) : "memory");
         if (MAP) {
           if (kPerByte == 2) {
             const uint32_t other = __shfl_xor_sync(kFull, bin, 1);
             bin = bin > other ? bin : other;
           }
-          if (kPerByte == 1 || (g & 1) == 0) ws.seen_max[g / kPerByte] = (uint8_t)seen_byte(bin);
+          if (kPerByte == 1 || (g & 1) == 0)
+            asm volatile("st.shared.u8 [%0], %1;" ::"r"(seen_at + (uint32_t)(g / kPerByte)), "r"(seen_byte(bin)) : "memory");
         }
       }
     };
